@@ -1,0 +1,200 @@
+/*
+ * melinoe_moe.h - C ABI of the cached Mixture-of-Experts layer for NVIDIA B200 (sm_100a).
+ *
+ * One handle is one MoE layer (Section 2 of the paper, Eq. 1-3) executed under a bounded,
+ * GPU-resident expert cache (Section 2 "Expert Offloading Systems", Section 3.2): all experts
+ * live in page-locked host memory, `cache_slots` of them are resident in device memory, and a
+ * forward call fetches the experts it misses over the host link, evicting by LRU.
+ *
+ * Conventions
+ *  - Every function returns a melinoe_status (0 = OK).  Nothing throws, aborts or exits.
+ *  - "dev" pointers are device memory on the device that was current at create time; "host"
+ *    pointers are host memory.  The library never takes ownership of caller memory.
+ *  - bf16 tensors are raw 16-bit patterns, row-major.
+ *  - A handle is driven by one host thread at a time, and all forward calls of one handle must
+ *    be ordered with respect to each other on the device (same stream, or caller-made
+ *    dependencies): a call's cache decisions depend on the previous call's.
+ *  - melinoe_moe_forward is asynchronous with respect to the host.
+ */
+#ifndef MELINOE_MOE_H_
+#define MELINOE_MOE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct melinoe_moe melinoe_moe_t;
+
+typedef enum melinoe_status {
+    MELINOE_OK = 0,
+    MELINOE_ERR_INVALID = 1,     /* bad argument (null, misaligned, out of range, not pinned) */
+    MELINOE_ERR_STATE = 2,       /* call order: e.g. forward before router / experts are set  */
+    MELINOE_ERR_CUDA = 3,        /* a CUDA call failed; melinoe_last_cuda_error() has its code */
+    MELINOE_ERR_NOMEM = 4,       /* device or host allocation failed                           */
+    MELINOE_ERR_TIMEOUT = 5,     /* a bounded device-side or service-side wait ran out         */
+    MELINOE_ERR_UNSUPPORTED = 6  /* shape outside what the kernels cover                       */
+} melinoe_status;
+
+/*
+ * Per-call statistics, written on the device in stream order by the call's planning kernel.
+ * The caller passes device-accessible memory (device memory or page-locked host memory) and
+ * reads it after synchronising the stream.  `misses` is the paper's hard miss count of the
+ * call (Appendix C.1: one miss = one host-to-device expert transfer).
+ */
+typedef struct melinoe_moe_stats {
+    int32_t status;       /* melinoe_status of the device-side part of the call            */
+    int32_t n_tokens;     /* T                                                             */
+    int32_t n_distinct;   /* number of distinct experts the call's tokens selected         */
+    int32_t hits;         /* requests served from the cache                                */
+    int32_t misses;       /* requests fetched from host memory                             */
+    int32_t evictions;    /* misses that displaced a resident expert                       */
+    int32_t groups;       /* compute groups the call was split in (1 + miss waves)         */
+    int32_t reserved;
+    uint64_t bytes_h2d;   /* misses * bytes_per_expert                                     */
+    uint64_t call_no;     /* 1-based count of forward calls on this handle since reset     */
+} melinoe_moe_stats;
+
+/* One cache request of a call, in the order the cache saw it (hits in ascending expert id,
+ * then misses in ascending expert id).  evicted = expert displaced, or -1. */
+typedef struct melinoe_moe_request {
+    int32_t expert, slot, hit, evicted;
+} melinoe_moe_request;
+
+/*
+ * Create one layer.  Shapes follow Eq. 1-3: router W_r [n_experts][d_model]; each expert has
+ * W_g, W_u [d_ff][d_model] and W_d [d_model][d_ff].  Allocates, on the current device,
+ * cache_slots expert slots of melinoe_moe_expert_bytes() each plus small tables, and creates
+ * a copy stream.  Limits: d_model in {256, 512, 1024, 2048, 3072, 4096}, d_ff % 8 == 0,
+ * 1 <= top_k <= n_experts <= 64, top_k <= cache_slots <= n_experts  (INVALID / UNSUPPORTED
+ * otherwise).
+ */
+int melinoe_moe_create(int d_model, int d_ff, int n_experts, int top_k, int cache_slots,
+                       melinoe_moe_t **out);
+
+/* Waits for the handle's outstanding transfers and device work, then frees everything the
+ * library allocated.  Caller memory (router, experts, bias) is untouched. */
+int melinoe_moe_destroy(melinoe_moe_t *h);
+
+/* Bytes of one packed expert: 3 * d_model * d_ff * 2. */
+size_t melinoe_moe_expert_bytes(int d_model, int d_ff);
+
+/*
+ * Pack one expert from the paper's matrix shapes (Eq. 3; bf16, row-major, host memory) into
+ * the library's streaming layout (host memory, `melinoe_moe_expert_bytes` long):
+ *     rows 0 .. 2*d_ff-1 of [d_model] values: row 2f = W_g[f][:], row 2f+1 = W_u[f][:]
+ *     then d_ff rows of [d_model] values:      row f = W_d[:][f]   (W_d transposed)
+ * so that every d_ff-slice of an expert is two contiguous byte ranges.  Pure host code; does
+ * not touch the device.  blob_out must not overlap the inputs.
+ */
+int melinoe_moe_pack_expert(int d_model, int d_ff, const void *w_gate_host, const void *w_up_host,
+                            const void *w_down_host, void *blob_out_host);
+
+/* Router matrix W_r (Eq. 1): dev pointer, [n_experts][d_model] bf16, 16-byte aligned, borrowed
+ * until the handle is destroyed or the router is replaced. */
+int melinoe_moe_set_router(melinoe_moe_t *h, const void *w_router_dev);
+
+/*
+ * The host-resident expert store (Section 3.2: offloaded experts stay in pinned CPU memory).
+ * expert_host_ptrs[e] points to expert e packed by melinoe_moe_pack_expert, in page-locked
+ * host memory, 16-byte aligned; bytes_per_expert must equal melinoe_moe_expert_bytes().
+ * Pointers are checked with the CUDA runtime: pageable memory is rejected with INVALID (the
+ * library never stages silently).  Borrowed, read-only, must outlive the handle.
+ */
+int melinoe_moe_register_host_experts(melinoe_moe_t *h, const void *const *expert_host_ptrs,
+                                      size_t bytes_per_expert);
+
+/* Always-resident shared experts (not in the paper; DeepSeekMoE-style stacks): packed blobs
+ * in DEVICE memory, applied to every token with gate 1, never cached, never counted in
+ * hits or misses.  n_shared <= 8.  Borrowed. */
+int melinoe_moe_register_shared_experts(melinoe_moe_t *h, int n_shared,
+                                        const void *const *expert_dev_ptrs);
+
+/*
+ * Optional additive router bias (emulates a fine-tuned, sequence-concentrated router):
+ * logits = W_r x + seq_bias[token_seq[t]].  seq_bias_dev [n_seq][n_experts] fp32;
+ * token_seq_dev [T] int32 with values in [0, n_seq), or NULL = every token uses row 0.
+ * seq_bias_dev == NULL restores Eq. 1 exactly.  Borrowed; takes effect for later calls.
+ */
+int melinoe_moe_set_router_bias(melinoe_moe_t *h, const float *seq_bias_dev,
+                                const int32_t *token_seq_dev, int n_seq);
+
+/* Make room for calls of up to max_tokens tokens (scratch grows on demand otherwise, which
+ * synchronises the device). */
+int melinoe_moe_reserve(melinoe_moe_t *h, int max_tokens);
+
+/*
+ * One forward call of the layer for n_tokens tokens (Eq. 1-3 under the cache):
+ * router softmax + top-k (ties to the lowest expert id), slot lookup with LRU eviction,
+ * asynchronous fetch of the missed experts from host memory on the handle's copy stream
+ * overlapped with the compute of the resident ones, token-to-expert gather, SwiGLU expert
+ * FFN with fp32 accumulation, and the gate-weighted sum, rounded once to bf16.
+ * Gates are renormalised over the selected experts (they sum to 1 per token).
+ *
+ * cuda_stream: a cudaStream_t (NULL = legacy default stream).  hidden_dev [n_tokens][d_model]
+ * bf16 and out_dev [n_tokens][d_model] bf16 are device memory, 16-byte aligned, borrowed
+ * until the stream work of this call has finished.  stats_dev: see melinoe_moe_stats; may be
+ * NULL.  n_tokens == 0 is a no-op.  Returns without waiting for the device.
+ */
+int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_dev,
+                        int n_tokens, void *out_dev, melinoe_moe_stats *stats_dev);
+
+/*
+ * Same call with HOST buffers: copies hidden_host to the device, runs the layer, copies the
+ * result to out_host and (if not NULL) the statistics to stats_host, all in stream order.
+ * Page-locked buffers make the copies asynchronous; pageable buffers work but block.
+ */
+int melinoe_moe_forward_host(melinoe_moe_t *h, void *cuda_stream, const void *hidden_host,
+                             int n_tokens, void *out_host, melinoe_moe_stats *stats_host);
+
+/* Cold start: all slots empty, stamps and totals zero.  Synchronises the handle first. */
+int melinoe_moe_reset_cache(melinoe_moe_t *h);
+
+/*
+ * Post-deployment prefetch of Section 3.2 (Eq. 5: preload the Top-C predicted experts before
+ * generation).  Loads up to cache_slots experts, in the order given, as if each were a miss
+ * of its own call (counted in the totals).  Synchronous.
+ */
+int melinoe_moe_preload(melinoe_moe_t *h, const int32_t *expert_ids_host, int n);
+
+/*
+ * Inspection (synchronise the stream first; these copy from the device and block).
+ * last_routing: idx [T][top_k] int32 and gates [T][top_k] fp32 of the most recent call.
+ * last_logits: the router logits (argument of the softmax in Eq. 1, bias included).
+ * last_requests: the most recent call's cache requests in order; *n_out receives their count
+ *   (capacity n_experts records).
+ * last_gather: counts [n_experts], offsets [n_experts+1], perm [T*top_k] (flat pair indices
+ *   t*top_k + j grouped by expert, ascending within an expert).
+ * cache_state: expert_of_slot [cache_slots] (-1 = empty) and totals {hits, misses, evictions}.
+ * Any output pointer may be NULL.
+ */
+int melinoe_moe_last_routing(melinoe_moe_t *h, int32_t *idx_host, float *gate_host);
+int melinoe_moe_last_logits(melinoe_moe_t *h, float *logits_host /* [T][n_experts] fp32 */);
+int melinoe_moe_last_requests(melinoe_moe_t *h, melinoe_moe_request *req_host, int *n_out);
+int melinoe_moe_last_gather(melinoe_moe_t *h, int32_t *counts_host, int32_t *offsets_host,
+                            int32_t *perm_host);
+int melinoe_moe_cache_state(melinoe_moe_t *h, int32_t *expert_of_slot_host, uint64_t *totals_host);
+
+/*
+ * Kernel timing for benchmarks: when enabled, every forward call brackets its expert-FFN
+ * launches with CUDA events on the caller's stream; melinoe_moe_ffn_time_ms returns, for the
+ * calls since the last query, the summed FFN time (ms) and the number of FFN launches and
+ * resets both.  Synchronises the recorded events.
+ */
+int melinoe_moe_enable_timing(melinoe_moe_t *h, int enable);
+int melinoe_moe_ffn_time_ms(melinoe_moe_t *h, double *ms_out, int64_t *launches_out);
+
+/* Number of kernels this library has launched in this process (all handles). */
+int64_t melinoe_launch_count(void);
+
+/* Last CUDA error code seen by the library in this process (0 = none). */
+int melinoe_last_cuda_error(void);
+
+const char *melinoe_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MELINOE_MOE_H_ */

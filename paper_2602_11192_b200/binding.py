@@ -1,0 +1,245 @@
+"""ctypes binding with the same names as include/melinoe_moe.h.  Argument marshalling only."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+__all__ = [
+    "MelinoeError", "Stats", "Request", "lib", "library_path", "STATUS_NAMES", "MoELayer",
+    "melinoe_moe_expert_bytes", "melinoe_moe_pack_expert", "melinoe_launch_count",
+    "melinoe_last_cuda_error", "melinoe_strerror", "EXPORTED_SYMBOLS",
+]
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+
+EXPORTED_SYMBOLS = [
+    "melinoe_moe_create", "melinoe_moe_destroy", "melinoe_moe_expert_bytes", "melinoe_moe_pack_expert",
+    "melinoe_moe_set_router", "melinoe_moe_register_host_experts", "melinoe_moe_register_shared_experts",
+    "melinoe_moe_set_router_bias", "melinoe_moe_reserve", "melinoe_moe_forward", "melinoe_moe_forward_host",
+    "melinoe_moe_reset_cache", "melinoe_moe_preload", "melinoe_moe_last_routing", "melinoe_moe_last_logits",
+    "melinoe_moe_last_requests", "melinoe_moe_last_gather", "melinoe_moe_cache_state",
+    "melinoe_moe_enable_timing", "melinoe_moe_ffn_time_ms", "melinoe_launch_count",
+    "melinoe_last_cuda_error", "melinoe_strerror",
+]
+
+STATUS_NAMES = {0: "OK", 1: "INVALID", 2: "STATE", 3: "CUDA", 4: "NOMEM", 5: "TIMEOUT", 6: "UNSUPPORTED"}
+
+
+class MelinoeError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = int(status)
+        super().__init__("%s: %s (%d)" % (where, melinoe_strerror(status), status))
+
+
+class Stats(C.Structure):
+    _fields_ = [("status", C.c_int32), ("n_tokens", C.c_int32), ("n_distinct", C.c_int32),
+                ("hits", C.c_int32), ("misses", C.c_int32), ("evictions", C.c_int32),
+                ("groups", C.c_int32), ("reserved", C.c_int32),
+                ("bytes_h2d", C.c_uint64), ("call_no", C.c_uint64)]
+
+
+class Request(C.Structure):
+    _fields_ = [("expert", C.c_int32), ("slot", C.c_int32), ("hit", C.c_int32), ("evicted", C.c_int32)]
+
+
+def library_path() -> str:
+    return os.path.join(HERE, "libmelinoe_moe.so")
+
+
+_lib = None
+
+
+def lib():
+    """The loaded shared library.  Raises if it has not been built (no CPU fallback exists)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = library_path()
+    if not os.path.exists(path):
+        raise ImportError("libmelinoe_moe.so is not built: run `python -m paper_2602_11192_b200.build` "
+                          "(there is no fallback implementation)")
+    L = C.CDLL(path)
+    vp, i32, sz = C.c_void_p, C.c_int, C.c_size_t
+    L.melinoe_moe_create.argtypes = [i32, i32, i32, i32, i32, C.POINTER(vp)]
+    L.melinoe_moe_destroy.argtypes = [vp]
+    L.melinoe_moe_expert_bytes.argtypes = [i32, i32]
+    L.melinoe_moe_expert_bytes.restype = sz
+    L.melinoe_moe_pack_expert.argtypes = [i32, i32, vp, vp, vp, vp]
+    L.melinoe_moe_set_router.argtypes = [vp, vp]
+    L.melinoe_moe_register_host_experts.argtypes = [vp, C.POINTER(vp), sz]
+    L.melinoe_moe_register_shared_experts.argtypes = [vp, i32, C.POINTER(vp)]
+    L.melinoe_moe_set_router_bias.argtypes = [vp, vp, vp, i32]
+    L.melinoe_moe_reserve.argtypes = [vp, i32]
+    L.melinoe_moe_forward.argtypes = [vp, vp, vp, i32, vp, vp]
+    L.melinoe_moe_forward_host.argtypes = [vp, vp, vp, i32, vp, vp]
+    L.melinoe_moe_reset_cache.argtypes = [vp]
+    L.melinoe_moe_preload.argtypes = [vp, vp, i32]
+    L.melinoe_moe_last_routing.argtypes = [vp, vp, vp]
+    L.melinoe_moe_last_logits.argtypes = [vp, vp]
+    L.melinoe_moe_last_requests.argtypes = [vp, vp, C.POINTER(i32)]
+    L.melinoe_moe_last_gather.argtypes = [vp, vp, vp, vp]
+    L.melinoe_moe_cache_state.argtypes = [vp, vp, vp]
+    L.melinoe_moe_enable_timing.argtypes = [vp, i32]
+    L.melinoe_moe_ffn_time_ms.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
+    L.melinoe_launch_count.restype = C.c_int64
+    L.melinoe_last_cuda_error.restype = i32
+    L.melinoe_strerror.argtypes = [i32]
+    L.melinoe_strerror.restype = C.c_char_p
+    _lib = L
+    return L
+
+
+def melinoe_strerror(status: int) -> str:
+    try:
+        return lib().melinoe_strerror(int(status)).decode()
+    except Exception:
+        return STATUS_NAMES.get(int(status), "?")
+
+
+def melinoe_moe_expert_bytes(d_model: int, d_ff: int) -> int:
+    return int(lib().melinoe_moe_expert_bytes(d_model, d_ff))
+
+
+def melinoe_moe_pack_expert(d_model: int, d_ff: int, w_gate_ptr: int, w_up_ptr: int, w_down_ptr: int,
+                            blob_ptr: int) -> None:
+    rc = lib().melinoe_moe_pack_expert(d_model, d_ff, w_gate_ptr, w_up_ptr, w_down_ptr, blob_ptr)
+    if rc:
+        raise MelinoeError(rc, "melinoe_moe_pack_expert")
+
+
+def melinoe_launch_count() -> int:
+    return int(lib().melinoe_launch_count())
+
+
+def melinoe_last_cuda_error() -> int:
+    return int(lib().melinoe_last_cuda_error())
+
+
+def _ptr(t) -> Optional[int]:
+    """Address of a torch tensor / numpy array / int / None."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    if hasattr(t, "data_ptr"):
+        return int(t.data_ptr())
+    return int(t.ctypes.data)
+
+
+class MoELayer:
+    """One handle (= one MoE layer).  Methods mirror the C entry points one to one."""
+
+    def __init__(self, d_model: int, d_ff: int, n_experts: int, top_k: int, cache_slots: int):
+        self.d_model, self.d_ff, self.n_experts, self.top_k, self.cache_slots = (
+            int(d_model), int(d_ff), int(n_experts), int(top_k), int(cache_slots))
+        self._h = C.c_void_p()
+        self._keep = {}
+        rc = lib().melinoe_moe_create(d_model, d_ff, n_experts, top_k, cache_slots, C.byref(self._h))
+        if rc:
+            self._h = C.c_void_p()
+            raise MelinoeError(rc, "melinoe_moe_create")
+
+    # -- lifetime
+    def destroy(self) -> None:
+        if getattr(self, "_h", None) and self._h.value:
+            lib().melinoe_moe_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+    def _ck(self, rc: int, where: str) -> None:
+        if rc:
+            raise MelinoeError(rc, where)
+
+    # -- configuration
+    def set_router(self, w_router_dev) -> None:
+        self._keep["router"] = w_router_dev
+        self._ck(lib().melinoe_moe_set_router(self._h, _ptr(w_router_dev)), "melinoe_moe_set_router")
+
+    def register_host_experts(self, expert_host_ptrs: Sequence[int], bytes_per_expert: int, keep=None) -> None:
+        arr = (C.c_void_p * len(expert_host_ptrs))(*[int(p) for p in expert_host_ptrs])
+        self._keep["experts"] = keep
+        self._ck(lib().melinoe_moe_register_host_experts(self._h, arr, bytes_per_expert),
+                 "melinoe_moe_register_host_experts")
+
+    def register_shared_experts(self, expert_dev_ptrs: Sequence[int], keep=None) -> None:
+        n = len(expert_dev_ptrs)
+        arr = (C.c_void_p * max(n, 1))(*[int(p) for p in expert_dev_ptrs])
+        self._keep["shared"] = keep
+        self._ck(lib().melinoe_moe_register_shared_experts(self._h, n, arr), "melinoe_moe_register_shared_experts")
+
+    def set_router_bias(self, seq_bias_dev, token_seq_dev, n_seq: int) -> None:
+        self._keep["bias"] = (seq_bias_dev, token_seq_dev)
+        self._ck(lib().melinoe_moe_set_router_bias(self._h, _ptr(seq_bias_dev), _ptr(token_seq_dev), n_seq),
+                 "melinoe_moe_set_router_bias")
+
+    def reserve(self, max_tokens: int) -> None:
+        self._ck(lib().melinoe_moe_reserve(self._h, max_tokens), "melinoe_moe_reserve")
+
+    # -- the hot path
+    def forward(self, stream: int, hidden_dev, n_tokens: int, out_dev, stats_dev=None) -> None:
+        self._ck(lib().melinoe_moe_forward(self._h, stream, _ptr(hidden_dev), n_tokens, _ptr(out_dev),
+                                           _ptr(stats_dev)), "melinoe_moe_forward")
+
+    def forward_host(self, stream: int, hidden_host, n_tokens: int, out_host, stats_host=None) -> None:
+        self._ck(lib().melinoe_moe_forward_host(self._h, stream, _ptr(hidden_host), n_tokens, _ptr(out_host),
+                                                _ptr(stats_host)), "melinoe_moe_forward_host")
+
+    def reset_cache(self) -> None:
+        self._ck(lib().melinoe_moe_reset_cache(self._h), "melinoe_moe_reset_cache")
+
+    def preload(self, expert_ids) -> None:
+        import numpy as np
+        ids = np.ascontiguousarray(expert_ids, dtype=np.int32)
+        self._ck(lib().melinoe_moe_preload(self._h, ids.ctypes.data, ids.size), "melinoe_moe_preload")
+
+    # -- inspection (blocking)
+    def last_routing(self, n_tokens: int):
+        import numpy as np
+        idx = np.empty((n_tokens, self.top_k), np.int32)
+        gate = np.empty((n_tokens, self.top_k), np.float32)
+        self._ck(lib().melinoe_moe_last_routing(self._h, idx.ctypes.data, gate.ctypes.data), "melinoe_moe_last_routing")
+        return idx, gate
+
+    def last_logits(self, n_tokens: int):
+        import numpy as np
+        lg = np.empty((n_tokens, self.n_experts), np.float32)
+        self._ck(lib().melinoe_moe_last_logits(self._h, lg.ctypes.data), "melinoe_moe_last_logits")
+        return lg
+
+    def last_requests(self):
+        import numpy as np
+        buf = np.empty((self.n_experts, 4), np.int32)
+        n = C.c_int(0)
+        self._ck(lib().melinoe_moe_last_requests(self._h, buf.ctypes.data, C.byref(n)), "melinoe_moe_last_requests")
+        return buf[: n.value].copy()
+
+    def last_gather(self, n_tokens: int):
+        import numpy as np
+        counts = np.empty(self.n_experts, np.int32)
+        offsets = np.empty(self.n_experts + 1, np.int32)
+        perm = np.empty(n_tokens * self.top_k, np.int32)
+        self._ck(lib().melinoe_moe_last_gather(self._h, counts.ctypes.data, offsets.ctypes.data, perm.ctypes.data),
+                 "melinoe_moe_last_gather")
+        return counts, offsets, perm
+
+    def cache_state(self):
+        import numpy as np
+        eos = np.empty(self.cache_slots, np.int32)
+        tot = np.empty(3, np.uint64)
+        self._ck(lib().melinoe_moe_cache_state(self._h, eos.ctypes.data, tot.ctypes.data), "melinoe_moe_cache_state")
+        return eos, {"hits": int(tot[0]), "misses": int(tot[1]), "evictions": int(tot[2])}
+
+    def enable_timing(self, enable: bool = True) -> None:
+        self._ck(lib().melinoe_moe_enable_timing(self._h, int(enable)), "melinoe_moe_enable_timing")
+
+    def ffn_time_ms(self):
+        ms = C.c_double(0.0)
+        n = C.c_int64(0)
+        self._ck(lib().melinoe_moe_ffn_time_ms(self._h, C.byref(ms), C.byref(n)), "melinoe_moe_ffn_time_ms")
+        return ms.value, n.value

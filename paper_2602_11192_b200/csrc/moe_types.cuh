@@ -1,0 +1,86 @@
+// Shared host/device structures of the cached-MoE-layer library (sm_100a).
+//
+// Nothing here is seen by the CPU oracle; the two implementations share no code.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace melinoe {
+
+constexpr int kMaxExperts = 64;          // routed experts per layer (need-set is one 64-bit mask)
+constexpr int kMaxShared = 8;            // always-resident shared experts
+constexpr int kMaxReq = kMaxExperts + kMaxShared;
+constexpr int kMaxGroups = kMaxExperts + 2;  // 1 + ceil(E / C) with C >= 1
+constexpr int kTokPerVr = 8;             // tokens per virtual request of the streaming FFN kernel
+constexpr int kUnitRows = 8;             // d_ff rows per work unit of the streaming FFN kernel
+
+// Persistent cache state of one layer (device memory).  The reading of "LRU" used here:
+// every request takes stamp = ++counter; a hit re-stamps its slot; a miss takes the lowest
+// empty slot, else the slot with the smallest stamp.
+struct DevCache {
+    int32_t expert_of_slot[kMaxExperts];   // -1 = empty
+    int32_t slot_of_expert[kMaxExperts];   // -1 = not resident
+    uint64_t stamp[kMaxExperts];
+    uint64_t counter;
+    uint64_t tot_hits, tot_misses, tot_evictions;
+    uint64_t call_no;
+    uint64_t tot_vr;                        // virtual requests handed to the FFN kernels so far
+};
+
+// One cache request of a call plus what the compute kernels need to serve it.
+struct ReqRec {
+    int32_t expert;    // routed: 0..E-1; shared: E + s
+    int32_t slot;      // cache slot, or -1 for a shared expert
+    int32_t hit;
+    int32_t evicted;   // expert displaced by this request, or -1
+    int32_t tok_off;   // first entry of this expert's token list in the sorted arrays
+    int32_t n_tok;     // tokens routed to it
+    int32_t vr_start;  // first virtual request (global index within the call)
+    int32_t group;     // compute group: 0 = resident at call entry, g >= 1 = g-th miss wave
+};
+
+// A virtual request: up to kTokPerVr tokens of one expert.
+struct VrRec {
+    int32_t req;       // index into DevPlan::req
+    int32_t tok_off;   // first entry in tok_of_sorted
+    int32_t n_tok;     // 1..kTokPerVr
+    int32_t group;
+};
+
+// Per-call plan written by the planning kernel, read by the FFN and combine kernels.
+struct DevPlan {
+    int32_t n_tokens, n_req, n_hits, n_miss, n_evict, n_groups, n_vr, status;
+    int32_t group_vr_begin[kMaxGroups + 1];
+    int32_t counts[kMaxReq];
+    int32_t offsets[kMaxReq + 1];
+    int32_t req_of_expert[kMaxReq];        // -1 = expert not requested by this call
+    ReqRec req[kMaxReq];
+};
+
+// What the host-side transfer service needs to know about a call, written by the planning
+// kernel into page-locked host memory.  seq_open is written first, seq last.
+struct HostMiss {
+    int32_t expert, slot, group, dep_group;  // dep_group: compute group that must finish first, or -1
+};
+struct HostPlan {
+    uint32_t seq_open;
+    int32_t n_miss, n_groups, status;
+    uint32_t arrive_base, done_base, gmax, pad;
+    HostMiss miss[kMaxExperts];
+    uint32_t seq;
+};
+
+// Geometry shared by the streaming FFN kernel and the combine kernel.
+struct FfnGeom {
+    int d, F, k, E, n_shared;
+    int grid;              // CTAs of every streaming FFN launch
+    int units_per_vr;      // F / kUnitRows
+};
+
+// CTA that owns work unit u when nu units are split over g CTAs as [floor(i*nu/g), floor((i+1)*nu/g)).
+__host__ __device__ inline int cta_of_unit(long long u, long long nu, long long g)
+{
+    return (int)(((u + 1) * g - 1) / nu);
+}
+
+}  // namespace melinoe

@@ -1,0 +1,351 @@
+// Planning kernel: token-to-expert gather, slot lookup with LRU eviction, miss queue.
+//
+// One block per call.  It turns the router's indices into
+//   (a) per-expert token lists (stable counting sort of the (token, rank) pairs),
+//   (b) the call's cache requests: one per distinct expert, experts resident at call entry
+//       first (ascending id), then the missing ones (ascending id); a miss takes the lowest
+//       empty slot, else the least recently stamped slot (Section 3.2: experts are fetched on
+//       demand, "evicting cached experts as dictated by the cache policy"; the policy is LRU),
+//   (c) compute groups: group 0 = resident experts (+ shared experts); the misses follow in
+//       waves, a new wave starting whenever a miss would overwrite an expert of the current
+//       wave, so every wave's transfers can be in flight while earlier groups compute,
+//   (d) the miss queue for the host transfer service, in page-locked host memory, and
+//   (e) the call's statistics (hard miss count of Appendix C.1).
+#include "kernels.cuh"
+
+namespace melinoe {
+
+namespace {
+
+constexpr int kPlanThreads = 1024;
+constexpr int kPlanWarps = kPlanThreads / 32;
+
+__global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p)
+{
+    __shared__ int32_t s_counts[kMaxReq];
+    __shared__ int32_t s_offsets[kMaxReq + 1];
+    __shared__ int32_t s_running[kMaxExperts];
+    __shared__ int32_t s_warp_cnt[kPlanWarps][kMaxExperts];
+    __shared__ DevCache s_cache;
+    __shared__ int32_t s_group_of_expert[kMaxExperts];
+    __shared__ int32_t s_req_of_expert[kMaxReq];
+    __shared__ ReqRec s_req[kMaxReq];
+    __shared__ HostMiss s_miss[kMaxExperts];
+    __shared__ int32_t s_group_vr_begin[kMaxGroups + 1];
+    __shared__ int32_t s_misc[8];  // 0 n_req(routed) 1 n_hits 2 n_miss 3 n_evict 4 n_groups 5 n_vr 6 status 7 n_req_total
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int n_pairs = p.T * p.k;
+    const int E = p.E, C = p.C;
+
+    // ---- load persistent cache state, clear tables
+    {
+        const uint32_t *src = reinterpret_cast<const uint32_t *>(p.cache);
+        uint32_t *dst = reinterpret_cast<uint32_t *>(&s_cache);
+        for (int i = tid; i < (int)(sizeof(DevCache) / 4); i += kPlanThreads)
+            dst[i] = src[i];
+    }
+    for (int i = tid; i < kMaxReq; i += kPlanThreads) {
+        s_counts[i] = 0;
+        s_req_of_expert[i] = -1;
+    }
+    if (tid < 8)
+        s_misc[tid] = 0;
+    __syncthreads();
+
+    // ---- (a) histogram
+    for (int q = tid; q < n_pairs; q += kPlanThreads) {
+        const int e = p.idx[q];
+        if (e >= 0 && e < E)
+            atomicAdd(&s_counts[e], 1);
+        else
+            s_misc[6] = MELINOE_ERR_INVALID;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        int run = 0;
+        for (int e = 0; e < E; ++e) {
+            s_offsets[e] = run;
+            s_running[e] = run;
+            run += s_counts[e];
+        }
+        for (int s = 0; s < p.n_shared; ++s) {
+            s_counts[E + s] = p.T;
+            s_offsets[E + s] = run;
+            run += p.T;
+        }
+        s_offsets[E + p.n_shared] = run;
+    }
+    __syncthreads();
+
+    // ---- stable scatter, kPlanThreads pairs per pass, in pair order
+    for (int base = 0; base < n_pairs; base += kPlanThreads) {
+        for (int i = tid; i < kPlanWarps * kMaxExperts; i += kPlanThreads)
+            (&s_warp_cnt[0][0])[i] = 0;
+        __syncthreads();
+        const int q = base + tid;
+        int e = q < n_pairs ? p.idx[q] : kMaxExperts;
+        if (e < 0 || e >= E)
+            e = kMaxExperts;  // invalid or padding: takes no part
+        const unsigned same = __match_any_sync(0xffffffffu, e);
+        const int rank = __popc(same & ((1u << lane) - 1u));
+        if (e < kMaxExperts && rank == 0)
+            s_warp_cnt[warp][e] = __popc(same);
+        __syncthreads();
+        if (tid < E) {
+            int run = 0;
+            for (int w = 0; w < kPlanWarps; ++w) {
+                const int c = s_warp_cnt[w][tid];
+                s_warp_cnt[w][tid] = run;
+                run += c;
+            }
+            s_group_of_expert[tid] = run;  // scratch: this pass's total for expert tid
+        }
+        __syncthreads();
+        if (e < kMaxExperts) {
+            const int pos = s_running[e] + s_warp_cnt[warp][e] + rank;
+            p.perm[pos] = q;
+            p.inv_pos[q] = pos;
+            p.tok_of_sorted[pos] = q / p.k;
+        }
+        __syncthreads();
+        if (tid < E)
+            s_running[tid] += s_group_of_expert[tid];
+        __syncthreads();
+    }
+    for (int i = tid; i < p.n_shared * p.T; i += kPlanThreads)
+        p.tok_of_sorted[n_pairs + i] = i % p.T;
+
+    // ---- (b), (c): cache requests, by warp 0 (slots spread over lanes)
+    if (warp == 0) {
+        uint64_t need = 0, resident = 0;
+        {
+            const bool n0 = lane < E && s_counts[lane] > 0;
+            const bool n1 = lane + 32 < E && s_counts[lane + 32] > 0;
+            const bool r0 = lane < E && s_cache.slot_of_expert[lane] >= 0;
+            const bool r1 = lane + 32 < E && s_cache.slot_of_expert[lane + 32] >= 0;
+            need = (uint64_t)__ballot_sync(0xffffffffu, n0) | ((uint64_t)__ballot_sync(0xffffffffu, n1) << 32);
+            resident = (uint64_t)__ballot_sync(0xffffffffu, r0) | ((uint64_t)__ballot_sync(0xffffffffu, r1) << 32);
+        }
+        int n_req = 0, n_hits = 0, n_miss = 0, n_evict = 0;
+        uint64_t counter = s_cache.counter;
+        for (uint64_t m = need & resident; m; m &= m - 1) {
+            const int e = __ffsll((long long)m) - 1;
+            if (lane == 0) {
+                const int s = s_cache.slot_of_expert[e];
+                s_cache.stamp[s] = ++counter;
+                s_req[n_req] = ReqRec{e, s, 1, -1, s_offsets[e], s_counts[e], 0, 0};
+                s_req_of_expert[e] = n_req;
+                s_group_of_expert[e] = 0;
+            }
+            ++n_req;
+            ++n_hits;
+        }
+        counter = __shfl_sync(0xffffffffu, counter, 0);
+        __syncwarp();
+        int cur_group = 1;
+        for (uint64_t m = need & ~resident; m; m &= m - 1) {
+            const int e = __ffsll((long long)m) - 1;
+            // victim: lowest empty slot, else smallest stamp (stamps are unique)
+            uint64_t key = ~0ull;
+            int slot = -1;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int s = lane + 32 * h;
+                if (s < C) {
+                    const uint64_t ks = s_cache.expert_of_slot[s] < 0 ? (uint64_t)s
+                                                                       : ((1ull << 63) | s_cache.stamp[s]);
+                    if (ks < key) {
+                        key = ks;
+                        slot = s;
+                    }
+                }
+            }
+#pragma unroll
+            for (int mm = 16; mm >= 1; mm >>= 1) {
+                const uint64_t ok = __shfl_xor_sync(0xffffffffu, key, mm);
+                const int os = __shfl_xor_sync(0xffffffffu, slot, mm);
+                if (ok < key) {
+                    key = ok;
+                    slot = os;
+                }
+            }
+            const int ev = s_cache.expert_of_slot[slot];
+            int dep = -1;
+            if (ev >= 0) {
+                ++n_evict;
+                if ((need >> ev) & 1ull)
+                    dep = s_group_of_expert[ev];
+            }
+            if (dep == cur_group)
+                ++cur_group;
+            __syncwarp();
+            if (lane == 0) {
+                ++counter;
+                if (ev >= 0)
+                    s_cache.slot_of_expert[ev] = -1;
+                s_cache.expert_of_slot[slot] = e;
+                s_cache.slot_of_expert[e] = slot;
+                s_cache.stamp[slot] = counter;
+                s_req[n_req] = ReqRec{e, slot, 0, ev, s_offsets[e], s_counts[e], 0, cur_group};
+                s_req_of_expert[e] = n_req;
+                s_group_of_expert[e] = cur_group;
+                s_miss[n_miss] = HostMiss{e, slot, cur_group, dep};
+            }
+            counter = __shfl_sync(0xffffffffu, counter, 0);
+            ++n_req;
+            ++n_miss;
+            __syncwarp();
+        }
+        if (lane == 0) {
+            const int n_groups = n_miss ? cur_group + 1 : 1;
+            int n_req_total = n_req;
+            for (int s = 0; s < p.n_shared; ++s) {
+                s_req[n_req_total] = ReqRec{E + s, -1, 1, -1, s_offsets[E + s], p.T, 0, 0};
+                s_req_of_expert[E + s] = n_req_total;
+                ++n_req_total;
+            }
+            // virtual requests, grouped: group 0 = hits then shared, then the miss waves in order
+            int nvr = 0;
+            s_group_vr_begin[0] = 0;
+            for (int r = 0; r < n_hits; ++r) {
+                s_req[r].vr_start = nvr;
+                nvr += (s_req[r].n_tok + kTokPerVr - 1) / kTokPerVr;
+            }
+            for (int r = n_req; r < n_req_total; ++r) {
+                s_req[r].vr_start = nvr;
+                nvr += (s_req[r].n_tok + kTokPerVr - 1) / kTokPerVr;
+            }
+            int g = 0;
+            for (int r = n_hits; r < n_req; ++r) {
+                while (g < s_req[r].group)
+                    s_group_vr_begin[++g] = nvr;
+                s_req[r].vr_start = nvr;
+                nvr += (s_req[r].n_tok + kTokPerVr - 1) / kTokPerVr;
+            }
+            while (g < kMaxGroups)
+                s_group_vr_begin[++g] = nvr;
+            int status = s_misc[6];
+            if (nvr > p.vr_capacity || n_groups > (int)p.gmax)
+                status = MELINOE_ERR_STATE;
+            if (status != MELINOE_OK) {
+                // leave nothing for the compute kernels to do
+                for (int i = 0; i <= kMaxGroups; ++i)
+                    s_group_vr_begin[i] = 0;
+                nvr = 0;
+            }
+            s_cache.counter = counter;
+            s_cache.tot_hits += (uint64_t)n_hits;
+            s_cache.tot_misses += (uint64_t)n_miss;
+            s_cache.tot_evictions += (uint64_t)n_evict;
+            s_cache.call_no += 1;
+            s_cache.tot_vr += (uint64_t)nvr;
+            s_misc[0] = n_req;
+            s_misc[1] = n_hits;
+            s_misc[2] = n_miss;
+            s_misc[3] = n_evict;
+            s_misc[4] = n_groups;
+            s_misc[5] = nvr;
+            s_misc[6] = status;
+            s_misc[7] = n_req_total;
+        }
+    }
+    __syncthreads();
+
+    // ---- write the plan, the virtual requests and the cache state back
+    const int n_req_total = s_misc[7];
+    const bool ok = s_misc[6] == MELINOE_OK;
+    DevPlan *plan = p.plan;
+    if (tid == 0) {
+        plan->n_tokens = p.T;
+        plan->n_req = s_misc[0];
+        plan->n_hits = s_misc[1];
+        plan->n_miss = s_misc[2];
+        plan->n_evict = s_misc[3];
+        plan->n_groups = s_misc[4];
+        plan->n_vr = s_misc[5];
+        plan->status = s_misc[6];
+    }
+    for (int i = tid; i <= kMaxGroups; i += kPlanThreads)
+        plan->group_vr_begin[i] = s_group_vr_begin[i];
+    for (int i = tid; i < kMaxReq; i += kPlanThreads) {
+        plan->counts[i] = s_counts[i];
+        plan->req_of_expert[i] = s_req_of_expert[i];
+    }
+    for (int i = tid; i <= kMaxReq; i += kPlanThreads)
+        plan->offsets[i] = i <= E + p.n_shared ? s_offsets[i] : 0;
+    for (int i = tid; i < n_req_total; i += kPlanThreads)
+        plan->req[i] = s_req[i];
+    if (ok) {
+        for (int r = 0; r < n_req_total; ++r) {
+            const ReqRec rec = s_req[r];
+            const int nv = (rec.n_tok + kTokPerVr - 1) / kTokPerVr;
+            for (int v = tid; v < nv; v += kPlanThreads) {
+                VrRec vr;
+                vr.req = r;
+                vr.tok_off = rec.tok_off + v * kTokPerVr;
+                vr.n_tok = min(kTokPerVr, rec.n_tok - v * kTokPerVr);
+                vr.group = rec.group;
+                p.vrs[rec.vr_start + v] = vr;
+            }
+        }
+    }
+    {
+        uint32_t *dst = reinterpret_cast<uint32_t *>(p.cache);
+        const uint32_t *src = reinterpret_cast<const uint32_t *>(&s_cache);
+        for (int i = tid; i < (int)(sizeof(DevCache) / 4); i += kPlanThreads)
+            dst[i] = src[i];
+    }
+
+    // ---- (d) miss queue for the host service, (e) statistics
+    if (tid == 0) {
+        const int n_miss = s_misc[2];
+        if (p.stats) {
+            melinoe_moe_stats st;
+            st.status = s_misc[6];
+            st.n_tokens = p.T;
+            st.n_distinct = s_misc[0];
+            st.hits = s_misc[1];
+            st.misses = n_miss;
+            st.evictions = s_misc[3];
+            st.groups = s_misc[4];
+            st.reserved = 0;
+            st.bytes_h2d = (uint64_t)n_miss * (uint64_t)p.expert_bytes;
+            st.call_no = s_cache.call_no;
+            *p.stats = st;
+        }
+        volatile HostPlan *hp = p.hplan;
+        hp->seq_open = p.call_seq;
+        __threadfence_system();
+        hp->n_miss = n_miss;
+        hp->n_groups = s_misc[4];
+        hp->status = s_misc[6];
+        hp->arrive_base = p.arrive_base;
+        hp->done_base = p.done_base;
+        hp->gmax = p.gmax;
+        for (int i = 0; i < n_miss; ++i) {
+            hp->miss[i].expert = s_miss[i].expert;
+            hp->miss[i].slot = s_miss[i].slot;
+            hp->miss[i].group = s_miss[i].group;
+            hp->miss[i].dep_group = s_miss[i].dep_group;
+        }
+        __threadfence_system();
+        hp->seq = p.call_seq;
+        if (n_miss == 0 || !ok) {
+            // nothing to wait for: release every wave of this call on the device
+            *reinterpret_cast<volatile uint32_t *>(p.arrive_word) = p.arrive_base + p.gmax - 1u;
+        }
+        __threadfence_system();
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_plan(cudaStream_t stream, const PlanParams &p)
+{
+    plan_kernel<<<1, kPlanThreads, 0, stream>>>(p);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace melinoe

@@ -1,0 +1,88 @@
+"""Helpers for the GPU-vs-oracle parity tests: build the same layer on both sides from the
+seeded generators and compare call by call."""
+from __future__ import annotations
+
+import numpy as np
+
+import gen
+import oracle
+
+REL_TOL = 2e-2      # per-token ||y_gpu - y_ref|| / ||y_ref||, the bound the layer is specified to
+TIGHT_TOL = 8e-3    # what bf16 rounding of h and of the output actually allows (2 x 2^-9 rms-ish)
+GATE_RTOL = 1e-5
+
+
+def make_weights(seed, layer, E, d, F, n_shared=0):
+    return [gen.expert_weights(seed, layer, e, d, F) for e in range(E + n_shared)]
+
+
+def rel_err_per_token(y_gpu_bits: np.ndarray, y_ref: np.ndarray) -> np.ndarray:
+    yg = gen.bf16_bits_to_f32(y_gpu_bits).astype(np.float64)
+    num = np.linalg.norm(yg - y_ref, axis=1)
+    den = np.linalg.norm(y_ref, axis=1)
+    return num / np.maximum(den, 1e-30)
+
+
+class Pair:
+    """The CUDA layer and the oracle side by side on identical weights."""
+
+    def __init__(self, d, F, E, k, C, seed=0, layer=0, n_shared=0):
+        from paper_2602_11192_b200.runner import LayerSetup
+        self.d, self.F, self.E, self.k, self.C, self.n_shared = d, F, E, k, C, n_shared
+        self.weights = make_weights(seed, layer, E, d, F, n_shared)
+        self.w_r = gen.router_weights(seed, layer, E, d)
+        self.gpu = LayerSetup(d, F, E, k, C, n_shared)
+        self.gpu.set_experts(self.weights[:E], self.weights[E:])
+        self.gpu.set_router(self.w_r)
+        self.cache = oracle.ExpertCache(C, E)
+        self.bias = None
+        self.seq = None
+
+    def set_bias(self, bias, seq):
+        self.bias, self.seq = bias, seq
+        self.gpu.set_bias(bias, seq)
+
+    def reset(self):
+        self.gpu.layer.reset_cache()
+        self.cache.reset()
+
+    def step(self, x_bits, check_y=True, tokens=None, tol=TIGHT_TOL):
+        """One forward call on both sides; asserts parity; returns (gpu result, oracle result)."""
+        T = x_bits.shape[0]
+        res = self.gpu.forward_np(x_bits)
+        L = self.gpu.layer
+        idx_g, gate_g = L.last_routing(T)
+        lg_g = L.last_logits(T)
+        req_g = L.last_requests()
+        cnt_g, off_g, perm_g = L.last_gather(T)
+        eos_g, tot_g = L.cache_state()
+
+        idx_o, gate_o, lg_o = oracle.route(x_bits, self.w_r, self.k, self.bias, self.seq)
+        req_o = self.cache.call(idx_o)
+        cnt_o, off_o, perm_o = oracle.gather(idx_o, self.E)
+        eos_o, _, tot_o = self.cache.state()
+
+        assert np.array_equal(lg_g.view(np.uint32), lg_o.view(np.uint32)), "router logits differ in bits"
+        assert np.array_equal(idx_g, idx_o), "routing indices differ"
+        assert np.allclose(gate_g, gate_o, rtol=GATE_RTOL, atol=1e-7), "gates differ"
+        assert np.allclose(gate_g.sum(axis=1), 1.0, atol=1e-5)
+        assert np.array_equal(req_g, req_o), "cache trace differs:\n%s\n%s" % (req_g, req_o)
+        assert np.array_equal(cnt_g, cnt_o) and np.array_equal(off_g, off_o) and np.array_equal(perm_g, perm_o)
+        assert np.array_equal(eos_g, eos_o) and tot_g == tot_o
+        st = res["stats"]
+        assert st["status"] == 0 and st["n_tokens"] == T and st["n_distinct"] == len(req_o)
+        assert st["hits"] == int(req_o[:, 2].sum()) and st["misses"] == len(req_o) - int(req_o[:, 2].sum())
+        assert st["evictions"] == int((req_o[:, 3] >= 0).sum())
+        assert st["bytes_h2d"] == st["misses"] * 3 * self.d * self.F * 2
+        out = {"idx": idx_o, "gate": gate_o, "req": req_o, "stats": st}
+        if check_y:
+            y_ref = oracle.ffn_combine(x_bits, idx_o, gate_o, self.weights, self.F, self.n_shared, tokens)
+            yb = res["out_bits"] if tokens is None else res["out_bits"][np.asarray(tokens)]
+            err = rel_err_per_token(yb, y_ref)
+            assert np.all(np.isfinite(gen.bf16_bits_to_f32(res["out_bits"]))), "non-finite output"
+            assert err.max() <= tol, "activation rel err %.3e > %.1e" % (err.max(), tol)
+            out["err"] = err
+        return res, out
+
+    def close(self):
+        self.gpu.close()

@@ -1,0 +1,58 @@
+"""CPU-side checks of the CUDA library: it loads, exports what the header declares, and its
+pure-host helpers work.  No kernel is launched here."""
+import os
+import re
+
+import numpy as np
+import pytest
+
+import gen
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def m():
+    from paper_2602_11192_b200 import build
+    build.build()
+    import paper_2602_11192_b200 as mod
+    return mod
+
+
+def test_library_exports_every_declared_symbol(m):
+    hdr = open(os.path.join(ROOT, "include", "melinoe_moe.h")).read()
+    declared = set(re.findall(r"^(?:int|size_t|int64_t|const char \*)\s*(melinoe_[a-z0-9_]+)\s*\(", hdr, re.M))
+    assert declared, "no declarations found"
+    L = m.lib()
+    for name in sorted(declared):
+        assert hasattr(L, name), "library does not export %s" % name
+    assert declared == set(m.EXPORTED_SYMBOLS), declared ^ set(m.EXPORTED_SYMBOLS)
+
+
+def test_status_strings_and_sizes(m):
+    assert m.melinoe_strerror(0) == "ok" and "argument" in m.melinoe_strerror(1)
+    assert m.melinoe_moe_expert_bytes(4096, 14336) == 352321536
+    assert m.melinoe_moe_expert_bytes(2048, 1024) == 12 * 2 ** 20
+    assert m.melinoe_moe_expert_bytes(0, 5) == 0
+
+
+def test_pack_expert_layout(m):
+    d, F = 256, 24
+    wg, wu, wd = gen.expert_weights(1, 0, 0, d, F)
+    blob = np.zeros(3 * d * F, np.uint16)
+    m.melinoe_moe_pack_expert(d, F, wg.ctypes.data, wu.ctypes.data, wd.ctypes.data, blob.ctypes.data)
+    gu = blob[: 2 * F * d].reshape(2 * F, d)
+    dt = blob[2 * F * d:].reshape(F, d)
+    assert np.array_equal(gu[0::2], wg) and np.array_equal(gu[1::2], wu)
+    assert np.array_equal(dt, wd.T)
+    with pytest.raises(m.MelinoeError):
+        m.melinoe_moe_pack_expert(d, F, 0, wu.ctypes.data, wd.ctypes.data, blob.ctypes.data)
+
+
+def test_create_fails_loudly_without_a_device(m):
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a device is present")
+    with pytest.raises(m.MelinoeError) as ei:
+        m.MoELayer(256, 64, 8, 2, 4)
+    assert ei.value.status == 3          # CUDA error, never a CPU fallback
