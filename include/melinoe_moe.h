@@ -14,7 +14,8 @@
  *  - A handle is driven by one host thread at a time, and all forward calls of one handle must
  *    be ordered with respect to each other on the device (same stream, or caller-made
  *    dependencies): a call's cache decisions depend on the previous call's.
- *  - melinoe_moe_forward is asynchronous with respect to the host.
+ *  - melinoe_moe_forward returns once the call's cache decisions are known to the host and all
+ *    of its transfers and kernels are queued; it does not wait for transfers or compute.
  */
 #ifndef MELINOE_MOE_H_
 #define MELINOE_MOE_H_
@@ -34,7 +35,7 @@ typedef enum melinoe_status {
     MELINOE_ERR_STATE = 2,       /* call order: e.g. forward before router / experts are set  */
     MELINOE_ERR_CUDA = 3,        /* a CUDA call failed; melinoe_last_cuda_error() has its code */
     MELINOE_ERR_NOMEM = 4,       /* device or host allocation failed                           */
-    MELINOE_ERR_TIMEOUT = 5,     /* a bounded device-side or service-side wait ran out         */
+    MELINOE_ERR_TIMEOUT = 5,     /* a bounded device-side or host-side wait ran out            */
     MELINOE_ERR_UNSUPPORTED = 6  /* shape outside what the kernels cover                       */
 } melinoe_status;
 
@@ -136,7 +137,14 @@ int melinoe_moe_reserve(melinoe_moe_t *h, int max_tokens);
  * cuda_stream: a cudaStream_t (NULL = legacy default stream).  hidden_dev [n_tokens][d_model]
  * bf16 and out_dev [n_tokens][d_model] bf16 are device memory, 16-byte aligned, borrowed
  * until the stream work of this call has finished.  stats_dev: see melinoe_moe_stats; may be
- * NULL.  n_tokens == 0 is a no-op.  Returns without waiting for the device.
+ * NULL.  n_tokens == 0 is a no-op.
+ *
+ * Host behaviour: the router, planning and resident-expert FFN kernels are queued first; the
+ * call then waits (bounded; TIMEOUT after 60 s) until the planning kernel has published the
+ * call's miss queue in page-locked memory, issues one cudaMemcpyAsync per missed expert on the
+ * handle's copy stream, ties the streams together with events, queues the remaining kernels and
+ * returns.  It therefore waits for earlier work on cuda_stream, but never for its own transfers,
+ * FFN kernels or combine.
  */
 int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_dev,
                         int n_tokens, void *out_dev, melinoe_moe_stats *stats_dev);

@@ -1,23 +1,21 @@
-// Host side of the C ABI: handle management, launch sequencing, and the transfer service that
-// turns the device-written miss queue into cudaMemcpyAsync calls on a side copy stream.
+// Host side of the C ABI: handle management, launch sequencing, and the miss path that turns
+// the device-written miss queue into cudaMemcpyAsync calls on a side copy stream.
 //
-// Ordering of one forward call on the caller's stream:
-//   router -> plan -> FFN(group 0: resident experts) -> [wait wave 1] FFN(group 1) -> ...
-//   -> combine.
-// The waits are stream memory operations (cuStreamWaitValue32) on a device word that the copy
-// stream advances (cuStreamWriteValue32) after each wave's transfers, so the host never blocks
-// in forward(), and a call without misses is released by the planning kernel itself without
-// touching the host at all.  The number of FFN launches is fixed per call shape
-// (1 + ceil(min(E, T*k) / C)); launches whose group turns out empty exit immediately.
-#include <cuda.h>
+// One forward call on the caller's stream:
+//   router -> plan -> FFN(group 0: experts resident at call entry)
+//   -> [host reads the miss queue; per miss wave: copies on the copy stream, event] ->
+//   wait(event) FFN(group 1) -> ... -> combine.
+// Group 0 is queued before the host knows the plan, so resident experts compute while the
+// miss queue travels to the host and while the transfers run.  Every cross-stream dependency
+// is a CUDA event (copy stream -> compute stream for arrival, compute stream -> copy stream
+// when a wave overwrites a slot that an earlier group of the same call still reads), so the
+// ordering is visible to the driver and cannot deadlock however streams share hardware queues.
 #include <cuda_runtime.h>
 
 #include <atomic>
 #include <chrono>
-#include <condition_variable>
 #include <cstdlib>
 #include <cstring>
-#include <mutex>
 #include <new>
 #include <thread>
 #include <vector>
@@ -36,23 +34,6 @@ void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
 }  // namespace melinoe
 
 namespace {
-
-typedef CUresult (*stream_value_fn)(CUstream, CUdeviceptr, cuuint32_t, unsigned int);
-stream_value_fn g_wait_value = nullptr, g_write_value = nullptr;
-std::once_flag g_entry_once;
-
-void load_entry_points()
-{
-    std::call_once(g_entry_once, [] {
-        cudaDriverEntryPointQueryResult qr;
-        void *fw = nullptr, *fr = nullptr;
-        if (cudaGetDriverEntryPoint("cuStreamWaitValue32", &fw, cudaEnableDefault, &qr) == cudaSuccess)
-            g_wait_value = reinterpret_cast<stream_value_fn>(fw);
-        if (cudaGetDriverEntryPoint("cuStreamWriteValue32", &fr, cudaEnableDefault, &qr) == cudaSuccess)
-            g_write_value = reinterpret_cast<stream_value_fn>(fr);
-        (void)cudaGetLastError();
-    });
-}
 
 int cuda_fail(cudaError_t e)
 {
@@ -88,7 +69,6 @@ struct melinoe_moe {
     char *slots = nullptr;
     DevCache *cache = nullptr;
     DevPlan *plan = nullptr;
-    uint32_t *arrive_word = nullptr;
     int *err_word = nullptr;
     const char **shared_dev = nullptr;
 
@@ -107,22 +87,18 @@ struct melinoe_moe {
     int n_seq = 0, n_shared = 0;
     std::vector<const void *> host_experts;
 
-    // page-locked host memory
+    // page-locked host memory: the miss queue the planning kernel writes
     HostPlan *hplan = nullptr;
-    uint32_t *done_word = nullptr;
 
     cudaStream_t copy_stream = nullptr;
-    cudaEvent_t ev_last = nullptr;
+    cudaEvent_t ev_last = nullptr;      // end of the most recent call on the caller's stream
+    cudaEvent_t ev_plan = nullptr;      // caller's stream: the planning kernel of the current call is done
+    cudaEvent_t ev_arrive = nullptr;    // copy stream: a wave's transfers have landed
+    std::vector<cudaEvent_t> ev_group;  // compute stream: FFN group g of the current call is done
     bool has_last = false;
-    uint32_t call_seq = 0, arrive_base = 0, done_base = 0;
+    uint32_t call_seq = 0;
     int last_T = 0;
-
-    // shared with the service thread
-    std::atomic<uint32_t> enqueued{0};
-    uint32_t serviced_seq = 0;
-    std::atomic<uint32_t> retired{0};
     std::atomic<int> sticky{0};
-    bool inline_service = false;
 
     // kernel timing
     bool timing = false;
@@ -130,162 +106,6 @@ struct melinoe_moe {
 };
 
 namespace {
-
-// ---------------------------------------------------------------- transfer service
-
-// Issue the transfers of the call whose plan record sits in h->hplan.  Called with the record
-// already validated (snapshot taken by the caller).
-void issue_transfers(melinoe_moe *h, const HostPlan &hp)
-{
-    if (hp.n_miss <= 0 || hp.status != MELINOE_OK)
-        return;  // the planning kernel released the waves itself
-    int cur_group = -1;
-    auto signal = [&](uint32_t value) {
-        CUresult r = g_write_value((CUstream)h->copy_stream, (CUdeviceptr)(uintptr_t)h->arrive_word, value, 0);
-        if (r != CUDA_SUCCESS) {
-            // last resort so the compute stream is never left waiting: write from the host
-            h->sticky.store(MELINOE_ERR_CUDA);
-            cudaStreamSynchronize(h->copy_stream);
-            cudaMemcpy(h->arrive_word, &value, 4, cudaMemcpyHostToDevice);
-        }
-    };
-    for (int i = 0; i < hp.n_miss; ++i) {
-        const HostMiss m = hp.miss[i];
-        if (m.group != cur_group) {
-            if (cur_group >= 0)
-                signal(hp.arrive_base + (uint32_t)cur_group);
-            cur_group = m.group;
-        }
-        if (m.dep_group >= 0) {
-            // the slot still feeds an earlier compute group of this call: wait for that group
-            const uint32_t target = hp.done_base + (uint32_t)m.dep_group + 1u;
-            const double t0 = now_s();
-            while ((int32_t)(*(volatile uint32_t *)h->done_word - target) < 0) {
-                if (now_s() - t0 > 20.0) {
-                    h->sticky.store(MELINOE_ERR_TIMEOUT);
-                    break;
-                }
-            }
-        }
-        bool ok = m.expert >= 0 && m.expert < h->E && m.slot >= 0 && m.slot < h->C;
-        if (ok) {
-            cudaError_t e = cudaMemcpyAsync(h->slots + (size_t)m.slot * h->slot_stride, h->host_experts[m.expert],
-                                            h->expert_bytes, cudaMemcpyHostToDevice, h->copy_stream);
-            if (e != cudaSuccess) {
-                g_last_cuda_error.store((int)e);
-                h->sticky.store(MELINOE_ERR_CUDA);
-            }
-        } else {
-            h->sticky.store(MELINOE_ERR_STATE);
-        }
-    }
-    signal(hp.arrive_base + hp.gmax - 1u);
-}
-
-// Look at a handle's plan record; if a new, consistent one is there, serve it.
-// Returns the number of calls retired.
-uint32_t poll_handle(melinoe_moe *h)
-{
-    volatile HostPlan *vp = h->hplan;
-    const uint32_t s = vp->seq;
-    if (s == h->serviced_seq)
-        return 0;
-    std::atomic_thread_fence(std::memory_order_acquire);
-    HostPlan snap;
-    snap.n_miss = vp->n_miss;
-    snap.n_groups = vp->n_groups;
-    snap.status = vp->status;
-    snap.arrive_base = vp->arrive_base;
-    snap.done_base = vp->done_base;
-    snap.gmax = vp->gmax;
-    const int nm = snap.n_miss < 0 ? 0 : (snap.n_miss > kMaxExperts ? kMaxExperts : snap.n_miss);
-    for (int i = 0; i < nm; ++i) {
-        snap.miss[i].expert = vp->miss[i].expert;
-        snap.miss[i].slot = vp->miss[i].slot;
-        snap.miss[i].group = vp->miss[i].group;
-        snap.miss[i].dep_group = vp->miss[i].dep_group;
-    }
-    std::atomic_thread_fence(std::memory_order_acquire);
-    if (vp->seq_open != s)
-        return 0;  // a later call without misses is overwriting the record: look again
-    snap.n_miss = nm;
-    issue_transfers(h, snap);
-    const uint32_t n = s - h->serviced_seq;
-    h->serviced_seq = s;
-    h->retired.fetch_add(n);
-    return n;
-}
-
-class Service {
-public:
-    static Service &get()
-    {
-        static Service *s = new Service();  // never destroyed: the thread may outlive static teardown
-        return *s;
-    }
-    void add(melinoe_moe *h)
-    {
-        std::lock_guard<std::mutex> lk(mu_);
-        handles_.push_back(h);
-        if (!started_) {
-            started_ = true;
-            std::thread(&Service::run, this).detach();
-        }
-    }
-    void remove(melinoe_moe *h)
-    {
-        std::lock_guard<std::mutex> lk(mu_);
-        for (size_t i = 0; i < handles_.size(); ++i)
-            if (handles_[i] == h) {
-                handles_.erase(handles_.begin() + i);
-                break;
-            }
-    }
-    void notify(melinoe_moe *h)
-    {
-        h->enqueued.fetch_add(1);
-        pending_.fetch_add(1);
-        std::lock_guard<std::mutex> lk(cv_mu_);
-        cv_.notify_one();
-    }
-
-private:
-    void run()
-    {
-        int cur_dev = -1;
-        for (;;) {
-            {
-                std::unique_lock<std::mutex> lk(cv_mu_);
-                cv_.wait(lk, [&] { return pending_.load() > 0; });
-            }
-            while (pending_.load() > 0) {
-                std::lock_guard<std::mutex> lk(mu_);
-                bool any = false;
-                for (melinoe_moe *h : handles_) {
-                    if (h->enqueued.load() == h->retired.load())
-                        continue;
-                    any = true;
-                    if (h->device != cur_dev) {
-                        cudaSetDevice(h->device);
-                        cur_dev = h->device;
-                    }
-                    const uint32_t n = poll_handle(h);
-                    if (n)
-                        pending_.fetch_sub((int)n);
-                }
-                if (!any) {
-                    // every live handle is drained (e.g. a handle was destroyed with calls pending)
-                    pending_.store(0);
-                }
-            }
-        }
-    }
-    std::mutex mu_, cv_mu_;
-    std::condition_variable cv_;
-    std::vector<melinoe_moe *> handles_;
-    std::atomic<int> pending_{0};
-    bool started_ = false;
-};
 
 // ---------------------------------------------------------------- helpers
 
@@ -330,15 +150,35 @@ int wait_idle(melinoe_moe *h)
     if (h->has_last)
         CU_TRY(cudaEventSynchronize(h->ev_last));
     CU_TRY(cudaStreamSynchronize(h->copy_stream));
-    if (!h->inline_service) {
-        const double t0 = now_s();
-        while (h->retired.load() != h->enqueued.load()) {
-            if (now_s() - t0 > 30.0)
-                return MELINOE_ERR_TIMEOUT;
+    return MELINOE_OK;
+}
+
+// Bounded host wait for the planning kernel of call `seq` to publish its miss queue.
+// ev_plan was recorded right behind that kernel.
+int wait_for_plan(melinoe_moe *h, uint32_t seq)
+{
+    volatile uint32_t *w = &h->hplan->seq;
+    for (int i = 0; i < 4096; ++i)
+        if (*w == seq)
+            return MELINOE_OK;
+    const double t0 = now_s();
+    for (;;) {
+        for (int i = 0; i < 256; ++i)
+            if (*w == seq)
+                return MELINOE_OK;
+        const double dt = now_s() - t0;
+        if (dt > 60.0)
+            return MELINOE_ERR_TIMEOUT;
+        if (dt > 0.001) {
+            // a long queue ahead of this call: stop burning the core, and notice a dead stream
             std::this_thread::yield();
+            const cudaError_t q = cudaEventQuery(h->ev_plan);
+            if (q == cudaSuccess)
+                return *w == seq ? MELINOE_OK : MELINOE_ERR_STATE;  // kernel done, record absent
+            if (q != cudaErrorNotReady)
+                return cuda_fail(q);
         }
     }
-    return MELINOE_OK;
 }
 
 int ensure_capacity(melinoe_moe *h, int T)
@@ -444,9 +284,6 @@ int melinoe_moe_create(int d, int F, int E, int k, int C, melinoe_moe_t **out)
         if (e != cudaSuccess)
             return cuda_fail(e);  // no usable device: there is no other execution path
     }
-    load_entry_points();
-    if (!g_wait_value || !g_write_value)
-        return MELINOE_ERR_UNSUPPORTED;
     melinoe_moe *h = new (std::nothrow) melinoe_moe();
     if (!h)
         return MELINOE_ERR_NOMEM;
@@ -458,8 +295,6 @@ int melinoe_moe_create(int d, int F, int E, int k, int C, melinoe_moe_t **out)
     h->expert_bytes = melinoe_moe_expert_bytes(d, F);
     h->slot_stride = (h->expert_bytes + 1023) / 1024 * 1024;
     h->host_experts.assign(E, nullptr);
-    const char *mode = std::getenv("MELINOE_SERVICE");
-    h->inline_service = mode && std::strcmp(mode, "inline") == 0;
     int rc = MELINOE_OK;
     auto fail = [&](int code) {
         melinoe_moe_destroy(h);
@@ -482,11 +317,9 @@ int melinoe_moe_create(int d, int F, int E, int k, int C, melinoe_moe_t **out)
     CR(cudaMalloc(&h->slots, h->slot_stride * (size_t)C));
     CR(cudaMalloc(&h->cache, sizeof(DevCache)));
     CR(cudaMalloc(&h->plan, sizeof(DevPlan)));
-    CR(cudaMalloc(&h->arrive_word, 256));
     CR(cudaMalloc(&h->err_word, 256));
     CR(cudaMalloc(&h->shared_dev, sizeof(char *) * kMaxShared));
     CR(cudaMalloc(&h->stage_stats, sizeof(melinoe_moe_stats)));
-    CR(cudaMemset(h->arrive_word, 0, 256));
     CR(cudaMemset(h->err_word, 0, 256));
     CR(cudaMemset(h->plan, 0, sizeof(DevPlan)));
     CR(cudaMemset(h->shared_dev, 0, sizeof(char *) * kMaxShared));
@@ -494,14 +327,12 @@ int melinoe_moe_create(int d, int F, int E, int k, int C, melinoe_moe_t **out)
     init_cache_host(c0);
     CR(cudaMemcpy(h->cache, &c0, sizeof c0, cudaMemcpyHostToDevice));
     CR(cudaHostAlloc(&h->hplan, sizeof(HostPlan), cudaHostAllocMapped | cudaHostAllocPortable));
-    CR(cudaHostAlloc(&h->done_word, 256, cudaHostAllocMapped | cudaHostAllocPortable));
     std::memset(h->hplan, 0, sizeof(HostPlan));
-    std::memset(h->done_word, 0, 256);
     CR(cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking));
     CR(cudaEventCreateWithFlags(&h->ev_last, cudaEventDisableTiming));
+    CR(cudaEventCreateWithFlags(&h->ev_plan, cudaEventDisableTiming));
+    CR(cudaEventCreateWithFlags(&h->ev_arrive, cudaEventDisableTiming));
 #undef CR
-    if (!h->inline_service)
-        Service::get().add(h);
     (void)rc;
     *out = h;
     return MELINOE_OK;
@@ -514,24 +345,25 @@ int melinoe_moe_destroy(melinoe_moe_t *h)
     int rc = MELINOE_OK;
     if (h->copy_stream)
         rc = wait_idle(h);
-    if (!h->inline_service)
-        Service::get().remove(h);
     free_scratch(h);
     cudaFree(h->slots);
     cudaFree(h->cache);
     cudaFree(h->plan);
-    cudaFree(h->arrive_word);
     cudaFree(h->err_word);
     cudaFree(h->shared_dev);
     cudaFree(h->stage_stats);
     if (h->hplan)
         cudaFreeHost(h->hplan);
-    if (h->done_word)
-        cudaFreeHost(h->done_word);
     if (h->copy_stream)
         cudaStreamDestroy(h->copy_stream);
     if (h->ev_last)
         cudaEventDestroy(h->ev_last);
+    if (h->ev_plan)
+        cudaEventDestroy(h->ev_plan);
+    if (h->ev_arrive)
+        cudaEventDestroy(h->ev_arrive);
+    for (cudaEvent_t e : h->ev_group)
+        cudaEventDestroy(e);
     for (auto &p : h->timed) {
         cudaEventDestroy(p.a);
         cudaEventDestroy(p.b);
@@ -640,8 +472,6 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
     const uint32_t gmax = (uint32_t)gmax_for(h, T);
     h->call_seq += 1;
     h->last_T = T;
-    if (!h->inline_service)
-        Service::get().notify(h);  // before any device work is queued: the service must be polling
 
     CU_TRY(launch_router(s, static_cast<const uint16_t *>(hidden_dev), h->w_router, h->bias, h->token_seq, T, h->d,
                          h->E, h->k, h->idx, h->gate, h->logits));
@@ -659,15 +489,13 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
     pp.inv_pos = h->inv_pos;
     pp.tok_of_sorted = h->tok_of_sorted;
     pp.hplan = h->hplan;
-    pp.arrive_word = h->arrive_word;
-    pp.arrive_base = h->arrive_base;
-    pp.done_base = h->done_base;
     pp.gmax = gmax;
     pp.call_seq = h->call_seq;
     pp.stats = stats_dev;
     pp.expert_bytes = h->expert_bytes;
     pp.vr_capacity = h->vr_capacity;
     CU_TRY(launch_plan(s, pp));
+    CU_TRY(cudaEventRecord(h->ev_plan, s));
 
     FfnParams fp;
     fp.slots = h->slots;
@@ -682,16 +510,7 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
     fp.d = h->d;
     fp.F = h->F;
     fp.E = h->E;
-    int status = MELINOE_OK;
-    for (uint32_t g = 0; g < gmax; ++g) {
-        if (g >= 1) {
-            CUresult r = g_wait_value((CUstream)s, (CUdeviceptr)(uintptr_t)h->arrive_word, h->arrive_base + g,
-                                      CU_STREAM_WAIT_VALUE_GEQ);
-            if (r != CUDA_SUCCESS) {
-                status = MELINOE_ERR_CUDA;
-                break;
-            }
-        }
+    auto launch_group = [&](int g) -> int {
         TimedPair tp{nullptr, nullptr};
         if (h->timing) {
             if (!h->free_pairs.empty()) {
@@ -703,55 +522,93 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
             }
             CU_TRY(cudaEventRecord(tp.a, s));
         }
-        fp.group = (int)g;
+        fp.group = g;
         CU_TRY(launch_ffn_stream(s, h->cfg, fp));
         if (h->timing) {
             CU_TRY(cudaEventRecord(tp.b, s));
             h->timed.push_back(tp);
         }
-        if (gmax > 2 && g + 1 < gmax) {
-            CUresult r = g_write_value((CUstream)s, (CUdeviceptr)(uintptr_t)h->done_word, h->done_base + g + 1u, 0);
-            if (r != CUDA_SUCCESS) {
-                status = MELINOE_ERR_CUDA;
-                break;
+        return MELINOE_OK;
+    };
+    // group 0 (experts resident at call entry, shared experts) goes out before the plan is known
+    rc = launch_group(0);
+    if (rc != MELINOE_OK)
+        return rc;
+
+    // the miss queue of this call
+    rc = wait_for_plan(h, h->call_seq);
+    if (rc != MELINOE_OK) {
+        h->sticky.store(rc);
+        return rc;
+    }
+    const HostPlan &hp = *h->hplan;
+    int n_miss = hp.n_miss, n_groups = hp.n_groups;
+    if (hp.status != MELINOE_OK || n_miss < 0 || n_miss > h->E || n_groups < 1 || n_groups > (int)gmax)
+        n_miss = 0, n_groups = 1;  // the device-side status already tells the caller; nothing to fetch
+    // which groups must signal their completion to the copy stream
+    bool need_done[kMaxGroups + 1] = {false};
+    for (int i = 0; i < n_miss; ++i)
+        if (hp.miss[i].dep_group >= 0 && hp.miss[i].dep_group <= kMaxGroups)
+            need_done[hp.miss[i].dep_group] = true;
+    auto group_event = [&](int g) -> cudaEvent_t {
+        while ((int)h->ev_group.size() <= g) {
+            cudaEvent_t e = nullptr;
+            if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess)
+                return nullptr;
+            h->ev_group.push_back(e);
+        }
+        return h->ev_group[g];
+    };
+    if (need_done[0]) {
+        cudaEvent_t e = group_event(0);
+        if (!e)
+            return cuda_fail(cudaGetLastError());
+        CU_TRY(cudaEventRecord(e, s));
+    }
+    int i = 0;
+    for (int g = 1; g < n_groups; ++g) {
+        for (; i < n_miss && hp.miss[i].group == g; ++i) {
+            const HostMiss m = hp.miss[i];
+            if (m.expert < 0 || m.expert >= h->E || m.slot < 0 || m.slot >= h->C || m.dep_group >= g) {
+                h->sticky.store(MELINOE_ERR_STATE);
+                return MELINOE_ERR_STATE;
             }
+            if (m.dep_group >= 0)  // the slot still feeds an earlier compute group of this call
+                CU_TRY(cudaStreamWaitEvent(h->copy_stream, h->ev_group[m.dep_group], 0));
+            CU_TRY(cudaMemcpyAsync(h->slots + (size_t)m.slot * h->slot_stride, h->host_experts[m.expert],
+                                   h->expert_bytes, cudaMemcpyHostToDevice, h->copy_stream));
+        }
+        CU_TRY(cudaEventRecord(h->ev_arrive, h->copy_stream));
+        CU_TRY(cudaStreamWaitEvent(s, h->ev_arrive, 0));
+        rc = launch_group(g);
+        if (rc != MELINOE_OK)
+            return rc;
+        if (need_done[g]) {
+            cudaEvent_t e = group_event(g);
+            if (!e)
+                return cuda_fail(cudaGetLastError());
+            CU_TRY(cudaEventRecord(e, s));
         }
     }
-    if (status == MELINOE_OK) {
-        CombineParams cp;
-        cp.plan = h->plan;
-        cp.idx = h->idx;
-        cp.gate = h->gate;
-        cp.inv_pos = h->inv_pos;
-        cp.part = h->part;
-        cp.out = static_cast<uint16_t *>(out_dev);
-        cp.T = T;
-        cp.d = h->d;
-        cp.k = h->k;
-        cp.E = h->E;
-        cp.n_shared = h->n_shared;
-        cp.grid = h->cfg.grid;
-        cp.units_per_vr = h->F / kUnitRows;
-        CU_TRY(launch_combine(s, cp));
-    }
+
+    CombineParams cp;
+    cp.plan = h->plan;
+    cp.idx = h->idx;
+    cp.gate = h->gate;
+    cp.inv_pos = h->inv_pos;
+    cp.part = h->part;
+    cp.out = static_cast<uint16_t *>(out_dev);
+    cp.T = T;
+    cp.d = h->d;
+    cp.k = h->k;
+    cp.E = h->E;
+    cp.n_shared = h->n_shared;
+    cp.grid = h->cfg.grid;
+    cp.units_per_vr = h->F / kUnitRows;
+    CU_TRY(launch_combine(s, cp));
     CU_TRY(cudaEventRecord(h->ev_last, s));
     h->has_last = true;
-    h->arrive_base += gmax;
-    h->done_base += gmax;
-
-    if (h->inline_service) {
-        // debugging mode: the calling thread serves this call's misses itself (blocks until the
-        // planning kernel has run)
-        const double t0 = now_s();
-        while (*(volatile uint32_t *)&h->hplan->seq != h->call_seq) {
-            if (now_s() - t0 > 30.0)
-                return MELINOE_ERR_TIMEOUT;
-        }
-        poll_handle(h);
-    }
-    if (status != MELINOE_OK)
-        h->sticky.store(status);
-    return status;
+    return MELINOE_OK;
 }
 
 int melinoe_moe_forward_host(melinoe_moe_t *h, void *cuda_stream, const void *hidden_host, int T, void *out_host,

@@ -24,8 +24,8 @@ struct PlanParams {
     VrRec *vrs;
     int32_t *perm, *inv_pos, *tok_of_sorted;
     HostPlan *hplan;          // page-locked host memory (device-visible address)
-    uint32_t *arrive_word;    // device word the compute stream waits on
-    uint32_t arrive_base, done_base, gmax, call_seq;
+    uint32_t gmax;            // compute groups the caller has room for
+    uint32_t call_seq;        // written to the miss queue's seq word when the record is complete
     melinoe_moe_stats *stats; // may be null
     size_t expert_bytes;
     int vr_capacity;

@@ -57,15 +57,14 @@ struct DevPlan {
     ReqRec req[kMaxReq];
 };
 
-// What the host-side transfer service needs to know about a call, written by the planning
-// kernel into page-locked host memory.  seq_open is written first, seq last.
+// The miss queue of a call: what the host needs in order to issue the transfers, written by
+// the planning kernel into page-locked host memory.  seq is written last (after a system-wide
+// fence); the host reads the record once seq equals the call's sequence number.
 struct HostMiss {
     int32_t expert, slot, group, dep_group;  // dep_group: compute group that must finish first, or -1
 };
 struct HostPlan {
-    uint32_t seq_open;
-    int32_t n_miss, n_groups, status;
-    uint32_t arrive_base, done_base, gmax, pad;
+    int32_t n_miss, n_groups, status, pad;
     HostMiss miss[kMaxExperts];
     uint32_t seq;
 };

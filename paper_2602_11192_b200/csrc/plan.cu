@@ -9,7 +9,7 @@
 //   (c) compute groups: group 0 = resident experts (+ shared experts); the misses follow in
 //       waves, a new wave starting whenever a miss would overwrite an expert of the current
 //       wave, so every wave's transfers can be in flight while earlier groups compute,
-//   (d) the miss queue for the host transfer service, in page-locked host memory, and
+//   (d) the miss queue, in page-locked host memory, from which the host issues the transfers, and
 //   (e) the call's statistics (hard miss count of Appendix C.1).
 #include "kernels.cuh"
 
@@ -315,14 +315,9 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p)
             *p.stats = st;
         }
         volatile HostPlan *hp = p.hplan;
-        hp->seq_open = p.call_seq;
-        __threadfence_system();
         hp->n_miss = n_miss;
         hp->n_groups = s_misc[4];
         hp->status = s_misc[6];
-        hp->arrive_base = p.arrive_base;
-        hp->done_base = p.done_base;
-        hp->gmax = p.gmax;
         for (int i = 0; i < n_miss; ++i) {
             hp->miss[i].expert = s_miss[i].expert;
             hp->miss[i].slot = s_miss[i].slot;
@@ -331,10 +326,6 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p)
         }
         __threadfence_system();
         hp->seq = p.call_seq;
-        if (n_miss == 0 || !ok) {
-            // nothing to wait for: release every wave of this call on the device
-            *reinterpret_cast<volatile uint32_t *>(p.arrive_word) = p.arrive_base + p.gmax - 1u;
-        }
         __threadfence_system();
     }
 }

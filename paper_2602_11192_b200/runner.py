@@ -82,6 +82,18 @@ class LayerSetup:
             list(ex.map(one, range(self.E)))
         self.layer.register_host_experts([base + e * eb for e in range(self.E)], eb, keep=self.store)
 
+    def set_shared_stacked(self, wg: torch.Tensor, wu: torch.Tensor, wd: torch.Tensor) -> None:
+        """Shared experts of the layer: wg/wu [n_shared][F][d], wd [n_shared][d][F] bf16 CPU tensors."""
+        assert wg.shape[0] == self.n_shared
+        tmp = torch.empty((self.n_shared, self.expert_bytes), dtype=torch.uint8)
+        for s in range(self.n_shared):
+            B.melinoe_moe_pack_expert(self.d, self.F, wg[s].data_ptr(), wu[s].data_ptr(), wd[s].data_ptr(),
+                                      tmp.data_ptr() + s * self.expert_bytes)
+        self.shared_store = tmp.cuda()
+        sb = self.shared_store.data_ptr()
+        self.layer.register_shared_experts([sb + s * self.expert_bytes for s in range(self.n_shared)],
+                                           keep=self.shared_store)
+
     def set_router(self, w_r_bits: np.ndarray) -> None:
         self.router_dev = to_dev_bf16(w_r_bits)
         self.layer.set_router(self.router_dev)
