@@ -68,7 +68,7 @@ typedef struct melinoe_moe_request {
  * Create one layer.  Shapes follow Eq. 1-3: router W_r [n_experts][d_model]; each expert has
  * W_g, W_u [d_ff][d_model] and W_d [d_model][d_ff].  Allocates, on the current device,
  * cache_slots expert slots of melinoe_moe_expert_bytes() each plus small tables, and creates
- * a copy stream.  Limits: d_model in {256, 512, 1024, 2048, 3072, 4096}, d_ff % 8 == 0,
+ * a copy stream.  Limits: d_model % 256 == 0, d_model <= 8192, d_ff % 8 == 0,
  * 1 <= top_k <= n_experts <= 64, top_k <= cache_slots <= n_experts  (INVALID / UNSUPPORTED
  * otherwise).
  */
@@ -83,12 +83,12 @@ int melinoe_moe_destroy(melinoe_moe_t *h);
 size_t melinoe_moe_expert_bytes(int d_model, int d_ff);
 
 /*
- * Pack one expert from the paper's matrix shapes (Eq. 3; bf16, row-major, host memory) into
- * the library's streaming layout (host memory, `melinoe_moe_expert_bytes` long):
- *     rows 0 .. 2*d_ff-1 of [d_model] values: row 2f = W_g[f][:], row 2f+1 = W_u[f][:]
- *     then d_ff rows of [d_model] values:      row f = W_d[:][f]   (W_d transposed)
- * so that every d_ff-slice of an expert is two contiguous byte ranges.  Pure host code; does
- * not touch the device.  blob_out must not overlap the inputs.
+ * Pack one expert from the paper's matrices (Eq. 3; bf16, row-major, host memory) into one
+ * contiguous blob (host memory, `melinoe_moe_expert_bytes` long):
+ *     W_g [d_ff][d_model] | W_u [d_ff][d_model] | W_d [d_model][d_ff]
+ * i.e. the three matrices back to back in the paper's own shapes, so every row that a kernel
+ * streams is one contiguous byte range.  Pure host code; does not touch the device.  blob_out
+ * must not overlap the inputs.
  */
 int melinoe_moe_pack_expert(int d_model, int d_ff, const void *w_gate_host, const void *w_up_host,
                             const void *w_down_host, void *blob_out_host);

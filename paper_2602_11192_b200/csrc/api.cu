@@ -4,7 +4,7 @@
 // One forward call on the caller's stream:
 //   router -> plan -> FFN(group 0: experts resident at call entry)
 //   -> [host reads the miss queue; per miss wave: copies on the copy stream, event] ->
-//   wait(event) FFN(group 1) -> ... -> combine.
+//   wait(event) FFN(group 1) -> ...   (the last group's FFN kernel also does the combine).
 // Group 0 is queued before the host knows the plan, so resident experts compute while the
 // miss queue travels to the host and while the transfers run.  Every cross-stream dependency
 // is a CUDA event (copy stream -> compute stream for arrival, compute stream -> copy stream
@@ -75,7 +75,9 @@ struct melinoe_moe {
     // scratch sized for cap_tokens
     int cap_tokens = 0, cap_shared = -1, vr_capacity = 0;
     int32_t *idx = nullptr, *perm = nullptr, *inv_pos = nullptr, *tok_of_sorted = nullptr;
-    float *gate = nullptr, *logits = nullptr, *part = nullptr;
+    float *gate = nullptr, *logits = nullptr, *zbuf = nullptr;
+    uint16_t *hbuf = nullptr;
+    unsigned *sync = nullptr, *row_done = nullptr;
     VrRec *vrs = nullptr;
     uint16_t *stage_in = nullptr, *stage_out = nullptr;
     melinoe_moe_stats *stage_stats = nullptr;
@@ -134,12 +136,14 @@ void free_scratch(melinoe_moe *h)
     cudaFree(h->tok_of_sorted);
     cudaFree(h->gate);
     cudaFree(h->logits);
-    cudaFree(h->part);
+    cudaFree(h->zbuf);
+    cudaFree(h->hbuf);
     cudaFree(h->vrs);
     cudaFree(h->stage_in);
     cudaFree(h->stage_out);
     h->idx = h->perm = h->inv_pos = h->tok_of_sorted = nullptr;
-    h->gate = h->logits = h->part = nullptr;
+    h->gate = h->logits = h->zbuf = nullptr;
+    h->hbuf = nullptr;
     h->vrs = nullptr;
     h->stage_in = h->stage_out = nullptr;
     h->cap_tokens = 0;
@@ -194,7 +198,8 @@ int ensure_capacity(melinoe_moe *h, int T)
     const size_t pairs = (size_t)cap * h->k;
     const size_t sorted = pairs + (size_t)h->n_shared * cap;
     const int vr_cap = (int)(pairs / kTokPerVr) + h->E + h->n_shared * (cap / kTokPerVr + 1) + 8;
-    const size_t part_rows = ((size_t)gmax_for(h, cap) * h->cfg.grid + vr_cap) * kTokPerVr;
+    const size_t fpad = ((size_t)h->F + 255) / 256 * 256;
+    const size_t hbytes = (size_t)vr_cap * kTokPerVr * fpad * 2;
     CU_TRY(cudaMalloc(&h->idx, pairs * 4));
     CU_TRY(cudaMalloc(&h->gate, pairs * 4));
     CU_TRY(cudaMalloc(&h->logits, (size_t)cap * h->E * 4));
@@ -202,7 +207,9 @@ int ensure_capacity(melinoe_moe *h, int T)
     CU_TRY(cudaMalloc(&h->inv_pos, pairs * 4));
     CU_TRY(cudaMalloc(&h->tok_of_sorted, sorted * 4));
     CU_TRY(cudaMalloc(&h->vrs, (size_t)vr_cap * sizeof(VrRec)));
-    CU_TRY(cudaMalloc(&h->part, part_rows * h->d * sizeof(float)));
+    CU_TRY(cudaMalloc(&h->zbuf, sorted * h->d * sizeof(float)));
+    CU_TRY(cudaMalloc(&h->hbuf, hbytes));
+    CU_TRY(cudaMemset(h->hbuf, 0, hbytes));   // the padding of every h row stays zero for good
     CU_TRY(cudaMalloc(&h->stage_in, (size_t)cap * h->d * 2));
     CU_TRY(cudaMalloc(&h->stage_out, (size_t)cap * h->d * 2));
     h->vr_capacity = vr_cap;
@@ -247,23 +254,11 @@ int melinoe_moe_pack_expert(int d, int F, const void *wg_, const void *wu_, cons
 {
     if (d <= 0 || F <= 0 || !wg_ || !wu_ || !wd_ || !blob_)
         return MELINOE_ERR_INVALID;
-    const uint16_t *wg = static_cast<const uint16_t *>(wg_);
-    const uint16_t *wu = static_cast<const uint16_t *>(wu_);
-    const uint16_t *wd = static_cast<const uint16_t *>(wd_);
-    uint16_t *blob = static_cast<uint16_t *>(blob_);
-    for (int f = 0; f < F; ++f) {
-        std::memcpy(blob + (size_t)(2 * f) * d, wg + (size_t)f * d, (size_t)d * 2);
-        std::memcpy(blob + (size_t)(2 * f + 1) * d, wu + (size_t)f * d, (size_t)d * 2);
-    }
-    uint16_t *dt = blob + (size_t)2 * F * d;  // [F][d], dt[f][r] = wd[r][f]
-    constexpr int B = 32;
-    for (int r0 = 0; r0 < d; r0 += B)
-        for (int f0 = 0; f0 < F; f0 += B) {
-            const int r1 = r0 + B < d ? r0 + B : d, f1 = f0 + B < F ? f0 + B : F;
-            for (int r = r0; r < r1; ++r)
-                for (int f = f0; f < f1; ++f)
-                    dt[(size_t)f * d + r] = wd[(size_t)r * F + f];
-        }
+    const size_t m = (size_t)d * F * 2;
+    char *blob = static_cast<char *>(blob_);
+    std::memcpy(blob, wg_, m);
+    std::memcpy(blob + m, wu_, m);
+    std::memcpy(blob + 2 * m, wd_, m);
     return MELINOE_OK;
 }
 
@@ -274,7 +269,7 @@ int melinoe_moe_create(int d, int F, int E, int k, int C, melinoe_moe_t **out)
     *out = nullptr;
     if (d <= 0 || F <= 0 || E <= 0 || k <= 0 || C <= 0 || k > E || C < k || C > E)
         return MELINOE_ERR_INVALID;
-    if (d % 256 != 0 || F % kUnitRows != 0 || E > kMaxExperts || !ffn_stream_supported(d))
+    if (d % 256 != 0 || d > 8192 || F % kUnitRows != 0 || E > kMaxExperts)
         return MELINOE_ERR_UNSUPPORTED;
     {
         int dev = 0;
@@ -306,8 +301,11 @@ int melinoe_moe_create(int d, int F, int E, int k, int C, melinoe_moe_t **out)
     if (prop.major != 10)
         return fail(MELINOE_ERR_UNSUPPORTED);
     h->n_sms = prop.multiProcessorCount;
-    if (ffn_stream_configure(d, h->n_sms, prop.sharedMemPerBlockOptin, &h->cfg) != cudaSuccess)
+    if (!prop.cooperativeLaunch ||
+        ffn_stream_configure(h->n_sms, prop.sharedMemPerBlockOptin, &h->cfg) != cudaSuccess) {
+        (void)cudaGetLastError();
         return fail(MELINOE_ERR_UNSUPPORTED);
+    }
 #define CR(expr)                                   \
     do {                                           \
         cudaError_t e__ = (expr);                  \
@@ -318,6 +316,10 @@ int melinoe_moe_create(int d, int F, int E, int k, int C, melinoe_moe_t **out)
     CR(cudaMalloc(&h->cache, sizeof(DevCache)));
     CR(cudaMalloc(&h->plan, sizeof(DevPlan)));
     CR(cudaMalloc(&h->err_word, 256));
+    CR(cudaMalloc(&h->sync, sizeof(unsigned) * (kMaxGroups + 1)));
+    CR(cudaMalloc(&h->row_done, sizeof(unsigned) * (d / 16)));
+    CR(cudaMemset(h->sync, 0, sizeof(unsigned) * (kMaxGroups + 1)));
+    CR(cudaMemset(h->row_done, 0, sizeof(unsigned) * (d / 16)));
     CR(cudaMalloc(&h->shared_dev, sizeof(char *) * kMaxShared));
     CR(cudaMalloc(&h->stage_stats, sizeof(melinoe_moe_stats)));
     CR(cudaMemset(h->err_word, 0, 256));
@@ -350,6 +352,8 @@ int melinoe_moe_destroy(melinoe_moe_t *h)
     cudaFree(h->cache);
     cudaFree(h->plan);
     cudaFree(h->err_word);
+    cudaFree(h->sync);
+    cudaFree(h->row_done);
     cudaFree(h->shared_dev);
     cudaFree(h->stage_stats);
     if (h->hplan)
@@ -489,6 +493,7 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
     pp.inv_pos = h->inv_pos;
     pp.tok_of_sorted = h->tok_of_sorted;
     pp.hplan = h->hplan;
+    pp.sync = h->sync;
     pp.gmax = gmax;
     pp.call_seq = h->call_seq;
     pp.stats = stats_dev;
@@ -504,12 +509,22 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
     fp.plan = h->plan;
     fp.vrs = h->vrs;
     fp.tok_of_sorted = h->tok_of_sorted;
+    fp.perm = h->perm;
     fp.x = static_cast<const uint16_t *>(hidden_dev);
-    fp.part = h->part;
+    fp.gate = h->gate;
+    fp.hbuf = h->hbuf;
+    fp.zbuf = h->zbuf;
+    fp.out = static_cast<uint16_t *>(out_dev);
+    fp.sync = h->sync;
+    fp.row_done = h->row_done;
     fp.err = h->err_word;
     fp.d = h->d;
     fp.F = h->F;
+    fp.Fpad = (h->F + 255) / 256 * 256;
     fp.E = h->E;
+    fp.k = h->k;
+    fp.T = T;
+    fp.n_shared = h->n_shared;
     auto launch_group = [&](int g) -> int {
         TimedPair tp{nullptr, nullptr};
         if (h->timing) {
@@ -591,21 +606,6 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
         }
     }
 
-    CombineParams cp;
-    cp.plan = h->plan;
-    cp.idx = h->idx;
-    cp.gate = h->gate;
-    cp.inv_pos = h->inv_pos;
-    cp.part = h->part;
-    cp.out = static_cast<uint16_t *>(out_dev);
-    cp.T = T;
-    cp.d = h->d;
-    cp.k = h->k;
-    cp.E = h->E;
-    cp.n_shared = h->n_shared;
-    cp.grid = h->cfg.grid;
-    cp.units_per_vr = h->F / kUnitRows;
-    CU_TRY(launch_combine(s, cp));
     CU_TRY(cudaEventRecord(h->ev_last, s));
     h->has_last = true;
     return MELINOE_OK;
@@ -647,6 +647,7 @@ int melinoe_moe_reset_cache(melinoe_moe_t *h)
     init_cache_host(c0);
     CU_TRY(cudaMemcpy(h->cache, &c0, sizeof c0, cudaMemcpyHostToDevice));
     CU_TRY(cudaMemset(h->err_word, 0, 4));
+    CU_TRY(cudaMemset(h->row_done, 0, sizeof(unsigned) * (h->d / 16)));
     h->sticky.store(MELINOE_OK);
     return MELINOE_OK;
 }

@@ -1,36 +1,46 @@
-// Streaming SwiGLU expert FFN (Eq. 3) for calls with at most a few tokens per expert
-// (decode): the work is reading every needed expert once from HBM, so the kernel is built
-// around keeping the memory system full, not around arithmetic.
+// Streaming SwiGLU expert FFN (Eq. 3) with the gate-weighted combine (Eq. 2) fused in, for
+// calls with few tokens per expert (decode).  The work is reading every needed expert once
+// from HBM, so the kernel is built around keeping the memory system full.
 //
-// Work decomposition.  A "virtual request" is one expert with up to 8 of its tokens.  Each
-// virtual request is cut along d_ff into units of 8 rows; in the packed expert layout a unit
-// is two contiguous byte ranges: 16 rows of [W_g; W_u] interleaved and 8 rows of W_d^T.  All
-// units of the launch are split evenly over the CTAs (one per SM), so any number of experts
-// loads every SM equally.  A CTA that covers only part of an expert writes a partial output
-// row set; the combine kernel adds the partials in a fixed order.
+// One cooperative launch per compute group, one CTA per SM, eight independent warps per CTA.
+// A "virtual request" is one expert with up to 8 of its tokens.
 //
-// Per CTA: one producer warp issues bulk asynchronous copies (cp.async.bulk, completion on
-// mbarriers) of weight rows into a shared-memory ring, far ahead of the math; eight consumer
-// warps run the two small products with mma.sync (bf16 inputs, fp32 accumulation):
-//   phase 1  [g;u] (16 rows) x hidden (<= 8 tokens): weights are the 8-wide operand, the
-//            tokens the 16-wide one; each warp owns d/8 of the columns, partial sums meet in
-//            shared memory, h = bf16(SiLU(g) * u);
-//   phase 2  z += W_d^T rows (8) x h: each warp owns d/8 of the output columns and keeps its
-//            accumulators in registers across all units of the virtual request.
-// Weight rows land in shared memory at a pitch of 2*d + 16 bytes, which makes every ldmatrix
-// access (plain for phase 1, transposed for phase 2) conflict-free.
+//   phase 1  tile = 8 rows of W_g plus the same 8 rows of W_u of one virtual request.
+//            D[16 x 8] = [W_g rows; W_u rows] (16 x d) * x^T (d x 8 tokens) on mma.sync
+//            (bf16 in, fp32 accumulate).  In the accumulator layout a thread holds g_f and u_f
+//            of the same f and the same two tokens, so h = SiLU(g) * u is thread-local;
+//            h goes to global memory as bf16.
+//   barrier  grid-wide (bounded spin on a device counter); before waiting, each warp already
+//            has the first W_d stages of its phase-2 work in flight.
+//   phase 2  tile = 16 rows of W_d of one virtual request: D[16 x 8] = W_d rows (16 x F) * h^T.
+//            Every tile is a complete dot product over d_ff, so z needs no cross-CTA reduction
+//            and goes to z[pair][d] in fp32.
+//   combine  the warp that finishes the last tile of a 16-row block in the call's last
+//            compute group sums gate * z over the ranks in rank order (plus shared experts)
+//            and writes the bf16 output rows.  The result does not depend on which warp does
+//            it, nor on how the experts were split over groups.
 //
-// Every wait is bounded: if an mbarrier wait runs out, the CTA raises an abort flag, skips
-// all later waits, finishes its loops without hanging and reports through the error word.
+// Data movement: every warp owns a private ring of S stages in shared memory.  A stage holds
+// a KC-column slice of the tile's 16 weight rows plus the matching slice of up to 8 operand rows
+// (hidden rows in phase 1, h rows in phase 2), each fetched by its own cp.async.bulk (one lane
+// per row) completing on the stage's mbarrier.  Rows sit at a pitch of 2*KC+16 bytes, which
+// makes the ldmatrix reads and the operand-fragment reads bank-conflict free.  There is no
+// CTA-wide synchronisation after start-up.
+//
+// Every wait is bounded: when an mbarrier or the grid barrier does not complete in time the
+// warp raises the CTA's abort flag, later waits fall through, the kernel ends normally and the
+// error word tells the host.
+#include <cooperative_groups.h>
+
 #include "kernels.cuh"
 
 namespace melinoe {
 
 namespace {
 
-constexpr int kConsumerWarps = 8;
-constexpr int kFfnThreads = (kConsumerWarps + 1) * 32;
-constexpr int kMaxStages = 16;
+constexpr int kWarps = 8;
+constexpr int kThreads = kWarps * 32;
+constexpr int kStageRows = 24;            // 16 weight rows + 8 operand rows
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p)
@@ -61,13 +71,13 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity)
 // Bounded wait.  Returns false (and raises the CTA's abort flag) when the limit runs out.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
 {
-    if (*abort_flag)
-        return false;
     if (mbar_try(bar, parity))
         return true;
+    if (*abort_flag)
+        return false;
     const unsigned long long t0 = globaltimer_ns();
     for (;;) {
-        for (int i = 0; i < 256; ++i)
+        for (int i = 0; i < 64; ++i)
             if (mbar_try(bar, parity))
                 return true;
         if (*abort_flag)
@@ -79,16 +89,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
 }
 
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-
-__device__ __forceinline__ void consumer_bar()
-{
-    asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory");
-}
-
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3)
 {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
@@ -96,334 +96,419 @@ __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t &r0, uint32_
                  : "r"(addr));
 }
 
-__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2,
-                                                  uint32_t &r3)
+// D(16x8) += A(16x16) * B(16x8), bf16 in, fp32 accumulate.
+__device__ __forceinline__ void mma_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                          uint32_t b0, uint32_t b1)
 {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
-                 : "r"(addr));
-}
-
-// D(16x8) += A(16x16) * B(16x8), bf16 in, fp32 accumulate.  Rows 8..15 of A are zero here.
-__device__ __forceinline__ void mma_k16_top(float (&c)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1)
-{
-    const uint32_t z = 0u;
     asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-                 : "r"(a0), "r"(z), "r"(a2), "r"(z), "r"(b0), "r"(b1));
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// D(16x8) += A(16x8) * B(8x8)
-__device__ __forceinline__ void mma_k8(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t b0)
+__device__ __forceinline__ uint32_t lds32(uint32_t addr)
 {
-    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%0,%1,%2,%3};"
-                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-                 : "r"(a0), "r"(a1), "r"(b0));
+    uint32_t v;
+    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
 }
 
-__device__ __forceinline__ uint32_t f32_to_bf16_rne_bits(float v)
+__device__ __forceinline__ uint16_t bf16_rne(float v)
 {
     uint32_t u = __float_as_uint(v);
     u += 0x7fffu + ((u >> 16) & 1u);
-    return u >> 16;
+    return (uint16_t)(u >> 16);
 }
 
-// KW = d / 8: the columns one consumer warp owns in both phases.
-template <int KW>
-__global__ void __launch_bounds__(kFfnThreads, 1)
-ffn_stream_kernel(FfnParams p, int rpe, int ns)
+__device__ __forceinline__ void fence_proxy_async()
 {
-    constexpr int KS2 = KW / 32;   // pairs of 16-wide k-steps in phase 1
-    constexpr int MT2 = KW / 32;   // pairs of 16-row output tiles in phase 2
+    asm volatile("fence.proxy.async;" ::: "memory");
+}
+
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+
+__device__ __forceinline__ void mbar_expect(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+
+// What a warp needs to know about the tile it fetches or computes.
+struct Tile {
+    const char *src;     // this lane's source row (weights: lanes 0..15, operand rows: lanes 16..23)
+    int n_tok;           // tokens of the virtual request
+    int vr;              // virtual request (index within the call)
+    int blk;             // f-block (phase 1) or 16-row block (phase 2)
+};
+
+template <int KC, int S>
+__global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p)
+{
+    constexpr int PITCH = 2 * KC + 16;
+    constexpr int STAGE = kStageRows * PITCH;
+    constexpr int KSTEPS = KC / 16;
 
     extern __shared__ __align__(128) unsigned char smem[];
-    const int d = p.d, F = p.F;
-    const int P = 2 * d + 16;                    // smem pitch of one weight / hidden row
-    const int row_bytes = 2 * d;
-    const int entry_bytes = rpe * P;
-    unsigned char *ring = smem;
-    unsigned char *xs = ring + (size_t)ns * entry_bytes;
-    float *s_part = reinterpret_cast<float *>(xs + 8 * P);
-    uint32_t *s_h32 = reinterpret_cast<uint32_t *>(s_part + kConsumerWarps * 2 * 8 * 8);
-    uint64_t *bars = reinterpret_cast<uint64_t *>(s_h32 + 32);
-    volatile int *s_abort = reinterpret_cast<volatile int *>(bars + 2 * kMaxStages);
-
-    const DevPlan *plan = p.plan;
-    const int vr_begin = plan->group_vr_begin[p.group];
-    const int nvr = plan->group_vr_begin[p.group + 1] - vr_begin;
-    if (nvr <= 0)
-        return;
-    const int upe = F / kUnitRows;
-    const long long NU = (long long)nvr * upe;
-    // CTAs that share this launch: never more than there are units, so no CTA's range is empty
-    const long long G = NU < (long long)gridDim.x ? NU : (long long)gridDim.x;
-    if ((long long)blockIdx.x >= G)
-        return;
-    const long long u0 = (long long)blockIdx.x * NU / G;
-    const long long u1 = (long long)(blockIdx.x + 1) * NU / G;
-    if (u0 >= u1)
-        return;
+    __shared__ int s_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + kMaxStages);
-    if (tid == 0) {
-        *s_abort = 0;
-        for (int i = 0; i < ns; ++i) {
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(full0 + 8 * i), "r"(1));
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(empty0 + 8 * i), "r"(kConsumerWarps));
-        }
+    const int g = lane >> 2, tig = lane & 3;
+    const int d = p.d, F = p.F, Fpad = p.Fpad;
+    const DevPlan *plan = p.plan;
+    const int G = (int)gridDim.x;
+
+    if (plan->status != MELINOE_OK) {
+        // the call was refused on the device: the output is all zeros, the status tells why
+        if (p.group == 0)
+            for (size_t i = (size_t)blockIdx.x * kThreads + tid; i < (size_t)p.T * d; i += (size_t)G * kThreads)
+                p.out[i] = 0;
+        return;
+    }
+    const int vb = plan->group_vr_begin[p.group];
+    const int nv = plan->group_vr_begin[p.group + 1] - vb;
+    const bool final_group = p.group == plan->n_groups - 1;
+    if (nv <= 0 && !final_group)
+        return;
+
+    unsigned char *ring = smem + (size_t)warp * S * STAGE;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + (size_t)kWarps * S * STAGE) + warp * S;
+    const uint32_t ring_s = smem_u32(ring), bar_s = smem_u32(bars);
+    volatile int *abort_flag = &s_abort;
+
+    if (tid == 0)
+        s_abort = 0;
+    if (lane == 0) {
+        for (int i = 0; i < S; ++i)
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar_s + 8 * i), "r"(1));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (F % KC != 0) {
+        // the last d_ff slice of a W_d row is shorter than a stage row: what it leaves untouched
+        // must be finite, because it meets zeros of the padded h rows in the product
+        uint4 *z = reinterpret_cast<uint4 *>(ring);
+        for (int i = lane; i < S * STAGE / 16; i += 32)
+            z[i] = make_uint4(0, 0, 0, 0);
+        fence_proxy_async();
     }
     __syncthreads();
 
-    const int epu = 24 / rpe;      // ring entries per unit
-    const int gue = 16 / rpe;      // of which [W_g;W_u] rows
-    const int half = 8 / rpe;      // entries per 8 rows
-    const uint32_t ring_s = smem_u32(ring);
+    // ---- this warp's tiles: a contiguous range per CTA, dealt round-robin to its warps
+    const int upe1 = F / 8, upe2 = d / 16;
+    const int nk1 = d / KC, nk2 = (F + KC - 1) / KC;
+    const long long NT1 = (long long)nv * upe1, NT2 = (long long)nv * upe2;
+    const int lo1 = (int)(blockIdx.x * NT1 / G) + warp, hi1 = (int)((blockIdx.x + 1) * NT1 / G);
+    const int lo2 = (int)(blockIdx.x * NT2 / G) + warp, hi2 = (int)((blockIdx.x + 1) * NT2 / G);
 
-    if (warp == kConsumerWarps) {
-        // ------------------------------------------------------------ producer
+    auto blob_of = [&](const VrRec &v) -> const char * {
+        const ReqRec rec = plan->req[v.req];
+        return rec.slot >= 0 ? p.slots + (size_t)rec.slot * p.slot_stride : p.shared_blobs[rec.expert - p.E];
+    };
+    // lane's source row for a phase-1 tile: lanes 0..7 W_g rows, 8..15 W_u rows, 16..23 hidden rows
+    auto tile1 = [&](int t) -> Tile {
+        Tile ti;
+        ti.vr = vb + t / upe1;
+        ti.blk = t % upe1;
+        const VrRec v = p.vrs[ti.vr];
+        ti.n_tok = v.n_tok;
+        ti.src = nullptr;
+        if (lane < 16) {
+            const int row = (lane < 8 ? 0 : F) + ti.blk * 8 + (lane & 7);
+            ti.src = blob_of(v) + (size_t)row * d * 2;
+        } else if (lane - 16 < v.n_tok) {
+            const int tok = p.tok_of_sorted[v.tok_off + lane - 16];
+            ti.src = reinterpret_cast<const char *>(p.x) + (size_t)tok * d * 2;
+        }
+        return ti;
+    };
+    // phase 2: lanes 0..15 W_d rows, 16..23 rows of h
+    auto tile2 = [&](int t) -> Tile {
+        Tile ti;
+        ti.vr = vb + t / upe2;
+        ti.blk = t % upe2;
+        const VrRec v = p.vrs[ti.vr];
+        ti.n_tok = v.n_tok;
+        ti.src = nullptr;
+        if (lane < 16)
+            ti.src = blob_of(v) + ((size_t)2 * F * d + (size_t)(ti.blk * 16 + lane) * F) * 2;
+        else if (lane - 16 < v.n_tok)
+            ti.src = reinterpret_cast<const char *>(p.hbuf) + ((size_t)ti.vr * kTokPerVr + lane - 16) * Fpad * 2;
+        return ti;
+    };
+
+    uint32_t n_issued = 0, n_consumed = 0;   // stages, over both phases (ring slot and parity)
+
+    // issue one stage: parts bit 0 = weight rows and the barrier's byte count, bit 1 = operand rows
+    auto issue = [&](const Tile &ti, int kc, int wbytes, int parts, uint32_t n) {
+        const uint32_t slot = n % S;
+        const uint32_t bar = bar_s + 8 * slot;
+        if ((parts & 1) && lane == 0)
+            mbar_expect(bar, 16u * wbytes + (uint32_t)ti.n_tok * KC * 2);
+        __syncwarp();
+        if (ti.src) {
+            const bool is_w = lane < 16;
+            if (is_w ? (parts & 1) : (parts & 2))
+                bulk_g2s(ring_s + slot * STAGE + lane * PITCH, ti.src + (size_t)kc * KC * 2,
+                         is_w ? (uint32_t)wbytes : (uint32_t)(KC * 2), bar);
+        }
+    };
+
+    // the mma loop over one stage
+    const uint32_t a_off = ((lane & 7) + ((lane >> 3) & 1) * 8) * PITCH + (lane >> 4) * 16;
+    const uint32_t b_off = (16 + g) * PITCH + tig * 4;
+    auto compute = [&](uint32_t n, int n_tok, float (&c0)[4], float (&c1)[4]) {
+        const uint32_t slot = n % S;
+        mbar_wait(bar_s + 8 * slot, (n / S) & 1u, abort_flag);
+        const uint32_t base = ring_s + slot * STAGE;
+        const bool has_tok = g < n_tok;
+#pragma unroll
+        for (int ks = 0; ks < KSTEPS; ks += 2) {
+            uint32_t a0, a1, a2, a3, e0, e1, e2, e3;
+            ldmatrix_x4(base + a_off + ks * 32, a0, a1, a2, a3);
+            ldmatrix_x4(base + a_off + ks * 32 + 32, e0, e1, e2, e3);
+            uint32_t b0 = 0, b1 = 0, f0 = 0, f1 = 0;
+            if (has_tok) {
+                b0 = lds32(base + b_off + ks * 32);
+                b1 = lds32(base + b_off + ks * 32 + 16);
+                f0 = lds32(base + b_off + ks * 32 + 32);
+                f1 = lds32(base + b_off + ks * 32 + 48);
+            }
+            mma_16816(c0, a0, a1, a2, a3, b0, b1);
+            mma_16816(c1, e0, e1, e2, e3, f0, f1);
+        }
+        __syncwarp();
+    };
+
+    // =========================================================== phase 1: h = SiLU(W_g x) * (W_u x)
+    {
+        int pt = lo1, pk = 0, ct = lo1, ck = 0;
+        Tile ptile{}, ctile{};
+        if (pt < hi1)
+            ptile = tile1(pt);
+        ctile = ptile;
+        for (int i = 0; i < S && pt < hi1; ++i) {
+            issue(ptile, pk, KC * 2, 3, n_issued++);
+            if (++pk == nk1) {
+                pk = 0;
+                pt += kWarps;
+                if (pt < hi1)
+                    ptile = tile1(pt);
+            }
+        }
+        float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
+        while (ct < hi1) {
+            compute(n_consumed++, ctile.n_tok, c0, c1);
+            if (pt < hi1) {
+                issue(ptile, pk, KC * 2, 3, n_issued++);
+                if (++pk == nk1) {
+                    pk = 0;
+                    pt += kWarps;
+                    if (pt < hi1)
+                        ptile = tile1(pt);
+                }
+            }
+            if (++ck == nk1) {
+                // rows g and g + 8 of the tile are g_f and u_f for f = 8 * blk + g
+                const int f = ctile.blk * 8 + g;
+                const float gv0 = c0[0] + c1[0], gv1 = c0[1] + c1[1], uv0 = c0[2] + c1[2], uv1 = c0[3] + c1[3];
+                uint16_t *hrow = p.hbuf + ((size_t)ctile.vr * kTokPerVr) * Fpad + f;
+                if (tig * 2 < ctile.n_tok)
+                    hrow[(size_t)(tig * 2) * Fpad] = bf16_rne(gv0 / (1.0f + __expf(-gv0)) * uv0);
+                if (tig * 2 + 1 < ctile.n_tok)
+                    hrow[(size_t)(tig * 2 + 1) * Fpad] = bf16_rne(gv1 / (1.0f + __expf(-gv1)) * uv1);
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    c0[i] = c1[i] = 0.f;
+                ck = 0;
+                ct += kWarps;
+                if (ct < hi1)
+                    ctile = tile1(ct);
+            }
+        }
+    }
+
+    // =========================================================== grid barrier, W_d already in flight
+    __threadfence();
+    fence_proxy_async();       // h was written through the generic proxy, bulk copies will read it
+    __syncwarp();
+    if (lane == 0)
+        atomicAdd(p.sync + p.group, 1u);
+    int pt = lo2, pk = 0;
+    Tile ptile{};
+    if (pt < hi2)
+        ptile = tile2(pt);
+    auto wbytes2 = [&](int kc) { return 2 * min(KC, F - kc * KC); };
+    {
+        // first stages of phase 2: weight rows only; their h rows follow once h is complete
+        int qt = pt, qk = pk;
+        Tile qtile = ptile;
+        const uint32_t n0 = n_issued;
+        int pre = 0;
+        for (; pre < S && pt < hi2; ++pre) {
+            issue(ptile, pk, wbytes2(pk), 1, n_issued++);
+            if (++pk == nk2) {
+                pk = 0;
+                pt += kWarps;
+                if (pt < hi2)
+                    ptile = tile2(pt);
+            }
+        }
         if (lane == 0) {
-            long long n = 0;
-            bool stop = false;
-            for (long long u = u0; u < u1 && !stop; ++u) {
-                const int vr = vr_begin + (int)(u / upe);
-                const int fb = (int)(u % upe) * kUnitRows;
-                const ReqRec rec = plan->req[p.vrs[vr].req];
-                const char *blob = rec.slot >= 0 ? p.slots + (size_t)rec.slot * p.slot_stride
-                                                 : p.shared_blobs[rec.expert - p.E];
-                const char *gu = blob + (size_t)(2 * fb) * row_bytes;
-                const char *dt = blob + (size_t)(2 * F + fb) * row_bytes;
-                for (int e = 0; e < epu; ++e, ++n) {
-                    const int slot = (int)(n % ns);
-                    if (n >= ns && !mbar_wait(empty0 + 8 * slot, (uint32_t)((n / ns - 1) & 1), s_abort)) {
-                        stop = true;
+            const unsigned target = (unsigned)G * kWarps;
+            volatile unsigned *w = p.sync + p.group;
+            if (*w < target && !*abort_flag) {
+                const unsigned long long t0 = globaltimer_ns();
+                while (*w < target) {
+                    if (*abort_flag || globaltimer_ns() - t0 > kWaitLimitNs) {
+                        *abort_flag = 1;
                         break;
                     }
-                    const char *src = e < gue ? gu + (size_t)e * rpe * row_bytes
-                                              : dt + (size_t)(e - gue) * rpe * row_bytes;
-                    const uint32_t bar = full0 + 8 * slot;
-                    const uint32_t dst = ring_s + slot * entry_bytes;
-                    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar),
-                                 "r"(rpe * row_bytes)
-                                 : "memory");
-                    for (int r = 0; r < rpe; ++r) {
-                        asm volatile(
-                            "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                            ::"r"(dst + r * P), "l"(src + (size_t)r * row_bytes), "r"(row_bytes), "r"(bar)
-                            : "memory");
-                    }
                 }
             }
-            if (stop) {
-                // the consumers gave up or a wait ran out: let the copies already issued land
-                // (bounded) before this CTA's shared memory goes away
-                const long long first = n > ns ? n - ns : 0;
-                const unsigned long long t0 = globaltimer_ns();
-                for (long long m = first; m < n; ++m) {
-                    const uint32_t bar = full0 + 8 * (int)(m % ns);
-                    const uint32_t par = (uint32_t)((m / ns) & 1);
-                    while (!mbar_try(bar, par) && globaltimer_ns() - t0 < kWaitLimitNs) {
-                    }
-                }
+            __threadfence();
+        }
+        __syncwarp();
+        fence_proxy_async();
+        for (int i = 0; i < pre; ++i) {
+            issue(qtile, qk, 0, 2, n0 + i);
+            if (++qk == nk2) {
+                qk = 0;
+                qt += kWarps;
+                if (qt < hi2)
+                    qtile = tile2(qt);
             }
         }
-    } else {
-        // ------------------------------------------------------------ consumers
-        const int g = lane >> 2, tig = lane & 3;
-        const int colbase = warp * KW;           // this warp's hidden columns / output columns
-        float zacc[2 * MT2][4];
-#pragma unroll
-        for (int i = 0; i < 2 * MT2; ++i)
-            zacc[i][0] = zacc[i][1] = zacc[i][2] = zacc[i][3] = 0.0f;
-        const uint32_t xs_s = smem_u32(xs);
-        float *my_part = s_part + warp * (2 * 8 * 8);
-        int cur_vr = -1, cur_ntok = 0;
+    }
 
-        auto flush = [&](int vr, int n_tok) {
-            const long long prow = ((long long)p.group * gridDim.x + blockIdx.x + vr) * kTokPerVr;
-            const int t0 = tig * 2;
-#pragma unroll
-            for (int mt = 0; mt < 2 * MT2; ++mt) {
-                const int r = colbase + mt * 16 + g;
-                if (t0 < n_tok) {
-                    p.part[(prow + t0) * d + r] = zacc[mt][0];
-                    p.part[(prow + t0) * d + r + 8] = zacc[mt][2];
+    // =========================================================== phase 2: z = W_d h, then the combine
+    {
+        int ct = lo2, ck = 0;
+        Tile ctile{};
+        if (ct < hi2)
+            ctile = tile2(ct);
+        float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
+        const int n_pairs = p.T * p.k;
+        while (ct < hi2) {
+            compute(n_consumed++, ctile.n_tok, c0, c1);
+            if (pt < hi2) {
+                issue(ptile, pk, wbytes2(pk), 3, n_issued++);
+                if (++pk == nk2) {
+                    pk = 0;
+                    pt += kWarps;
+                    if (pt < hi2)
+                        ptile = tile2(pt);
                 }
-                if (t0 + 1 < n_tok) {
-                    p.part[(prow + t0 + 1) * d + r] = zacc[mt][1];
-                    p.part[(prow + t0 + 1) * d + r + 8] = zacc[mt][3];
-                }
-                zacc[mt][0] = zacc[mt][1] = zacc[mt][2] = zacc[mt][3] = 0.0f;
             }
-        };
-
-        for (long long u = u0; u < u1; ++u) {
-            const int vr = vr_begin + (int)(u / upe);
-            if (vr != cur_vr) {
-                if (cur_vr >= 0)
-                    flush(cur_vr, cur_ntok);
-                const VrRec v = p.vrs[vr];
-                // hidden rows of this virtual request's tokens -> shared memory (zero padded to 8)
-                for (int t = 0; t < kTokPerVr; ++t) {
-                    const int tok = t < v.n_tok ? p.tok_of_sorted[v.tok_off + t] : -1;
-                    const uint4 *src = reinterpret_cast<const uint4 *>(p.x + (size_t)(tok < 0 ? 0 : tok) * d);
-                    uint4 *dst = reinterpret_cast<uint4 *>(xs + t * P);
-                    for (int i = tid; i < d / 8; i += kConsumerWarps * 32)
-                        dst[i] = tok >= 0 ? src[i] : make_uint4(0, 0, 0, 0);
-                }
-                cur_vr = vr;
-                cur_ntok = v.n_tok;
-                consumer_bar();
-            }
-            const long long nb = (u - u0) * epu;
-
-            // ---- phase 1: two blocks of 8 [W_g;W_u] rows
+            if (++ck == nk2) {
+                const VrRec v = p.vrs[ctile.vr];
+                const int r = ctile.blk * 16 + g;
 #pragma unroll
-            for (int blk = 0; blk < 2; ++blk) {
-                for (int e = 0; e < half; ++e) {
-                    const long long n = nb + blk * half + e;
-                    mbar_wait(full0 + 8 * (int)(n % ns), (uint32_t)((n / ns) & 1), s_abort);
+                for (int h = 0; h < 2; ++h) {
+                    const int ts = tig * 2 + h;
+                    if (ts < ctile.n_tok) {
+                        const int pos = v.tok_off + ts;
+                        const int pair = pos < n_pairs ? p.perm[pos] : pos;
+                        float *zr = p.zbuf + (size_t)pair * d + r;
+                        zr[0] = c0[h] + c1[h];
+                        zr[8] = c0[2 + h] + c1[2 + h];
+                    }
                 }
-                // lane's row for ldmatrix: unit-local row blk*8 + (lane & 7); k offset (lane >> 3) * 8
-                const int li = blk * 8 + (lane & 7);
-                const long long ne = nb + li / rpe;
-                const uint32_t rowaddr = ring_s + (int)(ne % ns) * entry_bytes + (li % rpe) * P
-                                         + (colbase + (lane >> 3) * 8) * 2;
-                const uint32_t xaddr = xs_s + g * P + (colbase + tig * 2) * 2;
-                float c[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
-                for (int ks = 0; ks < KS2; ++ks) {
-                    uint32_t b00, b01, b10, b11;
-                    ldmatrix_x4(rowaddr + ks * 64, b00, b01, b10, b11);
-                    uint32_t a0, a2, a0n, a2n;
-                    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(a0) : "r"(xaddr + ks * 64));
-                    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(a2) : "r"(xaddr + ks * 64 + 16));
-                    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(a0n) : "r"(xaddr + ks * 64 + 32));
-                    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(a2n) : "r"(xaddr + ks * 64 + 48));
-                    mma_k16_top(c, a0, a2, b00, b01);
-                    mma_k16_top(c, a0n, a2n, b10, b11);
+                for (int i = 0; i < 4; ++i)
+                    c0[i] = c1[i] = 0.f;
+                if (final_group) {
+                    // count the finished tiles of this 16-row block; the last one combines it
+                    unsigned old = 0;
+                    __threadfence();
+                    __syncwarp();
+                    if (lane == 0)
+                        old = atomicAdd(p.row_done + ctile.blk, 1u);
+                    old = __shfl_sync(0xffffffffu, old, 0);
+                    if (old == (unsigned)nv - 1u) {
+                        __threadfence();
+                        const int row = ctile.blk * 16 + (lane & 15);
+                        for (int t = lane >> 4; t < p.T; t += 2) {
+                            float y = 0.f;
+                            for (int j = 0; j < p.k; ++j)
+                                y = fmaf(p.gate[t * p.k + j], __ldcg(p.zbuf + (size_t)(t * p.k + j) * d + row), y);
+                            for (int s = 0; s < p.n_shared; ++s)
+                                y += __ldcg(p.zbuf + (size_t)(n_pairs + s * p.T + t) * d + row);
+                            p.out[(size_t)t * d + row] = bf16_rne(y);
+                        }
+                        if (lane == 0)
+                            p.row_done[ctile.blk] = 0;
+                    }
                 }
-                __syncwarp();
-                if (lane == 0)
-                    for (int e = 0; e < half; ++e)
-                        mbar_arrive(empty0 + 8 * (int)((nb + blk * half + e) % ns));
-                // c[0], c[1]: token g, rows tig*2 and tig*2+1 of this block (g_f and u_f, f = tig)
-                *reinterpret_cast<float2 *>(my_part + (blk * 8 + g) * 8 + tig * 2) = make_float2(c[0], c[1]);
-            }
-            consumer_bar();
-            if (tid < 64) {
-                const int t = tid >> 3, f = tid & 7, blk = f >> 2, fl = f & 3;
-                float gs = 0.0f, us = 0.0f;
-#pragma unroll
-                for (int w = 0; w < kConsumerWarps; ++w) {
-                    const float2 v = *reinterpret_cast<const float2 *>(s_part + w * 128 + (blk * 8 + t) * 8 + fl * 2);
-                    gs += v.x;
-                    us += v.y;
-                }
-                const float h = gs / (1.0f + __expf(-gs)) * us;
-                reinterpret_cast<uint16_t *>(s_h32)[t * 8 + f] = (uint16_t)f32_to_bf16_rne_bits(h);
-            }
-            consumer_bar();
-
-            // ---- phase 2: 8 rows of W_d^T
-            for (int e = 0; e < half; ++e) {
-                const long long n = nb + gue + e;
-                mbar_wait(full0 + 8 * (int)(n % ns), (uint32_t)((n / ns) & 1), s_abort);
-            }
-            {
-                const int li = lane & 7;                       // W_d^T row of the unit
-                const long long ne = nb + gue + li / rpe;
-                const uint32_t rowaddr = ring_s + (int)(ne % ns) * entry_bytes + (li % rpe) * P
-                                         + (colbase + (lane >> 3) * 8) * 2;
-                const uint32_t b0 = s_h32[g * 4 + tig];        // h[f = tig*2, tig*2+1][token g]
-#pragma unroll
-                for (int mt = 0; mt < MT2; ++mt) {
-                    uint32_t a00, a01, a10, a11;
-                    ldmatrix_x4_trans(rowaddr + mt * 64, a00, a01, a10, a11);
-                    mma_k8(zacc[2 * mt], a00, a01, b0);
-                    mma_k8(zacc[2 * mt + 1], a10, a11, b0);
-                }
-                __syncwarp();
-                if (lane == 0)
-                    for (int e = 0; e < half; ++e)
-                        mbar_arrive(empty0 + 8 * (int)((nb + gue + e) % ns));
+                ck = 0;
+                ct += kWarps;
+                if (ct < hi2)
+                    ctile = tile2(ct);
             }
         }
-        if (cur_vr >= 0)
-            flush(cur_vr, cur_ntok);
-        if (*s_abort && tid == 0)
-            atomicExch(p.err, MELINOE_ERR_TIMEOUT);
+    }
+    if (final_group && nv <= 0) {
+        // nothing computed in the last group (cannot happen for a well-formed plan): combine all rows
+        const int n_pairs = p.T * p.k;
+        for (int blk = blockIdx.x * kWarps + warp; blk < upe2; blk += G * kWarps) {
+            const int row = blk * 16 + (lane & 15);
+            for (int t = lane >> 4; t < p.T; t += 2) {
+                float y = 0.f;
+                for (int j = 0; j < p.k; ++j)
+                    y = fmaf(p.gate[t * p.k + j], __ldcg(p.zbuf + (size_t)(t * p.k + j) * d + row), y);
+                for (int s = 0; s < p.n_shared; ++s)
+                    y += __ldcg(p.zbuf + (size_t)(n_pairs + s * p.T + t) * d + row);
+                p.out[(size_t)t * d + row] = bf16_rne(y);
+            }
+        }
+    }
+    __syncwarp();
+    if (*abort_flag && lane == 0) {
+        // a wait ran out: give the copies this warp still has in flight a bounded time to land
+        // before its shared memory goes away, then report
+        const unsigned long long t0 = globaltimer_ns();
+        const uint32_t first = n_issued > (uint32_t)S ? n_issued - S : 0u;
+        for (uint32_t n = first; n < n_issued; ++n)
+            while (!mbar_try(bar_s + 8 * (n % S), (n / S) & 1u) && globaltimer_ns() - t0 < kWaitLimitNs) {
+            }
+        atomicExch(p.err, MELINOE_ERR_TIMEOUT);
     }
 }
 
-template <int KW>
-cudaError_t launch_kw(cudaStream_t stream, const FfnLaunchCfg &cfg, const FfnParams &p)
-{
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(ffn_stream_kernel<KW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)cfg.smem_bytes);
-        if (e != cudaSuccess)
-            return e;
-        attr_set = true;
-    }
-    ffn_stream_kernel<KW><<<cfg.grid, kFfnThreads, cfg.smem_bytes, stream>>>(p, cfg.rows_per_entry, cfg.n_stages);
-    count_launch();
-    return cudaGetLastError();
-}
+constexpr int kKC = 128;
+constexpr int kS = 4;
 
 }  // namespace
 
-bool ffn_stream_supported(int d)
+cudaError_t ffn_stream_configure(int n_sms, size_t max_smem, FfnLaunchCfg *cfg)
 {
-    switch (d) {
-    case 256: case 512: case 1024: case 2048: case 3072: case 4096:
-        return true;
-    default:
-        return false;
-    }
-}
-
-cudaError_t ffn_stream_configure(int d, int n_sms, size_t max_smem, FfnLaunchCfg *cfg)
-{
-    if (!ffn_stream_supported(d))
-        return cudaErrorInvalidValue;
-    const size_t P = 2 * (size_t)d + 16;
-    const size_t fixed = 8 * P + kConsumerWarps * 2 * 8 * 8 * sizeof(float) + 128 + 2 * kMaxStages * 8 + 16;
-    int best_rpe = 1, best_ns = 0;
-    for (int rpe = 8; rpe >= 1; rpe >>= 1) {
-        if (max_smem <= fixed)
-            break;
-        int ns = (int)((max_smem - fixed) / (rpe * P));
-        if (ns > kMaxStages)
-            ns = kMaxStages;
-        best_rpe = rpe;
-        best_ns = ns;
-        if (ns >= 6)
-            break;
-    }
-    // a unit holds at most 8 rows at a time; the ring must cover that plus copies in flight
-    if (best_ns * best_rpe < 16)
+    const size_t need = (size_t)kWarps * kS * kStageRows * (2 * kKC + 16) + (size_t)kWarps * kS * 8 + 64;
+    if (need > max_smem)
         return cudaErrorInvalidConfiguration;
-    cfg->grid = n_sms;
-    cfg->rows_per_entry = best_rpe;
-    cfg->n_stages = best_ns;
-    cfg->smem_bytes = fixed + (size_t)best_ns * best_rpe * P;
+    cudaError_t e = cudaFuncSetAttribute(ffn_stream_kernel<kKC, kS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)need);
+    if (e != cudaSuccess)
+        return e;
+    int per_sm = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ffn_stream_kernel<kKC, kS>, kThreads, need);
+    if (e != cudaSuccess)
+        return e;
+    if (per_sm < 1)
+        return cudaErrorInvalidConfiguration;
+    cfg->grid = n_sms;          // one CTA per SM: all of them resident, which the grid barrier needs
+    cfg->smem_bytes = need;
     return cudaSuccess;
 }
 
 cudaError_t launch_ffn_stream(cudaStream_t stream, const FfnLaunchCfg &cfg, const FfnParams &p)
 {
-    switch (p.d) {
-    case 256: return launch_kw<32>(stream, cfg, p);
-    case 512: return launch_kw<64>(stream, cfg, p);
-    case 1024: return launch_kw<128>(stream, cfg, p);
-    case 2048: return launch_kw<256>(stream, cfg, p);
-    case 3072: return launch_kw<384>(stream, cfg, p);
-    case 4096: return launch_kw<512>(stream, cfg, p);
-    default: return cudaErrorInvalidValue;
-    }
+    FfnParams q = p;
+    void *args[] = {&q};
+    cudaError_t e = cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(ffn_stream_kernel<kKC, kS>),
+                                                dim3(cfg.grid), dim3(kThreads), args, cfg.smem_bytes, stream);
+    count_launch();
+    return e;
 }
 
 }  // namespace melinoe

@@ -24,6 +24,7 @@ struct PlanParams {
     VrRec *vrs;
     int32_t *perm, *inv_pos, *tok_of_sorted;
     HostPlan *hplan;          // page-locked host memory (device-visible address)
+    unsigned *sync;           // grid-barrier counters of the FFN launches, zeroed here
     uint32_t gmax;            // compute groups the caller has room for
     uint32_t call_seq;        // written to the miss queue's seq word when the record is complete
     melinoe_moe_stats *stats; // may be null
@@ -32,7 +33,7 @@ struct PlanParams {
 };
 cudaError_t launch_plan(cudaStream_t stream, const PlanParams &p);
 
-// ---- streaming expert FFN (Eq. 3) for calls with few tokens per expert
+// ---- streaming expert FFN (Eq. 3) with the gate-weighted combine (Eq. 2) fused in
 struct FfnParams {
     const char *slots;               // device cache: slot s at slots + s * slot_stride
     size_t slot_stride;
@@ -40,30 +41,23 @@ struct FfnParams {
     const DevPlan *plan;
     const VrRec *vrs;
     const int32_t *tok_of_sorted;
+    const int32_t *perm;             // sorted position -> flat pair index t * k + j
     const uint16_t *x;               // hidden [T][d] bf16
-    float *part;                     // partial outputs, rows of d floats
+    const float *gate;               // [T][k]
+    uint16_t *hbuf;                  // h = SiLU(g) * u: [virtual request][8 token slots][Fpad] bf16
+    float *zbuf;                     // expert outputs: [T*k routed pairs, then n_shared*T][d] fp32
+    uint16_t *out;                   // [T][d] bf16
+    unsigned *sync;                  // grid-barrier counters, one per compute group (zero at launch)
+    unsigned *row_done;              // per 16-row block: finished tiles of the last group (self-resetting)
     int *err;                        // device error word (0 = ok)
-    int d, F, E;
+    int d, F, Fpad, E, k, T, n_shared;
     int group;
 };
 struct FfnLaunchCfg {
-    int grid, rows_per_entry, n_stages;
+    int grid;
     size_t smem_bytes;
 };
-bool ffn_stream_supported(int d);
-cudaError_t ffn_stream_configure(int d, int n_sms, size_t max_smem, FfnLaunchCfg *cfg);
+cudaError_t ffn_stream_configure(int n_sms, size_t max_smem, FfnLaunchCfg *cfg);
 cudaError_t launch_ffn_stream(cudaStream_t stream, const FfnLaunchCfg &cfg, const FfnParams &p);
-
-// ---- gate-weighted combine (Eq. 2) over the streaming kernel's partial outputs
-struct CombineParams {
-    const DevPlan *plan;
-    const int32_t *idx;
-    const float *gate;
-    const int32_t *inv_pos;
-    const float *part;
-    uint16_t *out;                   // [T][d] bf16
-    int T, d, k, E, n_shared, grid, units_per_vr;
-};
-cudaError_t launch_combine(cudaStream_t stream, const CombineParams &p);
 
 }  // namespace melinoe

@@ -12,7 +12,7 @@ constexpr int kMaxShared = 8;            // always-resident shared experts
 constexpr int kMaxReq = kMaxExperts + kMaxShared;
 constexpr int kMaxGroups = kMaxExperts + 2;  // 1 + ceil(E / C) with C >= 1
 constexpr int kTokPerVr = 8;             // tokens per virtual request of the streaming FFN kernel
-constexpr int kUnitRows = 8;             // d_ff rows per work unit of the streaming FFN kernel
+constexpr int kUnitRows = 8;             // d_ff must be a multiple of this (one phase-1 tile of the FFN kernel)
 
 // Persistent cache state of one layer (device memory).  The reading of "LRU" used here:
 // every request takes stamp = ++counter; a hit re-stamps its slot; a miss takes the lowest
@@ -68,18 +68,5 @@ struct HostPlan {
     HostMiss miss[kMaxExperts];
     uint32_t seq;
 };
-
-// Geometry shared by the streaming FFN kernel and the combine kernel.
-struct FfnGeom {
-    int d, F, k, E, n_shared;
-    int grid;              // CTAs of every streaming FFN launch
-    int units_per_vr;      // F / kUnitRows
-};
-
-// CTA that owns work unit u when nu units are split over g CTAs as [floor(i*nu/g), floor((i+1)*nu/g)).
-__host__ __device__ inline int cta_of_unit(long long u, long long nu, long long g)
-{
-    return (int)(((u + 1) * g - 1) / nu);
-}
 
 }  // namespace melinoe

@@ -115,6 +115,8 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p)
     }
     for (int i = tid; i < p.n_shared * p.T; i += kPlanThreads)
         p.tok_of_sorted[n_pairs + i] = i % p.T;
+    for (int i = tid; i <= kMaxGroups; i += kPlanThreads)
+        p.sync[i] = 0u;
 
     // ---- (b), (c): cache requests, by warp 0 (slots spread over lanes)
     if (warp == 0) {

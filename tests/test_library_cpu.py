@@ -41,10 +41,9 @@ def test_pack_expert_layout(m):
     wg, wu, wd = gen.expert_weights(1, 0, 0, d, F)
     blob = np.zeros(3 * d * F, np.uint16)
     m.melinoe_moe_pack_expert(d, F, wg.ctypes.data, wu.ctypes.data, wd.ctypes.data, blob.ctypes.data)
-    gu = blob[: 2 * F * d].reshape(2 * F, d)
-    dt = blob[2 * F * d:].reshape(F, d)
-    assert np.array_equal(gu[0::2], wg) and np.array_equal(gu[1::2], wu)
-    assert np.array_equal(dt, wd.T)
+    n = d * F
+    assert np.array_equal(blob[:n].reshape(F, d), wg) and np.array_equal(blob[n:2 * n].reshape(F, d), wu)
+    assert np.array_equal(blob[2 * n:].reshape(d, F), wd)
     with pytest.raises(m.MelinoeError):
         m.melinoe_moe_pack_expert(d, F, 0, wu.ctypes.data, wd.ctypes.data, blob.ctypes.data)
 
