@@ -77,7 +77,7 @@ struct melinoe_moe {
     int32_t *idx = nullptr, *perm = nullptr, *inv_pos = nullptr, *tok_of_sorted = nullptr;
     float *gate = nullptr, *logits = nullptr, *zbuf = nullptr;
     uint16_t *hbuf = nullptr;
-    unsigned *sync = nullptr, *row_done = nullptr;
+    unsigned *sync = nullptr;
     VrRec *vrs = nullptr;
     uint16_t *stage_in = nullptr, *stage_out = nullptr;
     melinoe_moe_stats *stage_stats = nullptr;
@@ -317,9 +317,7 @@ int melinoe_moe_create(int d, int F, int E, int k, int C, melinoe_moe_t **out)
     CR(cudaMalloc(&h->plan, sizeof(DevPlan)));
     CR(cudaMalloc(&h->err_word, 256));
     CR(cudaMalloc(&h->sync, sizeof(unsigned) * (kMaxGroups + 1)));
-    CR(cudaMalloc(&h->row_done, sizeof(unsigned) * (d / 16)));
     CR(cudaMemset(h->sync, 0, sizeof(unsigned) * (kMaxGroups + 1)));
-    CR(cudaMemset(h->row_done, 0, sizeof(unsigned) * (d / 16)));
     CR(cudaMalloc(&h->shared_dev, sizeof(char *) * kMaxShared));
     CR(cudaMalloc(&h->stage_stats, sizeof(melinoe_moe_stats)));
     CR(cudaMemset(h->err_word, 0, 256));
@@ -353,7 +351,6 @@ int melinoe_moe_destroy(melinoe_moe_t *h)
     cudaFree(h->plan);
     cudaFree(h->err_word);
     cudaFree(h->sync);
-    cudaFree(h->row_done);
     cudaFree(h->shared_dev);
     cudaFree(h->stage_stats);
     if (h->hplan)
@@ -516,7 +513,6 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
     fp.zbuf = h->zbuf;
     fp.out = static_cast<uint16_t *>(out_dev);
     fp.sync = h->sync;
-    fp.row_done = h->row_done;
     fp.err = h->err_word;
     fp.d = h->d;
     fp.F = h->F;
@@ -525,6 +521,9 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
     fp.k = h->k;
     fp.T = T;
     fp.n_shared = h->n_shared;
+    FfnGeometry geo;
+    if (ffn_stream_geometry(h->cfg, h->d, h->F, T, &geo) != cudaSuccess)
+        return MELINOE_ERR_UNSUPPORTED;
     auto launch_group = [&](int g) -> int {
         TimedPair tp{nullptr, nullptr};
         if (h->timing) {
@@ -538,7 +537,7 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
             CU_TRY(cudaEventRecord(tp.a, s));
         }
         fp.group = g;
-        CU_TRY(launch_ffn_stream(s, h->cfg, fp));
+        CU_TRY(launch_ffn_stream(s, h->cfg, geo, fp));
         if (h->timing) {
             CU_TRY(cudaEventRecord(tp.b, s));
             h->timed.push_back(tp);
@@ -647,7 +646,6 @@ int melinoe_moe_reset_cache(melinoe_moe_t *h)
     init_cache_host(c0);
     CU_TRY(cudaMemcpy(h->cache, &c0, sizeof c0, cudaMemcpyHostToDevice));
     CU_TRY(cudaMemset(h->err_word, 0, 4));
-    CU_TRY(cudaMemset(h->row_done, 0, sizeof(unsigned) * (h->d / 16)));
     h->sticky.store(MELINOE_OK);
     return MELINOE_OK;
 }

@@ -1,46 +1,52 @@
 // Streaming SwiGLU expert FFN (Eq. 3) with the gate-weighted combine (Eq. 2) fused in, for
 // calls with few tokens per expert (decode).  The work is reading every needed expert once
-// from HBM, so the kernel is built around keeping the memory system full.
+// from HBM, so the kernel is built around keeping the memory system full: measured on B200,
+// bulk copies of whole 4 KB rows stream at the full HBM rate while 256-byte pieces reach
+// little more than half of it, so the unit of transfer is a whole row (or a 4 KB piece of a
+// longer one).
 //
-// One cooperative launch per compute group, one CTA per SM, eight independent warps per CTA.
-// A "virtual request" is one expert with up to 8 of its tokens.
+// One cooperative launch per compute group, one CTA per SM: one producer warp and eight
+// consumer warps.  A "virtual request" is one expert with up to 8 of its tokens.
 //
 //   phase 1  tile = 8 rows of W_g plus the same 8 rows of W_u of one virtual request.
 //            D[16 x 8] = [W_g rows; W_u rows] (16 x d) * x^T (d x 8 tokens) on mma.sync
-//            (bf16 in, fp32 accumulate).  In the accumulator layout a thread holds g_f and u_f
-//            of the same f and the same two tokens, so h = SiLU(g) * u is thread-local;
-//            h goes to global memory as bf16.
-//   barrier  grid-wide (bounded spin on a device counter); before waiting, each warp already
-//            has the first W_d stages of its phase-2 work in flight.
-//   phase 2  tile = 16 rows of W_d of one virtual request: D[16 x 8] = W_d rows (16 x F) * h^T.
-//            Every tile is a complete dot product over d_ff, so z needs no cross-CTA reduction
-//            and goes to z[pair][d] in fp32.
-//   combine  the warp that finishes the last tile of a 16-row block in the call's last
-//            compute group sums gate * z over the ranks in rank order (plus shared experts)
-//            and writes the bf16 output rows.  The result does not depend on which warp does
-//            it, nor on how the experts were split over groups.
+//            (bf16 in, fp32 accumulate); the eight warps split the columns of a stage and
+//            their partial sums meet in shared memory once per tile.  In the accumulator
+//            layout a thread holds g_f and u_f of the same f and the same two tokens, so
+//            h = SiLU(g) * u is thread-local; h goes to global memory as bf16.
+//   barrier  grid-wide, crossed by the producer warps only (bounded spin on a device counter):
+//            the consumers never wait for it, and the first W_d stages of phase 2 are already
+//            in flight when the producer reaches it.
+//   phase 2  every CTA owns a contiguous range of the d_model output rows (d/G of them, so the
+//            split is even to within one row) for ALL virtual requests of the launch.  Tile =
+//            up to 16 of those W_d rows of one virtual request: D[16 x 8] = W_d rows * h^T, a
+//            complete dot product over d_ff, so z needs no cross-CTA reduction; it goes to
+//            z[pair][d] in fp32.
+//   combine  in the call's last compute group every CTA, having finished its rows, sums
+//            gate * z over the ranks in rank order (plus shared experts) for those rows and
+//            writes them as bf16: it reads only what itself (or an earlier launch) wrote, so
+//            no device-wide synchronisation is involved.  The result does not depend on how the
+//            experts were split over groups.
 //
-// Data movement: every warp owns a private ring of S stages in shared memory.  A stage holds
-// a KC-column slice of the tile's 16 weight rows plus the matching slice of up to 8 operand rows
-// (hidden rows in phase 1, h rows in phase 2), each fetched by its own cp.async.bulk (one lane
-// per row) completing on the stage's mbarrier.  Rows sit at a pitch of 2*KC+16 bytes, which
-// makes the ldmatrix reads and the operand-fragment reads bank-conflict free.  There is no
-// CTA-wide synchronisation after start-up.
+// A stage of the shared-memory ring holds one piece (at most 4 KB) of each of the tile's 16
+// weight rows plus the matching piece of up to 8 operand rows (hidden rows in phase 1, h rows
+// in phase 2), each fetched by its own cp.async.bulk (one producer lane per row) completing on
+// the stage's mbarrier.  Rows sit at a pitch of 16 bytes more than a multiple of 128, which
+// makes the ldmatrix reads and the operand-fragment reads bank-conflict free.
 //
 // Every wait is bounded: when an mbarrier or the grid barrier does not complete in time the
 // warp raises the CTA's abort flag, later waits fall through, the kernel ends normally and the
 // error word tells the host.
-#include <cooperative_groups.h>
-
 #include "kernels.cuh"
 
 namespace melinoe {
 
 namespace {
 
-constexpr int kWarps = 8;
-constexpr int kThreads = kWarps * 32;
-constexpr int kStageRows = 24;            // 16 weight rows + 8 operand rows
+constexpr int kConsumerWarps = 8;
+constexpr int kThreads = (kConsumerWarps + 1) * 32;
+constexpr int kMaxStages = 8;
+constexpr int kMaxChunk = 4096;                      // bytes of one row piece
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p)
@@ -89,6 +95,21 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
 }
 
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void mbar_expect(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+
+__device__ __forceinline__ void consumer_bar()
+{
+    asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory");
+}
+
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3)
 {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
@@ -131,34 +152,24 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t
                  : "memory");
 }
 
-__device__ __forceinline__ void mbar_expect(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-
-// What a warp needs to know about the tile it fetches or computes.
+// What the producer needs to know about a tile.
 struct Tile {
-    const char *src;     // this lane's source row (weights: lanes 0..15, operand rows: lanes 16..23)
+    const char *src;     // this lane's source row (weights: lanes 0..15, operand rows: 16..23)
     int n_tok;           // tokens of the virtual request
-    int vr;              // virtual request (index within the call)
-    int blk;             // f-block (phase 1) or 16-row block (phase 2)
+    int n_rows;          // weight rows in the tile (16 except at the end of a CTA's row range)
 };
 
-template <int KC, int S>
-__global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p)
+__global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, FfnGeometry geo)
 {
-    constexpr int PITCH = 2 * KC + 16;
-    constexpr int STAGE = kStageRows * PITCH;
-    constexpr int KSTEPS = KC / 16;
-
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ int s_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int g = lane >> 2, tig = lane & 3;
     const int d = p.d, F = p.F, Fpad = p.Fpad;
     const DevPlan *plan = p.plan;
     const int G = (int)gridDim.x;
+    const int S = geo.n_stages, PITCH = geo.pitch, CB = geo.chunk_bytes;
+    const int STAGE = (16 + geo.n_op_rows) * PITCH;
 
     if (plan->status != MELINOE_OK) {
         // the call was refused on the device: the output is all zeros, the status tells why
@@ -173,190 +184,148 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p)
     if (nv <= 0 && !final_group)
         return;
 
-    unsigned char *ring = smem + (size_t)warp * S * STAGE;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + (size_t)kWarps * S * STAGE) + warp * S;
-    const uint32_t ring_s = smem_u32(ring), bar_s = smem_u32(bars);
+    unsigned char *ring = smem;
+    float *red = reinterpret_cast<float *>(smem + (size_t)S * STAGE);          // [2][8 warps][4][32]
+    uint64_t *bars = reinterpret_cast<uint64_t *>(red + 2 * kConsumerWarps * 128);
+    const uint32_t ring_s = smem_u32(ring);
+    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + kMaxStages);
     volatile int *abort_flag = &s_abort;
 
-    if (tid == 0)
+    if (tid == 0) {
         s_abort = 0;
-    if (lane == 0) {
-        for (int i = 0; i < S; ++i)
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar_s + 8 * i), "r"(1));
+        for (int i = 0; i < S; ++i) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(full0 + 8 * i), "r"(1));
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(empty0 + 8 * i), "r"(kConsumerWarps));
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (F % KC != 0) {
-        // the last d_ff slice of a W_d row is shorter than a stage row: what it leaves untouched
-        // must be finite, because it meets zeros of the padded h rows in the product
+    if (F % 16 != 0) {
+        // the last 16-column step of a W_d row is half filled: what the copy leaves untouched
+        // must be finite, because it meets the zero padding of the h rows in the product
         uint4 *z = reinterpret_cast<uint4 *>(ring);
-        for (int i = lane; i < S * STAGE / 16; i += 32)
+        for (int i = tid; i < S * STAGE / 16; i += kThreads)
             z[i] = make_uint4(0, 0, 0, 0);
         fence_proxy_async();
     }
     __syncthreads();
 
-    // ---- this warp's tiles: a contiguous range per CTA, dealt round-robin to its warps
-    const int upe1 = F / 8, upe2 = d / 16;
-    const int nk1 = d / KC, nk2 = (F + KC - 1) / KC;
-    const long long NT1 = (long long)nv * upe1, NT2 = (long long)nv * upe2;
-    const int lo1 = (int)(blockIdx.x * NT1 / G) + warp, hi1 = (int)((blockIdx.x + 1) * NT1 / G);
-    const int lo2 = (int)(blockIdx.x * NT2 / G) + warp, hi2 = (int)((blockIdx.x + 1) * NT2 / G);
+    // ---- phase 1: a contiguous range of (virtual request, 8-row f-block) tiles per CTA
+    const int upe1 = F / 8;
+    const int rb1 = 2 * d, rb2 = 2 * F;                       // row bytes
+    const int nk1 = (rb1 + CB - 1) / CB, nk2 = (rb2 + CB - 1) / CB;
+    const long long NT1 = (long long)nv * upe1;
+    const int lo1 = (int)(blockIdx.x * NT1 / G), hi1 = (int)((blockIdx.x + 1) * NT1 / G);
+    // ---- phase 2: output rows [r_lo, r_hi) of every virtual request, in tiles of up to 16 rows
+    const int r_lo = (int)((long long)blockIdx.x * d / G), r_hi = (int)((long long)(blockIdx.x + 1) * d / G);
+    const int mt = (r_hi - r_lo + 15) / 16;
+    const int hi2 = nv * mt;
 
-    auto blob_of = [&](const VrRec &v) -> const char * {
-        const ReqRec rec = plan->req[v.req];
-        return rec.slot >= 0 ? p.slots + (size_t)rec.slot * p.slot_stride : p.shared_blobs[rec.expert - p.E];
-    };
-    // lane's source row for a phase-1 tile: lanes 0..7 W_g rows, 8..15 W_u rows, 16..23 hidden rows
-    auto tile1 = [&](int t) -> Tile {
-        Tile ti;
-        ti.vr = vb + t / upe1;
-        ti.blk = t % upe1;
-        const VrRec v = p.vrs[ti.vr];
-        ti.n_tok = v.n_tok;
-        ti.src = nullptr;
-        if (lane < 16) {
-            const int row = (lane < 8 ? 0 : F) + ti.blk * 8 + (lane & 7);
-            ti.src = blob_of(v) + (size_t)row * d * 2;
-        } else if (lane - 16 < v.n_tok) {
-            const int tok = p.tok_of_sorted[v.tok_off + lane - 16];
-            ti.src = reinterpret_cast<const char *>(p.x) + (size_t)tok * d * 2;
-        }
-        return ti;
-    };
-    // phase 2: lanes 0..15 W_d rows, 16..23 rows of h
-    auto tile2 = [&](int t) -> Tile {
-        Tile ti;
-        ti.vr = vb + t / upe2;
-        ti.blk = t % upe2;
-        const VrRec v = p.vrs[ti.vr];
-        ti.n_tok = v.n_tok;
-        ti.src = nullptr;
-        if (lane < 16)
-            ti.src = blob_of(v) + ((size_t)2 * F * d + (size_t)(ti.blk * 16 + lane) * F) * 2;
-        else if (lane - 16 < v.n_tok)
-            ti.src = reinterpret_cast<const char *>(p.hbuf) + ((size_t)ti.vr * kTokPerVr + lane - 16) * Fpad * 2;
-        return ti;
-    };
-
-    uint32_t n_issued = 0, n_consumed = 0;   // stages, over both phases (ring slot and parity)
-
-    // issue one stage: parts bit 0 = weight rows and the barrier's byte count, bit 1 = operand rows
-    auto issue = [&](const Tile &ti, int kc, int wbytes, int parts, uint32_t n) {
-        const uint32_t slot = n % S;
-        const uint32_t bar = bar_s + 8 * slot;
-        if ((parts & 1) && lane == 0)
-            mbar_expect(bar, 16u * wbytes + (uint32_t)ti.n_tok * KC * 2);
-        __syncwarp();
-        if (ti.src) {
-            const bool is_w = lane < 16;
-            if (is_w ? (parts & 1) : (parts & 2))
-                bulk_g2s(ring_s + slot * STAGE + lane * PITCH, ti.src + (size_t)kc * KC * 2,
-                         is_w ? (uint32_t)wbytes : (uint32_t)(KC * 2), bar);
-        }
-    };
-
-    // the mma loop over one stage
-    const uint32_t a_off = ((lane & 7) + ((lane >> 3) & 1) * 8) * PITCH + (lane >> 4) * 16;
-    const uint32_t b_off = (16 + g) * PITCH + tig * 4;
-    auto compute = [&](uint32_t n, int n_tok, float (&c0)[4], float (&c1)[4]) {
-        const uint32_t slot = n % S;
-        mbar_wait(bar_s + 8 * slot, (n / S) & 1u, abort_flag);
-        const uint32_t base = ring_s + slot * STAGE;
-        const bool has_tok = g < n_tok;
-#pragma unroll
-        for (int ks = 0; ks < KSTEPS; ks += 2) {
-            uint32_t a0, a1, a2, a3, e0, e1, e2, e3;
-            ldmatrix_x4(base + a_off + ks * 32, a0, a1, a2, a3);
-            ldmatrix_x4(base + a_off + ks * 32 + 32, e0, e1, e2, e3);
-            uint32_t b0 = 0, b1 = 0, f0 = 0, f1 = 0;
-            if (has_tok) {
-                b0 = lds32(base + b_off + ks * 32);
-                b1 = lds32(base + b_off + ks * 32 + 16);
-                f0 = lds32(base + b_off + ks * 32 + 32);
-                f1 = lds32(base + b_off + ks * 32 + 48);
-            }
-            mma_16816(c0, a0, a1, a2, a3, b0, b1);
-            mma_16816(c1, e0, e1, e2, e3, f0, f1);
-        }
-        __syncwarp();
-    };
-
-    // =========================================================== phase 1: h = SiLU(W_g x) * (W_u x)
-    {
-        int pt = lo1, pk = 0, ct = lo1, ck = 0;
-        Tile ptile{}, ctile{};
-        if (pt < hi1)
-            ptile = tile1(pt);
-        ctile = ptile;
-        for (int i = 0; i < S && pt < hi1; ++i) {
-            issue(ptile, pk, KC * 2, 3, n_issued++);
-            if (++pk == nk1) {
-                pk = 0;
-                pt += kWarps;
-                if (pt < hi1)
-                    ptile = tile1(pt);
-            }
-        }
-        float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
-        while (ct < hi1) {
-            compute(n_consumed++, ctile.n_tok, c0, c1);
-            if (pt < hi1) {
-                issue(ptile, pk, KC * 2, 3, n_issued++);
-                if (++pk == nk1) {
-                    pk = 0;
-                    pt += kWarps;
-                    if (pt < hi1)
-                        ptile = tile1(pt);
+    if (warp == kConsumerWarps) {
+        // =================================================================== producer
+        auto blob_of = [&](const VrRec &v) -> const char * {
+            const ReqRec rec = plan->req[v.req];
+            return rec.slot >= 0 ? p.slots + (size_t)rec.slot * p.slot_stride : p.shared_blobs[rec.expert - p.E];
+        };
+        // Per virtual request (looked up only when the tile sequence moves on to the next one):
+        // this lane's source row of block 0 and its stride from one block to the next.
+        int cur_vr = -1, cur_ntok = 0;
+        const char *lane_base = nullptr;
+        size_t lane_step = 0;
+        // phase 1: lanes 0..7 W_g rows, 8..15 W_u rows, 16..23 hidden rows of the request's tokens
+        auto tile1 = [&](int t) -> Tile {
+            const int vr = vb + t / upe1, blk = t % upe1;
+            if (vr != cur_vr) {
+                const VrRec v = p.vrs[vr];
+                cur_vr = vr;
+                cur_ntok = v.n_tok;
+                lane_base = nullptr;
+                lane_step = 0;
+                if (lane < 16) {
+                    lane_base = blob_of(v) + (size_t)((lane < 8 ? 0 : F) + (lane & 7)) * rb1;
+                    lane_step = (size_t)8 * rb1;
+                } else if (lane - 16 < v.n_tok) {
+                    const int tok = p.tok_of_sorted[v.tok_off + lane - 16];
+                    lane_base = reinterpret_cast<const char *>(p.x) + (size_t)tok * rb1;
                 }
             }
-            if (++ck == nk1) {
-                // rows g and g + 8 of the tile are g_f and u_f for f = 8 * blk + g
-                const int f = ctile.blk * 8 + g;
-                const float gv0 = c0[0] + c1[0], gv1 = c0[1] + c1[1], uv0 = c0[2] + c1[2], uv1 = c0[3] + c1[3];
-                uint16_t *hrow = p.hbuf + ((size_t)ctile.vr * kTokPerVr) * Fpad + f;
-                if (tig * 2 < ctile.n_tok)
-                    hrow[(size_t)(tig * 2) * Fpad] = bf16_rne(gv0 / (1.0f + __expf(-gv0)) * uv0);
-                if (tig * 2 + 1 < ctile.n_tok)
-                    hrow[(size_t)(tig * 2 + 1) * Fpad] = bf16_rne(gv1 / (1.0f + __expf(-gv1)) * uv1);
-#pragma unroll
-                for (int i = 0; i < 4; ++i)
-                    c0[i] = c1[i] = 0.f;
-                ck = 0;
-                ct += kWarps;
-                if (ct < hi1)
-                    ctile = tile1(ct);
+            Tile ti;
+            ti.n_tok = cur_ntok;
+            ti.n_rows = 16;
+            ti.src = lane_base ? lane_base + (size_t)blk * lane_step : nullptr;
+            return ti;
+        };
+        // phase 2: lanes 0..15 W_d rows, 16..23 rows of h
+        auto tile2 = [&](int t) -> Tile {
+            const int vr = vb + t / mt, blk = t % mt;
+            if (vr != cur_vr) {
+                const VrRec v = p.vrs[vr];
+                cur_vr = vr;
+                cur_ntok = v.n_tok;
+                lane_base = nullptr;
+                lane_step = 0;
+                if (lane < 16) {
+                    lane_base = blob_of(v) + (size_t)2 * F * rb1 + (size_t)(r_lo + lane) * rb2;
+                    lane_step = (size_t)16 * rb2;
+                } else if (lane - 16 < v.n_tok) {
+                    lane_base = reinterpret_cast<const char *>(p.hbuf) + ((size_t)vr * kTokPerVr + lane - 16) * Fpad * 2;
+                }
+            }
+            Tile ti;
+            ti.n_tok = cur_ntok;
+            ti.n_rows = min(16, r_hi - r_lo - 16 * blk);
+            ti.src = lane_base ? lane_base + (size_t)blk * lane_step : nullptr;
+            if (lane < 16 && lane >= ti.n_rows)
+                ti.src = nullptr;
+            return ti;
+        };
+        uint32_t n = 0;   // stages issued so far, over both phases
+        bool dead = false;
+        // parts bit 0: wait for the slot, arm the barrier, fetch the weight rows; bit 1: operand rows.
+        // wbytes: bytes of each weight-row piece; obytes: bytes of each operand-row piece.
+        auto issue = [&](const Tile &ti, int kc, int wbytes, int obytes, int parts, uint32_t nn) {
+            const uint32_t slot = nn % S;
+            const uint32_t bar = full0 + 8 * slot;
+            if (parts & 1) {
+                if (nn >= (uint32_t)S && !dead)
+                    dead = !mbar_wait(empty0 + 8 * slot, ((nn / S) - 1u) & 1u, abort_flag);
+                if (lane == 0)
+                    mbar_expect(bar, (uint32_t)ti.n_rows * wbytes + (uint32_t)ti.n_tok * obytes);
+                __syncwarp();
+            }
+            if (ti.src && !dead) {
+                const bool is_w = lane < 16;
+                if (is_w ? (parts & 1) : (parts & 2))
+                    bulk_g2s(ring_s + slot * STAGE + lane * PITCH, ti.src + (size_t)kc * CB,
+                             (uint32_t)(is_w ? wbytes : obytes), bar);
+            }
+        };
+        for (int t = lo1; t < hi1; ++t) {
+            const Tile ti = tile1(t);
+            for (int kc = 0; kc < nk1; ++kc) {
+                const int b = min(CB, rb1 - kc * CB);
+                issue(ti, kc, b, b, 3, n++);
             }
         }
-    }
-
-    // =========================================================== grid barrier, W_d already in flight
-    __threadfence();
-    fence_proxy_async();       // h was written through the generic proxy, bulk copies will read it
-    __syncwarp();
-    if (lane == 0)
-        atomicAdd(p.sync + p.group, 1u);
-    int pt = lo2, pk = 0;
-    Tile ptile{};
-    if (pt < hi2)
-        ptile = tile2(pt);
-    auto wbytes2 = [&](int kc) { return 2 * min(KC, F - kc * KC); };
-    {
-        // first stages of phase 2: weight rows only; their h rows follow once h is complete
-        int qt = pt, qk = pk;
-        Tile qtile = ptile;
-        const uint32_t n0 = n_issued;
+        // phase 2: the first stages go out with their weight rows only; h is not complete yet
+        cur_vr = -1;
+        int t2 = 0, k2 = 0;
+        Tile ti2{};
+        if (t2 < hi2)
+            ti2 = tile2(t2);
+        auto op_bytes2 = [&](int kc) { return min(CB, Fpad * 2 - kc * CB); };
+        const uint32_t n_pre0 = n;
         int pre = 0;
-        for (; pre < S && pt < hi2; ++pre) {
-            issue(ptile, pk, wbytes2(pk), 1, n_issued++);
-            if (++pk == nk2) {
-                pk = 0;
-                pt += kWarps;
-                if (pt < hi2)
-                    ptile = tile2(pt);
+        for (; pre < S && t2 < hi2; ++pre) {
+            issue(ti2, k2, min(CB, rb2 - k2 * CB), op_bytes2(k2), 1, n++);
+            if (++k2 == nk2) {
+                k2 = 0;
+                if (++t2 < hi2)
+                    ti2 = tile2(t2);
             }
         }
+        // grid barrier: every CTA's consumers have written their part of h
         if (lane == 0) {
-            const unsigned target = (unsigned)G * kWarps;
+            const unsigned target = (unsigned)G;
             volatile unsigned *w = p.sync + p.group;
             if (*w < target && !*abort_flag) {
                 const unsigned long long t0 = globaltimer_ns();
@@ -371,142 +340,244 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p)
         }
         __syncwarp();
         fence_proxy_async();
-        for (int i = 0; i < pre; ++i) {
-            issue(qtile, qk, 0, 2, n0 + i);
-            if (++qk == nk2) {
-                qk = 0;
-                qt += kWarps;
-                if (qt < hi2)
-                    qtile = tile2(qt);
+        {
+            // the operand rows of the stages already under way: replay the tile sequence from the
+            // start of phase 2 with a cache of its own, then restore the main sequence's cache
+            const int keep_vr = cur_vr, keep_ntok = cur_ntok;
+            const char *keep_base = lane_base;
+            const size_t keep_step = lane_step;
+            cur_vr = -1;
+            int qt = 0, qk = 0;
+            Tile qtile{};
+            if (pre > 0)
+                qtile = tile2(0);
+            for (int i = 0; i < pre; ++i) {
+                issue(qtile, qk, 0, op_bytes2(qk), 2, n_pre0 + i);
+                if (++qk == nk2) {
+                    qk = 0;
+                    if (++qt < hi2)
+                        qtile = tile2(qt);
+                }
+            }
+            cur_vr = keep_vr;
+            cur_ntok = keep_ntok;
+            lane_base = keep_base;
+            lane_step = keep_step;
+        }
+        while (t2 < hi2) {
+            issue(ti2, k2, min(CB, rb2 - k2 * CB), op_bytes2(k2), 3, n++);
+            if (++k2 == nk2) {
+                k2 = 0;
+                if (++t2 < hi2)
+                    ti2 = tile2(t2);
             }
         }
+        if (*abort_flag && lane == 0) {
+            // a wait ran out: give the copies still in flight a bounded time to land before this
+            // CTA's shared memory goes away
+            const unsigned long long t0 = globaltimer_ns();
+            const uint32_t first = n > (uint32_t)S ? n - S : 0u;
+            for (uint32_t m = first; m < n; ++m)
+                while (!mbar_try(full0 + 8 * (m % S), (m / S) & 1u) && globaltimer_ns() - t0 < kWaitLimitNs) {
+                }
+            atomicExch(p.err, MELINOE_ERR_TIMEOUT);
+        }
+        return;
     }
 
-    // =========================================================== phase 2: z = W_d h, then the combine
-    {
-        int ct = lo2, ck = 0;
-        Tile ctile{};
-        if (ct < hi2)
-            ctile = tile2(ct);
-        float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
-        const int n_pairs = p.T * p.k;
-        while (ct < hi2) {
-            compute(n_consumed++, ctile.n_tok, c0, c1);
-            if (pt < hi2) {
-                issue(ptile, pk, wbytes2(pk), 3, n_issued++);
-                if (++pk == nk2) {
-                    pk = 0;
-                    pt += kWarps;
-                    if (pt < hi2)
-                        ptile = tile2(pt);
-                }
+    // ======================================================================= consumers
+    const int g = lane >> 2, tig = lane & 3;
+    const uint32_t a_off = ((lane & 7) + ((lane >> 3) & 1) * 8) * PITCH + (lane >> 4) * 16;
+    const uint32_t b_off = (16 + g) * PITCH + tig * 4;
+    uint32_t n = 0;        // stages consumed so far
+    int n_tiles = 0;       // tiles finished so far (selects the reduction buffer and the epilogue warp)
+    float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
+
+    // this warp's share of one stage: some of the 16-column steps of the piece
+    auto compute = [&](int bytes, int n_tok) {
+        const uint32_t slot = n % S;
+        mbar_wait(full0 + 8 * slot, (n / S) & 1u, abort_flag);
+        const uint32_t base = ring_s + slot * STAGE;
+        const int ks_total = (bytes + 31) >> 5;
+        const int ks_lo = warp * ks_total / kConsumerWarps, ks_hi = (warp + 1) * ks_total / kConsumerWarps;
+        const bool has_tok = g < n_tok;
+        int ks = ks_lo;
+        for (; ks + 1 < ks_hi; ks += 2) {
+            uint32_t a0, a1, a2, a3, e0, e1, e2, e3;
+            ldmatrix_x4(base + a_off + ks * 32, a0, a1, a2, a3);
+            ldmatrix_x4(base + a_off + ks * 32 + 32, e0, e1, e2, e3);
+            uint32_t b0 = 0, b1 = 0, f0 = 0, f1 = 0;
+            if (has_tok) {
+                b0 = lds32(base + b_off + ks * 32);
+                b1 = lds32(base + b_off + ks * 32 + 16);
+                f0 = lds32(base + b_off + ks * 32 + 32);
+                f1 = lds32(base + b_off + ks * 32 + 48);
             }
-            if (++ck == nk2) {
-                const VrRec v = p.vrs[ctile.vr];
-                const int r = ctile.blk * 16 + g;
+            mma_16816(c0, a0, a1, a2, a3, b0, b1);
+            mma_16816(c1, e0, e1, e2, e3, f0, f1);
+        }
+        if (ks < ks_hi) {
+            uint32_t a0, a1, a2, a3;
+            ldmatrix_x4(base + a_off + ks * 32, a0, a1, a2, a3);
+            uint32_t b0 = 0, b1 = 0;
+            if (has_tok) {
+                b0 = lds32(base + b_off + ks * 32);
+                b1 = lds32(base + b_off + ks * 32 + 16);
+            }
+            mma_16816(c0, a0, a1, a2, a3, b0, b1);
+        }
+        __syncwarp();
+        if (lane == 0)
+            mbar_arrive(empty0 + 8 * slot);
+        ++n;
+    };
+    // end of a tile: the warps' partial accumulators meet in shared memory; one warp (they take
+    // turns) ends up with the complete 16 x 8 tile in the usual accumulator layout
+    auto reduce_tile = [&](float (&out)[4]) -> bool {
+        float *buf = red + (n_tiles & 1) * (kConsumerWarps * 128);
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const int ts = tig * 2 + h;
-                    if (ts < ctile.n_tok) {
-                        const int pos = v.tok_off + ts;
-                        const int pair = pos < n_pairs ? p.perm[pos] : pos;
-                        float *zr = p.zbuf + (size_t)pair * d + r;
-                        zr[0] = c0[h] + c1[h];
-                        zr[8] = c0[2 + h] + c1[2 + h];
-                    }
-                }
+        for (int i = 0; i < 4; ++i) {
+            buf[warp * 128 + i * 32 + lane] = c0[i] + c1[i];
+            c0[i] = c1[i] = 0.f;
+        }
+        consumer_bar();
+        const bool mine = warp == (n_tiles & (kConsumerWarps - 1));
+        if (mine) {
 #pragma unroll
-                for (int i = 0; i < 4; ++i)
-                    c0[i] = c1[i] = 0.f;
-                if (final_group) {
-                    // count the finished tiles of this 16-row block; the last one combines it
-                    unsigned old = 0;
-                    __threadfence();
-                    __syncwarp();
-                    if (lane == 0)
-                        old = atomicAdd(p.row_done + ctile.blk, 1u);
-                    old = __shfl_sync(0xffffffffu, old, 0);
-                    if (old == (unsigned)nv - 1u) {
-                        __threadfence();
-                        const int row = ctile.blk * 16 + (lane & 15);
-                        for (int t = lane >> 4; t < p.T; t += 2) {
-                            float y = 0.f;
-                            for (int j = 0; j < p.k; ++j)
-                                y = fmaf(p.gate[t * p.k + j], __ldcg(p.zbuf + (size_t)(t * p.k + j) * d + row), y);
-                            for (int s = 0; s < p.n_shared; ++s)
-                                y += __ldcg(p.zbuf + (size_t)(n_pairs + s * p.T + t) * d + row);
-                            p.out[(size_t)t * d + row] = bf16_rne(y);
-                        }
-                        if (lane == 0)
-                            p.row_done[ctile.blk] = 0;
-                    }
+            for (int i = 0; i < 4; ++i) {
+                float s = 0.f;
+#pragma unroll
+                for (int w = 0; w < kConsumerWarps; ++w)
+                    s += buf[w * 128 + i * 32 + lane];
+                out[i] = s;
+            }
+        }
+        ++n_tiles;
+        return mine;
+    };
+
+    // ---- phase 1: h = SiLU(W_g x) * (W_u x)
+    int cur_vr = -1;
+    VrRec v{};
+    for (int t = lo1; t < hi1; ++t) {
+        const int vr = vb + t / upe1, blk = t % upe1;
+        if (vr != cur_vr) {
+            v = p.vrs[vr];
+            cur_vr = vr;
+        }
+        for (int kc = 0; kc < nk1; ++kc)
+            compute(min(CB, rb1 - kc * CB), v.n_tok);
+        float r[4];
+        if (reduce_tile(r)) {
+            // rows g and g + 8 of the tile are g_f and u_f for f = 8 * blk + g
+            uint16_t *hrow = p.hbuf + ((size_t)vr * kTokPerVr) * Fpad + blk * 8 + g;
+            if (tig * 2 < v.n_tok)
+                hrow[(size_t)(tig * 2) * Fpad] = bf16_rne(r[0] / (1.0f + __expf(-r[0])) * r[2]);
+            if (tig * 2 + 1 < v.n_tok)
+                hrow[(size_t)(tig * 2 + 1) * Fpad] = bf16_rne(r[1] / (1.0f + __expf(-r[1])) * r[3]);
+        }
+    }
+    // this CTA's part of h is complete: tell the grid
+    __threadfence();
+    fence_proxy_async();       // h was written through the generic proxy, bulk copies will read it
+    consumer_bar();
+    if (tid == 0)
+        atomicAdd(p.sync + p.group, 1u);
+
+    // ---- phase 2: z = W_d h for this CTA's output rows
+    const int n_pairs = p.T * p.k;
+    for (int t = 0; t < hi2; ++t) {
+        const int vr = vb + t / mt, r0 = r_lo + 16 * (t % mt);
+        if (vr != cur_vr) {
+            v = p.vrs[vr];
+            cur_vr = vr;
+        }
+        for (int kc = 0; kc < nk2; ++kc)
+            compute(min(CB, rb2 - kc * CB), v.n_tok);
+        float r[4];
+        if (reduce_tile(r)) {
+            const int row = r0 + g;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int ts = tig * 2 + h;
+                if (ts < v.n_tok) {
+                    const int pos = v.tok_off + ts;
+                    const int pair = pos < n_pairs ? p.perm[pos] : pos;
+                    float *zr = p.zbuf + (size_t)pair * d + row;
+                    if (row < r_hi)
+                        zr[0] = r[h];
+                    if (row + 8 < r_hi)
+                        zr[8] = r[2 + h];
                 }
-                ck = 0;
-                ct += kWarps;
-                if (ct < hi2)
-                    ctile = tile2(ct);
             }
         }
     }
-    if (final_group && nv <= 0) {
-        // nothing computed in the last group (cannot happen for a well-formed plan): combine all rows
-        const int n_pairs = p.T * p.k;
-        for (int blk = blockIdx.x * kWarps + warp; blk < upe2; blk += G * kWarps) {
-            const int row = blk * 16 + (lane & 15);
-            for (int t = lane >> 4; t < p.T; t += 2) {
-                float y = 0.f;
-                for (int j = 0; j < p.k; ++j)
-                    y = fmaf(p.gate[t * p.k + j], __ldcg(p.zbuf + (size_t)(t * p.k + j) * d + row), y);
-                for (int s = 0; s < p.n_shared; ++s)
-                    y += __ldcg(p.zbuf + (size_t)(n_pairs + s * p.T + t) * d + row);
-                p.out[(size_t)t * d + row] = bf16_rne(y);
-            }
+    // ---- combine (Eq. 2) of this CTA's rows, once the call's last group has produced its z
+    if (final_group) {
+        __threadfence_block();
+        consumer_bar();
+        const int nr = r_hi - r_lo;
+        for (int i = tid; i < nr * p.T; i += kConsumerWarps * 32) {
+            const int tk = i / nr, orow = r_lo + i % nr;
+            float y = 0.f;
+            for (int j = 0; j < p.k; ++j)
+                y = fmaf(p.gate[tk * p.k + j], __ldcg(p.zbuf + (size_t)(tk * p.k + j) * d + orow), y);
+            for (int sh = 0; sh < p.n_shared; ++sh)
+                y += __ldcg(p.zbuf + (size_t)(n_pairs + sh * p.T + tk) * d + orow);
+            p.out[(size_t)tk * d + orow] = bf16_rne(y);
         }
     }
-    __syncwarp();
-    if (*abort_flag && lane == 0) {
-        // a wait ran out: give the copies this warp still has in flight a bounded time to land
-        // before its shared memory goes away, then report
-        const unsigned long long t0 = globaltimer_ns();
-        const uint32_t first = n_issued > (uint32_t)S ? n_issued - S : 0u;
-        for (uint32_t n = first; n < n_issued; ++n)
-            while (!mbar_try(bar_s + 8 * (n % S), (n / S) & 1u) && globaltimer_ns() - t0 < kWaitLimitNs) {
-            }
+    if (*abort_flag && tid == 0)
         atomicExch(p.err, MELINOE_ERR_TIMEOUT);
-    }
 }
-
-constexpr int kKC = 128;
-constexpr int kS = 4;
 
 }  // namespace
 
 cudaError_t ffn_stream_configure(int n_sms, size_t max_smem, FfnLaunchCfg *cfg)
 {
-    const size_t need = (size_t)kWarps * kS * kStageRows * (2 * kKC + 16) + (size_t)kWarps * kS * 8 + 64;
-    if (need > max_smem)
-        return cudaErrorInvalidConfiguration;
-    cudaError_t e = cudaFuncSetAttribute(ffn_stream_kernel<kKC, kS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)need);
+    const size_t usable = max_smem - 1024;   // room for the kernel's static shared memory
+    cudaError_t e = cudaFuncSetAttribute(ffn_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)usable);
     if (e != cudaSuccess)
         return e;
     int per_sm = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ffn_stream_kernel<kKC, kS>, kThreads, need);
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ffn_stream_kernel, kThreads, usable);
     if (e != cudaSuccess)
         return e;
     if (per_sm < 1)
         return cudaErrorInvalidConfiguration;
     cfg->grid = n_sms;          // one CTA per SM: all of them resident, which the grid barrier needs
-    cfg->smem_bytes = need;
+    cfg->max_smem = usable;
     return cudaSuccess;
 }
 
-cudaError_t launch_ffn_stream(cudaStream_t stream, const FfnLaunchCfg &cfg, const FfnParams &p)
+// Ring geometry for a call of T tokens on a d x F layer.
+cudaError_t ffn_stream_geometry(const FfnLaunchCfg &cfg, int d, int F, int T, FfnGeometry *geo)
+{
+    int longest = 2 * (d > F ? d : F);
+    if (longest > kMaxChunk)
+        longest = kMaxChunk;
+    geo->chunk_bytes = (longest + 127) / 128 * 128;
+    geo->pitch = geo->chunk_bytes + 16;
+    geo->n_op_rows = T < kTokPerVr ? T : kTokPerVr;
+    const size_t stage = (size_t)(16 + geo->n_op_rows) * geo->pitch;
+    const size_t fixed = 2 * kConsumerWarps * 128 * sizeof(float) + 2 * kMaxStages * 8 + 128;
+    if (cfg.max_smem < fixed + 2 * stage)
+        return cudaErrorInvalidConfiguration;
+    size_t s = (cfg.max_smem - fixed) / stage;
+    if (s > (size_t)kMaxStages)
+        s = kMaxStages;
+    geo->n_stages = (int)s;
+    geo->smem_bytes = fixed + s * stage;
+    return cudaSuccess;
+}
+
+cudaError_t launch_ffn_stream(cudaStream_t stream, const FfnLaunchCfg &cfg, const FfnGeometry &geo, const FfnParams &p)
 {
     FfnParams q = p;
-    void *args[] = {&q};
-    cudaError_t e = cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(ffn_stream_kernel<kKC, kS>),
-                                                dim3(cfg.grid), dim3(kThreads), args, cfg.smem_bytes, stream);
+    FfnGeometry gq = geo;
+    void *args[] = {&q, &gq};
+    cudaError_t e = cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(ffn_stream_kernel), dim3(cfg.grid),
+                                                dim3(kThreads), args, geo.smem_bytes, stream);
     count_launch();
     return e;
 }

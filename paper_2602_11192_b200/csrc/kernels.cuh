@@ -48,16 +48,22 @@ struct FfnParams {
     float *zbuf;                     // expert outputs: [T*k routed pairs, then n_shared*T][d] fp32
     uint16_t *out;                   // [T][d] bf16
     unsigned *sync;                  // grid-barrier counters, one per compute group (zero at launch)
-    unsigned *row_done;              // per 16-row block: finished tiles of the last group (self-resetting)
     int *err;                        // device error word (0 = ok)
     int d, F, Fpad, E, k, T, n_shared;
     int group;
 };
 struct FfnLaunchCfg {
-    int grid;
+    int grid;                        // one CTA per SM
+    size_t max_smem;                 // dynamic shared memory the kernel may use
+};
+// Shape of the shared-memory ring for one call.
+struct FfnGeometry {
+    int n_stages, pitch, chunk_bytes, n_op_rows;
     size_t smem_bytes;
 };
 cudaError_t ffn_stream_configure(int n_sms, size_t max_smem, FfnLaunchCfg *cfg);
-cudaError_t launch_ffn_stream(cudaStream_t stream, const FfnLaunchCfg &cfg, const FfnParams &p);
+cudaError_t ffn_stream_geometry(const FfnLaunchCfg &cfg, int d, int F, int T, FfnGeometry *geo);
+cudaError_t launch_ffn_stream(cudaStream_t stream, const FfnLaunchCfg &cfg, const FfnGeometry &geo,
+                              const FfnParams &p);
 
 }  // namespace melinoe
