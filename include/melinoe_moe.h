@@ -194,6 +194,17 @@ int melinoe_moe_cache_state(melinoe_moe_t *h, int32_t *expert_of_slot_host, uint
 int melinoe_moe_enable_timing(melinoe_moe_t *h, int enable);
 int melinoe_moe_ffn_time_ms(melinoe_moe_t *h, double *ms_out, int64_t *launches_out);
 
+/*
+ * Kernel timeline for profiling (no counterpart in the paper).  trace_dev: device memory of at
+ * least 8 * 8 bytes per SM of the device (melinoe_moe_trace_ctas() * 64 bytes), 8-byte aligned,
+ * borrowed; NULL switches tracing off.  Every expert-FFN launch then overwrites, per CTA, eight
+ * 64-bit nanosecond stamps of the device's global timer: 0 entry, 1 set-up done, 2 first weight
+ * stage landed, 3 gate/up phase done, 4 arrived at the grid barrier, 5 barrier passed (producer),
+ * 6 down-projection phase done, 7 exit.  Stamps of steps a CTA skipped keep their old value.
+ */
+int melinoe_moe_set_trace(melinoe_moe_t *h, void *trace_dev, size_t bytes);
+int melinoe_moe_trace_ctas(melinoe_moe_t *h);
+
 /* Number of kernels this library has launched in this process (all handles). */
 int64_t melinoe_launch_count(void);
 

@@ -78,6 +78,7 @@ struct melinoe_moe {
     float *gate = nullptr, *logits = nullptr, *zbuf = nullptr;
     uint16_t *hbuf = nullptr;
     unsigned *sync = nullptr;
+    unsigned long long *trace = nullptr;   // borrowed; see melinoe_moe_set_trace
     VrRec *vrs = nullptr;
     uint16_t *stage_in = nullptr, *stage_out = nullptr;
     melinoe_moe_stats *stage_stats = nullptr;
@@ -486,6 +487,9 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
     pp.cache = h->cache;
     pp.plan = h->plan;
     pp.vrs = h->vrs;
+    pp.slots = h->slots;
+    pp.slot_stride = h->slot_stride;
+    pp.shared_blobs = h->shared_dev;
     pp.perm = h->perm;
     pp.inv_pos = h->inv_pos;
     pp.tok_of_sorted = h->tok_of_sorted;
@@ -500,13 +504,8 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
     CU_TRY(cudaEventRecord(h->ev_plan, s));
 
     FfnParams fp;
-    fp.slots = h->slots;
-    fp.slot_stride = h->slot_stride;
-    fp.shared_blobs = h->shared_dev;
     fp.plan = h->plan;
     fp.vrs = h->vrs;
-    fp.tok_of_sorted = h->tok_of_sorted;
-    fp.perm = h->perm;
     fp.x = static_cast<const uint16_t *>(hidden_dev);
     fp.gate = h->gate;
     fp.hbuf = h->hbuf;
@@ -514,6 +513,7 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
     fp.out = static_cast<uint16_t *>(out_dev);
     fp.sync = h->sync;
     fp.err = h->err_word;
+    fp.trace = h->trace;
     fp.d = h->d;
     fp.F = h->F;
     fp.Fpad = (h->F + 255) / 256 * 256;
@@ -782,6 +782,22 @@ int melinoe_moe_cache_state(melinoe_moe_t *h, int32_t *expert_of_slot_host, uint
         return err;
     return h->sticky.load();
 }
+
+int melinoe_moe_set_trace(melinoe_moe_t *h, void *trace_dev, size_t bytes)
+{
+    if (!h)
+        return MELINOE_ERR_INVALID;
+    if (!trace_dev) {
+        h->trace = nullptr;
+        return MELINOE_OK;
+    }
+    if (bytes < (size_t)h->cfg.grid * 8 * sizeof(unsigned long long) || (reinterpret_cast<uintptr_t>(trace_dev) & 7u))
+        return MELINOE_ERR_INVALID;
+    h->trace = static_cast<unsigned long long *>(trace_dev);
+    return MELINOE_OK;
+}
+
+int melinoe_moe_trace_ctas(melinoe_moe_t *h) { return h ? h->cfg.grid : 0; }
 
 int melinoe_moe_enable_timing(melinoe_moe_t *h, int enable)
 {

@@ -15,8 +15,9 @@
 //            layout a thread holds g_f and u_f of the same f and the same two tokens, so
 //            h = SiLU(g) * u is thread-local; h goes to global memory as bf16.
 //   barrier  grid-wide, crossed by the producer warps only (bounded spin on a device counter):
-//            the consumers never wait for it, and the first W_d stages of phase 2 are already
-//            in flight when the producer reaches it.
+//            the consumers never wait for it.  The ring is cut anew for the (usually shorter)
+//            W_d rows as soon as the CTA's own phase 1 has drained, and as many W_d stages as
+//            fit are in flight before the producer reaches the barrier.
 //   phase 2  every CTA owns a contiguous range of the d_model output rows (d/G of them, so the
 //            split is even to within one row) for ALL virtual requests of the launch.  Tile =
 //            up to 16 of those W_d rows of one virtual request: D[16 x 8] = W_d rows * h^T, a
@@ -168,34 +169,45 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
     const int d = p.d, F = p.F, Fpad = p.Fpad;
     const DevPlan *plan = p.plan;
     const int G = (int)gridDim.x;
-    const int S = geo.n_stages, PITCH = geo.pitch, CB = geo.chunk_bytes;
-    const int STAGE = (16 + geo.n_op_rows) * PITCH;
+    const int NOP = geo.n_op_rows;
+    const int S1 = geo.n_stages, PITCH1 = geo.pitch, CB1 = geo.chunk_bytes, STAGE1 = (16 + NOP) * PITCH1;
+    const int S2 = geo.n_stages2, PITCH2 = geo.pitch2, CB2 = geo.chunk_bytes2, STAGE2 = (16 + NOP) * PITCH2;
 
-    if (plan->status != MELINOE_OK) {
+    // optional timeline: 8 device-clock stamps per CTA (see melinoe_moe_set_trace)
+    unsigned long long *trace = p.trace ? p.trace + (size_t)blockIdx.x * 8 : nullptr;
+    if (trace && tid == 0)
+        trace[0] = globaltimer_ns();
+
+    const int status = plan->status, n_groups = plan->n_groups;
+    const int vb = plan->group_vr_begin[p.group];
+    const int nv = plan->group_vr_begin[p.group + 1] - vb;
+    if (status != MELINOE_OK) {
         // the call was refused on the device: the output is all zeros, the status tells why
         if (p.group == 0)
             for (size_t i = (size_t)blockIdx.x * kThreads + tid; i < (size_t)p.T * d; i += (size_t)G * kThreads)
                 p.out[i] = 0;
         return;
     }
-    const int vb = plan->group_vr_begin[p.group];
-    const int nv = plan->group_vr_begin[p.group + 1] - vb;
-    const bool final_group = p.group == plan->n_groups - 1;
+    const bool final_group = p.group == n_groups - 1;
     if (nv <= 0 && !final_group)
         return;
 
+    // ring | reduction buffers | barriers (phase 1 full/empty, phase 2 full/empty)
     unsigned char *ring = smem;
-    float *red = reinterpret_cast<float *>(smem + (size_t)S * STAGE);          // [2][8 warps][4][32]
+    float *red = reinterpret_cast<float *>(smem + geo.ring_bytes);              // [2][8 warps][4][32]
     uint64_t *bars = reinterpret_cast<uint64_t *>(red + 2 * kConsumerWarps * 128);
     const uint32_t ring_s = smem_u32(ring);
-    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + kMaxStages);
+    const uint32_t full1 = smem_u32(bars), empty1 = full1 + 8 * kMaxStages;
+    const uint32_t full2 = empty1 + 8 * kMaxStages, empty2 = full2 + 8 * kMaxStages;
     volatile int *abort_flag = &s_abort;
 
     if (tid == 0) {
         s_abort = 0;
-        for (int i = 0; i < S; ++i) {
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(full0 + 8 * i), "r"(1));
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(empty0 + 8 * i), "r"(kConsumerWarps));
+        for (int i = 0; i < kMaxStages; ++i) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(full1 + 8 * i), "r"(1));
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(empty1 + 8 * i), "r"(kConsumerWarps));
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(full2 + 8 * i), "r"(1));
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(empty2 + 8 * i), "r"(kConsumerWarps));
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -203,16 +215,18 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
         // the last 16-column step of a W_d row is half filled: what the copy leaves untouched
         // must be finite, because it meets the zero padding of the h rows in the product
         uint4 *z = reinterpret_cast<uint4 *>(ring);
-        for (int i = tid; i < S * STAGE / 16; i += kThreads)
+        for (int i = tid; i < (int)(geo.ring_bytes / 16); i += kThreads)
             z[i] = make_uint4(0, 0, 0, 0);
         fence_proxy_async();
     }
     __syncthreads();
+    if (trace && tid == 0)
+        trace[1] = globaltimer_ns();
 
     // ---- phase 1: a contiguous range of (virtual request, 8-row f-block) tiles per CTA
     const int upe1 = F / 8;
     const int rb1 = 2 * d, rb2 = 2 * F;                       // row bytes
-    const int nk1 = (rb1 + CB - 1) / CB, nk2 = (rb2 + CB - 1) / CB;
+    const int nk1 = (rb1 + CB1 - 1) / CB1, nk2 = (rb2 + CB2 - 1) / CB2;
     const long long NT1 = (long long)nv * upe1;
     const int lo1 = (int)(blockIdx.x * NT1 / G), hi1 = (int)((blockIdx.x + 1) * NT1 / G);
     // ---- phase 2: output rows [r_lo, r_hi) of every virtual request, in tiles of up to 16 rows
@@ -222,10 +236,6 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
 
     if (warp == kConsumerWarps) {
         // =================================================================== producer
-        auto blob_of = [&](const VrRec &v) -> const char * {
-            const ReqRec rec = plan->req[v.req];
-            return rec.slot >= 0 ? p.slots + (size_t)rec.slot * p.slot_stride : p.shared_blobs[rec.expert - p.E];
-        };
         // Per virtual request (looked up only when the tile sequence moves on to the next one):
         // this lane's source row of block 0 and its stride from one block to the next.
         int cur_vr = -1, cur_ntok = 0;
@@ -235,17 +245,16 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
         auto tile1 = [&](int t) -> Tile {
             const int vr = vb + t / upe1, blk = t % upe1;
             if (vr != cur_vr) {
-                const VrRec v = p.vrs[vr];
+                const VrRec *v = p.vrs + vr;
                 cur_vr = vr;
-                cur_ntok = v.n_tok;
+                cur_ntok = v->n_tok;
                 lane_base = nullptr;
                 lane_step = 0;
                 if (lane < 16) {
-                    lane_base = blob_of(v) + (size_t)((lane < 8 ? 0 : F) + (lane & 7)) * rb1;
+                    lane_base = v->blob + (size_t)((lane < 8 ? 0 : F) + (lane & 7)) * rb1;
                     lane_step = (size_t)8 * rb1;
-                } else if (lane - 16 < v.n_tok) {
-                    const int tok = p.tok_of_sorted[v.tok_off + lane - 16];
-                    lane_base = reinterpret_cast<const char *>(p.x) + (size_t)tok * rb1;
+                } else if (lane - 16 < cur_ntok) {
+                    lane_base = reinterpret_cast<const char *>(p.x) + (size_t)v->tok[lane - 16] * rb1;
                 }
             }
             Tile ti;
@@ -258,15 +267,15 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
         auto tile2 = [&](int t) -> Tile {
             const int vr = vb + t / mt, blk = t % mt;
             if (vr != cur_vr) {
-                const VrRec v = p.vrs[vr];
+                const VrRec *v = p.vrs + vr;
                 cur_vr = vr;
-                cur_ntok = v.n_tok;
+                cur_ntok = v->n_tok;
                 lane_base = nullptr;
                 lane_step = 0;
                 if (lane < 16) {
-                    lane_base = blob_of(v) + (size_t)2 * F * rb1 + (size_t)(r_lo + lane) * rb2;
+                    lane_base = v->blob + (size_t)2 * F * rb1 + (size_t)(r_lo + lane) * rb2;
                     lane_step = (size_t)16 * rb2;
-                } else if (lane - 16 < v.n_tok) {
+                } else if (lane - 16 < cur_ntok) {
                     lane_base = reinterpret_cast<const char *>(p.hbuf) + ((size_t)vr * kTokPerVr + lane - 16) * Fpad * 2;
                 }
             }
@@ -278,11 +287,11 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
                 ti.src = nullptr;
             return ti;
         };
-        uint32_t n = 0;   // stages issued so far, over both phases
         bool dead = false;
-        // parts bit 0: wait for the slot, arm the barrier, fetch the weight rows; bit 1: operand rows.
-        // wbytes: bytes of each weight-row piece; obytes: bytes of each operand-row piece.
-        auto issue = [&](const Tile &ti, int kc, int wbytes, int obytes, int parts, uint32_t nn) {
+        // One stage of either phase.  parts bit 0: wait for the slot, arm the barrier, fetch the
+        // weight rows; bit 1: operand rows.  wbytes / obytes: bytes of each weight / operand piece.
+        auto issue = [&](const Tile &ti, uint32_t full0, uint32_t empty0, int S, int STAGE, int PITCH, size_t src_off,
+                         int wbytes, int obytes, int parts, uint32_t nn) {
             const uint32_t slot = nn % S;
             const uint32_t bar = full0 + 8 * slot;
             if (parts & 1) {
@@ -295,28 +304,33 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
             if (ti.src && !dead) {
                 const bool is_w = lane < 16;
                 if (is_w ? (parts & 1) : (parts & 2))
-                    bulk_g2s(ring_s + slot * STAGE + lane * PITCH, ti.src + (size_t)kc * CB,
+                    bulk_g2s(ring_s + slot * STAGE + lane * PITCH, ti.src + src_off,
                              (uint32_t)(is_w ? wbytes : obytes), bar);
             }
         };
+        uint32_t n1 = 0;
         for (int t = lo1; t < hi1; ++t) {
             const Tile ti = tile1(t);
             for (int kc = 0; kc < nk1; ++kc) {
-                const int b = min(CB, rb1 - kc * CB);
-                issue(ti, kc, b, b, 3, n++);
+                const int b = min(CB1, rb1 - kc * CB1);
+                issue(ti, full1, empty1, S1, STAGE1, PITCH1, (size_t)kc * CB1, b, b, 3, n1++);
             }
         }
+        // the ring is cut anew for phase 2: wait until the consumers have let go of every phase-1 stage
+        for (uint32_t m = n1 > (uint32_t)S1 ? n1 - S1 : 0u; m < n1 && !dead; ++m)
+            dead = !mbar_wait(empty1 + 8 * (m % S1), (m / S1) & 1u, abort_flag);
         // phase 2: the first stages go out with their weight rows only; h is not complete yet
         cur_vr = -1;
+        uint32_t n2 = 0;
         int t2 = 0, k2 = 0;
         Tile ti2{};
         if (t2 < hi2)
             ti2 = tile2(t2);
-        auto op_bytes2 = [&](int kc) { return min(CB, Fpad * 2 - kc * CB); };
-        const uint32_t n_pre0 = n;
+        auto w_bytes2 = [&](int kc) { return min(CB2, rb2 - kc * CB2); };
+        auto op_bytes2 = [&](int kc) { return min(CB2, Fpad * 2 - kc * CB2); };
         int pre = 0;
-        for (; pre < S && t2 < hi2; ++pre) {
-            issue(ti2, k2, min(CB, rb2 - k2 * CB), op_bytes2(k2), 1, n++);
+        for (; pre < S2 && t2 < hi2; ++pre) {
+            issue(ti2, full2, empty2, S2, STAGE2, PITCH2, (size_t)k2 * CB2, w_bytes2(k2), op_bytes2(k2), 1, n2++);
             if (++k2 == nk2) {
                 k2 = 0;
                 if (++t2 < hi2)
@@ -337,6 +351,8 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
                 }
             }
             __threadfence();
+            if (trace)
+                trace[5] = globaltimer_ns();
         }
         __syncwarp();
         fence_proxy_async();
@@ -352,7 +368,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
             if (pre > 0)
                 qtile = tile2(0);
             for (int i = 0; i < pre; ++i) {
-                issue(qtile, qk, 0, op_bytes2(qk), 2, n_pre0 + i);
+                issue(qtile, full2, empty2, S2, STAGE2, PITCH2, (size_t)qk * CB2, 0, op_bytes2(qk), 2, (uint32_t)i);
                 if (++qk == nk2) {
                     qk = 0;
                     if (++qt < hi2)
@@ -365,7 +381,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
             lane_step = keep_step;
         }
         while (t2 < hi2) {
-            issue(ti2, k2, min(CB, rb2 - k2 * CB), op_bytes2(k2), 3, n++);
+            issue(ti2, full2, empty2, S2, STAGE2, PITCH2, (size_t)k2 * CB2, w_bytes2(k2), op_bytes2(k2), 3, n2++);
             if (++k2 == nk2) {
                 k2 = 0;
                 if (++t2 < hi2)
@@ -376,9 +392,11 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
             // a wait ran out: give the copies still in flight a bounded time to land before this
             // CTA's shared memory goes away
             const unsigned long long t0 = globaltimer_ns();
-            const uint32_t first = n > (uint32_t)S ? n - S : 0u;
-            for (uint32_t m = first; m < n; ++m)
-                while (!mbar_try(full0 + 8 * (m % S), (m / S) & 1u) && globaltimer_ns() - t0 < kWaitLimitNs) {
+            for (uint32_t m = n1 > (uint32_t)S1 ? n1 - S1 : 0u; m < n1; ++m)
+                while (!mbar_try(full1 + 8 * (m % S1), (m / S1) & 1u) && globaltimer_ns() - t0 < kWaitLimitNs) {
+                }
+            for (uint32_t m = n2 > (uint32_t)S2 ? n2 - S2 : 0u; m < n2; ++m)
+                while (!mbar_try(full2 + 8 * (m % S2), (m / S2) & 1u) && globaltimer_ns() - t0 < kWaitLimitNs) {
                 }
             atomicExch(p.err, MELINOE_ERR_TIMEOUT);
         }
@@ -387,14 +405,12 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
 
     // ======================================================================= consumers
     const int g = lane >> 2, tig = lane & 3;
-    const uint32_t a_off = ((lane & 7) + ((lane >> 3) & 1) * 8) * PITCH + (lane >> 4) * 16;
-    const uint32_t b_off = (16 + g) * PITCH + tig * 4;
-    uint32_t n = 0;        // stages consumed so far
     int n_tiles = 0;       // tiles finished so far (selects the reduction buffer and the epilogue warp)
     float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
 
     // this warp's share of one stage: some of the 16-column steps of the piece
-    auto compute = [&](int bytes, int n_tok) {
+    auto compute = [&](uint32_t full0, uint32_t empty0, int S, int STAGE, uint32_t a_off, uint32_t b_off, uint32_t n,
+                       int bytes, int n_tok) {
         const uint32_t slot = n % S;
         mbar_wait(full0 + 8 * slot, (n / S) & 1u, abort_flag);
         const uint32_t base = ring_s + slot * STAGE;
@@ -429,7 +445,6 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
         __syncwarp();
         if (lane == 0)
             mbar_arrive(empty0 + 8 * slot);
-        ++n;
     };
     // end of a tile: the warps' partial accumulators meet in shared memory; one warp (they take
     // turns) ends up with the complete 16 x 8 tile in the usual accumulator layout
@@ -455,67 +470,103 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
         ++n_tiles;
         return mine;
     };
+    // what a consumer lane needs of a virtual request: its token count and the z rows of the two
+    // token slots this lane's accumulators belong to
+    struct VrInfo {
+        int n_tok, pair0, pair1;
+    };
+    auto load_vr = [&](int vr) -> VrInfo {
+        const VrRec *v = p.vrs + vr;
+        VrInfo r;
+        r.n_tok = v->n_tok;
+        const int2 pr = *reinterpret_cast<const int2 *>(v->pair + tig * 2);
+        r.pair0 = pr.x;
+        r.pair1 = pr.y;
+        return r;
+    };
 
     // ---- phase 1: h = SiLU(W_g x) * (W_u x)
-    int cur_vr = -1;
-    VrRec v{};
-    for (int t = lo1; t < hi1; ++t) {
-        const int vr = vb + t / upe1, blk = t % upe1;
-        if (vr != cur_vr) {
-            v = p.vrs[vr];
-            cur_vr = vr;
-        }
-        for (int kc = 0; kc < nk1; ++kc)
-            compute(min(CB, rb1 - kc * CB), v.n_tok);
-        float r[4];
-        if (reduce_tile(r)) {
-            // rows g and g + 8 of the tile are g_f and u_f for f = 8 * blk + g
-            uint16_t *hrow = p.hbuf + ((size_t)vr * kTokPerVr) * Fpad + blk * 8 + g;
-            if (tig * 2 < v.n_tok)
-                hrow[(size_t)(tig * 2) * Fpad] = bf16_rne(r[0] / (1.0f + __expf(-r[0])) * r[2]);
-            if (tig * 2 + 1 < v.n_tok)
-                hrow[(size_t)(tig * 2 + 1) * Fpad] = bf16_rne(r[1] / (1.0f + __expf(-r[1])) * r[3]);
+    {
+        const uint32_t a_off = ((lane & 7) + ((lane >> 3) & 1) * 8) * PITCH1 + (lane >> 4) * 16;
+        const uint32_t b_off = (16 + g) * PITCH1 + tig * 4;
+        uint32_t n = 0;
+        int cur_vr = -1;
+        VrInfo v{};
+        for (int t = lo1; t < hi1; ++t) {
+            const int vr = vb + t / upe1, blk = t % upe1;
+            if (vr != cur_vr) {
+                v = load_vr(vr);
+                cur_vr = vr;
+            }
+            for (int kc = 0; kc < nk1; ++kc) {
+                compute(full1, empty1, S1, STAGE1, a_off, b_off, n, min(CB1, rb1 - kc * CB1), v.n_tok);
+                if (trace && n == 0 && tid == 0)
+                    trace[2] = globaltimer_ns();
+                ++n;
+            }
+            float r[4];
+            if (reduce_tile(r)) {
+                // rows g and g + 8 of the tile are g_f and u_f for f = 8 * blk + g
+                uint16_t *hrow = p.hbuf + ((size_t)vr * kTokPerVr) * Fpad + blk * 8 + g;
+                if (tig * 2 < v.n_tok)
+                    hrow[(size_t)(tig * 2) * Fpad] = bf16_rne(r[0] / (1.0f + __expf(-r[0])) * r[2]);
+                if (tig * 2 + 1 < v.n_tok)
+                    hrow[(size_t)(tig * 2 + 1) * Fpad] = bf16_rne(r[1] / (1.0f + __expf(-r[1])) * r[3]);
+            }
         }
     }
+    if (trace && tid == 0)
+        trace[3] = globaltimer_ns();
     // this CTA's part of h is complete: tell the grid
     __threadfence();
     fence_proxy_async();       // h was written through the generic proxy, bulk copies will read it
     consumer_bar();
-    if (tid == 0)
+    if (tid == 0) {
         atomicAdd(p.sync + p.group, 1u);
+        if (trace)
+            trace[4] = globaltimer_ns();
+    }
 
     // ---- phase 2: z = W_d h for this CTA's output rows
-    const int n_pairs = p.T * p.k;
-    for (int t = 0; t < hi2; ++t) {
-        const int vr = vb + t / mt, r0 = r_lo + 16 * (t % mt);
-        if (vr != cur_vr) {
-            v = p.vrs[vr];
-            cur_vr = vr;
-        }
-        for (int kc = 0; kc < nk2; ++kc)
-            compute(min(CB, rb2 - kc * CB), v.n_tok);
-        float r[4];
-        if (reduce_tile(r)) {
-            const int row = r0 + g;
+    {
+        const uint32_t a_off = ((lane & 7) + ((lane >> 3) & 1) * 8) * PITCH2 + (lane >> 4) * 16;
+        const uint32_t b_off = (16 + g) * PITCH2 + tig * 4;
+        uint32_t n = 0;
+        VrInfo v{}, nxt{};
+        if (hi2 > 0)
+            nxt = load_vr(vb);
+        for (int t = 0; t < hi2; ++t) {
+            const int blk = t % mt, r0 = r_lo + 16 * blk;
+            if (blk == 0) {
+                v = nxt;
+                if (t + mt < hi2)
+                    nxt = load_vr(vb + t / mt + 1);   // in flight while this request's tiles are computed
+            }
+            for (int kc = 0; kc < nk2; ++kc, ++n)
+                compute(full2, empty2, S2, STAGE2, a_off, b_off, n, min(CB2, rb2 - kc * CB2), v.n_tok);
+            float r[4];
+            if (reduce_tile(r)) {
+                const int row = r0 + g;
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const int ts = tig * 2 + h;
-                if (ts < v.n_tok) {
-                    const int pos = v.tok_off + ts;
-                    const int pair = pos < n_pairs ? p.perm[pos] : pos;
-                    float *zr = p.zbuf + (size_t)pair * d + row;
-                    if (row < r_hi)
-                        zr[0] = r[h];
-                    if (row + 8 < r_hi)
-                        zr[8] = r[2 + h];
+                for (int h = 0; h < 2; ++h) {
+                    if (tig * 2 + h < v.n_tok) {
+                        float *zr = p.zbuf + (size_t)(h ? v.pair1 : v.pair0) * d + row;
+                        if (row < r_hi)
+                            zr[0] = r[h];
+                        if (row + 8 < r_hi)
+                            zr[8] = r[2 + h];
+                    }
                 }
             }
         }
     }
+    if (trace && tid == 0)
+        trace[6] = globaltimer_ns();
     // ---- combine (Eq. 2) of this CTA's rows, once the call's last group has produced its z
     if (final_group) {
         __threadfence_block();
         consumer_bar();
+        const int n_pairs = p.T * p.k;
         const int nr = r_hi - r_lo;
         for (int i = tid; i < nr * p.T; i += kConsumerWarps * 32) {
             const int tk = i / nr, orow = r_lo + i % nr;
@@ -527,6 +578,8 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
             p.out[(size_t)tk * d + orow] = bf16_rne(y);
         }
     }
+    if (trace && tid == 0)
+        trace[7] = globaltimer_ns();
     if (*abort_flag && tid == 0)
         atomicExch(p.err, MELINOE_ERR_TIMEOUT);
 }
@@ -550,24 +603,38 @@ cudaError_t ffn_stream_configure(int n_sms, size_t max_smem, FfnLaunchCfg *cfg)
     return cudaSuccess;
 }
 
-// Ring geometry for a call of T tokens on a d x F layer.
+// Ring geometry for a call of T tokens on a d x F layer: the same shared memory is cut into
+// stages of (16 + operand rows) row pieces twice, once for rows of 2*d bytes (gate/up phase)
+// and once for rows of 2*F bytes (down phase).
 cudaError_t ffn_stream_geometry(const FfnLaunchCfg &cfg, int d, int F, int T, FfnGeometry *geo)
 {
-    int longest = 2 * (d > F ? d : F);
-    if (longest > kMaxChunk)
-        longest = kMaxChunk;
-    geo->chunk_bytes = (longest + 127) / 128 * 128;
-    geo->pitch = geo->chunk_bytes + 16;
+    auto chunk_of = [](int row_bytes) {
+        const int c = row_bytes < kMaxChunk ? row_bytes : kMaxChunk;
+        return (c + 127) / 128 * 128;
+    };
     geo->n_op_rows = T < kTokPerVr ? T : kTokPerVr;
-    const size_t stage = (size_t)(16 + geo->n_op_rows) * geo->pitch;
-    const size_t fixed = 2 * kConsumerWarps * 128 * sizeof(float) + 2 * kMaxStages * 8 + 128;
-    if (cfg.max_smem < fixed + 2 * stage)
+    geo->chunk_bytes = chunk_of(2 * d);
+    geo->pitch = geo->chunk_bytes + 16;
+    geo->chunk_bytes2 = chunk_of(2 * F);
+    geo->pitch2 = geo->chunk_bytes2 + 16;
+    const size_t rows = 16 + geo->n_op_rows;
+    const size_t stage1 = rows * geo->pitch, stage2 = rows * geo->pitch2;
+    const size_t fixed = 2 * kConsumerWarps * 128 * sizeof(float) + 4 * kMaxStages * 8 + 128;
+    const size_t big = stage1 > stage2 ? stage1 : stage2;
+    if (cfg.max_smem < fixed + 2 * big)
         return cudaErrorInvalidConfiguration;
-    size_t s = (cfg.max_smem - fixed) / stage;
-    if (s > (size_t)kMaxStages)
-        s = kMaxStages;
-    geo->n_stages = (int)s;
-    geo->smem_bytes = fixed + s * stage;
+    const size_t avail = (cfg.max_smem - fixed) / 128 * 128;
+    size_t s1 = avail / stage1, s2 = avail / stage2;
+    if (s1 > (size_t)kMaxStages)
+        s1 = kMaxStages;
+    if (s2 > (size_t)kMaxStages)
+        s2 = kMaxStages;
+    geo->n_stages = (int)s1;
+    geo->n_stages2 = (int)s2;
+    size_t ring = s1 * stage1 > s2 * stage2 ? s1 * stage1 : s2 * stage2;
+    ring = (ring + 127) / 128 * 128;
+    geo->ring_bytes = ring;
+    geo->smem_bytes = ring + fixed;
     return cudaSuccess;
 }
 

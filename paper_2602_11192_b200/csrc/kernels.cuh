@@ -22,6 +22,9 @@ struct PlanParams {
     DevCache *cache;
     DevPlan *plan;
     VrRec *vrs;
+    const char *slots;        // device cache (slot s at slots + s * slot_stride), for the vrs' blob pointers
+    size_t slot_stride;
+    const char *const *shared_blobs;
     int32_t *perm, *inv_pos, *tok_of_sorted;
     HostPlan *hplan;          // page-locked host memory (device-visible address)
     unsigned *sync;           // grid-barrier counters of the FFN launches, zeroed here
@@ -35,13 +38,8 @@ cudaError_t launch_plan(cudaStream_t stream, const PlanParams &p);
 
 // ---- streaming expert FFN (Eq. 3) with the gate-weighted combine (Eq. 2) fused in
 struct FfnParams {
-    const char *slots;               // device cache: slot s at slots + s * slot_stride
-    size_t slot_stride;
-    const char *const *shared_blobs; // device array of shared-expert blobs, or null
     const DevPlan *plan;
     const VrRec *vrs;
-    const int32_t *tok_of_sorted;
-    const int32_t *perm;             // sorted position -> flat pair index t * k + j
     const uint16_t *x;               // hidden [T][d] bf16
     const float *gate;               // [T][k]
     uint16_t *hbuf;                  // h = SiLU(g) * u: [virtual request][8 token slots][Fpad] bf16
@@ -49,6 +47,7 @@ struct FfnParams {
     uint16_t *out;                   // [T][d] bf16
     unsigned *sync;                  // grid-barrier counters, one per compute group (zero at launch)
     int *err;                        // device error word (0 = ok)
+    unsigned long long *trace;       // null, or 8 clock stamps per CTA of the most recent launch
     int d, F, Fpad, E, k, T, n_shared;
     int group;
 };
@@ -58,8 +57,10 @@ struct FfnLaunchCfg {
 };
 // Shape of the shared-memory ring for one call.
 struct FfnGeometry {
-    int n_stages, pitch, chunk_bytes, n_op_rows;
-    size_t smem_bytes;
+    int n_op_rows;                   // operand rows per stage: min(T, 8)
+    int n_stages, pitch, chunk_bytes;        // gate/up phase: the ring as n_stages stages of (16 + n_op_rows) rows
+    int n_stages2, pitch2, chunk_bytes2;     // down phase: the same memory cut for rows of 2 * d_ff bytes
+    size_t ring_bytes, smem_bytes;
 };
 cudaError_t ffn_stream_configure(int n_sms, size_t max_smem, FfnLaunchCfg *cfg);
 cudaError_t ffn_stream_geometry(const FfnLaunchCfg &cfg, int d, int F, int T, FfnGeometry *geo);

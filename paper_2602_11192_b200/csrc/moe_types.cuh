@@ -39,12 +39,14 @@ struct ReqRec {
     int32_t group;     // compute group: 0 = resident at call entry, g >= 1 = g-th miss wave
 };
 
-// A virtual request: up to kTokPerVr tokens of one expert.
-struct VrRec {
-    int32_t req;       // index into DevPlan::req
-    int32_t tok_off;   // first entry in tok_of_sorted
-    int32_t n_tok;     // 1..kTokPerVr
+// A virtual request: up to kTokPerVr tokens of one expert, with everything the FFN kernel
+// needs to serve it in one 80-byte record (one dependent load instead of a chain of them).
+struct __align__(16) VrRec {
+    const char *blob;            // the expert's weights: its cache slot, or a shared expert's blob
+    int32_t n_tok;               // 1..kTokPerVr
     int32_t group;
+    int32_t tok[kTokPerVr];      // token (row of hidden) of each slot, -1 beyond n_tok
+    int32_t pair[kTokPerVr];     // row of the z buffer: t * k + j for routed pairs, T*k + s*T + t for shared
 };
 
 // Per-call plan written by the planning kernel, read by the FFN and combine kernels.

@@ -284,10 +284,15 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p)
             const int nv = (rec.n_tok + kTokPerVr - 1) / kTokPerVr;
             for (int v = tid; v < nv; v += kPlanThreads) {
                 VrRec vr;
-                vr.req = r;
-                vr.tok_off = rec.tok_off + v * kTokPerVr;
+                vr.blob = rec.slot >= 0 ? p.slots + (size_t)rec.slot * p.slot_stride : p.shared_blobs[rec.expert - E];
                 vr.n_tok = min(kTokPerVr, rec.n_tok - v * kTokPerVr);
                 vr.group = rec.group;
+                const int off = rec.tok_off + v * kTokPerVr;
+                for (int i = 0; i < kTokPerVr; ++i) {
+                    const int pos = off + i;
+                    vr.tok[i] = i < vr.n_tok ? p.tok_of_sorted[pos] : -1;
+                    vr.pair[i] = i < vr.n_tok ? (pos < n_pairs ? p.perm[pos] : pos) : -1;
+                }
                 p.vrs[rec.vr_start + v] = vr;
             }
         }
