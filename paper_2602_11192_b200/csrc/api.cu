@@ -317,8 +317,8 @@ int melinoe_moe_create(int d, int F, int E, int k, int C, melinoe_moe_t **out)
     CR(cudaMalloc(&h->cache, sizeof(DevCache)));
     CR(cudaMalloc(&h->plan, sizeof(DevPlan)));
     CR(cudaMalloc(&h->err_word, 256));
-    CR(cudaMalloc(&h->sync, sizeof(unsigned) * (kMaxGroups + 1)));
-    CR(cudaMemset(h->sync, 0, sizeof(unsigned) * (kMaxGroups + 1)));
+    CR(cudaMalloc(&h->sync, sizeof(unsigned) * 2 * (kMaxGroups + 1)));
+    CR(cudaMemset(h->sync, 0, sizeof(unsigned) * 2 * (kMaxGroups + 1)));
     CR(cudaMalloc(&h->shared_dev, sizeof(char *) * kMaxShared));
     CR(cudaMalloc(&h->stage_stats, sizeof(melinoe_moe_stats)));
     CR(cudaMemset(h->err_word, 0, 256));

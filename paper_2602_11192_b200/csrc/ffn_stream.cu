@@ -5,19 +5,20 @@
 // little more than half of it, so the unit of transfer is a whole row (or a 4 KB piece of a
 // longer one).
 //
-// One cooperative launch per compute group, one CTA per SM: one producer warp and eight
+// One cooperative launch per compute group, one CTA per SM: four producer warps and eight
 // consumer warps.  A "virtual request" is one expert with up to 8 of its tokens.
 //
-//   phase 1  tile = 8 rows of W_g plus the same 8 rows of W_u of one virtual request.
+//   phase 1  tile = up to 8 rows of W_g plus the same rows of W_u of one virtual request.
 //            D[16 x 8] = [W_g rows; W_u rows] (16 x d) * x^T (d x 8 tokens) on mma.sync
 //            (bf16 in, fp32 accumulate); the eight warps split the columns of a stage and
 //            their partial sums meet in shared memory once per tile.  In the accumulator
 //            layout a thread holds g_f and u_f of the same f and the same two tokens, so
 //            h = SiLU(g) * u is thread-local; h goes to global memory as bf16.
-//   barrier  grid-wide, crossed by the producer warps only (bounded spin on a device counter):
-//            the consumers never wait for it.  The ring is cut anew for the (usually shorter)
-//            W_d rows as soon as the CTA's own phase 1 has drained, and as many W_d stages as
-//            fit are in flight before the producer reaches the barrier.
+//   barrier  grid-wide, crossed by the producer warps only (bounded polling of a device counter):
+//            the consumers never wait for it.  The requests go through the kernel in two halves,
+//            so each half's barrier latency is covered by the other half's streaming; the ring is
+//            cut anew for the (usually shorter) W_d rows as soon as the CTA's own phase 1 has
+//            drained, and W_d rows run ahead of the barrier as far as the ring allows.
 //   phase 2  every CTA owns a contiguous range of the d_model output rows (d/G of them, so the
 //            split is even to within one row) for ALL virtual requests of the launch.  Tile =
 //            up to 16 of those W_d rows of one virtual request: D[16 x 8] = W_d rows * h^T, a
@@ -31,13 +32,14 @@
 //
 // A stage of the shared-memory ring holds one piece (at most 4 KB) of each of the tile's 16
 // weight rows plus the matching piece of up to 8 operand rows (hidden rows in phase 1, h rows
-// in phase 2), each fetched by its own cp.async.bulk (one producer lane per row) completing on
-// the stage's mbarrier.  Rows sit at a pitch of 16 bytes more than a multiple of 128, which
+// in phase 2), each fetched by its own cp.async.bulk (one producer lane per row; the producer
+// warps share out the ring slots) completing on the stage's mbarrier.  Rows sit at a pitch of 16 bytes more than a multiple of 128, which
 // makes the ldmatrix reads and the operand-fragment reads bank-conflict free.
 //
 // Every wait is bounded: when an mbarrier or the grid barrier does not complete in time the
 // warp raises the CTA's abort flag, later waits fall through, the kernel ends normally and the
 // error word tells the host.
+#include <cstdlib>
 #include "kernels.cuh"
 
 namespace melinoe {
@@ -45,9 +47,11 @@ namespace melinoe {
 namespace {
 
 constexpr int kConsumerWarps = 8;
-constexpr int kThreads = (kConsumerWarps + 1) * 32;
+constexpr int kProducerWarps = 4;                    // a warp needs ~0.6 us to get one stage's copies out
+constexpr int kThreads = (kConsumerWarps + kProducerWarps) * 32;
 constexpr int kMaxStages = 8;
 constexpr int kMaxChunk = 4096;                      // bytes of one row piece
+constexpr int kVrShared = 72;                        // virtual-request records kept in shared memory
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p)
@@ -153,17 +157,11 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t
                  : "memory");
 }
 
-// What the producer needs to know about a tile.
-struct Tile {
-    const char *src;     // this lane's source row (weights: lanes 0..15, operand rows: 16..23)
-    int n_tok;           // tokens of the virtual request
-    int n_rows;          // weight rows in the tile (16 except at the end of a CTA's row range)
-};
-
 __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, FfnGeometry geo)
 {
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ int s_abort;
+    __shared__ VrRec s_vrs[kVrShared];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int d = p.d, F = p.F, Fpad = p.Fpad;
@@ -211,6 +209,16 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    // the launch's virtual-request records: from shared memory when they fit (always in decode),
+    // so that nobody's critical path holds a dependent global load per tile
+    const VrRec *vrs = p.vrs + vb;
+    if (nv <= kVrShared) {
+        const uint4 *src = reinterpret_cast<const uint4 *>(p.vrs + vb);
+        uint4 *dst = reinterpret_cast<uint4 *>(s_vrs);
+        for (int i = tid; i < nv * (int)(sizeof(VrRec) / 16); i += kThreads)
+            dst[i] = src[i];
+        vrs = s_vrs;
+    }
     if (F % 16 != 0) {
         // the last 16-column step of a W_d row is half filled: what the copy leaves untouched
         // must be finite, because it meets the zero padding of the h rows in the product
@@ -223,172 +231,207 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
     if (trace && tid == 0)
         trace[1] = globaltimer_ns();
 
-    // ---- phase 1: a contiguous range of (virtual request, 8-row f-block) tiles per CTA
-    const int upe1 = F / 8;
+    // ---- work of this CTA.  The launch's virtual requests are cut into two halves (one when there
+    // is a single request) that go through the kernel one behind the other:
+    //     gate/up(A)  gate/up(B)  down(A)  down(B)
+    // so that the grid-wide wait for h of half A is covered by the streaming of half B's W_g/W_u
+    // rows, and the wait for half B by half A's W_d rows.
+    // gate/up: rows f of W_g and W_u of the half's requests, numbered request-major, are split
+    // evenly over the CTAs at single-row granularity; a tile is up to 8 consecutive f of one
+    // request (g rows in tile rows 0..7, u rows in 8..15).
+    // down: output rows [r_lo, r_hi) of every request, in tiles of up to 16 rows.
     const int rb1 = 2 * d, rb2 = 2 * F;                       // row bytes
     const int nk1 = (rb1 + CB1 - 1) / CB1, nk2 = (rb2 + CB2 - 1) / CB2;
-    const long long NT1 = (long long)nv * upe1;
-    const int lo1 = (int)(blockIdx.x * NT1 / G), hi1 = (int)((blockIdx.x + 1) * NT1 / G);
-    // ---- phase 2: output rows [r_lo, r_hi) of every virtual request, in tiles of up to 16 rows
+    const int n_half = nv >= 2 ? 2 : 1;
+    const int nvA = n_half == 2 ? nv / 2 : nv;                // requests in half A
+    int q_lo[2], q_hi[2];                                     // f-row ranges, relative to the half's first request
+    {
+        const long long rowsA = (long long)nvA * F, rowsB = (long long)(nv - nvA) * F;
+        q_lo[0] = (int)(blockIdx.x * rowsA / G);
+        q_hi[0] = (int)((blockIdx.x + 1) * rowsA / G);
+        q_lo[1] = (int)(blockIdx.x * rowsB / G);
+        q_hi[1] = (int)((blockIdx.x + 1) * rowsB / G);
+    }
     const int r_lo = (int)((long long)blockIdx.x * d / G), r_hi = (int)((long long)(blockIdx.x + 1) * d / G);
     const int mt = (r_hi - r_lo + 15) / 16;
-    const int hi2 = nv * mt;
+    const int hi2 = nv * mt, hi2A = nvA * mt;                 // down tiles: request-major, half A first
+    unsigned *sync_word = p.sync + 2 * p.group;               // [half]
 
-    if (warp == kConsumerWarps) {
-        // =================================================================== producer
-        // Per virtual request (looked up only when the tile sequence moves on to the next one):
-        // this lane's source row of block 0 and its stride from one block to the next.
-        int cur_vr = -1, cur_ntok = 0;
-        const char *lane_base = nullptr;
-        size_t lane_step = 0;
-        // phase 1: lanes 0..7 W_g rows, 8..15 W_u rows, 16..23 hidden rows of the request's tokens
-        auto tile1 = [&](int t) -> Tile {
-            const int vr = vb + t / upe1, blk = t % upe1;
-            if (vr != cur_vr) {
-                const VrRec *v = p.vrs + vr;
-                cur_vr = vr;
-                cur_ntok = v->n_tok;
-                lane_base = nullptr;
-                lane_step = 0;
-                if (lane < 16) {
-                    lane_base = v->blob + (size_t)((lane < 8 ? 0 : F) + (lane & 7)) * rb1;
-                    lane_step = (size_t)8 * rb1;
-                } else if (lane - 16 < cur_ntok) {
-                    lane_base = reinterpret_cast<const char *>(p.x) + (size_t)v->tok[lane - 16] * rb1;
-                }
-            }
-            Tile ti;
-            ti.n_tok = cur_ntok;
-            ti.n_rows = 16;
-            ti.src = lane_base ? lane_base + (size_t)blk * lane_step : nullptr;
-            return ti;
-        };
-        // phase 2: lanes 0..15 W_d rows, 16..23 rows of h
-        auto tile2 = [&](int t) -> Tile {
-            const int vr = vb + t / mt, blk = t % mt;
-            if (vr != cur_vr) {
-                const VrRec *v = p.vrs + vr;
-                cur_vr = vr;
-                cur_ntok = v->n_tok;
-                lane_base = nullptr;
-                lane_step = 0;
-                if (lane < 16) {
-                    lane_base = v->blob + (size_t)2 * F * rb1 + (size_t)(r_lo + lane) * rb2;
-                    lane_step = (size_t)16 * rb2;
-                } else if (lane - 16 < cur_ntok) {
-                    lane_base = reinterpret_cast<const char *>(p.hbuf) + ((size_t)vr * kTokPerVr + lane - 16) * Fpad * 2;
-                }
-            }
-            Tile ti;
-            ti.n_tok = cur_ntok;
-            ti.n_rows = min(16, r_hi - r_lo - 16 * blk);
-            ti.src = lane_base ? lane_base + (size_t)blk * lane_step : nullptr;
-            if (lane < 16 && lane >= ti.n_rows)
-                ti.src = nullptr;
-            return ti;
-        };
+    if (warp >= kConsumerWarps) {
+        // =================================================================== producers
+        // The producer warps walk the same stage sequence and share the stages out (a warp is busy
+        // for ~0.6 us with one bulk-copy instruction, however few lanes take part, so the stages
+        // of a 28 KB-per-stage phase would otherwise leave faster than one warp can issue them).
+        // A ring slot always belongs to the same warp (slot s to warp s mod 4), so every wait on a
+        // slot's "empty" barrier is made by the one warp that has followed all its earlier phases.
+        // Lanes 0..15 fetch the tile's weight rows, lanes 16..23 the operand rows.
+        const int pw = warp - kConsumerWarps;
+        const bool is_w = lane < 16;
+        const int my_row = is_w ? lane : lane - 16;                        // tile row, or token slot
+        const int dst_row = lane;
+        const bool lane_used = lane < 24;
         bool dead = false;
-        // One stage of either phase.  parts bit 0: wait for the slot, arm the barrier, fetch the
-        // weight rows; bit 1: operand rows.  wbytes / obytes: bytes of each weight / operand piece.
-        auto issue = [&](const Tile &ti, uint32_t full0, uint32_t empty0, int S, int STAGE, int PITCH, size_t src_off,
-                         int wbytes, int obytes, int parts, uint32_t nn) {
+        // One stage of either phase.  src: this lane's source row or null.  parts bit 0: arm the
+        // barrier and fetch the weight rows (the caller has made sure the slot is free); bit 1:
+        // operand rows.
+        auto issue = [&](const char *src, uint32_t full0, int S, int STAGE, int PITCH, size_t src_off, int wbytes,
+                         int obytes, int parts, uint32_t nn) {
             const uint32_t slot = nn % S;
             const uint32_t bar = full0 + 8 * slot;
+            const bool active = lane_used && src != nullptr;
             if (parts & 1) {
-                if (nn >= (uint32_t)S && !dead)
-                    dead = !mbar_wait(empty0 + 8 * slot, ((nn / S) - 1u) & 1u, abort_flag);
+                const unsigned mw = __ballot_sync(0xffffffffu, active && is_w);
+                const unsigned mo = __ballot_sync(0xffffffffu, active && !is_w);
                 if (lane == 0)
-                    mbar_expect(bar, (uint32_t)ti.n_rows * wbytes + (uint32_t)ti.n_tok * obytes);
+                    mbar_expect(bar, (uint32_t)__popc(mw) * wbytes + (uint32_t)__popc(mo) * obytes);
                 __syncwarp();
             }
-            if (ti.src && !dead) {
-                const bool is_w = lane < 16;
-                if (is_w ? (parts & 1) : (parts & 2))
-                    bulk_g2s(ring_s + slot * STAGE + lane * PITCH, ti.src + src_off,
-                             (uint32_t)(is_w ? wbytes : obytes), bar);
-            }
+            if (active && !dead && (is_w ? (parts & 1) : (parts & 2)))
+                bulk_g2s(ring_s + slot * STAGE + dst_row * PITCH, src + src_off, (uint32_t)(is_w ? wbytes : obytes), bar);
         };
+        // ---- gate/up: lanes 0..7 W_g rows, 8..15 W_u rows, 16..23 hidden rows of the request's tokens
         uint32_t n1 = 0;
-        for (int t = lo1; t < hi1; ++t) {
-            const Tile ti = tile1(t);
-            for (int kc = 0; kc < nk1; ++kc) {
-                const int b = min(CB1, rb1 - kc * CB1);
-                issue(ti, full1, empty1, S1, STAGE1, PITCH1, (size_t)kc * CB1, b, b, 3, n1++);
-            }
-        }
-        // the ring is cut anew for phase 2: wait until the consumers have let go of every phase-1 stage
-        for (uint32_t m = n1 > (uint32_t)S1 ? n1 - S1 : 0u; m < n1 && !dead; ++m)
-            dead = !mbar_wait(empty1 + 8 * (m % S1), (m / S1) & 1u, abort_flag);
-        // phase 2: the first stages go out with their weight rows only; h is not complete yet
-        cur_vr = -1;
-        uint32_t n2 = 0;
-        int t2 = 0, k2 = 0;
-        Tile ti2{};
-        if (t2 < hi2)
-            ti2 = tile2(t2);
-        auto w_bytes2 = [&](int kc) { return min(CB2, rb2 - kc * CB2); };
-        auto op_bytes2 = [&](int kc) { return min(CB2, Fpad * 2 - kc * CB2); };
-        int pre = 0;
-        for (; pre < S2 && t2 < hi2; ++pre) {
-            issue(ti2, full2, empty2, S2, STAGE2, PITCH2, (size_t)k2 * CB2, w_bytes2(k2), op_bytes2(k2), 1, n2++);
-            if (++k2 == nk2) {
-                k2 = 0;
-                if (++t2 < hi2)
-                    ti2 = tile2(t2);
-            }
-        }
-        // grid barrier: every CTA's consumers have written their part of h
-        if (lane == 0) {
-            const unsigned target = (unsigned)G;
-            volatile unsigned *w = p.sync + p.group;
-            if (*w < target && !*abort_flag) {
-                const unsigned long long t0 = globaltimer_ns();
-                while (*w < target) {
-                    if (*abort_flag || globaltimer_ns() - t0 > kWaitLimitNs) {
-                        *abort_flag = 1;
-                        break;
+        for (int half = 0; half < n_half; ++half) {
+            const int v0 = vb + (half ? nvA : 0);
+            int q = q_lo[half];
+            while (q < q_hi[half]) {
+                const int vr = v0 + q / F, f0 = q % F;
+                const int m = min(min(8, F - f0), q_hi[half] - q);
+                const VrRec *v = vrs + (vr - vb);
+                const char *src = nullptr;
+                if (lane_used) {
+                    if (is_w) {
+                        if ((my_row & 7) < m)
+                            src = v->blob + (size_t)((my_row < 8 ? 0 : F) + f0 + (my_row & 7)) * rb1;
+                    } else if (my_row < v->n_tok) {
+                        src = reinterpret_cast<const char *>(p.x) + (size_t)v->tok[my_row] * rb1;
                     }
                 }
+                for (int kc = 0; kc < nk1; ++kc, ++n1) {
+                    if ((int)((n1 % S1) % kProducerWarps) != pw)
+                        continue;
+                    if (n1 >= (uint32_t)S1 && !dead)
+                        dead = !mbar_wait(empty1 + 8 * (n1 % S1), ((n1 / S1) - 1u) & 1u, abort_flag);
+                    const int b = min(CB1, rb1 - kc * CB1);
+                    issue(src, full1, S1, STAGE1, PITCH1, (size_t)kc * CB1, b, b, 3, n1);
+                }
+                q += m;
             }
-            __threadfence();
-            if (trace)
-                trace[5] = globaltimer_ns();
         }
-        __syncwarp();
-        fence_proxy_async();
-        {
-            // the operand rows of the stages already under way: replay the tile sequence from the
-            // start of phase 2 with a cache of its own, then restore the main sequence's cache
-            const int keep_vr = cur_vr, keep_ntok = cur_ntok;
-            const char *keep_base = lane_base;
-            const size_t keep_step = lane_step;
-            cur_vr = -1;
-            int qt = 0, qk = 0;
-            Tile qtile{};
-            if (pre > 0)
-                qtile = tile2(0);
-            for (int i = 0; i < pre; ++i) {
-                issue(qtile, full2, empty2, S2, STAGE2, PITCH2, (size_t)qk * CB2, 0, op_bytes2(qk), 2, (uint32_t)i);
-                if (++qk == nk2) {
-                    qk = 0;
-                    if (++qt < hi2)
-                        qtile = tile2(qt);
+        // the ring is cut anew for the down phase: wait until the consumers have let go of every
+        // gate/up stage
+        // (each warp for the slots it owns, then the producer warps meet)
+        for (uint32_t m = n1 > (uint32_t)S1 ? n1 - S1 : 0u; m < n1 && !dead; ++m)
+            if ((int)((m % S1) % kProducerWarps) == pw)
+                dead = !mbar_wait(empty1 + 8 * (m % S1), (m / S1) & 1u, abort_flag);
+        asm volatile("bar.sync 2, %0;" ::"n"(kProducerWarps * 32) : "memory");
+
+        // ---- down: lanes 0..15 W_d rows, 16..23 rows of h.  Two cursors walk the same stage
+        // sequence: the weight rows run ahead as far as the ring allows, the h rows of a stage
+        // follow once the grid has finished the h of the stage's half.
+        struct Cursor {
+            int t, k, vr;
+            const char *base;
+        };
+        auto tile_of = [&](Cursor &c) -> const char * {
+            const int vr = vb + c.t / mt, blk = c.t % mt;
+            if (vr != c.vr) {
+                const VrRec *v = vrs + (vr - vb);
+                c.vr = vr;
+                c.base = nullptr;
+                if (lane_used) {
+                    if (is_w)
+                        c.base = v->blob + (size_t)2 * F * rb1 + (size_t)(r_lo + my_row) * rb2;
+                    else if (my_row < v->n_tok)
+                        c.base = reinterpret_cast<const char *>(p.hbuf) + ((size_t)vr * kTokPerVr + my_row) * Fpad * 2;
                 }
             }
-            cur_vr = keep_vr;
-            cur_ntok = keep_ntok;
-            lane_base = keep_base;
-            lane_step = keep_step;
-        }
-        while (t2 < hi2) {
-            issue(ti2, full2, empty2, S2, STAGE2, PITCH2, (size_t)k2 * CB2, w_bytes2(k2), op_bytes2(k2), 3, n2++);
-            if (++k2 == nk2) {
-                k2 = 0;
-                if (++t2 < hi2)
-                    ti2 = tile2(t2);
+            if (!is_w)
+                return c.base;
+            return (c.base && r_lo + 16 * blk + my_row < r_hi) ? c.base + (size_t)blk * 16 * rb2 : nullptr;
+        };
+        auto advance = [&](Cursor &c) {
+            if (++c.k == nk2) {
+                c.k = 0;
+                ++c.t;
+            }
+        };
+        auto w_bytes2 = [&](int kc) { return min(CB2, rb2 - kc * CB2); };
+        auto op_bytes2 = [&](int kc) { return min(CB2, Fpad * 2 - kc * CB2); };
+        const uint32_t N2 = (uint32_t)hi2 * nk2;
+        Cursor wc{0, 0, -1, nullptr}, oc{0, 0, -1, nullptr};
+        uint32_t wn = 0, on = 0;
+        bool passed[2] = {false, false};
+        unsigned long long t_idle = 0;
+        while (on < N2 && !dead) {
+            bool progress = false;
+            // weight rows of as many stages as there are free slots
+            while (wn < N2) {
+                if ((int)((wn % S2) % kProducerWarps) != pw) {
+                    (void)tile_of(wc);
+                    advance(wc);
+                    ++wn;
+                    progress = true;
+                    continue;
+                }
+                if (wn >= (uint32_t)S2) {
+                    int ok = 0;
+                    if (lane == 0)
+                        ok = mbar_try(empty2 + 8 * (wn % S2), ((wn / S2) - 1u) & 1u);
+                    if (!__shfl_sync(0xffffffffu, ok, 0))
+                        break;
+                }
+                const char *src = tile_of(wc);
+                issue(src, full2, S2, STAGE2, PITCH2, (size_t)wc.k * CB2, w_bytes2(wc.k), op_bytes2(wc.k), 1, wn);
+                advance(wc);
+                ++wn;
+                progress = true;
+            }
+            // h rows of the next stages, once their half of h is complete everywhere
+            if (on < wn) {
+                const int half = oc.t < hi2A ? 0 : 1;
+                if (!passed[half]) {
+                    int ok = 0;
+                    if (lane == 0) {
+                        ok = *reinterpret_cast<volatile unsigned *>(sync_word + half) >= (unsigned)G;
+                        if (ok) {
+                            __threadfence();
+                            if (trace && pw == 0)
+                                trace[5] = globaltimer_ns();
+                        }
+                    }
+                    passed[half] = __shfl_sync(0xffffffffu, ok, 0) != 0;
+                }
+                while (on < wn && passed[oc.t < hi2A ? 0 : 1]) {
+                    const char *src = tile_of(oc);
+                    if ((int)((on % S2) % kProducerWarps) != pw) {
+                        advance(oc);
+                        ++on;
+                        progress = true;
+                        continue;
+                    }
+                    issue(src, full2, S2, STAGE2, PITCH2, (size_t)oc.k * CB2, 0, op_bytes2(oc.k), 2, on);
+                    advance(oc);
+                    ++on;
+                    progress = true;
+                }
+            }
+            if (progress) {
+                t_idle = 0;
+            } else {
+                const unsigned long long now = globaltimer_ns();
+                if (t_idle == 0)
+                    t_idle = now;
+                int give_up = (now - t_idle > kWaitLimitNs) || *abort_flag;
+                give_up = __shfl_sync(0xffffffffu, give_up, 0);
+                if (give_up) {
+                    *abort_flag = 1;
+                    dead = true;
+                }
             }
         }
-        if (*abort_flag && lane == 0) {
+        const uint32_t n2 = on;
+        if (*abort_flag && lane == 0 && pw == 0) {
             // a wait ran out: give the copies still in flight a bounded time to land before this
             // CTA's shared memory goes away
             const unsigned long long t0 = globaltimer_ns();
@@ -408,16 +451,17 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
     int n_tiles = 0;       // tiles finished so far (selects the reduction buffer and the epilogue warp)
     float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
 
-    // this warp's share of one stage: some of the 16-column steps of the piece
+    // this warp's share of one stage: some of the 16-column steps of the piece.  Weights in tile
+    // rows 0..15, the operand rows (hidden or h) of the request's tokens behind them.
     auto compute = [&](uint32_t full0, uint32_t empty0, int S, int STAGE, uint32_t a_off, uint32_t b_off, uint32_t n,
                        int bytes, int n_tok) {
         const uint32_t slot = n % S;
         mbar_wait(full0 + 8 * slot, (n / S) & 1u, abort_flag);
         const uint32_t base = ring_s + slot * STAGE;
         const int ks_total = (bytes + 31) >> 5;
-        const int ks_lo = warp * ks_total / kConsumerWarps, ks_hi = (warp + 1) * ks_total / kConsumerWarps;
+        const int ks_hi = (warp + 1) * ks_total / kConsumerWarps;
+        int ks = warp * ks_total / kConsumerWarps;
         const bool has_tok = g < n_tok;
-        int ks = ks_lo;
         for (; ks + 1 < ks_hi; ks += 2) {
             uint32_t a0, a1, a2, a3, e0, e1, e2, e3;
             ldmatrix_x4(base + a_off + ks * 32, a0, a1, a2, a3);
@@ -476,7 +520,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
         int n_tok, pair0, pair1;
     };
     auto load_vr = [&](int vr) -> VrInfo {
-        const VrRec *v = p.vrs + vr;
+        const VrRec *v = vrs + (vr - vb);
         VrInfo r;
         r.n_tok = v->n_tok;
         const int2 pr = *reinterpret_cast<const int2 *>(v->pair + tig * 2);
@@ -485,68 +529,81 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
         return r;
     };
 
-    // ---- phase 1: h = SiLU(W_g x) * (W_u x)
+    // ---- gate/up: h = SiLU(W_g x) * (W_u x), half by half
     {
         const uint32_t a_off = ((lane & 7) + ((lane >> 3) & 1) * 8) * PITCH1 + (lane >> 4) * 16;
         const uint32_t b_off = (16 + g) * PITCH1 + tig * 4;
         uint32_t n = 0;
-        int cur_vr = -1;
-        VrInfo v{};
-        for (int t = lo1; t < hi1; ++t) {
-            const int vr = vb + t / upe1, blk = t % upe1;
-            if (vr != cur_vr) {
-                v = load_vr(vr);
-                cur_vr = vr;
+        for (int half = 0; half < n_half; ++half) {
+            const int v0 = vb + (half ? nvA : 0);
+            int cur_vr = -1;
+            VrInfo v{};
+            int q = q_lo[half];
+            while (q < q_hi[half]) {
+                const int vr = v0 + q / F, f0 = q % F;
+                const int m = min(min(8, F - f0), q_hi[half] - q);
+                if (vr != cur_vr) {
+                    v = load_vr(vr);
+                    cur_vr = vr;
+                }
+                for (int kc = 0; kc < nk1; ++kc) {
+                    compute(full1, empty1, S1, STAGE1, a_off, b_off, n, min(CB1, rb1 - kc * CB1), v.n_tok);
+                    if (trace && n == 0 && tid == 0)
+                        trace[2] = globaltimer_ns();
+                    ++n;
+                }
+                float r[4];
+                if (reduce_tile(r) && g < m) {
+                    // rows g and g + 8 of the tile are g_f and u_f for f = f0 + g
+                    uint16_t *hrow = p.hbuf + ((size_t)vr * kTokPerVr) * Fpad + f0 + g;
+                    if (tig * 2 < v.n_tok)
+                        hrow[(size_t)(tig * 2) * Fpad] = bf16_rne(r[0] / (1.0f + __expf(-r[0])) * r[2]);
+                    if (tig * 2 + 1 < v.n_tok)
+                        hrow[(size_t)(tig * 2 + 1) * Fpad] = bf16_rne(r[1] / (1.0f + __expf(-r[1])) * r[3]);
+                }
+                q += m;
             }
-            for (int kc = 0; kc < nk1; ++kc) {
-                compute(full1, empty1, S1, STAGE1, a_off, b_off, n, min(CB1, rb1 - kc * CB1), v.n_tok);
-                if (trace && n == 0 && tid == 0)
-                    trace[2] = globaltimer_ns();
-                ++n;
-            }
-            float r[4];
-            if (reduce_tile(r)) {
-                // rows g and g + 8 of the tile are g_f and u_f for f = 8 * blk + g
-                uint16_t *hrow = p.hbuf + ((size_t)vr * kTokPerVr) * Fpad + blk * 8 + g;
-                if (tig * 2 < v.n_tok)
-                    hrow[(size_t)(tig * 2) * Fpad] = bf16_rne(r[0] / (1.0f + __expf(-r[0])) * r[2]);
-                if (tig * 2 + 1 < v.n_tok)
-                    hrow[(size_t)(tig * 2 + 1) * Fpad] = bf16_rne(r[1] / (1.0f + __expf(-r[1])) * r[3]);
+            if (trace && tid == 0 && half == n_half - 1)
+                trace[3] = globaltimer_ns();
+            // this CTA's part of the half's h is complete: tell the grid
+            __threadfence();
+            fence_proxy_async();       // h was written through the generic proxy, bulk copies will read it
+            consumer_bar();
+            if (tid == 0) {
+                atomicAdd(sync_word + half, 1u);
+                if (trace && half == n_half - 1)
+                    trace[4] = globaltimer_ns();
             }
         }
     }
-    if (trace && tid == 0)
-        trace[3] = globaltimer_ns();
-    // this CTA's part of h is complete: tell the grid
-    __threadfence();
-    fence_proxy_async();       // h was written through the generic proxy, bulk copies will read it
-    consumer_bar();
-    if (tid == 0) {
-        atomicAdd(p.sync + p.group, 1u);
-        if (trace)
-            trace[4] = globaltimer_ns();
-    }
 
-    // ---- phase 2: z = W_d h for this CTA's output rows
+    // ---- down: z = W_d h for this CTA's output rows
     {
         const uint32_t a_off = ((lane & 7) + ((lane >> 3) & 1) * 8) * PITCH2 + (lane >> 4) * 16;
         const uint32_t b_off = (16 + g) * PITCH2 + tig * 4;
         uint32_t n = 0;
-        VrInfo v{}, nxt{};
-        if (hi2 > 0)
+        // the requests' records are read two requests ahead of their use
+        VrInfo v{}, nxt{}, nxt2{};
+        if (hi2 > 0) {
             nxt = load_vr(vb);
+            nxt2 = nv > 1 ? load_vr(vb + 1) : nxt;
+        }
         for (int t = 0; t < hi2; ++t) {
-            const int blk = t % mt, r0 = r_lo + 16 * blk;
+            const int blk = t % mt, iv = t / mt;
             if (blk == 0) {
                 v = nxt;
-                if (t + mt < hi2)
-                    nxt = load_vr(vb + t / mt + 1);   // in flight while this request's tiles are computed
+                nxt = nxt2;
+                if (iv + 2 < nv)
+                    nxt2 = load_vr(vb + iv + 2);
             }
-            for (int kc = 0; kc < nk2; ++kc, ++n)
+            for (int kc = 0; kc < nk2; ++kc, ++n) {
                 compute(full2, empty2, S2, STAGE2, a_off, b_off, n, min(CB2, rb2 - kc * CB2), v.n_tok);
+                if (trace && n == 0 && tid == 0)
+                    trace[2] = globaltimer_ns();
+            }
             float r[4];
             if (reduce_tile(r)) {
-                const int row = r0 + g;
+                const int row = r_lo + 16 * blk + g;
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
                     if (tig * 2 + h < v.n_tok) {
@@ -588,7 +645,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
 
 cudaError_t ffn_stream_configure(int n_sms, size_t max_smem, FfnLaunchCfg *cfg)
 {
-    const size_t usable = max_smem - 1024;   // room for the kernel's static shared memory
+    const size_t usable = max_smem - 8192;   // room for the kernel's static shared memory
     cudaError_t e = cudaFuncSetAttribute(ffn_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)usable);
     if (e != cudaSuccess)
         return e;
@@ -629,6 +686,8 @@ cudaError_t ffn_stream_geometry(const FfnLaunchCfg &cfg, int d, int F, int T, Ff
         s1 = kMaxStages;
     if (s2 > (size_t)kMaxStages)
         s2 = kMaxStages;
+    if (const char *e = getenv("MELINOE_DBG_S1")) { size_t v = atoi(e); if (v >= 1 && v < s1) s1 = v; }
+    if (const char *e = getenv("MELINOE_DBG_S2")) { size_t v = atoi(e); if (v >= 1 && v < s2) s2 = v; }
     geo->n_stages = (int)s1;
     geo->n_stages2 = (int)s2;
     size_t ring = s1 * stage1 > s2 * stage2 ? s1 * stage1 : s2 * stage2;
