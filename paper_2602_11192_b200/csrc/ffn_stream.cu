@@ -16,9 +16,10 @@
 //            h = SiLU(g) * u is thread-local; h goes to global memory as bf16.
 //   barrier  grid-wide, crossed by the producer warps only (bounded polling of a device counter):
 //            the consumers never wait for it.  The requests go through the kernel in two halves,
-//            so each half's barrier latency is covered by the other half's streaming; the ring is
-//            cut anew for the (usually shorter) W_d rows as soon as the CTA's own phase 1 has
-//            drained, and W_d rows run ahead of the barrier as far as the ring allows.
+//            so each half's barrier latency is covered by the other half's streaming.  Both
+//            phases run through one ring and one stage sequence, so the first W_d rows are
+//            requested the moment a slot comes free, before the CTA has finished phase 1, and run
+//            ahead of the barrier as far as the ring allows; only the h rows wait for it.
 //   phase 2  every CTA owns a contiguous range of the d_model output rows (d/G of them, so the
 //            split is even to within one row) for ALL virtual requests of the launch.  Tile =
 //            up to 16 of those W_d rows of one virtual request: D[16 x 8] = W_d rows * h^T, a
@@ -52,7 +53,10 @@ constexpr int kThreads = (kConsumerWarps + kProducerWarps) * 32;
 constexpr int kMaxStages = 8;
 constexpr int kMaxChunk = 4096;                      // bytes of one row piece
 constexpr int kVrShared = 72;                        // virtual-request records kept in shared memory
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+// Bound of every wait, in SM clock cycles (about 2 s).  Waits are timed with the SM's cycle
+// counter: reading the device-wide nanosecond timer costs about 0.6 us each time, which would
+// quantise every wait that does not succeed at once.
+constexpr long long kWaitLimitCycles = 4000000000ll;
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p)
 {
@@ -86,14 +90,14 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         return true;
     if (*abort_flag)
         return false;
-    const unsigned long long t0 = globaltimer_ns();
+    const long long t0 = clock64();
     for (;;) {
         for (int i = 0; i < 64; ++i)
             if (mbar_try(bar, parity))
                 return true;
         if (*abort_flag)
             return false;
-        if (globaltimer_ns() - t0 > kWaitLimitNs) {
+        if (clock64() - t0 > kWaitLimitCycles) {
             *abort_flag = 1;
             return false;
         }
@@ -168,8 +172,9 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
     const DevPlan *plan = p.plan;
     const int G = (int)gridDim.x;
     const int NOP = geo.n_op_rows;
-    const int S1 = geo.n_stages, PITCH1 = geo.pitch, CB1 = geo.chunk_bytes, STAGE1 = (16 + NOP) * PITCH1;
-    const int S2 = geo.n_stages2, PITCH2 = geo.pitch2, CB2 = geo.chunk_bytes2, STAGE2 = (16 + NOP) * PITCH2;
+    (void)NOP;
+    const int S1 = geo.n_stages, PITCH1 = geo.pitch, CB1 = geo.chunk_bytes, STAGE1 = geo.stage_bytes;
+    const int S2 = S1, PITCH2 = geo.pitch2, CB2 = geo.chunk_bytes2, STAGE2 = STAGE1;
 
     // optional timeline: 8 device-clock stamps per CTA (see melinoe_moe_set_trace)
     unsigned long long *trace = p.trace ? p.trace + (size_t)blockIdx.x * 8 : nullptr;
@@ -196,7 +201,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
     uint64_t *bars = reinterpret_cast<uint64_t *>(red + 2 * kConsumerWarps * 128);
     const uint32_t ring_s = smem_u32(ring);
     const uint32_t full1 = smem_u32(bars), empty1 = full1 + 8 * kMaxStages;
-    const uint32_t full2 = empty1 + 8 * kMaxStages, empty2 = full2 + 8 * kMaxStages;
+    const uint32_t full2 = full1, empty2 = empty1;          // one ring, one stage sequence for both phases
     volatile int *abort_flag = &s_abort;
 
     if (tid == 0) {
@@ -204,8 +209,6 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
         for (int i = 0; i < kMaxStages; ++i) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(full1 + 8 * i), "r"(1));
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(empty1 + 8 * i), "r"(kConsumerWarps));
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(full2 + 8 * i), "r"(1));
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(empty2 + 8 * i), "r"(kConsumerWarps));
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -318,14 +321,6 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
                 q += m;
             }
         }
-        // the ring is cut anew for the down phase: wait until the consumers have let go of every
-        // gate/up stage
-        // (each warp for the slots it owns, then the producer warps meet)
-        for (uint32_t m = n1 > (uint32_t)S1 ? n1 - S1 : 0u; m < n1 && !dead; ++m)
-            if ((int)((m % S1) % kProducerWarps) == pw)
-                dead = !mbar_wait(empty1 + 8 * (m % S1), (m / S1) & 1u, abort_flag);
-        asm volatile("bar.sync 2, %0;" ::"n"(kProducerWarps * 32) : "memory");
-
         // ---- down: lanes 0..15 W_d rows, 16..23 rows of h.  Two cursors walk the same stage
         // sequence: the weight rows run ahead as far as the ring allows, the h rows of a stage
         // follow once the grid has finished the h of the stage's half.
@@ -358,11 +353,12 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
         };
         auto w_bytes2 = [&](int kc) { return min(CB2, rb2 - kc * CB2); };
         auto op_bytes2 = [&](int kc) { return min(CB2, Fpad * 2 - kc * CB2); };
-        const uint32_t N2 = (uint32_t)hi2 * nk2;
+        // the down stages follow the gate/up stages in the same ring: stage numbers run on from n1
+        const uint32_t N2 = n1 + (uint32_t)hi2 * nk2;
         Cursor wc{0, 0, -1, nullptr}, oc{0, 0, -1, nullptr};
-        uint32_t wn = 0, on = 0;
+        uint32_t wn = n1, on = n1;
         bool passed[2] = {false, false};
-        unsigned long long t_idle = 0;
+        long long t_idle = 0;
         while (on < N2 && !dead) {
             bool progress = false;
             // weight rows of as many stages as there are free slots
@@ -419,10 +415,10 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
             if (progress) {
                 t_idle = 0;
             } else {
-                const unsigned long long now = globaltimer_ns();
+                const long long now = clock64();
                 if (t_idle == 0)
                     t_idle = now;
-                int give_up = (now - t_idle > kWaitLimitNs) || *abort_flag;
+                int give_up = (now - t_idle > kWaitLimitCycles) || *abort_flag;
                 give_up = __shfl_sync(0xffffffffu, give_up, 0);
                 if (give_up) {
                     *abort_flag = 1;
@@ -434,12 +430,9 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
         if (*abort_flag && lane == 0 && pw == 0) {
             // a wait ran out: give the copies still in flight a bounded time to land before this
             // CTA's shared memory goes away
-            const unsigned long long t0 = globaltimer_ns();
-            for (uint32_t m = n1 > (uint32_t)S1 ? n1 - S1 : 0u; m < n1; ++m)
-                while (!mbar_try(full1 + 8 * (m % S1), (m / S1) & 1u) && globaltimer_ns() - t0 < kWaitLimitNs) {
-                }
+            const long long t0 = clock64();
             for (uint32_t m = n2 > (uint32_t)S2 ? n2 - S2 : 0u; m < n2; ++m)
-                while (!mbar_try(full2 + 8 * (m % S2), (m / S2) & 1u) && globaltimer_ns() - t0 < kWaitLimitNs) {
+                while (!mbar_try(full2 + 8 * (m % S2), (m / S2) & 1u) && clock64() - t0 < kWaitLimitCycles) {
                 }
             atomicExch(p.err, MELINOE_ERR_TIMEOUT);
         }
@@ -529,11 +522,11 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
         return r;
     };
 
+    uint32_t n = 0;        // stages consumed so far, over both phases
     // ---- gate/up: h = SiLU(W_g x) * (W_u x), half by half
     {
         const uint32_t a_off = ((lane & 7) + ((lane >> 3) & 1) * 8) * PITCH1 + (lane >> 4) * 16;
         const uint32_t b_off = (16 + g) * PITCH1 + tig * 4;
-        uint32_t n = 0;
         for (int half = 0; half < n_half; ++half) {
             const int v0 = vb + (half ? nvA : 0);
             int cur_vr = -1;
@@ -581,7 +574,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
     {
         const uint32_t a_off = ((lane & 7) + ((lane >> 3) & 1) * 8) * PITCH2 + (lane >> 4) * 16;
         const uint32_t b_off = (16 + g) * PITCH2 + tig * 4;
-        uint32_t n = 0;
+        const uint32_t n_first = n;
         // the requests' records are read two requests ahead of their use
         VrInfo v{}, nxt{}, nxt2{};
         if (hi2 > 0) {
@@ -598,7 +591,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
             }
             for (int kc = 0; kc < nk2; ++kc, ++n) {
                 compute(full2, empty2, S2, STAGE2, a_off, b_off, n, min(CB2, rb2 - kc * CB2), v.n_tok);
-                if (trace && n == 0 && tid == 0)
+                if (trace && n == n_first && tid == 0)
                     trace[2] = globaltimer_ns();
             }
             float r[4];
@@ -660,9 +653,9 @@ cudaError_t ffn_stream_configure(int n_sms, size_t max_smem, FfnLaunchCfg *cfg)
     return cudaSuccess;
 }
 
-// Ring geometry for a call of T tokens on a d x F layer: the same shared memory is cut into
-// stages of (16 + operand rows) row pieces twice, once for rows of 2*d bytes (gate/up phase)
-// and once for rows of 2*F bytes (down phase).
+// Ring geometry for a call of T tokens on a d x F layer: stages of (16 + operand rows) row
+// pieces, sized for the longer of the two phases' pieces; each phase lays its rows out at its
+// own pitch inside a stage.
 cudaError_t ffn_stream_geometry(const FfnLaunchCfg &cfg, int d, int F, int T, FfnGeometry *geo)
 {
     auto chunk_of = [](int row_bytes) {
@@ -675,25 +668,18 @@ cudaError_t ffn_stream_geometry(const FfnLaunchCfg &cfg, int d, int F, int T, Ff
     geo->chunk_bytes2 = chunk_of(2 * F);
     geo->pitch2 = geo->chunk_bytes2 + 16;
     const size_t rows = 16 + geo->n_op_rows;
-    const size_t stage1 = rows * geo->pitch, stage2 = rows * geo->pitch2;
-    const size_t fixed = 2 * kConsumerWarps * 128 * sizeof(float) + 4 * kMaxStages * 8 + 128;
-    const size_t big = stage1 > stage2 ? stage1 : stage2;
-    if (cfg.max_smem < fixed + 2 * big)
+    const size_t stage = rows * (geo->pitch > geo->pitch2 ? geo->pitch : geo->pitch2);
+    const size_t fixed = 2 * kConsumerWarps * 128 * sizeof(float) + 2 * kMaxStages * 8 + 128;
+    if (cfg.max_smem < fixed + 2 * stage)
         return cudaErrorInvalidConfiguration;
     const size_t avail = (cfg.max_smem - fixed) / 128 * 128;
-    size_t s1 = avail / stage1, s2 = avail / stage2;
-    if (s1 > (size_t)kMaxStages)
-        s1 = kMaxStages;
-    if (s2 > (size_t)kMaxStages)
-        s2 = kMaxStages;
-    if (const char *e = getenv("MELINOE_DBG_S1")) { size_t v = atoi(e); if (v >= 1 && v < s1) s1 = v; }
-    if (const char *e = getenv("MELINOE_DBG_S2")) { size_t v = atoi(e); if (v >= 1 && v < s2) s2 = v; }
-    geo->n_stages = (int)s1;
-    geo->n_stages2 = (int)s2;
-    size_t ring = s1 * stage1 > s2 * stage2 ? s1 * stage1 : s2 * stage2;
-    ring = (ring + 127) / 128 * 128;
-    geo->ring_bytes = ring;
-    geo->smem_bytes = ring + fixed;
+    size_t n = avail / stage;
+    if (n > (size_t)kMaxStages)
+        n = kMaxStages;
+    geo->n_stages = (int)n;
+    geo->stage_bytes = (int)stage;
+    geo->ring_bytes = (n * stage + 127) / 128 * 128;
+    geo->smem_bytes = geo->ring_bytes + fixed;
     return cudaSuccess;
 }
 

@@ -58,8 +58,9 @@ struct FfnLaunchCfg {
 // Shape of the shared-memory ring for one call.
 struct FfnGeometry {
     int n_op_rows;                   // operand rows per stage: min(T, 8)
-    int n_stages, pitch, chunk_bytes;        // gate/up phase: the ring as n_stages stages of (16 + n_op_rows) rows
-    int n_stages2, pitch2, chunk_bytes2;     // down phase: the same memory cut for rows of 2 * d_ff bytes
+    int n_stages, stage_bytes;       // the ring
+    int pitch, chunk_bytes;          // gate/up phase: row pitch in a stage, bytes per row piece (rows of 2*d bytes)
+    int pitch2, chunk_bytes2;        // down phase (rows of 2*d_ff bytes)
     size_t ring_bytes, smem_bytes;
 };
 cudaError_t ffn_stream_configure(int n_sms, size_t max_smem, FfnLaunchCfg *cfg);
