@@ -69,7 +69,7 @@ typedef struct melinoe_moe_request {
  * W_g, W_u [d_ff][d_model] and W_d [d_model][d_ff].  Allocates, on the current device,
  * cache_slots expert slots of melinoe_moe_expert_bytes() each plus small tables, and creates
  * a copy stream.  Limits: d_model % 256 == 0, d_model <= 8192, d_ff % 8 == 0,
- * 1 <= top_k <= n_experts <= 64, top_k <= cache_slots <= n_experts  (INVALID / UNSUPPORTED
+ * 1 <= top_k <= n_experts <= 64, top_k <= 32, top_k <= cache_slots <= n_experts  (INVALID / UNSUPPORTED
  * otherwise).
  */
 int melinoe_moe_create(int d_model, int d_ff, int n_experts, int top_k, int cache_slots,

@@ -162,7 +162,7 @@ int wait_idle(melinoe_moe *h)
 // ev_plan was recorded right behind that kernel.
 int wait_for_plan(melinoe_moe *h, uint32_t seq)
 {
-    volatile uint32_t *w = &h->hplan->seq;
+    volatile uint32_t *w = &h->hplan->hdr.seq;
     for (int i = 0; i < 4096; ++i)
         if (*w == seq)
             return MELINOE_OK;
@@ -270,7 +270,7 @@ int melinoe_moe_create(int d, int F, int E, int k, int C, melinoe_moe_t **out)
     *out = nullptr;
     if (d <= 0 || F <= 0 || E <= 0 || k <= 0 || C <= 0 || k > E || C < k || C > E)
         return MELINOE_ERR_INVALID;
-    if (d % 256 != 0 || d > 8192 || F % kUnitRows != 0 || E > kMaxExperts)
+    if (d % 256 != 0 || d > 8192 || F % kUnitRows != 0 || E > kMaxExperts || k > 32)
         return MELINOE_ERR_UNSUPPORTED;
     {
         int dev = 0;
@@ -475,8 +475,6 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
     h->call_seq += 1;
     h->last_T = T;
 
-    CU_TRY(launch_router(s, static_cast<const uint16_t *>(hidden_dev), h->w_router, h->bias, h->token_seq, T, h->d,
-                         h->E, h->k, h->idx, h->gate, h->logits));
     PlanParams pp;
     pp.idx = h->idx;
     pp.T = T;
@@ -500,7 +498,14 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
     pp.stats = stats_dev;
     pp.expert_bytes = h->expert_bytes;
     pp.vr_capacity = h->vr_capacity;
-    CU_TRY(launch_plan(s, pp));
+    if (route_plan_small_supported(T, h->k, h->d)) {
+        CU_TRY(launch_route_plan_small(s, static_cast<const uint16_t *>(hidden_dev), h->w_router, h->bias, h->token_seq,
+                                       h->d, h->idx, h->gate, h->logits, pp));
+    } else {
+        CU_TRY(launch_router(s, static_cast<const uint16_t *>(hidden_dev), h->w_router, h->bias, h->token_seq, T, h->d,
+                             h->E, h->k, h->idx, h->gate, h->logits));
+        CU_TRY(launch_plan(s, pp));
+    }
     CU_TRY(cudaEventRecord(h->ev_plan, s));
 
     FfnParams fp;
@@ -555,10 +560,33 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
         h->sticky.store(rc);
         return rc;
     }
-    const HostPlan &hp = *h->hplan;
-    int n_miss = hp.n_miss, n_groups = hp.n_groups;
-    if (hp.status != MELINOE_OK || n_miss < 0 || n_miss > h->E || n_groups < 1 || n_groups > (int)gmax)
+    const volatile HostPlan &vhp = *h->hplan;
+    int n_miss = vhp.hdr.n_miss, n_groups = vhp.hdr.n_groups;
+    if (vhp.hdr.status != MELINOE_OK || n_miss < 0 || n_miss > h->E || n_groups < 1 || n_groups > (int)gmax)
         n_miss = 0, n_groups = 1;  // the device-side status already tells the caller; nothing to fetch
+    // every miss record carries the call's sequence number: take a copy once they have all arrived
+    struct {
+        HostMiss miss[kMaxExperts];
+    } hp;
+    for (int i = 0; i < n_miss; ++i) {
+        const double t0 = now_s();
+        for (;;) {
+            HostMiss m;
+            m.expert = vhp.miss[i].expert;
+            m.slot = vhp.miss[i].slot;
+            m.group = vhp.miss[i].group;
+            m.dep_group = vhp.miss[i].dep_group;
+            m.seq = vhp.miss[i].seq;
+            if (m.seq == h->call_seq && vhp.miss[i].expert == m.expert && vhp.miss[i].slot == m.slot) {
+                hp.miss[i] = m;
+                break;
+            }
+            if (now_s() - t0 > 10.0) {
+                h->sticky.store(MELINOE_ERR_TIMEOUT);
+                return MELINOE_ERR_TIMEOUT;
+            }
+        }
+    }
     // which groups must signal their completion to the copy stream
     bool need_done[kMaxGroups + 1] = {false};
     for (int i = 0; i < n_miss; ++i)

@@ -60,15 +60,41 @@ struct DevPlan {
 };
 
 // The miss queue of a call: what the host needs in order to issue the transfers, written by
-// the planning kernel into page-locked host memory.  seq is written last (after a system-wide
-// fence); the host reads the record once seq equals the call's sequence number.
-struct HostMiss {
-    int32_t expert, slot, group, dep_group;  // dep_group: compute group that must finish first, or -1
-};
-struct HostPlan {
-    int32_t n_miss, n_groups, status, pad;
-    HostMiss miss[kMaxExperts];
+// the planning kernel into page-locked host memory.  Every 16-byte record carries the call's
+// sequence number and is written with one 16-byte store, so a record is valid exactly when its
+// seq field matches and no fence is needed between records (a system-wide fence costs several
+// microseconds over the host link).
+struct __align__(16) HostMiss {
+    int32_t expert, slot;
+    int16_t group, dep_group;    // dep_group: compute group that must finish first, or -1
     uint32_t seq;
 };
+struct __align__(16) HostPlanHeader {
+    int32_t n_miss, n_groups, status;
+    uint32_t seq;
+};
+struct __align__(16) HostPlan {
+    HostPlanHeader hdr;
+    HostMiss miss[kMaxExperts];
+};
+
+// Device side: publish the miss queue of call `seq` (one 16-byte store per record).
+__device__ inline void store16_host(void *dst, const void *rec)
+{
+    const int4 v = *reinterpret_cast<const int4 *>(rec);
+    asm volatile("st.volatile.global.v4.s32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+                 : "memory");
+}
+__device__ inline void publish_miss_queue(HostPlan *hp, const HostMiss *miss, int n_miss, int n_groups, int status,
+                                          uint32_t seq)
+{
+    for (int i = 0; i < n_miss; ++i) {
+        HostMiss m = miss[i];
+        m.seq = seq;
+        store16_host(&hp->miss[i], &m);
+    }
+    HostPlanHeader h{n_miss, n_groups, status, seq};
+    store16_host(&hp->hdr, &h);
+}
 
 }  // namespace melinoe

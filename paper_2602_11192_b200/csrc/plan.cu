@@ -192,7 +192,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p)
                 s_req[n_req] = ReqRec{e, slot, 0, ev, s_offsets[e], s_counts[e], 0, cur_group};
                 s_req_of_expert[e] = n_req;
                 s_group_of_expert[e] = cur_group;
-                s_miss[n_miss] = HostMiss{e, slot, cur_group, dep};
+                s_miss[n_miss] = HostMiss{e, slot, (int16_t)cur_group, (int16_t)dep, 0u};
             }
             counter = __shfl_sync(0xffffffffu, counter, 0);
             ++n_req;
@@ -321,19 +321,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p)
             st.call_no = s_cache.call_no;
             *p.stats = st;
         }
-        volatile HostPlan *hp = p.hplan;
-        hp->n_miss = n_miss;
-        hp->n_groups = s_misc[4];
-        hp->status = s_misc[6];
-        for (int i = 0; i < n_miss; ++i) {
-            hp->miss[i].expert = s_miss[i].expert;
-            hp->miss[i].slot = s_miss[i].slot;
-            hp->miss[i].group = s_miss[i].group;
-            hp->miss[i].dep_group = s_miss[i].dep_group;
-        }
-        __threadfence_system();
-        hp->seq = p.call_seq;
-        __threadfence_system();
+        publish_miss_queue(p.hplan, s_miss, n_miss, s_misc[4], s_misc[6], p.call_seq);
     }
 }
 
