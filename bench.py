@@ -26,6 +26,11 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one ffn_stream_kernel launch divided by the launch's
+# algorithmic bytes (8 experts x 12.58 MB), from the ncu capture summarised in
+# profiles/ffn_stream_kernel_olmoe_decode.md; traffic grows in proportion to the experts streamed.
+DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.04
+
 METRIC = "decode tokens/s (OLMoE-shaped, cache-limited)"
 UNIT = "tokens/s"
 WORKLOAD = "olmoe"
@@ -187,6 +192,25 @@ def run_ours(args):
         stack.set_phase("decode")
         torch.cuda.synchronize()
 
+    copy_acc = [0.0, 0.0]   # copy-stream ms and bytes of the most recent run with kernel timing
+
+    def host_link_gbs():
+        """Pinned host -> device copy of 512 MiB on a side stream: the link's own rate."""
+        n = 512 << 20
+        hb = torch.empty(n, dtype=torch.uint8).pin_memory()
+        db = torch.empty(n, dtype=torch.uint8, device="cuda")
+        st_ = torch.cuda.Stream()
+        best = 0.0
+        with torch.cuda.stream(st_):
+            for _ in range(4):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(st_)
+                db.copy_(hb, non_blocking=True)
+                b.record(st_)
+                st_.synchronize()
+                best = max(best, n / (a.elapsed_time(b) * 1e-3) / 1e9)
+        return best
+
     def timed_device(alpha, with_kernel_timing=False):
         prepare(alpha)
         stats_dev.zero_()
@@ -209,11 +233,15 @@ def run_ours(args):
         ms = e0.elapsed_time(e1)
         launches = M.melinoe_launch_count() - n0
         ffn_ms, ffn_n = 0.0, 0
+        copy_acc[0] = copy_acc[1] = 0.0
         if with_kernel_timing:
             for ls in stack.layers:
                 a, b = ls.layer.ffn_time_ms()
                 ffn_ms += a
                 ffn_n += b
+                cm, cb = ls.layer.transfer_time_ms()
+                copy_acc[0] += cm
+                copy_acc[1] += cb
                 ls.layer.enable_timing(False)
         st = stats_rows(stats_dev[W:W + K])
         if int(st["status"].max()) != 0:
@@ -280,8 +308,16 @@ def run_ours(args):
     _, _, st2, ffn_ms, ffn_n = timed_device(alpha0, with_kernel_timing=True)
     ffn_bytes = float((st2["n_distinct"].astype(np.int64) + cfg.n_shared).sum()) * B_e
     achieved = ffn_bytes / (ffn_ms * 1e-3) / 1e9 if ffn_ms > 0 else 0.0
+    link_peak = host_link_gbs()
+    miss_path = {"achieved_gbs": (copy_acc[1] / (copy_acc[0] * 1e-3) / 1e9) if copy_acc[0] > 0 else None,
+                 "peak_gbs": link_peak, "bytes": copy_acc[1], "copy_stream_ms": copy_acc[0],
+                 "note": "expert bytes moved by cudaMemcpyAsync from pinned host memory / time between events on the "
+                         "copy stream around each wave of transfers; peak = a 512 MiB pinned copy measured in this run"}
+    if miss_path["achieved_gbs"]:
+        miss_path["frac"] = miss_path["achieved_gbs"] / link_peak
     roofline = {"bound": "hbm", "kernel": "ffn_stream_kernel", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
-                "frac": achieved / hbm_peak, "peak_source": peak_src, "traffic": None,
+                "frac": achieved / hbm_peak, "peak_source": peak_src,
+                "traffic": DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE * ffn_bytes / max(ffn_n, 1),
                 "launches": int(ffn_n), "avg_launch_us": 1e3 * ffn_ms / max(ffn_n, 1),
                 "bytes_per_launch": ffn_bytes / max(ffn_n, 1),
                 "note": "bytes = experts streamed x bytes per expert; launches that found no missed expert to "
@@ -325,7 +361,7 @@ def run_ours(args):
             "dtype": "bf16", "data": "synthetic",
             "config": workload_config(cfg, alpha0, C, L),
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
-            "roofline": roofline, "cpu_baseline": cpu_baseline,
+            "roofline": roofline, "miss_path": miss_path, "cpu_baseline": cpu_baseline,
             "hit_stats": hit_summary(st), "other_runs": extra,
         }
         if args.layers is not None:

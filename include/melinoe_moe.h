@@ -193,6 +193,10 @@ int melinoe_moe_cache_state(melinoe_moe_t *h, int32_t *expert_of_slot_host, uint
  */
 int melinoe_moe_enable_timing(melinoe_moe_t *h, int enable);
 int melinoe_moe_ffn_time_ms(melinoe_moe_t *h, double *ms_out, int64_t *launches_out);
+/* With timing enabled, every wave of miss transfers is bracketed by events on the copy stream
+ * as well: summed copy-stream time (ms) and bytes moved host-to-device since the last query
+ * (Eq. 4's N_miss * Time_transfer, measured).  Resets both. */
+int melinoe_moe_transfer_time_ms(melinoe_moe_t *h, double *ms_out, uint64_t *bytes_out);
 
 /*
  * Kernel timeline for profiling (no counterpart in the paper).  trace_dev: device memory of at

@@ -19,7 +19,8 @@ EXPORTED_SYMBOLS = [
     "melinoe_moe_set_router_bias", "melinoe_moe_reserve", "melinoe_moe_forward", "melinoe_moe_forward_host",
     "melinoe_moe_reset_cache", "melinoe_moe_preload", "melinoe_moe_last_routing", "melinoe_moe_last_logits",
     "melinoe_moe_last_requests", "melinoe_moe_last_gather", "melinoe_moe_cache_state",
-    "melinoe_moe_enable_timing", "melinoe_moe_ffn_time_ms", "melinoe_moe_set_trace", "melinoe_moe_trace_ctas", "melinoe_launch_count",
+    "melinoe_moe_enable_timing", "melinoe_moe_ffn_time_ms", "melinoe_moe_set_trace", "melinoe_moe_trace_ctas",
+    "melinoe_moe_transfer_time_ms", "melinoe_launch_count",
     "melinoe_last_cuda_error", "melinoe_strerror",
 ]
 
@@ -82,6 +83,7 @@ def lib():
     L.melinoe_moe_cache_state.argtypes = [vp, vp, vp]
     L.melinoe_moe_enable_timing.argtypes = [vp, i32]
     L.melinoe_moe_ffn_time_ms.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
+    L.melinoe_moe_transfer_time_ms.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_uint64)]
     L.melinoe_moe_set_trace.argtypes = [vp, vp, sz]
     L.melinoe_moe_trace_ctas.argtypes = [vp]
     L.melinoe_launch_count.restype = C.c_int64
@@ -239,6 +241,12 @@ class MoELayer:
 
     def enable_timing(self, enable: bool = True) -> None:
         self._ck(lib().melinoe_moe_enable_timing(self._h, int(enable)), "melinoe_moe_enable_timing")
+
+    def transfer_time_ms(self):
+        ms = C.c_double(0.0)
+        nb = C.c_uint64(0)
+        self._ck(lib().melinoe_moe_transfer_time_ms(self._h, C.byref(ms), C.byref(nb)), "melinoe_moe_transfer_time_ms")
+        return ms.value, nb.value
 
     def set_trace(self, trace_dev, n_bytes: int) -> None:
         self._keep["trace"] = trace_dev

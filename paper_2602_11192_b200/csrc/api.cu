@@ -105,7 +105,8 @@ struct melinoe_moe {
 
     // kernel timing
     bool timing = false;
-    std::vector<TimedPair> timed, free_pairs;
+    std::vector<TimedPair> timed, free_pairs, timed_copy;
+    uint64_t timed_copy_bytes = 0;
 };
 
 namespace {
@@ -374,6 +375,10 @@ int melinoe_moe_destroy(melinoe_moe_t *h)
         cudaEventDestroy(p.a);
         cudaEventDestroy(p.b);
     }
+    for (auto &p : h->timed_copy) {
+        cudaEventDestroy(p.a);
+        cudaEventDestroy(p.b);
+    }
     (void)cudaGetLastError();
     delete h;
     return rc;
@@ -609,6 +614,8 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
     }
     int i = 0;
     for (int g = 1; g < n_groups; ++g) {
+        TimedPair ctp{nullptr, nullptr};
+        bool wave_started = false;
         for (; i < n_miss && hp.miss[i].group == g; ++i) {
             const HostMiss m = hp.miss[i];
             if (m.expert < 0 || m.expert >= h->E || m.slot < 0 || m.slot >= h->C || m.dep_group >= g) {
@@ -617,8 +624,25 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
             }
             if (m.dep_group >= 0)  // the slot still feeds an earlier compute group of this call
                 CU_TRY(cudaStreamWaitEvent(h->copy_stream, h->ev_group[m.dep_group], 0));
+            if (h->timing && !wave_started) {
+                if (!h->free_pairs.empty()) {
+                    ctp = h->free_pairs.back();
+                    h->free_pairs.pop_back();
+                } else {
+                    CU_TRY(cudaEventCreate(&ctp.a));
+                    CU_TRY(cudaEventCreate(&ctp.b));
+                }
+                CU_TRY(cudaEventRecord(ctp.a, h->copy_stream));
+                wave_started = true;
+            }
+            if (h->timing)
+                h->timed_copy_bytes += h->expert_bytes;
             CU_TRY(cudaMemcpyAsync(h->slots + (size_t)m.slot * h->slot_stride, h->host_experts[m.expert],
                                    h->expert_bytes, cudaMemcpyHostToDevice, h->copy_stream));
+        }
+        if (wave_started) {
+            CU_TRY(cudaEventRecord(ctp.b, h->copy_stream));
+            h->timed_copy.push_back(ctp);
         }
         CU_TRY(cudaEventRecord(h->ev_arrive, h->copy_stream));
         CU_TRY(cudaStreamWaitEvent(s, h->ev_arrive, 0));
@@ -809,6 +833,28 @@ int melinoe_moe_cache_state(melinoe_moe_t *h, int32_t *expert_of_slot_host, uint
     if (err != 0)
         return err;
     return h->sticky.load();
+}
+
+int melinoe_moe_transfer_time_ms(melinoe_moe_t *h, double *ms_out, uint64_t *bytes_out)
+{
+    if (!h)
+        return MELINOE_ERR_INVALID;
+    double total = 0.0;
+    for (auto &p : h->timed_copy) {
+        CU_TRY(cudaEventSynchronize(p.b));
+        float ms = 0.f;
+        CU_TRY(cudaEventElapsedTime(&ms, p.a, p.b));
+        total += ms;
+    }
+    if (ms_out)
+        *ms_out = total;
+    if (bytes_out)
+        *bytes_out = h->timed_copy_bytes;
+    for (auto &p : h->timed_copy)
+        h->free_pairs.push_back(p);
+    h->timed_copy.clear();
+    h->timed_copy_bytes = 0;
+    return MELINOE_OK;
 }
 
 int melinoe_moe_set_trace(melinoe_moe_t *h, void *trace_dev, size_t bytes)
