@@ -157,6 +157,39 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
 int melinoe_moe_forward_host(melinoe_moe_t *h, void *cuda_stream, const void *hidden_host,
                              int n_tokens, void *out_host, melinoe_moe_stats *stats_host);
 
+/*
+ * melinoe_moe_forward for callers that must not allocate (no counterpart in the paper).
+ *
+ * melinoe_moe_forward grows its per-handle scratch with cudaMalloc when a call is larger than
+ * anything seen before, and creates CUDA events on demand.  Some callers cannot have that happen
+ * inside the call: a serving loop that has handed all remaining device memory to a KV cache or to
+ * another allocator and would get an out-of-memory error (or a device-wide synchronisation) from a
+ * stray cudaMalloc, and code that runs where the CUDA allocator must not be entered at all.  This
+ * entry point runs the same layer, same kernels and same cache state, but takes every byte of
+ * scratch (routing tables, gather lists, the h and z buffers of the expert FFN) from one array
+ * of melinoe_moe_static_scratch_bytes() (about 8.6 MiB) that is part of the library's device
+ * image: each GPU that loads the library holds it until the process exits.  It calls no
+ * cudaMalloc, cudaFree, event-creating or otherwise allocating routine.
+ *
+ * Limits, all checked, MELINOE_ERR_UNSUPPORTED beyond them (nothing is launched then):
+ *   n_tokens <= 8, n_tokens * top_k <= 16, n_tokens * top_k <= cache_slots,
+ *   n_shared * n_tokens <= 64, d_model <= 8192, d_ff <= 16384.
+ * MELINOE_ERR_STATE if kernel timing is enabled on the handle (timed calls create events).
+ *
+ * The first call on a device looks up the array's device address (cudaGetSymbolAddress) with
+ * that device current; make this first call before any stream capture begins.
+ * Every call on a device, of every handle, uses the same array: it keeps the previous call's
+ * contents (what has to start from zero is cleared on the caller's stream at the start of each
+ * call), and two such calls that can overlap on the GPU (different streams without an ordering
+ * between them) race on it.  Calls on one stream, or ordered by events, are safe, and may be
+ * mixed freely with melinoe_moe_forward on the same handle.
+ * The inspection calls (melinoe_moe_last_*) do not see calls made through this entry point.
+ * Arguments and results otherwise as melinoe_moe_forward.
+ */
+int melinoe_moe_forward_static(melinoe_moe_t *h, void *cuda_stream, const void *hidden_dev,
+                               int n_tokens, void *out_dev, melinoe_moe_stats *stats_dev);
+size_t melinoe_moe_static_scratch_bytes(void);
+
 /* Cold start: all slots empty, stamps and totals zero.  Synchronises the handle first. */
 int melinoe_moe_reset_cache(melinoe_moe_t *h);
 

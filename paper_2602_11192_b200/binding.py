@@ -20,7 +20,7 @@ EXPORTED_SYMBOLS = [
     "melinoe_moe_reset_cache", "melinoe_moe_preload", "melinoe_moe_last_routing", "melinoe_moe_last_logits",
     "melinoe_moe_last_requests", "melinoe_moe_last_gather", "melinoe_moe_cache_state",
     "melinoe_moe_enable_timing", "melinoe_moe_ffn_time_ms", "melinoe_moe_set_trace", "melinoe_moe_trace_ctas",
-    "melinoe_moe_transfer_time_ms", "melinoe_launch_count",
+    "melinoe_moe_transfer_time_ms", "melinoe_moe_forward_static", "melinoe_moe_static_scratch_bytes", "melinoe_launch_count",
     "melinoe_last_cuda_error", "melinoe_strerror",
 ]
 
@@ -74,6 +74,8 @@ def lib():
     L.melinoe_moe_reserve.argtypes = [vp, i32]
     L.melinoe_moe_forward.argtypes = [vp, vp, vp, i32, vp, vp]
     L.melinoe_moe_forward_host.argtypes = [vp, vp, vp, i32, vp, vp]
+    L.melinoe_moe_forward_static.argtypes = [vp, vp, vp, i32, vp, vp]
+    L.melinoe_moe_static_scratch_bytes.restype = sz
     L.melinoe_moe_reset_cache.argtypes = [vp]
     L.melinoe_moe_preload.argtypes = [vp, vp, i32]
     L.melinoe_moe_last_routing.argtypes = [vp, vp, vp]
@@ -189,6 +191,11 @@ class MoELayer:
     def forward(self, stream: int, hidden_dev, n_tokens: int, out_dev, stats_dev=None) -> None:
         self._ck(lib().melinoe_moe_forward(self._h, stream, _ptr(hidden_dev), n_tokens, _ptr(out_dev),
                                            _ptr(stats_dev)), "melinoe_moe_forward")
+
+    def forward_static(self, stream: int, hidden_dev, n_tokens: int, out_dev, stats_dev=None) -> None:
+        """melinoe_moe_forward_static: the same call on the library's static scratch (allocates nothing)."""
+        self._ck(lib().melinoe_moe_forward_static(self._h, stream, _ptr(hidden_dev), n_tokens, _ptr(out_dev),
+                                                  _ptr(stats_dev)), "melinoe_moe_forward_static")
 
     def forward_host(self, stream: int, hidden_host, n_tokens: int, out_host, stats_host=None) -> None:
         self._ck(lib().melinoe_moe_forward_host(self._h, stream, _ptr(hidden_host), n_tokens, _ptr(out_host),

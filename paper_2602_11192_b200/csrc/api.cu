@@ -16,6 +16,7 @@
 #include <chrono>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <thread>
 #include <vector>
@@ -661,6 +662,128 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
     h->has_last = true;
     return MELINOE_OK;
 }
+
+}  // extern "C"
+
+// ---------------------------------------------------------------- forward without allocation
+//
+// Scratch of melinoe_moe_forward_static: one array in the library's device image, shared by every
+// call on the device, instead of per-handle cudaMalloc'd buffers.
+constexpr int kStaticMaxTokens = 8;
+constexpr int kStaticMaxPairs = 16;                         // n_tokens * top_k
+constexpr int kStaticMaxSharedRows = 64;                    // n_shared * n_tokens
+constexpr int kStaticMaxVr = kStaticMaxPairs + kMaxShared;  // one virtual request per routed pair or shared expert
+constexpr int kStaticMaxD = 8192, kStaticMaxF = 16384;
+constexpr size_t kStaticSmall = 16 * 1024;                  // idx, gate, logits, perm, inv_pos, tok_of_sorted, vrs
+constexpr size_t kStaticZ = (size_t)(kStaticMaxPairs + kStaticMaxSharedRows) * kStaticMaxD * sizeof(float);
+constexpr size_t kStaticH = (size_t)kStaticMaxVr * kTokPerVr * kStaticMaxF * 2;
+constexpr size_t kStaticBytes = kStaticSmall + kStaticZ + kStaticH;   // about 8.6 MiB
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];
+
+namespace {
+// Device address of g_static_scratch per device ordinal.  In host code the array's name is
+// only a handle for the runtime, not an address a kernel could use.
+constexpr int kMaxDevices = 64;
+unsigned char *g_static_ptr[kMaxDevices] = {nullptr};
+std::mutex g_static_mu;
+}  // namespace
+
+extern "C" int melinoe_moe_forward_static(melinoe_moe_t *h, void *cuda_stream, const void *hidden_dev, int T,
+                                          void *out_dev, melinoe_moe_stats *stats_dev)
+{
+    if (!h || T < 0)
+        return MELINOE_ERR_INVALID;
+    if (T == 0)
+        return MELINOE_OK;
+    // everything beyond the static scratch's sizes is refused, never served by allocating
+    if (T > kStaticMaxTokens || T * h->k > kStaticMaxPairs || T * h->k > h->C || h->n_shared * T > kStaticMaxSharedRows ||
+        h->d > kStaticMaxD || h->F > kStaticMaxF)
+        return MELINOE_ERR_UNSUPPORTED;
+    if (h->timing)
+        return MELINOE_ERR_STATE;   // timed calls create events on demand
+    if (h->device < 0 || h->device >= kMaxDevices)
+        return MELINOE_ERR_UNSUPPORTED;
+    unsigned char *base = nullptr;
+    {
+        std::lock_guard<std::mutex> lk(g_static_mu);
+        base = g_static_ptr[h->device];
+        if (!base) {
+            // first call on this device (the handle's device must be current, as for every call)
+            int cur = -1;
+            CU_TRY(cudaGetDevice(&cur));
+            if (cur != h->device)
+                return MELINOE_ERR_STATE;
+            void *p = nullptr;
+            CU_TRY(cudaGetSymbolAddress(&p, g_static_scratch));
+            base = g_static_ptr[h->device] = static_cast<unsigned char *>(p);
+        }
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    // carve the scratch: small tables first, then z, then h
+    unsigned char *q = base;
+    auto take = [&](size_t bytes) {
+        unsigned char *r = q;
+        q += (bytes + 255) / 256 * 256;
+        return r;
+    };
+    const size_t pairs = kStaticMaxPairs, sorted = kStaticMaxPairs + kStaticMaxSharedRows;
+    int32_t *idx = reinterpret_cast<int32_t *>(take(pairs * 4));
+    float *gate = reinterpret_cast<float *>(take(pairs * 4));
+    float *logits = reinterpret_cast<float *>(take((size_t)kStaticMaxTokens * kMaxExperts * 4));
+    int32_t *perm = reinterpret_cast<int32_t *>(take(sorted * 4));
+    int32_t *inv_pos = reinterpret_cast<int32_t *>(take(pairs * 4));
+    int32_t *tok_of_sorted = reinterpret_cast<int32_t *>(take(sorted * 4));
+    VrRec *vrs = reinterpret_cast<VrRec *>(take((size_t)kStaticMaxVr * sizeof(VrRec)));
+    if ((size_t)(q - base) > kStaticSmall)
+        return MELINOE_ERR_STATE;
+    float *zbuf = reinterpret_cast<float *>(base + kStaticSmall);
+    uint16_t *hbuf = reinterpret_cast<uint16_t *>(base + kStaticSmall + kStaticZ);
+    // the padding behind every h row has to read as zero, and the array keeps whatever the last
+    // call (of any handle, with any d_ff) left there
+    const size_t fpad = ((size_t)h->F + 255) / 256 * 256;
+    CU_TRY(cudaMemsetAsync(hbuf, 0, (size_t)kStaticMaxVr * kTokPerVr * fpad * 2, s));
+
+    // run the ordinary call on the static scratch: swap the handle's scratch pointers for its duration
+    struct Saved {
+        int32_t *idx, *perm, *inv_pos, *tok_of_sorted;
+        float *gate, *logits, *zbuf;
+        uint16_t *hbuf;
+        VrRec *vrs;
+        int cap_tokens, cap_shared, vr_capacity;
+    } keep{h->idx, h->perm, h->inv_pos, h->tok_of_sorted, h->gate, h->logits, h->zbuf, h->hbuf, h->vrs,
+           h->cap_tokens, h->cap_shared, h->vr_capacity};
+    h->idx = idx;
+    h->perm = perm;
+    h->inv_pos = inv_pos;
+    h->tok_of_sorted = tok_of_sorted;
+    h->gate = gate;
+    h->logits = logits;
+    h->zbuf = zbuf;
+    h->hbuf = hbuf;
+    h->vrs = vrs;
+    h->cap_tokens = kStaticMaxTokens;
+    h->cap_shared = h->n_shared;
+    h->vr_capacity = kStaticMaxVr;
+    const int rc = melinoe_moe_forward(h, cuda_stream, hidden_dev, T, out_dev, stats_dev);
+    h->idx = keep.idx;
+    h->perm = keep.perm;
+    h->inv_pos = keep.inv_pos;
+    h->tok_of_sorted = keep.tok_of_sorted;
+    h->gate = keep.gate;
+    h->logits = keep.logits;
+    h->zbuf = keep.zbuf;
+    h->hbuf = keep.hbuf;
+    h->vrs = keep.vrs;
+    h->cap_tokens = keep.cap_tokens;
+    h->cap_shared = keep.cap_shared;
+    h->vr_capacity = keep.vr_capacity;
+    h->last_T = 0;   // the inspection calls read the handle's own scratch, which this call did not touch
+    return rc;
+}
+
+extern "C" size_t melinoe_moe_static_scratch_bytes(void) { return kStaticBytes; }
+
+extern "C" {
 
 int melinoe_moe_forward_host(melinoe_moe_t *h, void *cuda_stream, const void *hidden_host, int T, void *out_host,
                              melinoe_moe_stats *stats_host)
