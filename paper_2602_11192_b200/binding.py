@@ -20,7 +20,8 @@ EXPORTED_SYMBOLS = [
     "melinoe_moe_reset_cache", "melinoe_moe_preload", "melinoe_moe_last_routing", "melinoe_moe_last_logits",
     "melinoe_moe_last_requests", "melinoe_moe_last_gather", "melinoe_moe_cache_state",
     "melinoe_moe_enable_timing", "melinoe_moe_ffn_time_ms", "melinoe_moe_set_trace", "melinoe_moe_trace_ctas",
-    "melinoe_moe_transfer_time_ms", "melinoe_moe_forward_static", "melinoe_moe_static_scratch_bytes", "melinoe_launch_count",
+    "melinoe_moe_transfer_time_ms", "melinoe_moe_forward_static", "melinoe_moe_static_scratch_bytes",
+    "melinoe_moe_last_call_used_gemm", "melinoe_launch_count",
     "melinoe_last_cuda_error", "melinoe_strerror",
 ]
 
@@ -76,6 +77,7 @@ def lib():
     L.melinoe_moe_forward_host.argtypes = [vp, vp, vp, i32, vp, vp]
     L.melinoe_moe_forward_static.argtypes = [vp, vp, vp, i32, vp, vp]
     L.melinoe_moe_static_scratch_bytes.restype = sz
+    L.melinoe_moe_last_call_used_gemm.argtypes = [vp]
     L.melinoe_moe_reset_cache.argtypes = [vp]
     L.melinoe_moe_preload.argtypes = [vp, vp, i32]
     L.melinoe_moe_last_routing.argtypes = [vp, vp, vp]
@@ -248,6 +250,9 @@ class MoELayer:
 
     def enable_timing(self, enable: bool = True) -> None:
         self._ck(lib().melinoe_moe_enable_timing(self._h, int(enable)), "melinoe_moe_enable_timing")
+
+    def last_call_used_gemm(self) -> bool:
+        return bool(lib().melinoe_moe_last_call_used_gemm(self._h))
 
     def transfer_time_ms(self):
         ms = C.c_double(0.0)

@@ -10,6 +10,7 @@
 // is a CUDA event (copy stream -> compute stream for arrival, compute stream -> copy stream
 // when a wave overwrites a slot that an earlier group of the same call still reads), so the
 // ordering is visible to the driver and cannot deadlock however streams share hardware queues.
+#include <cuda.h>
 #include <cuda_runtime.h>
 
 #include <atomic>
@@ -50,6 +51,34 @@ int cuda_fail(cudaError_t e)
             return cuda_fail(e__);        \
     } while (0)
 
+typedef CUresult (*encode_tiled_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                    const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+encode_tiled_fn g_encode_tiled = nullptr;
+std::once_flag g_encode_once;
+
+// 2-D bf16 tensor [rows][cols], row-major, 128-byte swizzle, box of box_rows x 64 columns.
+bool encode_map(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows, uint32_t box_rows)
+{
+    std::call_once(g_encode_once, [] {
+        cudaDriverEntryPointQueryResult qr;
+        void *fn = nullptr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qr) == cudaSuccess &&
+            qr == cudaDriverEntryPointSuccess)
+            g_encode_tiled = reinterpret_cast<encode_tiled_fn>(fn);
+        (void)cudaGetLastError();
+    });
+    if (!g_encode_tiled || rows == 0)
+        return false;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * 2};
+    const cuuint32_t box[2] = {64, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return g_encode_tiled(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 double now_s()
 {
     return std::chrono::duration<double>(std::chrono::steady_clock::now().time_since_epoch()).count();
@@ -82,6 +111,12 @@ struct melinoe_moe {
     unsigned long long *trace = nullptr;   // borrowed; see melinoe_moe_set_trace
     VrRec *vrs = nullptr;
     uint16_t *stage_in = nullptr, *stage_out = nullptr;
+    // grouped-GEMM path (calls of more than 8 tokens): gathered activations, h, tensor maps
+    bool gemm_ok = false, last_used_gemm = false;
+    uint16_t *xs = nullptr, *hs = nullptr;
+    CUtensorMap *maps_dev = nullptr;
+    CUtensorMap maps_host[kMapCount];
+    const void *shared_ptrs[kMaxShared] = {nullptr};
     melinoe_moe_stats *stage_stats = nullptr;
 
     // borrowed
@@ -144,6 +179,9 @@ void free_scratch(melinoe_moe *h)
     cudaFree(h->vrs);
     cudaFree(h->stage_in);
     cudaFree(h->stage_out);
+    cudaFree(h->xs);
+    cudaFree(h->hs);
+    h->xs = h->hs = nullptr;
     h->idx = h->perm = h->inv_pos = h->tok_of_sorted = nullptr;
     h->gate = h->logits = h->zbuf = nullptr;
     h->hbuf = nullptr;
@@ -215,6 +253,14 @@ int ensure_capacity(melinoe_moe *h, int T)
     CU_TRY(cudaMemset(h->hbuf, 0, hbytes));   // the padding of every h row stays zero for good
     CU_TRY(cudaMalloc(&h->stage_in, (size_t)cap * h->d * 2));
     CU_TRY(cudaMalloc(&h->stage_out, (size_t)cap * h->d * 2));
+    if (h->gemm_ok && cap > kTokPerVr) {
+        CU_TRY(cudaMalloc(&h->xs, sorted * h->d * 2));
+        CU_TRY(cudaMalloc(&h->hs, sorted * h->F * 2));
+        if (!encode_map(&h->maps_host[kMapXs], h->xs, h->d, sorted, 128) ||
+            !encode_map(&h->maps_host[kMapHs], h->hs, h->F, sorted, 128))
+            return MELINOE_ERR_CUDA;
+        CU_TRY(cudaMemcpy(h->maps_dev, h->maps_host, sizeof(h->maps_host), cudaMemcpyHostToDevice));
+    }
     h->vr_capacity = vr_cap;
     h->cap_tokens = cap;
     h->cap_shared = h->n_shared;
@@ -335,6 +381,18 @@ int melinoe_moe_create(int d, int F, int E, int k, int C, melinoe_moe_t **out)
     CR(cudaEventCreateWithFlags(&h->ev_last, cudaEventDisableTiming));
     CR(cudaEventCreateWithFlags(&h->ev_plan, cudaEventDisableTiming));
     CR(cudaEventCreateWithFlags(&h->ev_arrive, cudaEventDisableTiming));
+    // grouped GEMM for calls of many tokens: the slots are contiguous, so one tensor map per view
+    // (rows of d elements: W_g, W_u; rows of F elements: W_d) covers every slot
+    std::memset(h->maps_host, 0, sizeof(h->maps_host));
+    if (ffn_gemm_supported(d, F) && h->slot_stride == h->expert_bytes && ffn_gemm_configure() == cudaSuccess) {
+        CR(cudaMalloc(&h->maps_dev, sizeof(h->maps_host)));
+        if (encode_map(&h->maps_host[kMapSlotsD], h->slots, d, (uint64_t)C * 3 * F, 128) &&
+            encode_map(&h->maps_host[kMapSlotsF], h->slots, F, (uint64_t)C * 3 * d, 256)) {
+            CR(cudaMemcpy(h->maps_dev, h->maps_host, sizeof(h->maps_host), cudaMemcpyHostToDevice));
+            h->gemm_ok = true;
+        }
+    }
+    (void)cudaGetLastError();
 #undef CR
     (void)rc;
     *out = h;
@@ -355,6 +413,7 @@ int melinoe_moe_destroy(melinoe_moe_t *h)
     cudaFree(h->err_word);
     cudaFree(h->sync);
     cudaFree(h->shared_dev);
+    cudaFree(h->maps_dev);
     cudaFree(h->stage_stats);
     if (h->hplan)
         cudaFreeHost(h->hplan);
@@ -438,6 +497,13 @@ int melinoe_moe_register_shared_experts(melinoe_moe_t *h, int n_shared, const vo
     for (int s = 0; s < n_shared; ++s)
         tmp[s] = static_cast<const char *>(ptrs[s]);
     CU_TRY(cudaMemcpy(h->shared_dev, tmp, sizeof tmp, cudaMemcpyHostToDevice));
+    if (h->gemm_ok) {
+        for (int s = 0; s < n_shared; ++s)
+            if (!encode_map(&h->maps_host[kMapShared0 + 2 * s], ptrs[s], h->d, (uint64_t)3 * h->F, 128) ||
+                !encode_map(&h->maps_host[kMapShared0 + 2 * s + 1], ptrs[s], h->F, (uint64_t)3 * h->d, 256))
+                return MELINOE_ERR_CUDA;
+        CU_TRY(cudaMemcpy(h->maps_dev, h->maps_host, sizeof(h->maps_host), cudaMemcpyHostToDevice));
+    }
     h->n_shared = n_shared;
     return MELINOE_OK;
 }
@@ -535,6 +601,22 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
     FfnGeometry geo;
     if (ffn_stream_geometry(h->cfg, h->d, h->F, T, &geo) != cudaSuccess)
         return MELINOE_ERR_UNSUPPORTED;
+    // calls of more than 8 tokens go through the grouped GEMM (where the shapes allow it)
+    const bool use_gemm = h->gemm_ok && T > kTokPerVr && h->xs != nullptr;
+    GemmParams gp;
+    gp.plan = h->plan;
+    gp.maps = h->maps_dev;
+    gp.hs = h->hs;
+    gp.zs = h->zbuf;
+    gp.err = h->err_word;
+    gp.d = h->d;
+    gp.F = h->F;
+    gp.E = h->E;
+    gp.n_shared = h->n_shared;
+    h->last_used_gemm = use_gemm;
+    if (use_gemm)
+        CU_TRY(launch_gather_rows(s, h->plan, static_cast<const uint16_t *>(hidden_dev), h->tok_of_sorted, h->xs, h->d,
+                                  T * h->k + h->n_shared * T, h->n_sms));
     auto launch_group = [&](int g) -> int {
         TimedPair tp{nullptr, nullptr};
         if (h->timing) {
@@ -547,8 +629,14 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
             }
             CU_TRY(cudaEventRecord(tp.a, s));
         }
-        fp.group = g;
-        CU_TRY(launch_ffn_stream(s, h->cfg, geo, fp));
+        if (use_gemm) {
+            gp.group = g;
+            CU_TRY(launch_ffn_gemm(s, 1, h->n_sms, gp));
+            CU_TRY(launch_ffn_gemm(s, 2, h->n_sms, gp));
+        } else {
+            fp.group = g;
+            CU_TRY(launch_ffn_stream(s, h->cfg, geo, fp));
+        }
         if (h->timing) {
             CU_TRY(cudaEventRecord(tp.b, s));
             h->timed.push_back(tp);
@@ -658,6 +746,9 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
         }
     }
 
+    if (use_gemm)
+        CU_TRY(launch_combine_rows(s, h->plan, h->gate, h->inv_pos, h->zbuf, static_cast<uint16_t *>(out_dev), T, h->d,
+                                   h->k, h->n_shared, h->n_sms));
     CU_TRY(cudaEventRecord(h->ev_last, s));
     h->has_last = true;
     return MELINOE_OK;
@@ -995,6 +1086,8 @@ int melinoe_moe_set_trace(melinoe_moe_t *h, void *trace_dev, size_t bytes)
 }
 
 int melinoe_moe_trace_ctas(melinoe_moe_t *h) { return h ? h->cfg.grid : 0; }
+
+int melinoe_moe_last_call_used_gemm(melinoe_moe_t *h) { return h && h->last_used_gemm ? 1 : 0; }
 
 int melinoe_moe_enable_timing(melinoe_moe_t *h, int enable)
 {

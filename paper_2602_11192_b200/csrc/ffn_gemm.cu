@@ -1,0 +1,476 @@
+// Expert FFN (Eq. 3) for calls with many tokens per expert (prefill): a grouped GEMM on the
+// fifth-generation tensor cores (tcgen05.mma, accumulators in tensor memory, operands staged
+// in shared memory by TMA), plus the token gather in front of it and the combine (Eq. 2) behind.
+//
+//   gather    Xs[pos] = hidden[token of sorted position pos]: the tokens of one expert become
+//             consecutive rows, so an expert's activations are one 2-D box for TMA.
+//   GEMM 1    per expert: [G | U] = Xs_e (M_e x d) * [W_g ; W_u]^T, tile 128 tokens x 128 f:
+//             one MMA of N = 256 whose B tile stacks 128 rows of W_g on 128 rows of W_u, so the
+//             accumulator holds g in columns 0..127 and u in 128..255 of the same token row and
+//             the epilogue forms h = SiLU(g) * u in registers; h is stored as bf16.
+//   GEMM 2    per expert: Z = H_e (M_e x F) * W_d^T, tile 128 tokens x 256 output columns, fp32.
+//   combine   y_t = sum_j gate[t][j] * Z[pos(t, j)] (+ shared experts), rank order, one rounding.
+//
+// Both GEMMs use the paper's own matrix shapes: W_g, W_u [F][d] and W_d [d][F] are "N x K,
+// K contiguous", and so are Xs and H, i.e. every operand is K-major with 128-byte swizzle.
+// The experts of all slots are addressed through one tensor map per view (rows of d elements
+// for GEMM 1, rows of F elements for GEMM 2), because the slots are contiguous.
+//
+// One persistent CTA per SM, warp-specialised: warp 0 issues TMA loads into a 4-stage ring,
+// warp 1 issues the MMAs (one elected thread) and commits them to mbarriers, warps 2..5 drain
+// the accumulator (tcgen05.ld, 32 rows per warp) and write the tile.  Two accumulators of 256
+// columns alternate so the epilogue of a tile overlaps the MMAs of the next.  Work items are
+// (request, n-tile, m-tile) triples of the launch's compute group, dealt round-robin.
+//
+// Ragged M: an m-tile may run past its expert's last row; those rows are computed on whatever
+// the next rows hold (or zeros past the end of the buffer) and never stored.
+//
+// Every wait is bounded; on a timeout the CTA raises its abort flag, every role leaves its
+// loops, tensor memory is freed and the error word tells the host.
+#include <cuda.h>
+
+#include "kernels.cuh"
+
+namespace melinoe {
+
+namespace {
+
+constexpr int kGemmThreads = 192;          // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
+constexpr int kBM = 128, kBK = 64;         // tile rows (tokens), K elements per stage (128 bytes)
+constexpr int kBN = 256;                   // accumulator columns: 128 g + 128 u, or 256 outputs
+constexpr int kStages = 4;
+constexpr int kABytes = kBM * kBK * 2, kBBytes = kBN * kBK * 2, kStageBytes = kABytes + kBBytes;
+constexpr long long kGemmWaitCycles = 4000000000ll;
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
+{
+    if (mbar_try(bar, parity))
+        return true;
+    if (*abort_flag)
+        return false;
+    const long long t0 = clock64();
+    for (;;) {
+        for (int i = 0; i < 64; ++i)
+            if (mbar_try(bar, parity))
+                return true;
+        if (*abort_flag)
+            return false;
+        if (clock64() - t0 > kGemmWaitCycles) {
+            *abort_flag = 1;
+            return false;
+        }
+    }
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+
+// 2-D tiled TMA load: box at (x = element column, y = row) of the tensor map into shared memory.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes, groups
+// of 8 rows 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3FFFFu) >> 4);          // start address
+    d |= (uint64_t)(1024u >> 4) << 32;                // stride between 8-row groups
+    d |= (uint64_t)1 << 46;                           // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;                           // 128-byte swizzle
+    return d;
+}
+
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = 256.
+__device__ __forceinline__ uint32_t instr_desc_bf16(int m, int n)
+{
+    uint32_t d = 0;
+    d |= 1u << 4;                    // D format: fp32
+    d |= 1u << 7;                    // A format: bf16
+    d |= 1u << 10;                   // B format: bf16
+    d |= (uint32_t)(n >> 3) << 17;
+    d |= (uint32_t)(m >> 4) << 24;
+    return d;
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+}
+
+__device__ __forceinline__ uint32_t bf16_rne(float v)
+{
+    uint32_t u = __float_as_uint(v);
+    u += 0x7fffu + ((u >> 16) & 1u);
+    return u >> 16;
+}
+
+struct GemmItem {
+    int row0;      // first sorted row of the m-tile
+    int row_end;   // one past the expert's last sorted row
+    int b_row;     // first row of the B tile in its tensor map (GEMM 1: the W_g rows; W_u = + F)
+    int n0;        // first output column of the tile (f for GEMM 1, output column for GEMM 2)
+    int shared;    // B comes from a shared expert's tensor map: index of that expert, else -1
+};
+
+// PHASE 1: h = SiLU(Xs W_g^T) * (Xs W_u^T) -> hs (bf16).  PHASE 2: z = hs W_d^T -> zs (fp32).
+template <int PHASE>
+__global__ void __launch_bounds__(kGemmThreads, 1) ffn_gemm_kernel(GemmParams p)
+{
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    __shared__ uint64_t s_bars[2 * kStages + 4];
+    __shared__ uint32_t s_tmem_base;
+    __shared__ int s_abort;
+    __shared__ int s_req[kMaxReq], s_tile0[kMaxReq + 1], s_nreq;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const DevPlan *plan = p.plan;
+    if (plan->status != MELINOE_OK)
+        return;
+    // 1024-byte aligned ring (the swizzle pattern repeats every 1024 bytes)
+    unsigned char *ring = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const uint32_t ring_s = smem_u32(ring);
+    const uint32_t full0 = smem_u32(s_bars), empty0 = full0 + 8 * kStages;
+    const uint32_t tfull0 = empty0 + 8 * kStages, tempty0 = tfull0 + 16;
+    volatile int *abort_flag = &s_abort;
+
+    // ---- the launch's requests and their m-tiles
+    const int K = PHASE == 1 ? p.d : p.F;                 // reduction length
+    const int n_tiles_n = PHASE == 1 ? p.F / 128 : p.d / kBN;
+    if (tid == 0) {
+        s_abort = 0;
+        int n = 0, tiles = 0;
+        const int n_req_total = plan->n_req + p.n_shared;
+        for (int r = 0; r < n_req_total; ++r) {
+            const ReqRec rec = plan->req[r];
+            if (rec.group == p.group && rec.n_tok > 0) {
+                s_req[n] = r;
+                s_tile0[n] = tiles;
+                tiles += (rec.n_tok + kBM - 1) / kBM * n_tiles_n;
+                ++n;
+            }
+        }
+        s_tile0[n] = tiles;
+        s_nreq = n;
+        for (int i = 0; i < kStages; ++i) {
+            mbar_init(full0 + 8 * i, 1);
+            mbar_init(empty0 + 8 * i, 1);
+        }
+        mbar_init(tfull0, 1);
+        mbar_init(tfull0 + 8, 1);
+        mbar_init(tempty0, 4);
+        mbar_init(tempty0 + 8, 4);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    const int n_reqs = s_nreq;
+    const int total_items = s_tile0[n_reqs];
+    if (total_items == 0)
+        return;
+
+    if (warp == 2) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)),
+                     "r"(512));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = s_tmem_base;
+
+    // item w -> (request, n-tile, m-tile): within a request the m-tiles of one n-tile are adjacent,
+    // so CTAs working side by side share the weight tile in L2
+    auto item_of = [&](int w) -> GemmItem {
+        int q = 0;
+        while (q + 1 < n_reqs && s_tile0[q + 1] <= w)
+            ++q;
+        const ReqRec rec = plan->req[s_req[q]];
+        const int local = w - s_tile0[q];
+        const int mtiles = (rec.n_tok + kBM - 1) / kBM;
+        const int nt = local / mtiles, mt = local % mtiles;
+        GemmItem it;
+        it.row0 = rec.tok_off + mt * kBM;
+        it.row_end = rec.tok_off + rec.n_tok;
+        it.shared = rec.slot >= 0 ? -1 : rec.expert - p.E;
+        const int base_expert = rec.slot >= 0 ? rec.slot : 0;     // shared experts have a map each
+        if (PHASE == 1) {
+            it.n0 = nt * 128;
+            it.b_row = base_expert * 3 * p.F + it.n0;
+        } else {
+            it.n0 = nt * kBN;
+            it.b_row = base_expert * 3 * p.d + 2 * p.d + it.n0;
+        }
+        return it;
+    };
+    const int kblocks = K / kBK;
+
+    if (warp == 0) {
+        // ============================================================ TMA producer
+        if (lane == 0) {
+            const CUtensorMap *map_a = p.maps + (PHASE == 1 ? kMapXs : kMapHs);
+            uint32_t n = 0;
+            for (int w = blockIdx.x; w < total_items && !*abort_flag; w += gridDim.x) {
+                const GemmItem it = item_of(w);
+                const CUtensorMap *map_b = it.shared < 0 ? p.maps + (PHASE == 1 ? kMapSlotsD : kMapSlotsF)
+                                                         : p.maps + kMapShared0 + 2 * it.shared + (PHASE == 1 ? 0 : 1);
+                for (int kb = 0; kb < kblocks; ++kb, ++n) {
+                    const uint32_t s = n % kStages;
+                    if (n >= (uint32_t)kStages && !mbar_wait(empty0 + 8 * s, ((n / kStages) - 1u) & 1u, abort_flag))
+                        break;
+                    const uint32_t bar = full0 + 8 * s;
+                    const uint32_t a_dst = ring_s + s * kStageBytes, b_dst = a_dst + kABytes;
+                    mbar_expect(bar, kStageBytes);
+                    tma_load_2d(a_dst, map_a, kb * kBK, it.row0, bar);
+                    if (PHASE == 1) {
+                        tma_load_2d(b_dst, map_b, kb * kBK, it.b_row, bar);                     // 128 rows of W_g
+                        tma_load_2d(b_dst + kBBytes / 2, map_b, kb * kBK, it.b_row + p.F, bar); // 128 rows of W_u
+                    } else {
+                        tma_load_2d(b_dst, map_b, kb * kBK, it.b_row, bar);                     // 256 rows of W_d
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ============================================================ MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = instr_desc_bf16(kBM, kBN);
+            uint32_t n = 0, item = 0;
+            for (int w = blockIdx.x; w < total_items && !*abort_flag; w += gridDim.x, ++item) {
+                const uint32_t acc = item & 1u;
+                if (item >= 2 && !mbar_wait(tempty0 + 8 * acc, ((item >> 1) - 1u) & 1u, abort_flag))
+                    break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t d_tmem = tmem_base + acc * kBN;
+                bool ok = true;
+                for (int kb = 0; kb < kblocks; ++kb, ++n) {
+                    const uint32_t s = n % kStages;
+                    if (!mbar_wait(full0 + 8 * s, (n / kStages) & 1u, abort_flag)) {
+                        ok = false;
+                        break;
+                    }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t a_addr = ring_s + s * kStageBytes, b_addr = a_addr + kABytes;
+                    const uint64_t a_desc = smem_desc_sw128(a_addr), b_desc = smem_desc_sw128(b_addr);
+#pragma unroll
+                    for (int ks = 0; ks < kBK / 16; ++ks)   // 16 K elements = 32 bytes = 2 descriptor units
+                        umma_bf16(d_tmem, a_desc + 2 * ks, b_desc + 2 * ks, idesc, (kb | ks) != 0);
+                    umma_commit(empty0 + 8 * s);             // the stage is free once these MMAs have read it
+                }
+                if (!ok)
+                    break;
+                umma_commit(tfull0 + 8 * acc);               // the accumulator is complete
+            }
+        }
+    } else {
+        // ============================================================ epilogue (warps 2..5)
+        const int quarter = warp & 3;                        // the 32 accumulator rows this warp may read
+        uint32_t item = 0;
+        for (int w = blockIdx.x; w < total_items && !*abort_flag; w += gridDim.x, ++item) {
+            const GemmItem it = item_of(w);
+            const uint32_t acc = item & 1u;
+            if (!mbar_wait(tfull0 + 8 * acc, (item >> 1) & 1u, abort_flag))
+                break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const int row = it.row0 + quarter * 32 + lane;
+            const bool live = row < it.row_end;
+            const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * kBN;
+            if (PHASE == 1) {
+#pragma unroll 1
+                for (int c = 0; c < 128; c += 32) {
+                    uint32_t g[32], u[32];
+                    tmem_ld32(t_row + c, g);
+                    tmem_ld32(t_row + 128 + c, u);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                    if (live) {
+                        uint4 *dst = reinterpret_cast<uint4 *>(p.hs + (size_t)row * p.F + it.n0 + c);
+#pragma unroll
+                        for (int v = 0; v < 4; ++v) {
+                            uint32_t o[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const float g0 = __uint_as_float(g[v * 8 + 2 * e]), g1 = __uint_as_float(g[v * 8 + 2 * e + 1]);
+                                const float u0 = __uint_as_float(u[v * 8 + 2 * e]), u1 = __uint_as_float(u[v * 8 + 2 * e + 1]);
+                                const float h0 = g0 / (1.0f + __expf(-g0)) * u0, h1 = g1 / (1.0f + __expf(-g1)) * u1;
+                                o[e] = bf16_rne(h0) | (bf16_rne(h1) << 16);
+                            }
+                            dst[v] = make_uint4(o[0], o[1], o[2], o[3]);
+                        }
+                    }
+                }
+            } else {
+#pragma unroll 1
+                for (int c = 0; c < kBN; c += 32) {
+                    uint32_t z[32];
+                    tmem_ld32(t_row + c, z);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                    if (live) {
+                        uint4 *dst = reinterpret_cast<uint4 *>(p.zs + (size_t)row * p.d + it.n0 + c);
+#pragma unroll
+                        for (int v = 0; v < 8; ++v)
+                            dst[v] = make_uint4(z[4 * v], z[4 * v + 1], z[4 * v + 2], z[4 * v + 3]);
+                    }
+                }
+            }
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0)
+                mbar_arrive(tempty0 + 8 * acc);
+        }
+    }
+
+    // ---- everyone is done with tensor memory: free it
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if (warp == 2)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512));
+    if (*abort_flag && tid == 0)
+        atomicExch(p.err, MELINOE_ERR_TIMEOUT);
+}
+
+// Xs[pos] = hidden[tok_of_sorted[pos]], one block per sorted row.
+__global__ void __launch_bounds__(256) gather_rows_kernel(const DevPlan *plan, const uint16_t *__restrict__ x,
+                                                          const int32_t *__restrict__ tok_of_sorted, uint16_t *xs, int d,
+                                                          int n_sorted)
+{
+    if (plan->status != MELINOE_OK)
+        return;
+    for (int pos = blockIdx.x; pos < n_sorted; pos += gridDim.x) {
+        const uint4 *src = reinterpret_cast<const uint4 *>(x + (size_t)tok_of_sorted[pos] * d);
+        uint4 *dst = reinterpret_cast<uint4 *>(xs + (size_t)pos * d);
+        for (int i = threadIdx.x; i < d / 8; i += 256)
+            dst[i] = src[i];
+    }
+}
+
+// y_t = sum_j gate[t][j] * Z[inv_pos[t*k+j]] + sum_s Z[T*k + s*T + t], fp32 in rank order, bf16 out.
+__global__ void __launch_bounds__(256) combine_rows_kernel(const DevPlan *plan, const float *__restrict__ gate,
+                                                           const int32_t *__restrict__ inv_pos, const float *__restrict__ zs,
+                                                           uint16_t *out, int T, int d, int k, int n_shared)
+{
+    const bool ok = plan->status == MELINOE_OK;
+    for (int t = blockIdx.x; t < T; t += gridDim.x) {
+        for (int c = threadIdx.x * 4; c < d; c += 256 * 4) {
+            float4 y = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (ok) {
+                for (int j = 0; j < k; ++j) {
+                    const float gw = gate[t * k + j];
+                    const float4 z = *reinterpret_cast<const float4 *>(zs + (size_t)inv_pos[t * k + j] * d + c);
+                    y.x = fmaf(gw, z.x, y.x);
+                    y.y = fmaf(gw, z.y, y.y);
+                    y.z = fmaf(gw, z.z, y.z);
+                    y.w = fmaf(gw, z.w, y.w);
+                }
+                for (int s = 0; s < n_shared; ++s) {
+                    const float4 z = *reinterpret_cast<const float4 *>(zs + ((size_t)T * k + (size_t)s * T + t) * d + c);
+                    y.x += z.x;
+                    y.y += z.y;
+                    y.z += z.z;
+                    y.w += z.w;
+                }
+            }
+            uint2 o;
+            o.x = bf16_rne(y.x) | (bf16_rne(y.y) << 16);
+            o.y = bf16_rne(y.z) | (bf16_rne(y.w) << 16);
+            *reinterpret_cast<uint2 *>(out + (size_t)t * d + c) = o;
+        }
+    }
+}
+
+constexpr size_t kGemmSmem = (size_t)kStages * kStageBytes + 1024;
+
+}  // namespace
+
+bool ffn_gemm_supported(int d, int F) { return d % kBN == 0 && F % 128 == 0 && d >= kBN && F >= 128; }
+
+cudaError_t ffn_gemm_configure()
+{
+    cudaError_t e = cudaFuncSetAttribute(ffn_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmem);
+    if (e != cudaSuccess)
+        return e;
+    return cudaFuncSetAttribute(ffn_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmem);
+}
+
+cudaError_t launch_gather_rows(cudaStream_t stream, const DevPlan *plan, const uint16_t *x, const int32_t *tok_of_sorted,
+                               uint16_t *xs, int d, int n_sorted, int n_sms)
+{
+    const int grid = n_sorted < n_sms * 16 ? n_sorted : n_sms * 16;
+    gather_rows_kernel<<<grid, 256, 0, stream>>>(plan, x, tok_of_sorted, xs, d, n_sorted);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_ffn_gemm(cudaStream_t stream, int phase, int n_sms, const GemmParams &p)
+{
+    if (phase == 1)
+        ffn_gemm_kernel<1><<<n_sms, kGemmThreads, kGemmSmem, stream>>>(p);
+    else
+        ffn_gemm_kernel<2><<<n_sms, kGemmThreads, kGemmSmem, stream>>>(p);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_combine_rows(cudaStream_t stream, const DevPlan *plan, const float *gate, const int32_t *inv_pos,
+                                const float *zs, uint16_t *out, int T, int d, int k, int n_shared, int n_sms)
+{
+    const int grid = T < n_sms * 8 ? T : n_sms * 8;
+    combine_rows_kernel<<<grid, 256, 0, stream>>>(plan, gate, inv_pos, zs, out, T, d, k, n_shared);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace melinoe

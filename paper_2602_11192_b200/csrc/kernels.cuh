@@ -1,5 +1,6 @@
 // Launch interfaces of the library's kernels (all sm_100a, all launched by api.cu).
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -73,5 +74,24 @@ cudaError_t ffn_stream_configure(int n_sms, size_t max_smem, FfnLaunchCfg *cfg);
 cudaError_t ffn_stream_geometry(const FfnLaunchCfg &cfg, int d, int F, int T, FfnGeometry *geo);
 cudaError_t launch_ffn_stream(cudaStream_t stream, const FfnLaunchCfg &cfg, const FfnGeometry &geo,
                               const FfnParams &p);
+
+// ---- grouped GEMM expert FFN on tcgen05 for calls with many tokens per expert (prefill)
+// Tensor maps in device memory, in this order:
+enum { kMapXs = 0, kMapHs = 1, kMapSlotsD = 2, kMapSlotsF = 3, kMapShared0 = 4, kMapCount = kMapShared0 + 2 * kMaxShared };
+struct GemmParams {
+    const DevPlan *plan;
+    const CUtensorMap *maps;         // device array of kMapCount tensor maps
+    uint16_t *hs;                    // h, [sorted rows][F] bf16
+    float *zs;                       // expert outputs, [sorted rows][d] fp32
+    int *err;
+    int group, d, F, E, n_shared;
+};
+bool ffn_gemm_supported(int d, int F);
+cudaError_t ffn_gemm_configure();
+cudaError_t launch_gather_rows(cudaStream_t stream, const DevPlan *plan, const uint16_t *x, const int32_t *tok_of_sorted,
+                               uint16_t *xs, int d, int n_sorted, int n_sms);
+cudaError_t launch_ffn_gemm(cudaStream_t stream, int phase, int n_sms, const GemmParams &p);
+cudaError_t launch_combine_rows(cudaStream_t stream, const DevPlan *plan, const float *gate, const int32_t *inv_pos,
+                                const float *zs, uint16_t *out, int T, int d, int k, int n_shared, int n_sms);
 
 }  // namespace melinoe

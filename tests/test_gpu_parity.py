@@ -110,6 +110,32 @@ def test_prefill_then_decode_with_waves():
     P.close()
 
 
+@pytest.mark.parametrize("d,F,E,k,C,n_shared,Ts", [
+    (512, 256, 8, 2, 8, 0, (40, 300, 9)),        # everything fits the cache: one compute group after warm-up
+    (256, 128, 16, 4, 5, 0, (130, 64)),          # more distinct experts than slots: miss waves
+    (1024, 384, 6, 2, 3, 2, (257, 20)),          # shared experts, ragged last m-tile
+])
+def test_prefill_grouped_gemm(d, F, E, k, C, n_shared, Ts):
+    """Calls of more than 8 tokens run the tensor-core grouped GEMM (d_ff a multiple of 128)."""
+    P = _pair(d, F, E, k, C, seed=200 + d // 256, n_shared=n_shared)
+    n_seq = 4
+    bias = _bias(21, E, 0.5, n_seq)
+    step = 0
+    for T in Ts:
+        P.set_bias(bias, (np.arange(T) % n_seq).astype(np.int32))
+        x = gen.hidden_states(300 + d, 0, "prefill", step, T, d)
+        # the oracle evaluates a spread of tokens (first, last and every 7th): the FFN is per token
+        tokens = sorted(set([0, 1, T - 2, T - 1] + list(range(0, T, 7))))
+        P.step(x, tokens=tokens)
+        assert P.gpu.layer.last_call_used_gemm()
+        step += 1
+    # and decode-sized calls on the same handle afterwards (streaming kernel), sharing the cache state
+    P.set_bias(bias, np.zeros(2, np.int32))
+    P.step(gen.hidden_states(300 + d, 0, "decode", 0, 2, d))
+    assert not P.gpu.layer.last_call_used_gemm()
+    P.close()
+
+
 def test_forward_host_matches_forward_and_is_deterministic():
     import torch
     from paper_2602_11192_b200.runner import current_stream_ptr
