@@ -1,0 +1,99 @@
+"""Parity at the benchmark's sizes: the synthetic stacks of the five workload shapes, driven the
+way bench.py drives them (one handle per layer, device-resident inputs), against the oracle.
+
+Routing indices, gates, request traces and statistics are compared for every call (they are
+cheap to recompute on the CPU); activations are compared on a sample of (layer, token) pairs,
+which is sound because a token's output depends only on its inputs and routing, never on the
+cache state.  The largest shapes run with a reduced number of layers (each layer is an
+independent handle; their full width and call shapes are kept).
+"""
+import numpy as np
+import pytest
+
+import gen
+import oracle
+
+pytestmark = pytest.mark.gpu
+
+REL_TOL = 2e-2          # the specified bound at full size
+
+
+def _run_stack(name, n_layers, alpha, C, decode_steps, sample_layers, prefill=True, y_tokens=3):
+    import torch
+    from paper_2602_11192_b200.workload import Stack, bits_of, stats_rows
+    cfg = gen.config_by_name(name)
+    st = Stack(cfg, alpha, C, n_layers=n_layers)
+    L, B, k, E, d = st.L, cfg.batch, cfg.top_k, cfg.n_experts, cfg.d_model
+    caches = [oracle.ExpertCache(C, E) for _ in range(L)]
+    weights = {}
+    for l in sample_layers:
+        wg, wu, wd = st.layer_weights(l)
+        weights[l] = ([(bits_of(wg[e]), bits_of(wu[e]), bits_of(wd[e])) for e in range(E + cfg.n_shared)], (wg, wu, wd))
+
+    def check(phase, step, T, seq):
+        x = st.hidden_bits(phase, step)                                  # [L][T][d]
+        xd = torch.from_numpy(x.view(np.int16)).cuda()
+        out = torch.empty_like(xd)
+        stats = torch.zeros((L, 12), dtype=torch.int32, device="cuda")
+        st.set_phase(phase)
+        st.forward_all(xd, out, stats)
+        torch.cuda.synchronize()
+        out_bits = out.cpu().numpy().view(np.uint16)
+        sr = stats_rows(stats)
+        worst = 0.0
+        for l in range(L):
+            idx_o, gate_o, lg_o = oracle.route(x[l], st.w_r[l], k, st.bias[l], seq)
+            req_o = caches[l].call(idx_o)
+            layer = st.layers[l].layer
+            idx_g, gate_g = layer.last_routing(T)
+            assert np.array_equal(idx_g, idx_o), "routing differs: %s layer %d %s step %d" % (name, l, phase, step)
+            assert np.allclose(gate_g, gate_o, rtol=1e-5, atol=1e-7)
+            assert np.array_equal(layer.last_requests(), req_o), "trace differs: %s layer %d" % (name, l)
+            hits = int(req_o[:, 2].sum())
+            assert sr["status"][l] == 0 and sr["n_distinct"][l] == len(req_o)
+            assert sr["hits"][l] == hits and sr["misses"][l] == len(req_o) - hits
+            assert layer.last_call_used_gemm() == (T > 8 and cfg.d_ff % 128 == 0)
+            if l in weights:
+                toks = sorted(set(np.linspace(0, T - 1, min(T, y_tokens)).astype(int).tolist()))
+                y = oracle.ffn_combine(x[l], idx_o, gate_o, weights[l][0], cfg.d_ff, cfg.n_shared, toks)
+                yg = gen.bf16_bits_to_f32(out_bits[l][toks]).astype(np.float64)
+                err = np.linalg.norm(yg - y, axis=1) / np.maximum(np.linalg.norm(y, axis=1), 1e-30)
+                assert np.all(np.isfinite(yg)) and err.max() <= REL_TOL, "rel err %.3e" % err.max()
+                worst = max(worst, float(err.max()))
+        return worst
+
+    if prefill and cfg.prefill_tokens:
+        check("prefill", 0, B * cfg.prefill_tokens, st.prefill_seq)
+    for s in range(decode_steps):
+        check("decode", s, B, st.decode_seq)
+    tot = [st.layers[l].layer.cache_state()[1] for l in range(L)]
+    for l in range(L):
+        _, _, t_o = caches[l].state()
+        assert tot[l] == t_o
+    st.close()
+
+
+def test_olmoe_full_stack_as_benchmarked():
+    """configs[1]: all 16 layers, 16 slots per layer, the prompt and the first decode steps."""
+    _run_stack("olmoe", None, 0.1, 16, decode_steps=12, sample_layers=(0, 7, 15))
+
+
+def test_olmoe_near_uniform_routing_thrashes_the_cache():
+    _run_stack("olmoe", 2, 10.0, 16, decode_steps=6, sample_layers=(1,))
+
+
+def test_mixtral_shape_two_slots():
+    """configs[2]: d 4096, d_ff 14336, 8 experts, top-2, 2 slots; one layer of the 32."""
+    _run_stack("mixtral", 1, 0.2, 2, decode_steps=4, sample_layers=(0,), y_tokens=2)
+
+
+def test_phi35_shape_batch_of_eight():
+    """configs[3]: d 4096, d_ff 6400, 16 experts, top-2, 6 slots, 8 sequences: 4096-token prefill
+    through the grouped GEMM, then decode steps of 8 tokens; one layer of the 32."""
+    _run_stack("phi35", 1, 0.3, 6, decode_steps=3, sample_layers=(0,), y_tokens=3)
+
+
+def test_deepseek_shape_with_shared_experts():
+    """configs[4]: d 2048, d_ff 1408, 64 routed + 2 shared experts, top-6, 12 slots, 4 sequences:
+    8192-token prefill, then decode steps of 4 tokens; one layer of the 28."""
+    _run_stack("deepseek", 1, 0.1, 12, decode_steps=3, sample_layers=(0,), y_tokens=3)
