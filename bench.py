@@ -128,6 +128,24 @@ class ClockSampler:
         return out
 
 
+# --------------------------------------------------------------------------- ranks
+
+def max_over_ranks(value: float, dist=None, device="cpu") -> float:
+    """The slowest rank's time: every rank runs an independent replica, the job is as slow as the
+    slowest of them.  dist is torch.distributed (initialised) or None for a single process."""
+    if dist is None:
+        return float(value)
+    import torch
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput(tokens_per_rank: int, world: int, ms: float) -> float:
+    """Whole-job tokens/s of `world` replicas that each processed tokens_per_rank tokens in ms."""
+    return tokens_per_rank * world / (ms * 1e-3)
+
+
 # --------------------------------------------------------------------------- our arm
 
 def run_ours(args):
@@ -248,13 +266,6 @@ def run_ours(args):
             raise SystemExit("device-side status %d in the timed region" % int(st["status"].max()))
         return ms, launches, st, ffn_ms, ffn_n
 
-    def max_over_ranks(v):
-        if dist is None:
-            return v
-        t = torch.tensor([v], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
-
     gpu_index = local
     vis = os.environ.get("CUDA_VISIBLE_DEVICES")
     if vis:
@@ -268,9 +279,9 @@ def run_ours(args):
     phase("timed region: %d warm-up + %d decode steps, device-resident inputs" % (W, K))
     ms, launches, st, _, _ = timed_device(alpha0)
     clocks = sampler.stop() if rank == 0 else None
-    ms = max_over_ranks(ms)
+    ms = max_over_ranks(ms, dist, "cuda")
     tokens = cfg.batch * K * world
-    value = tokens / (ms * 1e-3)
+    value = job_throughput(cfg.batch * K, world, ms)
 
     # ---- end to end: host buffers in, host buffers out, one synchronisation per decode step
     phase("end-to-end region: host buffers, %.1f ms/step on the device path" % (ms / K))
@@ -289,7 +300,7 @@ def run_ours(args):
     e1.record()
     torch.cuda.synchronize()
     barrier()
-    e2e_ms = max_over_ranks(e0.elapsed_time(e1))
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1), dist, "cuda")
     e2e = {"value": tokens / (e2e_ms * 1e-3), "unit": UNIT,
            "h2d_bytes_per_step": L * cfg.batch * d * 2,
            "d2h_bytes_per_step": L * (cfg.batch * d * 2 + 48),
