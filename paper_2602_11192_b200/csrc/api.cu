@@ -365,8 +365,8 @@ int melinoe_moe_create(int d, int F, int E, int k, int C, melinoe_moe_t **out)
     CR(cudaMalloc(&h->cache, sizeof(DevCache)));
     CR(cudaMalloc(&h->plan, sizeof(DevPlan)));
     CR(cudaMalloc(&h->err_word, 256));
-    CR(cudaMalloc(&h->sync, sizeof(unsigned) * 2 * (kMaxGroups + 1)));
-    CR(cudaMemset(h->sync, 0, sizeof(unsigned) * 2 * (kMaxGroups + 1)));
+    CR(cudaMalloc(&h->sync, sizeof(unsigned) * (2 * (kMaxGroups + 1) + 1)));
+    CR(cudaMemset(h->sync, 0, sizeof(unsigned) * (2 * (kMaxGroups + 1) + 1)));
     CR(cudaMalloc(&h->shared_dev, sizeof(char *) * kMaxShared));
     CR(cudaMalloc(&h->stage_stats, sizeof(melinoe_moe_stats)));
     CR(cudaMemset(h->err_word, 0, 256));
@@ -572,7 +572,7 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
     pp.vr_capacity = h->vr_capacity;
     if (route_plan_small_supported(T, h->k, h->d)) {
         CU_TRY(launch_route_plan_small(s, static_cast<const uint16_t *>(hidden_dev), h->w_router, h->bias, h->token_seq,
-                                       h->d, h->idx, h->gate, h->logits, pp));
+                                       h->d, h->idx, h->gate, h->logits, h->sync + 2 * (kMaxGroups + 1), pp));
     } else {
         CU_TRY(launch_router(s, static_cast<const uint16_t *>(hidden_dev), h->w_router, h->bias, h->token_seq, T, h->d,
                              h->E, h->k, h->idx, h->gate, h->logits));

@@ -41,7 +41,7 @@ cudaError_t launch_plan(cudaStream_t stream, const PlanParams &p);
 bool route_plan_small_supported(int T, int k, int d);
 cudaError_t launch_route_plan_small(cudaStream_t stream, const uint16_t *x, const uint16_t *w_r, const float *bias,
                                     const int32_t *token_seq, int d, int32_t *idx, float *gate, float *logits_out,
-                                    const PlanParams &p);
+                                    unsigned *ticket, const PlanParams &p);
 
 // ---- streaming expert FFN (Eq. 3) with the gate-weighted combine (Eq. 2) fused in
 struct FfnParams {

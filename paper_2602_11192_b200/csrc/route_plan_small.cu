@@ -1,109 +1,131 @@
-// Router (Eq. 1) and planning fused into one single-block kernel for calls of at most 8 tokens
-// (decode): logits, top-k with lowest-index tie-breaking, renormalised gates, token-to-expert
-// lists, slot lookup with LRU eviction, compute groups, miss queue and statistics.
+// Router (Eq. 1) and planning fused into one kernel for calls of at most 8 tokens (decode):
+// logits, top-k with lowest-index tie-breaking, renormalised gates, token-to-expert lists, slot
+// lookup with LRU eviction, compute groups, miss queue and statistics.
 //
-// At this size every step is latency, not throughput: the router matrix (E x d bf16, a few
-// hundred KB) is pulled by one SM with all 32 warps loading at once, and everything after it
-// works on at most 64 (token, rank) pairs, so one kernel without any device-wide hand-over
-// replaces two launches.  The results are exactly those of the general router and planning
-// kernels: the logit sum uses the same fixed order (element j belongs to lane (j mod 256) / 8,
-// lanes add their elements in increasing j, xor-butterfly 16, 8, 4, 2, 1, bias last), and the
-// cache requests follow the same rules (hits in ascending expert id, then misses in ascending
-// id; a miss takes the lowest empty slot, else the least recently stamped one).
+// At this size every step is latency, not throughput, so the kernel is organised to take as
+// few dependent memory round trips as possible:
+//   - logits: one warp per expert, spread over E/4 blocks (a single SM pulling the whole router
+//     matrix takes ~9 us; sixteen SMs take ~2); each lane has all its loads in flight at once;
+//   - the block that finishes last (a ticket counter) does the rest, so there is no second launch;
+//   - planning is written for one warp with lane = expert / slot / request: ranks come from
+//     ballots and population counts, prefix sums from shuffles, and the LRU victims of a call are
+//     taken from one sorted list instead of one search per miss.
+//
+// The results are exactly those of the general router and planning kernels.  The logit sum uses
+// the same fixed order (element j belongs to lane (j mod 256) / 8, lanes add their elements in
+// increasing j, xor-butterfly 16, 8, 4, 2, 1, bias last).  The cache requests follow the same
+// rules (hits in ascending expert id, then misses in ascending id; a miss takes the lowest empty
+// slot, else the least recently stamped one), restated in closed form:
+//   - hit number r (ascending id) stamps its slot with counter + r + 1;
+//   - let V be the slots ordered by (empty first, by index), then by stamp after the hits were
+//     stamped.  Miss number i (ascending id) takes V[i mod C], because every slot it could prefer
+//     has either been taken by an earlier miss (and stamped newer) or comes later in V;
+//   - the expert it displaces is V[i]'s occupant at call entry for i < C, and miss i - C otherwise;
+//   - miss i belongs to compute group 1 + i / C: a new wave starts exactly when a miss would
+//     overwrite an expert of the current wave, which is every C misses; it must wait for group
+//     i / C (i >= C), for group 0 if it displaces one of the call's hits, for nothing otherwise.
 #include "kernels.cuh"
 
 namespace melinoe {
 
 namespace {
 
-constexpr int kThreads = 1024;
-constexpr int kWarps = kThreads / 32;
+constexpr int kWarpsPerBlock = 4;
+constexpr int kThreads = kWarpsPerBlock * 32;
 constexpr int kMaxT = kTokPerVr;                 // 8 tokens
 constexpr int kMaxPairs = kMaxExperts;           // T * k <= 64 is required by the launcher
 
 __device__ __forceinline__ float bf16lo(uint32_t v) { return __uint_as_float(v << 16); }
 __device__ __forceinline__ float bf16hi(uint32_t v) { return __uint_as_float(v & 0xffff0000u); }
 
-__global__ void __launch_bounds__(kThreads, 1)
+__device__ __forceinline__ int warp_excl_scan(int v, int lane, int &total)
+{
+    int inc = v;
+#pragma unroll
+    for (int m = 1; m < 32; m <<= 1) {
+        const int o = __shfl_up_sync(0xffffffffu, inc, m);
+        if (lane >= m)
+            inc += o;
+    }
+    total = __shfl_sync(0xffffffffu, inc, 31);
+    return inc - v;
+}
+
+__device__ __forceinline__ uint64_t ballot64(bool lo, bool hi)
+{
+    return (uint64_t)__ballot_sync(0xffffffffu, lo) | ((uint64_t)__ballot_sync(0xffffffffu, hi) << 32);
+}
+
+__device__ __forceinline__ int rank_below(uint64_t mask, int bit) { return __popcll(mask & ((1ull << bit) - 1ull)); }
+
+// The virtual request of one expert (at most 8 tokens here): its tokens and z rows from the sorted lists.
+__device__ __forceinline__ void write_vr(VrRec *dst, const char *blob, int n_tok, int group, int off, int k,
+                                         const int32_t *pair_at)
+{
+    VrRec vr;
+    vr.blob = blob;
+    vr.n_tok = n_tok;
+    vr.group = group;
+#pragma unroll
+    for (int j = 0; j < kTokPerVr; ++j) {
+        const int pr = j < n_tok ? pair_at[off + j] : -1;
+        vr.tok[j] = pr >= 0 ? pr / k : -1;
+        vr.pair[j] = pr;
+    }
+    *dst = vr;
+}
+
+__global__ void __launch_bounds__(kThreads)
 route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restrict__ w_r,
                         const float *__restrict__ bias, const int32_t *__restrict__ token_seq, int d,
-                        int32_t *__restrict__ idx_out, float *__restrict__ gate_out,
-                        float *__restrict__ logits_out, PlanParams p)
+                        int32_t *__restrict__ idx_out, float *__restrict__ gate_out, float *logits_out,
+                        unsigned *ticket, PlanParams p)
 {
-    extern __shared__ __align__(16) unsigned char dyn[];
-    uint4 *xs = reinterpret_cast<uint4 *>(dyn);                  // [T][d / 8]
     __shared__ float s_logit[kMaxT][kMaxExperts];
     __shared__ int32_t s_idx[kMaxPairs];
-    __shared__ int32_t s_pos[kMaxPairs];                         // sorted position of pair q
     __shared__ int32_t s_pair_at[kMaxPairs];                     // pair at sorted position
-    __shared__ int32_t s_counts[kMaxReq];
-    __shared__ int32_t s_offsets[kMaxReq + 1];
-    __shared__ __align__(16) DevCache s_cache;
-    __shared__ int32_t s_group_of_expert[kMaxExperts];
-    __shared__ int32_t s_req_of_expert[kMaxReq];
-    __shared__ ReqRec s_req[kMaxReq];
-    __shared__ HostMiss s_miss[kMaxExperts];
-    __shared__ int32_t s_group_vr_begin[kMaxGroups + 1];
+    __shared__ unsigned long long s_key[kMaxExperts];            // victim-order key of a slot
+    __shared__ int32_t s_victim[kMaxExperts];                    // V: slots in victim order
+    __shared__ int32_t s_miss_expert[kMaxExperts];               // expert of miss number i
+    __shared__ int32_t s_entry_occ[kMaxExperts];                 // occupant of a slot at call entry
+    __shared__ int s_last;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int T = p.T, k = p.k, E = p.E, C = p.C;
     const int n_pairs = T * k;
-    const int dv = d >> 3;                                       // uint4 per row
 
-    // ---- stage the hidden rows; warp 0 fetches the cache state meanwhile
-    for (int i = tid; i < T * dv; i += kThreads)
-        xs[i] = reinterpret_cast<const uint4 *>(x)[i];
-    if (warp == 1) {
-        const uint4 *src = reinterpret_cast<const uint4 *>(p.cache);
-        uint4 *dst = reinterpret_cast<uint4 *>(&s_cache);
-        for (int i = lane; i < (int)(sizeof(DevCache) / 16); i += 32)
-            dst[i] = src[i];
-    }
-    for (int i = tid; i < 2 * (kMaxGroups + 1); i += kThreads)
-        p.sync[i] = 0u;
-    __syncthreads();
-
-    // ---- logits: warp w computes experts w and w + 32 for every token.  The weight row pieces
-    // of a lane are fetched eight at a time before any arithmetic, so that a row costs one
-    // memory latency instead of one per piece.
-    const int n_chunks = d >> 8;
-    for (int e = warp; e < E; e += kWarps) {
-        float acc[kMaxT];
+    // ================================================================ logits: one warp per expert
+    {
+        const int e = blockIdx.x * kWarpsPerBlock + warp;
+        if (e < E) {
+            const int n_chunks = d >> 8;
+            const uint4 *wrow = reinterpret_cast<const uint4 *>(w_r + (size_t)e * d) + lane;
+            for (int t = 0; t < T; ++t) {
+                const uint4 *xrow = reinterpret_cast<const uint4 *>(x + (size_t)t * d) + lane;
+                float a = 0.0f;
+                for (int c0 = 0; c0 < n_chunks; c0 += 8) {
+                    // all of a lane's loads for these 8 pieces go out before any arithmetic
+                    uint4 wv[8], xv[8];
 #pragma unroll
-        for (int t = 0; t < kMaxT; ++t)
-            acc[t] = 0.0f;
-        const uint4 *wrow = reinterpret_cast<const uint4 *>(w_r + (size_t)e * d) + lane;
-        for (int c0 = 0; c0 < n_chunks; c0 += 8) {
-            uint4 wv[8];
+                    for (int i = 0; i < 8; ++i) {
+                        const bool on = c0 + i < n_chunks;
+                        wv[i] = on ? __ldg(wrow + (c0 + i) * 32) : make_uint4(0, 0, 0, 0);
+                        xv[i] = on ? __ldg(xrow + (c0 + i) * 32) : make_uint4(0, 0, 0, 0);
+                    }
 #pragma unroll
-            for (int i = 0; i < 8; ++i)
-                wv[i] = c0 + i < n_chunks ? __ldg(wrow + (c0 + i) * 32) : make_uint4(0, 0, 0, 0);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                if (c0 + i < n_chunks) {
-#pragma unroll
-                    for (int t = 0; t < kMaxT; ++t) {
-                        if (t < T) {
-                            const uint4 xv = xs[t * dv + (c0 + i) * 32 + lane];
-                            float a = acc[t];
-                            a = __fmaf_rn(bf16lo(xv.x), bf16lo(wv[i].x), a);
-                            a = __fmaf_rn(bf16hi(xv.x), bf16hi(wv[i].x), a);
-                            a = __fmaf_rn(bf16lo(xv.y), bf16lo(wv[i].y), a);
-                            a = __fmaf_rn(bf16hi(xv.y), bf16hi(wv[i].y), a);
-                            a = __fmaf_rn(bf16lo(xv.z), bf16lo(wv[i].z), a);
-                            a = __fmaf_rn(bf16hi(xv.z), bf16hi(wv[i].z), a);
-                            a = __fmaf_rn(bf16lo(xv.w), bf16lo(wv[i].w), a);
-                            a = __fmaf_rn(bf16hi(xv.w), bf16hi(wv[i].w), a);
-                            acc[t] = a;
+                    for (int i = 0; i < 8; ++i) {
+                        if (c0 + i < n_chunks) {
+                            a = __fmaf_rn(bf16lo(xv[i].x), bf16lo(wv[i].x), a);
+                            a = __fmaf_rn(bf16hi(xv[i].x), bf16hi(wv[i].x), a);
+                            a = __fmaf_rn(bf16lo(xv[i].y), bf16lo(wv[i].y), a);
+                            a = __fmaf_rn(bf16hi(xv[i].y), bf16hi(wv[i].y), a);
+                            a = __fmaf_rn(bf16lo(xv[i].z), bf16lo(wv[i].z), a);
+                            a = __fmaf_rn(bf16hi(xv[i].z), bf16hi(wv[i].z), a);
+                            a = __fmaf_rn(bf16lo(xv[i].w), bf16lo(wv[i].w), a);
+                            a = __fmaf_rn(bf16hi(xv[i].w), bf16hi(wv[i].w), a);
                         }
                     }
                 }
-            }
-        }
-#pragma unroll
-        for (int t = 0; t < kMaxT; ++t) {
-            if (t < T) {
-                float a = acc[t];
 #pragma unroll
                 for (int m = 16; m >= 1; m >>= 1)
                     a = __fadd_rn(a, __shfl_xor_sync(0xffffffffu, a, m));
@@ -112,18 +134,30 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
                         const int q = token_seq ? token_seq[t] : 0;
                         a = __fadd_rn(a, bias[(size_t)q * E + e]);
                     }
-                    s_logit[t][e] = a;
-                    if (logits_out)
-                        logits_out[(size_t)t * E + e] = a;
+                    logits_out[(size_t)t * E + e] = a;
                 }
             }
         }
     }
+    // ---- the block that finishes last carries on
+    __threadfence();
+    __syncthreads();
+    if (tid == 0)
+        s_last = atomicAdd(ticket, 1u) == gridDim.x - 1;
+    __syncthreads();
+    if (!s_last)
+        return;
+    __threadfence();
+    if (tid == 0)
+        *ticket = 0u;
+    for (int i = tid; i < T * E; i += kThreads)
+        s_logit[i / E][i % E] = __ldcg(logits_out + i);
+    for (int i = tid; i < 2 * (kMaxGroups + 1); i += kThreads)
+        p.sync[i] = 0u;
     __syncthreads();
 
-    // ---- top-k and gates: warp t serves token t.  Lane l holds experts l and l + 32.
-    if (warp < T) {
-        const int t = warp;
+    // ================================================================ top-k and gates: a warp per token
+    for (int t = warp; t < T; t += kWarpsPerBlock) {
         const float NEG = -__int_as_float(0x7f800000);  // -inf
         const float v0 = lane < E ? s_logit[t][lane] : NEG;
         const float v1 = lane + 32 < E ? s_logit[t][lane + 32] : NEG;
@@ -178,169 +212,164 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
     if (warp != 0)
         return;
 
-    // ================================================================ planning, by warp 0
+    // ================================================================ planning, by one warp
+    // lane owns experts lane and lane + 32, slots lane and lane + 32, pairs lane and lane + 32
+    DevCache *cache = p.cache;
+    DevPlan *plan = p.plan;
+    const int e0 = lane, e1 = lane + 32;
+    // cache state of my experts and slots (one round trip, all loads in flight together)
+    const int soe0 = e0 < E ? cache->slot_of_expert[e0] : -1, soe1 = e1 < E ? cache->slot_of_expert[e1] : -1;
+    const int eos0 = lane < C ? cache->expert_of_slot[lane] : -1, eos1 = lane + 32 < C ? cache->expert_of_slot[lane + 32] : -1;
+    const unsigned long long st0 = lane < C ? cache->stamp[lane] : 0ull, st1 = lane + 32 < C ? cache->stamp[lane + 32] : 0ull;
+    const unsigned long long counter = cache->counter;
+    const unsigned long long call_no = cache->call_no + 1ull;
+
     // ---- token lists: counts, offsets, stable positions (pairs in increasing flat index)
-    for (int e = lane; e < kMaxReq; e += 32) {
-        int c = 0;
-        if (e < E)
-            for (int q = 0; q < n_pairs; ++q)
-                c += s_idx[q] == e;
-        else if (e < E + p.n_shared)
-            c = T;
-        s_counts[e] = c;
-        s_req_of_expert[e] = -1;
-    }
-    __syncwarp();
-    if (lane == 0) {
-        int run = 0;
-        for (int e = 0; e < E + p.n_shared; ++e) {
-            s_offsets[e] = run;
-            run += s_counts[e];
-        }
-        s_offsets[E + p.n_shared] = run;
-    }
-    __syncwarp();
-    for (int q = lane; q < n_pairs; q += 32) {
+    int c0 = 0, c1 = 0;
+    for (int q = 0; q < n_pairs; ++q) {
         const int e = s_idx[q];
+        c0 += e == e0;
+        c1 += e == e1;
+    }
+    int tot0, tot1;
+    const int off0 = warp_excl_scan(c0, lane, tot0);
+    const int off1 = tot0 + warp_excl_scan(c1, lane, tot1);
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int q = lane + 32 * h;
+        const int e = q < n_pairs ? s_idx[q] : 0;
         int r = 0;
-        for (int q2 = 0; q2 < q; ++q2)
+        for (int q2 = 0; q2 < q && q2 < n_pairs; ++q2)
             r += s_idx[q2] == e;
-        const int pos = s_offsets[e] + r;
-        s_pos[q] = pos;
-        s_pair_at[pos] = q;
-        p.perm[pos] = q;
-        p.inv_pos[q] = pos;
-        p.tok_of_sorted[pos] = q / k;
+        const int o0 = __shfl_sync(0xffffffffu, off0, e & 31), o1 = __shfl_sync(0xffffffffu, off1, e & 31);
+        if (q < n_pairs) {
+            const int pos = (e < 32 ? o0 : o1) + r;
+            s_pair_at[pos] = q;
+            p.perm[pos] = q;
+            p.inv_pos[q] = pos;
+            p.tok_of_sorted[pos] = q / k;
+        }
     }
     for (int i = lane; i < p.n_shared * T; i += 32)
         p.tok_of_sorted[n_pairs + i] = i % T;
-    __syncwarp();
 
-    // ---- cache requests: hits in ascending expert id, then misses in ascending id
-    uint64_t need = 0, resident = 0;
-    {
-        const bool n0 = lane < E && s_counts[lane] > 0;
-        const bool n1 = lane + 32 < E && s_counts[lane + 32] > 0;
-        const bool r0 = lane < E && s_cache.slot_of_expert[lane] >= 0;
-        const bool r1 = lane + 32 < E && s_cache.slot_of_expert[lane + 32] >= 0;
-        need = (uint64_t)__ballot_sync(0xffffffffu, n0) | ((uint64_t)__ballot_sync(0xffffffffu, n1) << 32);
-        resident = (uint64_t)__ballot_sync(0xffffffffu, r0) | ((uint64_t)__ballot_sync(0xffffffffu, r1) << 32);
-    }
-    int n_req = 0, n_hits = 0, n_miss = 0, n_evict = 0;
-    uint64_t counter = s_cache.counter;
-    for (uint64_t m = need & resident; m; m &= m - 1) {
-        const int e = __ffsll((long long)m) - 1;
-        if (lane == 0) {
-            const int s = s_cache.slot_of_expert[e];
-            s_cache.stamp[s] = ++counter;
-            s_req[n_req] = ReqRec{e, s, 1, -1, s_offsets[e], s_counts[e], 0, 0};
-            s_req_of_expert[e] = n_req;
-            s_group_of_expert[e] = 0;
-        }
-        ++n_req;
-        ++n_hits;
-    }
-    counter = __shfl_sync(0xffffffffu, counter, 0);
-    __syncwarp();
-    int cur_group = 1;
-    for (uint64_t m = need & ~resident; m; m &= m - 1) {
-        const int e = __ffsll((long long)m) - 1;
-        // victim: lowest empty slot, else smallest stamp (stamps are unique)
-        uint64_t key = ~0ull;
-        int slot = -1;
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            const int s = lane + 32 * h;
-            if (s < C) {
-                const uint64_t ks = s_cache.expert_of_slot[s] < 0 ? (uint64_t)s : ((1ull << 63) | s_cache.stamp[s]);
-                if (ks < key) {
-                    key = ks;
-                    slot = s;
-                }
-            }
-        }
-#pragma unroll
-        for (int mm = 16; mm >= 1; mm >>= 1) {
-            const uint64_t ok = __shfl_xor_sync(0xffffffffu, key, mm);
-            const int os = __shfl_xor_sync(0xffffffffu, slot, mm);
-            if (ok < key) {
-                key = ok;
-                slot = os;
-            }
-        }
-        const int ev = s_cache.expert_of_slot[slot];
-        int dep = -1;
-        if (ev >= 0) {
-            ++n_evict;
-            if ((need >> ev) & 1ull)
-                dep = s_group_of_expert[ev];
-        }
-        if (dep == cur_group)
-            ++cur_group;
-        __syncwarp();
-        if (lane == 0) {
-            ++counter;
-            if (ev >= 0)
-                s_cache.slot_of_expert[ev] = -1;
-            s_cache.expert_of_slot[slot] = e;
-            s_cache.slot_of_expert[e] = slot;
-            s_cache.stamp[slot] = counter;
-            s_req[n_req] = ReqRec{e, slot, 0, ev, s_offsets[e], s_counts[e], 0, cur_group};
-            s_req_of_expert[e] = n_req;
-            s_group_of_expert[e] = cur_group;
-            s_miss[n_miss] = HostMiss{e, slot, (int16_t)cur_group, (int16_t)dep, 0u};
-        }
-        counter = __shfl_sync(0xffffffffu, counter, 0);
-        ++n_req;
-        ++n_miss;
-        __syncwarp();
-    }
-    const int n_groups = n_miss ? cur_group + 1 : 1;
-    int n_req_total = n_req;
-    int nvr = 0;
-    int status = MELINOE_OK;
-    if (lane == 0) {
-        for (int s = 0; s < p.n_shared; ++s) {
-            s_req[n_req_total] = ReqRec{E + s, -1, 1, -1, s_offsets[E + s], T, 0, 0};
-            s_req_of_expert[E + s] = n_req_total;
-            ++n_req_total;
-        }
-        // virtual requests (one per request here: at most 8 tokens), grouped: group 0 = hits then
-        // shared, then the miss waves in order
-        s_group_vr_begin[0] = 0;
-        for (int r = 0; r < n_hits; ++r)
-            s_req[r].vr_start = nvr++;
-        for (int r = n_req; r < n_req_total; ++r)
-            s_req[r].vr_start = nvr++;
-        int g = 0;
-        for (int r = n_hits; r < n_req; ++r) {
-            while (g < s_req[r].group)
-                s_group_vr_begin[++g] = nvr;
-            s_req[r].vr_start = nvr++;
-        }
-        while (g < kMaxGroups)
-            s_group_vr_begin[++g] = nvr;
-        if (nvr > p.vr_capacity || n_groups > (int)p.gmax)
-            status = MELINOE_ERR_STATE;
-        if (status != MELINOE_OK) {
-            for (int i = 0; i <= kMaxGroups; ++i)
-                s_group_vr_begin[i] = 0;
-            nvr = 0;
-        }
-        s_cache.counter = counter;
-        s_cache.tot_hits += (uint64_t)n_hits;
-        s_cache.tot_misses += (uint64_t)n_miss;
-        s_cache.tot_evictions += (uint64_t)n_evict;
-        s_cache.call_no += 1;
-        s_cache.tot_vr += (uint64_t)nvr;
-    }
-    n_req_total = __shfl_sync(0xffffffffu, n_req_total, 0);
-    nvr = __shfl_sync(0xffffffffu, nvr, 0);
-    status = __shfl_sync(0xffffffffu, status, 0);
-    __syncwarp();
+    // ---- hits and misses
+    const uint64_t need = ballot64(c0 > 0, c1 > 0);
+    const uint64_t resident = ballot64(soe0 >= 0, soe1 >= 0);
+    const uint64_t hit_mask = need & resident, miss_mask = need & ~resident;
+    const int n_hits = __popcll(hit_mask), n_miss = __popcll(miss_mask), n_req = n_hits + n_miss;
+    const int n_groups = n_miss ? 1 + (n_miss + C - 1) / C : 1;
+    const int nvr = n_req + p.n_shared;
+    const int status = (nvr > p.vr_capacity || n_groups > (int)p.gmax) ? MELINOE_ERR_STATE : MELINOE_OK;
+    const bool ok = status == MELINOE_OK;
 
-    // ---- write the plan, the virtual requests and the cache state back
-    DevPlan *plan = p.plan;
+    // victim-order key of every slot: empty slots by index, then occupied ones by stamp, with the
+    // stamps this call's hits receive
+    s_key[lane] = lane < C ? (eos0 < 0 ? (unsigned long long)lane : ((1ull << 63) | st0)) : ~0ull;
+    s_key[lane + 32] = lane + 32 < C ? (eos1 < 0 ? (unsigned long long)(lane + 32) : ((1ull << 63) | st1)) : ~0ull;
+    s_entry_occ[lane] = eos0;
+    s_entry_occ[lane + 32] = eos1;
+    __syncwarp();
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int e = h ? e1 : e0, soe = h ? soe1 : soe0, cnt = h ? c1 : c0, off = h ? off1 : off0;
+        if ((hit_mask >> e) & 1ull) {
+            const int r = rank_below(hit_mask, e);
+            const unsigned long long st = counter + (unsigned long long)r + 1ull;
+            s_key[soe] = (1ull << 63) | st;
+            cache->stamp[soe] = st;
+            plan->req[r] = ReqRec{e, soe, 1, -1, off, cnt, r, 0};
+            if (ok)
+                write_vr(p.vrs + r, p.slots + (size_t)soe * p.slot_stride, cnt, 0, off, k, s_pair_at);
+        }
+        if ((miss_mask >> e) & 1ull)
+            s_miss_expert[rank_below(miss_mask, e)] = e;
+    }
+    __syncwarp();
+    // V: rank of each slot among the keys (keys are distinct)
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int s = lane + 32 * h;
+        if (s < C) {
+            const unsigned long long mine = s_key[s];
+            int r = 0;
+            for (int s2 = 0; s2 < C; ++s2)
+                r += s_key[s2] < mine;
+            s_victim[r] = s;
+        }
+    }
+    __syncwarp();
+    bool ev_flag[2] = {false, false};
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int e = h ? e1 : e0, cnt = h ? c1 : c0, off = h ? off1 : off0;
+        if ((miss_mask >> e) & 1ull) {
+            const int i = rank_below(miss_mask, e);
+            const int slot = s_victim[i % C];
+            const int ev = i < C ? s_entry_occ[slot] : s_miss_expert[i - C];
+            const int group = 1 + i / C;
+            int dep = -1;
+            if (i >= C)
+                dep = i / C;
+            else if (ev >= 0 && ((need >> ev) & 1ull))
+                dep = 0;
+            ev_flag[h] = ev >= 0;
+            const int vr_at = n_hits + p.n_shared + i;
+            plan->req[n_hits + i] = ReqRec{e, slot, 0, ev, off, cnt, vr_at, group};
+            if (ok)
+                write_vr(p.vrs + vr_at, p.slots + (size_t)slot * p.slot_stride, cnt, group, off, k, s_pair_at);
+            // cache update: the last miss that lands in a slot keeps it
+            const bool stays = i + C >= n_miss;
+            cache->slot_of_expert[e] = stays ? slot : -1;
+            if (stays) {
+                cache->expert_of_slot[slot] = e;
+                cache->stamp[slot] = counter + (unsigned long long)(n_hits + i) + 1ull;
+            }
+            if (i < C && ev >= 0)
+                cache->slot_of_expert[ev] = -1;
+            const HostMiss m{e, slot, (int16_t)group, (int16_t)dep, p.call_seq};
+            store16_host(&p.hplan->miss[i], &m);
+        }
+    }
+    const int n_evict = __popcll(ballot64(ev_flag[0], ev_flag[1]));
+    // shared experts: always resident, group 0, behind the hits
+    for (int s = lane; s < p.n_shared; s += 32) {
+        const int off = n_pairs + s * T;
+        plan->req[n_req + s] = ReqRec{E + s, -1, 1, -1, off, T, n_hits + s, 0};
+        if (ok) {
+            VrRec vr;
+            vr.blob = p.shared_blobs[s];
+            vr.n_tok = T;
+            vr.group = 0;
+            for (int j = 0; j < kTokPerVr; ++j) {
+                vr.tok[j] = j < T ? j : -1;
+                vr.pair[j] = j < T ? off + j : -1;
+            }
+            p.vrs[n_hits + s] = vr;
+        }
+    }
+    // group boundaries, counts and offsets (what the FFN launches and the inspection calls read)
+    for (int g = lane; g <= kMaxGroups; g += 32) {
+        int b = 0;
+        if (ok && g >= 1) {
+            const int done = (g - 1) * C;
+            b = n_hits + p.n_shared + (done < n_miss ? done : n_miss);
+        }
+        plan->group_vr_begin[g] = b;
+    }
+    if (e0 < E) {
+        plan->counts[e0] = c0;
+        plan->offsets[e0] = off0;
+    }
+    if (e1 < E) {
+        plan->counts[e1] = c1;
+        plan->offsets[e1] = off1;
+    }
+    if (lane <= p.n_shared) {
+        if (lane < p.n_shared)
+            plan->counts[E + lane] = T;
+        plan->offsets[E + lane] = n_pairs + lane * T;
+    }
     if (lane == 0) {
         plan->n_tokens = T;
         plan->n_req = n_req;
@@ -348,44 +377,14 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
         plan->n_miss = n_miss;
         plan->n_evict = n_evict;
         plan->n_groups = n_groups;
-        plan->n_vr = nvr;
+        plan->n_vr = ok ? nvr : 0;
         plan->status = status;
-    }
-    for (int i = lane; i <= kMaxGroups; i += 32)
-        plan->group_vr_begin[i] = s_group_vr_begin[i];
-    for (int i = lane; i < kMaxReq; i += 32) {
-        plan->counts[i] = s_counts[i];
-        plan->req_of_expert[i] = s_req_of_expert[i];
-    }
-    for (int i = lane; i <= kMaxReq; i += 32)
-        plan->offsets[i] = i <= E + p.n_shared ? s_offsets[i] : 0;
-    for (int r = lane; r < n_req_total; r += 32) {
-        const ReqRec rec = s_req[r];
-        plan->req[r] = rec;
-        if (status == MELINOE_OK) {
-            VrRec vr;
-            vr.blob = rec.slot >= 0 ? p.slots + (size_t)rec.slot * p.slot_stride : p.shared_blobs[rec.expert - E];
-            vr.n_tok = rec.n_tok;
-            vr.group = rec.group;
-            for (int i = 0; i < kTokPerVr; ++i) {
-                const int pos = rec.tok_off + i;
-                const bool on = i < rec.n_tok;
-                const bool routed = pos < n_pairs;
-                vr.tok[i] = on ? (routed ? s_pair_at[pos] / k : (pos - n_pairs) % T) : -1;
-                vr.pair[i] = on ? (routed ? s_pair_at[pos] : pos) : -1;
-            }
-            p.vrs[rec.vr_start] = vr;
-        }
-    }
-    {
-        uint4 *dst = reinterpret_cast<uint4 *>(p.cache);
-        const uint4 *src = reinterpret_cast<const uint4 *>(&s_cache);
-        for (int i = lane; i < (int)(sizeof(DevCache) / 16); i += 32)
-            dst[i] = src[i];
-    }
-
-    // ---- statistics and the miss queue for the host
-    if (lane == 0) {
+        cache->counter = counter + (unsigned long long)n_req;
+        cache->tot_hits += (unsigned long long)n_hits;
+        cache->tot_misses += (unsigned long long)n_miss;
+        cache->tot_evictions += (unsigned long long)n_evict;
+        cache->call_no = call_no;
+        cache->tot_vr += (unsigned long long)(ok ? nvr : 0);
         if (p.stats) {
             melinoe_moe_stats st;
             st.status = status;
@@ -397,10 +396,11 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
             st.groups = n_groups;
             st.reserved = 0;
             st.bytes_h2d = (uint64_t)n_miss * (uint64_t)p.expert_bytes;
-            st.call_no = s_cache.call_no;
+            st.call_no = call_no;
             *p.stats = st;
         }
-        publish_miss_queue(p.hplan, s_miss, n_miss, n_groups, status, p.call_seq);
+        const HostPlanHeader hdr{n_miss, n_groups, status, p.call_seq};
+        store16_host(&p.hplan->hdr, &hdr);
     }
 }
 
@@ -408,23 +408,16 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
 
 bool route_plan_small_supported(int T, int k, int d)
 {
-    return T >= 1 && T <= kMaxT && T * k <= kMaxPairs && (size_t)T * d * 2 <= 160 * 1024;
+    (void)d;
+    return T >= 1 && T <= kMaxT && T * k <= kMaxPairs;
 }
 
 cudaError_t launch_route_plan_small(cudaStream_t stream, const uint16_t *x, const uint16_t *w_r, const float *bias,
                                     const int32_t *token_seq, int d, int32_t *idx, float *gate, float *logits_out,
-                                    const PlanParams &p)
+                                    unsigned *ticket, const PlanParams &p)
 {
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(route_plan_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             160 * 1024);
-        if (e != cudaSuccess)
-            return e;
-        attr_set = true;
-    }
-    const size_t smem = (size_t)p.T * d * 2;
-    route_plan_small_kernel<<<1, kThreads, smem, stream>>>(x, w_r, bias, token_seq, d, idx, gate, logits_out, p);
+    const int grid = (p.E + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    route_plan_small_kernel<<<grid, kThreads, 0, stream>>>(x, w_r, bias, token_seq, d, idx, gate, logits_out, ticket, p);
     count_launch();
     return cudaGetLastError();
 }
