@@ -22,9 +22,10 @@
 //            ahead of the barrier as far as the ring allows; only the h rows wait for it.
 //   phase 2  every CTA owns a contiguous range of the d_model output rows (d/G of them, so the
 //            split is even to within one row) for ALL virtual requests of the launch.  Tile =
-//            up to 16 of those W_d rows of one virtual request: D[16 x 8] = W_d rows * h^T, a
-//            complete dot product over d_ff, so z needs no cross-CTA reduction; it goes to
-//            z[pair][d] in fp32.
+//            up to 16 of those W_d rows of one virtual request; warp w computes rows w and w + 8
+//            as plain fp32 dot products over d_ff against the h rows (the arithmetic is a few
+//            hundred FMAs per lane and tile), complete sums, so z needs no reduction across
+//            warps or CTAs; it goes to z[pair][d] in fp32.
 //   combine  in the call's last compute group every CTA, having finished its rows, sums
 //            gate * z over the ranks in rank order (plus shared experts) for those rows and
 //            writes them as bf16: it reads only what itself (or an earlier launch) wrote, so
@@ -41,6 +42,8 @@
 // warp raises the CTA's abort flag, later waits fall through, the kernel ends normally and the
 // error word tells the host.
 #include <cstdlib>
+#include <type_traits>
+
 #include "kernels.cuh"
 
 namespace melinoe {
@@ -51,6 +54,7 @@ constexpr int kConsumerWarps = 8;
 constexpr int kProducerWarps = 4;                    // a warp needs ~0.6 us to get one stage's copies out
 constexpr int kThreads = (kConsumerWarps + kProducerWarps) * 32;
 constexpr int kMaxStages = 8;
+constexpr int kMaxSub = 16;                          // sub-stages of the down phase, over the whole ring
 constexpr int kMaxChunk = 4096;                      // bytes of one row piece
 constexpr int kVrShared = 72;                        // virtual-request records kept in shared memory
 // Bound of every wait, in SM clock cycles (about 2 s).  Waits are timed with the SM's cycle
@@ -174,7 +178,16 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
     const int NOP = geo.n_op_rows;
     (void)NOP;
     const int S1 = geo.n_stages, PITCH1 = geo.pitch, CB1 = geo.chunk_bytes, STAGE1 = geo.stage_bytes;
-    const int S2 = S1, PITCH2 = geo.pitch2, CB2 = geo.chunk_bytes2, STAGE2 = STAGE1;
+    // down phase: rows of 2*F bytes.  When a whole row fits one piece, the CTA's rows of an expert
+    // are one contiguous block of global memory and travel as ONE bulk copy (the bulk-copy engine
+    // keeps a limited number of requests in flight, so 2 KB requests stream at half the rate of
+    // 4 KB ones); rows sit unpadded in the stage, which is fine because this phase reads them
+    // with plain 16-byte loads, one row per warp.
+    // A down stage is often much smaller than a gate/up stage (short W_d rows), so a ring slot is
+    // cut into NS2 sub-stages for the down phase: more tiles in flight where each tile is small.
+    const int CB2 = geo.chunk_bytes2, NS2 = geo.sub2, SUB2 = geo.sub_bytes2;
+    const bool contig2 = 2 * F <= CB2;
+    const int PITCH2 = contig2 ? 2 * F : CB2;
 
     // optional timeline: 8 device-clock stamps per CTA (see melinoe_moe_set_trace)
     unsigned long long *trace = p.trace ? p.trace + (size_t)blockIdx.x * 8 : nullptr;
@@ -201,11 +214,15 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
     uint64_t *bars = reinterpret_cast<uint64_t *>(red + 2 * kConsumerWarps * 128);
     const uint32_t ring_s = smem_u32(ring);
     const uint32_t full1 = smem_u32(bars), empty1 = full1 + 8 * kMaxStages;
-    const uint32_t full2 = full1, empty2 = empty1;          // one ring, one stage sequence for both phases
+    const uint32_t full2 = empty1 + 8 * kMaxStages, empty2 = full2 + 8 * kMaxSub;
     volatile int *abort_flag = &s_abort;
 
     if (tid == 0) {
         s_abort = 0;
+        for (int i = 0; i < kMaxSub; ++i) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(full2 + 8 * i), "r"(1));
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(empty2 + 8 * i), "r"(kConsumerWarps));
+        }
         for (int i = 0; i < kMaxStages; ++i) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(full1 + 8 * i), "r"(1));
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(empty1 + 8 * i), "r"(kConsumerWarps));
@@ -221,14 +238,6 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
         for (int i = tid; i < nv * (int)(sizeof(VrRec) / 16); i += kThreads)
             dst[i] = src[i];
         vrs = s_vrs;
-    }
-    if (F % 16 != 0) {
-        // the last 16-column step of a W_d row is half filled: what the copy leaves untouched
-        // must be finite, because it meets the zero padding of the h rows in the product
-        uint4 *z = reinterpret_cast<uint4 *>(ring);
-        for (int i = tid; i < (int)(geo.ring_bytes / 16); i += kThreads)
-            z[i] = make_uint4(0, 0, 0, 0);
-        fence_proxy_async();
     }
     __syncthreads();
     if (trace && tid == 0)
@@ -260,6 +269,21 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
     const int hi2 = nv * mt, hi2A = nvA * mt;                 // down tiles: request-major, half A first
     unsigned *sync_word = p.sync + 2 * p.group;               // [half]
 
+    // Down stage j (counted from 0 within the phase) lives in ring slot (n1 + j / NS2) mod S1, sub-stage
+    // j mod NS2: the slots are taken in the order in which the gate/up phase lets go of them.
+    struct Down {
+        uint32_t slot, bar, use, off;
+    };
+    auto down_stage = [&](uint32_t n1_, uint32_t j) -> Down {
+        Down x;
+        x.slot = (n1_ + j / NS2) % S1;
+        const uint32_t sub = j % NS2;
+        x.bar = x.slot * NS2 + sub;
+        x.use = j / (uint32_t)(S1 * NS2);
+        x.off = x.slot * STAGE1 + sub * SUB2;
+        return x;
+    };
+
     if (warp >= kConsumerWarps) {
         // =================================================================== producers
         // The producer warps walk the same stage sequence and share the stages out (a warp is busy
@@ -277,10 +301,8 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
         // One stage of either phase.  src: this lane's source row or null.  parts bit 0: arm the
         // barrier and fetch the weight rows (the caller has made sure the slot is free); bit 1:
         // operand rows.
-        auto issue = [&](const char *src, uint32_t full0, int S, int STAGE, int PITCH, size_t src_off, int wbytes,
-                         int obytes, int parts, uint32_t nn) {
-            const uint32_t slot = nn % S;
-            const uint32_t bar = full0 + 8 * slot;
+        auto issue = [&](const char *src, uint32_t bar, uint32_t stage_off, int PITCH, size_t src_off, int wbytes,
+                         int obytes, int parts) {
             const bool active = lane_used && src != nullptr;
             if (parts & 1) {
                 const unsigned mw = __ballot_sync(0xffffffffu, active && is_w);
@@ -290,7 +312,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
                 __syncwarp();
             }
             if (active && !dead && (is_w ? (parts & 1) : (parts & 2)))
-                bulk_g2s(ring_s + slot * STAGE + dst_row * PITCH, src + src_off, (uint32_t)(is_w ? wbytes : obytes), bar);
+                bulk_g2s(ring_s + stage_off + dst_row * PITCH, src + src_off, (uint32_t)(is_w ? wbytes : obytes), bar);
         };
         // ---- gate/up: lanes 0..7 W_g rows, 8..15 W_u rows, 16..23 hidden rows of the request's tokens
         uint32_t n1 = 0;
@@ -316,7 +338,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
                     if (n1 >= (uint32_t)S1 && !dead)
                         dead = !mbar_wait(empty1 + 8 * (n1 % S1), ((n1 / S1) - 1u) & 1u, abort_flag);
                     const int b = min(CB1, rb1 - kc * CB1);
-                    issue(src, full1, S1, STAGE1, PITCH1, (size_t)kc * CB1, b, b, 3, n1);
+                    issue(src, full1 + 8 * (n1 % S1), (n1 % S1) * STAGE1, PITCH1, (size_t)kc * CB1, b, b, 3);
                 }
                 q += m;
             }
@@ -343,42 +365,52 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
             }
             if (!is_w)
                 return c.base;
+            if (contig2 && lane != 0)
+                return nullptr;          // lane 0 fetches the tile's rows as one block
             return (c.base && r_lo + 16 * blk + my_row < r_hi) ? c.base + (size_t)blk * 16 * rb2 : nullptr;
         };
+        auto rows_of = [&](const Cursor &c) { return min(16, r_hi - r_lo - 16 * (c.t % mt)); };
         auto advance = [&](Cursor &c) {
             if (++c.k == nk2) {
                 c.k = 0;
                 ++c.t;
             }
         };
-        auto w_bytes2 = [&](int kc) { return min(CB2, rb2 - kc * CB2); };
-        auto op_bytes2 = [&](int kc) { return min(CB2, Fpad * 2 - kc * CB2); };
-        // the down stages follow the gate/up stages in the same ring: stage numbers run on from n1
-        const uint32_t N2 = n1 + (uint32_t)hi2 * nk2;
+        auto w_bytes2 = [&](int kc) { return min(CB2, rb2 - kc * CB2); };    // one row's piece
+        auto op_bytes2 = [&](int kc) { return min(CB2, rb2 - kc * CB2); };
+        const uint32_t N2 = (uint32_t)hi2 * nk2;
         Cursor wc{0, 0, -1, nullptr}, oc{0, 0, -1, nullptr};
-        uint32_t wn = n1, on = n1;
+        uint32_t wn = 0, on = 0;
         bool passed[2] = {false, false};
         long long t_idle = 0;
         while (on < N2 && !dead) {
             bool progress = false;
-            // weight rows of as many stages as there are free slots
+            // weight rows of as many stages as there are free sub-stages
             while (wn < N2) {
-                if ((int)((wn % S2) % kProducerWarps) != pw) {
+                const Down ds = down_stage(n1, wn);
+                if ((int)(ds.slot % kProducerWarps) != pw) {
                     (void)tile_of(wc);
                     advance(wc);
                     ++wn;
                     progress = true;
                     continue;
                 }
-                if (wn >= (uint32_t)S2) {
-                    int ok = 0;
-                    if (lane == 0)
-                        ok = mbar_try(empty2 + 8 * (wn % S2), ((wn / S2) - 1u) & 1u);
-                    if (!__shfl_sync(0xffffffffu, ok, 0))
-                        break;
+                // free when its previous down-phase use has been consumed, or, on first use, when the
+                // gate/up phase has let go of the slot for good
+                int ok = 1;
+                if (lane == 0) {
+                    if (ds.use > 0) {
+                        ok = mbar_try(empty2 + 8 * ds.bar, (ds.use - 1u) & 1u);
+                    } else if (n1 > ds.slot) {
+                        const uint32_t m_last = n1 - 1u - ((n1 - 1u - ds.slot) % S1);
+                        ok = mbar_try(empty1 + 8 * ds.slot, (m_last / S1) & 1u);
+                    }
                 }
+                if (!__shfl_sync(0xffffffffu, ok, 0))
+                    break;
                 const char *src = tile_of(wc);
-                issue(src, full2, S2, STAGE2, PITCH2, (size_t)wc.k * CB2, w_bytes2(wc.k), op_bytes2(wc.k), 1, wn);
+                issue(src, full2 + 8 * ds.bar, ds.off, PITCH2, (size_t)wc.k * CB2,
+                      contig2 ? rows_of(wc) * rb2 : w_bytes2(wc.k), op_bytes2(wc.k), 1);
                 advance(wc);
                 ++wn;
                 progress = true;
@@ -400,13 +432,9 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
                 }
                 while (on < wn && passed[oc.t < hi2A ? 0 : 1]) {
                     const char *src = tile_of(oc);
-                    if ((int)((on % S2) % kProducerWarps) != pw) {
-                        advance(oc);
-                        ++on;
-                        progress = true;
-                        continue;
-                    }
-                    issue(src, full2, S2, STAGE2, PITCH2, (size_t)oc.k * CB2, 0, op_bytes2(oc.k), 2, on);
+                    const Down ds = down_stage(n1, on);
+                    if ((int)(ds.slot % kProducerWarps) == pw)
+                        issue(src, full2 + 8 * ds.bar, ds.off, PITCH2, (size_t)oc.k * CB2, 0, op_bytes2(oc.k), 2);
                     advance(oc);
                     ++on;
                     progress = true;
@@ -431,9 +459,12 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
             // a wait ran out: give the copies still in flight a bounded time to land before this
             // CTA's shared memory goes away
             const long long t0 = clock64();
-            for (uint32_t m = n2 > (uint32_t)S2 ? n2 - S2 : 0u; m < n2; ++m)
-                while (!mbar_try(full2 + 8 * (m % S2), (m / S2) & 1u) && clock64() - t0 < kWaitLimitCycles) {
+            const uint32_t in_ring = (uint32_t)(S1 * NS2);
+            for (uint32_t j = n2 > in_ring ? n2 - in_ring : 0u; j < n2; ++j) {
+                const Down ds = down_stage(n1, j);
+                while (!mbar_try(full2 + 8 * ds.bar, ds.use & 1u) && clock64() - t0 < kWaitLimitCycles) {
                 }
+            }
             atomicExch(p.err, MELINOE_ERR_TIMEOUT);
         }
         return;
@@ -570,44 +601,92 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
         }
     }
 
-    // ---- down: z = W_d h for this CTA's output rows
+    // ---- down: z = W_d h for this CTA's output rows.  Warp w owns tile rows w and w + 8: plain
+    // 16-byte loads along the row, fp32 dot products against the h rows behind the weights, a warp
+    // reduction per (row, token), no synchronisation between the warps.
     {
-        const uint32_t a_off = ((lane & 7) + ((lane >> 3) & 1) * 8) * PITCH2 + (lane >> 4) * 16;
-        const uint32_t b_off = (16 + g) * PITCH2 + tig * 4;
-        const uint32_t n_first = n;
-        // the requests' records are read two requests ahead of their use
-        VrInfo v{}, nxt{}, nxt2{};
-        if (hi2 > 0) {
-            nxt = load_vr(vb);
-            nxt2 = nv > 1 ? load_vr(vb + 1) : nxt;
-        }
+        const uint32_t n1c = n;      // gate/up stages of this CTA: the down phase takes the slots in ring order
+        uint32_t j2 = 0;             // down stages consumed
         for (int t = 0; t < hi2; ++t) {
-            const int blk = t % mt, iv = t / mt;
-            if (blk == 0) {
-                v = nxt;
-                nxt = nxt2;
-                if (iv + 2 < nv)
-                    nxt2 = load_vr(vb + iv + 2);
-            }
-            for (int kc = 0; kc < nk2; ++kc, ++n) {
-                compute(full2, empty2, S2, STAGE2, a_off, b_off, n, min(CB2, rb2 - kc * CB2), v.n_tok);
-                if (trace && n == n_first && tid == 0)
-                    trace[2] = globaltimer_ns();
-            }
-            float r[4];
-            if (reduce_tile(r)) {
-                const int row = r_lo + 16 * blk + g;
+            const int blk = t % mt, vr = vb + t / mt;
+            const VrRec *vrec = vrs + (vr - vb);
+            const int n_tok = vrec->n_tok;
+            const int n_rows = min(16, r_hi - r_lo - 16 * blk);
+            // the token loops are unrolled for the smallest of 1, 2, 4, 8 that covers the request's
+            // tokens (predicated-off iterations would still cost issue slots)
+            auto run_tile = [&](auto nt_tag) {
+                constexpr int NT = decltype(nt_tag)::value;
+                float acc[2][NT];
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    if (tig * 2 + h < v.n_tok) {
-                        float *zr = p.zbuf + (size_t)(h ? v.pair1 : v.pair0) * d + row;
-                        if (row < r_hi)
-                            zr[0] = r[h];
-                        if (row + 8 < r_hi)
-                            zr[8] = r[2 + h];
+                for (int j = 0; j < 2; ++j)
+#pragma unroll
+                    for (int tk = 0; tk < NT; ++tk)
+                        acc[j][tk] = 0.f;
+                for (int kc = 0; kc < nk2; ++kc, ++j2) {
+                    const Down ds = down_stage(n1c, j2);
+                    mbar_wait(full2 + 8 * ds.bar, ds.use & 1u, abort_flag);
+                    if (trace && j2 == 0 && tid == 0)
+                        trace[2] = globaltimer_ns();
+                    const unsigned char *base = ring + ds.off;
+                    const int nch = min(CB2, rb2 - kc * CB2) >> 4;
+#pragma unroll
+                    for (int j = 0; j < 2; ++j) {
+                        const int rr = warp + 8 * j;
+                        if (rr < n_rows) {
+                            const uint4 *wr = reinterpret_cast<const uint4 *>(base + (size_t)rr * PITCH2);
+                            for (int c = lane; c < nch; c += 32) {
+                                const uint4 w = wr[c];
+                                const float w0 = __uint_as_float(w.x << 16), w1 = __uint_as_float(w.x & 0xffff0000u);
+                                const float w2 = __uint_as_float(w.y << 16), w3 = __uint_as_float(w.y & 0xffff0000u);
+                                const float w4 = __uint_as_float(w.z << 16), w5 = __uint_as_float(w.z & 0xffff0000u);
+                                const float w6 = __uint_as_float(w.w << 16), w7 = __uint_as_float(w.w & 0xffff0000u);
+#pragma unroll
+                                for (int tk = 0; tk < NT; ++tk) {
+                                    if (NT == 1 || tk < n_tok) {
+                                        const uint4 hv = reinterpret_cast<const uint4 *>(base + (size_t)(16 + tk) * PITCH2)[c];
+                                        float a = acc[j][tk];
+                                        a = fmaf(w0, __uint_as_float(hv.x << 16), a);
+                                        a = fmaf(w1, __uint_as_float(hv.x & 0xffff0000u), a);
+                                        a = fmaf(w2, __uint_as_float(hv.y << 16), a);
+                                        a = fmaf(w3, __uint_as_float(hv.y & 0xffff0000u), a);
+                                        a = fmaf(w4, __uint_as_float(hv.z << 16), a);
+                                        a = fmaf(w5, __uint_as_float(hv.z & 0xffff0000u), a);
+                                        a = fmaf(w6, __uint_as_float(hv.w << 16), a);
+                                        a = fmaf(w7, __uint_as_float(hv.w & 0xffff0000u), a);
+                                        acc[j][tk] = a;
+                                    }
+                                }
+                            }
+                        }
+                    }
+                    __syncwarp();
+                    if (lane == 0)
+                        mbar_arrive(empty2 + 8 * ds.bar);
+                }
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    const int rr = warp + 8 * j;
+#pragma unroll
+                    for (int tk = 0; tk < NT; ++tk) {
+                        if (tk < n_tok && rr < n_rows) {
+                            float a = acc[j][tk];
+#pragma unroll
+                            for (int m = 16; m >= 1; m >>= 1)
+                                a += __shfl_xor_sync(0xffffffffu, a, m);
+                            if (lane == 0)
+                                p.zbuf[(size_t)vrec->pair[tk] * d + r_lo + 16 * blk + rr] = a;
+                        }
                     }
                 }
-            }
+            };
+            if (n_tok <= 1)
+                run_tile(std::integral_constant<int, 1>{});
+            else if (n_tok <= 2)
+                run_tile(std::integral_constant<int, 2>{});
+            else if (n_tok <= 4)
+                run_tile(std::integral_constant<int, 4>{});
+            else
+                run_tile(std::integral_constant<int, 8>{});
         }
     }
     if (trace && tid == 0)
@@ -669,7 +748,7 @@ cudaError_t ffn_stream_geometry(const FfnLaunchCfg &cfg, int d, int F, int T, Ff
     geo->pitch2 = geo->chunk_bytes2 + 16;
     const size_t rows = 16 + geo->n_op_rows;
     const size_t stage = rows * (geo->pitch > geo->pitch2 ? geo->pitch : geo->pitch2);
-    const size_t fixed = 2 * kConsumerWarps * 128 * sizeof(float) + 2 * kMaxStages * 8 + 128;
+    const size_t fixed = 2 * kConsumerWarps * 128 * sizeof(float) + 2 * kMaxStages * 8 + 2 * kMaxSub * 8 + 128;
     if (cfg.max_smem < fixed + 2 * stage)
         return cudaErrorInvalidConfiguration;
     const size_t avail = (cfg.max_smem - fixed) / 128 * 128;
@@ -678,6 +757,16 @@ cudaError_t ffn_stream_geometry(const FfnLaunchCfg &cfg, int d, int F, int T, Ff
         n = kMaxStages;
     geo->n_stages = (int)n;
     geo->stage_bytes = (int)stage;
+    // down phase: rows unpadded (whole row if it fits a piece), as many sub-stages per slot as fit
+    const size_t pitch2u = (size_t)2 * F <= (size_t)geo->chunk_bytes2 ? (size_t)2 * F : (size_t)geo->chunk_bytes2;
+    const size_t sub = (rows * pitch2u + 127) / 128 * 128;
+    size_t ns2 = stage / sub;
+    if (ns2 < 1)
+        ns2 = 1;
+    while (ns2 * n > (size_t)kMaxSub)
+        --ns2;
+    geo->sub2 = (int)ns2;
+    geo->sub_bytes2 = (int)sub;
     geo->ring_bytes = (n * stage + 127) / 128 * 128;
     geo->smem_bytes = geo->ring_bytes + fixed;
     return cudaSuccess;
