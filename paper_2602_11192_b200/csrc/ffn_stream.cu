@@ -1,8 +1,9 @@
 // Streaming SwiGLU expert FFN (Eq. 3) with the gate-weighted combine (Eq. 2) fused in, for
 // calls with few tokens per expert (decode).  The work is reading every needed expert once
-// from HBM, so the kernel is built around keeping the memory system full.  Measured on B200,
-// bulk copies stream faster the larger they are (256-byte pieces reach little more than half the
-// rate of 4 KB rows), so the unit of transfer is a whole row, or a 4 KB piece of a longer one.
+// from HBM, so the kernel is built around keeping the memory system full: measured on B200,
+// bulk copies of whole 4 KB rows stream at the full HBM rate while 256-byte pieces reach
+// little more than half of it, so the unit of transfer is a whole row (or a 4 KB piece of a
+// longer one).
 //
 // One cooperative launch per compute group, one CTA per SM: four producer warps and eight
 // consumer warps.  A "virtual request" is one expert with up to 8 of its tokens.
@@ -15,9 +16,10 @@
 //            h = SiLU(g) * u is thread-local; h goes to global memory as bf16.
 //   barrier  grid-wide, crossed by the producer warps only (bounded polling of a device counter):
 //            the consumers never wait for it.  The requests go through the kernel in two halves,
-//            and both phases of both halves form one sequence of tiles through one ring
-//            (gate/up A | gate/up B and down A taking turns | down B), so each half's barrier
-//            latency is covered by the other half's streaming.
+//            so each half's barrier latency is covered by the other half's streaming.  Both
+//            phases run through one ring and one stage sequence, so the first W_d rows are
+//            requested the moment a slot comes free, before the CTA has finished phase 1, and run
+//            ahead of the barrier as far as the ring allows; only the h rows wait for it.
 //   phase 2  every CTA owns a contiguous range of the d_model output rows (d/G of them, so the
 //            split is even to within one row) for ALL virtual requests of the launch.  Tile =
 //            up to 16 of those W_d rows of one virtual request; warp w computes rows w and w + 8
@@ -32,15 +34,14 @@
 //
 // A stage of the shared-memory ring holds one piece (at most 4 KB) of each of the tile's 16
 // weight rows plus the matching piece of up to 8 operand rows (hidden rows in phase 1, h rows
-// in phase 2), fetched by cp.async.bulk (one producer lane per row; a down tile whose rows fit
-// one piece travels as a single block) completing on the stage's mbarrier; the producer warps
-// share out the ring slots.  Gate/up rows sit at a pitch of 16 bytes more than a multiple of
-// 128, which makes the ldmatrix reads and the operand-fragment reads bank-conflict free; down
-// rows sit unpadded and are read with plain 16-byte loads.
+// in phase 2), each fetched by its own cp.async.bulk (one producer lane per row; the producer
+// warps share out the ring slots) completing on the stage's mbarrier.  Rows sit at a pitch of 16 bytes more than a multiple of 128, which
+// makes the ldmatrix reads and the operand-fragment reads bank-conflict free.
 //
 // Every wait is bounded: when an mbarrier or the grid barrier does not complete in time the
 // warp raises the CTA's abort flag, later waits fall through, the kernel ends normally and the
 // error word tells the host.
+#include <cstdlib>
 #include <type_traits>
 
 #include "kernels.cuh"
@@ -53,6 +54,7 @@ constexpr int kConsumerWarps = 8;
 constexpr int kProducerWarps = 4;                    // a warp needs ~0.6 us to get one stage's copies out
 constexpr int kThreads = (kConsumerWarps + kProducerWarps) * 32;
 constexpr int kMaxStages = 8;
+constexpr int kMaxSub = 16;                          // sub-stages of the down phase, over the whole ring
 constexpr int kMaxChunk = 4096;                      // bytes of one row piece
 constexpr int kVrShared = 72;                        // virtual-request records kept in shared memory
 // Bound of every wait, in SM clock cycles (about 2 s).  Waits are timed with the SM's cycle
@@ -183,7 +185,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
     // with plain 16-byte loads, one row per warp.
     // A down stage is often much smaller than a gate/up stage (short W_d rows), so a ring slot is
     // cut into NS2 sub-stages for the down phase: more tiles in flight where each tile is small.
-    const int CB2 = geo.chunk_bytes2;
+    const int CB2 = geo.chunk_bytes2, NS2 = geo.sub2, SUB2 = geo.sub_bytes2;
     const bool contig2 = 2 * F <= CB2;
     const int PITCH2 = contig2 ? 2 * F : CB2;
 
@@ -212,10 +214,15 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
     uint64_t *bars = reinterpret_cast<uint64_t *>(red + 2 * kConsumerWarps * 128);
     const uint32_t ring_s = smem_u32(ring);
     const uint32_t full1 = smem_u32(bars), empty1 = full1 + 8 * kMaxStages;
+    const uint32_t full2 = empty1 + 8 * kMaxStages, empty2 = full2 + 8 * kMaxSub;
     volatile int *abort_flag = &s_abort;
 
     if (tid == 0) {
         s_abort = 0;
+        for (int i = 0; i < kMaxSub; ++i) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(full2 + 8 * i), "r"(1));
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(empty2 + 8 * i), "r"(kConsumerWarps));
+        }
         for (int i = 0; i < kMaxStages; ++i) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(full1 + 8 * i), "r"(1));
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(empty1 + 8 * i), "r"(kConsumerWarps));
@@ -236,13 +243,11 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
     if (trace && tid == 0)
         trace[1] = globaltimer_ns();
 
-    // ---- work of this CTA.  The launch's virtual requests are cut into two halves A and B (one
-    // when there is a single request).  Both phases of both halves go through ONE sequence of tiles
-    // and one ring:
-    //     gate/up(A) ... | gate/up(B) and down(A) tiles taking turns | down(B) ...
-    // so the grid-wide wait for h of half A is covered by half B's W_g/W_u rows, and the down tiles
-    // of half A (small, each a latency-bound fetch when the W_d rows are short) travel between
-    // gate/up stages that keep the memory system busy.
+    // ---- work of this CTA.  The launch's virtual requests are cut into two halves (one when there
+    // is a single request) that go through the kernel one behind the other:
+    //     gate/up(A)  gate/up(B)  down(A)  down(B)
+    // so that the grid-wide wait for h of half A is covered by the streaming of half B's W_g/W_u
+    // rows, and the wait for half B by half A's W_d rows.
     // gate/up: rows f of W_g and W_u of the half's requests, numbered request-major, are split
     // evenly over the CTAs at single-row granularity; a tile is up to 8 consecutive f of one
     // request (g rows in tile rows 0..7, u rows in 8..15).
@@ -264,169 +269,202 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
     const int hi2 = nv * mt, hi2A = nvA * mt;                 // down tiles: request-major, half A first
     unsigned *sync_word = p.sync + 2 * p.group;               // [half]
 
-    // The tile sequence, walked identically by the producer warps and the consumer warps.
-    struct Item {
-        int kind;      // 1 gate/up tile, 2 down tile, 0 end
-        int half;
-        int vr;        // virtual request
-        int f0, m;     // gate/up: first f and number of f (<= 8)
-        int blk;       // down: index of the 16-row tile within the CTA's rows
-        bool last_of_half;   // gate/up: the half's last tile of this CTA
+    // Down stage j (counted from 0 within the phase) lives in ring slot (n1 + j / NS2) mod S1, sub-stage
+    // j mod NS2: the slots are taken in the order in which the gate/up phase lets go of them.
+    struct Down {
+        uint32_t slot, bar, use, off;
     };
-    struct Sched {
-        int q[2];      // gate/up cursors of the halves
-        int t2;        // down tile cursor
-        int turn;      // in the mixed section: gate/up tiles of B emitted so far
+    auto down_stage = [&](uint32_t n1_, uint32_t j) -> Down {
+        Down x;
+        x.slot = (n1_ + j / NS2) % S1;
+        const uint32_t sub = j % NS2;
+        x.bar = x.slot * NS2 + sub;
+        x.use = j / (uint32_t)(S1 * NS2);
+        x.off = x.slot * STAGE1 + sub * SUB2;
+        return x;
     };
-    Sched sched_init{{q_lo[0], q_lo[1]}, 0, 0};
-    auto next_item = [&](Sched &sc) -> Item {
-        Item it{0, 0, 0, 0, 0, 0, false};
-        auto gate_up = [&](int half) {
-            const int v0 = vb + (half ? nvA : 0);
-            const int q = sc.q[half];
-            it.kind = 1;
-            it.half = half;
-            it.vr = v0 + q / F;
-            it.f0 = q % F;
-            it.m = min(min(8, F - it.f0), q_hi[half] - q);
-            sc.q[half] = q + it.m;
-            it.last_of_half = sc.q[half] >= q_hi[half];
-        };
-        auto down = [&]() {
-            it.kind = 2;
-            it.half = sc.t2 < hi2A ? 0 : 1;
-            it.vr = vb + sc.t2 / mt;
-            it.blk = sc.t2 % mt;
-            ++sc.t2;
-        };
-        if (sc.q[0] < q_hi[0]) {
-            gate_up(0);
-        } else if (n_half == 2 && (sc.q[1] < q_hi[1] || sc.t2 < hi2A)) {
-            // B's gate/up tiles and A's down tiles take turns; A's first down tile waits for two of
-            // B's tiles so that A's barrier has had time to complete
-            const bool b_left = sc.q[1] < q_hi[1], a_left = sc.t2 < hi2A;
-            const bool take_b = b_left && (!a_left || sc.turn < 2 || (sc.turn & 1) != 0);
-            if (take_b)
-                gate_up(1);
-            else
-                down();
-            ++sc.turn;
-        } else if (sc.t2 < hi2) {
-            down();
-        }
-        return it;
-    };
-    // a CTA with an empty gate/up range still has to announce the half
-    const bool emptyA = q_lo[0] >= q_hi[0], emptyB = n_half == 2 && q_lo[1] >= q_hi[1];
 
     if (warp >= kConsumerWarps) {
         // =================================================================== producers
-        // The producer warps walk the tile sequence and share the stages out.  A ring slot always
-        // belongs to the same warp (slot s to warp s mod 4), so every wait on a slot's "empty"
-        // barrier is made by the one warp that has followed all its earlier phases.
-        // Lanes 0..15 fetch the tile's weight rows, lanes 16..23 the operand rows; a down tile whose
-        // rows fit one piece is fetched as one block by lane 0.
+        // The producer warps walk the same stage sequence and share the stages out (a warp is busy
+        // for ~0.6 us with one bulk-copy instruction, however few lanes take part, so the stages
+        // of a 28 KB-per-stage phase would otherwise leave faster than one warp can issue them).
+        // A ring slot always belongs to the same warp (slot s to warp s mod 4), so every wait on a
+        // slot's "empty" barrier is made by the one warp that has followed all its earlier phases.
+        // Lanes 0..15 fetch the tile's weight rows, lanes 16..23 the operand rows.
         const int pw = warp - kConsumerWarps;
         const bool is_w = lane < 16;
         const int my_row = is_w ? lane : lane - 16;                        // tile row, or token slot
+        const int dst_row = lane;
         const bool lane_used = lane < 24;
         bool dead = false;
-        bool passed[2] = {false, false};
-        auto issue = [&](const char *src, uint32_t nn, int PITCH, size_t src_off, int wbytes, int obytes) {
-            const uint32_t slot = nn % S1;
-            const uint32_t bar = full1 + 8 * slot;
+        // One stage of either phase.  src: this lane's source row or null.  parts bit 0: arm the
+        // barrier and fetch the weight rows (the caller has made sure the slot is free); bit 1:
+        // operand rows.
+        auto issue = [&](const char *src, uint32_t bar, uint32_t stage_off, int PITCH, size_t src_off, int wbytes,
+                         int obytes, int parts) {
             const bool active = lane_used && src != nullptr;
-            const unsigned mw = __ballot_sync(0xffffffffu, active && is_w);
-            const unsigned mo = __ballot_sync(0xffffffffu, active && !is_w);
-            if (lane == 0)
-                mbar_expect(bar, (uint32_t)__popc(mw) * wbytes + (uint32_t)__popc(mo) * obytes);
-            __syncwarp();
-            if (active && !dead)
-                bulk_g2s(ring_s + slot * STAGE1 + lane * PITCH, src + src_off, (uint32_t)(is_w ? wbytes : obytes), bar);
-        };
-        // bounded wait until every CTA has written its part of the half's h
-        auto need_half = [&](int half) {
-            if (passed[half] || dead)
-                return;
-            int ok = 1;
-            if (lane == 0) {
-                volatile unsigned *w = sync_word + half;
-                if (*w < (unsigned)G) {
-                    const long long t0 = clock64();
-                    while (*w < (unsigned)G) {
-                        if (*abort_flag || clock64() - t0 > kWaitLimitCycles) {
-                            *abort_flag = 1;
-                            ok = 0;
-                            break;
-                        }
-                    }
-                }
-                __threadfence();
-                if (trace && pw == 0)
-                    trace[5] = globaltimer_ns();
+            if (parts & 1) {
+                const unsigned mw = __ballot_sync(0xffffffffu, active && is_w);
+                const unsigned mo = __ballot_sync(0xffffffffu, active && !is_w);
+                if (lane == 0)
+                    mbar_expect(bar, (uint32_t)__popc(mw) * wbytes + (uint32_t)__popc(mo) * obytes);
+                __syncwarp();
             }
-            ok = __shfl_sync(0xffffffffu, ok, 0);
-            if (!ok)
-                dead = true;
-            passed[half] = true;
+            if (active && !dead && (is_w ? (parts & 1) : (parts & 2)))
+                bulk_g2s(ring_s + stage_off + dst_row * PITCH, src + src_off, (uint32_t)(is_w ? wbytes : obytes), bar);
         };
-        uint32_t n = 0;
-        Sched sc = sched_init;
-        for (Item it = next_item(sc); it.kind != 0 && !dead; it = next_item(sc)) {
-            const VrRec *v = vrs + (it.vr - vb);
-            const int nk = it.kind == 1 ? nk1 : nk2;
-            // is any stage of this tile mine?
-            bool any = false;
-            for (int kc = 0; kc < nk; ++kc)
-                any = any || (int)(((n + kc) % S1) % kProducerWarps) == pw;
-            if (!any) {
-                n += nk;
-                continue;
-            }
-            const char *src = nullptr;
-            int n_rows = 16;
-            if (it.kind == 1) {
+        // ---- gate/up: lanes 0..7 W_g rows, 8..15 W_u rows, 16..23 hidden rows of the request's tokens
+        uint32_t n1 = 0;
+        for (int half = 0; half < n_half; ++half) {
+            const int v0 = vb + (half ? nvA : 0);
+            int q = q_lo[half];
+            while (q < q_hi[half]) {
+                const int vr = v0 + q / F, f0 = q % F;
+                const int m = min(min(8, F - f0), q_hi[half] - q);
+                const VrRec *v = vrs + (vr - vb);
+                const char *src = nullptr;
                 if (lane_used) {
                     if (is_w) {
-                        if ((my_row & 7) < it.m)
-                            src = v->blob + (size_t)((my_row < 8 ? 0 : F) + it.f0 + (my_row & 7)) * rb1;
+                        if ((my_row & 7) < m)
+                            src = v->blob + (size_t)((my_row < 8 ? 0 : F) + f0 + (my_row & 7)) * rb1;
                     } else if (my_row < v->n_tok) {
                         src = reinterpret_cast<const char *>(p.x) + (size_t)v->tok[my_row] * rb1;
                     }
                 }
-            } else {
-                need_half(it.half);
-                n_rows = min(16, r_hi - r_lo - 16 * it.blk);
+                for (int kc = 0; kc < nk1; ++kc, ++n1) {
+                    if ((int)((n1 % S1) % kProducerWarps) != pw)
+                        continue;
+                    if (n1 >= (uint32_t)S1 && !dead)
+                        dead = !mbar_wait(empty1 + 8 * (n1 % S1), ((n1 / S1) - 1u) & 1u, abort_flag);
+                    const int b = min(CB1, rb1 - kc * CB1);
+                    issue(src, full1 + 8 * (n1 % S1), (n1 % S1) * STAGE1, PITCH1, (size_t)kc * CB1, b, b, 3);
+                }
+                q += m;
+            }
+        }
+        // ---- down: lanes 0..15 W_d rows, 16..23 rows of h.  Two cursors walk the same stage
+        // sequence: the weight rows run ahead as far as the ring allows, the h rows of a stage
+        // follow once the grid has finished the h of the stage's half.
+        struct Cursor {
+            int t, k, vr;
+            const char *base;
+        };
+        auto tile_of = [&](Cursor &c) -> const char * {
+            const int vr = vb + c.t / mt, blk = c.t % mt;
+            if (vr != c.vr) {
+                const VrRec *v = vrs + (vr - vb);
+                c.vr = vr;
+                c.base = nullptr;
                 if (lane_used) {
-                    if (is_w) {
-                        if (contig2 ? lane == 0 : my_row < n_rows)
-                            src = v->blob + (size_t)2 * F * rb1 + (size_t)(r_lo + 16 * it.blk + my_row) * rb2;
-                    } else if (my_row < v->n_tok) {
-                        src = reinterpret_cast<const char *>(p.hbuf) + ((size_t)it.vr * kTokPerVr + my_row) * Fpad * 2;
-                    }
+                    if (is_w)
+                        c.base = v->blob + (size_t)2 * F * rb1 + (size_t)(r_lo + my_row) * rb2;
+                    else if (my_row < v->n_tok)
+                        c.base = reinterpret_cast<const char *>(p.hbuf) + ((size_t)vr * kTokPerVr + my_row) * Fpad * 2;
                 }
             }
-            for (int kc = 0; kc < nk; ++kc, ++n) {
-                if ((int)((n % S1) % kProducerWarps) != pw)
+            if (!is_w)
+                return c.base;
+            if (contig2 && lane != 0)
+                return nullptr;          // lane 0 fetches the tile's rows as one block
+            return (c.base && r_lo + 16 * blk + my_row < r_hi) ? c.base + (size_t)blk * 16 * rb2 : nullptr;
+        };
+        auto rows_of = [&](const Cursor &c) { return min(16, r_hi - r_lo - 16 * (c.t % mt)); };
+        auto advance = [&](Cursor &c) {
+            if (++c.k == nk2) {
+                c.k = 0;
+                ++c.t;
+            }
+        };
+        auto w_bytes2 = [&](int kc) { return min(CB2, rb2 - kc * CB2); };    // one row's piece
+        auto op_bytes2 = [&](int kc) { return min(CB2, rb2 - kc * CB2); };
+        const uint32_t N2 = (uint32_t)hi2 * nk2;
+        Cursor wc{0, 0, -1, nullptr}, oc{0, 0, -1, nullptr};
+        uint32_t wn = 0, on = 0;
+        bool passed[2] = {false, false};
+        long long t_idle = 0;
+        while (on < N2 && !dead) {
+            bool progress = false;
+            // weight rows of as many stages as there are free sub-stages
+            while (wn < N2) {
+                const Down ds = down_stage(n1, wn);
+                if ((int)(ds.slot % kProducerWarps) != pw) {
+                    (void)tile_of(wc);
+                    advance(wc);
+                    ++wn;
+                    progress = true;
                     continue;
-                if (n >= (uint32_t)S1 && !dead)
-                    dead = !mbar_wait(empty1 + 8 * (n % S1), ((n / S1) - 1u) & 1u, abort_flag);
-                if (it.kind == 1) {
-                    const int b = min(CB1, rb1 - kc * CB1);
-                    issue(src, n, PITCH1, (size_t)kc * CB1, b, b);
-                } else {
-                    const int b = min(CB2, rb2 - kc * CB2);
-                    issue(src, n, PITCH2, (size_t)kc * CB2, contig2 ? n_rows * rb2 : b, b);
+                }
+                // free when its previous down-phase use has been consumed, or, on first use, when the
+                // gate/up phase has let go of the slot for good
+                int ok = 1;
+                if (lane == 0) {
+                    if (ds.use > 0) {
+                        ok = mbar_try(empty2 + 8 * ds.bar, (ds.use - 1u) & 1u);
+                    } else if (n1 > ds.slot) {
+                        const uint32_t m_last = n1 - 1u - ((n1 - 1u - ds.slot) % S1);
+                        ok = mbar_try(empty1 + 8 * ds.slot, (m_last / S1) & 1u);
+                    }
+                }
+                if (!__shfl_sync(0xffffffffu, ok, 0))
+                    break;
+                const char *src = tile_of(wc);
+                issue(src, full2 + 8 * ds.bar, ds.off, PITCH2, (size_t)wc.k * CB2,
+                      contig2 ? rows_of(wc) * rb2 : w_bytes2(wc.k), op_bytes2(wc.k), 1);
+                advance(wc);
+                ++wn;
+                progress = true;
+            }
+            // h rows of the next stages, once their half of h is complete everywhere
+            if (on < wn) {
+                const int half = oc.t < hi2A ? 0 : 1;
+                if (!passed[half]) {
+                    int ok = 0;
+                    if (lane == 0) {
+                        ok = *reinterpret_cast<volatile unsigned *>(sync_word + half) >= (unsigned)G;
+                        if (ok) {
+                            __threadfence();
+                            if (trace && pw == 0)
+                                trace[5] = globaltimer_ns();
+                        }
+                    }
+                    passed[half] = __shfl_sync(0xffffffffu, ok, 0) != 0;
+                }
+                while (on < wn && passed[oc.t < hi2A ? 0 : 1]) {
+                    const char *src = tile_of(oc);
+                    const Down ds = down_stage(n1, on);
+                    if ((int)(ds.slot % kProducerWarps) == pw)
+                        issue(src, full2 + 8 * ds.bar, ds.off, PITCH2, (size_t)oc.k * CB2, 0, op_bytes2(oc.k), 2);
+                    advance(oc);
+                    ++on;
+                    progress = true;
+                }
+            }
+            if (progress) {
+                t_idle = 0;
+            } else {
+                const long long now = clock64();
+                if (t_idle == 0)
+                    t_idle = now;
+                int give_up = (now - t_idle > kWaitLimitCycles) || *abort_flag;
+                give_up = __shfl_sync(0xffffffffu, give_up, 0);
+                if (give_up) {
+                    *abort_flag = 1;
+                    dead = true;
                 }
             }
         }
+        const uint32_t n2 = on;
         if (*abort_flag && lane == 0 && pw == 0) {
             // a wait ran out: give the copies still in flight a bounded time to land before this
             // CTA's shared memory goes away
             const long long t0 = clock64();
-            for (uint32_t m = n > (uint32_t)S1 ? n - S1 : 0u; m < n; ++m)
-                while (!mbar_try(full1 + 8 * (m % S1), (m / S1) & 1u) && clock64() - t0 < kWaitLimitCycles) {
+            const uint32_t in_ring = (uint32_t)(S1 * NS2);
+            for (uint32_t j = n2 > in_ring ? n2 - in_ring : 0u; j < n2; ++j) {
+                const Down ds = down_stage(n1, j);
+                while (!mbar_try(full2 + 8 * ds.bar, ds.use & 1u) && clock64() - t0 < kWaitLimitCycles) {
                 }
+            }
             atomicExch(p.err, MELINOE_ERR_TIMEOUT);
         }
         return;
@@ -434,20 +472,16 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
 
     // ======================================================================= consumers
     const int g = lane >> 2, tig = lane & 3;
-    int n_tiles = 0;       // gate/up tiles finished so far (selects the reduction buffer and the epilogue warp)
+    int n_tiles = 0;       // tiles finished so far (selects the reduction buffer and the epilogue warp)
     float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
-    uint32_t n = 0;        // stages consumed so far
 
-    // gate/up stage: this warp's share of the 16-column steps of the piece.  Weights in tile rows
-    // 0..15, the hidden rows of the request's tokens behind them.
-    const uint32_t a_off = ((lane & 7) + ((lane >> 3) & 1) * 8) * PITCH1 + (lane >> 4) * 16;
-    const uint32_t b_off = (16 + g) * PITCH1 + tig * 4;
-    auto compute = [&](int bytes, int n_tok) {
-        const uint32_t slot = n % S1;
-        mbar_wait(full1 + 8 * slot, (n / S1) & 1u, abort_flag);
-        if (trace && n == 0 && tid == 0)
-            trace[2] = globaltimer_ns();
-        const uint32_t base = ring_s + slot * STAGE1;
+    // this warp's share of one stage: some of the 16-column steps of the piece.  Weights in tile
+    // rows 0..15, the operand rows (hidden or h) of the request's tokens behind them.
+    auto compute = [&](uint32_t full0, uint32_t empty0, int S, int STAGE, uint32_t a_off, uint32_t b_off, uint32_t n,
+                       int bytes, int n_tok) {
+        const uint32_t slot = n % S;
+        mbar_wait(full0 + 8 * slot, (n / S) & 1u, abort_flag);
+        const uint32_t base = ring_s + slot * STAGE;
         const int ks_total = (bytes + 31) >> 5;
         const int ks_hi = (warp + 1) * ks_total / kConsumerWarps;
         int ks = warp * ks_total / kConsumerWarps;
@@ -478,11 +512,10 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
         }
         __syncwarp();
         if (lane == 0)
-            mbar_arrive(empty1 + 8 * slot);
-        ++n;
+            mbar_arrive(empty0 + 8 * slot);
     };
-    // end of a gate/up tile: the warps' partial accumulators meet in shared memory; one warp (they
-    // take turns) ends up with the complete 16 x 8 tile in the usual accumulator layout
+    // end of a tile: the warps' partial accumulators meet in shared memory; one warp (they take
+    // turns) ends up with the complete 16 x 8 tile in the usual accumulator layout
     auto reduce_tile = [&](float (&out)[4]) -> bool {
         float *buf = red + (n_tiles & 1) * (kConsumerWarps * 128);
 #pragma unroll
@@ -505,124 +538,155 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
         ++n_tiles;
         return mine;
     };
-    // this CTA's part of a half's h is complete: tell the grid
-    auto announce = [&](int half) {
-        __threadfence();
-        fence_proxy_async();       // h was written through the generic proxy, bulk copies will read it
-        consumer_bar();
-        if (tid == 0) {
-            atomicAdd(sync_word + half, 1u);
-            if (trace && half == n_half - 1)
-                trace[4] = globaltimer_ns();
-        }
+    // what a consumer lane needs of a virtual request: its token count and the z rows of the two
+    // token slots this lane's accumulators belong to
+    struct VrInfo {
+        int n_tok, pair0, pair1;
     };
-    // down tile: warp w owns tile rows w and w + 8: plain 16-byte loads along the row, fp32 dot
-    // products against the h rows behind the weights, a warp reduction per (row, token), no
-    // synchronisation between the warps.  The token loops are unrolled for the smallest of 1, 2, 4, 8
-    // that covers the request's tokens (predicated-off iterations would still cost issue slots).
-    auto down_tile = [&](auto nt_tag, const VrRec *vrec, int n_tok, int blk) {
-        constexpr int NT = decltype(nt_tag)::value;
-        const int n_rows = min(16, r_hi - r_lo - 16 * blk);
-        float acc[2][NT];
+    auto load_vr = [&](int vr) -> VrInfo {
+        const VrRec *v = vrs + (vr - vb);
+        VrInfo r;
+        r.n_tok = v->n_tok;
+        const int2 pr = *reinterpret_cast<const int2 *>(v->pair + tig * 2);
+        r.pair0 = pr.x;
+        r.pair1 = pr.y;
+        return r;
+    };
+
+    uint32_t n = 0;        // stages consumed so far, over both phases
+    // ---- gate/up: h = SiLU(W_g x) * (W_u x), half by half
+    {
+        const uint32_t a_off = ((lane & 7) + ((lane >> 3) & 1) * 8) * PITCH1 + (lane >> 4) * 16;
+        const uint32_t b_off = (16 + g) * PITCH1 + tig * 4;
+        for (int half = 0; half < n_half; ++half) {
+            const int v0 = vb + (half ? nvA : 0);
+            int cur_vr = -1;
+            VrInfo v{};
+            int q = q_lo[half];
+            while (q < q_hi[half]) {
+                const int vr = v0 + q / F, f0 = q % F;
+                const int m = min(min(8, F - f0), q_hi[half] - q);
+                if (vr != cur_vr) {
+                    v = load_vr(vr);
+                    cur_vr = vr;
+                }
+                for (int kc = 0; kc < nk1; ++kc) {
+                    compute(full1, empty1, S1, STAGE1, a_off, b_off, n, min(CB1, rb1 - kc * CB1), v.n_tok);
+                    if (trace && n == 0 && tid == 0)
+                        trace[2] = globaltimer_ns();
+                    ++n;
+                }
+                float r[4];
+                if (reduce_tile(r) && g < m) {
+                    // rows g and g + 8 of the tile are g_f and u_f for f = f0 + g
+                    uint16_t *hrow = p.hbuf + ((size_t)vr * kTokPerVr) * Fpad + f0 + g;
+                    if (tig * 2 < v.n_tok)
+                        hrow[(size_t)(tig * 2) * Fpad] = bf16_rne(r[0] / (1.0f + __expf(-r[0])) * r[2]);
+                    if (tig * 2 + 1 < v.n_tok)
+                        hrow[(size_t)(tig * 2 + 1) * Fpad] = bf16_rne(r[1] / (1.0f + __expf(-r[1])) * r[3]);
+                }
+                q += m;
+            }
+            if (trace && tid == 0 && half == n_half - 1)
+                trace[3] = globaltimer_ns();
+            // this CTA's part of the half's h is complete: tell the grid
+            __threadfence();
+            fence_proxy_async();       // h was written through the generic proxy, bulk copies will read it
+            consumer_bar();
+            if (tid == 0) {
+                atomicAdd(sync_word + half, 1u);
+                if (trace && half == n_half - 1)
+                    trace[4] = globaltimer_ns();
+            }
+        }
+    }
+
+    // ---- down: z = W_d h for this CTA's output rows.  Warp w owns tile rows w and w + 8: plain
+    // 16-byte loads along the row, fp32 dot products against the h rows behind the weights, a warp
+    // reduction per (row, token), no synchronisation between the warps.
+    {
+        const uint32_t n1c = n;      // gate/up stages of this CTA: the down phase takes the slots in ring order
+        uint32_t j2 = 0;             // down stages consumed
+        for (int t = 0; t < hi2; ++t) {
+            const int blk = t % mt, vr = vb + t / mt;
+            const VrRec *vrec = vrs + (vr - vb);
+            const int n_tok = vrec->n_tok;
+            const int n_rows = min(16, r_hi - r_lo - 16 * blk);
+            // the token loops are unrolled for the smallest of 1, 2, 4, 8 that covers the request's
+            // tokens (predicated-off iterations would still cost issue slots)
+            auto run_tile = [&](auto nt_tag) {
+                constexpr int NT = decltype(nt_tag)::value;
+                float acc[2][NT];
 #pragma unroll
-        for (int j = 0; j < 2; ++j)
+                for (int j = 0; j < 2; ++j)
 #pragma unroll
-            for (int tk = 0; tk < NT; ++tk)
-                acc[j][tk] = 0.f;
-        for (int kc = 0; kc < nk2; ++kc, ++n) {
-            const uint32_t slot = n % S1;
-            mbar_wait(full1 + 8 * slot, (n / S1) & 1u, abort_flag);
-            const unsigned char *base = ring + (size_t)slot * STAGE1;
-            const int nch = min(CB2, rb2 - kc * CB2) >> 4;
+                    for (int tk = 0; tk < NT; ++tk)
+                        acc[j][tk] = 0.f;
+                for (int kc = 0; kc < nk2; ++kc, ++j2) {
+                    const Down ds = down_stage(n1c, j2);
+                    mbar_wait(full2 + 8 * ds.bar, ds.use & 1u, abort_flag);
+                    if (trace && j2 == 0 && tid == 0)
+                        trace[2] = globaltimer_ns();
+                    const unsigned char *base = ring + ds.off;
+                    const int nch = min(CB2, rb2 - kc * CB2) >> 4;
 #pragma unroll
-            for (int j = 0; j < 2; ++j) {
-                const int rr = warp + 8 * j;
-                if (rr < n_rows) {
-                    const uint4 *wr = reinterpret_cast<const uint4 *>(base + (size_t)rr * PITCH2);
-                    for (int c = lane; c < nch; c += 32) {
-                        const uint4 w = wr[c];
-                        const float w0 = __uint_as_float(w.x << 16), w1 = __uint_as_float(w.x & 0xffff0000u);
-                        const float w2 = __uint_as_float(w.y << 16), w3 = __uint_as_float(w.y & 0xffff0000u);
-                        const float w4 = __uint_as_float(w.z << 16), w5 = __uint_as_float(w.z & 0xffff0000u);
-                        const float w6 = __uint_as_float(w.w << 16), w7 = __uint_as_float(w.w & 0xffff0000u);
+                    for (int j = 0; j < 2; ++j) {
+                        const int rr = warp + 8 * j;
+                        if (rr < n_rows) {
+                            const uint4 *wr = reinterpret_cast<const uint4 *>(base + (size_t)rr * PITCH2);
+                            for (int c = lane; c < nch; c += 32) {
+                                const uint4 w = wr[c];
+                                const float w0 = __uint_as_float(w.x << 16), w1 = __uint_as_float(w.x & 0xffff0000u);
+                                const float w2 = __uint_as_float(w.y << 16), w3 = __uint_as_float(w.y & 0xffff0000u);
+                                const float w4 = __uint_as_float(w.z << 16), w5 = __uint_as_float(w.z & 0xffff0000u);
+                                const float w6 = __uint_as_float(w.w << 16), w7 = __uint_as_float(w.w & 0xffff0000u);
 #pragma unroll
-                        for (int tk = 0; tk < NT; ++tk) {
-                            if (NT == 1 || tk < n_tok) {
-                                const uint4 hv = reinterpret_cast<const uint4 *>(base + (size_t)(16 + tk) * PITCH2)[c];
-                                float a = acc[j][tk];
-                                a = fmaf(w0, __uint_as_float(hv.x << 16), a);
-                                a = fmaf(w1, __uint_as_float(hv.x & 0xffff0000u), a);
-                                a = fmaf(w2, __uint_as_float(hv.y << 16), a);
-                                a = fmaf(w3, __uint_as_float(hv.y & 0xffff0000u), a);
-                                a = fmaf(w4, __uint_as_float(hv.z << 16), a);
-                                a = fmaf(w5, __uint_as_float(hv.z & 0xffff0000u), a);
-                                a = fmaf(w6, __uint_as_float(hv.w << 16), a);
-                                a = fmaf(w7, __uint_as_float(hv.w & 0xffff0000u), a);
-                                acc[j][tk] = a;
+                                for (int tk = 0; tk < NT; ++tk) {
+                                    if (NT == 1 || tk < n_tok) {
+                                        const uint4 hv = reinterpret_cast<const uint4 *>(base + (size_t)(16 + tk) * PITCH2)[c];
+                                        float a = acc[j][tk];
+                                        a = fmaf(w0, __uint_as_float(hv.x << 16), a);
+                                        a = fmaf(w1, __uint_as_float(hv.x & 0xffff0000u), a);
+                                        a = fmaf(w2, __uint_as_float(hv.y << 16), a);
+                                        a = fmaf(w3, __uint_as_float(hv.y & 0xffff0000u), a);
+                                        a = fmaf(w4, __uint_as_float(hv.z << 16), a);
+                                        a = fmaf(w5, __uint_as_float(hv.z & 0xffff0000u), a);
+                                        a = fmaf(w6, __uint_as_float(hv.w << 16), a);
+                                        a = fmaf(w7, __uint_as_float(hv.w & 0xffff0000u), a);
+                                        acc[j][tk] = a;
+                                    }
+                                }
                             }
                         }
                     }
-                }
-            }
-            __syncwarp();
-            if (lane == 0)
-                mbar_arrive(empty1 + 8 * slot);
-        }
-#pragma unroll
-        for (int j = 0; j < 2; ++j) {
-            const int rr = warp + 8 * j;
-#pragma unroll
-            for (int tk = 0; tk < NT; ++tk) {
-                if (tk < n_tok && rr < n_rows) {
-                    float a = acc[j][tk];
-#pragma unroll
-                    for (int m = 16; m >= 1; m >>= 1)
-                        a += __shfl_xor_sync(0xffffffffu, a, m);
+                    __syncwarp();
                     if (lane == 0)
-                        p.zbuf[(size_t)vrec->pair[tk] * d + r_lo + 16 * blk + rr] = a;
+                        mbar_arrive(empty2 + 8 * ds.bar);
                 }
-            }
-        }
-    };
-
-    if (emptyA)
-        announce(0);
-    if (emptyB)
-        announce(1);
-    {
-        Sched sc = sched_init;
-        for (Item it = next_item(sc); it.kind != 0; it = next_item(sc)) {
-            const VrRec *vrec = vrs + (it.vr - vb);
-            const int n_tok = vrec->n_tok;
-            if (it.kind == 1) {
-                // ---- gate/up tile: h = SiLU(W_g x) * (W_u x)
-                for (int kc = 0; kc < nk1; ++kc)
-                    compute(min(CB1, rb1 - kc * CB1), n_tok);
-                float r[4];
-                if (reduce_tile(r) && g < it.m) {
-                    // rows g and g + 8 of the tile are g_f and u_f for f = f0 + g
-                    uint16_t *hrow = p.hbuf + ((size_t)it.vr * kTokPerVr) * Fpad + it.f0 + g;
-                    if (tig * 2 < n_tok)
-                        hrow[(size_t)(tig * 2) * Fpad] = bf16_rne(r[0] / (1.0f + __expf(-r[0])) * r[2]);
-                    if (tig * 2 + 1 < n_tok)
-                        hrow[(size_t)(tig * 2 + 1) * Fpad] = bf16_rne(r[1] / (1.0f + __expf(-r[1])) * r[3]);
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    const int rr = warp + 8 * j;
+#pragma unroll
+                    for (int tk = 0; tk < NT; ++tk) {
+                        if (tk < n_tok && rr < n_rows) {
+                            float a = acc[j][tk];
+#pragma unroll
+                            for (int m = 16; m >= 1; m >>= 1)
+                                a += __shfl_xor_sync(0xffffffffu, a, m);
+                            if (lane == 0)
+                                p.zbuf[(size_t)vrec->pair[tk] * d + r_lo + 16 * blk + rr] = a;
+                        }
+                    }
                 }
-                if (it.last_of_half) {
-                    if (trace && tid == 0 && it.half == n_half - 1)
-                        trace[3] = globaltimer_ns();
-                    announce(it.half);
-                }
-            } else {
-                // ---- down tile: z = W_d h for this CTA's output rows
-                if (n_tok <= 1)
-                    down_tile(std::integral_constant<int, 1>{}, vrec, n_tok, it.blk);
-                else if (n_tok <= 2)
-                    down_tile(std::integral_constant<int, 2>{}, vrec, n_tok, it.blk);
-                else if (n_tok <= 4)
-                    down_tile(std::integral_constant<int, 4>{}, vrec, n_tok, it.blk);
-                else
-                    down_tile(std::integral_constant<int, 8>{}, vrec, n_tok, it.blk);
-            }
+            };
+            if (n_tok <= 1)
+                run_tile(std::integral_constant<int, 1>{});
+            else if (n_tok <= 2)
+                run_tile(std::integral_constant<int, 2>{});
+            else if (n_tok <= 4)
+                run_tile(std::integral_constant<int, 4>{});
+            else
+                run_tile(std::integral_constant<int, 8>{});
         }
     }
     if (trace && tid == 0)
@@ -684,7 +748,7 @@ cudaError_t ffn_stream_geometry(const FfnLaunchCfg &cfg, int d, int F, int T, Ff
     geo->pitch2 = geo->chunk_bytes2 + 16;
     const size_t rows = 16 + geo->n_op_rows;
     const size_t stage = rows * (geo->pitch > geo->pitch2 ? geo->pitch : geo->pitch2);
-    const size_t fixed = 2 * kConsumerWarps * 128 * sizeof(float) + 2 * kMaxStages * 8 + 128;
+    const size_t fixed = 2 * kConsumerWarps * 128 * sizeof(float) + 2 * kMaxStages * 8 + 2 * kMaxSub * 8 + 128;
     if (cfg.max_smem < fixed + 2 * stage)
         return cudaErrorInvalidConfiguration;
     const size_t avail = (cfg.max_smem - fixed) / 128 * 128;
@@ -693,6 +757,16 @@ cudaError_t ffn_stream_geometry(const FfnLaunchCfg &cfg, int d, int F, int T, Ff
         n = kMaxStages;
     geo->n_stages = (int)n;
     geo->stage_bytes = (int)stage;
+    // down phase: rows unpadded (whole row if it fits a piece), as many sub-stages per slot as fit
+    const size_t pitch2u = (size_t)2 * F <= (size_t)geo->chunk_bytes2 ? (size_t)2 * F : (size_t)geo->chunk_bytes2;
+    const size_t sub = (rows * pitch2u + 127) / 128 * 128;
+    size_t ns2 = stage / sub;
+    if (ns2 < 1)
+        ns2 = 1;
+    while (ns2 * n > (size_t)kMaxSub)
+        --ns2;
+    geo->sub2 = (int)ns2;
+    geo->sub_bytes2 = (int)sub;
     geo->ring_bytes = (n * stage + 127) / 128 * 128;
     geo->smem_bytes = geo->ring_bytes + fixed;
     return cudaSuccess;
