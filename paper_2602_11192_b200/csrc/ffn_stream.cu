@@ -5,8 +5,9 @@
 // little more than half of it, so the unit of transfer is a whole row (or a 4 KB piece of a
 // longer one).
 //
-// One cooperative launch per compute group, one CTA per SM: four producer warps and eight
-// consumer warps.  A "virtual request" is one expert with up to 8 of its tokens.
+// One cooperative launch per compute group, one CTA per SM: eight consumer warps, three producer
+// warps and one warp for the grid barrier (twelve warps: a thirteenth would cost every thread
+// registers, which are handed out to warps in fours).  A "virtual request" is one expert with up to 8 of its tokens.
 //
 //   phase 1  tile = up to 8 rows of W_g plus the same rows of W_u of one virtual request.
 //            D[16 x 8] = [W_g rows; W_u rows] (16 x d) * x^T (d x 8 tokens) on mma.sync
@@ -14,12 +15,15 @@
 //            their partial sums meet in shared memory once per tile.  In the accumulator
 //            layout a thread holds g_f and u_f of the same f and the same two tokens, so
 //            h = SiLU(g) * u is thread-local; h goes to global memory as bf16.
-//   barrier  grid-wide, crossed by the producer warps only (bounded polling of a device counter):
-//            the consumers never wait for it.  The requests go through the kernel in two halves,
-//            so each half's barrier latency is covered by the other half's streaming.  Both
-//            phases run through one ring and one stage sequence, so the first W_d rows are
-//            requested the moment a slot comes free, before the CTA has finished phase 1, and run
-//            ahead of the barrier as far as the ring allows; only the h rows wait for it.
+//   barrier  grid-wide, and off everybody's critical path.  While the SM streams, any round trip
+//            to global memory (a fence after the h stores, a poll of a device counter) takes
+//            microseconds, so neither the consumers nor the producers ever make one: the consumer
+//            warps arrive on a shared-memory barrier when their part of h is stored and go on; a
+//            twelfth warp does the device-wide release (fence + atomic) for them, then polls the
+//            device counter and raises a shared-memory flag the producers look at.  The requests
+//            go through the kernel in two halves, so each half's barrier latency is covered by the
+//            other half's streaming.  The W_d rows do not wait for the barrier at all: they are
+//            requested the moment a ring slot comes free; only the h rows wait for it.
 //   phase 2  every CTA owns a contiguous range of the d_model output rows (d/G of them, so the
 //            split is even to within one row) for ALL virtual requests of the launch.  Tile =
 //            up to 16 of those W_d rows of one virtual request; warp w computes rows w and w + 8
@@ -51,8 +55,9 @@ namespace melinoe {
 namespace {
 
 constexpr int kConsumerWarps = 8;
-constexpr int kProducerWarps = 4;                    // a warp needs ~0.6 us to get one stage's copies out
-constexpr int kThreads = (kConsumerWarps + kProducerWarps) * 32;
+constexpr int kProducerWarps = 3;                    // a warp needs ~0.6 us to get one stage's copies out
+constexpr int kSyncWarp = kConsumerWarps + kProducerWarps;   // the warp that runs the grid barrier
+constexpr int kThreads = (kConsumerWarps + kProducerWarps + 1) * 32;
 constexpr int kMaxStages = 8;
 constexpr int kMaxSub = 16;                          // sub-stages of the down phase, over the whole ring
 constexpr int kMaxChunk = 4096;                      // bytes of one row piece
@@ -169,6 +174,8 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
 {
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ int s_abort;
+    __shared__ int s_passed[2];                 // half's h is complete on every CTA
+    __shared__ __align__(8) uint64_t s_harr[2]; // consumer warps that have stored their part of the half's h
     __shared__ VrRec s_vrs[kVrShared];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -217,11 +224,15 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
     const uint32_t full2 = empty1 + 8 * kMaxStages, empty2 = full2 + 8 * kMaxSub;
     volatile int *abort_flag = &s_abort;
 
+    const uint32_t harr = smem_u32(s_harr);
     if (tid == 0) {
         s_abort = 0;
+        s_passed[0] = s_passed[1] = 0;
+        for (int i = 0; i < 2; ++i)
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(harr + 8 * i), "r"(kConsumerWarps));
         for (int i = 0; i < kMaxSub; ++i) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(full2 + 8 * i), "r"(1));
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(empty2 + 8 * i), "r"(kConsumerWarps));
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(empty2 + 8 * i), "r"(kConsumerWarps / geo.groups2));
         }
         for (int i = 0; i < kMaxStages; ++i) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(full1 + 8 * i), "r"(1));
@@ -256,40 +267,93 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
     const int nk1 = (rb1 + CB1 - 1) / CB1, nk2 = (rb2 + CB2 - 1) / CB2;
     const int n_half = nv >= 2 ? 2 : 1;
     const int nvA = n_half == 2 ? nv / 2 : nv;                // requests in half A
-    int q_lo[2], q_hi[2];                                     // f-row ranges, relative to the half's first request
-    {
-        const long long rowsA = (long long)nvA * F, rowsB = (long long)(nv - nvA) * F;
-        q_lo[0] = (int)(blockIdx.x * rowsA / G);
-        q_hi[0] = (int)((blockIdx.x + 1) * rowsA / G);
-        q_lo[1] = (int)(blockIdx.x * rowsB / G);
-        q_hi[1] = (int)((blockIdx.x + 1) * rowsB / G);
-    }
+    // f-row ranges, relative to the half's first request (scalars, not arrays: an array indexed by
+    // the half would live in local memory)
+    const long long rowsA = (long long)nvA * F, rowsB = (long long)(nv - nvA) * F;
+    const int q_loA = (int)(blockIdx.x * rowsA / G), q_hiA = (int)((blockIdx.x + 1) * rowsA / G);
+    const int q_loB = (int)(blockIdx.x * rowsB / G), q_hiB = (int)((blockIdx.x + 1) * rowsB / G);
     const int r_lo = (int)((long long)blockIdx.x * d / G), r_hi = (int)((long long)(blockIdx.x + 1) * d / G);
     const int mt = (r_hi - r_lo + 15) / 16;
     const int hi2 = nv * mt, hi2A = nvA * mt;                 // down tiles: request-major, half A first
     unsigned *sync_word = p.sync + 2 * p.group;               // [half]
 
     // Down stage j (counted from 0 within the phase) lives in ring slot (n1 + j / NS2) mod S1, sub-stage
-    // j mod NS2: the slots are taken in the order in which the gate/up phase lets go of them.
+    // j mod NS2: the slots are taken in the order in which the gate/up phase lets go of them.  A
+    // cursor walks that sequence without divisions.
     struct Down {
-        uint32_t slot, bar, use, off;
+        uint32_t slot, sub, use, r;
     };
-    auto down_stage = [&](uint32_t n1_, uint32_t j) -> Down {
-        Down x;
-        x.slot = (n1_ + j / NS2) % S1;
-        const uint32_t sub = j % NS2;
-        x.bar = x.slot * NS2 + sub;
-        x.use = j / (uint32_t)(S1 * NS2);
-        x.off = x.slot * STAGE1 + sub * SUB2;
-        return x;
+    auto down_first = [&](uint32_t n1_) -> Down { return Down{n1_ % (uint32_t)S1, 0u, 0u, 0u}; };
+    auto down_next = [&](Down &x) {
+        if (++x.sub == (uint32_t)NS2) {
+            x.sub = 0;
+            if (++x.slot == (uint32_t)S1)
+                x.slot = 0;
+        }
+        if (++x.r == (uint32_t)(S1 * NS2)) {
+            x.r = 0;
+            ++x.use;
+        }
     };
+    auto down_bar = [&](const Down &x) -> uint32_t { return x.slot * NS2 + x.sub; };
+    auto down_off = [&](const Down &x) -> uint32_t { return x.slot * STAGE1 + x.sub * SUB2; };
+
+    if (warp == kSyncWarp) {
+        // =================================================================== grid barrier
+        // One lane: when the eight consumer warps have stored their part of a half's h, publish it
+        // device-wide (fence, then count this CTA in); then watch the half's counter and tell the
+        // producers when every CTA is in.
+        if (lane != 0)
+            return;
+        unsigned arrived = 0, passed = 0;
+        const unsigned all = (1u << n_half) - 1u;
+        const long long t0 = clock64();
+        while (passed != all) {
+            for (int half = 0; half < n_half; ++half) {
+                const unsigned bit = 1u << half;
+                if (!(arrived & bit)) {
+                    // the fence below takes microseconds while the SM streams: an earlier half that is
+                    // still being watched goes first
+                    if (half > 0 && !(passed & (bit >> 1)))
+                        continue;
+                    if (mbar_try(harr + 8 * half, 0)) {
+                        __threadfence();
+                        fence_proxy_async();   // h was written through the generic proxy, bulk copies will read it
+                        atomicAdd(sync_word + half, 1u);
+                        arrived |= bit;
+                        if (trace && half == n_half - 1)
+                            trace[4] = globaltimer_ns();
+                    }
+                } else if (!(passed & bit)) {
+                    unsigned v;
+                    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(sync_word + half) : "memory");
+                    if (v >= (unsigned)G) {
+                        fence_proxy_async();
+                        __threadfence_block();
+                        *reinterpret_cast<volatile int *>(&s_passed[half]) = 1;
+                        passed |= bit;
+                        if (trace && half == n_half - 1)
+                            trace[5] = globaltimer_ns();
+                    }
+                }
+            }
+            if (*abort_flag)
+                break;
+            if (clock64() - t0 > kWaitLimitCycles) {
+                *abort_flag = 1;
+                break;
+            }
+            __nanosleep(100);
+        }
+        return;
+    }
 
     if (warp >= kConsumerWarps) {
         // =================================================================== producers
         // The producer warps walk the same stage sequence and share the stages out (a warp is busy
         // for ~0.6 us with one bulk-copy instruction, however few lanes take part, so the stages
         // of a 28 KB-per-stage phase would otherwise leave faster than one warp can issue them).
-        // A ring slot always belongs to the same warp (slot s to warp s mod 4), so every wait on a
+        // A ring slot always belongs to the same warp (slot s to warp s mod 3), so every wait on a
         // slot's "empty" barrier is made by the one warp that has followed all its earlier phases.
         // Lanes 0..15 fetch the tile's weight rows, lanes 16..23 the operand rows.
         const int pw = warp - kConsumerWarps;
@@ -318,10 +382,11 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
         uint32_t n1 = 0;
         for (int half = 0; half < n_half; ++half) {
             const int v0 = vb + (half ? nvA : 0);
-            int q = q_lo[half];
-            while (q < q_hi[half]) {
+            const int q_end = half ? q_hiB : q_hiA;
+            int q = half ? q_loB : q_loA;
+            while (q < q_end) {
                 const int vr = v0 + q / F, f0 = q % F;
-                const int m = min(min(8, F - f0), q_hi[half] - q);
+                const int m = min(min(8, F - f0), q_end - q);
                 const VrRec *v = vrs + (vr - vb);
                 const char *src = nullptr;
                 if (lane_used) {
@@ -345,97 +410,103 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
         }
         // ---- down: lanes 0..15 W_d rows, 16..23 rows of h.  Two cursors walk the same stage
         // sequence: the weight rows run ahead as far as the ring allows, the h rows of a stage
-        // follow once the grid has finished the h of the stage's half.
+        // follow once the grid has finished the h of the stage's half.  A slot stays with the warp
+        // that served it in the gate/up phase: that warp has followed every phase of the slot's
+        // "empty" barrier, so its parity test of the slot's last gate/up use cannot be fooled by
+        // an older phase.
         struct Cursor {
-            int t, k, vr;
+            int t, k, blk, v, base_v;
             const char *base;
         };
         auto tile_of = [&](Cursor &c) -> const char * {
-            const int vr = vb + c.t / mt, blk = c.t % mt;
-            if (vr != c.vr) {
-                const VrRec *v = vrs + (vr - vb);
-                c.vr = vr;
+            if (c.v != c.base_v) {
+                const VrRec *v = vrs + c.v;
+                c.base_v = c.v;
                 c.base = nullptr;
                 if (lane_used) {
                     if (is_w)
                         c.base = v->blob + (size_t)2 * F * rb1 + (size_t)(r_lo + my_row) * rb2;
                     else if (my_row < v->n_tok)
-                        c.base = reinterpret_cast<const char *>(p.hbuf) + ((size_t)vr * kTokPerVr + my_row) * Fpad * 2;
+                        c.base = reinterpret_cast<const char *>(p.hbuf) + ((size_t)(vb + c.v) * kTokPerVr + my_row) * Fpad * 2;
                 }
             }
             if (!is_w)
                 return c.base;
             if (contig2 && lane != 0)
                 return nullptr;          // lane 0 fetches the tile's rows as one block
-            return (c.base && r_lo + 16 * blk + my_row < r_hi) ? c.base + (size_t)blk * 16 * rb2 : nullptr;
+            return (c.base && r_lo + 16 * c.blk + my_row < r_hi) ? c.base + (size_t)c.blk * 16 * rb2 : nullptr;
         };
-        auto rows_of = [&](const Cursor &c) { return min(16, r_hi - r_lo - 16 * (c.t % mt)); };
+        auto rows_of = [&](const Cursor &c) { return min(16, r_hi - r_lo - 16 * c.blk); };
         auto advance = [&](Cursor &c) {
             if (++c.k == nk2) {
                 c.k = 0;
                 ++c.t;
+                if (++c.blk == mt) {
+                    c.blk = 0;
+                    ++c.v;
+                }
             }
         };
-        auto w_bytes2 = [&](int kc) { return min(CB2, rb2 - kc * CB2); };    // one row's piece
-        auto op_bytes2 = [&](int kc) { return min(CB2, rb2 - kc * CB2); };
+        auto piece2 = [&](int kc) { return min(CB2, rb2 - kc * CB2); };    // one row's piece
         const uint32_t N2 = (uint32_t)hi2 * nk2;
-        Cursor wc{0, 0, -1, nullptr}, oc{0, 0, -1, nullptr};
+        Cursor wc{0, 0, 0, 0, -1, nullptr}, oc{0, 0, 0, 0, -1, nullptr};
+        Down wd = down_first(n1), od = wd;
         uint32_t wn = 0, on = 0;
-        bool passed[2] = {false, false};
+        bool passedA = false, passedB = false;
         long long t_idle = 0;
         while (on < N2 && !dead) {
             bool progress = false;
             // weight rows of as many stages as there are free sub-stages
             while (wn < N2) {
-                const Down ds = down_stage(n1, wn);
-                if ((int)(ds.slot % kProducerWarps) != pw) {
-                    (void)tile_of(wc);
-                    advance(wc);
-                    ++wn;
-                    progress = true;
-                    continue;
-                }
-                // free when its previous down-phase use has been consumed, or, on first use, when the
-                // gate/up phase has let go of the slot for good
-                int ok = 1;
-                if (lane == 0) {
-                    if (ds.use > 0) {
-                        ok = mbar_try(empty2 + 8 * ds.bar, (ds.use - 1u) & 1u);
-                    } else if (n1 > ds.slot) {
-                        const uint32_t m_last = n1 - 1u - ((n1 - 1u - ds.slot) % S1);
-                        ok = mbar_try(empty1 + 8 * ds.slot, (m_last / S1) & 1u);
+                const uint32_t bar = down_bar(wd);
+                if ((int)(wd.slot % kProducerWarps) == pw) {
+                    // free when its previous down-phase use has been consumed, or, on first use, when the
+                    // gate/up phase has let go of the slot for good
+                    int ok = 1;
+                    if (lane == 0) {
+                        if (wd.use > 0) {
+                            ok = mbar_try(empty2 + 8 * bar, (wd.use - 1u) & 1u);
+                        } else if (n1 > wd.slot) {
+                            const uint32_t m_last = n1 - 1u - ((n1 - 1u - wd.slot) % S1);
+                            ok = mbar_try(empty1 + 8 * wd.slot, (m_last / S1) & 1u);
+                        }
                     }
+                    if (!__shfl_sync(0xffffffffu, ok, 0))
+                        break;
+                    const char *src = tile_of(wc);
+                    issue(src, full2 + 8 * bar, down_off(wd), PITCH2, (size_t)wc.k * CB2,
+                          contig2 ? rows_of(wc) * rb2 : piece2(wc.k), piece2(wc.k), 1);
                 }
-                if (!__shfl_sync(0xffffffffu, ok, 0))
-                    break;
-                const char *src = tile_of(wc);
-                issue(src, full2 + 8 * ds.bar, ds.off, PITCH2, (size_t)wc.k * CB2,
-                      contig2 ? rows_of(wc) * rb2 : w_bytes2(wc.k), op_bytes2(wc.k), 1);
                 advance(wc);
+                down_next(wd);
                 ++wn;
                 progress = true;
             }
             // h rows of the next stages, once their half of h is complete everywhere
             if (on < wn) {
                 const int half = oc.t < hi2A ? 0 : 1;
-                if (!passed[half]) {
+                if (!(half ? passedB : passedA)) {
                     int ok = 0;
-                    if (lane == 0) {
-                        ok = *reinterpret_cast<volatile unsigned *>(sync_word + half) >= (unsigned)G;
-                        if (ok) {
-                            __threadfence();
-                            if (trace && pw == 0)
-                                trace[5] = globaltimer_ns();
-                        }
+                    if (lane == 0)
+                        ok = *reinterpret_cast<volatile int *>(&s_passed[half]);
+                    ok = __shfl_sync(0xffffffffu, ok, 0);
+                    if (ok) {
+                        __threadfence_block();
+                        fence_proxy_async();
+                        if (half)
+                            passedB = true;
+                        else
+                            passedA = true;
                     }
-                    passed[half] = __shfl_sync(0xffffffffu, ok, 0) != 0;
                 }
-                while (on < wn && passed[oc.t < hi2A ? 0 : 1]) {
-                    const char *src = tile_of(oc);
-                    const Down ds = down_stage(n1, on);
-                    if ((int)(ds.slot % kProducerWarps) == pw)
-                        issue(src, full2 + 8 * ds.bar, ds.off, PITCH2, (size_t)oc.k * CB2, 0, op_bytes2(oc.k), 2);
+                while (on < wn && (oc.t < hi2A ? passedA : passedB)) {
+                    const uint32_t bar = down_bar(od);
+                    if ((int)(od.slot % kProducerWarps) == pw) {
+                        const char *src = tile_of(oc);
+                        issue(src, full2 + 8 * bar, down_off(od), PITCH2, (size_t)oc.k * CB2, 0, piece2(oc.k), 2);
+                    }
                     advance(oc);
+                    down_next(od);
                     ++on;
                     progress = true;
                 }
@@ -452,6 +523,9 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
                     *abort_flag = 1;
                     dead = true;
                 }
+                // a warp that polls without pause takes issue slots and shared-memory pipeline
+                // cycles from the consumer warps
+                __nanosleep(100);
             }
         }
         const uint32_t n2 = on;
@@ -460,9 +534,11 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
             // CTA's shared memory goes away
             const long long t0 = clock64();
             const uint32_t in_ring = (uint32_t)(S1 * NS2);
-            for (uint32_t j = n2 > in_ring ? n2 - in_ring : 0u; j < n2; ++j) {
-                const Down ds = down_stage(n1, j);
-                while (!mbar_try(full2 + 8 * ds.bar, ds.use & 1u) && clock64() - t0 < kWaitLimitCycles) {
+            Down x = down_first(n1);
+            for (uint32_t j = 0; j < n2; ++j, down_next(x)) {
+                if (j + in_ring < n2)
+                    continue;
+                while (!mbar_try(full2 + 8 * down_bar(x), x.use & 1u) && clock64() - t0 < kWaitLimitCycles) {
                 }
             }
             atomicExch(p.err, MELINOE_ERR_TIMEOUT);
@@ -562,10 +638,11 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
             const int v0 = vb + (half ? nvA : 0);
             int cur_vr = -1;
             VrInfo v{};
-            int q = q_lo[half];
-            while (q < q_hi[half]) {
+            const int q_end = half ? q_hiB : q_hiA;
+            int q = half ? q_loB : q_loA;
+            while (q < q_end) {
                 const int vr = v0 + q / F, f0 = q % F;
-                const int m = min(min(8, F - f0), q_hi[half] - q);
+                const int m = min(min(8, F - f0), q_end - q);
                 if (vr != cur_vr) {
                     v = load_vr(vr);
                     cur_vr = vr;
@@ -589,104 +666,156 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
             }
             if (trace && tid == 0 && half == n_half - 1)
                 trace[3] = globaltimer_ns();
-            // this CTA's part of the half's h is complete: tell the grid
-            __threadfence();
-            fence_proxy_async();       // h was written through the generic proxy, bulk copies will read it
-            consumer_bar();
-            if (tid == 0) {
-                atomicAdd(sync_word + half, 1u);
-                if (trace && half == n_half - 1)
-                    trace[4] = globaltimer_ns();
-            }
+            // this warp's part of the half's h is stored: the barrier warp takes it from here
+            __syncwarp();
+            if (lane == 0)
+                mbar_arrive(harr + 8 * half);
         }
     }
 
-    // ---- down: z = W_d h for this CTA's output rows.  Warp w owns tile rows w and w + 8: plain
-    // 16-byte loads along the row, fp32 dot products against the h rows behind the weights, a warp
-    // reduction per (row, token), no synchronisation between the warps.
+    // ---- down: z = W_d h for this CTA's output rows, as plain fp32 dot products: 16-byte loads
+    // along the row, four per lane in flight, two independent chains per (row, token), a warp
+    // reduction per (row, token), complete sums.  The eight warps form NG groups; a sub-stage of the
+    // ring always belongs to the same group (its index mod NG: a warp that waited for phase k + 1 of a
+    // barrier whose phase k it has not seen could be let through by the parity test), a tile is
+    // worked on by the group of the sub-stage it lands in, and the group's warps share out its rows (warp wl of WPG = 8 / NG takes rows wl,
+    // wl + WPG, ...).  With short W_d rows a tile is small and what one tile costs is mostly
+    // latency (seeing the barrier, the loads, the shuffles), so the tiles of the ring are worked on
+    // side by side by single warps (NG = 8); with long rows NG = 1 and every stage is shared by all
+    // warps.  No synchronisation between the warps either way.
     {
-        const uint32_t n1c = n;      // gate/up stages of this CTA: the down phase takes the slots in ring order
-        uint32_t j2 = 0;             // down stages consumed
-        for (int t = 0; t < hi2; ++t) {
-            const int blk = t % mt, vr = vb + t / mt;
-            const VrRec *vrec = vrs + (vr - vb);
+        Down dc = down_first(n);     // the down phase takes the slots in ring order after the gate/up stages
+        bool first = true;
+        auto dot8 = [](const uint4 &w, const uint4 &h, float &a0, float &a1) {
+            a0 = fmaf(__uint_as_float(w.x << 16), __uint_as_float(h.x << 16), a0);
+            a1 = fmaf(__uint_as_float(w.x & 0xffff0000u), __uint_as_float(h.x & 0xffff0000u), a1);
+            a0 = fmaf(__uint_as_float(w.y << 16), __uint_as_float(h.y << 16), a0);
+            a1 = fmaf(__uint_as_float(w.y & 0xffff0000u), __uint_as_float(h.y & 0xffff0000u), a1);
+            a0 = fmaf(__uint_as_float(w.z << 16), __uint_as_float(h.z << 16), a0);
+            a1 = fmaf(__uint_as_float(w.z & 0xffff0000u), __uint_as_float(h.z & 0xffff0000u), a1);
+            a0 = fmaf(__uint_as_float(w.w << 16), __uint_as_float(h.w << 16), a0);
+            a1 = fmaf(__uint_as_float(w.w & 0xffff0000u), __uint_as_float(h.w & 0xffff0000u), a1);
+        };
+        const int NG = geo.groups2, WPG = kConsumerWarps / NG;
+        const int grp = warp / WPG, wl = warp % WPG;
+        for (int v = 0; v < nv; ++v) {
+            const VrRec *vrec = vrs + v;
             const int n_tok = vrec->n_tok;
-            const int n_rows = min(16, r_hi - r_lo - 16 * blk);
-            // the token loops are unrolled for the smallest of 1, 2, 4, 8 that covers the request's
-            // tokens (predicated-off iterations would still cost issue slots)
-            auto run_tile = [&](auto nt_tag) {
-                constexpr int NT = decltype(nt_tag)::value;
-                float acc[2][NT];
+            for (int blk = 0; blk < mt; ++blk) {
+                if ((int)(down_bar(dc) & (uint32_t)(NG - 1)) != grp) {
+                    for (int kc = 0; kc < nk2; ++kc)
+                        down_next(dc);
+                    continue;
+                }
+                const int n_rows = min(16, r_hi - r_lo - 16 * blk);
+                // RPW rows per warp; the token loops are unrolled for the smallest of 1, 2, 4, 8 that
+                // covers the request's tokens (predicated-off iterations would still cost issue slots)
+                auto run_tile = [&](auto rpw_tag, auto nt_tag) {
+                    constexpr int RPW = decltype(rpw_tag)::value;
+                    constexpr int NT = decltype(nt_tag)::value;
+                    // two chains per (row, token) where there are few of those, one where there are many
+                    constexpr int NC = RPW * NT >= 8 ? 1 : 2;
+                    float acc[RPW][NT][NC];
 #pragma unroll
-                for (int j = 0; j < 2; ++j)
+                    for (int j = 0; j < RPW; ++j)
 #pragma unroll
-                    for (int tk = 0; tk < NT; ++tk)
-                        acc[j][tk] = 0.f;
-                for (int kc = 0; kc < nk2; ++kc, ++j2) {
-                    const Down ds = down_stage(n1c, j2);
-                    mbar_wait(full2 + 8 * ds.bar, ds.use & 1u, abort_flag);
-                    if (trace && j2 == 0 && tid == 0)
-                        trace[2] = globaltimer_ns();
-                    const unsigned char *base = ring + ds.off;
-                    const int nch = min(CB2, rb2 - kc * CB2) >> 4;
+                        for (int tk = 0; tk < NT; ++tk)
 #pragma unroll
-                    for (int j = 0; j < 2; ++j) {
-                        const int rr = warp + 8 * j;
-                        if (rr < n_rows) {
-                            const uint4 *wr = reinterpret_cast<const uint4 *>(base + (size_t)rr * PITCH2);
-                            for (int c = lane; c < nch; c += 32) {
-                                const uint4 w = wr[c];
-                                const float w0 = __uint_as_float(w.x << 16), w1 = __uint_as_float(w.x & 0xffff0000u);
-                                const float w2 = __uint_as_float(w.y << 16), w3 = __uint_as_float(w.y & 0xffff0000u);
-                                const float w4 = __uint_as_float(w.z << 16), w5 = __uint_as_float(w.z & 0xffff0000u);
-                                const float w6 = __uint_as_float(w.w << 16), w7 = __uint_as_float(w.w & 0xffff0000u);
+                            for (int q = 0; q < NC; ++q)
+                                acc[j][tk][q] = 0.f;
+                    for (int kc = 0; kc < nk2; ++kc) {
+                        mbar_wait(full2 + 8 * down_bar(dc), dc.use & 1u, abort_flag);
+                        if (trace && first && tid == 0)
+                            trace[2] = globaltimer_ns();
+                        first = false;
+                        const unsigned char *base = ring + down_off(dc);
+                        const int nch = min(CB2, rb2 - kc * CB2) >> 4;
+                        const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+                        for (int pr = 0; pr < RPW / 2; ++pr) {
+                            const int ra = wl + WPG * (2 * pr), rb = ra + WPG;
+                            if (ra >= n_rows)
+                                break;
+                            const bool has_b = rb < n_rows;
+                            const uint4 *wra = reinterpret_cast<const uint4 *>(base + (size_t)ra * PITCH2);
+                            const uint4 *wrb = reinterpret_cast<const uint4 *>(base + (size_t)rb * PITCH2);
+                            for (int c0 = lane; c0 < nch; c0 += 128) {
+                                uint4 wa[4], wb[4];
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) {
+                                    const int c = c0 + 32 * i;
+                                    wa[i] = c < nch ? wra[c] : zero;
+                                    wb[i] = (c < nch && has_b) ? wrb[c] : zero;
+                                }
 #pragma unroll
                                 for (int tk = 0; tk < NT; ++tk) {
                                     if (NT == 1 || tk < n_tok) {
-                                        const uint4 hv = reinterpret_cast<const uint4 *>(base + (size_t)(16 + tk) * PITCH2)[c];
-                                        float a = acc[j][tk];
-                                        a = fmaf(w0, __uint_as_float(hv.x << 16), a);
-                                        a = fmaf(w1, __uint_as_float(hv.x & 0xffff0000u), a);
-                                        a = fmaf(w2, __uint_as_float(hv.y << 16), a);
-                                        a = fmaf(w3, __uint_as_float(hv.y & 0xffff0000u), a);
-                                        a = fmaf(w4, __uint_as_float(hv.z << 16), a);
-                                        a = fmaf(w5, __uint_as_float(hv.z & 0xffff0000u), a);
-                                        a = fmaf(w6, __uint_as_float(hv.w << 16), a);
-                                        a = fmaf(w7, __uint_as_float(hv.w & 0xffff0000u), a);
-                                        acc[j][tk] = a;
+                                        const uint4 *hr = reinterpret_cast<const uint4 *>(base + (size_t)(16 + tk) * PITCH2);
+                                        uint4 hv[4];
+#pragma unroll
+                                        for (int i = 0; i < 4; ++i) {
+                                            const int c = c0 + 32 * i;
+                                            hv[i] = c < nch ? hr[c] : zero;
+                                        }
+#pragma unroll
+                                        for (int i = 0; i < 4; ++i) {
+                                            dot8(wa[i], hv[i], acc[2 * pr][tk][0], acc[2 * pr][tk][NC - 1]);
+                                            dot8(wb[i], hv[i], acc[2 * pr + 1][tk][0], acc[2 * pr + 1][tk][NC - 1]);
+                                        }
                                     }
                                 }
                             }
                         }
+                        __syncwarp();
+                        if (lane == 0)
+                            mbar_arrive(empty2 + 8 * down_bar(dc));
+                        down_next(dc);
                     }
-                    __syncwarp();
-                    if (lane == 0)
-                        mbar_arrive(empty2 + 8 * ds.bar);
-                }
+                    if (wl < n_rows) {
+                        float vals[RPW * NT];
 #pragma unroll
-                for (int j = 0; j < 2; ++j) {
-                    const int rr = warp + 8 * j;
+                        for (int j = 0; j < RPW; ++j)
 #pragma unroll
-                    for (int tk = 0; tk < NT; ++tk) {
-                        if (tk < n_tok && rr < n_rows) {
-                            float a = acc[j][tk];
+                            for (int tk = 0; tk < NT; ++tk)
+                                vals[j * NT + tk] = NC == 2 ? acc[j][tk][0] + acc[j][tk][NC - 1] : acc[j][tk][0];
 #pragma unroll
-                            for (int m = 16; m >= 1; m >>= 1)
-                                a += __shfl_xor_sync(0xffffffffu, a, m);
-                            if (lane == 0)
-                                p.zbuf[(size_t)vrec->pair[tk] * d + r_lo + 16 * blk + rr] = a;
+                        for (int m = 16; m >= 1; m >>= 1)
+#pragma unroll
+                            for (int q = 0; q < RPW * NT; ++q)
+                                vals[q] += __shfl_xor_sync(0xffffffffu, vals[q], m);
+                        // every lane holds every sum: lane q stores sum q
+                        float mine = 0.f;
+#pragma unroll
+                        for (int q = 0; q < RPW * NT; ++q)
+                            mine = lane == q ? vals[q] : mine;
+                        if (lane < RPW * NT) {
+                            const int j = lane / NT, tk = lane % NT;
+                            const int rr = wl + WPG * j;
+                            if (tk < n_tok && rr < n_rows)
+                                p.zbuf[(size_t)vrec->pair[tk] * d + r_lo + 16 * blk + rr] = mine;
                         }
                     }
-                }
-            };
-            if (n_tok <= 1)
-                run_tile(std::integral_constant<int, 1>{});
-            else if (n_tok <= 2)
-                run_tile(std::integral_constant<int, 2>{});
-            else if (n_tok <= 4)
-                run_tile(std::integral_constant<int, 4>{});
-            else
-                run_tile(std::integral_constant<int, 8>{});
+                };
+                auto by_tokens = [&](auto rpw_tag) {
+                    constexpr int RPW = decltype(rpw_tag)::value;
+                    if (n_tok <= 1)
+                        run_tile(rpw_tag, std::integral_constant<int, 1>{});
+                    else if constexpr (RPW <= 8) {
+                        if (n_tok <= 2)
+                            run_tile(rpw_tag, std::integral_constant<int, 2>{});
+                        else if constexpr (RPW <= 4) {
+                            if (n_tok <= 4)
+                                run_tile(rpw_tag, std::integral_constant<int, 4>{});
+                            else if constexpr (RPW <= 2)
+                                run_tile(rpw_tag, std::integral_constant<int, 8>{});
+                        }
+                    }
+                };
+                if (NG == 2)
+                    by_tokens(std::integral_constant<int, 4>{});
+                else
+                    by_tokens(std::integral_constant<int, 2>{});
+            }
         }
     }
     if (trace && tid == 0)
@@ -766,6 +895,12 @@ cudaError_t ffn_stream_geometry(const FfnLaunchCfg &cfg, int d, int F, int T, Ff
     while (ns2 * n > (size_t)kMaxSub)
         --ns2;
     geo->sub2 = (int)ns2;
+    // down phase: warp groups working on different tiles side by side.  Only where a tile is a single
+    // stage and the request's tokens are few (the accumulators are rows per warp x tokens).
+    {
+        const int nt = geo->n_op_rows <= 1 ? 1 : geo->n_op_rows <= 2 ? 2 : geo->n_op_rows <= 4 ? 4 : 8;
+        geo->groups2 = ((size_t)2 * F <= (size_t)geo->chunk_bytes2 && nt <= 4) ? 2 : 1;
+    }
     geo->sub_bytes2 = (int)sub;
     geo->ring_bytes = (n * stage + 127) / 128 * 128;
     geo->smem_bytes = geo->ring_bytes + fixed;
