@@ -6,8 +6,7 @@
 // longer one).
 //
 // One cooperative launch per compute group, one CTA per SM: eight consumer warps, three producer
-// warps and one warp for the grid barrier (twelve warps: a thirteenth would cost every thread
-// registers, which are handed out to warps in fours).  A "virtual request" is one expert with up to 8 of its tokens.
+// warps and two warps for the grid barrier.  A "virtual request" is one expert with up to 8 of its tokens.
 //
 //   phase 1  tile = up to 8 rows of W_g plus the same rows of W_u of one virtual request.
 //            D[16 x 8] = [W_g rows; W_u rows] (16 x d) * x^T (d x 8 tokens) on mma.sync
@@ -19,7 +18,7 @@
 //            to global memory (a fence after the h stores, a poll of a device counter) takes
 //            microseconds, so neither the consumers nor the producers ever make one: the consumer
 //            warps arrive on a shared-memory barrier when their part of h is stored and go on; a
-//            twelfth warp does the device-wide release (fence + atomic) for them, then polls the
+//            warp of its own does the device-wide release (fence + atomic) for them, another polls the
 //            device counter and raises a shared-memory flag the producers look at.  The requests
 //            go through the kernel in two halves, so each half's barrier latency is covered by the
 //            other half's streaming.  The W_d rows do not wait for the barrier at all: they are
@@ -57,7 +56,7 @@ namespace {
 constexpr int kConsumerWarps = 8;
 constexpr int kProducerWarps = 3;                    // a warp needs ~0.6 us to get one stage's copies out
 constexpr int kSyncWarp = kConsumerWarps + kProducerWarps;   // the warp that runs the grid barrier
-constexpr int kThreads = (kConsumerWarps + kProducerWarps + 1) * 32;
+constexpr int kThreads = (kConsumerWarps + kProducerWarps + 2) * 32;
 constexpr int kMaxStages = 8;
 constexpr int kMaxSub = 16;                          // sub-stages of the down phase, over the whole ring
 constexpr int kMaxChunk = 4096;                      // bytes of one row piece
@@ -185,16 +184,12 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
     const int NOP = geo.n_op_rows;
     (void)NOP;
     const int S1 = geo.n_stages, PITCH1 = geo.pitch, CB1 = geo.chunk_bytes, STAGE1 = geo.stage_bytes;
-    // down phase: rows of 2*F bytes.  When a whole row fits one piece, the CTA's rows of an expert
-    // are one contiguous block of global memory and travel as ONE bulk copy (the bulk-copy engine
-    // keeps a limited number of requests in flight, so 2 KB requests stream at half the rate of
-    // 4 KB ones); rows sit unpadded in the stage, which is fine because this phase reads them
-    // with plain 16-byte loads, one row per warp.
-    // A down stage is often much smaller than a gate/up stage (short W_d rows), so a ring slot is
-    // cut into NS2 sub-stages for the down phase: more tiles in flight where each tile is small.
-    const int CB2 = geo.chunk_bytes2, NS2 = geo.sub2, SUB2 = geo.sub_bytes2;
-    const bool contig2 = 2 * F <= CB2;
-    const int PITCH2 = contig2 ? 2 * F : CB2;
+    // down phase: rows of 2*F bytes in pieces of at most CB2, laid out like the gate/up stages (one
+    // piece of every weight row of the tile, the h rows behind them at row ROWS2, padded pitch).  A
+    // down stage is often much smaller than a gate/up stage (short W_d rows, fewer than 16 rows per
+    // CTA), so a ring slot is cut into NS2 sub-stages for the down phase: more tiles in flight
+    // where each tile is small.
+    const int CB2 = geo.chunk_bytes2, NS2 = geo.sub2, SUB2 = geo.sub_bytes2, PITCH2 = geo.pitch2, ROWS2 = geo.rows2;
 
     // optional timeline: 8 device-clock stamps per CTA (see melinoe_moe_set_trace)
     unsigned long long *trace = p.trace ? p.trace + (size_t)blockIdx.x * 8 : nullptr;
@@ -232,7 +227,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(harr + 8 * i), "r"(kConsumerWarps));
         for (int i = 0; i < kMaxSub; ++i) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(full2 + 8 * i), "r"(1));
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(empty2 + 8 * i), "r"(kConsumerWarps / geo.groups2));
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(empty2 + 8 * i), "r"(1));
         }
         for (int i = 0; i < kMaxStages; ++i) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(full1 + 8 * i), "r"(1));
@@ -266,7 +261,9 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
     const int rb1 = 2 * d, rb2 = 2 * F;                       // row bytes
     const int nk1 = (rb1 + CB1 - 1) / CB1, nk2 = (rb2 + CB2 - 1) / CB2;
     const int n_half = nv >= 2 ? 2 : 1;
-    const int nvA = n_half == 2 ? nv / 2 : nv;                // requests in half A
+    // The second part is the smaller one: what follows its barrier is exposed, what follows the
+    // first part's barrier is covered by the second part's gate/up rows.
+    const int nvA = n_half == 2 ? nv - (nv + 2) / 4 : nv;     // requests in the first part
     // f-row ranges, relative to the half's first request (scalars, not arrays: an array indexed by
     // the half would live in local memory)
     const long long rowsA = (long long)nvA * F, rowsB = (long long)(nv - nvA) * F;
@@ -299,56 +296,54 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
     auto down_off = [&](const Down &x) -> uint32_t { return x.slot * STAGE1 + x.sub * SUB2; };
 
     if (warp == kSyncWarp) {
-        // =================================================================== grid barrier
+        // =================================================================== grid barrier, arriving
         // One lane: when the eight consumer warps have stored their part of a half's h, publish it
-        // device-wide (fence, then count this CTA in); then watch the half's counter and tell the
-        // producers when every CTA is in.
+        // device-wide (fence, then count this CTA in).  The fence takes microseconds while the SM
+        // streams, which is why no warp with other work makes it.
         if (lane != 0)
             return;
-        unsigned arrived = 0, passed = 0;
-        const unsigned all = (1u << n_half) - 1u;
+        for (int half = 0; half < n_half; ++half) {
+            if (!mbar_wait(harr + 8 * half, 0, abort_flag))
+                break;
+            __threadfence();
+            fence_proxy_async();   // h was written through the generic proxy, bulk copies will read it
+            atomicAdd(sync_word + half, 1u);
+            if (trace && half == n_half - 1)
+                trace[4] = globaltimer_ns();
+        }
+        return;
+    }
+    if (warp == kSyncWarp + 1) {
+        // =================================================================== grid barrier, watching
+        // One lane: watch the halves' counters (in order: the first half is complete everywhere
+        // before the second is) and tell the producers through a shared-memory flag.
+        if (lane != 0)
+            return;
         const long long t0 = clock64();
-        while (passed != all) {
-            for (int half = 0; half < n_half; ++half) {
-                const unsigned bit = 1u << half;
-                if (!(arrived & bit)) {
-                    // the fence below takes microseconds while the SM streams: an earlier half that is
-                    // still being watched goes first
-                    if (half > 0 && !(passed & (bit >> 1)))
-                        continue;
-                    if (mbar_try(harr + 8 * half, 0)) {
-                        __threadfence();
-                        fence_proxy_async();   // h was written through the generic proxy, bulk copies will read it
-                        atomicAdd(sync_word + half, 1u);
-                        arrived |= bit;
-                        if (trace && half == n_half - 1)
-                            trace[4] = globaltimer_ns();
-                    }
-                } else if (!(passed & bit)) {
-                    unsigned v;
-                    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(sync_word + half) : "memory");
-                    if (v >= (unsigned)G) {
-                        fence_proxy_async();
-                        __threadfence_block();
-                        *reinterpret_cast<volatile int *>(&s_passed[half]) = 1;
-                        passed |= bit;
-                        if (trace && half == n_half - 1)
-                            trace[5] = globaltimer_ns();
-                    }
+        for (int half = 0; half < n_half; ++half) {
+            for (;;) {
+                unsigned v;
+                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(sync_word + half) : "memory");
+                if (v >= (unsigned)G)
+                    break;
+                if (*abort_flag)
+                    return;
+                if (clock64() - t0 > kWaitLimitCycles) {
+                    *abort_flag = 1;
+                    return;
                 }
+                __nanosleep(100);
             }
-            if (*abort_flag)
-                break;
-            if (clock64() - t0 > kWaitLimitCycles) {
-                *abort_flag = 1;
-                break;
-            }
-            __nanosleep(100);
+            fence_proxy_async();
+            __threadfence_block();
+            *reinterpret_cast<volatile int *>(&s_passed[half]) = 1;
+            if (trace && half == n_half - 1)
+                trace[5] = globaltimer_ns();
         }
         return;
     }
 
-    if (warp >= kConsumerWarps) {
+    if (warp >= kConsumerWarps && warp < kSyncWarp) {
         // =================================================================== producers
         // The producer warps walk the same stage sequence and share the stages out (a warp is busy
         // for ~0.6 us with one bulk-copy instruction, however few lanes take part, so the stages
@@ -359,14 +354,14 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
         const int pw = warp - kConsumerWarps;
         const bool is_w = lane < 16;
         const int my_row = is_w ? lane : lane - 16;                        // tile row, or token slot
-        const int dst_row = lane;
+        const int dst_row2 = is_w ? lane : ROWS2 + my_row;             // row of a down sub-stage
         const bool lane_used = lane < 24;
         bool dead = false;
         // One stage of either phase.  src: this lane's source row or null.  parts bit 0: arm the
         // barrier and fetch the weight rows (the caller has made sure the slot is free); bit 1:
         // operand rows.
-        auto issue = [&](const char *src, uint32_t bar, uint32_t stage_off, int PITCH, size_t src_off, int wbytes,
-                         int obytes, int parts) {
+        auto issue = [&](const char *src, uint32_t bar, uint32_t stage_off, int PITCH, int dst_row, size_t src_off,
+                         int wbytes, int obytes, int parts) {
             const bool active = lane_used && src != nullptr;
             if (parts & 1) {
                 const unsigned mw = __ballot_sync(0xffffffffu, active && is_w);
@@ -403,7 +398,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
                     if (n1 >= (uint32_t)S1 && !dead)
                         dead = !mbar_wait(empty1 + 8 * (n1 % S1), ((n1 / S1) - 1u) & 1u, abort_flag);
                     const int b = min(CB1, rb1 - kc * CB1);
-                    issue(src, full1 + 8 * (n1 % S1), (n1 % S1) * STAGE1, PITCH1, (size_t)kc * CB1, b, b, 3);
+                    issue(src, full1 + 8 * (n1 % S1), (n1 % S1) * STAGE1, PITCH1, lane, (size_t)kc * CB1, b, b, 3);
                 }
                 q += m;
             }
@@ -432,11 +427,8 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
             }
             if (!is_w)
                 return c.base;
-            if (contig2 && lane != 0)
-                return nullptr;          // lane 0 fetches the tile's rows as one block
             return (c.base && r_lo + 16 * c.blk + my_row < r_hi) ? c.base + (size_t)c.blk * 16 * rb2 : nullptr;
         };
-        auto rows_of = [&](const Cursor &c) { return min(16, r_hi - r_lo - 16 * c.blk); };
         auto advance = [&](Cursor &c) {
             if (++c.k == nk2) {
                 c.k = 0;
@@ -474,8 +466,8 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
                     if (!__shfl_sync(0xffffffffu, ok, 0))
                         break;
                     const char *src = tile_of(wc);
-                    issue(src, full2 + 8 * bar, down_off(wd), PITCH2, (size_t)wc.k * CB2,
-                          contig2 ? rows_of(wc) * rb2 : piece2(wc.k), piece2(wc.k), 1);
+                    issue(src, full2 + 8 * bar, down_off(wd), PITCH2, dst_row2, (size_t)wc.k * CB2, piece2(wc.k),
+                          piece2(wc.k), 1);
                 }
                 advance(wc);
                 down_next(wd);
@@ -491,8 +483,9 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
                         ok = *reinterpret_cast<volatile int *>(&s_passed[half]);
                     ok = __shfl_sync(0xffffffffu, ok, 0);
                     if (ok) {
+                        // the barrier warp has made the generic-proxy writes of h visible to the bulk
+                        // copies before it raised the flag
                         __threadfence_block();
-                        fence_proxy_async();
                         if (half)
                             passedB = true;
                         else
@@ -503,7 +496,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
                     const uint32_t bar = down_bar(od);
                     if ((int)(od.slot % kProducerWarps) == pw) {
                         const char *src = tile_of(oc);
-                        issue(src, full2 + 8 * bar, down_off(od), PITCH2, (size_t)oc.k * CB2, 0, piece2(oc.k), 2);
+                        issue(src, full2 + 8 * bar, down_off(od), PITCH2, dst_row2, (size_t)oc.k * CB2, 0, piece2(oc.k), 2);
                     }
                     advance(oc);
                     down_next(od);
@@ -549,19 +542,29 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
     // ======================================================================= consumers
     const int g = lane >> 2, tig = lane & 3;
     int n_tiles = 0;       // tiles finished so far (selects the reduction buffer and the epilogue warp)
-    float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
+    // four accumulator chains: an mma waits some 30 cycles for the one it accumulates onto
+    float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f}, c2[4] = {0.f, 0.f, 0.f, 0.f}, c3[4] = {0.f, 0.f, 0.f, 0.f};
 
     // this warp's share of one stage: some of the 16-column steps of the piece.  Weights in tile
     // rows 0..15, the operand rows (hidden or h) of the request's tokens behind them.
-    auto compute = [&](uint32_t full0, uint32_t empty0, int S, int STAGE, uint32_t a_off, uint32_t b_off, uint32_t n,
-                       int bytes, int n_tok) {
-        const uint32_t slot = n % S;
-        mbar_wait(full0 + 8 * slot, (n / S) & 1u, abort_flag);
-        const uint32_t base = ring_s + slot * STAGE;
-        const int ks_total = (bytes + 31) >> 5;
-        const int ks_hi = (warp + 1) * ks_total / kConsumerWarps;
-        int ks = warp * ks_total / kConsumerWarps;
-        const bool has_tok = g < n_tok;
+    // 16-column steps [ks, ks_hi) of a stage at shared address base: weights in stage rows 0..15 (a_off
+    // is this lane's ldmatrix row), operand rows behind them (b_off is this lane's fragment row)
+    auto mma_steps = [&](uint32_t base, uint32_t a_off, uint32_t b_off, int ks, int ks_hi, bool has_tok) {
+        for (; ks + 3 < ks_hi; ks += 4) {
+            uint32_t a[4][4], b[4][2];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                ldmatrix_x4(base + a_off + (ks + i) * 32, a[i][0], a[i][1], a[i][2], a[i][3]);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                b[i][0] = has_tok ? lds32(base + b_off + (ks + i) * 32) : 0u;
+                b[i][1] = has_tok ? lds32(base + b_off + (ks + i) * 32 + 16) : 0u;
+            }
+            mma_16816(c0, a[0][0], a[0][1], a[0][2], a[0][3], b[0][0], b[0][1]);
+            mma_16816(c1, a[1][0], a[1][1], a[1][2], a[1][3], b[1][0], b[1][1]);
+            mma_16816(c2, a[2][0], a[2][1], a[2][2], a[2][3], b[2][0], b[2][1]);
+            mma_16816(c3, a[3][0], a[3][1], a[3][2], a[3][3], b[3][0], b[3][1]);
+        }
         for (; ks + 1 < ks_hi; ks += 2) {
             uint32_t a0, a1, a2, a3, e0, e1, e2, e3;
             ldmatrix_x4(base + a_off + ks * 32, a0, a1, a2, a3);
@@ -586,6 +589,15 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
             }
             mma_16816(c0, a0, a1, a2, a3, b0, b1);
         }
+    };
+    // gate/up: this warp's share of one stage, an eighth of the piece's 16-column steps
+    auto compute = [&](uint32_t full0, uint32_t empty0, int S, int STAGE, uint32_t a_off, uint32_t b_off, uint32_t n,
+                       int bytes, int n_tok) {
+        const uint32_t slot = n % S;
+        mbar_wait(full0 + 8 * slot, (n / S) & 1u, abort_flag);
+        const int ks_total = (bytes + 31) >> 5;
+        mma_steps(ring_s + slot * STAGE, a_off, b_off, warp * ks_total / kConsumerWarps,
+                  (warp + 1) * ks_total / kConsumerWarps, g < n_tok);
         __syncwarp();
         if (lane == 0)
             mbar_arrive(empty0 + 8 * slot);
@@ -596,8 +608,8 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
         float *buf = red + (n_tiles & 1) * (kConsumerWarps * 128);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            buf[warp * 128 + i * 32 + lane] = c0[i] + c1[i];
-            c0[i] = c1[i] = 0.f;
+            buf[warp * 128 + i * 32 + lane] = (c0[i] + c1[i]) + (c2[i] + c3[i]);
+            c0[i] = c1[i] = c2[i] = c3[i] = 0.f;
         }
         consumer_bar();
         const bool mine = warp == (n_tiles & (kConsumerWarps - 1));
@@ -673,148 +685,61 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
         }
     }
 
-    // ---- down: z = W_d h for this CTA's output rows, as plain fp32 dot products: 16-byte loads
-    // along the row, four per lane in flight, two independent chains per (row, token), a warp
-    // reduction per (row, token), complete sums.  The eight warps form NG groups; a sub-stage of the
-    // ring always belongs to the same group (its index mod NG: a warp that waited for phase k + 1 of a
-    // barrier whose phase k it has not seen could be let through by the parity test), a tile is
-    // worked on by the group of the sub-stage it lands in, and the group's warps share out its rows (warp wl of WPG = 8 / NG takes rows wl,
-    // wl + WPG, ...).  With short W_d rows a tile is small and what one tile costs is mostly
-    // latency (seeing the barrier, the loads, the shuffles), so the tiles of the ring are worked on
-    // side by side by single warps (NG = 8); with long rows NG = 1 and every stage is shared by all
-    // warps.  No synchronisation between the warps either way.
+    // ---- down: z = W_d h for this CTA's output rows.  A tile (up to 16 output rows of one request)
+    // belongs to ONE warp, tile j to warp j mod 8: D[16 rows x 8 tokens] accumulates in that warp's
+    // registers over all the pieces of the rows, so nothing is reduced across warps or lanes and
+    // the tiles in the ring are worked on side by side.  (A tile of short rows costs its warp a few
+    // hundred instructions; shared out over eight warps it would cost each of them mostly the
+    // latency of seeing the barrier and of meeting the others.)  Every warp waits for every stage
+    // in order, also those of other warps' tiles: a warp that waited for phase k + 1 of a barrier
+    // whose phase k it has not seen could be let through by the parity test.
     {
         Down dc = down_first(n);     // the down phase takes the slots in ring order after the gate/up stages
         bool first = true;
-        auto dot8 = [](const uint4 &w, const uint4 &h, float &a0, float &a1) {
-            a0 = fmaf(__uint_as_float(w.x << 16), __uint_as_float(h.x << 16), a0);
-            a1 = fmaf(__uint_as_float(w.x & 0xffff0000u), __uint_as_float(h.x & 0xffff0000u), a1);
-            a0 = fmaf(__uint_as_float(w.y << 16), __uint_as_float(h.y << 16), a0);
-            a1 = fmaf(__uint_as_float(w.y & 0xffff0000u), __uint_as_float(h.y & 0xffff0000u), a1);
-            a0 = fmaf(__uint_as_float(w.z << 16), __uint_as_float(h.z << 16), a0);
-            a1 = fmaf(__uint_as_float(w.z & 0xffff0000u), __uint_as_float(h.z & 0xffff0000u), a1);
-            a0 = fmaf(__uint_as_float(w.w << 16), __uint_as_float(h.w << 16), a0);
-            a1 = fmaf(__uint_as_float(w.w & 0xffff0000u), __uint_as_float(h.w & 0xffff0000u), a1);
-        };
-        const int NG = geo.groups2, WPG = kConsumerWarps / NG;
-        const int grp = warp / WPG, wl = warp % WPG;
+        const uint32_t a_off = ((lane & 7) + ((lane >> 3) & 1) * 8) * PITCH2 + (lane >> 4) * 16;
+        const uint32_t b_off = (ROWS2 + g) * PITCH2 + tig * 4;
+        int tile_no = 0;
         for (int v = 0; v < nv; ++v) {
-            const VrRec *vrec = vrs + v;
-            const int n_tok = vrec->n_tok;
-            for (int blk = 0; blk < mt; ++blk) {
-                if ((int)(down_bar(dc) & (uint32_t)(NG - 1)) != grp) {
-                    for (int kc = 0; kc < nk2; ++kc)
-                        down_next(dc);
-                    continue;
-                }
-                const int n_rows = min(16, r_hi - r_lo - 16 * blk);
-                // RPW rows per warp; the token loops are unrolled for the smallest of 1, 2, 4, 8 that
-                // covers the request's tokens (predicated-off iterations would still cost issue slots)
-                auto run_tile = [&](auto rpw_tag, auto nt_tag) {
-                    constexpr int RPW = decltype(rpw_tag)::value;
-                    constexpr int NT = decltype(nt_tag)::value;
-                    // two chains per (row, token) where there are few of those, one where there are many
-                    constexpr int NC = RPW * NT >= 8 ? 1 : 2;
-                    float acc[RPW][NT][NC];
-#pragma unroll
-                    for (int j = 0; j < RPW; ++j)
-#pragma unroll
-                        for (int tk = 0; tk < NT; ++tk)
-#pragma unroll
-                            for (int q = 0; q < NC; ++q)
-                                acc[j][tk][q] = 0.f;
-                    for (int kc = 0; kc < nk2; ++kc) {
-                        mbar_wait(full2 + 8 * down_bar(dc), dc.use & 1u, abort_flag);
-                        if (trace && first && tid == 0)
-                            trace[2] = globaltimer_ns();
-                        first = false;
-                        const unsigned char *base = ring + down_off(dc);
-                        const int nch = min(CB2, rb2 - kc * CB2) >> 4;
-                        const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
-#pragma unroll
-                        for (int pr = 0; pr < RPW / 2; ++pr) {
-                            const int ra = wl + WPG * (2 * pr), rb = ra + WPG;
-                            if (ra >= n_rows)
-                                break;
-                            const bool has_b = rb < n_rows;
-                            const uint4 *wra = reinterpret_cast<const uint4 *>(base + (size_t)ra * PITCH2);
-                            const uint4 *wrb = reinterpret_cast<const uint4 *>(base + (size_t)rb * PITCH2);
-                            for (int c0 = lane; c0 < nch; c0 += 128) {
-                                uint4 wa[4], wb[4];
-#pragma unroll
-                                for (int i = 0; i < 4; ++i) {
-                                    const int c = c0 + 32 * i;
-                                    wa[i] = c < nch ? wra[c] : zero;
-                                    wb[i] = (c < nch && has_b) ? wrb[c] : zero;
-                                }
-#pragma unroll
-                                for (int tk = 0; tk < NT; ++tk) {
-                                    if (NT == 1 || tk < n_tok) {
-                                        const uint4 *hr = reinterpret_cast<const uint4 *>(base + (size_t)(16 + tk) * PITCH2);
-                                        uint4 hv[4];
-#pragma unroll
-                                        for (int i = 0; i < 4; ++i) {
-                                            const int c = c0 + 32 * i;
-                                            hv[i] = c < nch ? hr[c] : zero;
-                                        }
-#pragma unroll
-                                        for (int i = 0; i < 4; ++i) {
-                                            dot8(wa[i], hv[i], acc[2 * pr][tk][0], acc[2 * pr][tk][NC - 1]);
-                                            dot8(wb[i], hv[i], acc[2 * pr + 1][tk][0], acc[2 * pr + 1][tk][NC - 1]);
-                                        }
-                                    }
-                                }
-                            }
+            const VrInfo vi = load_vr(vb + v);
+            for (int blk = 0; blk < mt; ++blk, ++tile_no) {
+                const bool mine = (tile_no & (kConsumerWarps - 1)) == warp;
+                for (int kc = 0; kc < nk2; ++kc) {
+                    mbar_wait(full2 + 8 * down_bar(dc), dc.use & 1u, abort_flag);
+                    if (trace && first && tid == 0)
+                        trace[2] = globaltimer_ns();
+                    first = false;
+                    if (mine) {
+                        const uint32_t base = ring_s + down_off(dc);
+                        const int bytes = min(CB2, rb2 - kc * CB2);
+                        const bool has_tok = g < vi.n_tok;
+                        mma_steps(base, a_off, b_off, 0, bytes >> 5, has_tok);
+                        if (bytes & 16) {
+                            // the row ends on half a step: columns 8..15 of both operands count as zero
+                            const int ks = bytes >> 5;
+                            uint32_t a0, a1, a2, a3;
+                            ldmatrix_x4(base + a_off + ks * 32, a0, a1, a2, a3);
+                            const uint32_t b0 = has_tok ? lds32(base + b_off + ks * 32) : 0u;
+                            mma_16816(c1, a0, a1, 0u, 0u, b0, 0u);
                         }
                         __syncwarp();
                         if (lane == 0)
                             mbar_arrive(empty2 + 8 * down_bar(dc));
-                        down_next(dc);
                     }
-                    if (wl < n_rows) {
-                        float vals[RPW * NT];
+                    down_next(dc);
+                }
+                if (mine) {
+                    // rows g and g + 8 of the tile, tokens 2 tig and 2 tig + 1 of the request
+                    const int n_rows = min(16, r_hi - r_lo - 16 * blk);
+                    float *z0 = p.zbuf + r_lo + 16 * blk + g;
 #pragma unroll
-                        for (int j = 0; j < RPW; ++j)
-#pragma unroll
-                            for (int tk = 0; tk < NT; ++tk)
-                                vals[j * NT + tk] = NC == 2 ? acc[j][tk][0] + acc[j][tk][NC - 1] : acc[j][tk][0];
-#pragma unroll
-                        for (int m = 16; m >= 1; m >>= 1)
-#pragma unroll
-                            for (int q = 0; q < RPW * NT; ++q)
-                                vals[q] += __shfl_xor_sync(0xffffffffu, vals[q], m);
-                        // every lane holds every sum: lane q stores sum q
-                        float mine = 0.f;
-#pragma unroll
-                        for (int q = 0; q < RPW * NT; ++q)
-                            mine = lane == q ? vals[q] : mine;
-                        if (lane < RPW * NT) {
-                            const int j = lane / NT, tk = lane % NT;
-                            const int rr = wl + WPG * j;
-                            if (tk < n_tok && rr < n_rows)
-                                p.zbuf[(size_t)vrec->pair[tk] * d + r_lo + 16 * blk + rr] = mine;
-                        }
+                    for (int i = 0; i < 4; ++i) {
+                        const float val = (c0[i] + c1[i]) + (c2[i] + c3[i]);
+                        c0[i] = c1[i] = c2[i] = c3[i] = 0.f;
+                        const int tok = tig * 2 + (i & 1), row = g + (i >> 1) * 8;
+                        if (tok < vi.n_tok && row < n_rows)
+                            z0[(size_t)((i & 1) ? vi.pair1 : vi.pair0) * d + (i >> 1) * 8] = val;
                     }
-                };
-                auto by_tokens = [&](auto rpw_tag) {
-                    constexpr int RPW = decltype(rpw_tag)::value;
-                    if (n_tok <= 1)
-                        run_tile(rpw_tag, std::integral_constant<int, 1>{});
-                    else if constexpr (RPW <= 8) {
-                        if (n_tok <= 2)
-                            run_tile(rpw_tag, std::integral_constant<int, 2>{});
-                        else if constexpr (RPW <= 4) {
-                            if (n_tok <= 4)
-                                run_tile(rpw_tag, std::integral_constant<int, 4>{});
-                            else if constexpr (RPW <= 2)
-                                run_tile(rpw_tag, std::integral_constant<int, 8>{});
-                        }
-                    }
-                };
-                if (NG == 2)
-                    by_tokens(std::integral_constant<int, 4>{});
-                else
-                    by_tokens(std::integral_constant<int, 2>{});
+                }
             }
         }
     }
@@ -886,21 +811,20 @@ cudaError_t ffn_stream_geometry(const FfnLaunchCfg &cfg, int d, int F, int T, Ff
         n = kMaxStages;
     geo->n_stages = (int)n;
     geo->stage_bytes = (int)stage;
-    // down phase: rows unpadded (whole row if it fits a piece), as many sub-stages per slot as fit
-    const size_t pitch2u = (size_t)2 * F <= (size_t)geo->chunk_bytes2 ? (size_t)2 * F : (size_t)geo->chunk_bytes2;
-    const size_t sub = (rows * pitch2u + 127) / 128 * 128;
+    // down phase: a CTA has at most ceil(d / grid) output rows, so a tile may have fewer than 16
+    // weight rows; the h rows follow them, and the sub-stage is at least 16 rows long because the
+    // tensor-core loads always read 16 (what lies in rows the tile does not have only reaches
+    // accumulator rows that are never stored).  As many sub-stages per slot as fit.
+    const int rows_cta = (d + cfg.grid - 1) / cfg.grid;
+    geo->rows2 = rows_cta < 16 ? rows_cta : 16;
+    const size_t sub_rows = (size_t)(geo->rows2 + geo->n_op_rows) > 16 ? (size_t)(geo->rows2 + geo->n_op_rows) : 16;
+    const size_t sub = (sub_rows * geo->pitch2 + 127) / 128 * 128;
     size_t ns2 = stage / sub;
     if (ns2 < 1)
         ns2 = 1;
     while (ns2 * n > (size_t)kMaxSub)
         --ns2;
     geo->sub2 = (int)ns2;
-    // down phase: warp groups working on different tiles side by side.  Only where a tile is a single
-    // stage and the request's tokens are few (the accumulators are rows per warp x tokens).
-    {
-        const int nt = geo->n_op_rows <= 1 ? 1 : geo->n_op_rows <= 2 ? 2 : geo->n_op_rows <= 4 ? 4 : 8;
-        geo->groups2 = ((size_t)2 * F <= (size_t)geo->chunk_bytes2 && nt <= 4) ? 2 : 1;
-    }
     geo->sub_bytes2 = (int)sub;
     geo->ring_bytes = (n * stage + 127) / 128 * 128;
     geo->smem_bytes = geo->ring_bytes + fixed;

@@ -69,7 +69,7 @@ struct FfnGeometry {
     int pitch, chunk_bytes;          // gate/up phase: row pitch in a stage, bytes per row piece (rows of 2*d bytes)
     int pitch2, chunk_bytes2;        // down phase (rows of 2*d_ff bytes)
     int sub2, sub_bytes2;            // down phase: sub-stages per ring slot and their size
-    int groups2;                     // down phase: groups of consumer warps working on different tiles (1 or 2)
+    int rows2;                       // down phase: weight rows of a sub-stage, min(16, ceil(d / grid)); the h rows follow
     size_t ring_bytes, smem_bytes;
 };
 cudaError_t ffn_stream_configure(int n_sms, size_t max_smem, FfnLaunchCfg *cfg);
