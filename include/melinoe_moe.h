@@ -94,7 +94,9 @@ int melinoe_moe_pack_expert(int d_model, int d_ff, const void *w_gate_host, cons
                             const void *w_down_host, void *blob_out_host);
 
 /* Router matrix W_r (Eq. 1): dev pointer, [n_experts][d_model] bf16, 16-byte aligned, borrowed
- * until the handle is destroyed or the router is replaced. */
+ * until the handle is destroyed or the router is replaced.  Its contents must not change while a
+ * forward call is queued or running (a decode call may read it before the work ahead of it in the
+ * stream has finished). */
 int melinoe_moe_set_router(melinoe_moe_t *h, const void *w_router_dev);
 
 /*

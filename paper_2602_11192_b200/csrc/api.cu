@@ -33,6 +33,12 @@ static std::atomic<int> g_last_cuda_error{0};
 
 void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
 
+bool pdl_enabled()
+{
+    static const bool on = std::getenv("MELINOE_MOE_NO_PDL") == nullptr;
+    return on;
+}
+
 }  // namespace melinoe
 
 namespace {
@@ -572,7 +578,7 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
     pp.vr_capacity = h->vr_capacity;
     if (route_plan_small_supported(T, h->k, h->d)) {
         CU_TRY(launch_route_plan_small(s, static_cast<const uint16_t *>(hidden_dev), h->w_router, h->bias, h->token_seq,
-                                       h->d, h->idx, h->gate, h->logits, h->sync + 2 * (kMaxGroups + 1), pp));
+                                       h->d, h->idx, h->gate, h->logits, pp));
     } else {
         CU_TRY(launch_router(s, static_cast<const uint16_t *>(hidden_dev), h->w_router, h->bias, h->token_seq, T, h->d,
                              h->E, h->k, h->idx, h->gate, h->logits));

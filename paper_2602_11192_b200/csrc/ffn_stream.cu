@@ -196,20 +196,6 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
     if (trace && tid == 0)
         trace[0] = globaltimer_ns();
 
-    const int status = plan->status, n_groups = plan->n_groups;
-    const int vb = plan->group_vr_begin[p.group];
-    const int nv = plan->group_vr_begin[p.group + 1] - vb;
-    if (status != MELINOE_OK) {
-        // the call was refused on the device: the output is all zeros, the status tells why
-        if (p.group == 0)
-            for (size_t i = (size_t)blockIdx.x * kThreads + tid; i < (size_t)p.T * d; i += (size_t)G * kThreads)
-                p.out[i] = 0;
-        return;
-    }
-    const bool final_group = p.group == n_groups - 1;
-    if (nv <= 0 && !final_group)
-        return;
-
     // ring | reduction buffers | barriers (phase 1 full/empty, phase 2 full/empty)
     unsigned char *ring = smem;
     float *red = reinterpret_cast<float *>(smem + geo.ring_bytes);              // [2][8 warps][4][32]
@@ -235,6 +221,26 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    // Everything above touches nothing an earlier kernel wrote.  The launch may have been made with
+    // programmatic stream serialisation, in which case this CTA can be running before the kernel
+    // ahead of it in the stream (the planner) has finished: wait for it here (returns at once in an
+    // ordinary launch), then let the kernel behind this one be scheduled early in the same way.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const int status = plan->status, n_groups = plan->n_groups;
+    const int vb = plan->group_vr_begin[p.group];
+    const int nv = plan->group_vr_begin[p.group + 1] - vb;
+    if (status != MELINOE_OK) {
+        // the call was refused on the device: the output is all zeros, the status tells why
+        if (p.group == 0)
+            for (size_t i = (size_t)blockIdx.x * kThreads + tid; i < (size_t)p.T * d; i += (size_t)G * kThreads)
+                p.out[i] = 0;
+        return;
+    }
+    const bool final_group = p.group == n_groups - 1;
+    if (nv <= 0 && !final_group)
+        return;
+
     // the launch's virtual-request records: from shared memory when they fit (always in decode),
     // so that nobody's critical path holds a dependent global load per tile
     const VrRec *vrs = p.vrs + vb;
@@ -783,6 +789,7 @@ cudaError_t ffn_stream_configure(int n_sms, size_t max_smem, FfnLaunchCfg *cfg)
         return cudaErrorInvalidConfiguration;
     cfg->grid = n_sms;          // one CTA per SM: all of them resident, which the grid barrier needs
     cfg->max_smem = usable;
+    cfg->pdl = pdl_enabled();
     return cudaSuccess;
 }
 
@@ -833,11 +840,22 @@ cudaError_t ffn_stream_geometry(const FfnLaunchCfg &cfg, int d, int F, int T, Ff
 
 cudaError_t launch_ffn_stream(cudaStream_t stream, const FfnLaunchCfg &cfg, const FfnGeometry &geo, const FfnParams &p)
 {
-    FfnParams q = p;
-    FfnGeometry gq = geo;
-    void *args[] = {&q, &gq};
-    cudaError_t e = cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(ffn_stream_kernel), dim3(cfg.grid),
-                                                dim3(kThreads), args, geo.smem_bytes, stream);
+    // cooperative (the grid barrier needs every CTA resident) and with programmatic stream
+    // serialisation (the CTAs may be scheduled, and set up their barriers, while the kernel ahead in
+    // the stream is still draining; the kernel waits for it before it reads the plan)
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3(cfg.grid);
+    lc.blockDim = dim3(kThreads);
+    lc.dynamicSmemBytes = geo.smem_bytes;
+    lc.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = cfg.pdl ? 2 : 1;
+    const cudaError_t e = cudaLaunchKernelEx(&lc, ffn_stream_kernel, p, geo);
     count_launch();
     return e;
 }

@@ -10,6 +10,8 @@
 namespace melinoe {
 
 void count_launch();
+// Programmatic stream serialisation for the decode kernels (on unless MELINOE_MOE_NO_PDL is set in the environment).
+bool pdl_enabled();
 
 // ---- router (Eq. 1): logits, top-k, gates
 cudaError_t launch_router(cudaStream_t stream, const uint16_t *x, const uint16_t *w_r,
@@ -37,11 +39,11 @@ struct PlanParams {
 };
 cudaError_t launch_plan(cudaStream_t stream, const PlanParams &p);
 
-// ---- router and planning in one single-block kernel, for calls of at most 8 tokens
+// ---- router and planning in one kernel (one thread-block cluster), for calls of at most 8 tokens
 bool route_plan_small_supported(int T, int k, int d);
 cudaError_t launch_route_plan_small(cudaStream_t stream, const uint16_t *x, const uint16_t *w_r, const float *bias,
                                     const int32_t *token_seq, int d, int32_t *idx, float *gate, float *logits_out,
-                                    unsigned *ticket, const PlanParams &p);
+                                    const PlanParams &p);
 
 // ---- streaming expert FFN (Eq. 3) with the gate-weighted combine (Eq. 2) fused in
 struct FfnParams {
@@ -61,6 +63,7 @@ struct FfnParams {
 struct FfnLaunchCfg {
     int grid;                        // one CTA per SM
     size_t max_smem;                 // dynamic shared memory the kernel may use
+    bool pdl;                        // launch with programmatic stream serialisation
 };
 // Shape of the shared-memory ring for one call.
 struct FfnGeometry {

@@ -4,9 +4,13 @@
 //
 // At this size every step is latency, not throughput, so the kernel is organised to take as
 // few dependent memory round trips as possible:
-//   - logits: one warp per expert, spread over E/4 blocks (a single SM pulling the whole router
-//     matrix takes ~9 us; sixteen SMs take ~2); each lane has all its loads in flight at once;
-//   - the block that finishes last (a ticket counter) does the rest, so there is no second launch;
+//   - logits: one warp per expert, spread over a thread-block cluster of 8 CTAs x 8 warps (a single
+//     SM pulling the whole router matrix takes ~9 us; eight take ~2); each lane has all its loads in
+//     flight at once, the router row already before the kernel ahead in the stream has finished;
+//   - the logits go straight into the shared memory of the cluster's first CTA and the cluster
+//     barrier tells it when they are all there: no fence, no device counter, no second launch;
+//   - top-k is a rank count (an element's rank is the number of elements that beat it), one warp
+//     per token, instead of k rounds of a warp-wide maximum;
 //   - planning is written for one warp with lane = expert / slot / request: ranks come from
 //     ballots and population counts, prefix sums from shuffles, and the LRU victims of a call are
 //     taken from one sorted list instead of one search per miss.
@@ -30,8 +34,9 @@ namespace melinoe {
 
 namespace {
 
-constexpr int kWarpsPerBlock = 4;
+constexpr int kWarpsPerBlock = 8;
 constexpr int kThreads = kWarpsPerBlock * 32;
+constexpr int kCluster = kMaxExperts / kWarpsPerBlock;   // 8 CTAs: a warp for each of up to 64 experts
 constexpr int kMaxT = kTokPerVr;                 // 8 tokens
 constexpr int kMaxPairs = kMaxExperts;           // T * k <= 64 is required by the launcher
 
@@ -75,11 +80,11 @@ __device__ __forceinline__ void write_vr(VrRec *dst, const char *blob, int n_tok
     *dst = vr;
 }
 
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 1)
 route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restrict__ w_r,
                         const float *__restrict__ bias, const int32_t *__restrict__ token_seq, int d,
                         int32_t *__restrict__ idx_out, float *__restrict__ gate_out, float *logits_out,
-                        unsigned *ticket, PlanParams p)
+                        PlanParams p)
 {
     __shared__ float s_logit[kMaxT][kMaxExperts];
     __shared__ int32_t s_idx[kMaxPairs];
@@ -88,123 +93,149 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
     __shared__ int32_t s_victim[kMaxExperts];                    // V: slots in victim order
     __shared__ int32_t s_miss_expert[kMaxExperts];               // expert of miss number i
     __shared__ int32_t s_entry_occ[kMaxExperts];                 // occupant of a slot at call entry
-    __shared__ int s_last;
+    __shared__ float s_sel[kMaxT][kMaxExperts];                  // a token's selected logits, by rank
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int T = p.T, k = p.k, E = p.E, C = p.C;
     const int n_pairs = T * k;
+    unsigned cta_rank;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(cta_rank));
 
     // ================================================================ logits: one warp per expert
-    {
-        const int e = blockIdx.x * kWarpsPerBlock + warp;
-        if (e < E) {
-            const int n_chunks = d >> 8;
-            const uint4 *wrow = reinterpret_cast<const uint4 *>(w_r + (size_t)e * d) + lane;
-            for (int t = 0; t < T; ++t) {
-                const uint4 *xrow = reinterpret_cast<const uint4 *>(x + (size_t)t * d) + lane;
-                float a = 0.0f;
-                for (int c0 = 0; c0 < n_chunks; c0 += 8) {
-                    // all of a lane's loads for these 8 pieces go out before any arithmetic
-                    uint4 wv[8], xv[8];
+    const int e_mine = (int)cta_rank * kWarpsPerBlock + warp;
+    const int n_chunks = d >> 8;
+    // The router matrix does not change while calls are queued, so the first eight pieces of the
+    // row go out before anything else.
+    uint4 wv0[8];
+    if (e_mine < E) {
+        const uint4 *wrow = reinterpret_cast<const uint4 *>(w_r + (size_t)e_mine * d) + lane;
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const bool on = c0 + i < n_chunks;
-                        wv[i] = on ? __ldg(wrow + (c0 + i) * 32) : make_uint4(0, 0, 0, 0);
-                        xv[i] = on ? __ldg(xrow + (c0 + i) * 32) : make_uint4(0, 0, 0, 0);
-                    }
+        for (int i = 0; i < 8; ++i)
+            wv0[i] = i < n_chunks ? __ldg(wrow + i * 32) : make_uint4(0, 0, 0, 0);
+    }
+    // The launch may have been made with programmatic stream serialisation: this block can then be
+    // running before the kernel ahead of it in the stream has finished.  Nothing before this point
+    // reads what that kernel may have written; wait for it here (returns at once in an ordinary
+    // launch).
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    // lane t holds token t's bias (two dependent loads, in flight under the dot products)
+    float my_bias = 0.0f;
+    if (e_mine < E && bias && lane < T) {
+        const int q = token_seq ? token_seq[lane] : 0;
+        my_bias = bias[(size_t)q * E + e_mine];
+    }
+
+    // the planner's view of the cache: its loads overlap the logits
+    DevCache *cache = p.cache;
+    int soe0 = -1, soe1 = -1, eos0 = -1, eos1 = -1;
+    unsigned long long st0 = 0ull, st1 = 0ull, counter = 0ull, call_no = 0ull;
+    if (cta_rank == 0 && warp == 0) {
+        if (lane < E)
+            soe0 = cache->slot_of_expert[lane];
+        if (lane + 32 < E)
+            soe1 = cache->slot_of_expert[lane + 32];
+        if (lane < C) {
+            eos0 = cache->expert_of_slot[lane];
+            st0 = cache->stamp[lane];
+        }
+        if (lane + 32 < C) {
+            eos1 = cache->expert_of_slot[lane + 32];
+            st1 = cache->stamp[lane + 32];
+        }
+        counter = cache->counter;
+        call_no = cache->call_no + 1ull;
+    }
+    if (e_mine < E) {
+        const uint4 *wrow = reinterpret_cast<const uint4 *>(w_r + (size_t)e_mine * d) + lane;
+        float my_logit = 0.0f;
+        for (int t = 0; t < T; ++t) {
+            const uint4 *xrow = reinterpret_cast<const uint4 *>(x + (size_t)t * d) + lane;
+            float a = 0.0f;
+            for (int c0 = 0; c0 < n_chunks; c0 += 8) {
+                // all of a lane's loads for these 8 pieces go out before any arithmetic
+                uint4 wv[8], xv[8];
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        if (c0 + i < n_chunks) {
-                            a = __fmaf_rn(bf16lo(xv[i].x), bf16lo(wv[i].x), a);
-                            a = __fmaf_rn(bf16hi(xv[i].x), bf16hi(wv[i].x), a);
-                            a = __fmaf_rn(bf16lo(xv[i].y), bf16lo(wv[i].y), a);
-                            a = __fmaf_rn(bf16hi(xv[i].y), bf16hi(wv[i].y), a);
-                            a = __fmaf_rn(bf16lo(xv[i].z), bf16lo(wv[i].z), a);
-                            a = __fmaf_rn(bf16hi(xv[i].z), bf16hi(wv[i].z), a);
-                            a = __fmaf_rn(bf16lo(xv[i].w), bf16lo(wv[i].w), a);
-                            a = __fmaf_rn(bf16hi(xv[i].w), bf16hi(wv[i].w), a);
-                        }
-                    }
+                for (int i = 0; i < 8; ++i) {
+                    const bool on = c0 + i < n_chunks;
+                    xv[i] = on ? __ldcg(xrow + (c0 + i) * 32) : make_uint4(0, 0, 0, 0);
+                }
+                if (c0 == 0) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        wv[i] = wv0[i];
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        wv[i] = c0 + i < n_chunks ? __ldg(wrow + (c0 + i) * 32) : make_uint4(0, 0, 0, 0);
                 }
 #pragma unroll
-                for (int m = 16; m >= 1; m >>= 1)
-                    a = __fadd_rn(a, __shfl_xor_sync(0xffffffffu, a, m));
-                if (lane == 0) {
-                    if (bias) {
-                        const int q = token_seq ? token_seq[t] : 0;
-                        a = __fadd_rn(a, bias[(size_t)q * E + e]);
+                for (int i = 0; i < 8; ++i) {
+                    if (c0 + i < n_chunks) {
+                        a = __fmaf_rn(bf16lo(xv[i].x), bf16lo(wv[i].x), a);
+                        a = __fmaf_rn(bf16hi(xv[i].x), bf16hi(wv[i].x), a);
+                        a = __fmaf_rn(bf16lo(xv[i].y), bf16lo(wv[i].y), a);
+                        a = __fmaf_rn(bf16hi(xv[i].y), bf16hi(wv[i].y), a);
+                        a = __fmaf_rn(bf16lo(xv[i].z), bf16lo(wv[i].z), a);
+                        a = __fmaf_rn(bf16hi(xv[i].z), bf16hi(wv[i].z), a);
+                        a = __fmaf_rn(bf16lo(xv[i].w), bf16lo(wv[i].w), a);
+                        a = __fmaf_rn(bf16hi(xv[i].w), bf16hi(wv[i].w), a);
                     }
-                    logits_out[(size_t)t * E + e] = a;
                 }
             }
+#pragma unroll
+            for (int m = 16; m >= 1; m >>= 1)
+                a = __fadd_rn(a, __shfl_xor_sync(0xffffffffu, a, m));
+            if (lane == t)
+                my_logit = bias ? __fadd_rn(a, my_bias) : a;
+        }
+        if (lane < T) {
+            // into the first CTA's shared memory, and to global memory for the inspection calls
+            uint32_t remote;
+            asm volatile("mapa.shared::cluster.u32 %0, %1, %2;"
+                         : "=r"(remote)
+                         : "r"((uint32_t)__cvta_generic_to_shared(&s_logit[lane][e_mine])), "r"(0));
+            asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(my_logit) : "memory");
+            logits_out[(size_t)lane * E + e_mine] = my_logit;
         }
     }
-    // ---- the block that finishes last carries on
-    __threadfence();
-    __syncthreads();
-    if (tid == 0)
-        s_last = atomicAdd(ticket, 1u) == gridDim.x - 1;
-    __syncthreads();
-    if (!s_last)
+    // ---- the cluster's first CTA carries on when every logit has arrived
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    if (cta_rank != 0)
         return;
-    __threadfence();
-    if (tid == 0)
-        *ticket = 0u;
-    for (int i = tid; i < T * E; i += kThreads)
-        s_logit[i / E][i % E] = __ldcg(logits_out + i);
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
     for (int i = tid; i < 2 * (kMaxGroups + 1); i += kThreads)
         p.sync[i] = 0u;
-    __syncthreads();
 
     // ================================================================ top-k and gates: a warp per token
+    // An element's rank is the number of elements that beat it (greater, or equal with a lower index).
     for (int t = warp; t < T; t += kWarpsPerBlock) {
         const float NEG = -__int_as_float(0x7f800000);  // -inf
         const float v0 = lane < E ? s_logit[t][lane] : NEG;
         const float v1 = lane + 32 < E ? s_logit[t][lane + 32] : NEG;
-        bool taken0 = !(lane < E), taken1 = !(lane + 32 < E);
-        float my_sel = 0.0f, top = 0.0f;
-        int my_idx = 0;
-        for (int j = 0; j < k; ++j) {
-            float bv;
-            int bi;
-            if (!taken0 && (taken1 || v0 >= v1)) {
-                bv = v0;
-                bi = lane;
-            } else if (!taken1) {
-                bv = v1;
-                bi = lane + 32;
-            } else {
-                bv = NEG;
-                bi = 1 << 20;
-            }
-#pragma unroll
-            for (int m = 16; m >= 1; m >>= 1) {
-                const float ov = __shfl_xor_sync(0xffffffffu, bv, m);
-                const int oi = __shfl_xor_sync(0xffffffffu, bi, m);
-                if (ov > bv || (ov == bv && oi < bi)) {
-                    bv = ov;
-                    bi = oi;
-                }
-            }
-            if (bi == lane)
-                taken0 = true;
-            if (bi == lane + 32)
-                taken1 = true;
-            if (j == 0)
-                top = bv;
-            if (lane == j) {
-                my_sel = bv;
-                my_idx = bi;
-            }
+        int r0 = 0, r1 = 0;
+        for (int e = 0; e < E; ++e) {
+            const float o = s_logit[t][e];
+            r0 += (o > v0) || (o == v0 && e < lane);
+            r1 += (o > v1) || (o == v1 && e < lane + 32);
         }
-        const float ev = lane < k ? expf(my_sel - top) : 0.0f;
+        if (lane < E && r0 < k) {
+            s_sel[t][r0] = v0;
+            s_idx[t * k + r0] = lane;
+        }
+        if (lane + 32 < E && r1 < k) {
+            s_sel[t][r1] = v1;
+            s_idx[t * k + r1] = lane + 32;
+        }
+        __syncwarp();
+        const float top = s_sel[t][0];
+        const float ev = lane < k ? expf(s_sel[t][lane] - top) : 0.0f;
         float sum = ev;
 #pragma unroll
         for (int m = 16; m >= 1; m >>= 1)
             sum += __shfl_xor_sync(0xffffffffu, sum, m);
         if (lane < k) {
-            s_idx[t * k + lane] = my_idx;
-            idx_out[(size_t)t * k + lane] = my_idx;
+            idx_out[(size_t)t * k + lane] = s_idx[t * k + lane];
             gate_out[(size_t)t * k + lane] = ev / sum;
         }
     }
@@ -214,15 +245,9 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
 
     // ================================================================ planning, by one warp
     // lane owns experts lane and lane + 32, slots lane and lane + 32, pairs lane and lane + 32
-    DevCache *cache = p.cache;
+    // (the cache state of this lane's experts and slots was loaded before the logits)
     DevPlan *plan = p.plan;
     const int e0 = lane, e1 = lane + 32;
-    // cache state of my experts and slots (one round trip, all loads in flight together)
-    const int soe0 = e0 < E ? cache->slot_of_expert[e0] : -1, soe1 = e1 < E ? cache->slot_of_expert[e1] : -1;
-    const int eos0 = lane < C ? cache->expert_of_slot[lane] : -1, eos1 = lane + 32 < C ? cache->expert_of_slot[lane + 32] : -1;
-    const unsigned long long st0 = lane < C ? cache->stamp[lane] : 0ull, st1 = lane + 32 < C ? cache->stamp[lane + 32] : 0ull;
-    const unsigned long long counter = cache->counter;
-    const unsigned long long call_no = cache->call_no + 1ull;
 
     // ---- token lists: counts, offsets, stable positions (pairs in increasing flat index)
     int c0 = 0, c1 = 0;
@@ -414,12 +439,28 @@ bool route_plan_small_supported(int T, int k, int d)
 
 cudaError_t launch_route_plan_small(cudaStream_t stream, const uint16_t *x, const uint16_t *w_r, const float *bias,
                                     const int32_t *token_seq, int d, int32_t *idx, float *gate, float *logits_out,
-                                    unsigned *ticket, const PlanParams &p)
+                                    const PlanParams &p)
 {
-    const int grid = (p.E + kWarpsPerBlock - 1) / kWarpsPerBlock;
-    route_plan_small_kernel<<<grid, kThreads, 0, stream>>>(x, w_r, bias, token_seq, d, idx, gate, logits_out, ticket, p);
+    // one cluster of 8 CTAs; programmatic stream serialisation: the blocks may be scheduled while the
+    // kernel ahead in the stream is still draining; the kernel itself waits for that kernel before it
+    // reads anything that kernel may have written
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(kCluster);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = kCluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl_enabled() ? 2 : 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, route_plan_small_kernel, x, w_r, bias, token_seq, d, idx, gate, logits_out, p);
     count_launch();
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace melinoe
