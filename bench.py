@@ -352,7 +352,8 @@ def run_ours(args):
         stack.close()
         full = Stack(cfg, alpha0, cfg.n_experts, n_layers=L)
         stack = full
-        ms_r, _, st_r, ffn_ms_r, ffn_n_r = timed_device(alpha0, with_kernel_timing=True)
+        ms_r, _, _, _, _ = timed_device(alpha0)                    # throughput: no per-launch events
+        _, _, st_r, ffn_ms_r, ffn_n_r = timed_device(alpha0, with_kernel_timing=True)
         by_r = float(st_r["n_distinct"].astype(np.int64).sum()) * B_e
         extra["all_resident"] = {"value": cfg.batch * K / (ms_r * 1e-3), "ffn_gbs": by_r / (ffn_ms_r * 1e-3) / 1e9,
                                  "ffn_frac_of_hbm": by_r / (ffn_ms_r * 1e-3) / 1e9 / hbm_peak,
