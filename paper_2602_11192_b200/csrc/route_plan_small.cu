@@ -64,8 +64,8 @@ __device__ __forceinline__ uint64_t ballot64(bool lo, bool hi)
 __device__ __forceinline__ int rank_below(uint64_t mask, int bit) { return __popcll(mask & ((1ull << bit) - 1ull)); }
 
 // The virtual request of one expert (at most 8 tokens here): its tokens and z rows from the sorted lists.
-__device__ __forceinline__ void write_vr(VrRec *dst, const char *blob, int n_tok, int group, int off, int k,
-                                         const int32_t *pair_at)
+__device__ __forceinline__ void write_vr(VrRec *dst, const char *blob, int n_tok, int group, int off,
+                                         const int32_t *pair_at, const int32_t *tok_of_pair)
 {
     VrRec vr;
     vr.blob = blob;
@@ -74,7 +74,7 @@ __device__ __forceinline__ void write_vr(VrRec *dst, const char *blob, int n_tok
 #pragma unroll
     for (int j = 0; j < kTokPerVr; ++j) {
         const int pr = j < n_tok ? pair_at[off + j] : -1;
-        vr.tok[j] = pr >= 0 ? pr / k : -1;
+        vr.tok[j] = pr >= 0 ? tok_of_pair[pr] : -1;
         vr.pair[j] = pr;
     }
     *dst = vr;
@@ -86,7 +86,9 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
                         int32_t *__restrict__ idx_out, float *__restrict__ gate_out, float *logits_out,
                         PlanParams p)
 {
-    __shared__ float s_logit[kMaxT][kMaxExperts];
+    __shared__ __align__(16) float s_logit[kMaxT][kMaxExperts];
+    __shared__ int32_t s_cnt[2][kMaxExperts];                    // pairs of an expert among pairs 0..31 / 32..63
+    __shared__ int32_t s_tok[kMaxPairs];                         // token of a pair
     __shared__ int32_t s_idx[kMaxPairs];
     __shared__ int32_t s_pair_at[kMaxPairs];                     // pair at sorted position
     __shared__ unsigned long long s_key[kMaxExperts];            // victim-order key of a slot
@@ -214,10 +216,18 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
         const float v0 = lane < E ? s_logit[t][lane] : NEG;
         const float v1 = lane + 32 < E ? s_logit[t][lane + 32] : NEG;
         int r0 = 0, r1 = 0;
-        for (int e = 0; e < E; ++e) {
-            const float o = s_logit[t][e];
-            r0 += (o > v0) || (o == v0 && e < lane);
-            r1 += (o > v1) || (o == v1 && e < lane + 32);
+        const float4 *row = reinterpret_cast<const float4 *>(s_logit[t]);
+#pragma unroll
+        for (int i = 0; i < kMaxExperts / 4; ++i) {
+            const float4 o4 = row[i];
+            const float ov[4] = {o4.x, o4.y, o4.z, o4.w};
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const int e = 4 * i + c;
+                const float o = e < E ? ov[c] : NEG;     // the row's tail beyond E was never written
+                r0 += (o > v0) || (o == v0 && e < lane);
+                r1 += (o > v1) || (o == v1 && e < lane + 32);
+            }
         }
         if (lane < E && r0 < k) {
             s_sel[t][r0] = v0;
@@ -250,29 +260,37 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
     const int e0 = lane, e1 = lane + 32;
 
     // ---- token lists: counts, offsets, stable positions (pairs in increasing flat index)
-    int c0 = 0, c1 = 0;
-    for (int q = 0; q < n_pairs; ++q) {
-        const int e = s_idx[q];
-        c0 += e == e0;
-        c1 += e == e1;
-    }
+    // Lane q also stands for pairs q and q + 32: the lanes whose pair names the same expert find
+    // one another with a match, so an expert's count and a pair's place among its expert's pairs
+    // are population counts.
+    const int qe[2] = {lane < n_pairs ? s_idx[lane] : -1 - lane, lane + 32 < n_pairs ? s_idx[lane + 32] : -1 - lane};
+    const unsigned lt = (1u << lane) - 1u;
+    const unsigned same[2] = {__match_any_sync(0xffffffffu, qe[0]), __match_any_sync(0xffffffffu, qe[1])};
+    s_cnt[0][lane] = s_cnt[0][lane + 32] = s_cnt[1][lane] = s_cnt[1][lane + 32] = 0;
+    s_tok[lane] = lane / k;
+    s_tok[lane + 32] = (lane + 32) / k;
+    __syncwarp();
+#pragma unroll
+    for (int h = 0; h < 2; ++h)
+        if (qe[h] >= 0 && (same[h] & lt) == 0u)
+            s_cnt[h][qe[h]] = __popc(same[h]);
+    __syncwarp();
+    const int c0 = s_cnt[0][e0] + s_cnt[1][e0], c1 = s_cnt[0][e1] + s_cnt[1][e1];
     int tot0, tot1;
     const int off0 = warp_excl_scan(c0, lane, tot0);
     const int off1 = tot0 + warp_excl_scan(c1, lane, tot1);
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
         const int q = lane + 32 * h;
-        const int e = q < n_pairs ? s_idx[q] : 0;
-        int r = 0;
-        for (int q2 = 0; q2 < q && q2 < n_pairs; ++q2)
-            r += s_idx[q2] == e;
+        const int e = qe[h] >= 0 ? qe[h] : 0;
+        const int r = __popc(same[h] & lt) + (h ? s_cnt[0][e] : 0);
         const int o0 = __shfl_sync(0xffffffffu, off0, e & 31), o1 = __shfl_sync(0xffffffffu, off1, e & 31);
         if (q < n_pairs) {
             const int pos = (e < 32 ? o0 : o1) + r;
             s_pair_at[pos] = q;
             p.perm[pos] = q;
             p.inv_pos[q] = pos;
-            p.tok_of_sorted[pos] = q / k;
+            p.tok_of_sorted[pos] = s_tok[q];
         }
     }
     for (int i = lane; i < p.n_shared * T; i += 32)
@@ -305,7 +323,7 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
             cache->stamp[soe] = st;
             plan->req[r] = ReqRec{e, soe, 1, -1, off, cnt, r, 0};
             if (ok)
-                write_vr(p.vrs + r, p.slots + (size_t)soe * p.slot_stride, cnt, 0, off, k, s_pair_at);
+                write_vr(p.vrs + r, p.slots + (size_t)soe * p.slot_stride, cnt, 0, off, s_pair_at, s_tok);
         }
         if ((miss_mask >> e) & 1ull)
             s_miss_expert[rank_below(miss_mask, e)] = e;
@@ -318,6 +336,7 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
         if (s < C) {
             const unsigned long long mine = s_key[s];
             int r = 0;
+#pragma unroll 8
             for (int s2 = 0; s2 < C; ++s2)
                 r += s_key[s2] < mine;
             s_victim[r] = s;
@@ -342,7 +361,7 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
             const int vr_at = n_hits + p.n_shared + i;
             plan->req[n_hits + i] = ReqRec{e, slot, 0, ev, off, cnt, vr_at, group};
             if (ok)
-                write_vr(p.vrs + vr_at, p.slots + (size_t)slot * p.slot_stride, cnt, group, off, k, s_pair_at);
+                write_vr(p.vrs + vr_at, p.slots + (size_t)slot * p.slot_stride, cnt, group, off, s_pair_at, s_tok);
             // cache update: the last miss that lands in a slot keeps it
             const bool stays = i + C >= n_miss;
             cache->slot_of_expert[e] = stays ? slot : -1;
