@@ -32,6 +32,10 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p)
     __shared__ ReqRec s_req[kMaxReq];
     __shared__ HostMiss s_miss[kMaxExperts];
     __shared__ int32_t s_group_vr_begin[kMaxGroups + 1];
+    __shared__ unsigned long long s_key[kMaxExperts];            // victim-order key of a slot
+    __shared__ int32_t s_victim[kMaxExperts];                    // V: slots in victim order
+    __shared__ int32_t s_miss_expert[kMaxExperts];               // expert of miss number i
+    __shared__ int32_t s_entry_occ[kMaxExperts];                 // occupant of a slot at call entry
     __shared__ int32_t s_misc[8];  // 0 n_req(routed) 1 n_hits 2 n_miss 3 n_evict 4 n_groups 5 n_vr 6 status 7 n_req_total
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -118,89 +122,101 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p)
     for (int i = tid; i <= kMaxGroups; i += kPlanThreads)
         p.sync[i] = 0u;
 
-    // ---- (b), (c): cache requests, by warp 0 (slots spread over lanes)
+    // ---- (b), (c): cache requests, by warp 0; lane owns experts lane and lane + 32 and slots lane and
+    // lane + 32.  The sequential rules (hits in ascending id, then misses in ascending id, a miss
+    // takes the lowest empty slot, else the least recently stamped one; a new wave starts when a
+    // miss would overwrite an expert of the current wave) have a closed form:
+    //   - hit number r (ascending id) stamps its slot with counter + r + 1;
+    //   - let V be the slots ordered by (empty first, by index), then by stamp after the hits were
+    //     stamped; miss number i (ascending id) takes V[i mod C], because every slot it could prefer
+    //     has either been taken by an earlier miss (and stamped newer) or comes later in V;
+    //   - the expert it displaces is V[i]'s occupant at call entry for i < C, and miss i - C otherwise;
+    //   - miss i belongs to wave 1 + i / C; it must wait for group i / C (i >= C), for group 0 if it
+    //     displaces one of the call's hits, for nothing otherwise.
     if (warp == 0) {
-        uint64_t need = 0, resident = 0;
-        {
-            const bool n0 = lane < E && s_counts[lane] > 0;
-            const bool n1 = lane + 32 < E && s_counts[lane + 32] > 0;
-            const bool r0 = lane < E && s_cache.slot_of_expert[lane] >= 0;
-            const bool r1 = lane + 32 < E && s_cache.slot_of_expert[lane + 32] >= 0;
-            need = (uint64_t)__ballot_sync(0xffffffffu, n0) | ((uint64_t)__ballot_sync(0xffffffffu, n1) << 32);
-            resident = (uint64_t)__ballot_sync(0xffffffffu, r0) | ((uint64_t)__ballot_sync(0xffffffffu, r1) << 32);
-        }
-        int n_req = 0, n_hits = 0, n_miss = 0, n_evict = 0;
+        const int e0 = lane, e1 = lane + 32;
+        const int c0 = e0 < E ? s_counts[e0] : 0, c1 = e1 < E ? s_counts[e1] : 0;
+        const int soe0 = e0 < E ? s_cache.slot_of_expert[e0] : -1, soe1 = e1 < E ? s_cache.slot_of_expert[e1] : -1;
+        const int eos0 = lane < C ? s_cache.expert_of_slot[lane] : -1, eos1 = lane + 32 < C ? s_cache.expert_of_slot[lane + 32] : -1;
+        const uint64_t st0 = lane < C ? s_cache.stamp[lane] : 0ull, st1 = lane + 32 < C ? s_cache.stamp[lane + 32] : 0ull;
         uint64_t counter = s_cache.counter;
-        for (uint64_t m = need & resident; m; m &= m - 1) {
-            const int e = __ffsll((long long)m) - 1;
-            if (lane == 0) {
-                const int s = s_cache.slot_of_expert[e];
-                s_cache.stamp[s] = ++counter;
-                s_req[n_req] = ReqRec{e, s, 1, -1, s_offsets[e], s_counts[e], 0, 0};
-                s_req_of_expert[e] = n_req;
-                s_group_of_expert[e] = 0;
-            }
-            ++n_req;
-            ++n_hits;
-        }
-        counter = __shfl_sync(0xffffffffu, counter, 0);
+        auto ballot64 = [](bool lo, bool hi) {
+            return (uint64_t)__ballot_sync(0xffffffffu, lo) | ((uint64_t)__ballot_sync(0xffffffffu, hi) << 32);
+        };
+        auto rank_below = [](uint64_t mask, int bit) { return __popcll(mask & ((1ull << bit) - 1ull)); };
+        const uint64_t need = ballot64(c0 > 0, c1 > 0);
+        const uint64_t resident = ballot64(soe0 >= 0, soe1 >= 0);
+        const uint64_t hit_mask = need & resident, miss_mask = need & ~resident;
+        const int n_hits = __popcll(hit_mask), n_miss = __popcll(miss_mask), n_req = n_hits + n_miss;
         __syncwarp();
-        int cur_group = 1;
-        for (uint64_t m = need & ~resident; m; m &= m - 1) {
-            const int e = __ffsll((long long)m) - 1;
-            // victim: lowest empty slot, else smallest stamp (stamps are unique)
-            uint64_t key = ~0ull;
-            int slot = -1;
+        s_key[lane] = lane < C ? (eos0 < 0 ? (uint64_t)lane : ((1ull << 63) | st0)) : ~0ull;
+        s_key[lane + 32] = lane + 32 < C ? (eos1 < 0 ? (uint64_t)(lane + 32) : ((1ull << 63) | st1)) : ~0ull;
+        s_entry_occ[lane] = eos0;
+        s_entry_occ[lane + 32] = eos1;
+        __syncwarp();
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const int s = lane + 32 * h;
-                if (s < C) {
-                    const uint64_t ks = s_cache.expert_of_slot[s] < 0 ? (uint64_t)s
-                                                                       : ((1ull << 63) | s_cache.stamp[s]);
-                    if (ks < key) {
-                        key = ks;
-                        slot = s;
-                    }
-                }
+        for (int h = 0; h < 2; ++h) {
+            const int e = h ? e1 : e0, soe = h ? soe1 : soe0;
+            if ((hit_mask >> e) & 1ull) {
+                const int r = rank_below(hit_mask, e);
+                const uint64_t st = counter + (uint64_t)r + 1ull;
+                s_key[soe] = (1ull << 63) | st;
+                s_cache.stamp[soe] = st;
+                s_req[r] = ReqRec{e, soe, 1, -1, s_offsets[e], s_counts[e], 0, 0};
+                s_req_of_expert[e] = r;
             }
-#pragma unroll
-            for (int mm = 16; mm >= 1; mm >>= 1) {
-                const uint64_t ok = __shfl_xor_sync(0xffffffffu, key, mm);
-                const int os = __shfl_xor_sync(0xffffffffu, slot, mm);
-                if (ok < key) {
-                    key = ok;
-                    slot = os;
-                }
-            }
-            const int ev = s_cache.expert_of_slot[slot];
-            int dep = -1;
-            if (ev >= 0) {
-                ++n_evict;
-                if ((need >> ev) & 1ull)
-                    dep = s_group_of_expert[ev];
-            }
-            if (dep == cur_group)
-                ++cur_group;
-            __syncwarp();
-            if (lane == 0) {
-                ++counter;
-                if (ev >= 0)
-                    s_cache.slot_of_expert[ev] = -1;
-                s_cache.expert_of_slot[slot] = e;
-                s_cache.slot_of_expert[e] = slot;
-                s_cache.stamp[slot] = counter;
-                s_req[n_req] = ReqRec{e, slot, 0, ev, s_offsets[e], s_counts[e], 0, cur_group};
-                s_req_of_expert[e] = n_req;
-                s_group_of_expert[e] = cur_group;
-                s_miss[n_miss] = HostMiss{e, slot, (int16_t)cur_group, (int16_t)dep, 0u};
-            }
-            counter = __shfl_sync(0xffffffffu, counter, 0);
-            ++n_req;
-            ++n_miss;
-            __syncwarp();
+            if ((miss_mask >> e) & 1ull)
+                s_miss_expert[rank_below(miss_mask, e)] = e;
         }
+        __syncwarp();
+        // V: rank of each slot among the keys (keys are distinct)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int sl = lane + 32 * h;
+            if (sl < C) {
+                const uint64_t mine = s_key[sl];
+                int r = 0;
+#pragma unroll 8
+                for (int s2 = 0; s2 < C; ++s2)
+                    r += s_key[s2] < mine;
+                s_victim[r] = sl;
+            }
+        }
+        __syncwarp();
+        bool ev_flag[2] = {false, false};
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int e = h ? e1 : e0;
+            if ((miss_mask >> e) & 1ull) {
+                const int i = rank_below(miss_mask, e);
+                const int slot = s_victim[i % C];
+                const int ev = i < C ? s_entry_occ[slot] : s_miss_expert[i - C];
+                const int group = 1 + i / C;
+                int dep = -1;
+                if (i >= C)
+                    dep = i / C;
+                else if (ev >= 0 && ((need >> ev) & 1ull))
+                    dep = 0;
+                ev_flag[h] = ev >= 0;
+                s_req[n_hits + i] = ReqRec{e, slot, 0, ev, s_offsets[e], s_counts[e], 0, group};
+                s_req_of_expert[e] = n_hits + i;
+                s_miss[i] = HostMiss{e, slot, (int16_t)group, (int16_t)dep, 0u};
+                // cache update: the last miss that lands in a slot keeps it
+                const bool stays = i + C >= n_miss;
+                s_cache.slot_of_expert[e] = stays ? slot : -1;
+                if (stays) {
+                    s_cache.expert_of_slot[slot] = e;
+                    s_cache.stamp[slot] = counter + (uint64_t)(n_hits + i) + 1ull;
+                }
+                if (i < C && ev >= 0)
+                    s_cache.slot_of_expert[ev] = -1;
+            }
+        }
+        const int n_evict = __popcll(ballot64(ev_flag[0], ev_flag[1]));
+        counter += (uint64_t)n_req;
+        __syncwarp();
         if (lane == 0) {
-            const int n_groups = n_miss ? cur_group + 1 : 1;
+            const int n_groups = n_miss ? 1 + (n_miss + C - 1) / C : 1;
             int n_req_total = n_req;
             for (int s = 0; s < p.n_shared; ++s) {
                 s_req[n_req_total] = ReqRec{E + s, -1, 1, -1, s_offsets[E + s], p.T, 0, 0};
@@ -279,10 +295,11 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p)
     for (int i = tid; i < n_req_total; i += kPlanThreads)
         plan->req[i] = s_req[i];
     if (ok) {
-        for (int r = 0; r < n_req_total; ++r) {
+        // a warp per request, a lane per virtual request
+        for (int r = warp; r < n_req_total; r += kPlanWarps) {
             const ReqRec rec = s_req[r];
             const int nv = (rec.n_tok + kTokPerVr - 1) / kTokPerVr;
-            for (int v = tid; v < nv; v += kPlanThreads) {
+            for (int v = lane; v < nv; v += 32) {
                 VrRec vr;
                 vr.blob = rec.slot >= 0 ? p.slots + (size_t)rec.slot * p.slot_stride : p.shared_blobs[rec.expert - E];
                 vr.n_tok = min(kTokPerVr, rec.n_tok - v * kTokPerVr);

@@ -26,7 +26,9 @@ router_topk_kernel(const uint16_t *__restrict__ x, const uint16_t *__restrict__ 
                    int T, int d, int E, int k, int32_t *__restrict__ idx,
                    float *__restrict__ gate, float *__restrict__ logits_out)
 {
-    __shared__ float s_logit[TT][kMaxExperts];
+    __shared__ __align__(16) float s_logit[TT][kMaxExperts];
+    __shared__ float s_sel[TT][32];
+    __shared__ int32_t s_sel_idx[TT][32];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int t0 = blockIdx.x * TT;
 
@@ -38,9 +40,11 @@ router_topk_kernel(const uint16_t *__restrict__ x, const uint16_t *__restrict__ 
             acc[i][t] = 0.0f;
 
     const int n_chunks = d >> 8;
+#pragma unroll 2
     for (int c = 0; c < n_chunks; ++c) {
         const int col = (c << 8) + (lane << 3);
-        uint4 xv[TT];
+        // all of this step's loads go out before any arithmetic
+        uint4 xv[TT], wvs[kMaxExpertsPerWarp];
 #pragma unroll
         for (int t = 0; t < TT; ++t) {
             const int tt = min(t0 + t, T - 1);
@@ -49,8 +53,13 @@ router_topk_kernel(const uint16_t *__restrict__ x, const uint16_t *__restrict__ 
 #pragma unroll
         for (int i = 0; i < kMaxExpertsPerWarp; ++i) {
             const int e = warp + i * kRouterWarps;
+            wvs[i] = e < E ? __ldg(reinterpret_cast<const uint4 *>(w_r + (size_t)e * d + col)) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int i = 0; i < kMaxExpertsPerWarp; ++i) {
+            const int e = warp + i * kRouterWarps;
             if (e < E) {
-                const uint4 wv = __ldg(reinterpret_cast<const uint4 *>(w_r + (size_t)e * d + col));
+                const uint4 wv = wvs[i];
 #pragma unroll
                 for (int t = 0; t < TT; ++t) {
                     float a = acc[i][t];
@@ -93,45 +102,36 @@ router_topk_kernel(const uint16_t *__restrict__ x, const uint16_t *__restrict__ 
     if (warp < TT && t0 + warp < T) {
         const int t = t0 + warp;
         const float NEG = -__int_as_float(0x7f800000);  // -inf
-        float v0 = lane < E ? s_logit[warp][lane] : NEG;
-        float v1 = lane + 32 < E ? s_logit[warp][lane + 32] : NEG;
-        bool taken0 = !(lane < E), taken1 = !(lane + 32 < E);
-        float my_sel = 0.0f, top = 0.0f;
-        int my_idx = 0;
-        for (int j = 0; j < k; ++j) {
-            // local candidate: higher value wins, lower index wins a tie
-            float bv;
-            int bi;
-            if (!taken0 && (taken1 || v0 >= v1)) {
-                bv = v0;
-                bi = lane;
-            } else if (!taken1) {
-                bv = v1;
-                bi = lane + 32;
-            } else {
-                bv = NEG;
-                bi = 1 << 20;
-            }
+        // an element's rank is the number of elements that beat it (greater, or equal with a lower
+        // index); the k elements of rank below k are the selection, in order
+        const float v0 = lane < E ? s_logit[warp][lane] : NEG;
+        const float v1 = lane + 32 < E ? s_logit[warp][lane + 32] : NEG;
+        int r0 = 0, r1 = 0;
+        const float4 *row = reinterpret_cast<const float4 *>(s_logit[warp]);
 #pragma unroll
-            for (int m = 16; m >= 1; m >>= 1) {
-                const float ov = __shfl_xor_sync(0xffffffffu, bv, m);
-                const int oi = __shfl_xor_sync(0xffffffffu, bi, m);
-                if (ov > bv || (ov == bv && oi < bi)) {
-                    bv = ov;
-                    bi = oi;
-                }
-            }
-            if (bi == lane)
-                taken0 = true;
-            if (bi == lane + 32)
-                taken1 = true;
-            if (j == 0)
-                top = bv;
-            if (lane == j) {
-                my_sel = bv;
-                my_idx = bi;
+        for (int i = 0; i < kMaxExperts / 4; ++i) {
+            const float4 o4 = row[i];
+            const float ov[4] = {o4.x, o4.y, o4.z, o4.w};
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const int e = 4 * i + c;
+                const float o = e < E ? ov[c] : NEG;     // the row's tail beyond E was never written
+                r0 += (o > v0) || (o == v0 && e < lane);
+                r1 += (o > v1) || (o == v1 && e < lane + 32);
             }
         }
+        if (lane < E && r0 < k) {
+            s_sel[warp][r0] = v0;
+            s_sel_idx[warp][r0] = lane;
+        }
+        if (lane + 32 < E && r1 < k) {
+            s_sel[warp][r1] = v1;
+            s_sel_idx[warp][r1] = lane + 32;
+        }
+        __syncwarp();
+        const float top = s_sel[warp][0];
+        const float my_sel = lane < k ? s_sel[warp][lane] : 0.0f;
+        const int my_idx = lane < k ? s_sel_idx[warp][lane] : 0;
         float ev = lane < k ? expf(my_sel - top) : 0.0f;
         float sum = ev;
 #pragma unroll
@@ -150,7 +150,8 @@ cudaError_t launch_router(cudaStream_t stream, const uint16_t *x, const uint16_t
                           const float *bias, const int32_t *token_seq, int T, int d, int E, int k,
                           int32_t *idx, float *gate, float *logits_out)
 {
-    if (T <= 16) {
+    // one token per block while that still fills the GPU no more than twice over
+    if (T <= 296) {
         router_topk_kernel<1><<<T, kRouterWarps * 32, 0, stream>>>(x, w_r, bias, token_seq, T, d, E, k,
                                                                     idx, gate, logits_out);
     } else {
