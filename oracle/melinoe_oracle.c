@@ -11,8 +11,8 @@
  *   expert FFN        Eq. 3   E_i(x) = W_d ( phi(W_g x) (.) W_u x ),  phi = SiLU
  *   offloading model  Section 2 "Expert Offloading Systems" and Section 3.2: a bounded
  *                     per-layer cache of resident experts, fetch on demand, eviction by
- *                     the cache policy (LRU here; Definition C.1's gamma-discounted
- *                     Top-C cache reduces to it for gamma -> 0+)
+ *                     the cache policy: LRU, or the gamma-discounted count of
+ *                     Definition C.1 (gamma = 1 is LFU, gamma -> 0+ reduces to LRU)
  *   miss count        Appendix C.1: number of cache misses = number of transfers
  *
  * Precision: the routing decision is an integer result, so the logits that decide it are
@@ -20,7 +20,10 @@
  * path must reproduce bit for bit.  Everything else (gates, FFN, combine) is fp64 with no
  * intermediate rounding: it is Eq. 2-3 written out.
  *
- * Parity status: router indices, cache trace, gather lists and the FFN/combine are pinned
+ * The discounted counts decide an integer result (the victim), so they too are fp32 with a
+ * fixed rounding order that the GPU path reproduces.
+ *
+ * Parity status: router indices, cache trace (both policies), gather lists and the FFN/combine are pinned
  * by the CPU tests (closed forms, brute force, library cross-checks, the paper's printed
  * transfer-time example).  Unpinned by design: exact bits of expf inside softmax gates
  * (the gates are compared within a tolerance, never bit for bit).
@@ -199,6 +202,19 @@ int moe_oracle_gather(const int32_t *idx, int T, int K, int E,
  *    first the experts resident at call entry in ascending expert id, then the others in
  *    ascending expert id.  (Hits first lets their compute overlap the transfers, and never
  *    evicts a needed resident expert while another victim exists.)
+ *
+ * Second policy: the gamma-discounted count of Definition C.1 (gamma = 1 is LFU, the policy of
+ * the paper's experiments; gamma -> 0+ is LRU, by the remark under the definition).  Reading:
+ *  - one forward call is one time step: before its requests are served, every expert's count
+ *    becomes gamma * count + r, r = 1 for the experts the call requests and 0 for the others
+ *    (the count recurrence of Definition C.1), in fp32, product rounded before the sum;
+ *  - requests, hits, stamps and empty slots exactly as above; only the victim differs: the
+ *    occupied slot whose expert has the smallest count, the smaller stamp deciding ties (so
+ *    the policy falls back to LRU order where counts are equal);
+ *  - a preloaded expert's count is raised by one without a decay step (the definition leaves
+ *    the initial count vector to the prefetch; C preloaded experts give it L1 norm C).
+ * Definition C.1's cache is the Top-C of the counts; a demand-fetched cache can only change
+ * where a miss occurs (the "lazy update" of the remark), which is what this does.
  */
 typedef struct moe_oracle_cache {
     int C, E;
@@ -207,6 +223,9 @@ typedef struct moe_oracle_cache {
     uint64_t *stamp;         /* [C] */
     int32_t *slot_of_expert; /* [E], -1 = not resident */
     uint64_t hits, misses, evictions;
+    int policy;              /* 0 = LRU, 1 = gamma-discounted count */
+    float gamma;
+    float *count;            /* [E] */
 } moe_oracle_cache;
 
 typedef struct moe_oracle_request {
@@ -221,8 +240,20 @@ void moe_oracle_cache_reset(moe_oracle_cache *c)
         c->expert_of_slot[s] = -1;
         c->stamp[s] = 0;
     }
-    for (int e = 0; e < c->E; ++e)
+    for (int e = 0; e < c->E; ++e) {
         c->slot_of_expert[e] = -1;
+        c->count[e] = 0.0f;
+    }
+}
+
+/* policy 0 = LRU, 1 = gamma-discounted count (0 <= gamma <= 1).  Keeps the cache contents. */
+int moe_oracle_cache_set_policy(moe_oracle_cache *c, int policy, float gamma)
+{
+    if (!c || (policy != 0 && policy != 1) || !(gamma >= 0.0f && gamma <= 1.0f))
+        return -1;
+    c->policy = policy;
+    c->gamma = gamma;
+    return 0;
 }
 
 moe_oracle_cache *moe_oracle_cache_create(int C, int E)
@@ -237,6 +268,9 @@ moe_oracle_cache *moe_oracle_cache_create(int C, int E)
     c->expert_of_slot = (int32_t *)malloc(sizeof(int32_t) * (size_t)C);
     c->stamp = (uint64_t *)malloc(sizeof(uint64_t) * (size_t)C);
     c->slot_of_expert = (int32_t *)malloc(sizeof(int32_t) * (size_t)E);
+    c->count = (float *)malloc(sizeof(float) * (size_t)E);
+    c->policy = 0;
+    c->gamma = 0.0f;
     moe_oracle_cache_reset(c);
     return c;
 }
@@ -248,6 +282,7 @@ void moe_oracle_cache_destroy(moe_oracle_cache *c)
     free(c->expert_of_slot);
     free(c->stamp);
     free(c->slot_of_expert);
+    free(c->count);
     free(c);
 }
 
@@ -273,9 +308,17 @@ static void cache_one_request(moe_oracle_cache *c, int e, moe_oracle_request *ou
             break;
         }
     if (victim < 0) {
-        for (int i = 0; i < c->C; ++i)
-            if (victim < 0 || c->stamp[i] < c->stamp[victim])
+        for (int i = 0; i < c->C; ++i) {
+            if (victim < 0) {
                 victim = i;
+            } else if (c->policy == 1) {
+                const float ci = c->count[c->expert_of_slot[i]], cv = c->count[c->expert_of_slot[victim]];
+                if (ci < cv || (ci == cv && c->stamp[i] < c->stamp[victim]))
+                    victim = i;
+            } else if (c->stamp[i] < c->stamp[victim]) {
+                victim = i;
+            }
+        }
         out->evicted = c->expert_of_slot[victim];
         c->slot_of_expert[out->evicted] = -1;
         c->evictions++;
@@ -306,6 +349,11 @@ int moe_oracle_cache_call(moe_oracle_cache *c, const int32_t *idx, int n_idx,
     }
     for (int e = 0; e < c->E; ++e)
         was_resident[e] = (unsigned char)(c->slot_of_expert[e] >= 0);
+    if (c->policy == 1)
+        for (int e = 0; e < c->E; ++e) {
+            const float decayed = c->gamma * c->count[e];   /* rounded before the sum */
+            c->count[e] = decayed + (needed[e] ? 1.0f : 0.0f);
+        }
     for (int e = 0; e < c->E; ++e)
         if (needed[e] && was_resident[e])
             cache_one_request(c, e, &out[n++]);
@@ -316,6 +364,26 @@ done:
     free(needed);
     free(was_resident);
     return n;
+}
+
+/* Fill the cache ahead of the first token (Eq. 5's preloading step): one request per id, in
+ * order, no decay step; under the count policy each id's count grows by one. */
+int moe_oracle_cache_preload(moe_oracle_cache *c, const int32_t *ids, int n, moe_oracle_request *out)
+{
+    for (int i = 0; i < n; ++i) {
+        if (ids[i] < 0 || ids[i] >= c->E)
+            return -1;
+        if (c->policy == 1)
+            c->count[ids[i]] += 1.0f;
+        cache_one_request(c, ids[i], &out[i]);
+    }
+    return n;
+}
+
+void moe_oracle_cache_counts(const moe_oracle_cache *c, float *count)
+{
+    for (int e = 0; e < c->E; ++e)
+        count[e] = c->count[e];
 }
 
 void moe_oracle_cache_state(const moe_oracle_cache *c, int32_t *expert_of_slot,

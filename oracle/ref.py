@@ -29,6 +29,11 @@ def _L():
         lib.moe_oracle_cache_call.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]
         lib.moe_oracle_cache_call.restype = C.c_int
         lib.moe_oracle_cache_state.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        lib.moe_oracle_cache_set_policy.argtypes = [C.c_void_p, C.c_int, C.c_float]
+        lib.moe_oracle_cache_set_policy.restype = C.c_int
+        lib.moe_oracle_cache_preload.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]
+        lib.moe_oracle_cache_preload.restype = C.c_int
+        lib.moe_oracle_cache_counts.argtypes = [C.c_void_p, C.c_void_p]
         lib.moe_oracle_logits.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                           C.c_int, C.c_int, C.c_int, C.c_void_p]
         lib.moe_oracle_topk.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p]
@@ -100,13 +105,38 @@ def gather(idx: np.ndarray, n_experts: int):
 
 
 class ExpertCache:
-    """LRU expert cache of one layer; `call` takes one forward call's routing indices."""
+    """Expert cache of one layer; `call` takes one forward call's routing indices.
 
-    def __init__(self, cache_slots: int, n_experts: int):
+    policy "lru" (default) or "count": the gamma-discounted count of Definition C.1
+    (gamma = 1 is LFU).
+    """
+
+    def __init__(self, cache_slots: int, n_experts: int, policy: str = "lru", gamma: float = 0.0):
         self.C, self.E = int(cache_slots), int(n_experts)
         self._h = _L().moe_oracle_cache_create(self.C, self.E)
         if not self._h:
             raise ValueError("bad cache shape")
+        if policy != "lru":
+            self.set_policy(policy, gamma)
+
+    def set_policy(self, policy: str, gamma: float = 0.0) -> None:
+        code = {"lru": 0, "count": 1}[policy]
+        if _L().moe_oracle_cache_set_policy(self._h, code, C.c_float(gamma)):
+            raise ValueError("bad policy or gamma")
+
+    def preload(self, expert_ids) -> np.ndarray:
+        """One request per id, in order, before the first token; returns the request records."""
+        ids = np.ascontiguousarray(expert_ids, dtype=np.int32).reshape(-1)
+        out = np.empty((max(ids.size, 1), 4), dtype=np.int32)
+        n = _L().moe_oracle_cache_preload(self._h, _p(ids), ids.size, _p(out))
+        if n < 0:
+            raise ValueError("expert index out of range")
+        return out[:n].copy()
+
+    def counts(self) -> np.ndarray:
+        c = np.empty(self.E, dtype=np.float32)
+        _L().moe_oracle_cache_counts(self._h, _p(c))
+        return c
 
     def __del__(self):
         if getattr(self, "_h", None):

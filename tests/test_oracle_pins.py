@@ -314,6 +314,77 @@ def test_lru_equals_discounted_topc_cache_for_small_gamma():
         assert set(int(x) for x in eos if x >= 0) == top and top <= nz_after
 
 
+def test_count_policy_hand_worked_traces():
+    """Definition C.1's discounted count as the eviction key: traces worked by hand."""
+    for g in _gold("count_policy_trace.json")["cases"]:
+        c = oracle.ExpertCache(g["cache_slots"], g["n_experts"], "count", g["gamma"])
+        for call, want in zip(g["calls"], g["requests"]):
+            assert c.call(np.array(call, np.int32)).tolist() == want, g["comment"]
+
+
+@pytest.mark.parametrize("C,E,k,T", [(4, 8, 2, 1), (16, 64, 8, 1), (6, 16, 2, 8), (2, 8, 2, 1)])
+def test_count_policy_with_vanishing_gamma_is_lru(C, E, k, T):
+    """Remark under Definition C.1: gamma -> 0+ gives LRU updates.  With a gamma so small that a
+    count is 1 for the experts of the latest call and (in fp32) below that for all others, older
+    ones tying at zero, the trace must be the LRU trace, request for request."""
+    rs = np.random.default_rng(C + 7 * E)
+    lru = oracle.ExpertCache(C, E)
+    cnt = oracle.ExpertCache(C, E, "count", 1e-30)
+    pref = rs.dirichlet(np.full(E, 0.5))
+    for _ in range(150):
+        idx = np.stack([rs.choice(E, size=k, replace=False, p=pref) for _ in range(T)]).astype(np.int32)
+        assert cnt.call(idx).tolist() == lru.call(idx).tolist()
+
+
+@pytest.mark.parametrize("gamma", [1.0, 0.9, 0.5])
+def test_count_policy_evicts_a_minimal_discounted_count(gamma):
+    """Every victim has the smallest discounted count among the experts resident at that moment,
+    the counts taken from the closed form sum_s gamma^(t - s) r_e(s) over the request history
+    (fp64, no recurrence), the resident set tracked from the request records alone."""
+    rs = np.random.default_rng(int(gamma * 100))
+    C, E, k = 5, 14, 2
+    cache = oracle.ExpertCache(C, E, "count", gamma)
+    history = []                      # request vectors r(s), one per call
+    slot_expert = {}
+    pref = rs.dirichlet(np.full(E, 0.7))
+    n_evictions = 0
+    for t in range(250):
+        idx = rs.choice(E, size=k, replace=False, p=pref).astype(np.int32)
+        r = np.zeros(E)
+        r[idx] = 1.0
+        history.append(r)
+        w = gamma ** np.arange(len(history) - 1, -1, -1, dtype=np.float64)
+        count = (w[:, None] * np.array(history)).sum(axis=0)
+        for e, slot, hit, ev in cache.call(idx[None, :]).tolist():
+            if hit:
+                assert slot_expert[slot] == e
+                continue
+            if ev >= 0:
+                n_evictions += 1
+                assert slot_expert[slot] == ev
+                others = [x for s_, x in slot_expert.items() if s_ != slot]
+                assert count[ev] <= min(count[x] for x in others) * (1 + 1e-5) + 1e-12
+            else:
+                assert slot not in slot_expert
+            slot_expert[slot] = e
+        assert np.allclose(cache.counts(), count, rtol=1e-4, atol=1e-30)
+    assert n_evictions > 50
+
+
+def test_count_policy_preload_gives_the_definitions_initial_counts():
+    """Definition C.1 starts from a count vector of L1 norm C set by the prefetch: C preloaded experts
+    carry count 1 each, sit in the cache, and hit on the first call."""
+    C, E = 4, 12
+    cache = oracle.ExpertCache(C, E, "count", 0.9)
+    rec = cache.preload([7, 2, 9, 4])
+    assert rec[:, 2].tolist() == [0, 0, 0, 0] and rec[:, 1].tolist() == [0, 1, 2, 3]
+    cnt = cache.counts()
+    assert cnt.sum() == C and set(np.nonzero(cnt)[0].tolist()) == {2, 4, 7, 9}
+    first = cache.call(np.array([[2, 9]], np.int32))
+    assert first[:, 2].tolist() == [1, 1]
+    assert np.allclose(cache.counts()[[2, 9, 4, 7]], [1.9, 1.9, 0.9, 0.9])
+
+
 def test_miss_bytes_match_papers_transfer_example():
     g = _gold("transfer_time.json")
     cfg = gen.config_by_name("mixtral")
