@@ -192,6 +192,32 @@ int melinoe_moe_forward_static(melinoe_moe_t *h, void *cuda_stream, const void *
                                int n_tokens, void *out_dev, melinoe_moe_stats *stats_dev);
 size_t melinoe_moe_static_scratch_bytes(void);
 
+/*
+ * Eviction policy of the handle's cache (Section 4: the paper's experiments run an LFU cache;
+ * Definition C.1: the gamma-discounted count whose Top-C is the cache state, gamma = 1 being LFU
+ * and gamma -> 0+ LRU).
+ *   MELINOE_POLICY_LRU    (default) a miss takes the lowest empty slot, else the least recently
+ *                         requested expert's slot;
+ *   MELINOE_POLICY_COUNT  every forward call is one time step: each expert's count becomes
+ *                         gamma * count + (requested by this call ? 1 : 0), in fp32 with the product
+ *                         rounded before the sum; a miss takes the lowest empty slot, else the slot
+ *                         of the expert with the smallest count, the less recently requested one on
+ *                         ties.  0 <= gamma <= 1.  A preloaded expert's count is raised by one
+ *                         without a decay step.
+ * Takes effect from the next call; the cache contents and the counts are kept (the counts are
+ * maintained only while the count policy is set; melinoe_moe_reset_cache zeroes them).  Under the
+ * count policy a call's misses may form up to one compute group each (a freshly fetched expert
+ * has the smallest count), so they are served with less overlap than under LRU.  Waits for the
+ * handle's queued calls.  Returns MELINOE_ERR_INVALID for an unknown policy or a gamma out of range.
+ */
+#define MELINOE_POLICY_LRU 0
+#define MELINOE_POLICY_COUNT 1
+int melinoe_moe_set_policy(melinoe_moe_t *h, int policy, float gamma);
+
+/* The experts' discounted counts (see melinoe_moe_set_policy): counts_host [n_experts] fp32.
+ * Waits for the handle's queued calls. */
+int melinoe_moe_cache_counts(melinoe_moe_t *h, float *counts_host);
+
 /* Cold start: all slots empty, stamps and totals zero.  Synchronises the handle first. */
 int melinoe_moe_reset_cache(melinoe_moe_t *h);
 

@@ -21,7 +21,7 @@ EXPORTED_SYMBOLS = [
     "melinoe_moe_last_requests", "melinoe_moe_last_gather", "melinoe_moe_cache_state",
     "melinoe_moe_enable_timing", "melinoe_moe_ffn_time_ms", "melinoe_moe_set_trace", "melinoe_moe_trace_ctas",
     "melinoe_moe_transfer_time_ms", "melinoe_moe_forward_static", "melinoe_moe_static_scratch_bytes",
-    "melinoe_moe_last_call_used_gemm", "melinoe_launch_count",
+    "melinoe_moe_last_call_used_gemm", "melinoe_moe_set_policy", "melinoe_moe_cache_counts", "melinoe_launch_count",
     "melinoe_last_cuda_error", "melinoe_strerror",
 ]
 
@@ -79,6 +79,8 @@ def lib():
     L.melinoe_moe_static_scratch_bytes.restype = sz
     L.melinoe_moe_last_call_used_gemm.argtypes = [vp]
     L.melinoe_moe_reset_cache.argtypes = [vp]
+    L.melinoe_moe_set_policy.argtypes = [vp, i32, C.c_float]
+    L.melinoe_moe_cache_counts.argtypes = [vp, vp]
     L.melinoe_moe_preload.argtypes = [vp, vp, i32]
     L.melinoe_moe_last_routing.argtypes = [vp, vp, vp]
     L.melinoe_moe_last_logits.argtypes = [vp, vp]
@@ -205,6 +207,17 @@ class MoELayer:
 
     def reset_cache(self) -> None:
         self._ck(lib().melinoe_moe_reset_cache(self._h), "melinoe_moe_reset_cache")
+
+    def set_policy(self, policy: str, gamma: float = 0.0) -> None:
+        """Eviction policy: "lru" (default) or "count" (Definition C.1's discounted count; gamma = 1 is LFU)."""
+        code = {"lru": 0, "count": 1}[policy]
+        self._ck(lib().melinoe_moe_set_policy(self._h, code, C.c_float(gamma)), "melinoe_moe_set_policy")
+
+    def cache_counts(self, n_experts: int):
+        import numpy as np
+        out = np.empty(n_experts, dtype=np.float32)
+        self._ck(lib().melinoe_moe_cache_counts(self._h, out.ctypes.data), "melinoe_moe_cache_counts")
+        return out
 
     def preload(self, expert_ids) -> None:
         import numpy as np

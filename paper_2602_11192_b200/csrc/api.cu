@@ -104,6 +104,8 @@ struct melinoe_moe {
     // device memory owned by the handle
     char *slots = nullptr;
     DevCache *cache = nullptr;
+    int policy = MELINOE_POLICY_LRU;   // eviction policy, see melinoe_moe_set_policy
+    float gamma = 0.0f;
     DevPlan *plan = nullptr;
     int *err_word = nullptr;
     const char **shared_dev = nullptr;
@@ -169,6 +171,8 @@ int gmax_for(const melinoe_moe *h, int T)
     long long u = (long long)T * h->k;
     if (u > h->E)
         u = h->E;
+    if (h->policy == MELINOE_POLICY_COUNT)
+        return 1 + (int)u;     // every miss may be a wave of its own
     return 1 + (int)((u + h->C - 1) / h->C);
 }
 
@@ -573,10 +577,12 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
     pp.sync = h->sync;
     pp.gmax = gmax;
     pp.call_seq = h->call_seq;
+    pp.policy = h->policy;
+    pp.gamma = h->gamma;
     pp.stats = stats_dev;
     pp.expert_bytes = h->expert_bytes;
     pp.vr_capacity = h->vr_capacity;
-    if (route_plan_small_supported(T, h->k, h->d)) {
+    if (h->policy == MELINOE_POLICY_LRU && route_plan_small_supported(T, h->k, h->d)) {
         CU_TRY(launch_route_plan_small(s, static_cast<const uint16_t *>(hidden_dev), h->w_router, h->bias, h->token_seq,
                                        h->d, h->idx, h->gate, h->logits, pp));
     } else {
@@ -922,6 +928,32 @@ int melinoe_moe_reset_cache(melinoe_moe_t *h)
     return MELINOE_OK;
 }
 
+int melinoe_moe_set_policy(melinoe_moe_t *h, int policy, float gamma)
+{
+    if (!h || (policy != MELINOE_POLICY_LRU && policy != MELINOE_POLICY_COUNT) || !(gamma >= 0.0f && gamma <= 1.0f))
+        return MELINOE_ERR_INVALID;
+    int rc = wait_idle(h);
+    if (rc != MELINOE_OK)
+        return rc;
+    h->policy = policy;
+    h->gamma = gamma;
+    return MELINOE_OK;
+}
+
+int melinoe_moe_cache_counts(melinoe_moe_t *h, float *counts_host)
+{
+    if (!h || !counts_host)
+        return MELINOE_ERR_INVALID;
+    int rc = wait_idle(h);
+    if (rc != MELINOE_OK)
+        return rc;
+    DevCache c;
+    CU_TRY(cudaMemcpy(&c, h->cache, sizeof c, cudaMemcpyDeviceToHost));
+    for (int e = 0; e < h->E; ++e)
+        counts_host[e] = c.count[e];
+    return MELINOE_OK;
+}
+
 int melinoe_moe_preload(melinoe_moe_t *h, const int32_t *ids, int n)
 {
     if (!h || n < 0 || (n > 0 && !ids) || n > h->C)
@@ -939,6 +971,8 @@ int melinoe_moe_preload(melinoe_moe_t *h, const int32_t *ids, int n)
             return MELINOE_ERR_INVALID;
         c.call_no += 1;
         const uint64_t st = ++c.counter;
+        if (h->policy == MELINOE_POLICY_COUNT)
+            c.count[e] += 1.0f;
         if (c.slot_of_expert[e] >= 0) {
             c.stamp[c.slot_of_expert[e]] = st;
             c.tot_hits += 1;
@@ -949,9 +983,17 @@ int melinoe_moe_preload(melinoe_moe_t *h, const int32_t *ids, int n)
             if (c.expert_of_slot[s] < 0)
                 victim = s;
         if (victim < 0) {
-            for (int s = 0; s < h->C; ++s)
-                if (victim < 0 || c.stamp[s] < c.stamp[victim])
+            for (int s = 0; s < h->C; ++s) {
+                if (victim < 0) {
                     victim = s;
+                } else if (h->policy == MELINOE_POLICY_COUNT) {
+                    const float cs = c.count[c.expert_of_slot[s]], cv = c.count[c.expert_of_slot[victim]];
+                    if (cs < cv || (cs == cv && c.stamp[s] < c.stamp[victim]))
+                        victim = s;
+                } else if (c.stamp[s] < c.stamp[victim]) {
+                    victim = s;
+                }
+            }
             c.slot_of_expert[c.expert_of_slot[victim]] = -1;
             c.tot_evictions += 1;
         }

@@ -25,6 +25,10 @@ struct DevCache {
     uint64_t tot_hits, tot_misses, tot_evictions;
     uint64_t call_no;
     uint64_t tot_vr;                        // virtual requests handed to the FFN kernels so far
+    // gamma-discounted request count of every expert (Definition C.1), kept for the count policy:
+    // one step per forward call, count <- gamma * count + (requested ? 1 : 0), fp32, the product
+    // rounded before the sum
+    float count[kMaxExperts];
 };
 
 // One cache request of a call plus what the compute kernels need to serve it.

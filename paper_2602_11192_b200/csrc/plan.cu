@@ -66,6 +66,9 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p)
             s_misc[6] = MELINOE_ERR_INVALID;
     }
     __syncthreads();
+    // count policy (Definition C.1): one time step per call, count <- gamma * count + request
+    if (p.policy == MELINOE_POLICY_COUNT && tid < E)
+        s_cache.count[tid] = __fadd_rn(__fmul_rn(p.gamma, s_cache.count[tid]), s_counts[tid] > 0 ? 1.0f : 0.0f);
     if (tid == 0) {
         int run = 0;
         for (int e = 0; e < E; ++e) {
@@ -119,8 +122,8 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p)
     }
     for (int i = tid; i < p.n_shared * p.T; i += kPlanThreads)
         p.tok_of_sorted[n_pairs + i] = i % p.T;
-    for (int i = tid; i <= kMaxGroups; i += kPlanThreads)
-        p.sync[i] = 0u;
+    for (int i = tid; i < 2 * (kMaxGroups + 1); i += kPlanThreads)
+        p.sync[i] = 0u;      // two barrier counters per compute group
 
     // ---- (b), (c): cache requests, by warp 0; lane owns experts lane and lane + 32 and slots lane and
     // lane + 32.  The sequential rules (hits in ascending id, then misses in ascending id, a miss
@@ -164,6 +167,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p)
                 s_cache.stamp[soe] = st;
                 s_req[r] = ReqRec{e, soe, 1, -1, s_offsets[e], s_counts[e], 0, 0};
                 s_req_of_expert[e] = r;
+                s_group_of_expert[e] = 0;
             }
             if ((miss_mask >> e) & 1ull)
                 s_miss_expert[rank_below(miss_mask, e)] = e;
@@ -184,6 +188,67 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p)
         }
         __syncwarp();
         bool ev_flag[2] = {false, false};
+        int n_groups = n_miss ? 1 + (n_miss + C - 1) / C : 1;
+        int n_evict_seq = 0;
+        if (p.policy == MELINOE_POLICY_COUNT) {
+            // The count policy has no closed form (a victim depends on the counts of what the
+            // earlier misses of the call brought in): one search per miss, in ascending expert id.
+            // Victim: lowest empty slot, else the smallest (count of the occupant, stamp).
+            int cur_group = 1, i = 0;
+            for (uint64_t m = miss_mask; m; m &= m - 1, ++i) {
+                const int e = __ffsll((long long)m) - 1;
+                uint64_t khi = ~0ull, klo = ~0ull;
+                int slot = -1;
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const int sl = lane + 32 * h;
+                    if (sl < C) {
+                        const int occ = s_cache.expert_of_slot[sl];
+                        const uint64_t hi = occ < 0 ? 0ull : ((1ull << 32) | (uint64_t)__float_as_uint(s_cache.count[occ]));
+                        const uint64_t lo = occ < 0 ? (uint64_t)sl : s_cache.stamp[sl];
+                        if (hi < khi || (hi == khi && lo < klo)) {
+                            khi = hi;
+                            klo = lo;
+                            slot = sl;
+                        }
+                    }
+                }
+#pragma unroll
+                for (int mm = 16; mm >= 1; mm >>= 1) {
+                    const uint64_t ohi = __shfl_xor_sync(0xffffffffu, khi, mm);
+                    const uint64_t olo = __shfl_xor_sync(0xffffffffu, klo, mm);
+                    const int os = __shfl_xor_sync(0xffffffffu, slot, mm);
+                    if (ohi < khi || (ohi == khi && olo < klo)) {
+                        khi = ohi;
+                        klo = olo;
+                        slot = os;
+                    }
+                }
+                const int ev = s_cache.expert_of_slot[slot];
+                int dep = -1;
+                if (ev >= 0) {
+                    ++n_evict_seq;
+                    if ((need >> ev) & 1ull)
+                        dep = s_group_of_expert[ev];
+                }
+                if (dep == cur_group)
+                    ++cur_group;      // it would overwrite an expert of the current wave: next wave
+                __syncwarp();
+                if (lane == 0) {
+                    if (ev >= 0)
+                        s_cache.slot_of_expert[ev] = -1;
+                    s_cache.expert_of_slot[slot] = e;
+                    s_cache.slot_of_expert[e] = slot;
+                    s_cache.stamp[slot] = counter + (uint64_t)(n_hits + i) + 1ull;
+                    s_req[n_hits + i] = ReqRec{e, slot, 0, ev, s_offsets[e], s_counts[e], 0, cur_group};
+                    s_req_of_expert[e] = n_hits + i;
+                    s_group_of_expert[e] = cur_group;
+                    s_miss[i] = HostMiss{e, slot, (int16_t)cur_group, (int16_t)dep, 0u};
+                }
+                __syncwarp();
+            }
+            n_groups = n_miss ? cur_group + 1 : 1;
+        } else
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             const int e = h ? e1 : e0;
@@ -212,11 +277,10 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p)
                     s_cache.slot_of_expert[ev] = -1;
             }
         }
-        const int n_evict = __popcll(ballot64(ev_flag[0], ev_flag[1]));
+        const int n_evict = p.policy == MELINOE_POLICY_COUNT ? n_evict_seq : __popcll(ballot64(ev_flag[0], ev_flag[1]));
         counter += (uint64_t)n_req;
         __syncwarp();
         if (lane == 0) {
-            const int n_groups = n_miss ? 1 + (n_miss + C - 1) / C : 1;
             int n_req_total = n_req;
             for (int s = 0; s < p.n_shared; ++s) {
                 s_req[n_req_total] = ReqRec{E + s, -1, 1, -1, s_offsets[E + s], p.T, 0, 0};

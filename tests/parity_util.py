@@ -42,6 +42,14 @@ class Pair:
         self.bias, self.seq = bias, seq
         self.gpu.set_bias(bias, seq)
 
+    def set_policy(self, policy, gamma=0.0):
+        self.gpu.layer.set_policy(policy, gamma)
+        self.cache.set_policy(policy, gamma)
+
+    def preload(self, ids):
+        self.gpu.layer.preload(np.asarray(ids, np.int32))
+        self.cache.preload(ids)
+
     def reset(self):
         self.gpu.layer.reset_cache()
         self.cache.reset()
@@ -69,6 +77,8 @@ class Pair:
         assert np.array_equal(req_g, req_o), "cache trace differs:\n%s\n%s" % (req_g, req_o)
         assert np.array_equal(cnt_g, cnt_o) and np.array_equal(off_g, off_o) and np.array_equal(perm_g, perm_o)
         assert np.array_equal(eos_g, eos_o) and tot_g == tot_o
+        # the discounted counts decide evictions: same bits on both sides
+        assert np.array_equal(L.cache_counts(self.E).view(np.uint32), self.cache.counts().view(np.uint32))
         st = res["stats"]
         assert st["status"] == 0 and st["n_tokens"] == T and st["n_distinct"] == len(req_o)
         assert st["hits"] == int(req_o[:, 2].sum()) and st["misses"] == len(req_o) - int(req_o[:, 2].sum())

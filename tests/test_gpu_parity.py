@@ -170,6 +170,44 @@ def test_preload_fills_the_cache_before_the_first_token():
     P.close()
 
 
+@pytest.mark.parametrize("gamma", [1.0, 0.9, 0.5])
+def test_count_policy_trace_matches_the_oracle(gamma):
+    """Definition C.1's discounted-count eviction (gamma = 1: LFU): requests, victims, compute
+    groups' results and the fp32 counts agree with the oracle call by call, decode and prefill."""
+    d, F, E, k, C = 256, 64, 16, 2, 4
+    P = _pair(d, F, E, k, C, seed=31)
+    P.set_policy("count", gamma)
+    bias = np.stack([gen.router_bias(31, 0, s, 0.3, E) for s in range(4)])
+    n_evict = 0
+    for step in range(40):
+        T = (1, 3, 8)[step % 3]
+        P.set_bias(bias, (np.arange(T) % 4).astype(np.int32))
+        _, out = P.step(gen.hidden_states(31, 0, "decode", step, T, d))
+        n_evict += int((out["req"][:, 3] >= 0).sum())
+    assert n_evict > 20
+    P.set_bias(bias, (np.arange(40) % 4).astype(np.int32))
+    P.step(gen.hidden_states(31, 0, "prefill", 0, 40, d))     # many misses in one call: one wave each at worst
+    # back to LRU on the same cache contents: the trace follows the LRU oracle again
+    P.set_policy("lru")
+    P.set_bias(bias, np.zeros(1, np.int32))
+    for step in range(6):
+        P.step(gen.hidden_states(31, 0, "decode", 100 + step, 1, d))
+    P.close()
+
+
+def test_count_policy_preload_and_lfu_keeps_the_hot_experts():
+    d, F, E, k, C = 256, 32, 8, 2, 4
+    P = _pair(d, F, E, k, C, seed=33)
+    P.set_policy("count", 1.0)
+    P.preload([5, 1, 6, 2])
+    assert np.array_equal(P.gpu.layer.cache_counts(E), P.cache.counts())
+    for step in range(12):
+        P.step(gen.hidden_states(33, 0, "decode", step, 2, d))
+    with pytest.raises(Exception):
+        P.gpu.layer.set_policy("count", 1.5)
+    P.close()
+
+
 def test_argument_and_state_errors():
     import torch
     from paper_2602_11192_b200 import MoELayer, MelinoeError, melinoe_moe_expert_bytes
