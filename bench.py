@@ -347,6 +347,15 @@ def run_ours(args):
             phase("alpha=%g" % a)
             ms_a, _, st_a, _, _ = timed_device(a)
             extra["alpha=%g" % a] = dict(value=cfg.batch * K / (ms_a * 1e-3), **hit_summary(st_a))
+        # the paper's other eviction policies on the same stream (its Table 13 compares transfers under
+        # LRU and LFU): Definition C.1's discounted count, gamma = 1 (LFU) and gamma = 0.9.  These runs
+        # plan with the general kernels, so their tokens/s also carries that difference.
+        for name, g in (("policy=lfu", 1.0), ("policy=count,gamma=0.9", 0.9)):
+            phase(name)
+            stack.set_policy("count", g)
+            ms_p, _, st_p, _, _ = timed_device(alpha0)
+            extra[name] = dict(value=cfg.batch * K / (ms_p * 1e-3), **hit_summary(st_p))
+        stack.set_policy("lru")
         # everything resident (cache = all experts, warm): the FFN kernel without the miss path
         phase("all experts resident")
         stack.close()

@@ -582,7 +582,7 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
     pp.stats = stats_dev;
     pp.expert_bytes = h->expert_bytes;
     pp.vr_capacity = h->vr_capacity;
-    if (h->policy == MELINOE_POLICY_LRU && route_plan_small_supported(T, h->k, h->d)) {
+    if (route_plan_small_supported(T, h->k, h->d)) {
         CU_TRY(launch_route_plan_small(s, static_cast<const uint16_t *>(hidden_dev), h->w_router, h->bias, h->token_seq,
                                        h->d, h->idx, h->gate, h->logits, pp));
     } else {

@@ -33,7 +33,7 @@ struct PlanParams {
     unsigned *sync;           // grid-barrier counters of the FFN launches, zeroed here
     uint32_t gmax;            // compute groups the caller has room for
     uint32_t call_seq;        // written to the miss queue's seq word when the record is complete
-    int policy;               // MELINOE_POLICY_LRU or MELINOE_POLICY_COUNT (general planning kernel only)
+    int policy;               // MELINOE_POLICY_LRU or MELINOE_POLICY_COUNT
     float gamma;              // decay of the count policy
     melinoe_moe_stats *stats; // may be null
     size_t expert_bytes;

@@ -89,6 +89,12 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
     __shared__ __align__(16) float s_logit[kMaxT][kMaxExperts];
     __shared__ int32_t s_cnt[2][kMaxExperts];                    // pairs of an expert among pairs 0..31 / 32..63
     __shared__ int32_t s_tok[kMaxPairs];                         // token of a pair
+    // count policy only: live slot table during the call's misses, counts, groups
+    __shared__ int32_t s_live_occ[kMaxExperts];
+    __shared__ unsigned long long s_live_stamp[kMaxExperts];
+    __shared__ float s_cntf[kMaxExperts];
+    __shared__ int32_t s_grp_of[kMaxExperts];
+    __shared__ int32_t s_grp_first[kMaxGroups + 1];              // first miss of a wave
     __shared__ int32_t s_idx[kMaxPairs];
     __shared__ int32_t s_pair_at[kMaxPairs];                     // pair at sorted position
     __shared__ unsigned long long s_key[kMaxExperts];            // victim-order key of a slot
@@ -132,7 +138,15 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
     DevCache *cache = p.cache;
     int soe0 = -1, soe1 = -1, eos0 = -1, eos1 = -1;
     unsigned long long st0 = 0ull, st1 = 0ull, counter = 0ull, call_no = 0ull;
+    float cnt0 = 0.0f, cnt1 = 0.0f;
+    const bool by_count = p.policy == MELINOE_POLICY_COUNT;
     if (cta_rank == 0 && warp == 0) {
+        if (by_count) {
+            if (lane < E)
+                cnt0 = cache->count[lane];
+            if (lane + 32 < E)
+                cnt1 = cache->count[lane + 32];
+        }
         if (lane < E)
             soe0 = cache->slot_of_expert[lane];
         if (lane + 32 < E)
@@ -301,10 +315,23 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
     const uint64_t resident = ballot64(soe0 >= 0, soe1 >= 0);
     const uint64_t hit_mask = need & resident, miss_mask = need & ~resident;
     const int n_hits = __popcll(hit_mask), n_miss = __popcll(miss_mask), n_req = n_hits + n_miss;
-    const int n_groups = n_miss ? 1 + (n_miss + C - 1) / C : 1;
+    // compute groups: closed form under LRU; under the count policy known only after the misses
+    // have been walked, one wave per miss at most
+    int n_groups = n_miss ? 1 + (by_count ? n_miss : (n_miss + C - 1) / C) : 1;
     const int nvr = n_req + p.n_shared;
     const int status = (nvr > p.vr_capacity || n_groups > (int)p.gmax) ? MELINOE_ERR_STATE : MELINOE_OK;
     const bool ok = status == MELINOE_OK;
+    if (by_count) {
+        // Definition C.1: one time step per call, count <- gamma * count + request
+        const float n0 = __fadd_rn(__fmul_rn(p.gamma, cnt0), c0 > 0 ? 1.0f : 0.0f);
+        const float n1 = __fadd_rn(__fmul_rn(p.gamma, cnt1), c1 > 0 ? 1.0f : 0.0f);
+        s_cntf[lane] = n0;
+        s_cntf[lane + 32] = n1;
+        if (e0 < E)
+            cache->count[e0] = n0;
+        if (e1 < E)
+            cache->count[e1] = n1;
+    }
 
     // victim-order key of every slot: empty slots by index, then occupied ones by stamp, with the
     // stamps this call's hits receive
@@ -322,6 +349,7 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
             s_key[soe] = (1ull << 63) | st;
             cache->stamp[soe] = st;
             plan->req[r] = ReqRec{e, soe, 1, -1, off, cnt, r, 0};
+            s_grp_of[e] = 0;
             if (ok)
                 write_vr(p.vrs + r, p.slots + (size_t)soe * p.slot_stride, cnt, 0, off, s_pair_at, s_tok);
         }
@@ -344,6 +372,87 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
     }
     __syncwarp();
     bool ev_flag[2] = {false, false};
+    int n_evict_seq = 0;
+    if (by_count) {
+        // The count policy has no closed form (a victim depends on the counts of what the earlier
+        // misses of the call brought in): one search per miss, in ascending expert id, over a live
+        // copy of the slot table.  Victim: lowest empty slot, else the smallest (count of the
+        // occupant, stamp).  A new wave starts when a miss would overwrite an expert of the
+        // current wave.
+        s_live_occ[lane] = eos0;
+        s_live_occ[lane + 32] = eos1;
+        s_live_stamp[lane] = s_key[lane] & ~(1ull << 63);
+        s_live_stamp[lane + 32] = s_key[lane + 32] & ~(1ull << 63);
+        if (lane == 0)
+            s_grp_first[1] = 0;
+        __syncwarp();
+        int cur_group = 1, i = 0;
+        for (uint64_t m = miss_mask; m; m &= m - 1, ++i) {
+            const int e = __ffsll((long long)m) - 1;
+            unsigned long long khi = ~0ull, klo = ~0ull;
+            int slot = -1;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int sl = lane + 32 * h;
+                if (sl < C) {
+                    const int occ = s_live_occ[sl];
+                    const unsigned long long hi = occ < 0 ? 0ull : ((1ull << 32) | (unsigned long long)__float_as_uint(s_cntf[occ]));
+                    const unsigned long long lo = occ < 0 ? (unsigned long long)sl : s_live_stamp[sl];
+                    if (hi < khi || (hi == khi && lo < klo)) {
+                        khi = hi;
+                        klo = lo;
+                        slot = sl;
+                    }
+                }
+            }
+#pragma unroll
+            for (int mm = 16; mm >= 1; mm >>= 1) {
+                const unsigned long long ohi = __shfl_xor_sync(0xffffffffu, khi, mm);
+                const unsigned long long olo = __shfl_xor_sync(0xffffffffu, klo, mm);
+                const int os = __shfl_xor_sync(0xffffffffu, slot, mm);
+                if (ohi < khi || (ohi == khi && olo < klo)) {
+                    khi = ohi;
+                    klo = olo;
+                    slot = os;
+                }
+            }
+            const int ev = s_live_occ[slot];
+            int dep = -1;
+            if (ev >= 0) {
+                ++n_evict_seq;
+                if ((need >> ev) & 1ull)
+                    dep = s_grp_of[ev];
+            }
+            if (dep == cur_group) {
+                ++cur_group;
+                if (lane == 0)
+                    s_grp_first[cur_group] = i;
+            }
+            __syncwarp();
+            // the expert's token list: offset and count live with the lane that owns the expert
+            const int cnt = __shfl_sync(0xffffffffu, e < 32 ? c0 : c1, e & 31);
+            const int off = __shfl_sync(0xffffffffu, e < 32 ? off0 : off1, e & 31);
+            if (lane == 0) {
+                const unsigned long long st = counter + (unsigned long long)(n_hits + i) + 1ull;
+                const int vr_at = n_hits + p.n_shared + i;
+                if (ev >= 0)
+                    cache->slot_of_expert[ev] = -1;
+                cache->expert_of_slot[slot] = e;
+                cache->slot_of_expert[e] = slot;
+                cache->stamp[slot] = st;
+                s_live_occ[slot] = e;
+                s_live_stamp[slot] = st;
+                s_grp_of[e] = cur_group;
+                plan->req[n_hits + i] = ReqRec{e, slot, 0, ev, off, cnt, vr_at, cur_group};
+                if (ok)
+                    write_vr(p.vrs + vr_at, p.slots + (size_t)slot * p.slot_stride, cnt, cur_group, off, s_pair_at, s_tok);
+                const HostMiss hm{e, slot, (int16_t)cur_group, (int16_t)dep, p.call_seq};
+                store16_host(&p.hplan->miss[i], &hm);
+            }
+            __syncwarp();
+        }
+        n_groups = n_miss ? cur_group + 1 : 1;
+    } else
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
         const int e = h ? e1 : e0, cnt = h ? c1 : c0, off = h ? off1 : off0;
@@ -375,7 +484,7 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
             store16_host(&p.hplan->miss[i], &m);
         }
     }
-    const int n_evict = __popcll(ballot64(ev_flag[0], ev_flag[1]));
+    const int n_evict = by_count ? n_evict_seq : __popcll(ballot64(ev_flag[0], ev_flag[1]));
     // shared experts: always resident, group 0, behind the hits
     for (int s = lane; s < p.n_shared; s += 32) {
         const int off = n_pairs + s * T;
@@ -396,7 +505,8 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
     for (int g = lane; g <= kMaxGroups; g += 32) {
         int b = 0;
         if (ok && g >= 1) {
-            const int done = (g - 1) * C;
+            // misses served before wave g: (g - 1) * C under LRU, the wave's recorded first miss otherwise
+            const int done = by_count ? (g < n_groups ? s_grp_first[g] : n_miss) : (g - 1) * C;
             b = n_hits + p.n_shared + (done < n_miss ? done : n_miss);
         }
         plan->group_vr_begin[g] = b;

@@ -33,7 +33,7 @@ class Stack:
     """
 
     def __init__(self, cfg: gen.MoEConfig, alpha: float, cache_slots: int, n_layers: Optional[int] = None,
-                 verbose: bool = False):
+                 verbose: bool = False, policy: str = "lru", gamma: float = 0.0):
         self.cfg, self.alpha, self.C = cfg, float(alpha), int(cache_slots)
         self.L = cfg.n_layers if n_layers is None else int(n_layers)
         self.layers: List[LayerSetup] = []
@@ -49,6 +49,8 @@ class Stack:
             del wg, wu, wd
             w_r = gen.router_weights(cfg.seed, l, cfg.n_experts, cfg.d_model)
             ls.set_router(w_r)
+            if policy != "lru":
+                ls.layer.set_policy(policy, gamma)
             bias = np.stack([gen.router_bias(cfg.seed, l, s, self.alpha, cfg.n_experts) for s in range(cfg.batch)])
             self.w_r.append(w_r)
             self.bias.append(bias)
@@ -78,6 +80,10 @@ class Stack:
         c = self.cfg
         T = c.batch if phase == "decode" else c.batch * c.prefill_tokens
         return np.stack([gen.hidden_states(c.seed, l, phase, step, T, c.d_model) for l in range(self.L)])
+
+    def set_policy(self, policy: str, gamma: float = 0.0) -> None:
+        for ls in self.layers:
+            ls.layer.set_policy(policy, gamma)
 
     def reset(self) -> None:
         for ls in self.layers:
