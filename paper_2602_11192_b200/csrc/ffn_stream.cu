@@ -213,7 +213,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(harr + 8 * i), "r"(kConsumerWarps));
         for (int i = 0; i < kMaxSub; ++i) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(full2 + 8 * i), "r"(1));
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(empty2 + 8 * i), "r"(1));
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(empty2 + 8 * i), "r"(2 * F > CB2 ? kConsumerWarps : 1));
         }
         for (int i = 0; i < kMaxStages; ++i) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(full1 + 8 * i), "r"(1));
@@ -691,24 +691,27 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
         }
     }
 
-    // ---- down: z = W_d h for this CTA's output rows.  A tile (up to 16 output rows of one request)
-    // belongs to ONE warp, tile j to warp j mod 8: D[16 rows x 8 tokens] accumulates in that warp's
-    // registers over all the pieces of the rows, so nothing is reduced across warps or lanes and
-    // the tiles in the ring are worked on side by side.  (A tile of short rows costs its warp a few
-    // hundred instructions; shared out over eight warps it would cost each of them mostly the
-    // latency of seeing the barrier and of meeting the others.)  Every warp waits for every stage
-    // in order, also those of other warps' tiles: a warp that waited for phase k + 1 of a barrier
-    // whose phase k it has not seen could be let through by the parity test.
+    // ---- down: z = W_d h for this CTA's output rows, D[16 rows x 8 tokens] per tile.
+    // Short rows (a tile is one stage): a tile belongs to ONE warp, tile j to warp j mod 8, so
+    // nothing is reduced across warps and the tiles in the ring are worked on side by side.  (Such
+    // a tile costs its warp a few hundred instructions; shared out over eight warps it would cost
+    // each of them mostly the latency of seeing the barrier and of meeting the others.)
+    // Long rows (a tile is several stages, each a 64 KB piece): one warp would need longer for a
+    // stage than the stage takes to arrive, so the eight warps share every stage as in the gate/up
+    // phase and meet in shared memory once per tile.
+    // Either way every warp waits for every stage in order: a warp that waited for phase k + 1 of a
+    // barrier whose phase k it has not seen could be let through by the parity test.
     {
         Down dc = down_first(n);     // the down phase takes the slots in ring order after the gate/up stages
         bool first = true;
+        const bool shared2 = nk2 > 1;
         const uint32_t a_off = ((lane & 7) + ((lane >> 3) & 1) * 8) * PITCH2 + (lane >> 4) * 16;
         const uint32_t b_off = (ROWS2 + g) * PITCH2 + tig * 4;
         int tile_no = 0;
         for (int v = 0; v < nv; ++v) {
             const VrInfo vi = load_vr(vb + v);
             for (int blk = 0; blk < mt; ++blk, ++tile_no) {
-                const bool mine = (tile_no & (kConsumerWarps - 1)) == warp;
+                const bool mine = shared2 || (tile_no & (kConsumerWarps - 1)) == warp;
                 for (int kc = 0; kc < nk2; ++kc) {
                     mbar_wait(full2 + 8 * down_bar(dc), dc.use & 1u, abort_flag);
                     if (trace && first && tid == 0)
@@ -718,8 +721,13 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
                         const uint32_t base = ring_s + down_off(dc);
                         const int bytes = min(CB2, rb2 - kc * CB2);
                         const bool has_tok = g < vi.n_tok;
-                        mma_steps(base, a_off, b_off, 0, bytes >> 5, has_tok);
-                        if (bytes & 16) {
+                        const int ks_total = bytes >> 5;
+                        if (shared2)
+                            mma_steps(base, a_off, b_off, warp * ks_total / kConsumerWarps,
+                                      (warp + 1) * ks_total / kConsumerWarps, has_tok);
+                        else
+                            mma_steps(base, a_off, b_off, 0, ks_total, has_tok);
+                        if ((bytes & 16) && (!shared2 || warp == kConsumerWarps - 1)) {
                             // the row ends on half a step: columns 8..15 of both operands count as zero
                             const int ks = bytes >> 5;
                             uint32_t a0, a1, a2, a3;
@@ -733,14 +741,24 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
                     }
                     down_next(dc);
                 }
-                if (mine) {
+                float r4[4];
+                bool store = mine;
+                if (shared2) {
+                    store = reduce_tile(r4);
+                } else if (mine) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        r4[i] = (c0[i] + c1[i]) + (c2[i] + c3[i]);
+                        c0[i] = c1[i] = c2[i] = c3[i] = 0.f;
+                    }
+                }
+                if (store) {
                     // rows g and g + 8 of the tile, tokens 2 tig and 2 tig + 1 of the request
                     const int n_rows = min(16, r_hi - r_lo - 16 * blk);
                     float *z0 = p.zbuf + r_lo + 16 * blk + g;
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
-                        const float val = (c0[i] + c1[i]) + (c2[i] + c3[i]);
-                        c0[i] = c1[i] = c2[i] = c3[i] = 0.f;
+                        const float val = r4[i];
                         const int tok = tig * 2 + (i & 1), row = g + (i >> 1) * 8;
                         if (tok < vi.n_tok && row < n_rows)
                             z0[(size_t)((i & 1) ? vi.pair1 : vi.pair0) * d + (i >> 1) * 8] = val;
