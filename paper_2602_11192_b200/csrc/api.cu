@@ -903,11 +903,28 @@ int melinoe_moe_forward_host(melinoe_moe_t *h, void *cuda_stream, const void *hi
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     const size_t bytes = (size_t)T * h->d * 2;
     CU_TRY(cudaMemcpyAsync(h->stage_in, hidden_host, bytes, cudaMemcpyHostToDevice, s));
-    rc = melinoe_moe_forward(h, cuda_stream, h->stage_in, T, h->stage_out, stats_host ? h->stage_stats : nullptr);
+    // A decode-sized result goes straight to page-locked host memory from the kernels that produce it
+    // (a few hundred posted writes) instead of through two more copy-engine operations, each of
+    // which costs the stream several microseconds.  Pageable buffers and large calls are staged.
+    void *out_direct = nullptr, *stats_direct = nullptr;
+    if (T <= kTokPerVr) {
+        cudaPointerAttributes a;
+        if (cudaPointerGetAttributes(&a, out_host) == cudaSuccess && a.type == cudaMemoryTypeHost && a.devicePointer &&
+            aligned16(a.devicePointer))
+            out_direct = a.devicePointer;
+        if (stats_host && cudaPointerGetAttributes(&a, stats_host) == cudaSuccess && a.type == cudaMemoryTypeHost &&
+            a.devicePointer && (reinterpret_cast<uintptr_t>(a.devicePointer) & 7u) == 0)
+            stats_direct = a.devicePointer;
+        (void)cudaGetLastError();
+    }
+    rc = melinoe_moe_forward(h, cuda_stream, h->stage_in, T, out_direct ? out_direct : h->stage_out,
+                             stats_host ? (stats_direct ? static_cast<melinoe_moe_stats *>(stats_direct) : h->stage_stats)
+                                        : nullptr);
     if (rc != MELINOE_OK)
         return rc;
-    CU_TRY(cudaMemcpyAsync(out_host, h->stage_out, bytes, cudaMemcpyDeviceToHost, s));
-    if (stats_host)
+    if (!out_direct)
+        CU_TRY(cudaMemcpyAsync(out_host, h->stage_out, bytes, cudaMemcpyDeviceToHost, s));
+    if (stats_host && !stats_direct)
         CU_TRY(cudaMemcpyAsync(stats_host, h->stage_stats, sizeof(melinoe_moe_stats), cudaMemcpyDeviceToHost, s));
     CU_TRY(cudaEventRecord(h->ev_last, s));
     return MELINOE_OK;

@@ -154,6 +154,15 @@ def test_forward_host_matches_forward_and_is_deterministic():
         assert np.array_equal(hy.numpy().view(np.uint16), a[i])
         assert int(hs[0]) == 0 and int(hs[1]) == 3
         P.cache.call(oracle.route(x, P.w_r, k)[0])
+    # pageable host buffers take the staged route and give the same bits
+    P.gpu.layer.reset_cache()
+    py, ps = np.empty((3, d), np.int16), np.zeros(12, np.int32)
+    for i, x in enumerate(xs):
+        px = np.ascontiguousarray(x.view(np.int16))
+        P.gpu.layer.forward_host(current_stream_ptr(), px, 3, py, ps)
+        torch.cuda.synchronize()
+        assert np.array_equal(py.view(np.uint16), a[i])
+        assert int(ps[0]) == 0 and int(ps[1]) == 3
     P.close()
 
 
