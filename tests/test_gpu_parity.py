@@ -54,6 +54,26 @@ def test_shapes_and_token_counts(d, F, E, k, C):
     P.close()
 
 
+def test_largest_supported_sizes_and_empty_call():
+    """d_model, n_experts and top_k at their limits; T * k = 64 is the largest call the fused
+    decode planner takes, T = 3 already goes through the general kernels; T = 0 is a no-op."""
+    import torch
+    from paper_2602_11192_b200.runner import current_stream_ptr
+    d, F, E, k, C = 8192, 64, 64, 32, 32
+    P = _pair(d, F, E, k, C, seed=41)
+    for step, T in enumerate((1, 2, 3, 9, 1)):
+        P.step(gen.hidden_states(41, 0, "decode", step, T, d), tokens=[0, T - 1] if T > 1 else None)
+    x = torch.zeros((1, d), dtype=torch.int16, device="cuda")
+    y = torch.full((1, d), 7, dtype=torch.int16, device="cuda")
+    before = P.gpu.layer.cache_state()
+    P.gpu.layer.forward(current_stream_ptr(), x, 0, y)
+    torch.cuda.synchronize()
+    assert int(y.min()) == 7 and int(y.max()) == 7          # nothing written
+    after = P.gpu.layer.cache_state()
+    assert np.array_equal(before[0], after[0]) and before[1] == after[1]
+    P.close()
+
+
 def test_full_cache_has_only_compulsory_misses():
     E, k = 8, 2
     P = _pair(256, 64, E, k, E, seed=3)
