@@ -174,6 +174,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ int s_abort;
     __shared__ int s_passed[2];                 // half's h is complete on every CTA
+    __shared__ int s_slot_free[kMaxStages];     // the gate/up phase has let go of the ring slot
     __shared__ __align__(8) uint64_t s_harr[2]; // consumer warps that have stored their part of the half's h
     __shared__ VrRec s_vrs[kVrShared];
 
@@ -209,6 +210,8 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
     if (tid == 0) {
         s_abort = 0;
         s_passed[0] = s_passed[1] = 0;
+        for (int i = 0; i < kMaxStages; ++i)
+            s_slot_free[i] = 0;
         for (int i = 0; i < 2; ++i)
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(harr + 8 * i), "r"(kConsumerWarps));
         for (int i = 0; i < kMaxSub; ++i) {
@@ -267,9 +270,9 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
     const int rb1 = 2 * d, rb2 = 2 * F;                       // row bytes
     const int nk1 = (rb1 + CB1 - 1) / CB1, nk2 = (rb2 + CB2 - 1) / CB2;
     const int n_half = nv >= 2 ? 2 : 1;
-    // The second part is the smaller one: what follows its barrier is exposed, what follows the
-    // first part's barrier is covered by the second part's gate/up rows.
-    const int nvA = n_half == 2 ? nv - (nv + 2) / 4 : nv;     // requests in the first part
+    // Equal parts measured best (OLMoE shape, 8 requests: 5 + 3, 4 + 4 and 3 + 5 within 0.2 us of one
+    // another per launch, 6 + 2 one microsecond slower, 7 + 1 two and a half).
+    const int nvA = n_half == 2 ? nv - nv / 2 : nv;           // requests in the first part
     // f-row ranges, relative to the half's first request (scalars, not arrays: an array indexed by
     // the half would live in local memory)
     const long long rowsA = (long long)nvA * F, rowsB = (long long)(nv - nvA) * F;
@@ -411,10 +414,9 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
         }
         // ---- down: lanes 0..15 W_d rows, 16..23 rows of h.  Two cursors walk the same stage
         // sequence: the weight rows run ahead as far as the ring allows, the h rows of a stage
-        // follow once the grid has finished the h of the stage's half.  A slot stays with the warp
-        // that served it in the gate/up phase: that warp has followed every phase of the slot's
-        // "empty" barrier, so its parity test of the slot's last gate/up use cannot be fooled by
-        // an older phase.
+        // follow once the grid has finished the h of the stage's half.  Sub-stage (slot, sub) belongs
+        // to warp (slot + sub) mod 3 throughout, so the two tiles that share a slot are requested by
+        // two warps side by side (a warp is busy for most of a microsecond with one tile's copies).
         struct Cursor {
             int t, k, blk, v, base_v;
             const char *base;
@@ -457,16 +459,28 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
             // weight rows of as many stages as there are free sub-stages
             while (wn < N2) {
                 const uint32_t bar = down_bar(wd);
-                if ((int)(wd.slot % kProducerWarps) == pw) {
+                if ((int)((wd.slot + wd.sub) % kProducerWarps) == pw) {
                     // free when its previous down-phase use has been consumed, or, on first use, when the
-                    // gate/up phase has let go of the slot for good
+                    // gate/up phase has let go of the slot for good.  Only the warp that served the slot
+                    // in the gate/up phase (it owns sub-stage 0) may read that off the slot's "empty"
+                    // barrier; it tells the owners of the slot's other sub-stages through a flag.
                     int ok = 1;
                     if (lane == 0) {
                         if (wd.use > 0) {
                             ok = mbar_try(empty2 + 8 * bar, (wd.use - 1u) & 1u);
                         } else if (n1 > wd.slot) {
-                            const uint32_t m_last = n1 - 1u - ((n1 - 1u - wd.slot) % S1);
-                            ok = mbar_try(empty1 + 8 * wd.slot, (m_last / S1) & 1u);
+                            if (wd.sub == 0) {
+                                const uint32_t m_last = n1 - 1u - ((n1 - 1u - wd.slot) % S1);
+                                ok = mbar_try(empty1 + 8 * wd.slot, (m_last / S1) & 1u);
+                                if (ok) {
+                                    __threadfence_block();
+                                    *reinterpret_cast<volatile int *>(&s_slot_free[wd.slot]) = 1;
+                                }
+                            } else {
+                                ok = *reinterpret_cast<volatile int *>(&s_slot_free[wd.slot]);
+                                if (ok)
+                                    __threadfence_block();
+                            }
                         }
                     }
                     if (!__shfl_sync(0xffffffffu, ok, 0))
@@ -500,7 +514,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(FfnParams p, Ff
                 }
                 while (on < wn && (oc.t < hi2A ? passedA : passedB)) {
                     const uint32_t bar = down_bar(od);
-                    if ((int)(od.slot % kProducerWarps) == pw) {
+                    if ((int)((od.slot + od.sub) % kProducerWarps) == pw) {
                         const char *src = tile_of(oc);
                         issue(src, full2 + 8 * bar, down_off(od), PITCH2, dst_row2, (size_t)oc.k * CB2, 0, piece2(oc.k), 2);
                     }
