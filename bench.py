@@ -29,7 +29,7 @@ if ROOT not in sys.path:
 # dram__bytes_read.sum + dram__bytes_write.sum of one ffn_stream_kernel launch divided by the launch's
 # algorithmic bytes (8 experts x 12.58 MB), from the ncu capture summarised in
 # profiles/ffn_stream_kernel_olmoe_decode.md; traffic grows in proportion to the experts streamed.
-DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.04
+DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.03
 
 METRIC = "decode tokens/s (OLMoE-shaped, cache-limited)"
 UNIT = "tokens/s"
