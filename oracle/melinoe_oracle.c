@@ -14,6 +14,8 @@
  *                     the cache policy: LRU, or the gamma-discounted count of
  *                     Definition C.1 (gamma = 1 is LFU, gamma -> 0+ reduces to LRU)
  *   miss count        Appendix C.1: number of cache misses = number of transfers
+ *   4-bit store       Section 3.2: experts kept in 4-bit form in host memory (plain symmetric
+ *                     group quantisation here, stated at moe_oracle_quantize_q4)
  *
  * Precision: the routing decision is an integer result, so the logits that decide it are
  * computed in fp32 in one fixed summation order (stated at moe_oracle_logits) that the GPU
@@ -56,6 +58,79 @@ int moe_oracle_threads(void)
 #else
     return 1;
 #endif
+}
+
+/* ---------------------------------------------------------------- 4-bit store --- */
+
+/*
+ * Group-quantised 4-bit experts (Section 3.2: expert weights are "maintained in HQQ INT4"; HQQ's
+ * calibration is a third-party method and is not reproduced: this is plain symmetric
+ * round-to-nearest quantisation, which is all the data path needs).  Reading:
+ *  - a matrix row is cut into groups of 64 consecutive elements (cols % 64 == 0);
+ *  - a group's scale is bf16( max|w| / 7 ), the division in fp32, rounded to nearest even;
+ *  - code = clamp( rint(w / scale), -8, 7 ) + 8 with the division in fp32 and ties to even; a
+ *    group whose scale is zero has code 8 everywhere;
+ *  - the weight the layer computes with is bf16( scale * (code - 8) ), product in fp32 (exact),
+ *    rounded to nearest even.
+ */
+static uint16_t f32_to_bf16_rne(float f)
+{
+    uint32_t u;
+    memcpy(&u, &f, sizeof u);
+    u += 0x7fffu + ((u >> 16) & 1u);
+    return (uint16_t)(u >> 16);
+}
+
+/* w [rows][cols] bf16 bits -> codes [rows][cols / 2] (low nibble = even column), scales [rows][cols / 64] bf16 bits */
+int moe_oracle_quantize_q4(const uint16_t *w, int rows, int cols, uint8_t *codes, uint16_t *scales)
+{
+    if (rows <= 0 || cols <= 0 || cols % 64)
+        return 1;
+    for (int r = 0; r < rows; ++r)
+        for (int g0 = 0; g0 < cols; g0 += 64) {
+            const uint16_t *src = w + (size_t)r * cols + g0;
+            float amax = 0.0f;
+            for (int j = 0; j < 64; ++j) {
+                float a = fabsf(bf16_to_f32(src[j]));
+                if (a > amax)
+                    amax = a;
+            }
+            uint16_t sb = f32_to_bf16_rne(amax / 7.0f);
+            float s = bf16_to_f32(sb);
+            scales[(size_t)r * (cols / 64) + g0 / 64] = sb;
+            for (int j = 0; j < 64; ++j) {
+                int q = 0;
+                if (s > 0.0f) {
+                    float t = rintf(bf16_to_f32(src[j]) / s);
+                    if (t < -8.0f)
+                        t = -8.0f;
+                    if (t > 7.0f)
+                        t = 7.0f;
+                    q = (int)t;
+                }
+                uint8_t c = (uint8_t)(q + 8);
+                uint8_t *dst = codes + ((size_t)r * cols + g0 + j) / 2;
+                if (j & 1)
+                    *dst = (uint8_t)((*dst & 0x0f) | (c << 4));
+                else
+                    *dst = (uint8_t)((*dst & 0xf0) | c);
+            }
+        }
+    return 0;
+}
+
+int moe_oracle_dequantize_q4(const uint8_t *codes, const uint16_t *scales, int rows, int cols, uint16_t *w_out)
+{
+    if (rows <= 0 || cols <= 0 || cols % 64)
+        return 1;
+    for (int r = 0; r < rows; ++r)
+        for (int j = 0; j < cols; ++j) {
+            size_t at = (size_t)r * cols + j;
+            int c = (j & 1) ? (codes[at / 2] >> 4) : (codes[at / 2] & 0x0f);
+            float s = bf16_to_f32(scales[(size_t)r * (cols / 64) + j / 64]);
+            w_out[at] = f32_to_bf16_rne(s * (float)(c - 8));
+        }
+    return 0;
 }
 
 /* ---------------------------------------------------------------- router -------- */

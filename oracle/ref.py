@@ -12,7 +12,7 @@ import numpy as np
 
 from . import build as _build
 
-__all__ = ["threads", "logits", "topk", "route", "gather", "ExpertCache", "ffn_combine", "layer_forward"]
+__all__ = ["threads", "logits", "topk", "route", "gather", "quantize_q4", "dequantize_q4", "ExpertCache", "ffn_combine", "layer_forward"]
 
 _lib = None
 
@@ -41,6 +41,8 @@ def _L():
         lib.moe_oracle_ffn_combine.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                                C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
                                                C.c_void_p, C.c_int, C.c_void_p]
+        lib.moe_oracle_quantize_q4.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p]
+        lib.moe_oracle_dequantize_q4.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p]
         _lib = lib
     return _lib
 
@@ -102,6 +104,28 @@ def gather(idx: np.ndarray, n_experts: int):
     if rc:
         raise ValueError("moe_oracle_gather rc=%d" % rc)
     return counts, offsets, perm
+
+
+def quantize_q4(w) -> Tuple[np.ndarray, np.ndarray]:
+    """w [rows][cols] bf16 bits -> (codes [rows][cols/2] uint8, scales [rows][cols/64] bf16 bits)."""
+    w = _u16(w)
+    rows, cols = w.shape
+    codes = np.zeros((rows, cols // 2), dtype=np.uint8)
+    scales = np.zeros((rows, max(cols // 64, 1)), dtype=np.uint16)
+    if _L().moe_oracle_quantize_q4(_p(w), rows, cols, _p(codes), _p(scales)):
+        raise ValueError("cols must be a positive multiple of 64")
+    return codes, scales
+
+
+def dequantize_q4(codes, scales) -> np.ndarray:
+    """The bf16 weights (bit patterns) the layer computes with for a 4-bit matrix."""
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    scales = _u16(scales)
+    rows, cols = codes.shape[0], codes.shape[1] * 2
+    out = np.empty((rows, cols), dtype=np.uint16)
+    if _L().moe_oracle_dequantize_q4(_p(codes), _p(scales), rows, cols, _p(out)):
+        raise ValueError("cols must be a positive multiple of 64")
+    return out
 
 
 class ExpertCache:

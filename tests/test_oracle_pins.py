@@ -385,6 +385,49 @@ def test_count_policy_preload_gives_the_definitions_initial_counts():
     assert np.allclose(cache.counts()[[2, 9, 4, 7]], [1.9, 1.9, 0.9, 0.9])
 
 
+def test_q4_hand_worked_groups():
+    for g in _gold("q4_groups.json")["groups"]:
+        row = np.zeros(64, np.float32)
+        row[:len(g["head"])] = g["head"]
+        codes, scales = oracle.quantize_q4(_bf16(row)[None, :])
+        assert gen.bf16_bits_to_f32(scales)[0, 0] == g["scale"], g["comment"]
+        nib = np.stack([codes[0] & 15, codes[0] >> 4], axis=1).reshape(-1)
+        n = len(g["head"])
+        assert nib[:n].tolist() == g["codes_head"] and np.all(nib[n:] == 8), g["comment"]
+        deq = gen.bf16_bits_to_f32(oracle.dequantize_q4(codes, scales))[0]
+        assert deq[:n].tolist() == g["dequant_head"] and np.all(deq[n:] == 0.0), g["comment"]
+
+
+def test_q4_error_bound_range_and_grid_points():
+    rs = np.random.default_rng(5)
+    w = _bf16(rs.normal(0.0, 0.02, (24, 256)).astype(np.float32))
+    codes, scales = oracle.quantize_q4(w)
+    wf = gen.bf16_bits_to_f32(w).astype(np.float64)
+    sf = np.repeat(gen.bf16_bits_to_f32(scales).astype(np.float64), 64, axis=1)
+    deq = gen.bf16_bits_to_f32(oracle.dequantize_q4(codes, scales)).astype(np.float64)
+    nib = np.stack([codes & 15, codes >> 4], axis=2).reshape(24, 256).astype(np.int64) - 8
+    assert nib.min() >= -8 and nib.max() <= 7
+    # rounding to the nearest code: half a step, plus half an ulp of bf16 on the product, plus the
+    # clamp at +-7 where the rounded-down scale makes max|w| / scale a little more than 7
+    step_err = np.abs(wf - sf * nib)
+    assert np.all(step_err <= sf * (0.5 + 7 * 2.0 ** -8) + 1e-12)
+    assert np.all(np.abs(deq - sf * nib) <= np.abs(sf * nib) * 2.0 ** -8 + 1e-30)
+    # the largest element of every group sits on the outermost code
+    wg, ng = np.abs(wf).reshape(24, 4, 64), np.abs(nib).reshape(24, 4, 64)
+    assert np.all(np.take_along_axis(ng, wg.argmax(axis=2)[..., None], axis=2) >= 7)
+    # weights that are already scale * integer with a power-of-two scale come back exactly
+    grid = (rs.integers(-7, 8, (6, 128)) * 2.0 ** -6).astype(np.float32)
+    grid[:, 0] = 7 * 2.0 ** -6
+    grid[:, 64] = -7 * 2.0 ** -6
+    c2, s2 = oracle.quantize_q4(_bf16(grid))
+    assert np.array_equal(gen.bf16_bits_to_f32(oracle.dequantize_q4(c2, s2)), grid)
+    # an all-zero group: scale 0, code 8, weight 0
+    c3, s3 = oracle.quantize_q4(np.zeros((2, 64), np.uint16))
+    assert np.all(s3 == 0) and np.all(c3 == 0x88) and np.all(oracle.dequantize_q4(c3, s3) == 0)
+    with pytest.raises(ValueError):
+        oracle.quantize_q4(np.zeros((2, 96), np.uint16))
+
+
 def test_miss_bytes_match_papers_transfer_example():
     g = _gold("transfer_time.json")
     cfg = gen.config_by_name("mixtral")
