@@ -93,6 +93,21 @@ size_t melinoe_moe_expert_bytes(int d_model, int d_ff);
 int melinoe_moe_pack_expert(int d_model, int d_ff, const void *w_gate_host, const void *w_up_host,
                             const void *w_down_host, void *blob_out_host);
 
+/*
+ * 4-bit host store (Section 3.2 keeps the expert weights in 4-bit form; the calibrated HQQ format
+ * of the paper is a third-party method, what is implemented is plain symmetric group
+ * quantisation).  A matrix row is cut into groups of 64 consecutive elements; a group's scale is
+ * bf16(max|w| / 7); code = clamp(rint(w / scale), -8, 7) + 8, ties to even; the weight the layer
+ * computes with is bf16(scale * (code - 8)).  Blob of one expert, `melinoe_moe_expert_bytes_q4`
+ * long (about 1.59 bytes per three weights, 3.76 times smaller than the bf16 blob): for W_g, W_u,
+ * W_d in this order the codes [rows][cols / 2] (even column in the low nibble) then the scales
+ * [rows][cols / 64] bf16.  Needs d_ff % 64 == 0 (else the size is 0 and packing returns
+ * MELINOE_ERR_UNSUPPORTED).  Pure host code.
+ */
+size_t melinoe_moe_expert_bytes_q4(int d_model, int d_ff);
+int melinoe_moe_pack_expert_q4(int d_model, int d_ff, const void *w_gate_host, const void *w_up_host,
+                               const void *w_down_host, void *blob_out_host);
+
 /* Router matrix W_r (Eq. 1): dev pointer, [n_experts][d_model] bf16, 16-byte aligned, borrowed
  * until the handle is destroyed or the router is replaced.  Its contents must not change while a
  * forward call is queued or running (a decode call may read it before the work ahead of it in the
@@ -108,6 +123,18 @@ int melinoe_moe_set_router(melinoe_moe_t *h, const void *w_router_dev);
  */
 int melinoe_moe_register_host_experts(melinoe_moe_t *h, const void *const *expert_host_ptrs,
                                       size_t bytes_per_expert);
+
+/*
+ * Same registration for a store of 4-bit blobs (melinoe_moe_pack_expert_q4): a miss then moves the
+ * 4-bit blob over the host link (3.76 times fewer bytes, which is what a miss costs, Eq. 4) and a
+ * kernel on the handle's copy stream expands it into the bf16 slot behind the copy, so the cache
+ * slots and the compute kernels are the same as with a bf16 store and the layer computes with
+ * exactly the weights the format defines.  The statistics count the bytes that travelled.
+ * Page-locked, 16-byte aligned, borrowed, as above.  Registering one kind of store replaces the
+ * other; the cache should be reset when the store changes.
+ */
+int melinoe_moe_register_host_experts_q4(melinoe_moe_t *h, const void *const *expert_host_ptrs,
+                                         size_t bytes_per_expert);
 
 /* Always-resident shared experts (not in the paper; DeepSeekMoE-style stacks): packed blobs
  * in DEVICE memory, applied to every token with gate 1, never cached, never counted in

@@ -7,7 +7,8 @@ from typing import Optional, Sequence
 
 __all__ = [
     "MelinoeError", "Stats", "Request", "lib", "library_path", "STATUS_NAMES", "MoELayer",
-    "melinoe_moe_expert_bytes", "melinoe_moe_pack_expert", "melinoe_launch_count",
+    "melinoe_moe_expert_bytes", "melinoe_moe_pack_expert", "melinoe_moe_expert_bytes_q4",
+    "melinoe_moe_pack_expert_q4", "melinoe_launch_count",
     "melinoe_last_cuda_error", "melinoe_strerror", "EXPORTED_SYMBOLS",
 ]
 
@@ -21,7 +22,8 @@ EXPORTED_SYMBOLS = [
     "melinoe_moe_last_requests", "melinoe_moe_last_gather", "melinoe_moe_cache_state",
     "melinoe_moe_enable_timing", "melinoe_moe_ffn_time_ms", "melinoe_moe_set_trace", "melinoe_moe_trace_ctas",
     "melinoe_moe_transfer_time_ms", "melinoe_moe_forward_static", "melinoe_moe_static_scratch_bytes",
-    "melinoe_moe_last_call_used_gemm", "melinoe_moe_set_policy", "melinoe_moe_cache_counts", "melinoe_launch_count",
+    "melinoe_moe_last_call_used_gemm", "melinoe_moe_set_policy", "melinoe_moe_cache_counts", "melinoe_moe_expert_bytes_q4",
+    "melinoe_moe_pack_expert_q4", "melinoe_moe_register_host_experts_q4", "melinoe_launch_count",
     "melinoe_last_cuda_error", "melinoe_strerror",
 ]
 
@@ -68,8 +70,12 @@ def lib():
     L.melinoe_moe_expert_bytes.argtypes = [i32, i32]
     L.melinoe_moe_expert_bytes.restype = sz
     L.melinoe_moe_pack_expert.argtypes = [i32, i32, vp, vp, vp, vp]
+    L.melinoe_moe_expert_bytes_q4.argtypes = [i32, i32]
+    L.melinoe_moe_expert_bytes_q4.restype = sz
+    L.melinoe_moe_pack_expert_q4.argtypes = [i32, i32, vp, vp, vp, vp]
     L.melinoe_moe_set_router.argtypes = [vp, vp]
     L.melinoe_moe_register_host_experts.argtypes = [vp, C.POINTER(vp), sz]
+    L.melinoe_moe_register_host_experts_q4.argtypes = [vp, C.POINTER(vp), sz]
     L.melinoe_moe_register_shared_experts.argtypes = [vp, i32, C.POINTER(vp)]
     L.melinoe_moe_set_router_bias.argtypes = [vp, vp, vp, i32]
     L.melinoe_moe_reserve.argtypes = [vp, i32]
@@ -116,6 +122,17 @@ def melinoe_moe_pack_expert(d_model: int, d_ff: int, w_gate_ptr: int, w_up_ptr: 
     rc = lib().melinoe_moe_pack_expert(d_model, d_ff, w_gate_ptr, w_up_ptr, w_down_ptr, blob_ptr)
     if rc:
         raise MelinoeError(rc, "melinoe_moe_pack_expert")
+
+
+def melinoe_moe_expert_bytes_q4(d_model: int, d_ff: int) -> int:
+    return int(lib().melinoe_moe_expert_bytes_q4(d_model, d_ff))
+
+
+def melinoe_moe_pack_expert_q4(d_model: int, d_ff: int, w_gate_ptr: int, w_up_ptr: int, w_down_ptr: int,
+                               blob_ptr: int) -> None:
+    rc = lib().melinoe_moe_pack_expert_q4(d_model, d_ff, w_gate_ptr, w_up_ptr, w_down_ptr, blob_ptr)
+    if rc:
+        raise MelinoeError(rc, "melinoe_moe_pack_expert_q4")
 
 
 def melinoe_launch_count() -> int:
@@ -176,6 +193,12 @@ class MoELayer:
         self._keep["experts"] = keep
         self._ck(lib().melinoe_moe_register_host_experts(self._h, arr, bytes_per_expert),
                  "melinoe_moe_register_host_experts")
+
+    def register_host_experts_q4(self, expert_host_ptrs: Sequence[int], bytes_per_expert: int, keep=None) -> None:
+        arr = (C.c_void_p * len(expert_host_ptrs))(*[int(p) for p in expert_host_ptrs])
+        self._keep["experts"] = keep
+        self._ck(lib().melinoe_moe_register_host_experts_q4(self._h, arr, bytes_per_expert),
+                 "melinoe_moe_register_host_experts_q4")
 
     def register_shared_experts(self, expert_dev_ptrs: Sequence[int], keep=None) -> None:
         n = len(expert_dev_ptrs)

@@ -15,6 +15,7 @@
 
 #include <atomic>
 #include <chrono>
+#include <cmath>
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
@@ -133,6 +134,11 @@ struct melinoe_moe {
     const int32_t *token_seq = nullptr;
     int n_seq = 0, n_shared = 0;
     std::vector<const void *> host_experts;
+    // 4-bit host store (melinoe_moe_register_host_experts_q4): what travels is the 4-bit blob, a
+    // kernel on the copy stream expands it from this staging buffer into the bf16 slot
+    bool store_q4 = false;
+    size_t q4_bytes = 0;
+    char *q4_stage = nullptr;
 
     // page-locked host memory: the miss queue the planning kernel writes
     HostPlan *hplan = nullptr;
@@ -321,6 +327,76 @@ int melinoe_moe_pack_expert(int d, int F, const void *wg_, const void *wu_, cons
     return MELINOE_OK;
 }
 
+size_t melinoe_moe_expert_bytes_q4(int d_model, int d_ff)
+{
+    if (d_model <= 0 || d_ff <= 0 || d_model % 64 != 0 || d_ff % 64 != 0)
+        return 0;
+    const size_t n = (size_t)d_model * (size_t)d_ff;
+    return 3 * (n / 2 + n / 32);
+}
+
+namespace {
+
+float host_bf16_to_f32(uint16_t b)
+{
+    const uint32_t u = (uint32_t)b << 16;
+    float f;
+    std::memcpy(&f, &u, sizeof f);
+    return f;
+}
+
+uint16_t host_f32_to_bf16(float f)
+{
+    uint32_t u;
+    std::memcpy(&u, &f, sizeof u);
+    u += 0x7fffu + ((u >> 16) & 1u);
+    return (uint16_t)(u >> 16);
+}
+
+// One matrix [rows][cols] into its section: codes [rows][cols / 2], then scales [rows][cols / 64].
+void pack_q4_matrix(const uint16_t *w, size_t rows, size_t cols, unsigned char *section)
+{
+    unsigned char *codes = section;
+    uint16_t *scales = reinterpret_cast<uint16_t *>(section + rows * cols / 2);
+    for (size_t r = 0; r < rows; ++r) {
+        for (size_t g = 0; g < cols / 64; ++g) {
+            const uint16_t *src = w + r * cols + g * 64;
+            float amax = 0.0f;
+            for (int j = 0; j < 64; ++j)
+                amax = std::fmax(amax, std::fabs(host_bf16_to_f32(src[j])));
+            const uint16_t sb = host_f32_to_bf16(amax / 7.0f);
+            const float sc = host_bf16_to_f32(sb);
+            scales[r * (cols / 64) + g] = sb;
+            unsigned char *dst = codes + (r * cols + g * 64) / 2;
+            for (int j = 0; j < 64; j += 2) {
+                int q[2] = {0, 0};
+                for (int h2 = 0; h2 < 2; ++h2)
+                    if (sc > 0.0f) {
+                        const float t = std::nearbyint(host_bf16_to_f32(src[j + h2]) / sc);   // ties to even
+                        q[h2] = (int)std::fmin(7.0f, std::fmax(-8.0f, t));
+                    }
+                dst[j / 2] = (unsigned char)((q[0] + 8) | ((q[1] + 8) << 4));
+            }
+        }
+    }
+}
+
+}  // namespace
+
+int melinoe_moe_pack_expert_q4(int d, int F, const void *wg_, const void *wu_, const void *wd_, void *blob_)
+{
+    if (d <= 0 || F <= 0 || !wg_ || !wu_ || !wd_ || !blob_)
+        return MELINOE_ERR_INVALID;
+    if (melinoe_moe_expert_bytes_q4(d, F) == 0)
+        return MELINOE_ERR_UNSUPPORTED;
+    const size_t n = (size_t)d * F, sec = n / 2 + n / 32;
+    unsigned char *blob = static_cast<unsigned char *>(blob_);
+    pack_q4_matrix(static_cast<const uint16_t *>(wg_), (size_t)F, (size_t)d, blob);
+    pack_q4_matrix(static_cast<const uint16_t *>(wu_), (size_t)F, (size_t)d, blob + sec);
+    pack_q4_matrix(static_cast<const uint16_t *>(wd_), (size_t)d, (size_t)F, blob + 2 * sec);
+    return MELINOE_OK;
+}
+
 int melinoe_moe_create(int d, int F, int E, int k, int C, melinoe_moe_t **out)
 {
     if (!out)
@@ -422,6 +498,7 @@ int melinoe_moe_destroy(melinoe_moe_t *h)
     cudaFree(h->plan);
     cudaFree(h->err_word);
     cudaFree(h->sync);
+    cudaFree(h->q4_stage);
     cudaFree(h->shared_dev);
     cudaFree(h->maps_dev);
     cudaFree(h->stage_stats);
@@ -485,6 +562,39 @@ int melinoe_moe_register_host_experts(melinoe_moe_t *h, const void *const *ptrs,
         return rc;
     for (int e = 0; e < h->E; ++e)
         h->host_experts[e] = ptrs[e];
+    h->store_q4 = false;
+    return MELINOE_OK;
+}
+
+int melinoe_moe_register_host_experts_q4(melinoe_moe_t *h, const void *const *ptrs, size_t bytes_per_expert)
+{
+    if (!h || !ptrs)
+        return MELINOE_ERR_INVALID;
+    const size_t qb = melinoe_moe_expert_bytes_q4(h->d, h->F);
+    if (qb == 0)
+        return MELINOE_ERR_UNSUPPORTED;
+    if (bytes_per_expert != qb)
+        return MELINOE_ERR_INVALID;
+    for (int e = 0; e < h->E; ++e) {
+        cudaPointerAttributes a;
+        if (!ptrs[e] || !aligned16(ptrs[e]) || cudaPointerGetAttributes(&a, ptrs[e]) != cudaSuccess ||
+            a.type != cudaMemoryTypeHost) {
+            (void)cudaGetLastError();
+            return MELINOE_ERR_INVALID;
+        }
+    }
+    int rc = wait_idle(h);
+    if (rc != MELINOE_OK)
+        return rc;
+    if (!h->q4_stage) {
+        const cudaError_t e = cudaMalloc(&h->q4_stage, qb);
+        if (e != cudaSuccess)
+            return cuda_fail(e);
+    }
+    for (int e = 0; e < h->E; ++e)
+        h->host_experts[e] = ptrs[e];
+    h->store_q4 = true;
+    h->q4_bytes = qb;
     return MELINOE_OK;
 }
 
@@ -580,7 +690,7 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
     pp.policy = h->policy;
     pp.gamma = h->gamma;
     pp.stats = stats_dev;
-    pp.expert_bytes = h->expert_bytes;
+    pp.expert_bytes = h->store_q4 ? h->q4_bytes : h->expert_bytes;   // bytes one miss moves over the host link
     pp.vr_capacity = h->vr_capacity;
     if (route_plan_small_supported(T, h->k, h->d)) {
         CU_TRY(launch_route_plan_small(s, static_cast<const uint16_t *>(hidden_dev), h->w_router, h->bias, h->token_seq,
@@ -737,9 +847,17 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
                 wave_started = true;
             }
             if (h->timing)
-                h->timed_copy_bytes += h->expert_bytes;
-            CU_TRY(cudaMemcpyAsync(h->slots + (size_t)m.slot * h->slot_stride, h->host_experts[m.expert],
-                                   h->expert_bytes, cudaMemcpyHostToDevice, h->copy_stream));
+                h->timed_copy_bytes += h->store_q4 ? h->q4_bytes : h->expert_bytes;
+            if (h->store_q4) {
+                // the 4-bit blob travels; the copy stream expands it into the slot behind the copy
+                CU_TRY(cudaMemcpyAsync(h->q4_stage, h->host_experts[m.expert], h->q4_bytes, cudaMemcpyHostToDevice,
+                                       h->copy_stream));
+                CU_TRY(launch_dequant_q4(h->copy_stream, h->q4_stage, h->slots + (size_t)m.slot * h->slot_stride, h->d,
+                                         h->F, h->n_sms));
+            } else {
+                CU_TRY(cudaMemcpyAsync(h->slots + (size_t)m.slot * h->slot_stride, h->host_experts[m.expert],
+                                       h->expert_bytes, cudaMemcpyHostToDevice, h->copy_stream));
+            }
         }
         if (wave_started) {
             CU_TRY(cudaEventRecord(ctp.b, h->copy_stream));
@@ -1014,8 +1132,15 @@ int melinoe_moe_preload(melinoe_moe_t *h, const int32_t *ids, int n)
             c.slot_of_expert[c.expert_of_slot[victim]] = -1;
             c.tot_evictions += 1;
         }
-        CU_TRY(cudaMemcpy(h->slots + (size_t)victim * h->slot_stride, h->host_experts[e], h->expert_bytes,
-                          cudaMemcpyHostToDevice));
+        if (h->store_q4) {
+            CU_TRY(cudaMemcpyAsync(h->q4_stage, h->host_experts[e], h->q4_bytes, cudaMemcpyHostToDevice, h->copy_stream));
+            CU_TRY(launch_dequant_q4(h->copy_stream, h->q4_stage, h->slots + (size_t)victim * h->slot_stride, h->d, h->F,
+                                     h->n_sms));
+            CU_TRY(cudaStreamSynchronize(h->copy_stream));
+        } else {
+            CU_TRY(cudaMemcpy(h->slots + (size_t)victim * h->slot_stride, h->host_experts[e], h->expert_bytes,
+                              cudaMemcpyHostToDevice));
+        }
         c.expert_of_slot[victim] = e;
         c.slot_of_expert[e] = victim;
         c.stamp[victim] = st;

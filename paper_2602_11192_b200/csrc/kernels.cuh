@@ -101,4 +101,7 @@ cudaError_t launch_ffn_gemm(cudaStream_t stream, int phase, int n_sms, const Gem
 cudaError_t launch_combine_rows(cudaStream_t stream, const DevPlan *plan, const float *gate, const int32_t *inv_pos,
                                 const float *zs, uint16_t *out, int T, int d, int k, int n_shared, int n_sms);
 
+// ---- 4-bit host store: expand one 4-bit expert (layout in dequant.cu) into a bf16 slot
+cudaError_t launch_dequant_q4(cudaStream_t stream, const void *q4_blob, void *slot, int d, int F, int n_sms);
+
 }  // namespace melinoe

@@ -70,6 +70,19 @@ class LayerSetup:
             self.layer.register_shared_experts([sb + s * self.expert_bytes for s in range(self.n_shared)],
                                                keep=self.shared_store)
 
+    def set_experts_q4(self, experts: Sequence[Tuple]) -> None:
+        """experts[e] = (W_g, W_u, W_d) numpy uint16 (bf16 bits): quantised into a 4-bit pinned store."""
+        assert len(experts) == self.E
+        qb = B.melinoe_moe_expert_bytes_q4(self.d, self.F)
+        assert qb > 0, "the 4-bit store needs d_ff % 64 == 0"
+        self.store_q4 = torch.empty((self.E, qb), dtype=torch.uint8, pin_memory=True)
+        base = self.store_q4.data_ptr()
+        for e, (wg, wu, wd) in enumerate(experts):
+            a = [np.ascontiguousarray(m) for m in (wg, wu, wd)]
+            B.melinoe_moe_pack_expert_q4(self.d, self.F, a[0].ctypes.data, a[1].ctypes.data, a[2].ctypes.data,
+                                         base + e * qb)
+        self.layer.register_host_experts_q4([base + e * qb for e in range(self.E)], qb, keep=self.store_q4)
+
     def set_experts_stacked(self, wg: torch.Tensor, wu: torch.Tensor, wd: torch.Tensor, threads: int = 8) -> None:
         """Whole layer at once: wg/wu [E][F][d], wd [E][d][F] bf16 CPU tensors."""
         base = self.store.data_ptr()
@@ -81,6 +94,20 @@ class LayerSetup:
         with cf.ThreadPoolExecutor(max_workers=threads) as ex:
             list(ex.map(one, range(self.E)))
         self.layer.register_host_experts([base + e * eb for e in range(self.E)], eb, keep=self.store)
+
+    def set_experts_stacked_q4(self, wg: torch.Tensor, wu: torch.Tensor, wd: torch.Tensor, threads: int = 8) -> None:
+        """Whole layer at once into a 4-bit pinned store: wg/wu [E][F][d], wd [E][d][F] bf16 CPU tensors."""
+        qb = B.melinoe_moe_expert_bytes_q4(self.d, self.F)
+        assert qb > 0, "the 4-bit store needs d_ff % 64 == 0"
+        self.store_q4 = torch.empty((self.E, qb), dtype=torch.uint8, pin_memory=True)
+        base = self.store_q4.data_ptr()
+
+        def one(e):
+            B.melinoe_moe_pack_expert_q4(self.d, self.F, wg[e].data_ptr(), wu[e].data_ptr(), wd[e].data_ptr(),
+                                         base + e * qb)
+        with cf.ThreadPoolExecutor(max_workers=threads) as ex:
+            list(ex.map(one, range(self.E)))
+        self.layer.register_host_experts_q4([base + e * qb for e in range(self.E)], qb, keep=self.store_q4)
 
     def set_shared_stacked(self, wg: torch.Tensor, wu: torch.Tensor, wd: torch.Tensor) -> None:
         """Shared experts of the layer: wg/wu [n_shared][F][d], wd [n_shared][d][F] bf16 CPU tensors."""

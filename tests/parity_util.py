@@ -26,13 +26,23 @@ def rel_err_per_token(y_gpu_bits: np.ndarray, y_ref: np.ndarray) -> np.ndarray:
 class Pair:
     """The CUDA layer and the oracle side by side on identical weights."""
 
-    def __init__(self, d, F, E, k, C, seed=0, layer=0, n_shared=0):
+    def __init__(self, d, F, E, k, C, seed=0, layer=0, n_shared=0, store="bf16"):
         from paper_2602_11192_b200.runner import LayerSetup
+        from paper_2602_11192_b200 import melinoe_moe_expert_bytes_q4
         self.d, self.F, self.E, self.k, self.C, self.n_shared = d, F, E, k, C, n_shared
         self.weights = make_weights(seed, layer, E, d, F, n_shared)
         self.w_r = gen.router_weights(seed, layer, E, d)
         self.gpu = LayerSetup(d, F, E, k, C, n_shared)
-        self.gpu.set_experts(self.weights[:E], self.weights[E:])
+        self.bytes_per_miss = 3 * d * F * 2
+        if store == "q4":
+            # the library quantises the original weights; the oracle computes with what the 4-bit
+            # format defines as the layer's weights (its own quantise + dequantise)
+            assert n_shared == 0
+            self.gpu.set_experts_q4(self.weights)
+            self.weights = [tuple(oracle.dequantize_q4(*oracle.quantize_q4(m)) for m in w) for w in self.weights]
+            self.bytes_per_miss = melinoe_moe_expert_bytes_q4(d, F)
+        else:
+            self.gpu.set_experts(self.weights[:E], self.weights[E:])
         self.gpu.set_router(self.w_r)
         self.cache = oracle.ExpertCache(C, E)
         self.bias = None
@@ -83,7 +93,7 @@ class Pair:
         assert st["status"] == 0 and st["n_tokens"] == T and st["n_distinct"] == len(req_o)
         assert st["hits"] == int(req_o[:, 2].sum()) and st["misses"] == len(req_o) - int(req_o[:, 2].sum())
         assert st["evictions"] == int((req_o[:, 3] >= 0).sum())
-        assert st["bytes_h2d"] == st["misses"] * 3 * self.d * self.F * 2
+        assert st["bytes_h2d"] == st["misses"] * self.bytes_per_miss
         out = {"idx": idx_o, "gate": gate_o, "req": req_o, "stats": st}
         if check_y:
             y_ref = oracle.ffn_combine(x_bits, idx_o, gate_o, self.weights, self.F, self.n_shared, tokens)

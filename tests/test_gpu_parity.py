@@ -237,6 +237,36 @@ def test_count_policy_preload_and_lfu_keeps_the_hot_experts():
     P.close()
 
 
+def test_q4_host_store_matches_the_oracle_and_a_bf16_store_of_the_same_weights():
+    """4-bit host store: the misses move 4-bit blobs, the layer computes with the weights the format
+    defines.  Against the oracle on its own dequantised weights (tolerance), and bit for bit against
+    a second layer whose bf16 store holds those dequantised weights."""
+    from paper_2602_11192_b200.runner import LayerSetup
+    d, F, E, k, C = 512, 128, 12, 2, 4
+    P = _pair(d, F, E, k, C, seed=51, store="q4")
+    assert P.bytes_per_miss == 3 * (d * F // 2 + d * F // 32)
+    ref = LayerSetup(d, F, E, k, C)
+    ref.set_experts(P.weights, [])
+    ref.set_router(P.w_r)
+    n_miss = 0
+    for step, T in enumerate((1, 2, 8, 1, 20, 3, 1, 1)):
+        x = gen.hidden_states(51, 0, "decode", step, T, d)
+        res, out = P.step(x)
+        n_miss += out["stats"]["misses"]
+        assert np.array_equal(res["out_bits"], ref.forward_np(x)["out_bits"])
+    assert n_miss > 10
+    # preload goes through the same expansion
+    P.reset()
+    ref.layer.reset_cache()
+    P.preload([3, 7])
+    ref.layer.preload(np.array([3, 7], np.int32))
+    x = gen.hidden_states(51, 0, "decode", 99, 4, d)
+    res, _ = P.step(x)
+    assert np.array_equal(res["out_bits"], ref.forward_np(x)["out_bits"])
+    ref.close()
+    P.close()
+
+
 def test_argument_and_state_errors():
     import torch
     from paper_2602_11192_b200 import MoELayer, MelinoeError, melinoe_moe_expert_bytes

@@ -48,6 +48,30 @@ def test_pack_expert_layout(m):
         m.melinoe_moe_pack_expert(d, F, 0, wu.ctypes.data, wd.ctypes.data, blob.ctypes.data)
 
 
+def test_pack_expert_q4_matches_the_oracle_bit_for_bit(m):
+    """The library's host-side quantiser against the oracle's (independent code, same definition)."""
+    import oracle
+    d, F = 256, 128
+    rs = np.random.default_rng(3)
+    w = [gen.f32_to_bf16_bits(rs.normal(0.0, 0.02, shp).astype(np.float32)) for shp in ((F, d), (F, d), (d, F))]
+    w[0][0, :64] = 0                                            # an all-zero group
+    w[1][1, :8] = gen.f32_to_bf16_bits(np.array([0.875, -0.875, 0.0625, 0.1875, -0.0625, -0.1875, 0.125, 0.0], np.float32))
+    w[1][1, 8:64] = 0                                           # ties exactly between two codes
+    qb = m.melinoe_moe_expert_bytes_q4(d, F)
+    assert qb == 3 * (d * F // 2 + d * F // 32)
+    assert m.melinoe_moe_expert_bytes_q4(256, 40) == 0
+    blob = np.full(qb, 0xAB, np.uint8)
+    m.melinoe_moe_pack_expert_q4(d, F, w[0].ctypes.data, w[1].ctypes.data, w[2].ctypes.data, blob.ctypes.data)
+    sec = d * F // 2 + d * F // 32
+    for i, mat in enumerate(w):
+        codes, scales = oracle.quantize_q4(mat)
+        part = blob[i * sec:(i + 1) * sec]
+        assert np.array_equal(part[:d * F // 2], codes.reshape(-1))
+        assert np.array_equal(part[d * F // 2:].view(np.uint16), scales.reshape(-1))
+    with pytest.raises(m.MelinoeError):
+        m.melinoe_moe_pack_expert_q4(256, 40, w[0].ctypes.data, w[1].ctypes.data, w[2].ctypes.data, blob.ctypes.data)
+
+
 def test_create_fails_loudly_without_a_device(m):
     import torch
     if torch.cuda.is_available():
