@@ -33,7 +33,7 @@ class Stack:
     """
 
     def __init__(self, cfg: gen.MoEConfig, alpha: float, cache_slots: int, n_layers: Optional[int] = None,
-                 verbose: bool = False, policy: str = "lru", gamma: float = 0.0):
+                 verbose: bool = False, policy: str = "lru", gamma: float = 0.0, store: str = "bf16"):
         self.cfg, self.alpha, self.C = cfg, float(alpha), int(cache_slots)
         self.L = cfg.n_layers if n_layers is None else int(n_layers)
         self.layers: List[LayerSetup] = []
@@ -43,7 +43,10 @@ class Stack:
         for l in range(self.L):
             ls = LayerSetup(cfg.d_model, cfg.d_ff, cfg.n_experts, cfg.top_k, self.C, cfg.n_shared)
             wg, wu, wd = gen.fill_expert_store_fast(cfg.seed, l, cfg.n_experts + cfg.n_shared, cfg.d_model, cfg.d_ff)
-            ls.set_experts_stacked(wg[:cfg.n_experts], wu[:cfg.n_experts], wd[:cfg.n_experts])
+            if store == "q4":
+                ls.set_experts_stacked_q4(wg[:cfg.n_experts], wu[:cfg.n_experts], wd[:cfg.n_experts])
+            else:
+                ls.set_experts_stacked(wg[:cfg.n_experts], wu[:cfg.n_experts], wd[:cfg.n_experts])
             if cfg.n_shared:
                 ls.set_shared_stacked(wg[cfg.n_experts:], wu[cfg.n_experts:], wd[cfg.n_experts:])
             del wg, wu, wd
