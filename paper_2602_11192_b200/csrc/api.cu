@@ -138,7 +138,11 @@ struct melinoe_moe {
     // kernel on the copy stream expands it from this staging buffer into the bf16 slot
     bool store_q4 = false;
     size_t q4_bytes = 0;
-    char *q4_stage = nullptr;
+    char *q4_stage = nullptr;              // two staging buffers of q4_bytes, used alternately
+    cudaStream_t dq_stream = nullptr;      // runs the expansion kernels, so the link does not wait for them
+    cudaEvent_t ev_q4_copied[2] = {nullptr, nullptr}, ev_q4_expanded[2] = {nullptr, nullptr};
+    unsigned q4_turn = 0;                  // staging buffer of the next miss
+    bool q4_used[2] = {false, false};
 
     // page-locked host memory: the miss queue the planning kernel writes
     HostPlan *hplan = nullptr;
@@ -211,6 +215,8 @@ int wait_idle(melinoe_moe *h)
     if (h->has_last)
         CU_TRY(cudaEventSynchronize(h->ev_last));
     CU_TRY(cudaStreamSynchronize(h->copy_stream));
+    if (h->dq_stream)
+        CU_TRY(cudaStreamSynchronize(h->dq_stream));
     return MELINOE_OK;
 }
 
@@ -499,6 +505,14 @@ int melinoe_moe_destroy(melinoe_moe_t *h)
     cudaFree(h->err_word);
     cudaFree(h->sync);
     cudaFree(h->q4_stage);
+    if (h->dq_stream)
+        cudaStreamDestroy(h->dq_stream);
+    for (int i = 0; i < 2; ++i) {
+        if (h->ev_q4_copied[i])
+            cudaEventDestroy(h->ev_q4_copied[i]);
+        if (h->ev_q4_expanded[i])
+            cudaEventDestroy(h->ev_q4_expanded[i]);
+    }
     cudaFree(h->shared_dev);
     cudaFree(h->maps_dev);
     cudaFree(h->stage_stats);
@@ -587,9 +601,12 @@ int melinoe_moe_register_host_experts_q4(melinoe_moe_t *h, const void *const *pt
     if (rc != MELINOE_OK)
         return rc;
     if (!h->q4_stage) {
-        const cudaError_t e = cudaMalloc(&h->q4_stage, qb);
-        if (e != cudaSuccess)
-            return cuda_fail(e);
+        CU_TRY(cudaMalloc(&h->q4_stage, 2 * qb));
+        CU_TRY(cudaStreamCreateWithFlags(&h->dq_stream, cudaStreamNonBlocking));
+        for (int i = 0; i < 2; ++i) {
+            CU_TRY(cudaEventCreateWithFlags(&h->ev_q4_copied[i], cudaEventDisableTiming));
+            CU_TRY(cudaEventCreateWithFlags(&h->ev_q4_expanded[i], cudaEventDisableTiming));
+        }
     }
     for (int e = 0; e < h->E; ++e)
         h->host_experts[e] = ptrs[e];
@@ -833,8 +850,11 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
                 h->sticky.store(MELINOE_ERR_STATE);
                 return MELINOE_ERR_STATE;
             }
-            if (m.dep_group >= 0)  // the slot still feeds an earlier compute group of this call
-                CU_TRY(cudaStreamWaitEvent(h->copy_stream, h->ev_group[m.dep_group], 0));
+            // the slot may still feed an earlier compute group of this call: whoever writes the slot
+            // (the copy itself, or the expansion kernel of a 4-bit store) waits for that group
+            cudaStream_t slot_writer = h->store_q4 ? h->dq_stream : h->copy_stream;
+            if (m.dep_group >= 0)
+                CU_TRY(cudaStreamWaitEvent(slot_writer, h->ev_group[m.dep_group], 0));
             if (h->timing && !wave_started) {
                 if (!h->free_pairs.empty()) {
                     ctp = h->free_pairs.back();
@@ -849,11 +869,20 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
             if (h->timing)
                 h->timed_copy_bytes += h->store_q4 ? h->q4_bytes : h->expert_bytes;
             if (h->store_q4) {
-                // the 4-bit blob travels; the copy stream expands it into the slot behind the copy
-                CU_TRY(cudaMemcpyAsync(h->q4_stage, h->host_experts[m.expert], h->q4_bytes, cudaMemcpyHostToDevice,
+                // the 4-bit blob travels into one of two staging buffers; a kernel on a stream of its own
+                // expands it into the slot, so the next blob is on the link meanwhile
+                const unsigned b = h->q4_turn++ & 1u;
+                char *stage = h->q4_stage + (size_t)b * h->q4_bytes;
+                if (h->q4_used[b])
+                    CU_TRY(cudaStreamWaitEvent(h->copy_stream, h->ev_q4_expanded[b], 0));
+                CU_TRY(cudaMemcpyAsync(stage, h->host_experts[m.expert], h->q4_bytes, cudaMemcpyHostToDevice,
                                        h->copy_stream));
-                CU_TRY(launch_dequant_q4(h->copy_stream, h->q4_stage, h->slots + (size_t)m.slot * h->slot_stride, h->d,
-                                         h->F, h->n_sms));
+                CU_TRY(cudaEventRecord(h->ev_q4_copied[b], h->copy_stream));
+                CU_TRY(cudaStreamWaitEvent(h->dq_stream, h->ev_q4_copied[b], 0));
+                CU_TRY(launch_dequant_q4(h->dq_stream, stage, h->slots + (size_t)m.slot * h->slot_stride, h->d, h->F,
+                                         h->n_sms));
+                CU_TRY(cudaEventRecord(h->ev_q4_expanded[b], h->dq_stream));
+                h->q4_used[b] = true;
             } else {
                 CU_TRY(cudaMemcpyAsync(h->slots + (size_t)m.slot * h->slot_stride, h->host_experts[m.expert],
                                        h->expert_bytes, cudaMemcpyHostToDevice, h->copy_stream));
@@ -863,7 +892,7 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
             CU_TRY(cudaEventRecord(ctp.b, h->copy_stream));
             h->timed_copy.push_back(ctp);
         }
-        CU_TRY(cudaEventRecord(h->ev_arrive, h->copy_stream));
+        CU_TRY(cudaEventRecord(h->ev_arrive, h->store_q4 ? h->dq_stream : h->copy_stream));
         CU_TRY(cudaStreamWaitEvent(s, h->ev_arrive, 0));
         rc = launch_group(g);
         if (rc != MELINOE_OK)
@@ -1133,10 +1162,11 @@ int melinoe_moe_preload(melinoe_moe_t *h, const int32_t *ids, int n)
             c.tot_evictions += 1;
         }
         if (h->store_q4) {
-            CU_TRY(cudaMemcpyAsync(h->q4_stage, h->host_experts[e], h->q4_bytes, cudaMemcpyHostToDevice, h->copy_stream));
-            CU_TRY(launch_dequant_q4(h->copy_stream, h->q4_stage, h->slots + (size_t)victim * h->slot_stride, h->d, h->F,
+            // the handle is idle (wait_idle above): stage, expand, wait
+            CU_TRY(cudaMemcpy(h->q4_stage, h->host_experts[e], h->q4_bytes, cudaMemcpyHostToDevice));
+            CU_TRY(launch_dequant_q4(h->dq_stream, h->q4_stage, h->slots + (size_t)victim * h->slot_stride, h->d, h->F,
                                      h->n_sms));
-            CU_TRY(cudaStreamSynchronize(h->copy_stream));
+            CU_TRY(cudaStreamSynchronize(h->dq_stream));
         } else {
             CU_TRY(cudaMemcpy(h->slots + (size_t)victim * h->slot_stride, h->host_experts[e], h->expert_bytes,
                               cudaMemcpyHostToDevice));
