@@ -267,6 +267,28 @@ def test_q4_host_store_matches_the_oracle_and_a_bf16_store_of_the_same_weights()
     P.close()
 
 
+def test_parity_without_programmatic_launch():
+    """The decode kernels are launched with programmatic stream serialisation by default; the
+    same parity must hold with the attribute switched off (the switch is read once per process,
+    hence the child process)."""
+    import os
+    import subprocess
+    import sys
+    here = os.path.dirname(os.path.abspath(__file__))
+    code = (
+        "import sys; sys.path.insert(0, %r); sys.path.insert(0, %r)\n"
+        "import numpy as np, gen\n"
+        "from parity_util import Pair\n"
+        "P = Pair(512, 64, 16, 2, 4, seed=61)\n"
+        "for step, T in enumerate((1, 4, 1, 8, 2, 1, 12, 1)):\n"
+        "    P.step(gen.hidden_states(61, 0, 'decode', step, T, 512))\n"
+        "P.close()\n"
+        "print('child ok')\n" % (os.path.dirname(here), here))
+    env = dict(os.environ, MELINOE_MOE_NO_PDL="1")
+    r = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0 and "child ok" in r.stdout, r.stdout[-2000:] + r.stderr[-2000:]
+
+
 def test_argument_and_state_errors():
     import torch
     from paper_2602_11192_b200 import MoELayer, MelinoeError, melinoe_moe_expert_bytes
