@@ -367,6 +367,14 @@ def run_ours(args):
                 extra["store=q4,alpha=%g" % a] = dict(value=cfg.batch * K / (ms_q * 1e-3), **hit_summary(st_q))
                 extra["store=q4,alpha=%g" % a]["h2d_expert_bytes_per_step"] = (
                     float(st_q["misses"].sum()) * M.melinoe_moe_expert_bytes_q4(cfg.d_model, cfg.d_ff) / K)
+            # the paper's own serving configuration: 4-bit experts and an LFU cache
+            phase("4-bit host store with the LFU policy")
+            stack.set_policy("count", 1.0)
+            ms_q, _, st_q, _, _ = timed_device(alpha0)
+            extra["store=q4,policy=lfu"] = dict(value=cfg.batch * K / (ms_q * 1e-3), **hit_summary(st_q))
+            extra["store=q4,policy=lfu"]["h2d_expert_bytes_per_step"] = (
+                float(st_q["misses"].sum()) * M.melinoe_moe_expert_bytes_q4(cfg.d_model, cfg.d_ff) / K)
+            stack.set_policy("lru")
         # everything resident (cache = all experts, warm): the FFN kernel without the miss path
         phase("all experts resident")
         stack.close()
