@@ -9,8 +9,9 @@
 //     flight at once, the router row already before the kernel ahead in the stream has finished;
 //   - the logits go straight into the shared memory of the cluster's first CTA and the cluster
 //     barrier tells it when they are all there: no fence, no device counter, no second launch;
-//   - top-k is a rank count (an element's rank is the number of elements that beat it), one warp
-//     per token, instead of k rounds of a warp-wide maximum;
+//   - top-k is a rank count (an element's rank is the number of elements that beat it) shared by
+//     the eight warps, instead of k rounds of a warp-wide maximum; the gates are computed by the
+//     other warps while the first one plans;
 //   - planning is written for one warp with lane = expert / slot / request: ranks come from
 //     ballots and population counts, prefix sums from shuffles, and the LRU victims of a call are
 //     taken from one sorted list instead of one search per miss.
@@ -89,6 +90,7 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
     __shared__ __align__(16) float s_logit[kMaxT][kMaxExperts];
     __shared__ int32_t s_cnt[2][kMaxExperts];                    // pairs of an expert among pairs 0..31 / 32..63
     __shared__ int32_t s_tok[kMaxPairs];                         // token of a pair
+    __shared__ int32_t s_rank[kMaxT][kMaxExperts];               // rank of an expert among a token's logits
     // count policy only: live slot table during the call's misses, counts, groups
     __shared__ int32_t s_live_occ[kMaxExperts];
     __shared__ unsigned long long s_live_stamp[kMaxExperts];
@@ -216,6 +218,9 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
         }
     }
     // ---- the cluster's first CTA carries on when every logit has arrived
+    if (cta_rank == 0)
+        for (int i = tid; i < kMaxT * kMaxExperts; i += kThreads)
+            (&s_rank[0][0])[i] = 0;
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     if (cta_rank != 0)
         return;
@@ -223,49 +228,66 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
     for (int i = tid; i < 2 * (kMaxGroups + 1); i += kThreads)
         p.sync[i] = 0u;
 
-    // ================================================================ top-k and gates: a warp per token
-    // An element's rank is the number of elements that beat it (greater, or equal with a lower index).
-    for (int t = warp; t < T; t += kWarpsPerBlock) {
+    // ================================================================ top-k
+    // An element's rank is the number of elements that beat it (greater, or equal with a lower
+    // index).  The eight warps share the count (warp w compares against elements 8w .. 8w + 7 of
+    // every token) and add their parts up in shared memory; then warp t writes token t's selection.
+    // Only the indices are on the way to the planner: the gates are left to the other warps.
+    {
         const float NEG = -__int_as_float(0x7f800000);  // -inf
-        const float v0 = lane < E ? s_logit[t][lane] : NEG;
-        const float v1 = lane + 32 < E ? s_logit[t][lane + 32] : NEG;
-        int r0 = 0, r1 = 0;
-        const float4 *row = reinterpret_cast<const float4 *>(s_logit[t]);
+        for (int t = 0; t < T; ++t) {
+            const float v0 = lane < E ? s_logit[t][lane] : NEG;
+            const float v1 = lane + 32 < E ? s_logit[t][lane + 32] : NEG;
+            int r0 = 0, r1 = 0;
+            const float4 *row = reinterpret_cast<const float4 *>(s_logit[t]) + 2 * warp;
 #pragma unroll
-        for (int i = 0; i < kMaxExperts / 4; ++i) {
-            const float4 o4 = row[i];
-            const float ov[4] = {o4.x, o4.y, o4.z, o4.w};
+            for (int i = 0; i < 2; ++i) {
+                const float4 o4 = row[i];
+                const float ov[4] = {o4.x, o4.y, o4.z, o4.w};
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                const int e = 4 * i + c;
-                const float o = e < E ? ov[c] : NEG;     // the row's tail beyond E was never written
-                r0 += (o > v0) || (o == v0 && e < lane);
-                r1 += (o > v1) || (o == v1 && e < lane + 32);
+                for (int c = 0; c < 4; ++c) {
+                    const int e = 8 * warp + 4 * i + c;
+                    const float o = e < E ? ov[c] : NEG;     // the row's tail beyond E was never written
+                    r0 += (o > v0) || (o == v0 && e < lane);
+                    r1 += (o > v1) || (o == v1 && e < lane + 32);
+                }
+            }
+            if (r0)
+                atomicAdd(&s_rank[t][lane], r0);
+            if (r1)
+                atomicAdd(&s_rank[t][lane + 32], r1);
+        }
+        __syncthreads();
+        if (warp < T) {
+            const int t = warp;
+            const int r0 = s_rank[t][lane], r1 = s_rank[t][lane + 32];
+            if (lane < E && r0 < k) {
+                s_sel[t][r0] = s_logit[t][lane];
+                s_idx[t * k + r0] = lane;
+            }
+            if (lane + 32 < E && r1 < k) {
+                s_sel[t][r1] = s_logit[t][lane + 32];
+                s_idx[t * k + r1] = lane + 32;
             }
         }
-        if (lane < E && r0 < k) {
-            s_sel[t][r0] = v0;
-            s_idx[t * k + r0] = lane;
-        }
-        if (lane + 32 < E && r1 < k) {
-            s_sel[t][r1] = v1;
-            s_idx[t * k + r1] = lane + 32;
-        }
-        __syncwarp();
-        const float top = s_sel[t][0];
-        const float ev = lane < k ? expf(s_sel[t][lane] - top) : 0.0f;
-        float sum = ev;
-#pragma unroll
-        for (int m = 16; m >= 1; m >>= 1)
-            sum += __shfl_xor_sync(0xffffffffu, sum, m);
-        if (lane < k) {
-            idx_out[(size_t)t * k + lane] = s_idx[t * k + lane];
-            gate_out[(size_t)t * k + lane] = ev / sum;
-        }
+        __syncthreads();
     }
-    __syncthreads();
-    if (warp != 0)
+    if (warp != 0) {
+        // ============================================================ gates (Eq. 1), off the planner's path
+        for (int t = warp - 1; t < T; t += kWarpsPerBlock - 1) {
+            const float top = s_sel[t][0];
+            const float ev = lane < k ? expf(s_sel[t][lane] - top) : 0.0f;
+            float sum = ev;
+#pragma unroll
+            for (int m = 16; m >= 1; m >>= 1)
+                sum += __shfl_xor_sync(0xffffffffu, sum, m);
+            if (lane < k) {
+                idx_out[(size_t)t * k + lane] = s_idx[t * k + lane];
+                gate_out[(size_t)t * k + lane] = ev / sum;
+            }
+        }
         return;
+    }
 
     // ================================================================ planning, by one warp
     // lane owns experts lane and lane + 32, slots lane and lane + 32, pairs lane and lane + 32
