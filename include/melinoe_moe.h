@@ -182,8 +182,9 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
  * Same call with HOST buffers: copies hidden_host to the device, runs the layer, copies the
  * result to out_host and (if not NULL) the statistics to stats_host, all in stream order.
  * Page-locked buffers make the copies asynchronous; pageable buffers work but block.  For calls of
- * at most 8 tokens with page-locked (device-mapped), 16-byte aligned out_host / 8-byte aligned
- * stats_host, the kernels write the result and the statistics straight into those buffers; they
+ * at most 8 tokens with page-locked (device-mapped), 16-byte aligned hidden_host / out_host and
+ * 8-byte aligned stats_host, a small kernel fetches the input and the layer's kernels write the
+ * result and the statistics straight into those buffers (no copy-engine operation at all); they
  * are complete when the stream reaches the end of the call, as with the copies.
  */
 int melinoe_moe_forward_host(melinoe_moe_t *h, void *cuda_stream, const void *hidden_host,

@@ -1049,7 +1049,18 @@ int melinoe_moe_forward_host(melinoe_moe_t *h, void *cuda_stream, const void *hi
         return rc;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     const size_t bytes = (size_t)T * h->d * 2;
-    CU_TRY(cudaMemcpyAsync(h->stage_in, hidden_host, bytes, cudaMemcpyHostToDevice, s));
+    {
+        // decode-sized input from page-locked (device-mapped) memory: fetched by a small kernel, which
+        // costs the stream less than a copy-engine operation; otherwise a plain copy
+        cudaPointerAttributes a;
+        if (T <= kTokPerVr && cudaPointerGetAttributes(&a, hidden_host) == cudaSuccess && a.type == cudaMemoryTypeHost &&
+            a.devicePointer && aligned16(a.devicePointer)) {
+            CU_TRY(launch_stage_in(s, a.devicePointer, h->stage_in, bytes));
+        } else {
+            (void)cudaGetLastError();
+            CU_TRY(cudaMemcpyAsync(h->stage_in, hidden_host, bytes, cudaMemcpyHostToDevice, s));
+        }
+    }
     // A decode-sized result goes straight to page-locked host memory from the kernels that produce it
     // (a few hundred posted writes) instead of through two more copy-engine operations, each of
     // which costs the stream several microseconds.  Pageable buffers and large calls are staged.

@@ -102,6 +102,8 @@ cudaError_t launch_combine_rows(cudaStream_t stream, const DevPlan *plan, const 
                                 const float *zs, uint16_t *out, int T, int d, int k, int n_shared, int n_sms);
 
 // ---- 4-bit host store: expand one 4-bit expert (layout in dequant.cu) into a bf16 slot
+// ---- decode-sized input from device-mapped host memory into device memory (bytes % 16 == 0)
+cudaError_t launch_stage_in(cudaStream_t stream, const void *src_mapped, void *dst, size_t bytes);
 cudaError_t launch_dequant_q4(cudaStream_t stream, const void *q4_blob, void *slot, int d, int F, int n_sms);
 
 }  // namespace melinoe
