@@ -12,7 +12,7 @@ import numpy as np
 
 from . import build as _build
 
-__all__ = ["threads", "logits", "topk", "route", "gather", "quantize_q4", "dequantize_q4", "ExpertCache", "ffn_combine", "layer_forward"]
+__all__ = ["threads", "logits", "topk", "route", "gather", "quantize_q4", "dequantize_q4", "miss_proxies", "ExpertCache", "ffn_combine", "layer_forward"]
 
 _lib = None
 
@@ -126,6 +126,51 @@ def dequantize_q4(codes, scales) -> np.ndarray:
     if _L().moe_oracle_dequantize_q4(_p(codes), _p(scales), rows, cols, _p(out)):
         raise ValueError("cols must be a positive multiple of 64")
     return out
+
+
+def miss_proxies(idx, n_experts: int, cache_slots: int, gamma: float):
+    """Cache-miss proxies of one layer's routing trace (Section 3.1's cache simulation and
+    Definition C.1), forward only.  idx [T][K]: the experts each token selected.
+
+    Returns (soft, hard):
+      soft  [T] fp64: sum_i r_i (1 - c_i) per token with the soft cache state c of Section 3.1
+            (c starts at 0 and follows c <- gamma c + r while its L1 norm is below C; the first
+            update that reaches C is rescaled to norm C and starts the normaliser Z = 1; from
+            then on c <- (gamma Z c + r) / Z', Z' = gamma Z + K / C, which keeps the norm at C);
+            their mean is the loss L_cs of that layer;
+      hard  [T] int: requested experts outside the hard cache Top-C(count) of Definition C.1
+            (count starts at 0, count <- gamma count + r; the cache holds the up to C experts of
+            largest non-zero count, lower index first among equals): the misses of a
+            gamma-discounted cache, whose sum is the number of transfers of Appendix C.1.
+    """
+    idx = np.asarray(idx, dtype=np.int64)
+    T, K = idx.shape
+    E, C = int(n_experts), int(cache_slots)
+    c = np.zeros(E)
+    Z, filled = 1.0, False
+    count = np.zeros(E)
+    soft = np.zeros(T)
+    hard = np.zeros(T, dtype=np.int64)
+    for t in range(T):
+        r = np.zeros(E)
+        r[idx[t]] = 1.0
+        soft[t] = float((r * (1.0 - c)).sum())
+        order = [i for i in np.argsort(-count, kind="stable") if count[i] > 0][:C]
+        resident = np.zeros(E)
+        resident[order] = 1.0
+        hard[t] = int((r * (1.0 - resident)).sum())
+        if not filled:
+            nxt = gamma * c + r
+            if nxt.sum() >= C:
+                nxt *= C / nxt.sum()
+                filled, Z = True, 1.0
+            c = nxt
+        else:
+            Zn = gamma * Z + r.sum() / C
+            c = (gamma * Z * c + r) / Zn
+            Z = Zn
+        count = gamma * count + r
+    return soft, hard
 
 
 class ExpertCache:

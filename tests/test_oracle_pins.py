@@ -428,6 +428,54 @@ def test_q4_error_bound_range_and_grid_points():
         oracle.quantize_q4(np.zeros((2, 96), np.uint16))
 
 
+def test_miss_proxies_closed_forms():
+    """Section 3.1's soft cache and Definition C.1's hard cache on traces whose answer is known."""
+    E, C, K = 12, 4, 2
+    # the same K experts every token: once the soft cache is full its whole mass C sits on them, so the
+    # proxy is K (1 - C / K) = K - C; the hard cache misses them once
+    same = np.tile(np.array([[3, 7]]), (60, 1))
+    soft, hard = oracle.miss_proxies(same, E, C, 0.9)
+    assert soft[0] == K and np.allclose(soft[-10:], K - C)
+    assert hard.tolist() == [2] + [0] * 59
+    # gamma = 0 with K < C: the state is the previous request (its norm K never reaches C, so it is never
+    # rescaled), soft and hard proxy are both K - |overlap with the previous token|
+    rs = np.random.default_rng(9)
+    tr = np.stack([rs.choice(E, size=K, replace=False) for _ in range(80)])
+    soft0, hard0 = oracle.miss_proxies(tr, E, C, 0.0)
+    for t in range(1, 80):
+        overlap = len(set(tr[t].tolist()) & set(tr[t - 1].tolist()))
+        assert soft0[t] == K - overlap and hard0[t] == K - overlap
+    # gamma = 1: the fill ends after C / K tokens with c0 = the sum of their requests (norm exactly C);
+    # from then on Z_n c_n = c0 + the requests since, Z_n = 1 + n K / C
+    soft1, _ = oracle.miss_proxies(tr, E, C, 1.0)
+    n0 = C // K
+    acc = np.zeros(E)
+    for t in range(80):
+        r = np.zeros(E)
+        r[tr[t]] = 1.0
+        if t >= n0:
+            c_t = acc / (1.0 + (t - n0) * K / C)
+            assert abs(soft1[t] - float((r * (1.0 - c_t)).sum())) < 1e-12
+        acc += r
+    # the norm of the soft state stays at C after the fill: sum_i (1 - c_i) r_i <= K and the mean proxy
+    # over a uniform trace is K (1 - C / E) up to sampling noise
+    big = np.stack([rs.choice(E, size=K, replace=False) for _ in range(4000)])
+    soft_u, _ = oracle.miss_proxies(big, E, C, 0.9)
+    assert abs(soft_u[100:].mean() - K * (1 - C / E)) < 0.03
+
+
+@pytest.mark.parametrize("C,E", [(4, 10), (6, 16)])
+def test_hard_miss_proxy_is_the_lru_miss_count_for_small_gamma(C, E):
+    """K = 1 and gamma < 1/2: Top-C of the discounted counts is the C most recent experts, so the
+    hard proxy equals the misses of the LRU cache oracle on the same trace."""
+    rs = np.random.default_rng(C)
+    tr = rs.integers(0, E, size=(400, 1))
+    _, hard = oracle.miss_proxies(tr, E, C, 0.25)
+    cache = oracle.ExpertCache(C, E)
+    lru = [int(1 - cache.call(tr[t:t + 1])[0, 2]) for t in range(400)]
+    assert hard.tolist() == lru
+
+
 def test_miss_bytes_match_papers_transfer_example():
     g = _gold("transfer_time.json")
     cfg = gen.config_by_name("mixtral")
