@@ -249,6 +249,34 @@ int melinoe_moe_set_policy(melinoe_moe_t *h, int policy, float gamma);
  * Waits for the handle's queued calls. */
 int melinoe_moe_cache_counts(melinoe_moe_t *h, float *counts_host);
 
+/*
+ * Cache-miss proxies of a recorded routing trace, forward only: what a cache of a given size
+ * would have cost on routing that has already happened, for choosing per-layer cache sizes under
+ * one memory budget.  No handle and no expert weights are involved.
+ *   soft  Section 3.1: the mean over the layer's tokens of sum_i r_i (1 - c_i), c the soft cache
+ *         state of the cache simulation loss (zero start, un-normalised fill until its L1 norm
+ *         reaches C, the update that reaches C rescaled to exactly C, then the normalised update
+ *         with Z' = gamma Z + K / C): the layer's term of L_cs;
+ *   hard  Definition C.1: requested experts outside Top-C of the gamma-discounted counts (zero
+ *         start, only non-zero counts are resident, lower index first among equal counts), summed
+ *         over the tokens: the transfers of a gamma-cache (Appendix C.1).
+ * trace_dev [n_layers][n_tokens][top_k] int32 expert ids (device); configs_dev [n_configs]
+ * (device), each naming a layer, a cache size in [1, n_experts] and a gamma in [0, 1];
+ * soft_mean_dev [n_configs] fp64 and hard_total_dev [n_configs] int64 (device) receive the
+ * results.  Asynchronous on cuda_stream.  fp64 throughout; n_experts <= 64, top_k <= n_experts.
+ * A configuration whose layer, cache size or gamma is out of range is not evaluated: its results
+ * are NaN and -1.  Expert ids outside [0, n_experts) match no expert; the trace is expected to be
+ * one the router produced (top_k distinct experts per token).
+ */
+typedef struct melinoe_proxy_config {
+    int32_t layer;
+    int32_t cache_slots;
+    double gamma;
+} melinoe_proxy_config;
+int melinoe_trace_miss_proxies(void *cuda_stream, const int32_t *trace_dev, int n_layers, int n_tokens, int top_k,
+                               int n_experts, const melinoe_proxy_config *configs_dev, int n_configs,
+                               double *soft_mean_dev, int64_t *hard_total_dev);
+
 /* Cold start: all slots empty, stamps and totals zero.  Synchronises the handle first. */
 int melinoe_moe_reset_cache(melinoe_moe_t *h);
 

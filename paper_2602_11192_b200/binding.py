@@ -8,7 +8,7 @@ from typing import Optional, Sequence
 __all__ = [
     "MelinoeError", "Stats", "Request", "lib", "library_path", "STATUS_NAMES", "MoELayer",
     "melinoe_moe_expert_bytes", "melinoe_moe_pack_expert", "melinoe_moe_expert_bytes_q4",
-    "melinoe_moe_pack_expert_q4", "melinoe_launch_count",
+    "melinoe_moe_pack_expert_q4", "melinoe_trace_miss_proxies", "ProxyConfig", "melinoe_launch_count",
     "melinoe_last_cuda_error", "melinoe_strerror", "EXPORTED_SYMBOLS",
 ]
 
@@ -23,7 +23,7 @@ EXPORTED_SYMBOLS = [
     "melinoe_moe_enable_timing", "melinoe_moe_ffn_time_ms", "melinoe_moe_set_trace", "melinoe_moe_trace_ctas",
     "melinoe_moe_transfer_time_ms", "melinoe_moe_forward_static", "melinoe_moe_static_scratch_bytes",
     "melinoe_moe_last_call_used_gemm", "melinoe_moe_set_policy", "melinoe_moe_cache_counts", "melinoe_moe_expert_bytes_q4",
-    "melinoe_moe_pack_expert_q4", "melinoe_moe_register_host_experts_q4", "melinoe_launch_count",
+    "melinoe_moe_pack_expert_q4", "melinoe_moe_register_host_experts_q4", "melinoe_trace_miss_proxies", "melinoe_launch_count",
     "melinoe_last_cuda_error", "melinoe_strerror",
 ]
 
@@ -85,6 +85,7 @@ def lib():
     L.melinoe_moe_static_scratch_bytes.restype = sz
     L.melinoe_moe_last_call_used_gemm.argtypes = [vp]
     L.melinoe_moe_reset_cache.argtypes = [vp]
+    L.melinoe_trace_miss_proxies.argtypes = [vp, vp, i32, i32, i32, i32, vp, i32, vp, vp]
     L.melinoe_moe_set_policy.argtypes = [vp, i32, C.c_float]
     L.melinoe_moe_cache_counts.argtypes = [vp, vp]
     L.melinoe_moe_preload.argtypes = [vp, vp, i32]
@@ -133,6 +134,18 @@ def melinoe_moe_pack_expert_q4(d_model: int, d_ff: int, w_gate_ptr: int, w_up_pt
     rc = lib().melinoe_moe_pack_expert_q4(d_model, d_ff, w_gate_ptr, w_up_ptr, w_down_ptr, blob_ptr)
     if rc:
         raise MelinoeError(rc, "melinoe_moe_pack_expert_q4")
+
+
+class ProxyConfig(C.Structure):
+    _fields_ = [("layer", C.c_int32), ("cache_slots", C.c_int32), ("gamma", C.c_double)]
+
+
+def melinoe_trace_miss_proxies(stream: int, trace_dev, n_layers: int, n_tokens: int, top_k: int, n_experts: int,
+                               configs_dev, n_configs: int, soft_mean_dev, hard_total_dev) -> None:
+    rc = lib().melinoe_trace_miss_proxies(stream, _ptr(trace_dev), n_layers, n_tokens, top_k, n_experts,
+                                          _ptr(configs_dev), n_configs, _ptr(soft_mean_dev), _ptr(hard_total_dev))
+    if rc:
+        raise MelinoeError(rc, "melinoe_trace_miss_proxies")
 
 
 def melinoe_launch_count() -> int:

@@ -1088,6 +1088,22 @@ int melinoe_moe_forward_host(melinoe_moe_t *h, void *cuda_stream, const void *hi
     return MELINOE_OK;
 }
 
+int melinoe_trace_miss_proxies(void *cuda_stream, const int32_t *trace_dev, int n_layers, int n_tokens, int top_k,
+                               int n_experts, const melinoe_proxy_config *configs_dev, int n_configs,
+                               double *soft_mean_dev, int64_t *hard_total_dev)
+{
+    if (!trace_dev || !configs_dev || !soft_mean_dev || !hard_total_dev || n_layers <= 0 || n_tokens < 0 || top_k <= 0 ||
+        n_experts <= 0 || n_configs < 0 || top_k > n_experts)
+        return MELINOE_ERR_INVALID;
+    if (n_experts > kMaxExperts)
+        return MELINOE_ERR_UNSUPPORTED;
+    if (n_configs == 0)
+        return MELINOE_OK;
+    CU_TRY(launch_miss_proxies(static_cast<cudaStream_t>(cuda_stream), trace_dev, n_layers, n_tokens, top_k, n_experts, configs_dev,
+                               n_configs, soft_mean_dev, reinterpret_cast<long long *>(hard_total_dev)));
+    return MELINOE_OK;
+}
+
 int melinoe_moe_reset_cache(melinoe_moe_t *h)
 {
     if (!h)

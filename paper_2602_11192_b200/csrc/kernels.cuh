@@ -101,6 +101,10 @@ cudaError_t launch_ffn_gemm(cudaStream_t stream, int phase, int n_sms, const Gem
 cudaError_t launch_combine_rows(cudaStream_t stream, const DevPlan *plan, const float *gate, const int32_t *inv_pos,
                                 const float *zs, uint16_t *out, int T, int d, int k, int n_shared, int n_sms);
 
+// ---- cache-miss proxies of a recorded routing trace (Section 3.1, Definition C.1)
+cudaError_t launch_miss_proxies(cudaStream_t stream, const int32_t *idx, int n_layers, int T, int K, int E,
+                                const melinoe_proxy_config *cfgs, int n_cfg, double *soft_mean, long long *hard_total);
+
 // ---- 4-bit host store: expand one 4-bit expert (layout in dequant.cu) into a bf16 slot
 // ---- decode-sized input from device-mapped host memory into device memory (bytes % 16 == 0)
 cudaError_t launch_stage_in(cudaStream_t stream, const void *src_mapped, void *dst, size_t bytes);

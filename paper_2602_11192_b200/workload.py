@@ -34,14 +34,17 @@ class Stack:
 
     def __init__(self, cfg: gen.MoEConfig, alpha: float, cache_slots: int, n_layers: Optional[int] = None,
                  verbose: bool = False, policy: str = "lru", gamma: float = 0.0, store: str = "bf16"):
-        self.cfg, self.alpha, self.C = cfg, float(alpha), int(cache_slots)
+        self.cfg, self.alpha = cfg, float(alpha)
         self.L = cfg.n_layers if n_layers is None else int(n_layers)
+        # one cache size for every layer, or one per layer (see budget.allocate_slots)
+        self.C = [int(cache_slots)] * self.L if np.isscalar(cache_slots) else [int(c) for c in cache_slots]
+        assert len(self.C) == self.L
         self.layers: List[LayerSetup] = []
         self.w_r: List[np.ndarray] = []
         self.bias: List[np.ndarray] = []
         t0 = time.time()
         for l in range(self.L):
-            ls = LayerSetup(cfg.d_model, cfg.d_ff, cfg.n_experts, cfg.top_k, self.C, cfg.n_shared)
+            ls = LayerSetup(cfg.d_model, cfg.d_ff, cfg.n_experts, cfg.top_k, self.C[l], cfg.n_shared)
             wg, wu, wd = gen.fill_expert_store_fast(cfg.seed, l, cfg.n_experts + cfg.n_shared, cfg.d_model, cfg.d_ff)
             if store == "q4":
                 ls.set_experts_stacked_q4(wg[:cfg.n_experts], wu[:cfg.n_experts], wd[:cfg.n_experts])

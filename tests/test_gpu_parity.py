@@ -289,6 +289,43 @@ def test_parity_without_programmatic_launch():
     assert r.returncode == 0 and "child ok" in r.stdout, r.stdout[-2000:] + r.stderr[-2000:]
 
 
+def test_trace_miss_proxies_match_the_oracle():
+    """Soft (Section 3.1) and hard (Definition C.1) miss proxies of recorded traces, every cache size
+    at once: hard misses exact, soft proxy to fp64 rounding; then a budget split over the layers."""
+    from paper_2602_11192_b200.budget import miss_curves, allocate_slots
+    rs = np.random.default_rng(71)
+    L, T, K, E = 3, 300, 2, 12
+    trace = np.empty((L, T, K), np.int32)
+    for l, alpha in enumerate((0.05, 0.5, 50.0)):             # from concentrated to uniform routing
+        pref = rs.dirichlet(np.full(E, alpha)) + 1e-6
+        pref /= pref.sum()
+        for t in range(T):
+            trace[l, t] = rs.choice(E, size=K, replace=False, p=pref)
+    sizes = list(range(K, E + 1))
+    for gamma in (1.0, 0.9, 0.0):
+        soft, hard = miss_curves(trace, E, gamma, sizes)
+        for l in range(L):
+            for j, c in enumerate(sizes):
+                so, ho = oracle.miss_proxies(trace[l], E, c, gamma)
+                assert hard[l, j] == int(ho.sum()), (gamma, l, c)
+                assert abs(soft[l, j] - so.mean()) <= 1e-10 * max(1.0, abs(so.mean())), (gamma, l, c)
+        assert np.all(np.diff(hard, axis=1) <= 0)            # a larger gamma-cache never transfers more
+    _, hard = miss_curves(trace, E, 0.9, sizes)
+    slots = allocate_slots(hard, sizes, 3 * K + 9)
+    assert sum(slots) == 3 * K + 9 and slots[0] <= slots[1]   # concentrated routing needs the fewest slots
+    # a configuration that names nothing is marked, not evaluated
+    import torch
+    from paper_2602_11192_b200 import binding as B
+    from paper_2602_11192_b200.runner import current_stream_ptr
+    cfg = (B.ProxyConfig * 2)(B.ProxyConfig(7, 4, 0.9), B.ProxyConfig(0, 0, 0.9))
+    cfg_dev = torch.frombuffer(bytearray(bytes(cfg)), dtype=torch.uint8).cuda()
+    so = torch.zeros(2, dtype=torch.float64, device="cuda")
+    ha = torch.zeros(2, dtype=torch.int64, device="cuda")
+    B.melinoe_trace_miss_proxies(current_stream_ptr(), torch.from_numpy(trace).cuda(), L, T, K, E, cfg_dev, 2, so, ha)
+    torch.cuda.synchronize()
+    assert bool(torch.isnan(so).all()) and ha.tolist() == [-1, -1]
+
+
 def test_argument_and_state_errors():
     import torch
     from paper_2602_11192_b200 import MoELayer, MelinoeError, melinoe_moe_expert_bytes

@@ -72,6 +72,29 @@ def test_pack_expert_q4_matches_the_oracle_bit_for_bit(m):
         m.melinoe_moe_pack_expert_q4(256, 40, w[0].ctypes.data, w[1].ctypes.data, w[2].ctypes.data, blob.ctypes.data)
 
 
+def test_budget_allocation_spends_slots_where_they_save_transfers():
+    """Host logic of the per-layer budget: greedy on the marginal transfers saved."""
+    import importlib.util
+    spec = importlib.util.spec_from_file_location("budget_src", os.path.join(ROOT, "paper_2602_11192_b200", "budget.py"))
+    src = open(spec.origin).read()
+    ns = {}
+    # the allocator itself needs neither the library nor a device: run it from its source
+    start = src.index("def allocate_slots")
+    exec("import numpy as np\nfrom typing import List, Sequence\n" + src[start:], ns)
+    alloc = ns["allocate_slots"]
+    sizes = [2, 3, 4, 5, 6]
+    hard = np.array([[100, 60, 50, 49, 49],      # layer 0: the third slot is worth 40, then little
+                     [100, 95, 90, 85, 80],      # layer 1: every slot is worth 5
+                     [30, 30, 30, 30, 30]])      # layer 2: nothing to gain
+    assert alloc(hard, sizes, 6) == [2, 2, 2]
+    assert alloc(hard, sizes, 7) == [3, 2, 2]
+    assert alloc(hard, sizes, 8) == [4, 2, 2]                 # 10 saved on layer 0 beats 5 on layer 1
+    assert alloc(hard, sizes, 10) == [4, 4, 2]
+    assert alloc(hard, sizes, 30) == [6, 6, 6]                # more budget than sizes: everything at the largest
+    with pytest.raises(ValueError):
+        alloc(hard, sizes, 5)
+
+
 def test_create_fails_loudly_without_a_device(m):
     import torch
     if torch.cuda.is_available():
