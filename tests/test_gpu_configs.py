@@ -97,3 +97,30 @@ def test_deepseek_shape_with_shared_experts():
     """configs[4]: d 2048, d_ff 1408, 64 routed + 2 shared experts, top-6, 12 slots, 4 sequences:
     8192-token prefill, then decode steps of 4 tokens; one layer of the 28."""
     _run_stack("deepseek", 1, 0.1, 12, decode_steps=3, sample_layers=(0,), y_tokens=3)
+
+
+def test_repeated_runs_with_heavy_miss_traffic_are_bit_identical():
+    """Two cold-start runs of the same OLMoE-shaped steps (near-uniform routing: several transfers
+    per layer and token, miss waves, slot reuse inside a call) give the same output bits and the
+    same statistics: nothing in the transfer / compute overlap is left to chance."""
+    import torch
+    from paper_2602_11192_b200.workload import Stack, stats_rows
+    cfg = gen.config_by_name("olmoe")
+    L, steps = 2, 60
+    runs = []
+    for rep in range(2):
+        st = Stack(cfg, 10.0, cfg.cache_slots[0], n_layers=L)
+        out = torch.empty((L, 1, cfg.d_model), dtype=torch.int16, device="cuda")
+        stats = torch.zeros((steps, L, 12), dtype=torch.int32, device="cuda")
+        outs = []
+        for s in range(steps):
+            x = torch.from_numpy(st.hidden_bits("decode", s).view(np.int16)).cuda()
+            st.forward_all(x, out, stats[s])
+            outs.append(out.clone())
+        torch.cuda.synchronize()
+        r = stats_rows(stats)
+        assert int(r["status"].max()) == 0 and int(r["misses"].sum()) > 3 * L * steps
+        runs.append((torch.stack(outs).cpu().numpy(), stats.cpu().numpy()[:, :, :8]))
+        st.close()
+    assert np.array_equal(runs[0][0], runs[1][0]) and np.array_equal(runs[0][1], runs[1][1])
+
