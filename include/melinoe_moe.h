@@ -329,9 +329,11 @@ int melinoe_moe_transfer_time_ms(melinoe_moe_t *h, double *ms_out, uint64_t *byt
 int melinoe_moe_set_trace(melinoe_moe_t *h, void *trace_dev, size_t bytes);
 int melinoe_moe_trace_ctas(melinoe_moe_t *h);
 
-/* 1 if the most recent forward call of the handle ran its expert FFN as the tensor-core grouped
- * GEMM (calls of more than 8 tokens on shapes with d_model % 256 == 0 and d_ff % 128 == 0),
- * 0 if it ran the streaming kernel. */
+/* Non-zero if the most recent forward call of the handle ran its expert FFN as the tensor-core
+ * grouped GEMM (calls of more than 8 tokens on shapes with d_model % 256 == 0 and d_ff % 128 == 0):
+ * 1 on single CTAs (128-token tiles), 2 on CTA pairs (256-token tiles: an alternative that runs only
+ * with MELINOE_MOE_PAIR set in the environment and at least 192 routed tokens per expert on
+ * average; it measured no faster); 0 if it ran the streaming kernel. */
 int melinoe_moe_last_call_used_gemm(melinoe_moe_t *h);
 
 /* Number of kernels this library has launched in this process (all handles). */

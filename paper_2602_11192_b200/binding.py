@@ -303,6 +303,10 @@ class MoELayer:
     def last_call_used_gemm(self) -> bool:
         return bool(lib().melinoe_moe_last_call_used_gemm(self._h))
 
+    def last_call_gemm_kind(self) -> int:
+        """0 streaming kernel, 1 grouped GEMM on single CTAs, 2 grouped GEMM on CTA pairs."""
+        return int(lib().melinoe_moe_last_call_used_gemm(self._h))
+
     def transfer_time_ms(self):
         ms = C.c_double(0.0)
         nb = C.c_uint64(0)

@@ -121,7 +121,7 @@ struct melinoe_moe {
     VrRec *vrs = nullptr;
     uint16_t *stage_in = nullptr, *stage_out = nullptr;
     // grouped-GEMM path (calls of more than 8 tokens): gathered activations, h, tensor maps
-    bool gemm_ok = false, last_used_gemm = false;
+    bool gemm_ok = false, pair_ok = false, last_used_gemm = false, last_used_pair = false;
     uint16_t *xs = nullptr, *hs = nullptr;
     CUtensorMap *maps_dev = nullptr;
     CUtensorMap maps_host[kMapCount];
@@ -479,9 +479,11 @@ int melinoe_moe_create(int d, int F, int E, int k, int C, melinoe_moe_t **out)
     if (ffn_gemm_supported(d, F) && h->slot_stride == h->expert_bytes && ffn_gemm_configure() == cudaSuccess) {
         CR(cudaMalloc(&h->maps_dev, sizeof(h->maps_host)));
         if (encode_map(&h->maps_host[kMapSlotsD], h->slots, d, (uint64_t)C * 3 * F, 128) &&
-            encode_map(&h->maps_host[kMapSlotsF], h->slots, F, (uint64_t)C * 3 * d, 256)) {
+            encode_map(&h->maps_host[kMapSlotsF], h->slots, F, (uint64_t)C * 3 * d, 256) &&
+            encode_map(&h->maps_host[kMapSlotsF128], h->slots, F, (uint64_t)C * 3 * d, 128)) {
             CR(cudaMemcpy(h->maps_dev, h->maps_host, sizeof(h->maps_host), cudaMemcpyHostToDevice));
             h->gemm_ok = true;
+            h->pair_ok = ffn_gemm_pair_configure() == cudaSuccess && (h->n_sms & ~1) >= 2;
         }
     }
     (void)cudaGetLastError();
@@ -637,7 +639,8 @@ int melinoe_moe_register_shared_experts(melinoe_moe_t *h, int n_shared, const vo
     if (h->gemm_ok) {
         for (int s = 0; s < n_shared; ++s)
             if (!encode_map(&h->maps_host[kMapShared0 + 2 * s], ptrs[s], h->d, (uint64_t)3 * h->F, 128) ||
-                !encode_map(&h->maps_host[kMapShared0 + 2 * s + 1], ptrs[s], h->F, (uint64_t)3 * h->d, 256))
+                !encode_map(&h->maps_host[kMapShared0 + 2 * s + 1], ptrs[s], h->F, (uint64_t)3 * h->d, 256) ||
+                !encode_map(&h->maps_host[kMapSharedF128 + s], ptrs[s], h->F, (uint64_t)3 * h->d, 128))
                 return MELINOE_ERR_CUDA;
         CU_TRY(cudaMemcpy(h->maps_dev, h->maps_host, sizeof(h->maps_host), cudaMemcpyHostToDevice));
     }
@@ -742,6 +745,11 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
         return MELINOE_ERR_UNSUPPORTED;
     // calls of more than 8 tokens go through the grouped GEMM (where the shapes allow it)
     const bool use_gemm = h->gemm_ok && T > kTokPerVr && h->xs != nullptr;
+    // Alternative for calls with many tokens per expert: 256-token tiles on CTA pairs (each B tile staged
+    // once per 256 rows).  Measured no faster than single CTAs (Phi-3.5-shaped prompt 1097 against
+    // 1126 TFLOP/s, DeepSeek-shaped 1026 against 1015), so it runs only when MELINOE_MOE_PAIR is set.
+    const bool use_pair = use_gemm && h->pair_ok && (long long)T * h->k >= (long long)192 * h->E &&
+                          std::getenv("MELINOE_MOE_PAIR") != nullptr;
     GemmParams gp;
     gp.plan = h->plan;
     gp.maps = h->maps_dev;
@@ -753,6 +761,7 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
     gp.E = h->E;
     gp.n_shared = h->n_shared;
     h->last_used_gemm = use_gemm;
+    h->last_used_pair = use_pair;
     if (use_gemm)
         CU_TRY(launch_gather_rows(s, h->plan, static_cast<const uint16_t *>(hidden_dev), h->tok_of_sorted, h->xs, h->d,
                                   T * h->k + h->n_shared * T, h->n_sms));
@@ -770,8 +779,13 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
         }
         if (use_gemm) {
             gp.group = g;
-            CU_TRY(launch_ffn_gemm(s, 1, h->n_sms, gp));
-            CU_TRY(launch_ffn_gemm(s, 2, h->n_sms, gp));
+            if (use_pair) {
+                CU_TRY(launch_ffn_gemm_pair(s, 1, h->n_sms, gp));
+                CU_TRY(launch_ffn_gemm_pair(s, 2, h->n_sms, gp));
+            } else {
+                CU_TRY(launch_ffn_gemm(s, 1, h->n_sms, gp));
+                CU_TRY(launch_ffn_gemm(s, 2, h->n_sms, gp));
+            }
         } else {
             fp.group = g;
             CU_TRY(launch_ffn_stream(s, h->cfg, geo, fp));
@@ -1334,7 +1348,7 @@ int melinoe_moe_set_trace(melinoe_moe_t *h, void *trace_dev, size_t bytes)
 
 int melinoe_moe_trace_ctas(melinoe_moe_t *h) { return h ? h->cfg.grid : 0; }
 
-int melinoe_moe_last_call_used_gemm(melinoe_moe_t *h) { return h && h->last_used_gemm ? 1 : 0; }
+int melinoe_moe_last_call_used_gemm(melinoe_moe_t *h) { return h && h->last_used_gemm ? (h->last_used_pair ? 2 : 1) : 0; }
 
 int melinoe_moe_enable_timing(melinoe_moe_t *h, int enable)
 {

@@ -84,7 +84,13 @@ cudaError_t launch_ffn_stream(cudaStream_t stream, const FfnLaunchCfg &cfg, cons
 
 // ---- grouped GEMM expert FFN on tcgen05 for calls with many tokens per expert (prefill)
 // Tensor maps in device memory, in this order:
-enum { kMapXs = 0, kMapHs = 1, kMapSlotsD = 2, kMapSlotsF = 3, kMapShared0 = 4, kMapCount = kMapShared0 + 2 * kMaxShared };
+enum {
+    kMapXs = 0, kMapHs = 1, kMapSlotsD = 2, kMapSlotsF = 3,          // boxes of 128, 128, 128 and 256 rows
+    kMapShared0 = 4,                                                 // per shared expert: rows of d (128), rows of F (256)
+    kMapSlotsF128 = kMapShared0 + 2 * kMaxShared,                    // rows of F in boxes of 128 rows (CTA-pair kernel)
+    kMapSharedF128 = kMapSlotsF128 + 1,                              // the same per shared expert
+    kMapCount = kMapSharedF128 + kMaxShared
+};
 struct GemmParams {
     const DevPlan *plan;
     const CUtensorMap *maps;         // device array of kMapCount tensor maps
@@ -98,6 +104,9 @@ cudaError_t ffn_gemm_configure();
 cudaError_t launch_gather_rows(cudaStream_t stream, const DevPlan *plan, const uint16_t *x, const int32_t *tok_of_sorted,
                                uint16_t *xs, int d, int n_sorted, int n_sms);
 cudaError_t launch_ffn_gemm(cudaStream_t stream, int phase, int n_sms, const GemmParams &p);
+// the same two GEMMs on CTA pairs (tcgen05.mma.cta_group::2), for calls with many tokens per expert
+cudaError_t ffn_gemm_pair_configure();
+cudaError_t launch_ffn_gemm_pair(cudaStream_t stream, int phase, int n_sms, const GemmParams &p);
 cudaError_t launch_combine_rows(cudaStream_t stream, const DevPlan *plan, const float *gate, const int32_t *inv_pos,
                                 const float *zs, uint16_t *out, int T, int d, int k, int n_shared, int n_sms);
 

@@ -1,4 +1,6 @@
 """GPU-vs-oracle parity through the C ABI (run with -m gpu on a B200)."""
+import os
+
 import numpy as np
 import pytest
 
@@ -134,6 +136,8 @@ def test_prefill_then_decode_with_waves():
     (512, 256, 8, 2, 8, 0, (40, 300, 9)),        # everything fits the cache: one compute group after warm-up
     (256, 128, 16, 4, 5, 0, (130, 64)),          # more distinct experts than slots: miss waves
     (1024, 384, 6, 2, 3, 2, (257, 20)),          # shared experts, ragged last m-tile
+    (512, 256, 4, 2, 4, 0, (600, 385, 40)),      # many tokens per expert, ragged
+    (1024, 384, 4, 2, 2, 1, (700,)),             # many tokens per expert with a shared expert and miss waves
 ])
 def test_prefill_grouped_gemm(d, F, E, k, C, n_shared, Ts):
     """Calls of more than 8 tokens run the tensor-core grouped GEMM (d_ff a multiple of 128)."""
@@ -148,12 +152,25 @@ def test_prefill_grouped_gemm(d, F, E, k, C, n_shared, Ts):
         tokens = sorted(set([0, 1, T - 2, T - 1] + list(range(0, T, 7))))
         P.step(x, tokens=tokens)
         assert P.gpu.layer.last_call_used_gemm()
+        pairs_on = os.environ.get("MELINOE_MOE_PAIR") is not None
+        assert P.gpu.layer.last_call_gemm_kind() == (2 if pairs_on and T * k >= 192 * E else 1)
         step += 1
     # and decode-sized calls on the same handle afterwards (streaming kernel), sharing the cache state
     P.set_bias(bias, np.zeros(2, np.int32))
     P.step(gen.hidden_states(300 + d, 0, "decode", 0, 2, d))
     assert not P.gpu.layer.last_call_used_gemm()
     P.close()
+
+
+def test_prefill_grouped_gemm_on_cta_pairs():
+    """The same cases with the CTA-pair variant of the grouped GEMM switched on (tcgen05.mma on two
+    SMs, 256-token tiles): a child process, because the switch is an environment variable."""
+    import subprocess
+    import sys
+    env = dict(os.environ, MELINOE_MOE_PAIR="1")
+    r = subprocess.run([sys.executable, "-m", "pytest", os.path.abspath(__file__), "-q", "-x", "-m", "gpu", "-k",
+                        "test_prefill_grouped_gemm and not cta_pairs"], env=env, capture_output=True, text=True, timeout=900)
+    assert r.returncode == 0 and "5 passed" in r.stdout, r.stdout[-3000:] + r.stderr[-2000:]
 
 
 def test_forward_host_matches_forward_and_is_deterministic():
