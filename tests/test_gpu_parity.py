@@ -241,6 +241,17 @@ def test_count_policy_trace_matches_the_oracle(gamma):
     P.close()
 
 
+def test_count_policy_with_shared_experts_and_batches():
+    """The count policy on a stack with always-resident shared experts (their requests sit between
+    the hits and the miss waves in the launch order) and token batches."""
+    d, F, E, k, C = 256, 64, 12, 3, 4
+    P = _pair(d, F, E, k, C, seed=35, n_shared=2)
+    P.set_policy("count", 0.9)
+    for step, T in enumerate((4, 1, 8, 2, 30, 1, 5)):
+        P.step(gen.hidden_states(35, 0, "decode", step, T, d))
+    P.close()
+
+
 def test_count_policy_preload_and_lfu_keeps_the_hot_experts():
     d, F, E, k, C = 256, 32, 8, 2, 4
     P = _pair(d, F, E, k, C, seed=33)
