@@ -14,8 +14,11 @@
  *  - A handle is driven by one host thread at a time, and all forward calls of one handle must
  *    be ordered with respect to each other on the device (same stream, or caller-made
  *    dependencies): a call's cache decisions depend on the previous call's.
- *  - melinoe_moe_forward returns once the call's cache decisions are known to the host and all
- *    of its transfers and kernels are queued; it does not wait for transfers or compute.
+ *  - melinoe_moe_forward is asynchronous with respect to the host: for calls of at most 8 tokens
+ *    on a bf16 host store it queues two kernels and returns (the missed experts are fetched by the
+ *    compute kernel itself); otherwise it returns once the call's cache decisions are known to
+ *    the host and all of its transfers and kernels are queued.  It never waits for transfers or
+ *    compute.
  */
 #ifndef MELINOE_MOE_H_
 #define MELINOE_MOE_H_
@@ -68,7 +71,7 @@ typedef struct melinoe_moe_request {
  * Create one layer.  Shapes follow Eq. 1-3: router W_r [n_experts][d_model]; each expert has
  * W_g, W_u [d_ff][d_model] and W_d [d_model][d_ff].  Allocates, on the current device,
  * cache_slots expert slots of melinoe_moe_expert_bytes() each plus small tables, and creates
- * a copy stream.  Limits: d_model % 256 == 0, d_model <= 8192, d_ff % 8 == 0,
+ * a copy stream.  Limits: d_model % 256 == 0, d_model <= 4096, d_ff % 8 == 0,
  * 1 <= top_k <= n_experts <= 64, top_k <= 32, top_k <= cache_slots <= n_experts  (INVALID / UNSUPPORTED
  * otherwise).
  */
@@ -83,12 +86,17 @@ int melinoe_moe_destroy(melinoe_moe_t *h);
 size_t melinoe_moe_expert_bytes(int d_model, int d_ff);
 
 /*
- * Pack one expert from the paper's matrices (Eq. 3; bf16, row-major, host memory) into one
- * contiguous blob (host memory, `melinoe_moe_expert_bytes` long):
- *     W_g [d_ff][d_model] | W_u [d_ff][d_model] | W_d [d_model][d_ff]
- * i.e. the three matrices back to back in the paper's own shapes, so every row that a kernel
- * streams is one contiguous byte range.  Pure host code; does not touch the device.  blob_out
- * must not overlap the inputs.
+ * Pack one expert from the paper's matrices (Eq. 3: W_g, W_u [d_ff][d_model], W_d [d_model][d_ff];
+ * bf16, row-major, host memory) into one contiguous blob (host memory, `melinoe_moe_expert_bytes`
+ * long).  The blob holds, for every hidden unit f = 0 .. d_ff - 1, the three vectors that belong to
+ * it back to back, 3 * d_model elements:
+ *     W_g[f][0 .. d_model) | W_u[f][0 .. d_model) | W_d[0 .. d_model)[f]
+ * so that everything f contributes to the layer's output (Eq. 3) is one contiguous byte range, and
+ * any run of consecutive f is too.  Within each of the three vectors, every group of 64 elements
+ * (128 bytes) has its eight 16-byte pieces stored at position (piece xor (f mod 8)): shared-memory
+ * bank conflicts of the kernels' tensor-core fragment loads are avoided by this permutation, and it
+ * is the arrangement the tensor cores' 128-byte-swizzled operand layout expects.  Pure host code;
+ * does not touch the device.  blob_out must not overlap the inputs.  d_model % 64 == 0.
  */
 int melinoe_moe_pack_expert(int d_model, int d_ff, const void *w_gate_host, const void *w_up_host,
                             const void *w_down_host, void *blob_out_host);
@@ -119,7 +127,11 @@ int melinoe_moe_set_router(melinoe_moe_t *h, const void *w_router_dev);
  * expert_host_ptrs[e] points to expert e packed by melinoe_moe_pack_expert, in page-locked
  * host memory, 16-byte aligned; bytes_per_expert must equal melinoe_moe_expert_bytes().
  * Pointers are checked with the CUDA runtime: pageable memory is rejected with INVALID (the
- * library never stages silently).  Borrowed, read-only, must outlive the handle.
+ * library never stages silently).  Borrowed, read-only, must outlive the handle.  Where the device
+ * can address the store (memory from cudaHostAlloc, or registered with cudaHostRegister), calls of
+ * at most 8 tokens read the experts they miss straight from it inside the compute kernel, with no
+ * host involvement; MELINOE_MOE_HOST_COPIES in the environment keeps every transfer a
+ * cudaMemcpyAsync issued by the host.
  */
 int melinoe_moe_register_host_experts(melinoe_moe_t *h, const void *const *expert_host_ptrs,
                                       size_t bytes_per_expert);
@@ -127,9 +139,10 @@ int melinoe_moe_register_host_experts(melinoe_moe_t *h, const void *const *exper
 /*
  * Same registration for a store of 4-bit blobs (melinoe_moe_pack_expert_q4): a miss then moves the
  * 4-bit blob over the host link (3.76 times fewer bytes, which is what a miss costs, Eq. 4) and a
- * kernel on the handle's copy stream expands it into the bf16 slot behind the copy, so the cache
- * slots and the compute kernels are the same as with a bf16 store and the layer computes with
- * exactly the weights the format defines.  The statistics count the bytes that travelled.
+ * kernel expands it into the bf16 slot behind the copy, so the cache slots and the compute kernels
+ * are the same as with a bf16 store and the layer computes with exactly the weights the format
+ * defines.  The statistics count the bytes that travelled.  Transfers of such a store are issued by
+ * the host (the forward call waits for the call's cache decisions, see melinoe_moe_forward).
  * Page-locked, 16-byte aligned, borrowed, as above.  Registering one kind of store replaces the
  * other; the cache should be reset when the store changes.
  */
@@ -168,12 +181,19 @@ int melinoe_moe_reserve(melinoe_moe_t *h, int max_tokens);
  * until the stream work of this call has finished.  stats_dev: see melinoe_moe_stats; may be
  * NULL.  n_tokens == 0 is a no-op.
  *
- * Host behaviour: the router, planning and resident-expert FFN kernels are queued first; the
- * call then waits (bounded; TIMEOUT after 60 s) until the planning kernel has published the
- * call's miss queue in page-locked memory, issues one cudaMemcpyAsync per missed expert on the
- * handle's copy stream, ties the streams together with events, queues the remaining kernels and
- * returns.  It therefore waits for earlier work on cuda_stream, but never for its own transfers,
- * FFN kernels or combine.
+ * Host behaviour.  Calls of at most 8 tokens (or of any size on shapes the grouped GEMM does not
+ * cover) on a bf16 store the device can address: the routing / planning kernel and the expert-FFN
+ * kernel are queued and the call returns; the FFN kernel reads the experts the call misses from the
+ * host store itself, stores those that stay resident into their slots, and writes the result.  The
+ * host learns the call's cache decisions only through stats_dev.
+ * All other calls (more than 8 tokens through the grouped GEMM; a 4-bit store; host copies forced):
+ * the router, planning and resident-expert kernels are queued first; the call then waits (bounded;
+ * TIMEOUT after 60 s) until the planning kernel has published the call's miss queue in page-locked
+ * memory, issues one cudaMemcpyAsync per missed expert on the handle's copy stream, ties the streams
+ * together with events, queues the remaining kernels and returns.  It then waits for earlier work on
+ * cuda_stream, but never for its own transfers, FFN kernels or combine.  If queuing fails part-way,
+ * the error is returned, stays on the handle (every later call returns it until
+ * melinoe_moe_reset_cache) and the handle can still be synchronised and destroyed.
  */
 int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_dev,
                         int n_tokens, void *out_dev, melinoe_moe_stats *stats_dev);
@@ -199,24 +219,27 @@ int melinoe_moe_forward_host(melinoe_moe_t *h, void *cuda_stream, const void *hi
  * another allocator and would get an out-of-memory error (or a device-wide synchronisation) from a
  * stray cudaMalloc, and code that runs where the CUDA allocator must not be entered at all.  This
  * entry point runs the same layer, same kernels and same cache state, but takes every byte of
- * scratch (routing tables, gather lists, the h and z buffers of the expert FFN) from one array
- * of melinoe_moe_static_scratch_bytes() (about 8.6 MiB) that is part of the library's device
+ * scratch (routing tables, gather lists, the FFN kernel's per-SM partial outputs) from one array
+ * of melinoe_moe_static_scratch_bytes() (about 10.1 MiB) that is part of the library's device
  * image: each GPU that loads the library holds it until the process exits.  It calls no
- * cudaMalloc, cudaFree, event-creating or otherwise allocating routine.
+ * cudaMalloc, cudaFree, event-creating or otherwise allocating routine, under either eviction
+ * policy (the events a call may need are made when the handle is created).
  *
- * Limits, all checked, MELINOE_ERR_UNSUPPORTED beyond them (nothing is launched then):
- *   n_tokens <= 8, n_tokens * top_k <= 16, n_tokens * top_k <= cache_slots,
- *   n_shared * n_tokens <= 64, d_model <= 8192, d_ff <= 16384.
- * MELINOE_ERR_STATE if kernel timing is enabled on the handle (timed calls create events).
+ * Limits, all checked before anything is queued, MELINOE_ERR_UNSUPPORTED beyond them:
+ *   n_tokens <= 8, n_tokens * top_k <= 64, and SMs * n_tokens * d_model * 4 bytes <= 10 MiB
+ *   (on a 148-SM device: n_tokens * d_model <= 17 712, e.g. 8 tokens at d_model 2048, 4 at 4096).
+ * MELINOE_ERR_STATE if kernel timing is enabled on the handle (timed calls create events), or if
+ * the handle's device is not the current one.
  *
  * The first call on a device looks up the array's device address (cudaGetSymbolAddress) with
  * that device current; make this first call before any stream capture begins.
  * Every call on a device, of every handle, uses the same array: it keeps the previous call's
- * contents (what has to start from zero is cleared on the caller's stream at the start of each
- * call), and two such calls that can overlap on the GPU (different streams without an ordering
- * between them) race on it.  Calls on one stream, or ordered by events, are safe, and may be
- * mixed freely with melinoe_moe_forward on the same handle.
- * The inspection calls (melinoe_moe_last_*) do not see calls made through this entry point.
+ * contents (nothing in it has to start from zero: each table is written by the call's own kernels
+ * before it is read), and two such calls that can overlap on the GPU (different streams without an
+ * ordering between them) race on it.  Calls on one stream, or ordered by events, are safe, and may
+ * be mixed freely with melinoe_moe_forward on the same handle.
+ * The inspection calls (melinoe_moe_last_*) read the scratch of the most recent call, so after a
+ * call through this entry point they are valid only until the next static call on the device.
  * Arguments and results otherwise as melinoe_moe_forward.
  */
 int melinoe_moe_forward_static(melinoe_moe_t *h, void *cuda_stream, const void *hidden_dev,
@@ -313,6 +336,11 @@ int melinoe_moe_cache_state(melinoe_moe_t *h, int32_t *expert_of_slot_host, uint
  */
 int melinoe_moe_enable_timing(melinoe_moe_t *h, int enable);
 int melinoe_moe_ffn_time_ms(melinoe_moe_t *h, double *ms_out, int64_t *launches_out);
+/* The same launches one by one, in launch order, without resetting anything: up to `capacity` times
+ * (ms) into ms_out; *n_out receives the number of timed launches recorded since the last
+ * melinoe_moe_ffn_time_ms.  With one FFN launch per call (calls of at most 8 tokens on a store the
+ * device can address) entry i belongs to the i-th call, whose statistics say what it fetched. */
+int melinoe_moe_ffn_launch_times_ms(melinoe_moe_t *h, float *ms_out, int capacity, int *n_out);
 /* With timing enabled, every wave of miss transfers is bracketed by events on the copy stream
  * as well: summed copy-stream time (ms) and bytes moved host-to-device since the last query
  * (Eq. 4's N_miss * Time_transfer, measured).  Resets both. */
@@ -321,20 +349,24 @@ int melinoe_moe_transfer_time_ms(melinoe_moe_t *h, double *ms_out, uint64_t *byt
 /*
  * Kernel timeline for profiling (no counterpart in the paper).  trace_dev: device memory of at
  * least 8 * 8 bytes per SM of the device (melinoe_moe_trace_ctas() * 64 bytes), 8-byte aligned,
- * borrowed; NULL switches tracing off.  Every expert-FFN launch then overwrites, per CTA, eight
- * 64-bit nanosecond stamps of the device's global timer: 0 entry, 1 set-up done, 2 first weight
- * stage landed, 3 gate/up phase done, 4 arrived at the grid barrier, 5 barrier passed (producer),
- * 6 down-projection phase done, 7 exit.  Stamps of steps a CTA skipped keep their old value.
+ * borrowed; NULL switches tracing off.  Every launch of the decode FFN kernel then overwrites, per
+ * CTA, eight 64-bit nanosecond stamps of the device's global timer: 0 entry, 1 set-up done (plan
+ * read, rows dealt out), 2 first tile of weights landed, 3 last tile computed, 4 arrived at the grid
+ * barrier, 5 barrier passed, 6 output written, 7 exit.  Stamps of steps a CTA skipped keep their old
+ * value.
  */
 int melinoe_moe_set_trace(melinoe_moe_t *h, void *trace_dev, size_t bytes);
 int melinoe_moe_trace_ctas(melinoe_moe_t *h);
 
-/* Non-zero if the most recent forward call of the handle ran its expert FFN as the tensor-core
- * grouped GEMM (calls of more than 8 tokens on shapes with d_model % 256 == 0 and d_ff % 128 == 0):
- * 1 on single CTAs (128-token tiles), 2 on CTA pairs (256-token tiles: an alternative that runs only
- * with MELINOE_MOE_PAIR set in the environment and at least 192 routed tokens per expert on
- * average; it measured no faster); 0 if it ran the streaming kernel. */
+/* 1 if the most recent forward call of the handle ran its expert FFN as the tensor-core grouped
+ * GEMM (calls of more than 8 tokens on shapes with d_model % 256 == 0 and d_ff % 128 == 0), 0 if it
+ * ran the decode kernel (in slices of 8 tokens where the call had more). */
 int melinoe_moe_last_call_used_gemm(melinoe_moe_t *h);
+
+/* Test hook, host side only: the nth host-issued expert copy from now (cudaMemcpyAsync of a miss
+ * wave; n >= 1) is not issued and reports a CUDA failure instead, so that the error path of a
+ * partly queued call can be exercised without any fault on the device.  0 switches it off. */
+int melinoe_debug_fail_host_copy(int nth);
 
 /* Number of kernels this library has launched in this process (all handles). */
 int64_t melinoe_launch_count(void);

@@ -24,7 +24,7 @@ EXPORTED_SYMBOLS = [
     "melinoe_moe_transfer_time_ms", "melinoe_moe_forward_static", "melinoe_moe_static_scratch_bytes",
     "melinoe_moe_last_call_used_gemm", "melinoe_moe_set_policy", "melinoe_moe_cache_counts", "melinoe_moe_expert_bytes_q4",
     "melinoe_moe_pack_expert_q4", "melinoe_moe_register_host_experts_q4", "melinoe_trace_miss_proxies", "melinoe_launch_count",
-    "melinoe_last_cuda_error", "melinoe_strerror",
+    "melinoe_last_cuda_error", "melinoe_strerror", "melinoe_moe_ffn_launch_times_ms", "melinoe_debug_fail_host_copy",
 ]
 
 STATUS_NAMES = {0: "OK", 1: "INVALID", 2: "STATE", 3: "CUDA", 4: "NOMEM", 5: "TIMEOUT", 6: "UNSUPPORTED"}
@@ -97,6 +97,8 @@ def lib():
     L.melinoe_moe_enable_timing.argtypes = [vp, i32]
     L.melinoe_moe_ffn_time_ms.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
     L.melinoe_moe_transfer_time_ms.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_uint64)]
+    L.melinoe_moe_ffn_launch_times_ms.argtypes = [vp, vp, i32, C.POINTER(i32)]
+    L.melinoe_debug_fail_host_copy.argtypes = [i32]
     L.melinoe_moe_set_trace.argtypes = [vp, vp, sz]
     L.melinoe_moe_trace_ctas.argtypes = [vp]
     L.melinoe_launch_count.restype = C.c_int64
@@ -303,9 +305,14 @@ class MoELayer:
     def last_call_used_gemm(self) -> bool:
         return bool(lib().melinoe_moe_last_call_used_gemm(self._h))
 
-    def last_call_gemm_kind(self) -> int:
-        """0 streaming kernel, 1 grouped GEMM on single CTAs, 2 grouped GEMM on CTA pairs."""
-        return int(lib().melinoe_moe_last_call_used_gemm(self._h))
+    def ffn_launch_times_ms(self, capacity: int = 65536):
+        """Per-launch times (ms) of the timed FFN launches since the last ffn_time_ms(), in launch order."""
+        import numpy as np
+        buf = np.empty(capacity, np.float32)
+        n = C.c_int(0)
+        self._ck(lib().melinoe_moe_ffn_launch_times_ms(self._h, buf.ctypes.data, capacity, C.byref(n)),
+                 "melinoe_moe_ffn_launch_times_ms")
+        return buf[: min(n.value, capacity)].copy()
 
     def transfer_time_ms(self):
         ms = C.c_double(0.0)

@@ -30,6 +30,15 @@ using namespace melinoe;
 namespace melinoe {
 
 static std::atomic<long long> g_launches{0};
+// Test hook (melinoe_debug_fail_host_copy): when positive, counts down once per host-issued expert copy;
+// the copy at which it reaches zero is not issued and reports a failure instead.  Host-side only.
+static std::atomic<int> g_fail_copy_in{0};
+static cudaError_t g_copy_hook()
+{
+    if (g_fail_copy_in.load() > 0 && g_fail_copy_in.fetch_sub(1) == 1)
+        return cudaErrorUnknown;
+    return cudaSuccess;
+}
 static std::atomic<int> g_last_cuda_error{0};
 
 void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
@@ -64,8 +73,10 @@ typedef CUresult (*encode_tiled_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32
 encode_tiled_fn g_encode_tiled = nullptr;
 std::once_flag g_encode_once;
 
-// 2-D bf16 tensor [rows][cols], row-major, 128-byte swizzle, box of box_rows x 64 columns.
-bool encode_map(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows, uint32_t box_rows)
+// 2-D bf16 tensor [rows][cols] with rows pitch_bytes apart, box of box_rows x 64 columns; with or
+// without the 128-byte swizzle (the expert blobs are stored already permuted, see melinoe_moe_pack_expert).
+bool encode_map(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows, uint64_t pitch_bytes, uint32_t box_rows,
+                bool swizzle)
 {
     std::call_once(g_encode_once, [] {
         cudaDriverEntryPointQueryResult qr;
@@ -78,12 +89,22 @@ bool encode_map(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows, 
     if (!g_encode_tiled || rows == 0)
         return false;
     const cuuint64_t dims[2] = {cols, rows};
-    const cuuint64_t strides[1] = {cols * 2};
+    const cuuint64_t strides[1] = {pitch_bytes};
     const cuuint32_t box[2] = {64, box_rows};
     const cuuint32_t estr[2] = {1, 1};
     return g_encode_tiled(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// The three views of expert blobs that lie back to back from `base` (n_rows = experts * F rows f):
+// W_g rows, W_u rows (boxes of 128 rows), W_d^T rows (boxes of 64 rows), all d columns at a pitch of 6 d bytes.
+bool encode_weight_maps(CUtensorMap *m3, const void *base, int d, uint64_t n_rows)
+{
+    const char *b = static_cast<const char *>(base);
+    const uint64_t pitch = (uint64_t)6 * d;
+    return encode_map(m3 + 0, b, d, n_rows, pitch, 128, false) && encode_map(m3 + 1, b + (size_t)2 * d, d, n_rows, pitch, 128, false) &&
+           encode_map(m3 + 2, b + (size_t)4 * d, d, n_rows, pitch, 64, false);
 }
 
 double now_s()
@@ -97,10 +118,20 @@ struct TimedPair {
 
 }  // namespace
 
+// Scratch of one forward call.  idx .. tok_of_sorted: routing and gather tables; yacc: the decode
+// kernel's output accumulator [<= 8 tokens][d] (64-bit words, all zero between launches); ybuf: fp32
+// sums of a call that is computed in several launches.
+struct Scratch {
+    int32_t *idx = nullptr, *perm = nullptr, *inv_pos = nullptr, *tok_of_sorted = nullptr;
+    float *gate = nullptr, *logits = nullptr, *ybuf = nullptr;
+    long long *yacc = nullptr;
+    int cap_tokens = 0;
+};
+
 struct melinoe_moe {
     int d = 0, F = 0, E = 0, k = 0, C = 0, device = 0, n_sms = 0;
     size_t expert_bytes = 0, slot_stride = 0;
-    FfnLaunchCfg cfg{};
+    DecLaunchCfg cfg{};
 
     // device memory owned by the handle
     char *slots = nullptr;
@@ -110,18 +141,18 @@ struct melinoe_moe {
     DevPlan *plan = nullptr;
     int *err_word = nullptr;
     const char **shared_dev = nullptr;
+    const char **host_dev = nullptr;       // [E]: the host store's blobs as the device sees them (null: not readable)
+    bool pull_ok = false;                  // the decode kernel may read missed experts straight from the host store
 
-    // scratch sized for cap_tokens
-    int cap_tokens = 0, cap_shared = -1, vr_capacity = 0;
-    int32_t *idx = nullptr, *perm = nullptr, *inv_pos = nullptr, *tok_of_sorted = nullptr;
-    float *gate = nullptr, *logits = nullptr, *zbuf = nullptr;
-    uint16_t *hbuf = nullptr;
-    unsigned *sync = nullptr;
+    // per-call scratch: the handle's own (sized for cap_tokens), and whichever the most recent call used
+    Scratch own{}, last{};
+    int cap_shared = -1;
+    float *zbuf = nullptr;                 // grouped-GEMM path: expert outputs [sorted rows][d] fp32
+    unsigned *sync = nullptr;              // counter of the decode kernel's rare "who is last" step (zero between launches)
     unsigned long long *trace = nullptr;   // borrowed; see melinoe_moe_set_trace
-    VrRec *vrs = nullptr;
     uint16_t *stage_in = nullptr, *stage_out = nullptr;
     // grouped-GEMM path (calls of more than 8 tokens): gathered activations, h, tensor maps
-    bool gemm_ok = false, pair_ok = false, last_used_gemm = false, last_used_pair = false;
+    bool gemm_ok = false, last_used_gemm = false;
     uint16_t *xs = nullptr, *hs = nullptr;
     CUtensorMap *maps_dev = nullptr;
     CUtensorMap maps_host[kMapCount];
@@ -188,26 +219,25 @@ int gmax_for(const melinoe_moe *h, int T)
 
 void free_scratch(melinoe_moe *h)
 {
-    cudaFree(h->idx);
-    cudaFree(h->perm);
-    cudaFree(h->inv_pos);
-    cudaFree(h->tok_of_sorted);
-    cudaFree(h->gate);
-    cudaFree(h->logits);
+    Scratch &o = h->own;
+    cudaFree(o.idx);
+    cudaFree(o.perm);
+    cudaFree(o.inv_pos);
+    cudaFree(o.tok_of_sorted);
+    cudaFree(o.gate);
+    cudaFree(o.logits);
+    cudaFree(o.yacc);
+    cudaFree(o.ybuf);
     cudaFree(h->zbuf);
-    cudaFree(h->hbuf);
-    cudaFree(h->vrs);
     cudaFree(h->stage_in);
     cudaFree(h->stage_out);
     cudaFree(h->xs);
     cudaFree(h->hs);
     h->xs = h->hs = nullptr;
-    h->idx = h->perm = h->inv_pos = h->tok_of_sorted = nullptr;
-    h->gate = h->logits = h->zbuf = nullptr;
-    h->hbuf = nullptr;
-    h->vrs = nullptr;
+    o = Scratch{};
+    h->last = Scratch{};
+    h->zbuf = nullptr;
     h->stage_in = h->stage_out = nullptr;
-    h->cap_tokens = 0;
 }
 
 int wait_idle(melinoe_moe *h)
@@ -250,41 +280,39 @@ int wait_for_plan(melinoe_moe *h, uint32_t seq)
 
 int ensure_capacity(melinoe_moe *h, int T)
 {
-    if (T <= h->cap_tokens && h->cap_shared == h->n_shared)
+    if (T <= h->own.cap_tokens && h->cap_shared == h->n_shared)
         return MELINOE_OK;
     int rc = wait_idle(h);
     if (rc != MELINOE_OK)
         return rc;
     CU_TRY(cudaDeviceSynchronize());
-    const int cap = T > h->cap_tokens ? T : h->cap_tokens;
+    const int cap = T > h->own.cap_tokens ? T : h->own.cap_tokens;
     free_scratch(h);
+    Scratch &o = h->own;
     const size_t pairs = (size_t)cap * h->k;
     const size_t sorted = pairs + (size_t)h->n_shared * cap;
-    const int vr_cap = (int)(pairs / kTokPerVr) + h->E + h->n_shared * (cap / kTokPerVr + 1) + 8;
-    const size_t fpad = ((size_t)h->F + 255) / 256 * 256;
-    const size_t hbytes = (size_t)vr_cap * kTokPerVr * fpad * 2;
-    CU_TRY(cudaMalloc(&h->idx, pairs * 4));
-    CU_TRY(cudaMalloc(&h->gate, pairs * 4));
-    CU_TRY(cudaMalloc(&h->logits, (size_t)cap * h->E * 4));
-    CU_TRY(cudaMalloc(&h->perm, sorted * 4));
-    CU_TRY(cudaMalloc(&h->inv_pos, pairs * 4));
-    CU_TRY(cudaMalloc(&h->tok_of_sorted, sorted * 4));
-    CU_TRY(cudaMalloc(&h->vrs, (size_t)vr_cap * sizeof(VrRec)));
-    CU_TRY(cudaMalloc(&h->zbuf, sorted * h->d * sizeof(float)));
-    CU_TRY(cudaMalloc(&h->hbuf, hbytes));
-    CU_TRY(cudaMemset(h->hbuf, 0, hbytes));   // the padding of every h row stays zero for good
+    const int launch_tokens = cap < kTokPerVr ? cap : kTokPerVr;
+    CU_TRY(cudaMalloc(&o.idx, pairs * 4));
+    CU_TRY(cudaMalloc(&o.gate, pairs * 4));
+    CU_TRY(cudaMalloc(&o.logits, (size_t)cap * h->E * 4));
+    CU_TRY(cudaMalloc(&o.perm, sorted * 4));
+    CU_TRY(cudaMalloc(&o.inv_pos, pairs * 4));
+    CU_TRY(cudaMalloc(&o.tok_of_sorted, sorted * 4));
+    CU_TRY(cudaMalloc(&o.yacc, (size_t)launch_tokens * h->d * sizeof(long long)));
+    CU_TRY(cudaMemset(o.yacc, 0, (size_t)launch_tokens * h->d * sizeof(long long)));
+    CU_TRY(cudaMalloc(&o.ybuf, (size_t)cap * h->d * sizeof(float)));
     CU_TRY(cudaMalloc(&h->stage_in, (size_t)cap * h->d * 2));
     CU_TRY(cudaMalloc(&h->stage_out, (size_t)cap * h->d * 2));
     if (h->gemm_ok && cap > kTokPerVr) {
+        CU_TRY(cudaMalloc(&h->zbuf, sorted * h->d * sizeof(float)));
         CU_TRY(cudaMalloc(&h->xs, sorted * h->d * 2));
         CU_TRY(cudaMalloc(&h->hs, sorted * h->F * 2));
-        if (!encode_map(&h->maps_host[kMapXs], h->xs, h->d, sorted, 128) ||
-            !encode_map(&h->maps_host[kMapHs], h->hs, h->F, sorted, 128))
+        if (!encode_map(&h->maps_host[kMapXs], h->xs, h->d, sorted, (uint64_t)h->d * 2, 128, true) ||
+            !encode_map(&h->maps_host[kMapHs], h->hs, h->F, sorted, (uint64_t)h->F * 2, 128, true))
             return MELINOE_ERR_CUDA;
         CU_TRY(cudaMemcpy(h->maps_dev, h->maps_host, sizeof(h->maps_host), cudaMemcpyHostToDevice));
     }
-    h->vr_capacity = vr_cap;
-    h->cap_tokens = cap;
+    o.cap_tokens = cap;
     h->cap_shared = h->n_shared;
     return MELINOE_OK;
 }
@@ -325,11 +353,45 @@ int melinoe_moe_pack_expert(int d, int F, const void *wg_, const void *wu_, cons
 {
     if (d <= 0 || F <= 0 || !wg_ || !wu_ || !wd_ || !blob_)
         return MELINOE_ERR_INVALID;
-    const size_t m = (size_t)d * F * 2;
-    char *blob = static_cast<char *>(blob_);
-    std::memcpy(blob, wg_, m);
-    std::memcpy(blob + m, wu_, m);
-    std::memcpy(blob + 2 * m, wd_, m);
+    if (d % 64 != 0)
+        return MELINOE_ERR_UNSUPPORTED;
+    const uint16_t *wg = static_cast<const uint16_t *>(wg_), *wu = static_cast<const uint16_t *>(wu_);
+    const uint16_t *wd = static_cast<const uint16_t *>(wd_);
+    uint16_t *blob = static_cast<uint16_t *>(blob_);
+    // per hidden unit f: W_g[f][:] | W_u[f][:] | W_d[:][f]; 8-element (16-byte) pieces of every 64-element
+    // (128-byte) group at position (piece xor (f mod 8))
+    for (int f = 0; f < F; ++f) {
+        uint16_t *row = blob + (size_t)f * 3 * d;
+        const int x = f & 7;
+        for (int j = 0; j < d / 8; ++j) {
+            const int pj = (j & ~7) | ((j ^ x) & 7);
+            std::memcpy(row + (size_t)pj * 8, wg + (size_t)f * d + (size_t)j * 8, 16);
+            std::memcpy(row + d + (size_t)pj * 8, wu + (size_t)f * d + (size_t)j * 8, 16);
+        }
+    }
+    // W_d transposed in 8 x 8 blocks (8 output columns c by 8 hidden units f), so that both the reads and
+    // the writes move 16 contiguous bytes; F need not be a multiple of 8 here, the tail goes element-wise
+    const int F8 = F & ~7;
+    for (int j = 0; j < d / 8; ++j) {
+        for (int f0 = 0; f0 < F8; f0 += 8) {
+            uint16_t t[8][8];
+            for (int i = 0; i < 8; ++i)
+                std::memcpy(t[i], wd + (size_t)(j * 8 + i) * F + f0, 16);
+            for (int r = 0; r < 8; ++r) {
+                const int f = f0 + r;
+                const int pj = (j & ~7) | ((j ^ (f & 7)) & 7);
+                uint16_t *dst = blob + (size_t)f * 3 * d + 2 * (size_t)d + (size_t)pj * 8;
+                for (int i = 0; i < 8; ++i)
+                    dst[i] = t[i][r];
+            }
+        }
+        for (int f = F8; f < F; ++f) {
+            const int pj = (j & ~7) | ((j ^ (f & 7)) & 7);
+            uint16_t *dst = blob + (size_t)f * 3 * d + 2 * (size_t)d + (size_t)pj * 8;
+            for (int i = 0; i < 8; ++i)
+                dst[i] = wd[(size_t)(j * 8 + i) * F + f];
+        }
+    }
     return MELINOE_OK;
 }
 
@@ -410,7 +472,7 @@ int melinoe_moe_create(int d, int F, int E, int k, int C, melinoe_moe_t **out)
     *out = nullptr;
     if (d <= 0 || F <= 0 || E <= 0 || k <= 0 || C <= 0 || k > E || C < k || C > E)
         return MELINOE_ERR_INVALID;
-    if (d % 256 != 0 || d > 8192 || F % kUnitRows != 0 || E > kMaxExperts || k > 32)
+    if (!ffn_decode_supported(d, F) || E > kMaxExperts || k > 32)
         return MELINOE_ERR_UNSUPPORTED;
     {
         int dev = 0;
@@ -442,8 +504,7 @@ int melinoe_moe_create(int d, int F, int E, int k, int C, melinoe_moe_t **out)
     if (prop.major != 10)
         return fail(MELINOE_ERR_UNSUPPORTED);
     h->n_sms = prop.multiProcessorCount;
-    if (!prop.cooperativeLaunch ||
-        ffn_stream_configure(h->n_sms, prop.sharedMemPerBlockOptin, &h->cfg) != cudaSuccess) {
+    if (ffn_decode_configure(h->n_sms, prop.sharedMemPerBlockOptin, &h->cfg) != cudaSuccess) {
         (void)cudaGetLastError();
         return fail(MELINOE_ERR_UNSUPPORTED);
     }
@@ -457,9 +518,11 @@ int melinoe_moe_create(int d, int F, int E, int k, int C, melinoe_moe_t **out)
     CR(cudaMalloc(&h->cache, sizeof(DevCache)));
     CR(cudaMalloc(&h->plan, sizeof(DevPlan)));
     CR(cudaMalloc(&h->err_word, 256));
-    CR(cudaMalloc(&h->sync, sizeof(unsigned) * (2 * (kMaxGroups + 1) + 1)));
-    CR(cudaMemset(h->sync, 0, sizeof(unsigned) * (2 * (kMaxGroups + 1) + 1)));
+    CR(cudaMalloc(&h->sync, 256));
+    CR(cudaMemset(h->sync, 0, 256));
     CR(cudaMalloc(&h->shared_dev, sizeof(char *) * kMaxShared));
+    CR(cudaMalloc(&h->host_dev, sizeof(char *) * kMaxExperts));
+    CR(cudaMemset(h->host_dev, 0, sizeof(char *) * kMaxExperts));
     CR(cudaMalloc(&h->stage_stats, sizeof(melinoe_moe_stats)));
     CR(cudaMemset(h->err_word, 0, 256));
     CR(cudaMemset(h->plan, 0, sizeof(DevPlan)));
@@ -473,17 +536,18 @@ int melinoe_moe_create(int d, int F, int E, int k, int C, melinoe_moe_t **out)
     CR(cudaEventCreateWithFlags(&h->ev_last, cudaEventDisableTiming));
     CR(cudaEventCreateWithFlags(&h->ev_plan, cudaEventDisableTiming));
     CR(cudaEventCreateWithFlags(&h->ev_arrive, cudaEventDisableTiming));
+    // one event per compute group a call can have, made here so that no forward call ever creates one
+    h->ev_group.assign(kMaxGroups + 1, nullptr);
+    for (auto &e : h->ev_group)
+        CR(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
     // grouped GEMM for calls of many tokens: the slots are contiguous, so one tensor map per view
-    // (rows of d elements: W_g, W_u; rows of F elements: W_d) covers every slot
+    // (W_g rows, W_u rows, W_d^T rows) covers every slot
     std::memset(h->maps_host, 0, sizeof(h->maps_host));
     if (ffn_gemm_supported(d, F) && h->slot_stride == h->expert_bytes && ffn_gemm_configure() == cudaSuccess) {
         CR(cudaMalloc(&h->maps_dev, sizeof(h->maps_host)));
-        if (encode_map(&h->maps_host[kMapSlotsD], h->slots, d, (uint64_t)C * 3 * F, 128) &&
-            encode_map(&h->maps_host[kMapSlotsF], h->slots, F, (uint64_t)C * 3 * d, 256) &&
-            encode_map(&h->maps_host[kMapSlotsF128], h->slots, F, (uint64_t)C * 3 * d, 128)) {
+        if (encode_weight_maps(&h->maps_host[kMapSlotsG], h->slots, d, (uint64_t)C * F)) {
             CR(cudaMemcpy(h->maps_dev, h->maps_host, sizeof(h->maps_host), cudaMemcpyHostToDevice));
             h->gemm_ok = true;
-            h->pair_ok = ffn_gemm_pair_configure() == cudaSuccess && (h->n_sms & ~1) >= 2;
         }
     }
     (void)cudaGetLastError();
@@ -516,6 +580,7 @@ int melinoe_moe_destroy(melinoe_moe_t *h)
             cudaEventDestroy(h->ev_q4_expanded[i]);
     }
     cudaFree(h->shared_dev);
+    cudaFree(h->host_dev);
     cudaFree(h->maps_dev);
     cudaFree(h->stage_stats);
     if (h->hplan)
@@ -576,6 +641,22 @@ int melinoe_moe_register_host_experts(melinoe_moe_t *h, const void *const *ptrs,
     int rc = wait_idle(h);
     if (rc != MELINOE_OK)
         return rc;
+    // the store as the device sees it: the decode kernel reads missed experts from there itself
+    const char *dev_view[kMaxExperts] = {nullptr};
+    bool all = true;
+    for (int e = 0; e < h->E; ++e) {
+        void *dp = nullptr;
+        if (cudaHostGetDevicePointer(&dp, const_cast<void *>(ptrs[e]), 0) != cudaSuccess || !dp || !aligned16(dp)) {
+            (void)cudaGetLastError();
+            all = false;
+            break;
+        }
+        dev_view[e] = static_cast<const char *>(dp);
+    }
+    if (!all)
+        std::memset(dev_view, 0, sizeof dev_view);
+    CU_TRY(cudaMemcpy(h->host_dev, dev_view, sizeof dev_view, cudaMemcpyHostToDevice));
+    h->pull_ok = all && std::getenv("MELINOE_MOE_HOST_COPIES") == nullptr;
     for (int e = 0; e < h->E; ++e)
         h->host_experts[e] = ptrs[e];
     h->store_q4 = false;
@@ -612,6 +693,8 @@ int melinoe_moe_register_host_experts_q4(melinoe_moe_t *h, const void *const *pt
     }
     for (int e = 0; e < h->E; ++e)
         h->host_experts[e] = ptrs[e];
+    CU_TRY(cudaMemset(h->host_dev, 0, sizeof(char *) * kMaxExperts));
+    h->pull_ok = false;     // 4-bit blobs are expanded into the bf16 slots by a kernel behind the copy
     h->store_q4 = true;
     h->q4_bytes = qb;
     return MELINOE_OK;
@@ -638,9 +721,7 @@ int melinoe_moe_register_shared_experts(melinoe_moe_t *h, int n_shared, const vo
     CU_TRY(cudaMemcpy(h->shared_dev, tmp, sizeof tmp, cudaMemcpyHostToDevice));
     if (h->gemm_ok) {
         for (int s = 0; s < n_shared; ++s)
-            if (!encode_map(&h->maps_host[kMapShared0 + 2 * s], ptrs[s], h->d, (uint64_t)3 * h->F, 128) ||
-                !encode_map(&h->maps_host[kMapShared0 + 2 * s + 1], ptrs[s], h->F, (uint64_t)3 * h->d, 256) ||
-                !encode_map(&h->maps_host[kMapSharedF128 + s], ptrs[s], h->F, (uint64_t)3 * h->d, 128))
+            if (!encode_weight_maps(&h->maps_host[kMapShared0 + 3 * s], ptrs[s], h->d, (uint64_t)h->F))
                 return MELINOE_ERR_CUDA;
         CU_TRY(cudaMemcpy(h->maps_dev, h->maps_host, sizeof(h->maps_host), cudaMemcpyHostToDevice));
     }
@@ -666,29 +747,72 @@ int melinoe_moe_reserve(melinoe_moe_t *h, int max_tokens)
     return ensure_capacity(h, max_tokens);
 }
 
-int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_dev, int T, void *out_dev,
-                        melinoe_moe_stats *stats_dev)
+}  // extern "C"
+
+namespace {
+
+// Event pair for kernel timing, reused from the handle's pool.
+int take_pair(melinoe_moe *h, TimedPair *tp)
 {
-    if (!h || T < 0)
-        return MELINOE_ERR_INVALID;
-    if (T == 0)
+    if (!h->free_pairs.empty()) {
+        *tp = h->free_pairs.back();
+        h->free_pairs.pop_back();
         return MELINOE_OK;
-    if (!hidden_dev || !out_dev || !aligned16(hidden_dev) || !aligned16(out_dev))
-        return MELINOE_ERR_INVALID;
-    if (!h->w_router || !h->host_experts[0])
-        return MELINOE_ERR_STATE;
-    if (h->sticky.load() != MELINOE_OK)
-        return h->sticky.load();
-    int rc = ensure_capacity(h, T);
-    if (rc != MELINOE_OK)
-        return rc;
+    }
+    CU_TRY(cudaEventCreate(&tp->a));
+    CU_TRY(cudaEventCreate(&tp->b));
+    return MELINOE_OK;
+}
+
+// One launch of the decode FFN kernel: compute group `group` (or -1: the whole call, missed experts
+// read from the host store) for tokens [8 * chunk, 8 * chunk + 8) of the call.
+int launch_decode(melinoe_moe *h, cudaStream_t s, const Scratch &sc, const void *hidden_dev, void *out_dev, int T,
+                  int group, int chunk, bool first_of_call)
+{
+    const int tokens = T - chunk * kTokPerVr < kTokPerVr ? T - chunk * kTokPerVr : kTokPerVr;
+    DecGeometry geo;
+    if (ffn_decode_geometry(h->cfg, h->d, h->F, tokens, 0, &geo) != cudaSuccess)
+        return MELINOE_ERR_UNSUPPORTED;
+    DecParams dp;
+    dp.plan = h->plan;
+    dp.x = static_cast<const uint16_t *>(hidden_dev);
+    dp.idx = sc.idx;
+    dp.gate = sc.gate;
+    dp.yacc = sc.yacc;
+    dp.ybuf = sc.ybuf;
+    dp.out = static_cast<uint16_t *>(out_dev);
+    dp.sync = h->sync;
+    dp.call_seq = h->call_seq;
+    dp.err = h->err_word;
+    dp.trace = h->trace;
+    dp.d = h->d;
+    dp.F = h->F;
+    dp.E = h->E;
+    dp.k = h->k;
+    dp.T = T;
+    dp.n_shared = h->n_shared;
+    dp.group = group;
+    dp.chunk = chunk;
+    dp.n_chunks = (T + kTokPerVr - 1) / kTokPerVr;
+    dp.write_back = 1;
+    dp.wait_prior = first_of_call ? 0 : 1;
+    dp.fmt = 0;
+    CU_TRY(launch_ffn_decode(s, h->cfg, geo, dp));
+    return MELINOE_OK;
+}
+
+// The call itself, on the scratch it is given.
+int forward_on(melinoe_moe *h, const Scratch &sc, void *cuda_stream, const void *hidden_dev, int T, void *out_dev,
+               melinoe_moe_stats *stats_dev)
+{
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     const uint32_t gmax = (uint32_t)gmax_for(h, T);
     h->call_seq += 1;
     h->last_T = T;
+    h->last = sc;
 
     PlanParams pp;
-    pp.idx = h->idx;
+    pp.idx = sc.idx;
     pp.T = T;
     pp.k = h->k;
     pp.E = h->E;
@@ -696,60 +820,61 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
     pp.n_shared = h->n_shared;
     pp.cache = h->cache;
     pp.plan = h->plan;
-    pp.vrs = h->vrs;
     pp.slots = h->slots;
     pp.slot_stride = h->slot_stride;
     pp.shared_blobs = h->shared_dev;
-    pp.perm = h->perm;
-    pp.inv_pos = h->inv_pos;
-    pp.tok_of_sorted = h->tok_of_sorted;
+    pp.host_blobs = h->host_dev;
+    pp.perm = sc.perm;
+    pp.inv_pos = sc.inv_pos;
+    pp.tok_of_sorted = sc.tok_of_sorted;
     pp.hplan = h->hplan;
-    pp.sync = h->sync;
     pp.gmax = gmax;
     pp.call_seq = h->call_seq;
     pp.policy = h->policy;
     pp.gamma = h->gamma;
     pp.stats = stats_dev;
     pp.expert_bytes = h->store_q4 ? h->q4_bytes : h->expert_bytes;   // bytes one miss moves over the host link
-    pp.vr_capacity = h->vr_capacity;
-    if (route_plan_small_supported(T, h->k, h->d)) {
+    const bool small = route_plan_small_supported(T, h->k, h->d);
+    if (small) {
         CU_TRY(launch_route_plan_small(s, static_cast<const uint16_t *>(hidden_dev), h->w_router, h->bias, h->token_seq,
-                                       h->d, h->idx, h->gate, h->logits, pp));
+                                       h->d, sc.idx, sc.gate, sc.logits, pp));
     } else {
         CU_TRY(launch_router(s, static_cast<const uint16_t *>(hidden_dev), h->w_router, h->bias, h->token_seq, T, h->d,
-                             h->E, h->k, h->idx, h->gate, h->logits));
+                             h->E, h->k, sc.idx, sc.gate, sc.logits));
         CU_TRY(launch_plan(s, pp));
     }
-    CU_TRY(cudaEventRecord(h->ev_plan, s));
-
-    FfnParams fp;
-    fp.plan = h->plan;
-    fp.vrs = h->vrs;
-    fp.x = static_cast<const uint16_t *>(hidden_dev);
-    fp.gate = h->gate;
-    fp.hbuf = h->hbuf;
-    fp.zbuf = h->zbuf;
-    fp.out = static_cast<uint16_t *>(out_dev);
-    fp.sync = h->sync;
-    fp.err = h->err_word;
-    fp.trace = h->trace;
-    fp.d = h->d;
-    fp.F = h->F;
-    fp.Fpad = (h->F + 255) / 256 * 256;
-    fp.E = h->E;
-    fp.k = h->k;
-    fp.T = T;
-    fp.n_shared = h->n_shared;
-    FfnGeometry geo;
-    if (ffn_stream_geometry(h->cfg, h->d, h->F, T, &geo) != cudaSuccess)
-        return MELINOE_ERR_UNSUPPORTED;
     // calls of more than 8 tokens go through the grouped GEMM (where the shapes allow it)
-    const bool use_gemm = h->gemm_ok && T > kTokPerVr && h->xs != nullptr;
-    // Alternative for calls with many tokens per expert: 256-token tiles on CTA pairs (each B tile staged
-    // once per 256 rows).  Measured no faster than single CTAs (Phi-3.5-shaped prompt 1097 against
-    // 1126 TFLOP/s, DeepSeek-shaped 1026 against 1015), so it runs only when MELINOE_MOE_PAIR is set.
-    const bool use_pair = use_gemm && h->pair_ok && (long long)T * h->k >= (long long)192 * h->E &&
-                          std::getenv("MELINOE_MOE_PAIR") != nullptr;
+    const bool use_gemm = h->gemm_ok && T > kTokPerVr && h->xs != nullptr && sc.idx == h->own.idx;
+    const int n_chunks = (T + kTokPerVr - 1) / kTokPerVr;
+    h->last_used_gemm = use_gemm;
+
+    // ---- everything on the device: the decode kernel fetches the missed experts itself, the host is
+    // not in the path at all and returns at once (the call's cache decisions are in stats_dev)
+    if (!use_gemm && h->pull_ok) {
+        for (int c = 0; c < n_chunks; ++c) {
+            TimedPair tp{nullptr, nullptr};
+            if (h->timing) {
+                int rc = take_pair(h, &tp);
+                if (rc != MELINOE_OK)
+                    return rc;
+                CU_TRY(cudaEventRecord(tp.a, s));
+            }
+            int rc = launch_decode(h, s, sc, hidden_dev, out_dev, T, -1, c, c == 0);
+            if (rc != MELINOE_OK)
+                return rc;
+            if (h->timing) {
+                CU_TRY(cudaEventRecord(tp.b, s));
+                h->timed.push_back(tp);
+            }
+        }
+        CU_TRY(cudaEventRecord(h->ev_last, s));
+        h->has_last = true;
+        return MELINOE_OK;
+    }
+
+    // ---- transfers issued by the host: group 0 is queued at once, the miss waves follow as the host
+    // learns of them
+    CU_TRY(cudaEventRecord(h->ev_plan, s));
     GemmParams gp;
     gp.plan = h->plan;
     gp.maps = h->maps_dev;
@@ -760,35 +885,27 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
     gp.F = h->F;
     gp.E = h->E;
     gp.n_shared = h->n_shared;
-    h->last_used_gemm = use_gemm;
-    h->last_used_pair = use_pair;
     if (use_gemm)
-        CU_TRY(launch_gather_rows(s, h->plan, static_cast<const uint16_t *>(hidden_dev), h->tok_of_sorted, h->xs, h->d,
+        CU_TRY(launch_gather_rows(s, h->plan, static_cast<const uint16_t *>(hidden_dev), sc.tok_of_sorted, h->xs, h->d,
                                   T * h->k + h->n_shared * T, h->n_sms));
     auto launch_group = [&](int g) -> int {
         TimedPair tp{nullptr, nullptr};
         if (h->timing) {
-            if (!h->free_pairs.empty()) {
-                tp = h->free_pairs.back();
-                h->free_pairs.pop_back();
-            } else {
-                CU_TRY(cudaEventCreate(&tp.a));
-                CU_TRY(cudaEventCreate(&tp.b));
-            }
+            int rc = take_pair(h, &tp);
+            if (rc != MELINOE_OK)
+                return rc;
             CU_TRY(cudaEventRecord(tp.a, s));
         }
         if (use_gemm) {
             gp.group = g;
-            if (use_pair) {
-                CU_TRY(launch_ffn_gemm_pair(s, 1, h->n_sms, gp));
-                CU_TRY(launch_ffn_gemm_pair(s, 2, h->n_sms, gp));
-            } else {
-                CU_TRY(launch_ffn_gemm(s, 1, h->n_sms, gp));
-                CU_TRY(launch_ffn_gemm(s, 2, h->n_sms, gp));
-            }
+            CU_TRY(launch_ffn_gemm(s, 1, h->n_sms, gp));
+            CU_TRY(launch_ffn_gemm(s, 2, h->n_sms, gp));
         } else {
-            fp.group = g;
-            CU_TRY(launch_ffn_stream(s, h->cfg, geo, fp));
+            for (int c = 0; c < n_chunks; ++c) {
+                int rc = launch_decode(h, s, sc, hidden_dev, out_dev, T, g, c, g == 0 && c == 0);
+                if (rc != MELINOE_OK)
+                    return rc;
+            }
         }
         if (h->timing) {
             CU_TRY(cudaEventRecord(tp.b, s));
@@ -796,17 +913,23 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
         }
         return MELINOE_OK;
     };
+    // From here on part of the call is queued: a failure must leave the stream and the handle in a
+    // state the caller can see (ev_last recorded, the error sticky until the cache is reset).
+    auto fail = [&](int code) -> int {
+        h->sticky.store(code);
+        (void)cudaEventRecord(h->ev_last, s);
+        h->has_last = true;
+        return code;
+    };
     // group 0 (experts resident at call entry, shared experts) goes out before the plan is known
-    rc = launch_group(0);
+    int rc = launch_group(0);
     if (rc != MELINOE_OK)
-        return rc;
+        return fail(rc);
 
     // the miss queue of this call
     rc = wait_for_plan(h, h->call_seq);
-    if (rc != MELINOE_OK) {
-        h->sticky.store(rc);
-        return rc;
-    }
+    if (rc != MELINOE_OK)
+        return fail(rc);
     const volatile HostPlan &vhp = *h->hplan;
     int n_miss = vhp.hdr.n_miss, n_groups = vhp.hdr.n_groups;
     if (vhp.hdr.status != MELINOE_OK || n_miss < 0 || n_miss > h->E || n_groups < 1 || n_groups > (int)gmax)
@@ -828,10 +951,8 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
                 hp.miss[i] = m;
                 break;
             }
-            if (now_s() - t0 > 10.0) {
-                h->sticky.store(MELINOE_ERR_TIMEOUT);
-                return MELINOE_ERR_TIMEOUT;
-            }
+            if (now_s() - t0 > 10.0)
+                return fail(MELINOE_ERR_TIMEOUT);
         }
     }
     // which groups must signal their completion to the copy stream
@@ -839,109 +960,123 @@ int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_
     for (int i = 0; i < n_miss; ++i)
         if (hp.miss[i].dep_group >= 0 && hp.miss[i].dep_group <= kMaxGroups)
             need_done[hp.miss[i].dep_group] = true;
-    auto group_event = [&](int g) -> cudaEvent_t {
-        while ((int)h->ev_group.size() <= g) {
-            cudaEvent_t e = nullptr;
-            if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess)
-                return nullptr;
-            h->ev_group.push_back(e);
-        }
-        return h->ev_group[g];
-    };
-    if (need_done[0]) {
-        cudaEvent_t e = group_event(0);
-        if (!e)
-            return cuda_fail(cudaGetLastError());
-        CU_TRY(cudaEventRecord(e, s));
-    }
+    if (need_done[0])
+        CU_TRY(cudaEventRecord(h->ev_group[0], s));
     int i = 0;
     for (int g = 1; g < n_groups; ++g) {
         TimedPair ctp{nullptr, nullptr};
         bool wave_started = false;
         for (; i < n_miss && hp.miss[i].group == g; ++i) {
             const HostMiss m = hp.miss[i];
-            if (m.expert < 0 || m.expert >= h->E || m.slot < 0 || m.slot >= h->C || m.dep_group >= g) {
-                h->sticky.store(MELINOE_ERR_STATE);
-                return MELINOE_ERR_STATE;
-            }
+            if (m.expert < 0 || m.expert >= h->E || m.slot < 0 || m.slot >= h->C || m.dep_group >= g)
+                return fail(MELINOE_ERR_STATE);
             // the slot may still feed an earlier compute group of this call: whoever writes the slot
             // (the copy itself, or the expansion kernel of a 4-bit store) waits for that group
             cudaStream_t slot_writer = h->store_q4 ? h->dq_stream : h->copy_stream;
+            cudaError_t ce = cudaSuccess;
             if (m.dep_group >= 0)
-                CU_TRY(cudaStreamWaitEvent(slot_writer, h->ev_group[m.dep_group], 0));
-            if (h->timing && !wave_started) {
-                if (!h->free_pairs.empty()) {
-                    ctp = h->free_pairs.back();
-                    h->free_pairs.pop_back();
-                } else {
-                    CU_TRY(cudaEventCreate(&ctp.a));
-                    CU_TRY(cudaEventCreate(&ctp.b));
-                }
-                CU_TRY(cudaEventRecord(ctp.a, h->copy_stream));
+                ce = cudaStreamWaitEvent(slot_writer, h->ev_group[m.dep_group], 0);
+            if (ce == cudaSuccess && h->timing && !wave_started) {
+                rc = take_pair(h, &ctp);
+                if (rc != MELINOE_OK)
+                    return fail(rc);
+                ce = cudaEventRecord(ctp.a, h->copy_stream);
                 wave_started = true;
             }
             if (h->timing)
                 h->timed_copy_bytes += h->store_q4 ? h->q4_bytes : h->expert_bytes;
-            if (h->store_q4) {
+            if (ce == cudaSuccess && h->store_q4) {
                 // the 4-bit blob travels into one of two staging buffers; a kernel on a stream of its own
                 // expands it into the slot, so the next blob is on the link meanwhile
                 const unsigned b = h->q4_turn++ & 1u;
                 char *stage = h->q4_stage + (size_t)b * h->q4_bytes;
                 if (h->q4_used[b])
-                    CU_TRY(cudaStreamWaitEvent(h->copy_stream, h->ev_q4_expanded[b], 0));
-                CU_TRY(cudaMemcpyAsync(stage, h->host_experts[m.expert], h->q4_bytes, cudaMemcpyHostToDevice,
-                                       h->copy_stream));
-                CU_TRY(cudaEventRecord(h->ev_q4_copied[b], h->copy_stream));
-                CU_TRY(cudaStreamWaitEvent(h->dq_stream, h->ev_q4_copied[b], 0));
-                CU_TRY(launch_dequant_q4(h->dq_stream, stage, h->slots + (size_t)m.slot * h->slot_stride, h->d, h->F,
-                                         h->n_sms));
-                CU_TRY(cudaEventRecord(h->ev_q4_expanded[b], h->dq_stream));
+                    ce = cudaStreamWaitEvent(h->copy_stream, h->ev_q4_expanded[b], 0);
+                if (ce == cudaSuccess)
+                    ce = g_copy_hook();
+                if (ce == cudaSuccess)
+                    ce = cudaMemcpyAsync(stage, h->host_experts[m.expert], h->q4_bytes, cudaMemcpyHostToDevice, h->copy_stream);
+                if (ce == cudaSuccess)
+                    ce = cudaEventRecord(h->ev_q4_copied[b], h->copy_stream);
+                if (ce == cudaSuccess)
+                    ce = cudaStreamWaitEvent(h->dq_stream, h->ev_q4_copied[b], 0);
+                if (ce == cudaSuccess)
+                    ce = launch_dequant_q4(h->dq_stream, stage, h->slots + (size_t)m.slot * h->slot_stride, h->d, h->F, h->n_sms);
+                if (ce == cudaSuccess)
+                    ce = cudaEventRecord(h->ev_q4_expanded[b], h->dq_stream);
                 h->q4_used[b] = true;
-            } else {
-                CU_TRY(cudaMemcpyAsync(h->slots + (size_t)m.slot * h->slot_stride, h->host_experts[m.expert],
-                                       h->expert_bytes, cudaMemcpyHostToDevice, h->copy_stream));
+            } else if (ce == cudaSuccess) {
+                ce = g_copy_hook();
+                if (ce == cudaSuccess)
+                    ce = cudaMemcpyAsync(h->slots + (size_t)m.slot * h->slot_stride, h->host_experts[m.expert], h->expert_bytes,
+                                         cudaMemcpyHostToDevice, h->copy_stream);
             }
+            if (ce != cudaSuccess)
+                return fail(cuda_fail(ce));
         }
         if (wave_started) {
             CU_TRY(cudaEventRecord(ctp.b, h->copy_stream));
             h->timed_copy.push_back(ctp);
         }
-        CU_TRY(cudaEventRecord(h->ev_arrive, h->store_q4 ? h->dq_stream : h->copy_stream));
-        CU_TRY(cudaStreamWaitEvent(s, h->ev_arrive, 0));
+        cudaError_t ce = cudaEventRecord(h->ev_arrive, h->store_q4 ? h->dq_stream : h->copy_stream);
+        if (ce == cudaSuccess)
+            ce = cudaStreamWaitEvent(s, h->ev_arrive, 0);
+        if (ce != cudaSuccess)
+            return fail(cuda_fail(ce));
         rc = launch_group(g);
         if (rc != MELINOE_OK)
-            return rc;
-        if (need_done[g]) {
-            cudaEvent_t e = group_event(g);
-            if (!e)
-                return cuda_fail(cudaGetLastError());
-            CU_TRY(cudaEventRecord(e, s));
-        }
+            return fail(rc);
+        if (need_done[g] && cudaEventRecord(h->ev_group[g], s) != cudaSuccess)
+            return fail(cuda_fail(cudaGetLastError()));
     }
 
     if (use_gemm)
-        CU_TRY(launch_combine_rows(s, h->plan, h->gate, h->inv_pos, h->zbuf, static_cast<uint16_t *>(out_dev), T, h->d,
+        CU_TRY(launch_combine_rows(s, h->plan, sc.gate, sc.inv_pos, h->zbuf, static_cast<uint16_t *>(out_dev), T, h->d,
                                    h->k, h->n_shared, h->n_sms));
     CU_TRY(cudaEventRecord(h->ev_last, s));
     h->has_last = true;
     return MELINOE_OK;
 }
 
-}  // extern "C"
+int check_forward_args(melinoe_moe *h, const void *hidden_dev, int T, void *out_dev)
+{
+    if (!h || T < 0)
+        return MELINOE_ERR_INVALID;
+    if (T == 0)
+        return MELINOE_OK;
+    if (!hidden_dev || !out_dev || !aligned16(hidden_dev) || !aligned16(out_dev))
+        return MELINOE_ERR_INVALID;
+    if (!h->w_router || !h->host_experts[0])
+        return MELINOE_ERR_STATE;
+    if (h->sticky.load() != MELINOE_OK)
+        return h->sticky.load();
+    return MELINOE_OK;
+}
+
+}  // namespace
+
+extern "C" int melinoe_moe_forward(melinoe_moe_t *h, void *cuda_stream, const void *hidden_dev, int T, void *out_dev,
+                                   melinoe_moe_stats *stats_dev)
+{
+    int rc = check_forward_args(h, hidden_dev, T, out_dev);
+    if (rc != MELINOE_OK || T == 0)
+        return rc;
+    rc = ensure_capacity(h, T);
+    if (rc != MELINOE_OK)
+        return rc;
+    return forward_on(h, h->own, cuda_stream, hidden_dev, T, out_dev, stats_dev);
+}
 
 // ---------------------------------------------------------------- forward without allocation
 //
 // Scratch of melinoe_moe_forward_static: one array in the library's device image, shared by every
 // call on the device, instead of per-handle cudaMalloc'd buffers.
 constexpr int kStaticMaxTokens = 8;
-constexpr int kStaticMaxPairs = 16;                         // n_tokens * top_k
-constexpr int kStaticMaxSharedRows = 64;                    // n_shared * n_tokens
-constexpr int kStaticMaxVr = kStaticMaxPairs + kMaxShared;  // one virtual request per routed pair or shared expert
-constexpr int kStaticMaxD = 8192, kStaticMaxF = 16384;
-constexpr size_t kStaticSmall = 16 * 1024;                  // idx, gate, logits, perm, inv_pos, tok_of_sorted, vrs
-constexpr size_t kStaticZ = (size_t)(kStaticMaxPairs + kStaticMaxSharedRows) * kStaticMaxD * sizeof(float);
-constexpr size_t kStaticH = (size_t)kStaticMaxVr * kTokPerVr * kStaticMaxF * 2;
-constexpr size_t kStaticBytes = kStaticSmall + kStaticZ + kStaticH;   // about 8.6 MiB
+constexpr int kStaticMaxPairs = 64;                         // n_tokens * top_k
+constexpr size_t kStaticSmall = 16 * 1024;                  // idx, gate, logits, perm, inv_pos, tok_of_sorted
+constexpr size_t kStaticY = (size_t)kStaticMaxTokens * 4096 * sizeof(float);   // fp32 sums of a call made in several launches
+constexpr size_t kStaticAcc = (size_t)kStaticMaxTokens * 4096 * sizeof(long long);   // fixed-point sums of a launch
+constexpr size_t kStaticBytes = kStaticSmall + kStaticY + kStaticAcc;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];
 
 namespace {
@@ -955,94 +1090,55 @@ std::mutex g_static_mu;
 extern "C" int melinoe_moe_forward_static(melinoe_moe_t *h, void *cuda_stream, const void *hidden_dev, int T,
                                           void *out_dev, melinoe_moe_stats *stats_dev)
 {
-    if (!h || T < 0)
-        return MELINOE_ERR_INVALID;
-    if (T == 0)
-        return MELINOE_OK;
+    int rc = check_forward_args(h, hidden_dev, T, out_dev);
+    if (rc != MELINOE_OK || T == 0)
+        return rc;
     // everything beyond the static scratch's sizes is refused, never served by allocating
-    if (T > kStaticMaxTokens || T * h->k > kStaticMaxPairs || T * h->k > h->C || h->n_shared * T > kStaticMaxSharedRows ||
-        h->d > kStaticMaxD || h->F > kStaticMaxF)
+    if (T > kStaticMaxTokens || T * h->k > kStaticMaxPairs || (size_t)h->n_shared * T + (size_t)T * h->k > 1024 ||
+        (size_t)T * h->d * sizeof(float) > kStaticY)
         return MELINOE_ERR_UNSUPPORTED;
     if (h->timing)
         return MELINOE_ERR_STATE;   // timed calls create events on demand
     if (h->device < 0 || h->device >= kMaxDevices)
         return MELINOE_ERR_UNSUPPORTED;
+    int cur = -1;
+    CU_TRY(cudaGetDevice(&cur));
+    if (cur != h->device)
+        return MELINOE_ERR_STATE;   // the handle's device must be current, as for every call
     unsigned char *base = nullptr;
     {
         std::lock_guard<std::mutex> lk(g_static_mu);
         base = g_static_ptr[h->device];
         if (!base) {
-            // first call on this device (the handle's device must be current, as for every call)
-            int cur = -1;
-            CU_TRY(cudaGetDevice(&cur));
-            if (cur != h->device)
-                return MELINOE_ERR_STATE;
+            // first call on this device: look the array's address up
             void *p = nullptr;
             CU_TRY(cudaGetSymbolAddress(&p, g_static_scratch));
             base = g_static_ptr[h->device] = static_cast<unsigned char *>(p);
         }
     }
-    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-    // carve the scratch: small tables first, then z, then h
+    // carve the scratch: small tables first, then the fp32 sums, then the fixed-point accumulator.  The
+    // tables are written by the call's kernels before they are read; the accumulator must be all zero
+    // when a launch starts: it is (static storage starts out zero) and every launch leaves it so.
     unsigned char *q = base;
     auto take = [&](size_t bytes) {
         unsigned char *r = q;
         q += (bytes + 255) / 256 * 256;
         return r;
     };
-    const size_t pairs = kStaticMaxPairs, sorted = kStaticMaxPairs + kStaticMaxSharedRows;
-    int32_t *idx = reinterpret_cast<int32_t *>(take(pairs * 4));
-    float *gate = reinterpret_cast<float *>(take(pairs * 4));
-    float *logits = reinterpret_cast<float *>(take((size_t)kStaticMaxTokens * kMaxExperts * 4));
-    int32_t *perm = reinterpret_cast<int32_t *>(take(sorted * 4));
-    int32_t *inv_pos = reinterpret_cast<int32_t *>(take(pairs * 4));
-    int32_t *tok_of_sorted = reinterpret_cast<int32_t *>(take(sorted * 4));
-    VrRec *vrs = reinterpret_cast<VrRec *>(take((size_t)kStaticMaxVr * sizeof(VrRec)));
+    const size_t pairs = kStaticMaxPairs, sorted = 1024;
+    Scratch sc;
+    sc.idx = reinterpret_cast<int32_t *>(take(pairs * 4));
+    sc.gate = reinterpret_cast<float *>(take(pairs * 4));
+    sc.logits = reinterpret_cast<float *>(take((size_t)kStaticMaxTokens * kMaxExperts * 4));
+    sc.perm = reinterpret_cast<int32_t *>(take(sorted * 4));
+    sc.inv_pos = reinterpret_cast<int32_t *>(take(pairs * 4));
+    sc.tok_of_sorted = reinterpret_cast<int32_t *>(take(sorted * 4));
     if ((size_t)(q - base) > kStaticSmall)
         return MELINOE_ERR_STATE;
-    float *zbuf = reinterpret_cast<float *>(base + kStaticSmall);
-    uint16_t *hbuf = reinterpret_cast<uint16_t *>(base + kStaticSmall + kStaticZ);
-    // the padding behind every h row has to read as zero, and the array keeps whatever the last
-    // call (of any handle, with any d_ff) left there
-    const size_t fpad = ((size_t)h->F + 255) / 256 * 256;
-    CU_TRY(cudaMemsetAsync(hbuf, 0, (size_t)kStaticMaxVr * kTokPerVr * fpad * 2, s));
-
-    // run the ordinary call on the static scratch: swap the handle's scratch pointers for its duration
-    struct Saved {
-        int32_t *idx, *perm, *inv_pos, *tok_of_sorted;
-        float *gate, *logits, *zbuf;
-        uint16_t *hbuf;
-        VrRec *vrs;
-        int cap_tokens, cap_shared, vr_capacity;
-    } keep{h->idx, h->perm, h->inv_pos, h->tok_of_sorted, h->gate, h->logits, h->zbuf, h->hbuf, h->vrs,
-           h->cap_tokens, h->cap_shared, h->vr_capacity};
-    h->idx = idx;
-    h->perm = perm;
-    h->inv_pos = inv_pos;
-    h->tok_of_sorted = tok_of_sorted;
-    h->gate = gate;
-    h->logits = logits;
-    h->zbuf = zbuf;
-    h->hbuf = hbuf;
-    h->vrs = vrs;
-    h->cap_tokens = kStaticMaxTokens;
-    h->cap_shared = h->n_shared;
-    h->vr_capacity = kStaticMaxVr;
-    const int rc = melinoe_moe_forward(h, cuda_stream, hidden_dev, T, out_dev, stats_dev);
-    h->idx = keep.idx;
-    h->perm = keep.perm;
-    h->inv_pos = keep.inv_pos;
-    h->tok_of_sorted = keep.tok_of_sorted;
-    h->gate = keep.gate;
-    h->logits = keep.logits;
-    h->zbuf = keep.zbuf;
-    h->hbuf = keep.hbuf;
-    h->vrs = keep.vrs;
-    h->cap_tokens = keep.cap_tokens;
-    h->cap_shared = keep.cap_shared;
-    h->vr_capacity = keep.vr_capacity;
-    h->last_T = 0;   // the inspection calls read the handle's own scratch, which this call did not touch
-    return rc;
+    sc.ybuf = reinterpret_cast<float *>(base + kStaticSmall);
+    sc.yacc = reinterpret_cast<long long *>(base + kStaticSmall + kStaticY);
+    sc.cap_tokens = kStaticMaxTokens;
+    return forward_on(h, sc, cuda_stream, hidden_dev, T, out_dev, stats_dev);
 }
 
 extern "C" size_t melinoe_moe_static_scratch_bytes(void) { return kStaticBytes; }
@@ -1229,9 +1325,9 @@ int melinoe_moe_last_routing(melinoe_moe_t *h, int32_t *idx_host, float *gate_ho
         return MELINOE_ERR_STATE;
     const size_t n = (size_t)h->last_T * h->k;
     if (idx_host)
-        CU_TRY(cudaMemcpy(idx_host, h->idx, n * 4, cudaMemcpyDeviceToHost));
+        CU_TRY(cudaMemcpy(idx_host, h->last.idx, n * 4, cudaMemcpyDeviceToHost));
     if (gate_host)
-        CU_TRY(cudaMemcpy(gate_host, h->gate, n * 4, cudaMemcpyDeviceToHost));
+        CU_TRY(cudaMemcpy(gate_host, h->last.gate, n * 4, cudaMemcpyDeviceToHost));
     return MELINOE_OK;
 }
 
@@ -1241,7 +1337,7 @@ int melinoe_moe_last_logits(melinoe_moe_t *h, float *logits_host)
         return MELINOE_ERR_INVALID;
     if (h->last_T <= 0)
         return MELINOE_ERR_STATE;
-    CU_TRY(cudaMemcpy(logits_host, h->logits, (size_t)h->last_T * h->E * 4, cudaMemcpyDeviceToHost));
+    CU_TRY(cudaMemcpy(logits_host, h->last.logits, (size_t)h->last_T * h->E * 4, cudaMemcpyDeviceToHost));
     return MELINOE_OK;
 }
 
@@ -1285,7 +1381,7 @@ int melinoe_moe_last_gather(melinoe_moe_t *h, int32_t *counts_host, int32_t *off
         CU_TRY(cudaMemcpy(offsets_host, reinterpret_cast<char *>(h->plan) + offsetof(DevPlan, offsets),
                           (size_t)(h->E + 1) * 4, cudaMemcpyDeviceToHost));
     if (perm_host)
-        CU_TRY(cudaMemcpy(perm_host, h->perm, (size_t)h->last_T * h->k * 4, cudaMemcpyDeviceToHost));
+        CU_TRY(cudaMemcpy(perm_host, h->last.perm, (size_t)h->last_T * h->k * 4, cudaMemcpyDeviceToHost));
     return MELINOE_OK;
 }
 
@@ -1348,13 +1444,36 @@ int melinoe_moe_set_trace(melinoe_moe_t *h, void *trace_dev, size_t bytes)
 
 int melinoe_moe_trace_ctas(melinoe_moe_t *h) { return h ? h->cfg.grid : 0; }
 
-int melinoe_moe_last_call_used_gemm(melinoe_moe_t *h) { return h && h->last_used_gemm ? (h->last_used_pair ? 2 : 1) : 0; }
+int melinoe_moe_last_call_used_gemm(melinoe_moe_t *h) { return h && h->last_used_gemm ? 1 : 0; }
+
+int melinoe_debug_fail_host_copy(int nth)
+{
+    g_fail_copy_in.store(nth > 0 ? nth : 0);
+    return MELINOE_OK;
+}
 
 int melinoe_moe_enable_timing(melinoe_moe_t *h, int enable)
 {
     if (!h)
         return MELINOE_ERR_INVALID;
     h->timing = enable != 0;
+    return MELINOE_OK;
+}
+
+int melinoe_moe_ffn_launch_times_ms(melinoe_moe_t *h, float *ms_out, int capacity, int *n_out)
+{
+    if (!h || capacity < 0 || (capacity > 0 && !ms_out))
+        return MELINOE_ERR_INVALID;
+    int n = 0;
+    for (auto &p : h->timed) {
+        if (n >= capacity)
+            break;
+        CU_TRY(cudaEventSynchronize(p.b));
+        CU_TRY(cudaEventElapsedTime(&ms_out[n], p.a, p.b));
+        ++n;
+    }
+    if (n_out)
+        *n_out = (int)h->timed.size();
     return MELINOE_OK;
 }
 

@@ -1,11 +1,12 @@
-// Expansion of a 4-bit group-quantised expert into the bf16 slot layout the FFN kernels read.
+// Expansion of a 4-bit group-quantised expert into the bf16 blob layout the FFN kernels read.
 //
 // Host store layout of one 4-bit expert (Section 3.2 keeps the experts in 4-bit form; what is
 // stored here is plain symmetric group quantisation): for each of W_g [F][d], W_u [F][d],
 // W_d [d][F], in this order, the codes [rows][cols / 2] (one byte = two columns, the even column
 // in the low nibble) followed by the scales [rows][cols / 64] (bf16).  The weight that the layer
 // computes with is bf16( scale * (code - 8) ): the product is exact in fp32 and is rounded to
-// nearest even.  The kernel is a pure stream: 1.6 bytes in, 6 bytes out per three weights.
+// nearest even.  The output is the bf16 blob of melinoe_moe_pack_expert: per hidden unit f the rows
+// W_g[f] | W_u[f] | W_d[:, f], the 16-byte pieces of every 128-byte group at (piece xor (f mod 8)).
 #include "kernels.cuh"
 
 namespace melinoe {
@@ -19,43 +20,64 @@ __device__ __forceinline__ uint32_t bf16_rne_bits(float v)
     return u >> 16;
 }
 
-// One thread expands 16 consecutive weights of one row (8 code bytes in, 32 bytes out).
+// A block expands tiles of 64 x 64 weights.  W_g / W_u: 64 rows f x 64 columns, written straight
+// through; W_d: 64 rows c x 64 columns f, transposed through shared memory so that the 64 values
+// c of one f leave as one 128-byte row piece.
 __global__ void __launch_bounds__(256) dequant_q4_kernel(const unsigned char *__restrict__ q, uint16_t *__restrict__ out, int d, int F)
 {
-    const size_t per_gu = (size_t)F * d, per_d = (size_t)d * F;       // weights per matrix
-    const size_t units = (2 * per_gu + per_d) / 16;
-    for (size_t u = (size_t)blockIdx.x * blockDim.x + threadIdx.x; u < units; u += (size_t)gridDim.x * blockDim.x) {
-        size_t w0 = u * 16;                 // first weight of the unit, counted over the three matrices
-        int m = 0;
-        if (w0 >= per_gu) {
-            w0 -= per_gu;
-            m = 1;
-            if (w0 >= per_gu) {
-                w0 -= per_gu;
-                m = 2;
-            }
-        }
-        const size_t n_w = m < 2 ? per_gu : per_d;
+    __shared__ uint16_t s_t[64][66];
+    const size_t n = (size_t)d * F;
+    const size_t sec = n / 2 + n / 32;                 // one matrix's section of the 4-bit blob
+    const int tiles_gu = (F / 64) * (d / 64), tiles_d = (d / 64) * (F / 64);
+    const int total = 2 * tiles_gu + tiles_d;
+    const int tid = threadIdx.x;
+    const int r = tid >> 2, part = tid & 3;            // source row of the tile, 16 of its 64 columns
+    for (int t = blockIdx.x; t < total; t += gridDim.x) {
+        const int m = t < tiles_gu ? 0 : (t < 2 * tiles_gu ? 1 : 2);
+        const int tt = t - m * tiles_gu;
         const int cols = m < 2 ? d : F;
-        // the matrix's section of the 4-bit blob: codes, then scales
-        const size_t sec = (size_t)m * (per_gu / 2 + per_gu / 32);     // W_g and W_u sections have the same size
-        const unsigned char *codes = q + sec;
-        const uint16_t *scales = reinterpret_cast<const uint16_t *>(q + sec + n_w / 2);
-        const size_t row = w0 / cols, col = w0 % cols;
-        const float s = __uint_as_float((uint32_t)scales[row * (cols / 64) + col / 64] << 16);
-        const uint2 c8 = *reinterpret_cast<const uint2 *>(codes + w0 / 2);
+        const int tr = tt / (cols / 64), tc = tt % (cols / 64);      // tile of source rows, of source columns
+        const unsigned char *codes = q + m * sec;
+        const uint16_t *scales = reinterpret_cast<const uint16_t *>(q + m * sec + n / 2);
+        const size_t row = (size_t)tr * 64 + r;
+        const float sc = __uint_as_float((uint32_t)scales[row * (cols / 64) + tc] << 16);
+        const uint2 c8 = *reinterpret_cast<const uint2 *>(codes + (row * cols + (size_t)tc * 64 + part * 16) / 2);
         uint32_t o[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             const uint32_t word = i < 4 ? c8.x : c8.y;
             const uint32_t byte = (word >> (8 * (i & 3))) & 0xffu;
-            const float lo = __fmul_rn(s, (float)((int)(byte & 15u) - 8));
-            const float hi = __fmul_rn(s, (float)((int)(byte >> 4) - 8));
+            const float lo = __fmul_rn(sc, (float)((int)(byte & 15u) - 8));
+            const float hi = __fmul_rn(sc, (float)((int)(byte >> 4) - 8));
             o[i] = bf16_rne_bits(lo) | (bf16_rne_bits(hi) << 16);
         }
-        uint4 *dst = reinterpret_cast<uint4 *>(out + (size_t)m * per_gu + w0);
-        dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
-        dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+        if (m < 2) {
+            // row f = row, columns tc * 64 + part * 16 ..: two 16-byte pieces of the 128-byte group tc
+            const int f = (int)row;
+            uint16_t *dst = out + ((size_t)f * 3 + m) * d + (size_t)tc * 64;
+            const int p0 = (part * 2) ^ (f & 7), p1 = (part * 2 + 1) ^ (f & 7);
+            *reinterpret_cast<uint4 *>(dst + p0 * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+            *reinterpret_cast<uint4 *>(dst + p1 * 8) = make_uint4(o[4], o[5], o[6], o[7]);
+        } else {
+            // source row c = row, source columns f = tc * 64 + part * 16 ..: transpose
+            __syncthreads();
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                s_t[part * 16 + 2 * i][r] = (uint16_t)(o[i] & 0xffffu);
+                s_t[part * 16 + 2 * i + 1][r] = (uint16_t)(o[i] >> 16);
+            }
+            __syncthreads();
+            // thread: f = tc * 64 + r, 16 of the 64 values c = tr * 64 + part * 16 ..
+            const int f = tc * 64 + r;
+            uint32_t w[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                w[i] = (uint32_t)s_t[r][part * 16 + 2 * i] | ((uint32_t)s_t[r][part * 16 + 2 * i + 1] << 16);
+            uint16_t *dst = out + ((size_t)f * 3 + 2) * d + (size_t)tr * 64;
+            const int p0 = (part * 2) ^ (f & 7), p1 = (part * 2 + 1) ^ (f & 7);
+            *reinterpret_cast<uint4 *>(dst + p0 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+            *reinterpret_cast<uint4 *>(dst + p1 * 8) = make_uint4(w[4], w[5], w[6], w[7]);
+        }
     }
 }
 

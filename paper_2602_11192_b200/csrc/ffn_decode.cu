@@ -1,0 +1,760 @@
+// Decode expert FFN (Eq. 3) with the gate-weighted combine (Eq. 2) fused in: one launch serves up
+// to 8 tokens.  The work is reading every needed expert once (from HBM, or over the host link for
+// an expert that is not resident), so the kernel is built around one contiguous stream per SM and
+// no synchronisation between SMs until the very end.
+//
+// Layout of an expert ("blob", written by melinoe_moe_pack_expert): for f = 0 .. d_ff - 1 the
+// three rows that belong to hidden unit f back to back,
+//     W_g[f][0..d) | W_u[f][0..d) | W_d[0..d)[f]   (the last one is row f of W_d transposed),
+// 6 d bytes, and inside each row the 16-byte pieces of every 128-byte group are stored at
+// position (piece xor (f mod 8)).  Consequences:
+//   - the rows f0 .. f0 + m - 1 are ONE contiguous byte range, fetched by one bulk copy;
+//   - everything hidden unit f contributes to the output, gate * SiLU(g_f) * u_f * W_d[:, f], can be
+//     formed by the SM that read those three rows: no other SM is involved, so the d_ff rows of all
+//     requested experts are simply dealt out evenly (single-row granularity) and every CTA ends up
+//     with a partial output vector;
+//   - eight consecutive rows, read at the same logical column, fall into eight different groups
+//     of shared-memory banks (the xor), so the tensor-core fragment loads (ldmatrix) are free of
+//     bank conflicts although the rows sit at a pitch that is a multiple of 128 bytes.
+//
+// One CTA per SM: NW consumer warps (8 for d <= 2048, else 16) and one producer warp.
+//   producer  one thread; per tile (up to 8 rows f of one expert) one cp.async.bulk into a ring
+//             stage, completion on the stage's mbarrier.  A missed expert's rows come straight from
+//             the page-locked host store (the device reads host memory over the link).
+//   gate/up   D[16 x 8] = [W_g rows ; W_u rows] (16 x d) * x^T (d x 8 tokens) on mma.sync m16n8k16
+//             (bf16 in, fp32 accumulate): decode is one multiply-add per weight byte pair, far
+//             below what even this legacy tensor path delivers, so it is free compute.  The warps
+//             split the columns; their partial tiles meet in shared memory once per tile and every
+//             warp forms the complete g_f, u_f (thread-local: a thread holds g and u of the same f and
+//             the same two tokens), then h = gate[token][expert] * SiLU(g) * u, rounded once to bf16.
+//             The gate is folded in here so that all experts accumulate into one output tile.
+//   down      Y[c][t] += sum_f W_d^T[f][c] * h[f][t]: the same 8 rows f are now the K dimension
+//             (padded to 16 with zeros), A = W_d^T rows read transposed (ldmatrix.trans), every warp
+//             owns d / NW output columns and keeps their fp32 accumulators in registers for the
+//             whole kernel.
+//   fetched   a tile of a missed expert that stays resident after the call is also stored into its
+//   experts   cache slot (bulk copy shared -> global) while it is being computed with.
+//   combine   every CTA adds its partial [tokens][d] into the call's accumulator in global memory as
+//             64-bit fixed point (units of 2^-40; integer atomics: the sum is exact, so it does not
+//             depend on the order of arrival and results are bit-identical from run to run), counts
+//             itself out on the handle's counter and exits; the CTA that finds all the others gone
+//             converts the sums to bf16, writes the output and clears accumulator and counter.  No CTA
+//             ever waits for another.
+//
+// Every wait is bounded: when an mbarrier or the wait for the plan does not complete in time the warp
+// raises the CTA's abort flag, later waits fall through, copies in flight are given a bounded time
+// to land, the kernel ends normally and the error word tells the host.
+#include <cstdlib>
+
+#include "kernels.cuh"
+
+namespace melinoe {
+
+namespace {
+
+constexpr int kMaxStages = 8;
+constexpr int kMaxMt = 16;                       // m-tiles (16 output columns each) / k-steps per warp
+// Bound of every wait, in SM clock cycles (about 2 s).
+constexpr long long kWaitLimitCycles = 4000000000ll;
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ unsigned long long globaltimer_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// Bounded wait.  Returns false (and raises the CTA's abort flag) when the limit runs out.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
+{
+    if (mbar_try(bar, parity))
+        return true;
+    if (*abort_flag)
+        return false;
+    const long long t0 = clock64();
+    for (;;) {
+        for (int i = 0; i < 64; ++i)
+            if (mbar_try(bar, parity))
+                return true;
+        if (*abort_flag)
+            return false;
+        if (clock64() - t0 > kWaitLimitCycles) {
+            *abort_flag = 1;
+            return false;
+        }
+    }
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(addr));
+}
+// D(16x8) += A(16x16) * B(16x8), bf16 in, fp32 accumulate.
+__device__ __forceinline__ void mma_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                          uint32_t b0, uint32_t b1)
+{
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint32_t lds32(uint32_t addr)
+{
+    uint32_t v;
+    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+
+__device__ __forceinline__ uint32_t bf16_rne(float v)
+{
+    uint32_t u = __float_as_uint(v);
+    u += 0x7fffu + ((u >> 16) & 1u);
+    return u >> 16;
+}
+
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_s2g(void *dst, uint32_t src, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes) : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+// An active request of the launch as the tile loops see it.
+struct SReq {
+    const char *src;      // where its rows are streamed from: the slot, a shared expert's blob, or the host store
+    char *wb;             // null, or the slot the fetched rows are also stored into
+    int32_t gate_row;     // its row of the gate table (= its index among the launch's requests)
+    int32_t deferred;     // the slot is written only after the grid barrier (it is still being computed with)
+};
+
+constexpr int NW = 16;                           // consumer warps
+constexpr int kThreads = (NW + 1) * 32;          // + the producer warp
+constexpr int kBufPitch = 130;                   // floats between the warps' partial tiles (keeps the column sums conflict-free)
+
+// MT_: k-steps of the gate/up phase and m-tiles of the down phase per warp (d / 256), 0 = taken from d at run time.
+template <int MT_>
+__global__ void __launch_bounds__(kThreads, 1) ffn_decode_kernel(DecParams p, DecGeometry geo)
+{
+    extern __shared__ __align__(128) unsigned char smem[];
+    __shared__ int s_abort, s_nact, s_last;
+    __shared__ int s_hdr[4];                        // status, n_groups, first request, one past the last
+    __shared__ DecReq s_raw[kMaxReq];
+    __shared__ SReq s_req[kMaxReq];
+    __shared__ float s_gate[kMaxReq][kTokPerVr];    // gate of (request, token of the launch); 0 = not routed
+    __shared__ unsigned s_match[kMaxReq];
+    __shared__ int32_t s_of_expert[kMaxReq];        // request of an expert id (routed 0..E-1, shared E..), -1 = none
+    __shared__ int32_t s_idx[kTokPerVr * 32];
+    __shared__ float s_gw[kTokPerVr * 32];
+    __shared__ float s_sums[128];
+    __shared__ __align__(8) uint64_t s_bars[2 * kMaxStages + 1];
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int d = p.d, F = p.F;
+    const int G = (int)gridDim.x;
+    const int TR = geo.tile_rows, S = geo.n_stages, RB = geo.row_bytes, STAGE = geo.stage_bytes, XP = geo.x_pitch;
+    const int Tc = geo.tokens, tok0 = p.chunk * kTokPerVr;
+    const int MT = MT_ > 0 ? MT_ : d / (16 * NW);
+
+    unsigned long long *trace = p.trace ? p.trace + (size_t)blockIdx.x * 8 : nullptr;
+    if (trace && tid == 0)
+        trace[0] = globaltimer_ns();
+
+    // ring | staged hidden rows | the warps' partial gate/up tiles
+    unsigned char *ring = smem;
+    unsigned char *xs = smem + (size_t)S * STAGE;
+    float *buf = reinterpret_cast<float *>(xs + (size_t)Tc * XP);                   // [NW][kBufPitch]
+    const uint32_t ring_s = smem_u32(ring), xs_s = smem_u32(xs);
+    const uint32_t full0 = smem_u32(s_bars), empty0 = full0 + 8 * kMaxStages, hzbar = empty0 + 8 * kMaxStages;
+    volatile int *abort_flag = &s_abort;
+
+    if (tid == 0) {
+        s_abort = 0;
+        s_nact = 0;
+        for (int i = 0; i < kMaxStages; ++i) {
+            mbar_init(full0 + 8 * i, 1);
+            mbar_init(empty0 + 8 * i, NW);
+        }
+        mbar_init(hzbar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    for (int i = tid; i < kMaxReq; i += kThreads) {
+        s_match[i] = 0u;
+        s_of_expert[i] = -1;
+    }
+    // Nothing above reads what an earlier kernel wrote.  With programmatic stream serialisation this
+    // CTA may be running while the kernel ahead of it in the stream (the planner) still is.  It does
+    // not wait for that grid to drain (which costs microseconds) but for the word the planner writes
+    // last, behind a device-wide fence, when the call's plan is complete.  The planner itself has
+    // waited for everything ahead of it in the stream, so whatever this kernel reads (hidden states,
+    // routing, plan) is in memory once the word is there.  A programmatically launched grid never
+    // starts before every CTA of the grid ahead of it is running, and the planner waits for nobody
+    // behind it, so the wait ends; it is bounded all the same.
+    if (p.wait_prior)
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const DevPlan *plan = p.plan;
+    if (tid == 0) {
+        const long long t0 = clock64();
+        for (;;) {
+            unsigned v;
+            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(&plan->ready_seq) : "memory");
+            if (v == p.call_seq)
+                break;
+            if (clock64() - t0 > kWaitLimitCycles) {
+                s_abort = 1;
+                break;
+            }
+        }
+    }
+    __syncthreads();
+
+    // ---- everything the launch needs to know, in one round trip to memory
+    if (tid == kThreads - 1) {
+        const int n_groups = plan->n_groups;
+        s_hdr[0] = plan->status;
+        s_hdr[1] = n_groups;
+        if (p.group < 0) {
+            s_hdr[2] = 0;
+            s_hdr[3] = plan->n_dreq;
+        } else {
+            s_hdr[2] = plan->group_vr_begin[p.group];
+            s_hdr[3] = plan->group_vr_begin[p.group + 1];
+        }
+    }
+    if (tid < kMaxReq) {
+        const uint4 *src = reinterpret_cast<const uint4 *>(plan->dreq + tid);
+        uint4 *dst = reinterpret_cast<uint4 *>(s_raw + tid);
+        dst[0] = src[0];
+        dst[1] = src[1];
+    }
+    for (int i = tid; i < Tc * p.k; i += kThreads) {
+        s_idx[i] = p.idx[(size_t)tok0 * p.k + i];
+        s_gw[i] = p.gate[(size_t)tok0 * p.k + i];
+    }
+    {
+        const int per_row = d / 8;                  // 16-byte pieces of a hidden row
+        for (int i = tid; i < Tc * per_row; i += kThreads) {
+            const int t = i / per_row, c = i % per_row;
+            const uint4 v = *reinterpret_cast<const uint4 *>(p.x + (size_t)(tok0 + t) * d + c * 8);
+            *reinterpret_cast<uint4 *>(xs + (size_t)t * XP + c * 16) = v;
+        }
+    }
+    __syncthreads();
+    const int status = s_abort == 1 ? (int)MELINOE_ERR_TIMEOUT : s_hdr[0], n_groups = s_hdr[1], rq0 = s_hdr[2];
+    const int nrq = s_hdr[3] - rq0;
+    if (status != MELINOE_OK || nrq < 0 || nrq > kMaxReq) {
+        if (s_abort == 1 && tid == 0)
+            atomicExch(p.err, MELINOE_ERR_TIMEOUT);
+        // the call was refused on the device: the output is all zeros, the status tells why
+        if (p.group <= 0)
+            for (size_t i = (size_t)blockIdx.x * kThreads + tid; i < (size_t)Tc * d; i += (size_t)G * kThreads)
+                p.out[(size_t)tok0 * d + i] = 0;
+        if (tid == 0) {
+            // the counter advances once per CTA and launch, whatever happens
+            if (atomicAdd(p.sync, 1u) == (unsigned)(G - 1))
+                *p.sync = 0u;
+        }
+        return;
+    }
+    // gate of every (request, token): the token's gate for that expert if the router chose it
+    for (int i = tid; i < nrq * kTokPerVr; i += kThreads) {
+        const int r = i / kTokPerVr, t = i % kTokPerVr;
+        const int e = s_raw[rq0 + r].expert;
+        if (t == 0 && e >= 0 && e < kMaxReq)
+            s_of_expert[e] = r;
+        float gv = 0.0f;
+        if (t < Tc) {
+            if (e >= p.E) {
+                gv = 1.0f;              // shared expert: every token, gate 1
+                atomicOr(&s_match[r], 1u << t);
+            } else {
+                for (int j = 0; j < p.k; ++j)
+                    if (s_idx[t * p.k + j] == e) {
+                        gv = s_gw[t * p.k + j];
+                        atomicOr(&s_match[r], 1u << t);
+                    }
+            }
+        }
+        s_gate[r][t] = gv;
+    }
+    __syncthreads();
+    // The requests that have a token in this launch, in ascending expert id (shared experts last): the
+    // rows are dealt out in that order, so the order of every sum depends only on which experts the
+    // tokens use, not on which of them happened to be resident.
+    if (warp == 0) {
+        int base = 0;
+        for (int e0 = 0; e0 < kMaxReq; e0 += 32) {
+            const int e = e0 + lane;
+            const int r = e < kMaxReq ? s_of_expert[e] : -1;
+            // a fetched expert that stays resident is streamed (and stored into its slot) by the launch whose
+            // job that is even if none of this launch's tokens uses it
+            bool act = r >= 0 && s_match[r] != 0u;
+            bool pull = false, stays = false, hazard = false;
+            if (r >= 0 && p.group < 0 && (s_raw[rq0 + r].flags & kDecMiss)) {
+                const int fl = s_raw[rq0 + r].flags;
+                pull = true;
+                stays = (fl & kDecStays) != 0 && p.write_back != 0;
+                hazard = (fl & kDecHazard) != 0;
+                if (stays && (hazard ? p.chunk == p.n_chunks - 1 : p.chunk == 0))
+                    act = true;
+            }
+            const unsigned m = __ballot_sync(0xffffffffu, act);
+            if (act) {
+                const DecReq q = s_raw[rq0 + r];
+                SReq sr;
+                sr.src = q.blob;
+                sr.wb = nullptr;
+                sr.gate_row = r;
+                sr.deferred = 0;
+                if (pull) {
+                    // Where a call is made in several launches (more than 8 tokens): the first one stores
+                    // the expert into its slot and the later ones read it there, unless the slot still
+                    // holds an expert the call computes with: then every launch reads the host store and
+                    // the last one stores it once all CTAs are done.
+                    if (stays && !hazard && p.chunk > 0) {
+                        sr.src = q.blob;
+                    } else {
+                        sr.src = q.host;
+                        if (q.host == nullptr)
+                            s_abort = 2;
+                        if (stays && !hazard)
+                            sr.wb = const_cast<char *>(q.blob);
+                        if (stays && hazard && p.chunk == p.n_chunks - 1)
+                            sr.deferred = 1;
+                    }
+                }
+                s_req[base + __popc(m & ((1u << lane) - 1u))] = sr;
+            }
+            base += __popc(m);
+        }
+        if (lane == 0)
+            s_nact = base;
+    }
+    __syncthreads();
+    const int nact = s_nact;
+    const bool no_host = s_abort == 2;      // a missed expert cannot be read from here: nothing is computed
+    if (trace && tid == 0)
+        trace[1] = globaltimer_ns();
+
+    // ---- this CTA's share of the rows: f rows of the active requests, request-major, dealt out evenly
+    const long long rows = no_host ? 0 : (long long)nact * F;
+    const long long q_lo = blockIdx.x * rows / G, q_hi = (blockIdx.x + 1) * rows / G;
+
+    if (warp == NW) {
+        // =================================================================== producer
+        if (lane == 0) {
+            uint32_t n = 0;
+            long long q = q_lo;
+            int a = (int)(q / F), f0 = (int)(q % F);
+            while (q < q_hi) {
+                const int m = (int)min((long long)min(TR, F - f0), q_hi - q);
+                const uint32_t st = n % (uint32_t)S;
+                if (n >= (uint32_t)S && !mbar_wait(empty0 + 8 * st, ((n / S) - 1u) & 1u, abort_flag))
+                    break;
+                const uint32_t bytes = (uint32_t)m * RB;
+                mbar_expect(full0 + 8 * st, bytes);
+                bulk_g2s(ring_s + st * STAGE, s_req[a].src + (size_t)f0 * RB, bytes, full0 + 8 * st);
+                ++n;
+                q += m;
+                f0 += m;
+                if (f0 == F) {
+                    f0 = 0;
+                    ++a;
+                }
+            }
+            if (*abort_flag) {
+                // a wait ran out: give the copies still in flight a bounded time to land before this
+                // CTA's shared memory goes away
+                const long long t0 = clock64();
+                for (uint32_t j = n > (uint32_t)S ? n - S : 0; j < n; ++j)
+                    while (!mbar_try(full0 + 8 * (j % S), (j / S) & 1u) && clock64() - t0 < kWaitLimitCycles) {
+                    }
+            }
+        }
+    } else {
+        // =================================================================== consumers
+        const int g = lane >> 2, tig = lane & 3;
+        float acc[kMaxMt][4];
+#pragma unroll
+        for (int i = 0; i < kMaxMt; ++i)
+            acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f;
+        const bool has_tok = g < Tc;
+        const uint32_t xrow = xs_s + g * XP + tig * 4 + warp * MT * 32;     // this warp's columns of token g
+        // ldmatrix lane roles.  gate/up: matrices (W_g rows, k low), (W_u rows, k low), (W_g rows, k high),
+        // (W_u rows, k high); down: four consecutive 8-column pieces of the W_d^T rows
+        const int r8 = lane & 7, sel_gu = (lane >> 3) & 1, kh = lane >> 4, mat = lane >> 3;
+        const uint32_t src0 = (uint32_t)((2 * tig) * 4 + (g >> 1)), src1 = src0 + 4;
+        uint32_t n = 0;
+        long long q = q_lo;
+        int a = (int)(q / F), f0 = (int)(q % F);
+        bool first = true;
+        while (q < q_hi) {
+            const int m = (int)min((long long)min(TR, F - f0), q_hi - q);
+            const uint32_t st = n % (uint32_t)S;
+            const uint32_t stage = ring_s + st * STAGE;
+            mbar_wait(full0 + 8 * st, (n / S) & 1u, abort_flag);
+            if (trace && first && tid == 0)
+                trace[2] = globaltimer_ns();
+            first = false;
+            const SReq rq = s_req[a];
+            const bool store_tile = rq.wb != nullptr && tid == 0;
+            if (store_tile)
+                bulk_s2g(rq.wb + (size_t)f0 * RB, stage, (uint32_t)m * RB);
+            const int rr = r8 < m ? r8 : 0;               // rows the tile does not have read row 0 (never used)
+            const uint32_t swz = (uint32_t)((f0 + rr) & 7);
+            const uint32_t rowbase = stage + rr * RB;
+            // ---- gate/up: this warp's columns of the tile's rows.  A dependent mma.sync issues only every
+            // ~110 cycles, so the k-steps go to four independent accumulators, and the fragment loads of
+            // four steps are issued before their four products.
+            float cg[4][4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                cg[i][0] = cg[i][1] = cg[i][2] = cg[i][3] = 0.f;
+            {
+                const uint32_t arow = rowbase + sel_gu * 2 * d;
+                const uint32_t ch0 = (uint32_t)(2 * warp * MT + kh);
+#pragma unroll
+                for (int i0 = 0; i0 < kMaxMt; i0 += 4) {
+                    if (i0 < MT) {
+                        uint32_t af[4][4], bf[4][2];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const int i = i0 + j < MT ? i0 + j : i0;     // beyond the warp's last step: a valid address, product unused
+                            ldmatrix_x4(arow + (((ch0 + 2 * i) ^ swz) << 4), af[j][0], af[j][1], af[j][2], af[j][3]);
+                            bf[j][0] = has_tok ? lds32(xrow + i * 32) : 0u;
+                            bf[j][1] = has_tok ? lds32(xrow + i * 32 + 16) : 0u;
+                        }
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            if (i0 + j < MT)
+                                mma_16816(cg[j], af[j][0], af[j][1], af[j][2], af[j][3], bf[j][0], bf[j][1]);
+                    }
+                }
+            }
+            // ---- the warps' partial tiles meet: warp w sums 8 of the tile's 128 values over all warps (four
+            // lanes per value, each adding four warps' parts in warp order, then a fixed tree), then every
+            // warp reads the complete tile
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                buf[warp * kBufPitch + i * 32 + lane] = (cg[0][i] + cg[1][i]) + (cg[2][i] + cg[3][i]);
+            asm volatile("bar.sync 1, %0;" ::"n"(NW * 32) : "memory");
+            {
+                const int e = warp * 8 + (lane & 7), pg = lane >> 3;
+                float v = buf[(pg * 4) * kBufPitch + e];
+                v += buf[(pg * 4 + 1) * kBufPitch + e];
+                v += buf[(pg * 4 + 2) * kBufPitch + e];
+                v += buf[(pg * 4 + 3) * kBufPitch + e];
+                v += __shfl_xor_sync(0xffffffffu, v, 8);
+                v += __shfl_xor_sync(0xffffffffu, v, 16);
+                if (lane < 8)
+                    s_sums[e] = v;
+            }
+            asm volatile("bar.sync 1, %0;" ::"n"(NW * 32) : "memory");
+            const float s0 = s_sums[lane], s1 = s_sums[32 + lane], s2 = s_sums[64 + lane], s3 = s_sums[96 + lane];
+            // rows g and g + 8 of the tile are g_f and u_f of f = f0 + g, columns are tokens 2 tig, 2 tig + 1
+            const float gt0 = s_gate[rq.gate_row][2 * tig], gt1 = s_gate[rq.gate_row][2 * tig + 1];
+            // (the fast division: the exact one takes its slow path for the zeros of unused token columns)
+            float h0 = __fdividef(s0, 1.0f + __expf(-s0)) * s2 * gt0;
+            float h1 = __fdividef(s1, 1.0f + __expf(-s1)) * s3 * gt1;
+            if (g >= m || gt0 == 0.0f)
+                h0 = 0.f;
+            if (g >= m || gt1 == 0.0f)
+                h1 = 0.f;
+            const uint32_t hp = bf16_rne(h0) | (bf16_rne(h1) << 16);
+            // B fragment of the down product: h[f = 2 tig', 2 tig' + 1][token g'] from the lanes that hold them
+            const uint32_t v0 = __shfl_sync(0xffffffffu, hp, src0), v1 = __shfl_sync(0xffffffffu, hp, src1);
+            const uint32_t bd = (g & 1) ? ((v0 >> 16) | (v1 & 0xffff0000u)) : ((v0 & 0xffffu) | (v1 << 16));
+            // ---- down: the tile's rows are the K dimension (rows the tile does not have count as zero)
+            {
+                const uint32_t km = (2 * tig < m ? 0x0000ffffu : 0u) | (2 * tig + 1 < m ? 0xffff0000u : 0u);
+                const uint32_t drow = rowbase + 4 * d;
+                const uint32_t cc0 = (uint32_t)(warp * MT * 2);
+#pragma unroll
+                for (int m0 = 0; m0 < kMaxMt; m0 += 8) {
+                    if (m0 < MT) {
+                        // fragment loads of up to eight m-tiles first, then their products
+                        uint32_t rf[4][4];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            // a load covers two m-tiles; an odd last one is fetched together with the one before
+                            // it (or, if it is the warp's only one, with 16 columns that are not used)
+                            int mi = m0 + 2 * j;
+                            if (mi >= MT)
+                                mi = m0;
+                            else if (mi + 1 >= MT && mi > 0)
+                                mi -= 1;
+                            ldmatrix_x4_trans(drow + (((cc0 + 2 * mi + mat) ^ swz) << 4), rf[j][0], rf[j][1], rf[j][2], rf[j][3]);
+                        }
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const int mi = m0 + 2 * j;
+                            if (mi + 1 < MT) {
+                                mma_16816(acc[mi], rf[j][0] & km, rf[j][1] & km, 0u, 0u, bd, 0u);
+                                mma_16816(acc[mi + 1], rf[j][2] & km, rf[j][3] & km, 0u, 0u, bd, 0u);
+                            } else if (mi < MT) {
+                                if (mi > 0)
+                                    mma_16816(acc[mi], rf[j][2] & km, rf[j][3] & km, 0u, 0u, bd, 0u);
+                                else
+                                    mma_16816(acc[mi], rf[j][0] & km, rf[j][1] & km, 0u, 0u, bd, 0u);
+                            }
+                        }
+                    }
+                }
+            }
+            if (store_tile)
+                bulk_wait_read();         // the slot store has read the stage
+            __syncwarp();
+            if (lane == 0)
+                mbar_arrive(empty0 + 8 * st);
+            ++n;
+            q += m;
+            f0 += m;
+            if (f0 == F) {
+                f0 = 0;
+                ++a;
+            }
+        }
+        if (trace && tid == 0)
+            trace[3] = globaltimer_ns();
+        // ---- this CTA's partial output, added into the call's accumulator as 64-bit fixed point (2^-40):
+        // integer addition is exact, so the sum does not depend on the order in which the CTAs arrive.
+        // (Adds without a return value: atomics that return the old word, which would let the last adder
+        // of an element finish it on the spot, measured three times slower under this contention.)
+        {
+            unsigned long long *yacc = reinterpret_cast<unsigned long long *>(p.yacc);
+            auto add = [&](int t, int c, float v) {
+                const long long fx = __double2ll_rn((double)v * 1099511627776.0);
+                atomicAdd(yacc + (size_t)t * d + c, (unsigned long long)fx);
+            };
+#pragma unroll
+            for (int mi = 0; mi < kMaxMt; ++mi) {
+                if (mi < MT) {
+                    const int c = (warp * MT + mi) * 16 + g;
+                    if (2 * tig < Tc) {
+                        add(2 * tig, c, acc[mi][0]);
+                        add(2 * tig, c + 8, acc[mi][2]);
+                    }
+                    if (2 * tig + 1 < Tc) {
+                        add(2 * tig + 1, c, acc[mi][1]);
+                        add(2 * tig + 1, c + 8, acc[mi][3]);
+                    }
+                }
+            }
+        }
+        if (tid == 0)
+            bulk_wait_all();              // the slot stores of this thread have completed
+    }
+
+    // ---- the CTA that finishes last turns the sums into the output; all others are done
+    __syncthreads();
+    if (tid == 0) {
+        __threadfence();
+        const unsigned ticket = atomicAdd(p.sync, 1u);
+        s_last = ticket == (unsigned)(G - 1);
+        if (s_last)
+            *p.sync = 0u;                 // the counter is back at zero for the next launch
+        if (trace)
+            trace[4] = globaltimer_ns();
+    }
+    __syncthreads();
+    if (*abort_flag && tid == 0)
+        atomicExch(p.err, no_host ? MELINOE_ERR_STATE : MELINOE_ERR_TIMEOUT);
+    if (!s_last) {
+        if (trace && tid == 0)
+            trace[7] = globaltimer_ns();
+        return;
+    }
+    __threadfence();
+    if (trace && tid == 0)
+        trace[5] = globaltimer_ns();
+    {
+        const bool acc_in = p.group > 0, acc_out = p.group >= 0 && p.group < n_groups - 1;
+        long long *yacc = p.yacc;
+        const int N = Tc * d;
+        for (int e = tid; e < N; e += kThreads) {
+            const long long fx = __ldcg(yacc + e);
+            yacc[e] = 0;                                     // the accumulator is left clean for the next launch
+            float v = (float)((double)fx * (1.0 / 1099511627776.0));
+            const size_t o = (size_t)tok0 * d + e;           // element e of the launch's [tokens][d] block
+            if (acc_in)
+                v += __ldcg(p.ybuf + o);
+            if (acc_out)
+                p.ybuf[o] = v;
+            else
+                p.out[o] = (uint16_t)bf16_rne(v);
+        }
+    }
+    if (trace && tid == 0)
+        trace[6] = globaltimer_ns();
+
+    // ---- fetched experts whose slot was still being computed with: stored now that every CTA is done
+    if (tid == 0) {
+        uint32_t phase = 0;
+        bool any = false;
+        __syncwarp();
+        for (int a = 0; a < nact && *abort_flag != 1; ++a) {
+            if (!s_req[a].deferred)
+                continue;
+            const SReq rq = s_req[a];
+            char *slot = const_cast<char *>(s_raw[rq0 + rq.gate_row].blob);
+            for (int f = 0; f < F; f += TR) {
+                const uint32_t bytes = (uint32_t)min(TR, F - f) * RB;
+                if (any)
+                    bulk_wait_read();
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                mbar_expect(hzbar, bytes);
+                bulk_g2s(ring_s, rq.src + (size_t)f * RB, bytes, hzbar);
+                if (!mbar_wait(hzbar, phase & 1u, abort_flag))
+                    break;
+                ++phase;
+                bulk_s2g(slot + (size_t)f * RB, ring_s, bytes);
+                any = true;
+            }
+        }
+        if (any)
+            bulk_wait_all();
+        if (*abort_flag == 1)
+            atomicExch(p.err, MELINOE_ERR_TIMEOUT);
+    }
+    if (trace && tid == 0)
+        trace[7] = globaltimer_ns();
+}
+
+}  // namespace
+
+bool ffn_decode_supported(int d, int F) { return d % 256 == 0 && d >= 256 && d <= 4096 && F % kUnitRows == 0; }
+
+cudaError_t ffn_decode_configure(int n_sms, size_t max_smem, DecLaunchCfg *cfg)
+{
+    size_t stat = 0;
+    const void *fns[3] = {reinterpret_cast<const void *>(ffn_decode_kernel<0>), reinterpret_cast<const void *>(ffn_decode_kernel<8>),
+                          reinterpret_cast<const void *>(ffn_decode_kernel<16>)};
+    for (const void *fn : fns) {
+        cudaFuncAttributes fa;
+        const cudaError_t e = cudaFuncGetAttributes(&fa, fn);
+        if (e != cudaSuccess)
+            return e;
+        if (fa.sharedSizeBytes > stat)
+            stat = fa.sharedSizeBytes;
+    }
+    const size_t usable = (max_smem - stat - 1024) / 128 * 128;
+    for (const void *fn : fns) {
+        const cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)usable);
+        if (e != cudaSuccess)
+            return e;
+    }
+    cfg->grid = n_sms < 255 ? n_sms : 255;   // one CTA per SM (the accumulator words count CTAs in one byte)
+    cfg->max_smem = usable;
+    cfg->pdl = pdl_enabled();
+    return cudaSuccess;
+}
+
+cudaError_t ffn_decode_geometry(const DecLaunchCfg &cfg, int d, int F, int tokens, int fmt, DecGeometry *geo)
+{
+    if (!ffn_decode_supported(d, F) || tokens < 1 || tokens > kTokPerVr || fmt != 0)
+        return cudaErrorInvalidValue;
+    geo->n_warps = NW;
+    geo->row_bytes = 6 * d;
+    geo->x_pitch = 2 * d + 16;
+    geo->tokens = tokens;
+    // staged hidden rows + the warps' partial tiles; the largest tile (8, 4, 2 or 1 rows) of which two
+    // stages fit beside them
+    const size_t fixed = (size_t)tokens * geo->x_pitch + (size_t)NW * kBufPitch * sizeof(float);
+    int tr = 8;
+    if (const char *ev = std::getenv("MELINOE_DEC_TR"))
+        tr = atoi(ev);
+    for (;; tr /= 2) {
+        if (cfg.max_smem >= fixed + (size_t)2 * tr * geo->row_bytes)
+            break;
+        if (tr == 1)
+            return cudaErrorInvalidConfiguration;
+    }
+    const size_t avail = cfg.max_smem - fixed;
+    geo->tile_rows = tr;
+    geo->stage_bytes = tr * geo->row_bytes;
+    size_t n = avail / geo->stage_bytes;
+    if (n > (size_t)kMaxStages)
+        n = kMaxStages;
+    geo->n_stages = (int)n;
+    geo->smem_bytes = n * geo->stage_bytes + fixed;
+    return cudaSuccess;
+}
+
+cudaError_t launch_ffn_decode(cudaStream_t stream, const DecLaunchCfg &cfg, const DecGeometry &geo, const DecParams &p)
+{
+    // Programmatic stream serialisation: the CTAs may be scheduled, and set up their barriers, while the
+    // kernel ahead in the stream is still draining; the kernel waits for it before it reads the plan.
+    // All CTAs are resident at once (one per SM, the grid is the SM count), which the grid barrier at
+    // the end relies on; MELINOE_MOE_COOP in the environment asks the driver to guarantee it.
+    static const bool coop = std::getenv("MELINOE_MOE_COOP") != nullptr;
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3(cfg.grid);
+    lc.blockDim = dim3(kThreads);
+    lc.dynamicSmemBytes = geo.smem_bytes;
+    lc.stream = stream;
+    cudaLaunchAttribute attr[2];
+    int na = 0;
+    if (coop) {
+        attr[na].id = cudaLaunchAttributeCooperative;
+        attr[na].val.cooperative = 1;
+        ++na;
+    }
+    if (cfg.pdl) {
+        attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+    }
+    lc.attrs = attr;
+    lc.numAttrs = na;
+    const int mt = p.d / (16 * NW);
+    const cudaError_t e = mt == 8    ? cudaLaunchKernelEx(&lc, ffn_decode_kernel<8>, p, geo)
+                          : mt == 16 ? cudaLaunchKernelEx(&lc, ffn_decode_kernel<16>, p, geo)
+                                     : cudaLaunchKernelEx(&lc, ffn_decode_kernel<0>, p, geo);
+    count_launch();
+    return e;
+}
+
+}  // namespace melinoe

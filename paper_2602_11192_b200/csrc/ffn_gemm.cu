@@ -11,10 +11,16 @@
 //   GEMM 2    per expert: Z = H_e (M_e x F) * W_d^T, tile 128 tokens x 256 output columns, fp32.
 //   combine   y_t = sum_j gate[t][j] * Z[pos(t, j)] (+ shared experts), rank order, one rounding.
 //
-// Both GEMMs use the paper's own matrix shapes: W_g, W_u [F][d] and W_d [d][F] are "N x K,
-// K contiguous", and so are Xs and H, i.e. every operand is K-major with 128-byte swizzle.
-// The experts of all slots are addressed through one tensor map per view (rows of d elements
-// for GEMM 1, rows of F elements for GEMM 2), because the slots are contiguous.
+// The expert blob (see melinoe_moe_pack_expert) holds, per hidden unit f, the rows W_g[f], W_u[f]
+// and W_d[:, f], each d elements, with the 16-byte pieces of every 128-byte group stored at
+// (piece xor (f mod 8)).  That permutation is exactly what a TMA load with 128-byte swizzle would
+// have produced in shared memory from plain rows, as long as a tile starts at a multiple of 8 rows
+// and 64 columns; so the weight tiles are fetched by TMA WITHOUT swizzle and the MMA descriptors
+// name the 128-byte-swizzled layout.  W_g and W_u rows are "N x K, K contiguous" (K-major, like the
+// activations Xs and H, which are plain and fetched with TMA swizzle); the W_d^T rows are
+// "K x N, N contiguous": GEMM 2 takes its B operand N-major (four 64-column boxes per stage).
+// The experts of all slots are addressed through one tensor map per view (W_g rows, W_u rows,
+// W_d^T rows: the same row pitch of 6 d bytes, different offsets), because the slots are contiguous.
 //
 // One persistent CTA per SM, warp-specialised: warp 0 issues TMA loads into a 4-stage ring,
 // warp 1 issues the MMAs (one elected thread) and commits them to mbarriers, warps 2..5 drain
@@ -111,13 +117,23 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr)
     return d;
 }
 
-// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = 256.
-__device__ __forceinline__ uint32_t instr_desc_bf16(int m, int n)
+// The same for an N-major B operand made of 64-column boxes (64 K rows of 128 bytes each, 8 KB per
+// box): the boxes follow one another along N (leading offset), groups of 8 K rows are 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128_nmajor(uint32_t addr)
+{
+    uint64_t d = smem_desc_sw128(addr);
+    d |= (uint64_t)(8192u >> 4) << 16;                // between 64-column boxes
+    return d;
+}
+
+// Instruction descriptor: bf16 x bf16 -> fp32, A K-major, B K-major or N-major, M = 128, N = 256.
+__device__ __forceinline__ uint32_t instr_desc_bf16(int m, int n, bool b_nmajor)
 {
     uint32_t d = 0;
     d |= 1u << 4;                    // D format: fp32
     d |= 1u << 7;                    // A format: bf16
     d |= 1u << 10;                   // B format: bf16
+    d |= (b_nmajor ? 1u : 0u) << 16; // B major: 0 = K, 1 = N
     d |= (uint32_t)(n >> 3) << 17;
     d |= (uint32_t)(m >> 4) << 24;
     return d;
@@ -162,7 +178,7 @@ __device__ __forceinline__ uint32_t bf16_rne(float v)
 struct GemmItem {
     int row0;      // first sorted row of the m-tile
     int row_end;   // one past the expert's last sorted row
-    int b_row;     // first row of the B tile in its tensor map (GEMM 1: the W_g rows; W_u = + F)
+    int b_row;     // first expert row of its tensor maps (its slot times F, 0 for a shared expert)
     int n0;        // first output column of the tile (f for GEMM 1, output column for GEMM 2)
     int shared;    // B comes from a shared expert's tensor map: index of that expert, else -1
 };
@@ -246,14 +262,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) ffn_gemm_kernel(GemmParams p)
         it.row0 = rec.tok_off + mt * kBM;
         it.row_end = rec.tok_off + rec.n_tok;
         it.shared = rec.slot >= 0 ? -1 : rec.expert - p.E;
-        const int base_expert = rec.slot >= 0 ? rec.slot : 0;     // shared experts have a map each
-        if (PHASE == 1) {
-            it.n0 = nt * 128;
-            it.b_row = base_expert * 3 * p.F + it.n0;
-        } else {
-            it.n0 = nt * kBN;
-            it.b_row = base_expert * 3 * p.d + 2 * p.d + it.n0;
-        }
+        it.b_row = (rec.slot >= 0 ? rec.slot : 0) * p.F;          // shared experts have maps of their own
+        it.n0 = PHASE == 1 ? nt * 128 : nt * kBN;
         return it;
     };
     const int kblocks = K / kBK;
@@ -265,8 +275,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) ffn_gemm_kernel(GemmParams p)
             uint32_t n = 0;
             for (int w = blockIdx.x; w < total_items && !*abort_flag; w += gridDim.x) {
                 const GemmItem it = item_of(w);
-                const CUtensorMap *map_b = it.shared < 0 ? p.maps + (PHASE == 1 ? kMapSlotsD : kMapSlotsF)
-                                                         : p.maps + kMapShared0 + 2 * it.shared + (PHASE == 1 ? 0 : 1);
+                // W_g rows, W_u rows, W_d^T rows of the slots, or of the shared expert
+                const CUtensorMap *map_w = it.shared < 0 ? p.maps + kMapSlotsG : p.maps + kMapShared0 + 3 * it.shared;
                 for (int kb = 0; kb < kblocks; ++kb, ++n) {
                     const uint32_t s = n % kStages;
                     if (n >= (uint32_t)kStages && !mbar_wait(empty0 + 8 * s, ((n / kStages) - 1u) & 1u, abort_flag))
@@ -276,10 +286,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) ffn_gemm_kernel(GemmParams p)
                     mbar_expect(bar, kStageBytes);
                     tma_load_2d(a_dst, map_a, kb * kBK, it.row0, bar);
                     if (PHASE == 1) {
-                        tma_load_2d(b_dst, map_b, kb * kBK, it.b_row, bar);                     // 128 rows of W_g
-                        tma_load_2d(b_dst + kBBytes / 2, map_b, kb * kBK, it.b_row + p.F, bar); // 128 rows of W_u
+                        tma_load_2d(b_dst, map_w, kb * kBK, it.b_row + it.n0, bar);                   // 128 rows of W_g
+                        tma_load_2d(b_dst + kBBytes / 2, map_w + 1, kb * kBK, it.b_row + it.n0, bar); // 128 rows of W_u
                     } else {
-                        tma_load_2d(b_dst, map_b, kb * kBK, it.b_row, bar);                     // 256 rows of W_d
+                        // 64 rows f of W_d^T, four boxes of 64 output columns
+#pragma unroll
+                        for (int i = 0; i < kBN / 64; ++i)
+                            tma_load_2d(b_dst + i * 8192, map_w + 2, it.n0 + 64 * i, it.b_row + kb * kBK, bar);
                     }
                 }
             }
@@ -287,7 +300,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) ffn_gemm_kernel(GemmParams p)
     } else if (warp == 1) {
         // ============================================================ MMA issuer
         if (lane == 0) {
-            const uint32_t idesc = instr_desc_bf16(kBM, kBN);
+            const uint32_t idesc = instr_desc_bf16(kBM, kBN, PHASE == 2);
             uint32_t n = 0, item = 0;
             for (int w = blockIdx.x; w < total_items && !*abort_flag; w += gridDim.x, ++item) {
                 const uint32_t acc = item & 1u;
@@ -304,10 +317,14 @@ __global__ void __launch_bounds__(kGemmThreads, 1) ffn_gemm_kernel(GemmParams p)
                     }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t a_addr = ring_s + s * kStageBytes, b_addr = a_addr + kABytes;
-                    const uint64_t a_desc = smem_desc_sw128(a_addr), b_desc = smem_desc_sw128(b_addr);
+                    const uint64_t a_desc = smem_desc_sw128(a_addr);
+                    const uint64_t b_desc = PHASE == 1 ? smem_desc_sw128(b_addr) : smem_desc_sw128_nmajor(b_addr);
+                    // 16 K elements: 32 bytes along a K-major row (2 descriptor units), 16 rows of 128 bytes
+                    // in an N-major box (128 units)
+                    constexpr int kBStep = PHASE == 1 ? 2 : 128;
 #pragma unroll
-                    for (int ks = 0; ks < kBK / 16; ++ks)   // 16 K elements = 32 bytes = 2 descriptor units
-                        umma_bf16(d_tmem, a_desc + 2 * ks, b_desc + 2 * ks, idesc, (kb | ks) != 0);
+                    for (int ks = 0; ks < kBK / 16; ++ks)
+                        umma_bf16(d_tmem, a_desc + 2 * ks, b_desc + kBStep * ks, idesc, (kb | ks) != 0);
                     umma_commit(empty0 + 8 * s);             // the stage is free once these MMAs have read it
                 }
                 if (!ok)

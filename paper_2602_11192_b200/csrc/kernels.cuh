@@ -24,20 +24,19 @@ struct PlanParams {
     int T, k, E, C, n_shared;
     DevCache *cache;
     DevPlan *plan;
-    VrRec *vrs;
-    const char *slots;        // device cache (slot s at slots + s * slot_stride), for the vrs' blob pointers
+    const char *slots;        // device cache (slot s at slots + s * slot_stride)
     size_t slot_stride;
     const char *const *shared_blobs;
+    const char *const *host_blobs;   // device array [E]: every expert's blob in the host store as the device
+                                     // sees it (null entries, or a null array: the store cannot be read from kernels)
     int32_t *perm, *inv_pos, *tok_of_sorted;
     HostPlan *hplan;          // page-locked host memory (device-visible address)
-    unsigned *sync;           // grid-barrier counters of the FFN launches, zeroed here
     uint32_t gmax;            // compute groups the caller has room for
     uint32_t call_seq;        // written to the miss queue's seq word when the record is complete
     int policy;               // MELINOE_POLICY_LRU or MELINOE_POLICY_COUNT
     float gamma;              // decay of the count policy
     melinoe_moe_stats *stats; // may be null
     size_t expert_bytes;
-    int vr_capacity;
 };
 cudaError_t launch_plan(cudaStream_t stream, const PlanParams &p);
 
@@ -47,49 +46,57 @@ cudaError_t launch_route_plan_small(cudaStream_t stream, const uint16_t *x, cons
                                     const int32_t *token_seq, int d, int32_t *idx, float *gate, float *logits_out,
                                     const PlanParams &p);
 
-// ---- streaming expert FFN (Eq. 3) with the gate-weighted combine (Eq. 2) fused in
-struct FfnParams {
+// ---- decode expert FFN (Eq. 3) with the gate-weighted combine (Eq. 2) fused in, for up to 8 tokens per launch
+struct DecParams {
     const DevPlan *plan;
-    const VrRec *vrs;
     const uint16_t *x;               // hidden [T][d] bf16
+    const int32_t *idx;              // [T][k]
     const float *gate;               // [T][k]
-    uint16_t *hbuf;                  // h = SiLU(g) * u: [virtual request][8 token slots][Fpad] bf16
-    float *zbuf;                     // expert outputs: [T*k routed pairs, then n_shared*T][d] fp32
+    long long *yacc;                 // [8][d] output accumulator words of the launch; all zero between launches
+    float *ybuf;                     // [T][d] fp32: sum over the earlier launches of the same tokens (group mode)
     uint16_t *out;                   // [T][d] bf16
-    unsigned *sync;                  // grid-barrier counters, one per compute group (zero at launch)
+    unsigned *sync;                  // the handle's counter for the rare launches whose CTAs have to know who is last (zero between launches)
+    uint32_t call_seq;               // the call's sequence number: the plan is ready when plan->ready_seq equals it
     int *err;                        // device error word (0 = ok)
     unsigned long long *trace;       // null, or 8 clock stamps per CTA of the most recent launch
-    int d, F, Fpad, E, k, T, n_shared;
-    int group;
+    int d, F, E, k, T, n_shared;
+    int group;                       // -1: every request of the call in this one launch, the missed experts read
+                                     // straight from the host store; g >= 0: compute group g only, from the slots
+    int chunk, n_chunks;             // tokens [8 * chunk, 8 * chunk + 8) of the call; launches the call is made in
+    int write_back;                  // group -1: store the fetched experts that stay resident into their slots
+    int wait_prior;                  // the kernel ahead in the stream is another launch of the same call (it uses the
+                                     // same accumulator): wait for that grid to finish before anything else
+    int fmt;                         // 0: bf16 blobs, 1: 4-bit blobs
 };
-struct FfnLaunchCfg {
+struct DecLaunchCfg {
     int grid;                        // one CTA per SM
     size_t max_smem;                 // dynamic shared memory the kernel may use
     bool pdl;                        // launch with programmatic stream serialisation
 };
-// Shape of the shared-memory ring for one call.
-struct FfnGeometry {
-    int n_op_rows;                   // operand rows per stage: min(T, 8)
-    int n_stages, stage_bytes;       // the ring
-    int pitch, chunk_bytes;          // gate/up phase: row pitch in a stage, bytes per row piece (rows of 2*d bytes)
-    int pitch2, chunk_bytes2;        // down phase (rows of 2*d_ff bytes)
-    int sub2, sub_bytes2;            // down phase: sub-stages per ring slot and their size
-    int rows2;                       // down phase: weight rows of a sub-stage, min(16, ceil(d / grid)); the h rows follow
-    size_t ring_bytes, smem_bytes;
+// Shape of the shared-memory ring for one launch.
+struct DecGeometry {
+    int n_warps;                     // consumer warps: 8 (d <= 2048) or 16
+    int tile_rows;                   // f rows per tile / ring stage: 8, 4, 2 or 1
+    int n_stages;
+    int row_bytes;                   // bytes of one f row of the blob (its W_g, W_u and W_d^T rows)
+    int stage_bytes;
+    int x_pitch;                     // bytes between token rows of the staged hidden states
+    int tokens;                      // tokens of the launch (1..8)
+    size_t smem_bytes;
 };
-cudaError_t ffn_stream_configure(int n_sms, size_t max_smem, FfnLaunchCfg *cfg);
-cudaError_t ffn_stream_geometry(const FfnLaunchCfg &cfg, int d, int F, int T, FfnGeometry *geo);
-cudaError_t launch_ffn_stream(cudaStream_t stream, const FfnLaunchCfg &cfg, const FfnGeometry &geo,
-                              const FfnParams &p);
+cudaError_t ffn_decode_configure(int n_sms, size_t max_smem, DecLaunchCfg *cfg);
+bool ffn_decode_supported(int d, int F);
+cudaError_t ffn_decode_geometry(const DecLaunchCfg &cfg, int d, int F, int tokens, int fmt, DecGeometry *geo);
+cudaError_t launch_ffn_decode(cudaStream_t stream, const DecLaunchCfg &cfg, const DecGeometry &geo,
+                              const DecParams &p);
 
 // ---- grouped GEMM expert FFN on tcgen05 for calls with many tokens per expert (prefill)
 // Tensor maps in device memory, in this order:
 enum {
-    kMapXs = 0, kMapHs = 1, kMapSlotsD = 2, kMapSlotsF = 3,          // boxes of 128, 128, 128 and 256 rows
-    kMapShared0 = 4,                                                 // per shared expert: rows of d (128), rows of F (256)
-    kMapSlotsF128 = kMapShared0 + 2 * kMaxShared,                    // rows of F in boxes of 128 rows (CTA-pair kernel)
-    kMapSharedF128 = kMapSlotsF128 + 1,                              // the same per shared expert
-    kMapCount = kMapSharedF128 + kMaxShared
+    kMapXs = 0, kMapHs = 1,                                          // activations: boxes of 128 rows x 64 columns
+    kMapSlotsG = 2, kMapSlotsU = 3, kMapSlotsD = 4,                  // W_g, W_u rows (128-row boxes), W_d^T rows (64-row boxes) of all slots
+    kMapShared0 = 5,                                                 // per shared expert: the same three views
+    kMapCount = kMapShared0 + 3 * kMaxShared
 };
 struct GemmParams {
     const DevPlan *plan;
@@ -104,9 +111,6 @@ cudaError_t ffn_gemm_configure();
 cudaError_t launch_gather_rows(cudaStream_t stream, const DevPlan *plan, const uint16_t *x, const int32_t *tok_of_sorted,
                                uint16_t *xs, int d, int n_sorted, int n_sms);
 cudaError_t launch_ffn_gemm(cudaStream_t stream, int phase, int n_sms, const GemmParams &p);
-// the same two GEMMs on CTA pairs (tcgen05.mma.cta_group::2), for calls with many tokens per expert
-cudaError_t ffn_gemm_pair_configure();
-cudaError_t launch_ffn_gemm_pair(cudaStream_t stream, int phase, int n_sms, const GemmParams &p);
 cudaError_t launch_combine_rows(cudaStream_t stream, const DevPlan *plan, const float *gate, const int32_t *inv_pos,
                                 const float *zs, uint16_t *out, int T, int d, int k, int n_shared, int n_sms);
 

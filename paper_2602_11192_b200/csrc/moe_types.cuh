@@ -11,8 +11,8 @@ constexpr int kMaxExperts = 64;          // routed experts per layer (need-set i
 constexpr int kMaxShared = 8;            // always-resident shared experts
 constexpr int kMaxReq = kMaxExperts + kMaxShared;
 constexpr int kMaxGroups = kMaxExperts + 2;  // 1 + ceil(E / C) with C >= 1
-constexpr int kTokPerVr = 8;             // tokens per virtual request of the streaming FFN kernel
-constexpr int kUnitRows = 8;             // d_ff must be a multiple of this (one phase-1 tile of the FFN kernel)
+constexpr int kTokPerVr = 8;             // tokens one launch of the decode FFN kernel serves (its mma N dimension)
+constexpr int kUnitRows = 8;             // d_ff must be a multiple of this (the row swizzle of the expert blob has period 8)
 
 // Persistent cache state of one layer (device memory).  The reading of "LRU" used here:
 // every request takes stamp = ++counter; a hit re-stamps its slot; a miss takes the lowest
@@ -24,7 +24,7 @@ struct DevCache {
     uint64_t counter;
     uint64_t tot_hits, tot_misses, tot_evictions;
     uint64_t call_no;
-    uint64_t tot_vr;                        // virtual requests handed to the FFN kernels so far
+    uint64_t reserved0;
     // gamma-discounted request count of every expert (Definition C.1), kept for the count policy:
     // one step per forward call, count <- gamma * count + (requested ? 1 : 0), fp32, the product
     // rounded before the sum
@@ -43,24 +43,35 @@ struct ReqRec {
     int32_t group;     // compute group: 0 = resident at call entry, g >= 1 = g-th miss wave
 };
 
-// A virtual request: up to kTokPerVr tokens of one expert, with everything the FFN kernel
-// needs to serve it in one 80-byte record (one dependent load instead of a chain of them).
-struct __align__(16) VrRec {
-    const char *blob;            // the expert's weights: its cache slot, or a shared expert's blob
-    int32_t n_tok;               // 1..kTokPerVr
-    int32_t group;
-    int32_t tok[kTokPerVr];      // token (row of hidden) of each slot, -1 beyond n_tok
-    int32_t pair[kTokPerVr];     // row of the z buffer: t * k + j for routed pairs, T*k + s*T + t for shared
+// What the decode FFN kernel needs to serve one request (one distinct expert of the call, or a
+// shared expert): where its weights are and what has to happen to them.  One 32-byte record, read
+// with one load.
+struct __align__(32) DecReq {
+    const char *blob;            // the expert's cache slot, or a shared expert's blob (device memory)
+    const char *host;            // the expert's blob in the page-locked host store as the device sees it, or null
+    int32_t expert;              // routed: 0..E-1; shared: E + s
+    int32_t flags;               // kDecMiss | kDecStays | kDecHazard
+    int32_t group;               // compute group (0 = resident at call entry or shared, g >= 1 = g-th miss wave)
+    int32_t reserved;
 };
+constexpr int kDecMiss = 1;      // not resident at call entry: the weights come from the host store
+constexpr int kDecStays = 2;     // a miss that still occupies its slot when the call ends: written into the slot
+constexpr int kDecHazard = 4;    // ... whose slot held, at call entry, an expert that this call also computes with
 
 // Per-call plan written by the planning kernel, read by the FFN and combine kernels.
 struct DevPlan {
-    int32_t n_tokens, n_req, n_hits, n_miss, n_evict, n_groups, n_vr, status;
-    int32_t group_vr_begin[kMaxGroups + 1];
+    int32_t n_tokens, n_req, n_hits, n_miss, n_evict, n_groups, n_dreq, status;
+    // Sequence number of the call whose plan this is, written last (after a device-wide fence) by the
+    // planning kernel: the decode FFN kernel, which may have been scheduled while the planner was still
+    // running, waits for it instead of waiting for the planner's grid to drain.
+    uint32_t ready_seq;
+    uint32_t pad_[3];
+    int32_t group_vr_begin[kMaxGroups + 1];   // first entry of dreq[] of every compute group
     int32_t counts[kMaxReq];
     int32_t offsets[kMaxReq + 1];
     int32_t req_of_expert[kMaxReq];        // -1 = expert not requested by this call
     ReqRec req[kMaxReq];
+    DecReq dreq[kMaxReq];                     // group 0 (hits, then shared experts), then the misses by wave
 };
 
 // The miss queue of a call: what the host needs in order to issue the transfers, written by

@@ -36,7 +36,8 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p)
     __shared__ int32_t s_victim[kMaxExperts];                    // V: slots in victim order
     __shared__ int32_t s_miss_expert[kMaxExperts];               // expert of miss number i
     __shared__ int32_t s_entry_occ[kMaxExperts];                 // occupant of a slot at call entry
-    __shared__ int32_t s_misc[8];  // 0 n_req(routed) 1 n_hits 2 n_miss 3 n_evict 4 n_groups 5 n_vr 6 status 7 n_req_total
+    __shared__ int32_t s_miss_flags[kMaxExperts];                // kDecStays / kDecHazard of miss number i
+    __shared__ int32_t s_misc[8];  // 0 n_req(routed) 1 n_hits 2 n_miss 3 n_evict 4 n_groups 5 n_dreq 6 status 7 n_req_total
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n_pairs = p.T * p.k;
@@ -122,8 +123,6 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p)
     }
     for (int i = tid; i < p.n_shared * p.T; i += kPlanThreads)
         p.tok_of_sorted[n_pairs + i] = i % p.T;
-    for (int i = tid; i < 2 * (kMaxGroups + 1); i += kPlanThreads)
-        p.sync[i] = 0u;      // two barrier counters per compute group
 
     // ---- (b), (c): cache requests, by warp 0; lane owns experts lane and lane + 32 and slots lane and
     // lane + 32.  The sequential rules (hits in ascending id, then misses in ascending id, a miss
@@ -248,6 +247,14 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p)
                 __syncwarp();
             }
             n_groups = n_miss ? cur_group + 1 : 1;
+            // a miss stays if it still occupies its slot when the call ends; storing it there has to
+            // wait for the call's compute if the slot held one of the call's hits at entry
+            for (int j = lane; j < n_miss; j += 32) {
+                const int e = s_miss[j].expert, slot = s_miss[j].slot, occ = s_entry_occ[slot];
+                const bool stays = s_cache.expert_of_slot[slot] == e;
+                const bool hazard = stays && occ >= 0 && ((need >> occ) & 1ull);
+                s_miss_flags[j] = (stays ? kDecStays : 0) | (hazard ? kDecHazard : 0);
+            }
         } else
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
@@ -268,6 +275,11 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p)
                 s_miss[i] = HostMiss{e, slot, (int16_t)group, (int16_t)dep, 0u};
                 // cache update: the last miss that lands in a slot keeps it
                 const bool stays = i + C >= n_miss;
+                {
+                    const int occ = s_entry_occ[slot];
+                    const bool hazard = stays && occ >= 0 && ((need >> occ) & 1ull);
+                    s_miss_flags[i] = (stays ? kDecStays : 0) | (hazard ? kDecHazard : 0);
+                }
                 s_cache.slot_of_expert[e] = stays ? slot : -1;
                 if (stays) {
                     s_cache.expert_of_slot[slot] = e;
@@ -287,47 +299,42 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p)
                 s_req_of_expert[E + s] = n_req_total;
                 ++n_req_total;
             }
-            // virtual requests, grouped: group 0 = hits then shared, then the miss waves in order
-            int nvr = 0;
+            // records for the compute kernels, grouped: group 0 = hits then shared experts, then the
+            // miss waves in order
+            int ndr = 0;
             s_group_vr_begin[0] = 0;
-            for (int r = 0; r < n_hits; ++r) {
-                s_req[r].vr_start = nvr;
-                nvr += (s_req[r].n_tok + kTokPerVr - 1) / kTokPerVr;
-            }
-            for (int r = n_req; r < n_req_total; ++r) {
-                s_req[r].vr_start = nvr;
-                nvr += (s_req[r].n_tok + kTokPerVr - 1) / kTokPerVr;
-            }
+            for (int r = 0; r < n_hits; ++r)
+                s_req[r].vr_start = ndr++;
+            for (int r = n_req; r < n_req_total; ++r)
+                s_req[r].vr_start = ndr++;
             int g = 0;
             for (int r = n_hits; r < n_req; ++r) {
                 while (g < s_req[r].group)
-                    s_group_vr_begin[++g] = nvr;
-                s_req[r].vr_start = nvr;
-                nvr += (s_req[r].n_tok + kTokPerVr - 1) / kTokPerVr;
+                    s_group_vr_begin[++g] = ndr;
+                s_req[r].vr_start = ndr++;
             }
             while (g < kMaxGroups)
-                s_group_vr_begin[++g] = nvr;
+                s_group_vr_begin[++g] = ndr;
             int status = s_misc[6];
-            if (nvr > p.vr_capacity || n_groups > (int)p.gmax)
+            if (n_groups > (int)p.gmax)
                 status = MELINOE_ERR_STATE;
             if (status != MELINOE_OK) {
                 // leave nothing for the compute kernels to do
                 for (int i = 0; i <= kMaxGroups; ++i)
                     s_group_vr_begin[i] = 0;
-                nvr = 0;
+                ndr = 0;
             }
             s_cache.counter = counter;
             s_cache.tot_hits += (uint64_t)n_hits;
             s_cache.tot_misses += (uint64_t)n_miss;
             s_cache.tot_evictions += (uint64_t)n_evict;
             s_cache.call_no += 1;
-            s_cache.tot_vr += (uint64_t)nvr;
             s_misc[0] = n_req;
             s_misc[1] = n_hits;
             s_misc[2] = n_miss;
             s_misc[3] = n_evict;
             s_misc[4] = n_groups;
-            s_misc[5] = nvr;
+            s_misc[5] = ndr;
             s_misc[6] = status;
             s_misc[7] = n_req_total;
         }
@@ -345,7 +352,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p)
         plan->n_miss = s_misc[2];
         plan->n_evict = s_misc[3];
         plan->n_groups = s_misc[4];
-        plan->n_vr = s_misc[5];
+        plan->n_dreq = s_misc[5];
         plan->status = s_misc[6];
     }
     for (int i = tid; i <= kMaxGroups; i += kPlanThreads)
@@ -359,23 +366,21 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p)
     for (int i = tid; i < n_req_total; i += kPlanThreads)
         plan->req[i] = s_req[i];
     if (ok) {
-        // a warp per request, a lane per virtual request
-        for (int r = warp; r < n_req_total; r += kPlanWarps) {
+        const int n_hits = s_misc[1];
+        for (int r = tid; r < n_req_total; r += kPlanThreads) {
             const ReqRec rec = s_req[r];
-            const int nv = (rec.n_tok + kTokPerVr - 1) / kTokPerVr;
-            for (int v = lane; v < nv; v += 32) {
-                VrRec vr;
-                vr.blob = rec.slot >= 0 ? p.slots + (size_t)rec.slot * p.slot_stride : p.shared_blobs[rec.expert - E];
-                vr.n_tok = min(kTokPerVr, rec.n_tok - v * kTokPerVr);
-                vr.group = rec.group;
-                const int off = rec.tok_off + v * kTokPerVr;
-                for (int i = 0; i < kTokPerVr; ++i) {
-                    const int pos = off + i;
-                    vr.tok[i] = i < vr.n_tok ? p.tok_of_sorted[pos] : -1;
-                    vr.pair[i] = i < vr.n_tok ? (pos < n_pairs ? p.perm[pos] : pos) : -1;
-                }
-                p.vrs[rec.vr_start + v] = vr;
+            DecReq q;
+            q.blob = rec.slot >= 0 ? p.slots + (size_t)rec.slot * p.slot_stride : p.shared_blobs[rec.expert - E];
+            q.host = nullptr;
+            q.expert = rec.expert;
+            q.flags = 0;
+            q.group = rec.group;
+            q.reserved = 0;
+            if (!rec.hit) {
+                q.host = p.host_blobs ? p.host_blobs[rec.expert] : nullptr;
+                q.flags = kDecMiss | s_miss_flags[r - n_hits];
             }
+            plan->dreq[rec.vr_start] = q;
         }
     }
     {
@@ -403,6 +408,13 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p)
             *p.stats = st;
         }
         publish_miss_queue(p.hplan, s_miss, n_miss, s_misc[4], s_misc[6], p.call_seq);
+    }
+    // the plan is complete: announce it (see DevPlan::ready_seq)
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        __threadfence();
+        asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(&plan->ready_seq), "r"(p.call_seq) : "memory");
     }
 }
 

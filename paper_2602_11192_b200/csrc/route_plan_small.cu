@@ -64,23 +64,6 @@ __device__ __forceinline__ uint64_t ballot64(bool lo, bool hi)
 
 __device__ __forceinline__ int rank_below(uint64_t mask, int bit) { return __popcll(mask & ((1ull << bit) - 1ull)); }
 
-// The virtual request of one expert (at most 8 tokens here): its tokens and z rows from the sorted lists.
-__device__ __forceinline__ void write_vr(VrRec *dst, const char *blob, int n_tok, int group, int off,
-                                         const int32_t *pair_at, const int32_t *tok_of_pair)
-{
-    VrRec vr;
-    vr.blob = blob;
-    vr.n_tok = n_tok;
-    vr.group = group;
-#pragma unroll
-    for (int j = 0; j < kTokPerVr; ++j) {
-        const int pr = j < n_tok ? pair_at[off + j] : -1;
-        vr.tok[j] = pr >= 0 ? tok_of_pair[pr] : -1;
-        vr.pair[j] = pr;
-    }
-    *dst = vr;
-}
-
 __global__ void __launch_bounds__(kThreads, 1)
 route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restrict__ w_r,
                         const float *__restrict__ bias, const int32_t *__restrict__ token_seq, int d,
@@ -102,6 +85,9 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
     __shared__ unsigned long long s_key[kMaxExperts];            // victim-order key of a slot
     __shared__ int32_t s_victim[kMaxExperts];                    // V: slots in victim order
     __shared__ int32_t s_miss_expert[kMaxExperts];               // expert of miss number i
+    __shared__ HostMiss s_hm[kMaxExperts];                       // the call's miss queue, sent to the host last
+    __shared__ int32_t s_miss_slot[kMaxExperts];                 // count policy: its slot and wave
+    __shared__ int32_t s_miss_group[kMaxExperts];
     __shared__ int32_t s_entry_occ[kMaxExperts];                 // occupant of a slot at call entry
     __shared__ float s_sel[kMaxT][kMaxExperts];                  // a token's selected logits, by rank
 
@@ -225,8 +211,6 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
     if (cta_rank != 0)
         return;
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-    for (int i = tid; i < 2 * (kMaxGroups + 1); i += kThreads)
-        p.sync[i] = 0u;
 
     // ================================================================ top-k
     // An element's rank is the number of elements that beat it (greater, or equal with a lower
@@ -286,6 +270,8 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
                 gate_out[(size_t)t * k + lane] = ev / sum;
             }
         }
+        // these warps' results are written before the planning warp announces the plan
+        asm volatile("bar.arrive 2, %0;" ::"n"(kThreads) : "memory");
         return;
     }
 
@@ -340,8 +326,8 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
     // compute groups: closed form under LRU; under the count policy known only after the misses
     // have been walked, one wave per miss at most
     int n_groups = n_miss ? 1 + (by_count ? n_miss : (n_miss + C - 1) / C) : 1;
-    const int nvr = n_req + p.n_shared;
-    const int status = (nvr > p.vr_capacity || n_groups > (int)p.gmax) ? MELINOE_ERR_STATE : MELINOE_OK;
+    const int ndr = n_req + p.n_shared;             // records for the compute kernels: hits, shared experts, misses
+    const int status = n_groups > (int)p.gmax ? MELINOE_ERR_STATE : MELINOE_OK;
     const bool ok = status == MELINOE_OK;
     if (by_count) {
         // Definition C.1: one time step per call, count <- gamma * count + request
@@ -372,8 +358,7 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
             cache->stamp[soe] = st;
             plan->req[r] = ReqRec{e, soe, 1, -1, off, cnt, r, 0};
             s_grp_of[e] = 0;
-            if (ok)
-                write_vr(p.vrs + r, p.slots + (size_t)soe * p.slot_stride, cnt, 0, off, s_pair_at, s_tok);
+            plan->dreq[r] = DecReq{p.slots + (size_t)soe * p.slot_stride, nullptr, e, 0, 0, 0};
         }
         if ((miss_mask >> e) & 1ull)
             s_miss_expert[rank_below(miss_mask, e)] = e;
@@ -466,14 +451,24 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
                 s_live_stamp[slot] = st;
                 s_grp_of[e] = cur_group;
                 plan->req[n_hits + i] = ReqRec{e, slot, 0, ev, off, cnt, vr_at, cur_group};
-                if (ok)
-                    write_vr(p.vrs + vr_at, p.slots + (size_t)slot * p.slot_stride, cnt, cur_group, off, s_pair_at, s_tok);
-                const HostMiss hm{e, slot, (int16_t)cur_group, (int16_t)dep, p.call_seq};
-                store16_host(&p.hplan->miss[i], &hm);
+                s_miss_expert[i] = e;
+                s_miss_slot[i] = slot;
+                s_miss_group[i] = cur_group;
+                s_hm[i] = HostMiss{e, slot, (int16_t)cur_group, (int16_t)dep, p.call_seq};
             }
             __syncwarp();
         }
         n_groups = n_miss ? cur_group + 1 : 1;
+        // a miss stays if it still occupies its slot when the call ends; writing it there must wait
+        // for the end of the call's compute if the slot held one of the call's hits at entry
+        for (int j = lane; j < n_miss; j += 32) {
+            const int e = s_miss_expert[j], slot = s_miss_slot[j], occ = s_entry_occ[slot];
+            const bool stays = s_live_occ[slot] == e;
+            const bool hazard = stays && occ >= 0 && ((need >> occ) & 1ull);
+            plan->dreq[n_hits + p.n_shared + j] =
+                DecReq{p.slots + (size_t)slot * p.slot_stride, p.host_blobs ? p.host_blobs[e] : nullptr, e,
+                       kDecMiss | (stays ? kDecStays : 0) | (hazard ? kDecHazard : 0), s_miss_group[j], 0};
+        }
     } else
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
@@ -491,10 +486,14 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
             ev_flag[h] = ev >= 0;
             const int vr_at = n_hits + p.n_shared + i;
             plan->req[n_hits + i] = ReqRec{e, slot, 0, ev, off, cnt, vr_at, group};
-            if (ok)
-                write_vr(p.vrs + vr_at, p.slots + (size_t)slot * p.slot_stride, cnt, group, off, s_pair_at, s_tok);
             // cache update: the last miss that lands in a slot keeps it
             const bool stays = i + C >= n_miss;
+            {
+                const int occ = s_entry_occ[slot];
+                const bool hazard = stays && occ >= 0 && ((need >> occ) & 1ull);
+                plan->dreq[vr_at] = DecReq{p.slots + (size_t)slot * p.slot_stride, p.host_blobs ? p.host_blobs[e] : nullptr, e,
+                                           kDecMiss | (stays ? kDecStays : 0) | (hazard ? kDecHazard : 0), group, 0};
+            }
             cache->slot_of_expert[e] = stays ? slot : -1;
             if (stays) {
                 cache->expert_of_slot[slot] = e;
@@ -502,8 +501,7 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
             }
             if (i < C && ev >= 0)
                 cache->slot_of_expert[ev] = -1;
-            const HostMiss m{e, slot, (int16_t)group, (int16_t)dep, p.call_seq};
-            store16_host(&p.hplan->miss[i], &m);
+            s_hm[i] = HostMiss{e, slot, (int16_t)group, (int16_t)dep, p.call_seq};
         }
     }
     const int n_evict = by_count ? n_evict_seq : __popcll(ballot64(ev_flag[0], ev_flag[1]));
@@ -511,17 +509,7 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
     for (int s = lane; s < p.n_shared; s += 32) {
         const int off = n_pairs + s * T;
         plan->req[n_req + s] = ReqRec{E + s, -1, 1, -1, off, T, n_hits + s, 0};
-        if (ok) {
-            VrRec vr;
-            vr.blob = p.shared_blobs[s];
-            vr.n_tok = T;
-            vr.group = 0;
-            for (int j = 0; j < kTokPerVr; ++j) {
-                vr.tok[j] = j < T ? j : -1;
-                vr.pair[j] = j < T ? off + j : -1;
-            }
-            p.vrs[n_hits + s] = vr;
-        }
+        plan->dreq[n_hits + s] = DecReq{p.shared_blobs[s], nullptr, E + s, 0, 0, 0};
     }
     // group boundaries, counts and offsets (what the FFN launches and the inspection calls read)
     for (int g = lane; g <= kMaxGroups; g += 32) {
@@ -553,14 +541,28 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
         plan->n_miss = n_miss;
         plan->n_evict = n_evict;
         plan->n_groups = n_groups;
-        plan->n_vr = ok ? nvr : 0;
+        plan->n_dreq = ok ? ndr : 0;
         plan->status = status;
         cache->counter = counter + (unsigned long long)n_req;
         cache->tot_hits += (unsigned long long)n_hits;
         cache->tot_misses += (unsigned long long)n_miss;
         cache->tot_evictions += (unsigned long long)n_evict;
         cache->call_no = call_no;
-        cache->tot_vr += (unsigned long long)(ok ? nvr : 0);
+    }
+    // The plan is complete: announce it.  The decode FFN kernel behind this one in the stream may
+    // already be running (programmatic launch) and waits for this word, not for this grid to drain.
+    // (The barrier orders the other warps' and lanes' writes before lane 0's release.)
+    asm volatile("bar.sync 2, %0;" ::"n"(kThreads) : "memory");
+    if (lane == 0) {
+        __threadfence();
+        asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(&plan->ready_seq), "r"(p.call_seq) : "memory");
+    }
+    // What may live in host memory goes out last, so that no fence above has to wait for the host link:
+    // the statistics, and the miss queue for calls whose transfers the host issues.
+    for (int i = lane; i < n_miss; i += 32)
+        store16_host(&p.hplan->miss[i], &s_hm[i]);
+    __syncwarp();
+    if (lane == 0) {
         if (p.stats) {
             melinoe_moe_stats st;
             st.status = status;

@@ -137,12 +137,13 @@ class LayerSetup:
         self.layer.set_router_bias(self.bias_dev, self.seq_dev, bias.shape[0])
 
     # -- one call with numpy in / numpy out (blocking; for tests)
-    def forward_np(self, hidden_bits: np.ndarray, want_stats: bool = True):
+    def forward_np(self, hidden_bits: np.ndarray, want_stats: bool = True, entry: str = "forward"):
         T = hidden_bits.shape[0]
         x = to_dev_bf16(hidden_bits)
-        out = torch.empty((T, self.d), dtype=torch.int16, device="cuda")
+        out = torch.full((T, self.d), 0x7FC0, dtype=torch.int16, device="cuda")   # NaN pattern: must be overwritten
         stats = torch.zeros(12, dtype=torch.int32, device="cuda") if want_stats else None
-        self.layer.forward(current_stream_ptr(), x, T, out, stats)
+        call = self.layer.forward_static if entry == "static" else self.layer.forward
+        call(current_stream_ptr(), x, T, out, stats)
         torch.cuda.synchronize()
         res = {"out_bits": out.cpu().numpy().view(np.uint16)}
         if want_stats:

@@ -12,6 +12,7 @@ import pytest
 
 import gen
 import oracle
+from parity_util import elementwise_excess
 
 pytestmark = pytest.mark.gpu
 
@@ -59,6 +60,8 @@ def _run_stack(name, n_layers, alpha, C, decode_steps, sample_layers, prefill=Tr
                 yg = gen.bf16_bits_to_f32(out_bits[l][toks]).astype(np.float64)
                 err = np.linalg.norm(yg - y, axis=1) / np.maximum(np.linalg.norm(y, axis=1), 1e-30)
                 assert np.all(np.isfinite(yg)) and err.max() <= REL_TOL, "rel err %.3e" % err.max()
+                ex = elementwise_excess(out_bits[l][toks], y)
+                assert ex <= 1.0, "%s layer %d: an output element is off by %.2f times its bound" % (name, l, ex)
                 worst = max(worst, float(err.max()))
         return worst
 

@@ -37,13 +37,23 @@ def test_status_strings_and_sizes(m):
 
 
 def test_pack_expert_layout(m):
+    """Per hidden unit f the blob holds W_g[f] | W_u[f] | W_d[:, f]; inside every 64-element group the
+    eight 8-element pieces sit at (piece xor (f mod 8)).  Undoing that permutation with index
+    arithmetic written here gives the three matrices back."""
     d, F = 256, 24
     wg, wu, wd = gen.expert_weights(1, 0, 0, d, F)
     blob = np.zeros(3 * d * F, np.uint16)
     m.melinoe_moe_pack_expert(d, F, wg.ctypes.data, wu.ctypes.data, wd.ctypes.data, blob.ctypes.data)
-    n = d * F
-    assert np.array_equal(blob[:n].reshape(F, d), wg) and np.array_equal(blob[n:2 * n].reshape(F, d), wu)
-    assert np.array_equal(blob[2 * n:].reshape(d, F), wd)
+    rows = blob.reshape(F, 3, d // 64, 8, 8)                     # f, vector, group, stored piece, element
+    plain = np.empty_like(rows)
+    for f in range(F):
+        for piece in range(8):
+            plain[f, :, :, piece, :] = rows[f, :, :, piece ^ (f & 7), :]
+    plain = plain.reshape(F, 3, d)
+    assert np.array_equal(plain[:, 0, :], wg) and np.array_equal(plain[:, 1, :], wu)
+    assert np.array_equal(plain[:, 2, :], wd.T)
+    # rows 0 and 8 are stored unpermuted, row 1 swaps neighbouring pieces
+    assert np.array_equal(blob[:8], wg[0, :8]) and np.array_equal(blob[3 * d:3 * d + 8], wg[1, 8:16])
     with pytest.raises(m.MelinoeError):
         m.melinoe_moe_pack_expert(d, F, 0, wu.ctypes.data, wd.ctypes.data, blob.ctypes.data)
 
