@@ -32,15 +32,15 @@ struct DevCache {
 };
 
 // One cache request of a call plus what the compute kernels need to serve it.
-struct ReqRec {
+struct __align__(16) ReqRec {
     int32_t expert;    // routed: 0..E-1; shared: E + s
     int32_t slot;      // cache slot, or -1 for a shared expert
     int32_t hit;
     int32_t evicted;   // expert displaced by this request, or -1
+    int32_t vr_start;  // its entry of DevPlan::dreq
+    int32_t group;     // compute group: 0 = resident at call entry, g >= 1 = g-th miss wave
     int32_t tok_off;   // first entry of this expert's token list in the sorted arrays
     int32_t n_tok;     // tokens routed to it
-    int32_t vr_start;  // first virtual request (global index within the call)
-    int32_t group;     // compute group: 0 = resident at call entry, g >= 1 = g-th miss wave
 };
 
 // What the decode FFN kernel needs to serve one request (one distinct expert of the call, or a

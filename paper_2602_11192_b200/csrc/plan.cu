@@ -164,7 +164,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p)
                 const uint64_t st = counter + (uint64_t)r + 1ull;
                 s_key[soe] = (1ull << 63) | st;
                 s_cache.stamp[soe] = st;
-                s_req[r] = ReqRec{e, soe, 1, -1, s_offsets[e], s_counts[e], 0, 0};
+                s_req[r] = ReqRec{e, soe, 1, -1, 0, 0, s_offsets[e], s_counts[e]};
                 s_req_of_expert[e] = r;
                 s_group_of_expert[e] = 0;
             }
@@ -239,7 +239,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p)
                     s_cache.expert_of_slot[slot] = e;
                     s_cache.slot_of_expert[e] = slot;
                     s_cache.stamp[slot] = counter + (uint64_t)(n_hits + i) + 1ull;
-                    s_req[n_hits + i] = ReqRec{e, slot, 0, ev, s_offsets[e], s_counts[e], 0, cur_group};
+                    s_req[n_hits + i] = ReqRec{e, slot, 0, ev, 0, cur_group, s_offsets[e], s_counts[e]};
                     s_req_of_expert[e] = n_hits + i;
                     s_group_of_expert[e] = cur_group;
                     s_miss[i] = HostMiss{e, slot, (int16_t)cur_group, (int16_t)dep, 0u};
@@ -270,7 +270,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p)
                 else if (ev >= 0 && ((need >> ev) & 1ull))
                     dep = 0;
                 ev_flag[h] = ev >= 0;
-                s_req[n_hits + i] = ReqRec{e, slot, 0, ev, s_offsets[e], s_counts[e], 0, group};
+                s_req[n_hits + i] = ReqRec{e, slot, 0, ev, 0, group, s_offsets[e], s_counts[e]};
                 s_req_of_expert[e] = n_hits + i;
                 s_miss[i] = HostMiss{e, slot, (int16_t)group, (int16_t)dep, 0u};
                 // cache update: the last miss that lands in a slot keeps it
@@ -295,7 +295,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p)
         if (lane == 0) {
             int n_req_total = n_req;
             for (int s = 0; s < p.n_shared; ++s) {
-                s_req[n_req_total] = ReqRec{E + s, -1, 1, -1, s_offsets[E + s], p.T, 0, 0};
+                s_req[n_req_total] = ReqRec{E + s, -1, 1, -1, 0, 0, s_offsets[E + s], p.T};
                 s_req_of_expert[E + s] = n_req_total;
                 ++n_req_total;
             }

@@ -64,6 +64,13 @@ __device__ __forceinline__ uint64_t ballot64(bool lo, bool hi)
 
 __device__ __forceinline__ int rank_below(uint64_t mask, int bit) { return __popcll(mask & ((1ull << bit) - 1ull)); }
 
+// The cache half of a request record (the gather warp writes tok_off / n_tok, the other two words).
+__device__ __forceinline__ void write_req(ReqRec *r, int expert, int slot, int hit, int evicted, int at, int group)
+{
+    *reinterpret_cast<int4 *>(&r->expert) = make_int4(expert, slot, hit, evicted);
+    *reinterpret_cast<int2 *>(&r->vr_start) = make_int2(at, group);
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
 route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restrict__ w_r,
                         const float *__restrict__ bias, const int32_t *__restrict__ token_seq, int d,
@@ -81,10 +88,10 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
     __shared__ int32_t s_grp_of[kMaxExperts];
     __shared__ int32_t s_grp_first[kMaxGroups + 1];              // first miss of a wave
     __shared__ int32_t s_idx[kMaxPairs];
-    __shared__ int32_t s_pair_at[kMaxPairs];                     // pair at sorted position
     __shared__ unsigned long long s_key[kMaxExperts];            // victim-order key of a slot
     __shared__ int32_t s_victim[kMaxExperts];                    // V: slots in victim order
     __shared__ int32_t s_miss_expert[kMaxExperts];               // expert of miss number i
+    __shared__ int32_t s_needflags[2][kMaxExperts];              // per planning warp: 1 = some pair of the call names this expert
     __shared__ HostMiss s_hm[kMaxExperts];                       // the call's miss queue, sent to the host last
     __shared__ int32_t s_miss_slot[kMaxExperts];                 // count policy: its slot and wave
     __shared__ int32_t s_miss_group[kMaxExperts];
@@ -128,6 +135,13 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
     unsigned long long st0 = 0ull, st1 = 0ull, counter = 0ull, call_no = 0ull;
     float cnt0 = 0.0f, cnt1 = 0.0f;
     const bool by_count = p.policy == MELINOE_POLICY_COUNT;
+    if (cta_rank == 0 && warp == 1) {
+        // the gather warp only needs to know which experts are resident
+        if (lane < E)
+            soe0 = cache->slot_of_expert[lane];
+        if (lane + 32 < E)
+            soe1 = cache->slot_of_expert[lane + 32];
+    }
     if (cta_rank == 0 && warp == 0) {
         if (by_count) {
             if (lane < E)
@@ -256,9 +270,9 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
         }
         __syncthreads();
     }
-    if (warp != 0) {
+    if (warp >= 2) {
         // ============================================================ gates (Eq. 1), off the planner's path
-        for (int t = warp - 1; t < T; t += kWarpsPerBlock - 1) {
+        for (int t = warp - 2; t < T; t += kWarpsPerBlock - 2) {
             const float top = s_sel[t][0];
             const float ev = lane < k ? expf(s_sel[t][lane] - top) : 0.0f;
             float sum = ev;
@@ -275,54 +289,96 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
         return;
     }
 
-    // ================================================================ planning, by one warp
+    // ================================================================ planning, by two warps side by side
+    // Warp 1 builds the token lists (what the gather and the inspection calls need), warp 0 the cache
+    // requests (what the compute kernel waits for).  Both know which experts are needed and which of
+    // those are resident, so both can tell a request's place in the call's request order.
     // lane owns experts lane and lane + 32, slots lane and lane + 32, pairs lane and lane + 32
     // (the cache state of this lane's experts and slots was loaded before the logits)
     DevPlan *plan = p.plan;
     const int e0 = lane, e1 = lane + 32;
-
-    // ---- token lists: counts, offsets, stable positions (pairs in increasing flat index)
-    // Lane q also stands for pairs q and q + 32: the lanes whose pair names the same expert find
-    // one another with a match, so an expert's count and a pair's place among its expert's pairs
-    // are population counts.
-    const int qe[2] = {lane < n_pairs ? s_idx[lane] : -1 - lane, lane + 32 < n_pairs ? s_idx[lane + 32] : -1 - lane};
-    const unsigned lt = (1u << lane) - 1u;
-    const unsigned same[2] = {__match_any_sync(0xffffffffu, qe[0]), __match_any_sync(0xffffffffu, qe[1])};
-    s_cnt[0][lane] = s_cnt[0][lane + 32] = s_cnt[1][lane] = s_cnt[1][lane + 32] = 0;
-    s_tok[lane] = lane / k;
-    s_tok[lane + 32] = (lane + 32) / k;
+    // which experts the call's pairs name
+    int32_t *s_needflag = s_needflags[warp];
+    s_needflag[lane] = 0;
+    s_needflag[lane + 32] = 0;
     __syncwarp();
-#pragma unroll
-    for (int h = 0; h < 2; ++h)
-        if (qe[h] >= 0 && (same[h] & lt) == 0u)
-            s_cnt[h][qe[h]] = __popc(same[h]);
+    if (lane < n_pairs)
+        s_needflag[s_idx[lane]] = 1;
+    if (lane + 32 < n_pairs)
+        s_needflag[s_idx[lane + 32]] = 1;
     __syncwarp();
-    const int c0 = s_cnt[0][e0] + s_cnt[1][e0], c1 = s_cnt[0][e1] + s_cnt[1][e1];
-    int tot0, tot1;
-    const int off0 = warp_excl_scan(c0, lane, tot0);
-    const int off1 = tot0 + warp_excl_scan(c1, lane, tot1);
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-        const int q = lane + 32 * h;
-        const int e = qe[h] >= 0 ? qe[h] : 0;
-        const int r = __popc(same[h] & lt) + (h ? s_cnt[0][e] : 0);
-        const int o0 = __shfl_sync(0xffffffffu, off0, e & 31), o1 = __shfl_sync(0xffffffffu, off1, e & 31);
-        if (q < n_pairs) {
-            const int pos = (e < 32 ? o0 : o1) + r;
-            s_pair_at[pos] = q;
-            p.perm[pos] = q;
-            p.inv_pos[q] = pos;
-            p.tok_of_sorted[pos] = s_tok[q];
-        }
-    }
-    for (int i = lane; i < p.n_shared * T; i += 32)
-        p.tok_of_sorted[n_pairs + i] = i % T;
-
-    // ---- hits and misses
-    const uint64_t need = ballot64(c0 > 0, c1 > 0);
+    const uint64_t need = ballot64(s_needflag[lane] != 0, s_needflag[lane + 32] != 0);
     const uint64_t resident = ballot64(soe0 >= 0, soe1 >= 0);
     const uint64_t hit_mask = need & resident, miss_mask = need & ~resident;
     const int n_hits = __popcll(hit_mask), n_miss = __popcll(miss_mask), n_req = n_hits + n_miss;
+
+    if (warp == 1) {
+        // ---- token lists: counts, offsets, stable positions (pairs in increasing flat index)
+        // Lane q also stands for pairs q and q + 32: the lanes whose pair names the same expert find
+        // one another with a match, so an expert's count and a pair's place among its expert's pairs
+        // are population counts.
+        const int qe[2] = {lane < n_pairs ? s_idx[lane] : -1 - lane, lane + 32 < n_pairs ? s_idx[lane + 32] : -1 - lane};
+        const unsigned lt = (1u << lane) - 1u;
+        const unsigned same[2] = {__match_any_sync(0xffffffffu, qe[0]), __match_any_sync(0xffffffffu, qe[1])};
+        s_cnt[0][lane] = s_cnt[0][lane + 32] = s_cnt[1][lane] = s_cnt[1][lane + 32] = 0;
+        s_tok[lane] = lane / k;
+        s_tok[lane + 32] = (lane + 32) / k;
+        __syncwarp();
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+            if (qe[h] >= 0 && (same[h] & lt) == 0u)
+                s_cnt[h][qe[h]] = __popc(same[h]);
+        __syncwarp();
+        const int c0 = s_cnt[0][e0] + s_cnt[1][e0], c1 = s_cnt[0][e1] + s_cnt[1][e1];
+        int tot0, tot1;
+        const int off0 = warp_excl_scan(c0, lane, tot0);
+        const int off1 = tot0 + warp_excl_scan(c1, lane, tot1);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int q = lane + 32 * h;
+            const int e = qe[h] >= 0 ? qe[h] : 0;
+            const int r = __popc(same[h] & lt) + (h ? s_cnt[0][e] : 0);
+            const int o0 = __shfl_sync(0xffffffffu, off0, e & 31), o1 = __shfl_sync(0xffffffffu, off1, e & 31);
+            if (q < n_pairs) {
+                const int pos = (e < 32 ? o0 : o1) + r;
+                p.perm[pos] = q;
+                p.inv_pos[q] = pos;
+                p.tok_of_sorted[pos] = s_tok[q];
+            }
+        }
+        for (int i = lane; i < p.n_shared * T; i += 32)
+            p.tok_of_sorted[n_pairs + i] = i % T;
+        // every request's token list: its record's place follows from the masks (hits in ascending
+        // id, then the misses in ascending id, then the shared experts)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int e = h ? e1 : e0, cnt = h ? c1 : c0, off = h ? off1 : off0;
+            if ((need >> e) & 1ull) {
+                const int r = ((hit_mask >> e) & 1ull) ? rank_below(hit_mask, e) : n_hits + rank_below(miss_mask, e);
+                *reinterpret_cast<int2 *>(&plan->req[r].tok_off) = make_int2(off, cnt);
+            }
+        }
+        for (int sh = lane; sh < p.n_shared; sh += 32)
+            *reinterpret_cast<int2 *>(&plan->req[n_req + sh].tok_off) = make_int2(n_pairs + sh * T, T);
+        if (e0 < E) {
+            plan->counts[e0] = c0;
+            plan->offsets[e0] = off0;
+        }
+        if (e1 < E) {
+            plan->counts[e1] = c1;
+            plan->offsets[e1] = off1;
+        }
+        if (lane <= p.n_shared) {
+            if (lane < p.n_shared)
+                plan->counts[E + lane] = T;
+            plan->offsets[E + lane] = n_pairs + lane * T;
+        }
+        asm volatile("bar.arrive 2, %0;" ::"n"(kThreads) : "memory");
+        return;
+    }
+
+    // ---- the cache requests (warp 0)
+    const bool req0 = (need >> e0) & 1ull, req1 = (need >> e1) & 1ull;
     // compute groups: closed form under LRU; under the count policy known only after the misses
     // have been walked, one wave per miss at most
     int n_groups = n_miss ? 1 + (by_count ? n_miss : (n_miss + C - 1) / C) : 1;
@@ -331,8 +387,8 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
     const bool ok = status == MELINOE_OK;
     if (by_count) {
         // Definition C.1: one time step per call, count <- gamma * count + request
-        const float n0 = __fadd_rn(__fmul_rn(p.gamma, cnt0), c0 > 0 ? 1.0f : 0.0f);
-        const float n1 = __fadd_rn(__fmul_rn(p.gamma, cnt1), c1 > 0 ? 1.0f : 0.0f);
+        const float n0 = __fadd_rn(__fmul_rn(p.gamma, cnt0), req0 ? 1.0f : 0.0f);
+        const float n1 = __fadd_rn(__fmul_rn(p.gamma, cnt1), req1 ? 1.0f : 0.0f);
         s_cntf[lane] = n0;
         s_cntf[lane + 32] = n1;
         if (e0 < E)
@@ -350,13 +406,13 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
     __syncwarp();
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
-        const int e = h ? e1 : e0, soe = h ? soe1 : soe0, cnt = h ? c1 : c0, off = h ? off1 : off0;
+        const int e = h ? e1 : e0, soe = h ? soe1 : soe0;
         if ((hit_mask >> e) & 1ull) {
             const int r = rank_below(hit_mask, e);
             const unsigned long long st = counter + (unsigned long long)r + 1ull;
             s_key[soe] = (1ull << 63) | st;
             cache->stamp[soe] = st;
-            plan->req[r] = ReqRec{e, soe, 1, -1, off, cnt, r, 0};
+            write_req(&plan->req[r], e, soe, 1, -1, r, 0);
             s_grp_of[e] = 0;
             plan->dreq[r] = DecReq{p.slots + (size_t)soe * p.slot_stride, nullptr, e, 0, 0, 0};
         }
@@ -436,9 +492,6 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
                     s_grp_first[cur_group] = i;
             }
             __syncwarp();
-            // the expert's token list: offset and count live with the lane that owns the expert
-            const int cnt = __shfl_sync(0xffffffffu, e < 32 ? c0 : c1, e & 31);
-            const int off = __shfl_sync(0xffffffffu, e < 32 ? off0 : off1, e & 31);
             if (lane == 0) {
                 const unsigned long long st = counter + (unsigned long long)(n_hits + i) + 1ull;
                 const int vr_at = n_hits + p.n_shared + i;
@@ -450,7 +503,7 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
                 s_live_occ[slot] = e;
                 s_live_stamp[slot] = st;
                 s_grp_of[e] = cur_group;
-                plan->req[n_hits + i] = ReqRec{e, slot, 0, ev, off, cnt, vr_at, cur_group};
+                write_req(&plan->req[n_hits + i], e, slot, 0, ev, vr_at, cur_group);
                 s_miss_expert[i] = e;
                 s_miss_slot[i] = slot;
                 s_miss_group[i] = cur_group;
@@ -472,7 +525,7 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
     } else
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
-        const int e = h ? e1 : e0, cnt = h ? c1 : c0, off = h ? off1 : off0;
+        const int e = h ? e1 : e0;
         if ((miss_mask >> e) & 1ull) {
             const int i = rank_below(miss_mask, e);
             const int slot = s_victim[i % C];
@@ -485,7 +538,7 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
                 dep = 0;
             ev_flag[h] = ev >= 0;
             const int vr_at = n_hits + p.n_shared + i;
-            plan->req[n_hits + i] = ReqRec{e, slot, 0, ev, off, cnt, vr_at, group};
+            write_req(&plan->req[n_hits + i], e, slot, 0, ev, vr_at, group);
             // cache update: the last miss that lands in a slot keeps it
             const bool stays = i + C >= n_miss;
             {
@@ -507,8 +560,7 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
     const int n_evict = by_count ? n_evict_seq : __popcll(ballot64(ev_flag[0], ev_flag[1]));
     // shared experts: always resident, group 0, behind the hits
     for (int s = lane; s < p.n_shared; s += 32) {
-        const int off = n_pairs + s * T;
-        plan->req[n_req + s] = ReqRec{E + s, -1, 1, -1, off, T, n_hits + s, 0};
+        write_req(&plan->req[n_req + s], E + s, -1, 1, -1, n_hits + s, 0);
         plan->dreq[n_hits + s] = DecReq{p.shared_blobs[s], nullptr, E + s, 0, 0, 0};
     }
     // group boundaries, counts and offsets (what the FFN launches and the inspection calls read)
@@ -520,19 +572,6 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
             b = n_hits + p.n_shared + (done < n_miss ? done : n_miss);
         }
         plan->group_vr_begin[g] = b;
-    }
-    if (e0 < E) {
-        plan->counts[e0] = c0;
-        plan->offsets[e0] = off0;
-    }
-    if (e1 < E) {
-        plan->counts[e1] = c1;
-        plan->offsets[e1] = off1;
-    }
-    if (lane <= p.n_shared) {
-        if (lane < p.n_shared)
-            plan->counts[E + lane] = T;
-        plan->offsets[E + lane] = n_pairs + lane * T;
     }
     if (lane == 0) {
         plan->n_tokens = T;

@@ -83,7 +83,7 @@ class LayerSetup:
                                          base + e * qb)
         self.layer.register_host_experts_q4([base + e * qb for e in range(self.E)], qb, keep=self.store_q4)
 
-    def set_experts_stacked(self, wg: torch.Tensor, wu: torch.Tensor, wd: torch.Tensor, threads: int = 8) -> None:
+    def set_experts_stacked(self, wg: torch.Tensor, wu: torch.Tensor, wd: torch.Tensor, threads: int = 16) -> None:
         """Whole layer at once: wg/wu [E][F][d], wd [E][d][F] bf16 CPU tensors."""
         base = self.store.data_ptr()
         eb = self.expert_bytes
@@ -95,7 +95,7 @@ class LayerSetup:
             list(ex.map(one, range(self.E)))
         self.layer.register_host_experts([base + e * eb for e in range(self.E)], eb, keep=self.store)
 
-    def set_experts_stacked_q4(self, wg: torch.Tensor, wu: torch.Tensor, wd: torch.Tensor, threads: int = 8) -> None:
+    def set_experts_stacked_q4(self, wg: torch.Tensor, wu: torch.Tensor, wd: torch.Tensor, threads: int = 16) -> None:
         """Whole layer at once into a 4-bit pinned store: wg/wu [E][F][d], wd [E][d][F] bf16 CPU tensors."""
         qb = B.melinoe_moe_expert_bytes_q4(self.d, self.F)
         assert qb > 0, "the 4-bit store needs d_ff % 64 == 0"

@@ -4,8 +4,10 @@ way bench.py drives them (one handle per layer, device-resident inputs), against
 Routing indices, gates, request traces and statistics are compared for every call (they are
 cheap to recompute on the CPU); activations are compared on a sample of (layer, token) pairs,
 which is sound because a token's output depends only on its inputs and routing, never on the
-cache state.  The largest shapes run with a reduced number of layers (each layer is an
-independent handle; their full width and call shapes are kept).
+cache state.  The largest shapes run with 4 of their layers (each layer is an independent
+handle with its own weights, router, bias and cache; full width and call shapes are kept) and
+32 of their decode steps; every call's sampled tokens (up to 8 per call, first and last
+included) are compared element by element as well as by norm.
 """
 import numpy as np
 import pytest
@@ -19,7 +21,7 @@ pytestmark = pytest.mark.gpu
 REL_TOL = 2e-2          # the specified bound at full size
 
 
-def _run_stack(name, n_layers, alpha, C, decode_steps, sample_layers, prefill=True, y_tokens=3):
+def _run_stack(name, n_layers, alpha, C, decode_steps, sample_layers, prefill=True, y_tokens=8):
     import torch
     from paper_2602_11192_b200.workload import Stack, bits_of, stats_rows
     cfg = gen.config_by_name(name)
@@ -81,25 +83,31 @@ def test_olmoe_full_stack_as_benchmarked():
     _run_stack("olmoe", None, 0.1, 16, decode_steps=12, sample_layers=(0, 7, 15))
 
 
-def test_olmoe_near_uniform_routing_thrashes_the_cache():
-    _run_stack("olmoe", 2, 10.0, 16, decode_steps=6, sample_layers=(1,))
+@pytest.mark.parametrize("alpha", [1.0, 10.0])
+def test_olmoe_other_routing_concentrations(alpha):
+    """configs[1], alpha = 1 and 10 (near-uniform routing thrashes the cache): 4 of the 16 layers, the
+    prompt and 32 decode steps."""
+    _run_stack("olmoe", 4, alpha, 16, decode_steps=32, sample_layers=(0, 3))
 
 
-def test_mixtral_shape_two_slots():
-    """configs[2]: d 4096, d_ff 14336, 8 experts, top-2, 2 slots; one layer of the 32."""
-    _run_stack("mixtral", 1, 0.2, 2, decode_steps=4, sample_layers=(0,), y_tokens=2)
+@pytest.mark.parametrize("C,alpha", [(2, 0.2), (2, 2.0), (4, 0.2), (4, 2.0)])
+def test_mixtral_shape(C, alpha):
+    """configs[2]: d 4096, d_ff 14336, 8 experts, top-2, 2 and 4 slots, alpha 0.2 and 2.0; 4 of the 32
+    layers, the 256-token prompt and 32 decode steps."""
+    _run_stack("mixtral", 4, alpha, C, decode_steps=32, sample_layers=(1,), y_tokens=8)
 
 
 def test_phi35_shape_batch_of_eight():
     """configs[3]: d 4096, d_ff 6400, 16 experts, top-2, 6 slots, 8 sequences: 4096-token prefill
-    through the grouped GEMM, then decode steps of 8 tokens; one layer of the 32."""
-    _run_stack("phi35", 1, 0.3, 6, decode_steps=3, sample_layers=(0,), y_tokens=3)
+    through the grouped GEMM, then 32 decode steps of 8 tokens; 4 of the 32 layers."""
+    _run_stack("phi35", 4, 0.3, 6, decode_steps=32, sample_layers=(2,), y_tokens=8)
 
 
-def test_deepseek_shape_with_shared_experts():
+@pytest.mark.parametrize("alpha", [0.1, 1.0])
+def test_deepseek_shape_with_shared_experts(alpha):
     """configs[4]: d 2048, d_ff 1408, 64 routed + 2 shared experts, top-6, 12 slots, 4 sequences:
-    8192-token prefill, then decode steps of 4 tokens; one layer of the 28."""
-    _run_stack("deepseek", 1, 0.1, 12, decode_steps=3, sample_layers=(0,), y_tokens=3)
+    8192-token prefill, then 32 decode steps of 4 tokens; 4 of the 28 layers."""
+    _run_stack("deepseek", 4, alpha, 12, decode_steps=32, sample_layers=(3,), y_tokens=8)
 
 
 def test_repeated_runs_with_heavy_miss_traffic_are_bit_identical():

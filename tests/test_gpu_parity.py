@@ -164,6 +164,63 @@ def test_prefill_grouped_gemm(d, F, E, k, C, n_shared, Ts):
     P.close()
 
 
+def test_prefill_router_breaks_ties_towards_the_lowest_expert_id():
+    """More than 8 tokens go through the general router kernel: with a zero router matrix the logits are
+    the bias alone, and a bias with equal entries makes ties that must go to the lowest ids (Eq. 1 with
+    the tie rule of the oracle's strict-greater arg-max); all-equal logits select experts 0 .. k-1."""
+    d, F, E, k, C = 512, 64, 12, 3, 6
+    P = _pair(d, F, E, k, C, seed=81)
+    P.w_r = np.zeros_like(P.w_r)
+    P.gpu.set_router(P.w_r)
+    bias = np.zeros((3, E), np.float32)
+    bias[0, [2, 5, 7, 9, 11]] = 1.0            # five tied winners: 2, 5, 7 are taken
+    bias[1, :] = 0.25                          # everything equal: 0, 1, 2
+    bias[2, [10, 4]] = 3.0                     # two clear winners, then the lowest of the tied rest: 4, 10, 0
+    for T in (20, 9, 33):
+        seq = (np.arange(T) % 3).astype(np.int32)
+        P.set_bias(bias, seq)
+        _, o = P.step(gen.hidden_states(81, 0, "prefill", T, T, d), tokens=[0, 1, 2, T - 1])
+        for t in range(T):
+            want = {0: [2, 5, 7], 1: [0, 1, 2], 2: [4, 10, 0]}[int(seq[t])]
+            assert o["idx"][t].tolist() == want
+    # the same ties through the decode router (at most 8 tokens)
+    P.set_bias(bias, np.arange(3, dtype=np.int32))
+    _, o = P.step(gen.hidden_states(81, 0, "decode", 0, 3, d))
+    assert o["idx"].tolist() == [[2, 5, 7], [0, 1, 2], [4, 10, 0]]
+    P.close()
+
+
+def test_a_failed_host_copy_leaves_the_handle_usable():
+    """Error path of a partly queued call.  The failure is made on the host: a hook makes the first
+    host-issued expert copy of the call report an error instead of being issued (nothing faults or
+    waits on the device).  The call returns the error, later calls return it too until the cache is
+    reset, the stream can be synchronised, and after the reset the layer works again."""
+    import torch
+    from paper_2602_11192_b200 import MelinoeError, lib
+    from paper_2602_11192_b200.runner import current_stream_ptr, to_dev_bf16
+    d, F, E, k, C = 512, 128, 8, 2, 4
+    P = _pair(d, F, E, k, C, seed=83)
+    T = 40                                              # grouped-GEMM path: the host issues the copies
+    x = gen.hidden_states(83, 0, "prefill", 0, T, d)
+    xd = to_dev_bf16(x)
+    out = torch.zeros((T, d), dtype=torch.int16, device="cuda")
+    lib().melinoe_debug_fail_host_copy(1)
+    with pytest.raises(MelinoeError) as ei:
+        P.gpu.layer.forward(current_stream_ptr(), xd, T, out)
+    assert ei.value.status == 3
+    lib().melinoe_debug_fail_host_copy(0)
+    torch.cuda.synchronize()                            # whatever was queued runs to its end
+    with pytest.raises(MelinoeError) as ei:
+        P.gpu.layer.forward(current_stream_ptr(), xd, T, out)
+    assert ei.value.status == 3                         # sticky
+    with pytest.raises(MelinoeError):
+        P.gpu.layer.cache_state()
+    P.reset()                                           # clears the error; both sides start cold again
+    P.step(x, tokens=[0, 7, T - 1])
+    P.step(gen.hidden_states(83, 0, "decode", 0, 2, d))
+    P.close()
+
+
 def test_forward_host_matches_forward_and_is_deterministic():
     import torch
     from paper_2602_11192_b200.runner import current_stream_ptr
