@@ -26,10 +26,10 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one ffn_stream_kernel launch divided by the launch's
-# algorithmic bytes (8 experts x 12.58 MB), from the ncu capture summarised in
-# profiles/ffn_stream_kernel_olmoe_decode.md; traffic grows in proportion to the experts streamed.
-DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.03
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the decode FFN kernel divided by the launch's
+# algorithmic bytes (8 experts x 12.58 MB), from an ncu capture of a two-layer case of this workload; traffic
+# grows in proportion to the experts streamed.  None until the counters have been taken for the current kernel.
+DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE = None
 
 METRIC = "decode tokens/s (OLMoE-shaped, cache-limited)"
 UNIT = "tokens/s"
@@ -148,6 +148,237 @@ def job_throughput(tokens_per_rank: int, world: int, ms: float) -> float:
 
 # --------------------------------------------------------------------------- our arm
 
+REPEATS = 5          # every timed region is measured this many times: median and best are reported
+
+
+class Runner:
+    """One synthetic stack plus its decode inputs: prepares (cold start, prompt, warm-up) and times regions."""
+
+    def __init__(self, torch, M, gen, cfg, alpha, C, L, K, W, store="bf16", dist=None):
+        from paper_2602_11192_b200.workload import Stack
+        self.torch, self.M, self.gen, self.cfg, self.dist = torch, M, gen, cfg, dist
+        self.L, self.K, self.W = L, K, W
+        self.stack = Stack(cfg, alpha, C, n_layers=L, store=store)
+        d = cfg.d_model
+        n_steps = W + K
+        dec = np.stack([self.stack.hidden_bits("decode", s) for s in range(n_steps)])          # [S][L][B][d]
+        self.dec_host = torch.from_numpy(dec.view(np.int16)).pin_memory()
+        self.dec_dev = self.dec_host.cuda()
+        self.pre_dev = None
+        if cfg.prefill_tokens:
+            self.pre_dev = torch.from_numpy(self.stack.hidden_bits("prefill", 0).view(np.int16)).cuda()
+            self.pre_out = torch.empty_like(self.pre_dev)
+        self.out_dev = torch.empty((L, cfg.batch, d), dtype=torch.int16, device="cuda")
+        self.out_host = torch.empty((L, cfg.batch, d), dtype=torch.int16).pin_memory()
+        self.stats_dev = torch.zeros((n_steps, L, 12), dtype=torch.int32, device="cuda")
+        self.stats_host = torch.zeros((L, 12), dtype=torch.int32).pin_memory()
+
+    def barrier(self):
+        if self.dist is not None:
+            self.dist.barrier()
+
+    def prepare(self, alpha, timing_prefill=False):
+        """Cold start, prompt, then the warm-up decode steps are left to the caller."""
+        st, cfg, gen = self.stack, self.cfg, self.gen
+        if alpha != st.alpha:
+            st.alpha = alpha
+            st.bias = [np.stack([gen.router_bias(cfg.seed, l, s, alpha, cfg.n_experts) for s in range(cfg.batch)])
+                       for l in range(self.L)]
+        st.reset()
+        if self.pre_dev is not None:
+            st.set_phase("prefill")
+            if timing_prefill:
+                for ls in st.layers:
+                    ls.layer.enable_timing(True)
+            st.forward_all(self.pre_dev, self.pre_out, None)
+        st.set_phase("decode")
+        self.torch.cuda.synchronize()
+
+    def timed_device(self, alpha, with_kernel_timing=False):
+        """W warm-up steps, then K timed steps with device-resident inputs.  Returns ms, launches, the
+        timed steps' statistics and, with kernel timing, the per-launch FFN times (ms) in call order."""
+        torch, M, st, W, K = self.torch, self.M, self.stack, self.W, self.K
+        self.prepare(alpha)
+        self.stats_dev.zero_()
+        for s in range(W):
+            st.forward_all(self.dec_dev[s], self.out_dev, self.stats_dev[s])
+        torch.cuda.synchronize()
+        if with_kernel_timing:
+            for ls in st.layers:
+                ls.layer.enable_timing(True)
+        self.barrier()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n0 = M.melinoe_launch_count()
+        e0.record()
+        for s in range(W, W + K):
+            st.forward_all(self.dec_dev[s], self.out_dev, self.stats_dev[s])
+        e1.record()
+        torch.cuda.synchronize()
+        self.barrier()
+        ms = e0.elapsed_time(e1)
+        launches = M.melinoe_launch_count() - n0
+        per_launch = None
+        if with_kernel_timing:
+            per_launch = []                                   # [layer] -> times of its K calls' launches
+            for ls in st.layers:
+                per_launch.append(ls.layer.ffn_launch_times_ms())
+                ls.layer.ffn_time_ms()
+                ls.layer.transfer_time_ms()
+                ls.layer.enable_timing(False)
+        stats = stats_arrays(self.stats_dev[W:W + K])
+        if int(stats["status"].max()) != 0:
+            raise SystemExit("device-side status %d in the timed region" % int(stats["status"].max()))
+        return ms, launches, stats, per_launch
+
+    def timed_e2e(self, alpha):
+        """The same steps through the host-buffer entry point, one stream synchronisation per step."""
+        torch, st, W, K = self.torch, self.stack, self.W, self.K
+        self.prepare(alpha)
+        s_ptr = torch.cuda.current_stream()
+        for s in range(W):
+            st.forward_all_host(self.dec_host[s], self.out_host, self.stats_host)
+            s_ptr.synchronize()
+        self.barrier()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for s in range(W, W + K):
+            st.forward_all_host(self.dec_host[s], self.out_host, self.stats_host)
+            s_ptr.synchronize()
+        e1.record()
+        torch.cuda.synchronize()
+        self.barrier()
+        return e0.elapsed_time(e1)
+
+    def close(self):
+        self.stack.close()
+
+
+def stats_arrays(stats_dev):
+    """[K][L][12] int32 statistics -> dict of [K][L] arrays."""
+    s = stats_dev.cpu().numpy()
+    return {"status": s[..., 0], "n_tokens": s[..., 1], "n_distinct": s[..., 2], "hits": s[..., 3], "misses": s[..., 4],
+            "evictions": s[..., 5], "groups": s[..., 6]}
+
+
+def med_best(vals, higher_is_better=True):
+    v = sorted(vals)
+    return statistics.median(v), (v[-1] if higher_is_better else v[0])
+
+
+def hit_summary(cfg, stats, K, L):
+    h, m = int(stats["hits"].sum()), int(stats["misses"].sum())
+    return {"hit_rate": h / max(h + m, 1), "misses_per_layer_per_token": m / (K * L * cfg.batch),
+            "h2d_expert_bytes_per_step": m * cfg.expert_bytes / K}
+
+
+def ffn_launch_analysis(cfg, stats, per_launch, hbm_peak, link_peak):
+    """Per-launch CUDA-event times of the decode FFN kernel against what each launch moved.
+    One launch per call here (the kernel fetches missed experts itself), so launch i of layer l is call i.
+    Launches whose experts were all resident are bound by HBM: bytes = experts x bytes per expert.  Launches
+    that fetched experts are bound by the host link for those: bytes over the link / launch time."""
+    B_e = cfg.expert_bytes
+    res_bytes = res_ms = 0.0
+    res_n = 0
+    miss_bytes = miss_ms = 0.0
+    miss_n = 0
+    all_bytes = all_ms = 0.0
+    K, L = stats["misses"].shape
+    for l in range(L):
+        t = per_launch[l]
+        if len(t) != K:
+            return None                     # not one launch per call (host-issued transfers): no per-call attribution
+        for i in range(K):
+            experts = int(stats["n_distinct"][i, l]) + cfg.n_shared
+            m = int(stats["misses"][i, l])
+            all_bytes += experts * B_e
+            all_ms += float(t[i])
+            if m == 0:
+                res_bytes += experts * B_e
+                res_ms += float(t[i])
+                res_n += 1
+            else:
+                miss_bytes += m * B_e
+                miss_ms += float(t[i])
+                miss_n += 1
+    out = {"resident": None, "fetching": None, "all": None}
+    if res_n:
+        g = res_bytes / (res_ms * 1e-3) / 1e9
+        out["resident"] = {"launches": res_n, "avg_launch_us": 1e3 * res_ms / res_n, "bytes_per_launch": res_bytes / res_n,
+                           "gbs": g, "frac_of_hbm": g / hbm_peak}
+    if miss_n:
+        g = miss_bytes / (miss_ms * 1e-3) / 1e9
+        out["fetching"] = {"launches": miss_n, "avg_launch_us": 1e3 * miss_ms / miss_n, "link_bytes_per_launch": miss_bytes / miss_n,
+                           "link_gbs": g, "frac_of_link": g / link_peak if link_peak else None}
+    g = all_bytes / (all_ms * 1e-3) / 1e9
+    out["all"] = {"launches": res_n + miss_n, "avg_launch_us": 1e3 * all_ms / max(res_n + miss_n, 1), "gbs": g,
+                  "frac_of_hbm": g / hbm_peak}
+    return out
+
+
+def host_link_gbs(torch):
+    """Pinned host -> device copy of 512 MiB on a side stream: the link's own rate."""
+    n = 512 << 20
+    hb = torch.empty(n, dtype=torch.uint8).pin_memory()
+    db = torch.empty(n, dtype=torch.uint8, device="cuda")
+    st_ = torch.cuda.Stream()
+    best = 0.0
+    with torch.cuda.stream(st_):
+        for _ in range(4):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(st_)
+            db.copy_(hb, non_blocking=True)
+            b.record(st_)
+            st_.synchronize()
+            best = max(best, n / (a.elapsed_time(b) * 1e-3) / 1e9)
+    del hb, db
+    return best
+
+
+def shape_record(torch, M, gen, name, n_layers, K, W, hbm_peak, link_peak, peaks):
+    """Decode throughput, FFN roofline and (where the prompt runs the grouped GEMM) the prefill GEMM's
+    rate of one of the other workload shapes, at its full width with a reduced number of layers."""
+    cfg = gen.config_by_name(name)
+    C, alpha = cfg.cache_slots[0], cfg.alphas[0]
+    R = Runner(torch, M, gen, cfg, alpha, C, n_layers, K, W)
+    rec = {"workload": "%s-shaped: d_model=%d, d_ff=%d, %d experts (+%d shared), top-%d, cache %d/layer, batch %d, "
+                       "%d-token prompts, alpha=%g" % (name, cfg.d_model, cfg.d_ff, cfg.n_experts, cfg.n_shared, cfg.top_k, C,
+                                                       cfg.batch, cfg.prefill_tokens, alpha),
+           "layers": n_layers, "reduced_layers": n_layers != cfg.n_layers, "decode_steps": K}
+    vals = []
+    for _ in range(3):
+        ms, _, st, _ = R.timed_device(alpha)
+        vals.append(cfg.batch * K / (ms * 1e-3))
+    rec["tokens_per_s_median"], rec["tokens_per_s_best"] = med_best(vals)
+    rec.update(hit_summary(cfg, st, K, n_layers))
+    _, _, st2, per_launch = R.timed_device(alpha, with_kernel_timing=True)
+    rec["ffn"] = ffn_launch_analysis(cfg, st2, per_launch, hbm_peak, link_peak)
+    # the prompt again with events around the grouped GEMM launches of every compute group
+    if cfg.prefill_tokens and cfg.d_ff % 128 == 0 and cfg.batch * cfg.prefill_tokens > 8:
+        R.prepare(alpha, timing_prefill=True)
+        ms_sum, n = 0.0, 0
+        for ls in R.stack.layers:
+            t = ls.layer.ffn_launch_times_ms()
+            ms_sum += float(t.sum())
+            n += len(t)
+            ls.layer.ffn_time_ms()
+            ls.layer.transfer_time_ms()
+            ls.layer.enable_timing(False)
+        T = cfg.batch * cfg.prefill_tokens
+        pairs = T * (cfg.top_k + cfg.n_shared)
+        flops = 6.0 * cfg.d_model * cfg.d_ff * pairs * n_layers
+        tf = flops / (ms_sum * 1e-3) / 1e12
+        rec["prefill_gemm"] = {"tokens": T, "token_expert_pairs_per_layer": pairs, "tflops": tf,
+                               "frac_of_bf16_burst": tf / peaks.get("bf16_tflops", 1590.0),
+                               "frac_of_bf16_sustained": tf / peaks.get("bf16_tflops_sustained", 1400.0),
+                               "gemm_launch_pairs": n, "gemm_ms_per_layer": ms_sum / n_layers,
+                               "note": "flops = 6 d_model d_ff per (token, expert) pair; time = CUDA events around the two "
+                                       "GEMM launches of every compute group, transfers excluded"}
+    R.close()
+    return rec
+
+
 def run_ours(args):
     import torch
     import gen
@@ -162,16 +393,12 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
-    def barrier():
-        if dist is not None:
-            dist.barrier()
-
     from paper_2602_11192_b200 import build as _build
     if rank == 0:
         _build.build()
-    barrier()
+    if dist is not None:
+        dist.barrier()
     import paper_2602_11192_b200 as M
-    from paper_2602_11192_b200.workload import Stack, stats_rows
 
     cfg = gen.config_by_name(WORKLOAD)
     C = cfg.cache_slots[0]
@@ -180,91 +407,16 @@ def run_ours(args):
     K, W = args.steps, args.warmup
     d = cfg.d_model
     B_e = cfg.expert_bytes
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except Exception:
+        pass
+    hbm_peak = float(peaks.get("hbm_gbs", 6650.0))
+    peak_src = "measured" if "hbm_gbs" in peaks else "fallback"
 
     phase("building the stack: %d layers x %d experts x %.1f MB in pinned host memory" % (L, cfg.n_experts, B_e / 1e6))
-    stack = Stack(cfg, alpha0, C, n_layers=L)
-    n_steps = W + K
-    # decode inputs for every step, on the device and in pinned host memory
-    dec = np.stack([stack.hidden_bits("decode", s) for s in range(n_steps)])          # [S][L][B][d]
-    dec_host = torch.from_numpy(dec.view(np.int16)).pin_memory()
-    dec_dev = dec_host.cuda()
-    pre_dev = None
-    if cfg.prefill_tokens:
-        pre_dev = torch.from_numpy(stack.hidden_bits("prefill", 0).view(np.int16)).cuda()
-        pre_out = torch.empty_like(pre_dev)
-    out_dev = torch.empty((L, cfg.batch, d), dtype=torch.int16, device="cuda")
-    out_host = torch.empty((L, cfg.batch, d), dtype=torch.int16).pin_memory()
-    stats_dev = torch.zeros((n_steps, L, 12), dtype=torch.int32, device="cuda")
-    stats_host = torch.zeros((L, 12), dtype=torch.int32).pin_memory()
-
-    def prepare(alpha):
-        """Cold start, prompt, then the warm-up decode steps."""
-        if alpha != stack.alpha:
-            stack.alpha = alpha
-            stack.bias = [np.stack([gen.router_bias(cfg.seed, l, s, alpha, cfg.n_experts) for s in range(cfg.batch)])
-                          for l in range(L)]
-        stack.reset()
-        if pre_dev is not None:
-            stack.set_phase("prefill")
-            stack.forward_all(pre_dev, pre_out, None)
-        stack.set_phase("decode")
-        torch.cuda.synchronize()
-
-    copy_acc = [0.0, 0.0]   # copy-stream ms and bytes of the most recent run with kernel timing
-
-    def host_link_gbs():
-        """Pinned host -> device copy of 512 MiB on a side stream: the link's own rate."""
-        n = 512 << 20
-        hb = torch.empty(n, dtype=torch.uint8).pin_memory()
-        db = torch.empty(n, dtype=torch.uint8, device="cuda")
-        st_ = torch.cuda.Stream()
-        best = 0.0
-        with torch.cuda.stream(st_):
-            for _ in range(4):
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record(st_)
-                db.copy_(hb, non_blocking=True)
-                b.record(st_)
-                st_.synchronize()
-                best = max(best, n / (a.elapsed_time(b) * 1e-3) / 1e9)
-        return best
-
-    def timed_device(alpha, with_kernel_timing=False):
-        prepare(alpha)
-        stats_dev.zero_()
-        for s in range(W):
-            stack.forward_all(dec_dev[s], out_dev, stats_dev[s])
-        torch.cuda.synchronize()
-        if with_kernel_timing:
-            for ls in stack.layers:
-                ls.layer.enable_timing(True)
-        barrier()
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        n0 = M.melinoe_launch_count()
-        e0.record()
-        for s in range(W, W + K):
-            stack.forward_all(dec_dev[s], out_dev, stats_dev[s])
-        e1.record()
-        torch.cuda.synchronize()
-        barrier()
-        ms = e0.elapsed_time(e1)
-        launches = M.melinoe_launch_count() - n0
-        ffn_ms, ffn_n = 0.0, 0
-        copy_acc[0] = copy_acc[1] = 0.0
-        if with_kernel_timing:
-            for ls in stack.layers:
-                a, b = ls.layer.ffn_time_ms()
-                ffn_ms += a
-                ffn_n += b
-                cm, cb = ls.layer.transfer_time_ms()
-                copy_acc[0] += cm
-                copy_acc[1] += cb
-                ls.layer.enable_timing(False)
-        st = stats_rows(stats_dev[W:W + K])
-        if int(st["status"].max()) != 0:
-            raise SystemExit("device-side status %d in the timed region" % int(st["status"].max()))
-        return ms, launches, st, ffn_ms, ffn_n
+    R = Runner(torch, M, gen, cfg, alpha0, C, L, K, W, dist=dist)
 
     gpu_index = local
     vis = os.environ.get("CUDA_VISIBLE_DEVICES")
@@ -276,68 +428,50 @@ def run_ours(args):
     sampler = ClockSampler(gpu_index)
     if rank == 0:
         sampler.start()
-    phase("timed region: %d warm-up + %d decode steps, device-resident inputs" % (W, K))
-    ms, launches, st, _, _ = timed_device(alpha0)
+    phase("timed region x %d: %d warm-up + %d decode steps each, device-resident inputs" % (REPEATS, W, K))
+    runs = []
+    for _ in range(REPEATS):
+        ms, launches, st, _ = R.timed_device(alpha0)
+        runs.append(max_over_ranks(ms, dist, "cuda"))
     clocks = sampler.stop() if rank == 0 else None
-    ms = max_over_ranks(ms, dist, "cuda")
+    ms = statistics.median(runs)
     tokens = cfg.batch * K * world
     value = job_throughput(cfg.batch * K, world, ms)
+    repeats = {"n": REPEATS, "tokens_per_s": [job_throughput(cfg.batch * K, world, m) for m in runs],
+               "median": value, "best": job_throughput(cfg.batch * K, world, min(runs))}
 
     # ---- end to end: host buffers in, host buffers out, one synchronisation per decode step
-    phase("end-to-end region: host buffers, %.1f ms/step on the device path" % (ms / K))
-    prepare(alpha0)
-    s_ptr = torch.cuda.current_stream()
-    for s in range(W):
-        stack.forward_all_host(dec_host[s], out_host, stats_host)
-        s_ptr.synchronize()
-    barrier()
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for s in range(W, W + K):
-        stack.forward_all_host(dec_host[s], out_host, stats_host)
-        s_ptr.synchronize()
-    e1.record()
-    torch.cuda.synchronize()
-    barrier()
-    e2e_ms = max_over_ranks(e0.elapsed_time(e1), dist, "cuda")
-    e2e = {"value": tokens / (e2e_ms * 1e-3), "unit": UNIT,
+    phase("end-to-end region x %d: host buffers, %.2f ms/step on the device path" % (REPEATS, ms / K))
+    e2e_runs = [max_over_ranks(R.timed_e2e(alpha0), dist, "cuda") for _ in range(REPEATS)]
+    e2e_ms = statistics.median(e2e_runs)
+    e2e = {"value": tokens / (e2e_ms * 1e-3), "unit": UNIT, "best": tokens / (min(e2e_runs) * 1e-3),
            "h2d_bytes_per_step": L * cfg.batch * d * 2,
            "d2h_bytes_per_step": L * (cfg.batch * d * 2 + 48),
            "note": "inputs from pinned host memory and outputs + statistics back to it inside the timed region, "
-                   "one stream synchronisation per decode step; expert miss traffic (counted in hit_stats) is extra"}
+                   "one stream synchronisation per decode step; expert miss traffic (counted in hit_stats) is extra; "
+                   "median of %d runs" % REPEATS}
 
-    # ---- roofline of the dominant kernel (streaming expert FFN): same region again with per-launch events
-    peaks = {}
-    try:
-        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
-    except Exception:
-        pass
-    hbm_peak = float(peaks.get("hbm_gbs", 6650.0))
-    peak_src = "measured" if "hbm_gbs" in peaks else "fallback"
+    # ---- roofline of the dominant kernel (decode expert FFN): same region again with per-launch events
     phase("same region with per-launch events around the FFN kernel")
-    _, _, st2, ffn_ms, ffn_n = timed_device(alpha0, with_kernel_timing=True)
-    ffn_bytes = float((st2["n_distinct"].astype(np.int64) + cfg.n_shared).sum()) * B_e
-    achieved = ffn_bytes / (ffn_ms * 1e-3) / 1e9 if ffn_ms > 0 else 0.0
-    link_peak = host_link_gbs()
-    miss_path = {"achieved_gbs": (copy_acc[1] / (copy_acc[0] * 1e-3) / 1e9) if copy_acc[0] > 0 else None,
-                 "peak_gbs": link_peak, "bytes": copy_acc[1], "copy_stream_ms": copy_acc[0],
-                 "note": "expert bytes moved by cudaMemcpyAsync from pinned host memory / time between events on the "
-                         "copy stream around each wave of transfers; peak = a 512 MiB pinned copy measured in this run"}
-    if miss_path["achieved_gbs"]:
-        miss_path["frac"] = miss_path["achieved_gbs"] / link_peak
-    roofline = {"bound": "hbm", "kernel": "ffn_stream_kernel", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
-                "frac": achieved / hbm_peak, "peak_source": peak_src,
-                "traffic": DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE * ffn_bytes / max(ffn_n, 1),
-                "launches": int(ffn_n), "avg_launch_us": 1e3 * ffn_ms / max(ffn_n, 1),
-                "bytes_per_launch": ffn_bytes / max(ffn_n, 1),
-                "note": "bytes = experts streamed x bytes per expert; launches that found no missed expert to "
-                        "compute are included in the time"}
-
-    def hit_summary(s):
-        h, m = int(s["hits"].sum()), int(s["misses"].sum())
-        return {"hit_rate": h / max(h + m, 1), "misses_per_layer_per_token": m / (K * L * cfg.batch),
-                "h2d_expert_bytes_per_step": m * B_e / K}
+    link_peak = host_link_gbs(torch)
+    _, _, st2, per_launch = R.timed_device(alpha0, with_kernel_timing=True)
+    ana = ffn_launch_analysis(cfg, st2, per_launch, hbm_peak, link_peak)
+    res = ana["resident"] if ana and ana["resident"] else {"gbs": 0.0, "launches": 0, "avg_launch_us": None, "bytes_per_launch": 0.0}
+    roofline = {"bound": "hbm", "kernel": "ffn_decode_kernel", "achieved": res["gbs"], "peak": hbm_peak, "unit": "GB/s",
+                "frac": res["gbs"] / hbm_peak, "peak_source": peak_src,
+                "traffic": (DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE * res["bytes_per_launch"]) if DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE else None,
+                "launches": res["launches"], "avg_launch_us": res["avg_launch_us"], "bytes_per_launch": res["bytes_per_launch"],
+                "all_launches": ana["all"] if ana else None,
+                "note": "launches whose experts were all resident (HBM-bound): bytes = experts streamed x bytes per expert, "
+                        "time = CUDA events around each launch; the launches that also fetched experts over the host link "
+                        "are in miss_path, all launches together in all_launches"}
+    fe = ana["fetching"] if ana else None
+    miss_path = {"achieved_gbs": fe["link_gbs"] if fe else None, "peak_gbs": link_peak,
+                 "frac": fe["frac_of_link"] if fe else None, "launches": fe["launches"] if fe else 0,
+                 "avg_launch_us": fe["avg_launch_us"] if fe else None,
+                 "note": "launches of the FFN kernel that read missed experts from pinned host memory themselves: expert "
+                         "bytes over the link / whole launch time by CUDA events (the resident experts' compute runs on "
+                         "other SMs meanwhile); peak = a 512 MiB pinned cudaMemcpyAsync measured in this run"}
 
     extra = {}
     if not args.no_extra and rank == 0 and world == 1:
@@ -345,54 +479,61 @@ def run_ours(args):
             if a == alpha0:
                 continue
             phase("alpha=%g" % a)
-            ms_a, _, st_a, _, _ = timed_device(a)
-            extra["alpha=%g" % a] = dict(value=cfg.batch * K / (ms_a * 1e-3), **hit_summary(st_a))
+            ms_a, _, st_a, _ = R.timed_device(a)
+            extra["alpha=%g" % a] = dict(value=cfg.batch * K / (ms_a * 1e-3), **hit_summary(cfg, st_a, K, L))
         # the paper's other eviction policies on the same stream (its Table 13 compares transfers under
-        # LRU and LFU): Definition C.1's discounted count, gamma = 1 (LFU) and gamma = 0.9.  These runs
-        # plan with the general kernels, so their tokens/s also carries that difference.
+        # LRU and LFU): Definition C.1's discounted count, gamma = 1 (LFU) and gamma = 0.9
         for name, g in (("policy=lfu", 1.0), ("policy=count,gamma=0.9", 0.9)):
             phase(name)
-            stack.set_policy("count", g)
-            ms_p, _, st_p, _, _ = timed_device(alpha0)
-            extra[name] = dict(value=cfg.batch * K / (ms_p * 1e-3), **hit_summary(st_p))
-        stack.set_policy("lru")
-        # 4-bit host store (the paper keeps its experts in 4-bit form): a miss moves 3.76 times fewer
-        # bytes; slots and compute stay bf16, computing with the dequantised weights
+            R.stack.set_policy("count", g)
+            ms_p, _, st_p, _ = R.timed_device(alpha0)
+            extra[name] = dict(value=cfg.batch * K / (ms_p * 1e-3), **hit_summary(cfg, st_p, K, L))
+        R.stack.set_policy("lru")
+        R.close()
+        # 4-bit host store (the paper keeps its experts in 4-bit form): a miss moves 3.76 times fewer bytes
         if cfg.d_ff % 64 == 0:
-            stack.close()
-            stack = Stack(cfg, alpha0, C, n_layers=L, store="q4")
+            Rq = Runner(torch, M, gen, cfg, alpha0, C, L, K, W, store="q4")
+            qb = M.melinoe_moe_expert_bytes_q4(cfg.d_model, cfg.d_ff)
             for a in cfg.alphas[:2]:
                 phase("4-bit host store, alpha=%g" % a)
-                ms_q, _, st_q, _, _ = timed_device(a)
-                extra["store=q4,alpha=%g" % a] = dict(value=cfg.batch * K / (ms_q * 1e-3), **hit_summary(st_q))
-                extra["store=q4,alpha=%g" % a]["h2d_expert_bytes_per_step"] = (
-                    float(st_q["misses"].sum()) * M.melinoe_moe_expert_bytes_q4(cfg.d_model, cfg.d_ff) / K)
+                ms_q, _, st_q, _ = Rq.timed_device(a)
+                extra["store=q4,alpha=%g" % a] = dict(value=cfg.batch * K / (ms_q * 1e-3), **hit_summary(cfg, st_q, K, L))
+                extra["store=q4,alpha=%g" % a]["h2d_expert_bytes_per_step"] = float(st_q["misses"].sum()) * qb / K
             # the paper's own serving configuration: 4-bit experts and an LFU cache
             phase("4-bit host store with the LFU policy")
-            stack.set_policy("count", 1.0)
-            ms_q, _, st_q, _, _ = timed_device(alpha0)
-            extra["store=q4,policy=lfu"] = dict(value=cfg.batch * K / (ms_q * 1e-3), **hit_summary(st_q))
-            extra["store=q4,policy=lfu"]["h2d_expert_bytes_per_step"] = (
-                float(st_q["misses"].sum()) * M.melinoe_moe_expert_bytes_q4(cfg.d_model, cfg.d_ff) / K)
-            stack.set_policy("lru")
-        # everything resident (cache = all experts, warm): the FFN kernel without the miss path
+            Rq.stack.set_policy("count", 1.0)
+            ms_q, _, st_q, _ = Rq.timed_device(alpha0)
+            extra["store=q4,policy=lfu"] = dict(value=cfg.batch * K / (ms_q * 1e-3), **hit_summary(cfg, st_q, K, L))
+            extra["store=q4,policy=lfu"]["h2d_expert_bytes_per_step"] = float(st_q["misses"].sum()) * qb / K
+            Rq.close()
+        # everything resident (cache = all experts, warm): the hit path alone
         phase("all experts resident")
-        stack.close()
-        full = Stack(cfg, alpha0, cfg.n_experts, n_layers=L)
-        stack = full
-        ms_r, _, _, _, _ = timed_device(alpha0)                    # throughput: no per-launch events
-        _, _, st_r, ffn_ms_r, ffn_n_r = timed_device(alpha0, with_kernel_timing=True)
-        by_r = float(st_r["n_distinct"].astype(np.int64).sum()) * B_e
-        extra["all_resident"] = {"value": cfg.batch * K / (ms_r * 1e-3), "ffn_gbs": by_r / (ffn_ms_r * 1e-3) / 1e9,
-                                 "ffn_frac_of_hbm": by_r / (ffn_ms_r * 1e-3) / 1e9 / hbm_peak,
-                                 "ffn_launches": int(ffn_n_r), **hit_summary(st_r)}
+        Rf = Runner(torch, M, gen, cfg, alpha0, cfg.n_experts, L, K, W)
+        vals = []
+        for _ in range(REPEATS):
+            ms_r, _, st_r, _ = Rf.timed_device(alpha0)
+            vals.append(cfg.batch * K / (ms_r * 1e-3))
+        _, _, st_r2, pl_r = Rf.timed_device(alpha0, with_kernel_timing=True)
+        ana_r = ffn_launch_analysis(cfg, st_r2, pl_r, hbm_peak, link_peak)
+        rr = ana_r["resident"] if ana_r and ana_r["resident"] else {"gbs": 0.0, "frac_of_hbm": 0.0, "launches": 0, "avg_launch_us": None}
+        med, best = med_best(vals)
+        extra["all_resident"] = {"value": med, "best": best, "ffn_gbs": rr["gbs"], "ffn_frac_of_hbm": rr["frac_of_hbm"],
+                                 "ffn_launches": rr["launches"], "ffn_avg_launch_us": rr["avg_launch_us"],
+                                 "us_per_layer": 1e6 / (med * L) * cfg.batch, **hit_summary(cfg, st_r, K, L)}
+        Rf.close()
+        # the other workload shapes at full width, fewer layers
+        Ks = min(K, 64)
+        for name, nl in (("mixtral", 2), ("phi35", 2), ("deepseek", 2)):
+            phase("%s-shaped stack, %d layers" % (name, nl))
+            extra["shape=" + name] = shape_record(torch, M, gen, name, nl, Ks, W, hbm_peak, link_peak, peaks)
+    else:
+        R.close()
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         phase("CPU oracle on a sample of the same steps")
         cpu_baseline = cpu_oracle_sample(cfg, alpha0, C, L, W, K, budget_s=15.0)
 
-    stack.close()
     faulthandler.cancel_dump_traceback_later()
     if rank == 0:
         line = {
@@ -400,9 +541,9 @@ def run_ours(args):
             "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
             "config": workload_config(cfg, alpha0, C, L),
-            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
+            "clocks": clocks, "repeats": repeats, "e2e": e2e, "gpu_launches": int(launches),
             "roofline": roofline, "miss_path": miss_path, "cpu_baseline": cpu_baseline,
-            "hit_stats": hit_summary(st), "other_runs": extra,
+            "hit_stats": hit_summary(cfg, st, K, L), "other_runs": extra,
         }
         if args.layers is not None:
             line["config"]["reduced_layers"] = True
@@ -459,11 +600,14 @@ def oracle_decode_steps(cfg, alpha, C, L, first_step, n_steps, max_seconds=None,
 
 
 def cpu_oracle_sample(cfg, alpha, C, L, W, K, budget_s):
+    """The oracle on the timed decode steps and, where those take it less than the budget, on the steps
+    of the same stream that follow them."""
     import oracle
-    secs, done = oracle_decode_steps(cfg, alpha, C, L, W, K, max_seconds=budget_s)
+    n = max(K, min(cfg.decode_steps - W, 512))
+    secs, done = oracle_decode_steps(cfg, alpha, C, L, W, n, max_seconds=budget_s)
     return {"value": cfg.batch * done / secs, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
-            "sample": "the first %d of the %d timed decode steps, all %d layers each (about %.0f s of CPU work)"
-                      % (done, K, L, secs)}
+            "sample": "%d decode steps of the same stream from the first timed one on (the %d timed steps first), all %d "
+                      "layers each: %.0f s of CPU work" % (done, K, L, secs)}
 
 
 def run_reference(args):

@@ -850,7 +850,10 @@ int forward_on(melinoe_moe *h, const Scratch &sc, void *cuda_stream, const void 
 
     // ---- everything on the device: the decode kernel fetches the missed experts itself, the host is
     // not in the path at all and returns at once (the call's cache decisions are in stats_dev)
-    if (!use_gemm && h->pull_ok) {
+    // (Only where the call cannot need more distinct experts than there are slots: otherwise a fetched
+    // expert may have to take the slot of an expert the same call still computes with, which needs an
+    // order between the SMs that only separate launches give; those calls take the path below.)
+    if (!use_gemm && h->pull_ok && (long long)T * h->k <= h->C) {
         for (int c = 0; c < n_chunks; ++c) {
             TimedPair tp{nullptr, nullptr};
             if (h->timing) {

@@ -449,26 +449,29 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_decode_kernel(DecParams p, De
             // ---- gate/up: this warp's columns of the tile's rows.  A dependent mma.sync issues only every
             // ~110 cycles, so the k-steps go to four independent accumulators, and the fragment loads of
             // four steps are issued before their four products.
-            float cg[4][4];
+            // (Where a warp has 16 m-tiles of output accumulators, d_model above 2048, registers only allow
+            // two steps at a time.)
+            constexpr int GG = (MT_ > 8 || MT_ == 0) ? 2 : 4;
+            float cg[GG][4];
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
+            for (int i = 0; i < GG; ++i)
                 cg[i][0] = cg[i][1] = cg[i][2] = cg[i][3] = 0.f;
             {
                 const uint32_t arow = rowbase + sel_gu * 2 * d;
                 const uint32_t ch0 = (uint32_t)(2 * warp * MT + kh);
 #pragma unroll
-                for (int i0 = 0; i0 < kMaxMt; i0 += 4) {
+                for (int i0 = 0; i0 < kMaxMt; i0 += GG) {
                     if (i0 < MT) {
-                        uint32_t af[4][4], bf[4][2];
+                        uint32_t af[GG][4], bf[GG][2];
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
+                        for (int j = 0; j < GG; ++j) {
                             const int i = i0 + j < MT ? i0 + j : i0;     // beyond the warp's last step: a valid address, product unused
                             ldmatrix_x4(arow + (((ch0 + 2 * i) ^ swz) << 4), af[j][0], af[j][1], af[j][2], af[j][3]);
                             bf[j][0] = has_tok ? lds32(xrow + i * 32) : 0u;
                             bf[j][1] = has_tok ? lds32(xrow + i * 32 + 16) : 0u;
                         }
 #pragma unroll
-                        for (int j = 0; j < 4; ++j)
+                        for (int j = 0; j < GG; ++j)
                             if (i0 + j < MT)
                                 mma_16816(cg[j], af[j][0], af[j][1], af[j][2], af[j][3], bf[j][0], bf[j][1]);
                     }
@@ -479,7 +482,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_decode_kernel(DecParams p, De
             // warp reads the complete tile
 #pragma unroll
             for (int i = 0; i < 4; ++i)
-                buf[warp * kBufPitch + i * 32 + lane] = (cg[0][i] + cg[1][i]) + (cg[2][i] + cg[3][i]);
+                buf[warp * kBufPitch + i * 32 + lane] = GG == 4 ? (cg[0][i] + cg[1][i]) + (cg[2][i] + cg[3][i]) : cg[0][i] + cg[GG - 1][i];
             asm volatile("bar.sync 1, %0;" ::"n"(NW * 32) : "memory");
             {
                 const int e = warp * 8 + (lane & 7), pg = lane >> 3;
@@ -512,13 +515,14 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_decode_kernel(DecParams p, De
                 const uint32_t km = (2 * tig < m ? 0x0000ffffu : 0u) | (2 * tig + 1 < m ? 0xffff0000u : 0u);
                 const uint32_t drow = rowbase + 4 * d;
                 const uint32_t cc0 = (uint32_t)(warp * MT * 2);
+                constexpr int DG = (MT_ > 8 || MT_ == 0) ? 2 : 4;      // loads (of two m-tiles each) per group
 #pragma unroll
-                for (int m0 = 0; m0 < kMaxMt; m0 += 8) {
+                for (int m0 = 0; m0 < kMaxMt; m0 += 2 * DG) {
                     if (m0 < MT) {
                         // fragment loads of up to eight m-tiles first, then their products
-                        uint32_t rf[4][4];
+                        uint32_t rf[DG][4];
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
+                        for (int j = 0; j < DG; ++j) {
                             // a load covers two m-tiles; an odd last one is fetched together with the one before
                             // it (or, if it is the warp's only one, with 16 columns that are not used)
                             int mi = m0 + 2 * j;
@@ -529,7 +533,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_decode_kernel(DecParams p, De
                             ldmatrix_x4_trans(drow + (((cc0 + 2 * mi + mat) ^ swz) << 4), rf[j][0], rf[j][1], rf[j][2], rf[j][3]);
                         }
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
+                        for (int j = 0; j < DG; ++j) {
                             const int mi = m0 + 2 * j;
                             if (mi + 1 < MT) {
                                 mma_16816(acc[mi], rf[j][0] & km, rf[j][1] & km, 0u, 0u, bd, 0u);
@@ -566,7 +570,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_decode_kernel(DecParams p, De
         {
             unsigned long long *yacc = reinterpret_cast<unsigned long long *>(p.yacc);
             auto add = [&](int t, int c, float v) {
-                const long long fx = __double2ll_rn((double)v * 1099511627776.0);
+                const long long fx = __float2ll_rn(v * 1099511627776.0f);    // exact scaling, then to the nearest 2^-40
                 atomicAdd(yacc + (size_t)t * d + c, (unsigned long long)fx);
             };
 #pragma unroll
@@ -617,7 +621,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_decode_kernel(DecParams p, De
         for (int e = tid; e < N; e += kThreads) {
             const long long fx = __ldcg(yacc + e);
             yacc[e] = 0;                                     // the accumulator is left clean for the next launch
-            float v = (float)((double)fx * (1.0 / 1099511627776.0));
+            float v = __ll2float_rn(fx) * (1.0f / 1099511627776.0f);     // one rounding, then an exact scaling
             const size_t o = (size_t)tok0 * d + e;           // element e of the launch's [tokens][d] block
             if (acc_in)
                 v += __ldcg(p.ybuf + o);
