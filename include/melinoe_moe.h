@@ -220,22 +220,22 @@ int melinoe_moe_forward_host(melinoe_moe_t *h, void *cuda_stream, const void *hi
  * stray cudaMalloc, and code that runs where the CUDA allocator must not be entered at all.  This
  * entry point runs the same layer, same kernels and same cache state, but takes every byte of
  * scratch (routing tables, gather lists, the FFN kernel's per-SM partial outputs) from one array
- * of melinoe_moe_static_scratch_bytes() (about 10.1 MiB) that is part of the library's device
+ * of melinoe_moe_static_scratch_bytes() (400 KiB) that is part of the library's device
  * image: each GPU that loads the library holds it until the process exits.  It calls no
  * cudaMalloc, cudaFree, event-creating or otherwise allocating routine, under either eviction
  * policy (the events a call may need are made when the handle is created).
  *
  * Limits, all checked before anything is queued, MELINOE_ERR_UNSUPPORTED beyond them:
- *   n_tokens <= 8, n_tokens * top_k <= 64, and SMs * n_tokens * d_model * 4 bytes <= 10 MiB
- *   (on a 148-SM device: n_tokens * d_model <= 17 712, e.g. 8 tokens at d_model 2048, 4 at 4096).
+ *   n_tokens <= 8 and n_tokens * top_k <= 64 (every width the library supports fits).
  * MELINOE_ERR_STATE if kernel timing is enabled on the handle (timed calls create events), or if
  * the handle's device is not the current one.
  *
  * The first call on a device looks up the array's device address (cudaGetSymbolAddress) with
  * that device current; make this first call before any stream capture begins.
  * Every call on a device, of every handle, uses the same array: it keeps the previous call's
- * contents (nothing in it has to start from zero: each table is written by the call's own kernels
- * before it is read), and two such calls that can overlap on the GPU (different streams without an
+ * contents (the tables are written by the call's own kernels before they are read; the one part that
+ * has to start from zero, the output accumulator, is cleared by the kernel that used it), and two
+ * such calls that can overlap on the GPU (different streams without an
  * ordering between them) race on it.  Calls on one stream, or ordered by events, are safe, and may
  * be mixed freely with melinoe_moe_forward on the same handle.
  * The inspection calls (melinoe_moe_last_*) read the scratch of the most recent call, so after a
@@ -304,11 +304,29 @@ int melinoe_trace_miss_proxies(void *cuda_stream, const int32_t *trace_dev, int 
 int melinoe_moe_reset_cache(melinoe_moe_t *h);
 
 /*
- * Post-deployment prefetch of Section 3.2 (Eq. 5: preload the Top-C predicted experts before
- * generation).  Loads up to cache_slots experts, in the order given, as if each were a miss
- * of its own call (counted in the totals).  Synchronous.
+ * Post-deployment prefetch of Section 3.2 (Eq. 5: the Top-C experts the activation predictor names
+ * are loaded into the cache before generation begins; the predictor itself is not part of this
+ * library, the caller supplies the set).  Up to cache_slots expert ids, host memory; each id is one
+ * cache request of its own, in the order given, as if it were the only expert of a call: a
+ * resident expert is re-stamped (counted as a hit), a missing one takes the lowest empty slot,
+ * else the policy's victim (counted as a miss; under the count policy every id's count is raised
+ * by one without a decay step).
+ * The call queues its work on the handle's copy stream, behind everything already queued on the
+ * handle, and returns: on a bf16 store the device can address, a planning kernel and a copy kernel
+ * that reads the experts over the host link itself (the host is not involved); otherwise the host
+ * waits for the planning kernel's list and issues one cudaMemcpyAsync per expert.  The next forward
+ * call of the handle, on whatever stream, waits for the preload on the device before it starts.
  */
 int melinoe_moe_preload(melinoe_moe_t *h, const int32_t *expert_ids_host, int n);
+
+/*
+ * The same for a batch (Section 4.3 "Effect of Batch Size": the predictor pools the most likely
+ * experts across all sequences of the batch; the paper does not say how, the reading taken here is
+ * a vote).  lists_host [n_seq][per_seq] int32: every sequence's own predicted set.  An expert's
+ * vote is the number of sequences whose list contains it; the cache_slots experts with the most
+ * votes (at least one), the lower id first among equals, are preloaded in that order.
+ */
+int melinoe_moe_preload_pooled(melinoe_moe_t *h, const int32_t *lists_host, int n_seq, int per_seq);
 
 /*
  * Inspection (synchronise the stream first; these copy from the device and block).

@@ -455,6 +455,49 @@ int moe_oracle_cache_preload(moe_oracle_cache *c, const int32_t *ids, int n, moe
     return n;
 }
 
+/*
+ * Pooled prefetch set of a batch (Section 4.3 "Effect of Batch Size": the predictor pools the most
+ * likely experts across the sequences of the batch; the paper gives no rule, the reading taken is
+ * a vote).  lists[n_seq][per_seq]: every sequence's own predicted set.  vote(e) = number of
+ * sequences whose list contains e.  The result is the C experts with the largest non-zero vote,
+ * by decreasing vote, the lower id first among equal votes; returns how many were written to out,
+ * or -1 on a bad id.  Written as a selection sort over the votes, nothing cleverer.
+ */
+int moe_oracle_pool_prefetch(const int32_t *lists, int n_seq, int per_seq, int E, int C, int32_t *out)
+{
+    int *vote = (int *)calloc((size_t)E, sizeof(int));
+    unsigned char *in_list = (unsigned char *)calloc((size_t)E, 1);
+    int n = 0;
+    for (int q = 0; q < n_seq; ++q) {
+        for (int e = 0; e < E; ++e)
+            in_list[e] = 0;
+        for (int j = 0; j < per_seq; ++j) {
+            const int e = lists[(size_t)q * per_seq + j];
+            if (e < 0 || e >= E) {
+                n = -1;
+                goto done;
+            }
+            in_list[e] = 1;
+        }
+        for (int e = 0; e < E; ++e)
+            vote[e] += in_list[e];
+    }
+    while (n < C) {
+        int best = -1;
+        for (int e = 0; e < E; ++e)
+            if (vote[e] > 0 && (best < 0 || vote[e] > vote[best]))
+                best = e;                      /* strict >: the lowest id wins among equal votes */
+        if (best < 0)
+            break;
+        out[n++] = best;
+        vote[best] = 0;
+    }
+done:
+    free(vote);
+    free(in_list);
+    return n;
+}
+
 void moe_oracle_cache_counts(const moe_oracle_cache *c, float *count)
 {
     for (int e = 0; e < c->E; ++e)

@@ -12,7 +12,7 @@ import numpy as np
 
 from . import build as _build
 
-__all__ = ["threads", "logits", "topk", "route", "gather", "quantize_q4", "dequantize_q4", "miss_proxies", "ExpertCache", "ffn_combine", "layer_forward"]
+__all__ = ["pool_prefetch", "threads", "logits", "topk", "route", "gather", "quantize_q4", "dequantize_q4", "miss_proxies", "ExpertCache", "ffn_combine", "layer_forward"]
 
 _lib = None
 
@@ -34,6 +34,8 @@ def _L():
         lib.moe_oracle_cache_preload.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]
         lib.moe_oracle_cache_preload.restype = C.c_int
         lib.moe_oracle_cache_counts.argtypes = [C.c_void_p, C.c_void_p]
+        lib.moe_oracle_pool_prefetch.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p]
+        lib.moe_oracle_pool_prefetch.restype = C.c_int
         lib.moe_oracle_logits.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                           C.c_int, C.c_int, C.c_int, C.c_void_p]
         lib.moe_oracle_topk.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p]
@@ -55,6 +57,18 @@ def _u16(a) -> np.ndarray:
     a = np.ascontiguousarray(a)
     assert a.dtype == np.uint16, "bf16 tensors are passed as uint16 bit patterns"
     return a
+
+
+def pool_prefetch(lists, n_experts: int, cache_slots: int) -> np.ndarray:
+    """Pooled prefetch set of a batch (Section 4.3, batch size): lists [n_seq][per_seq] of every
+    sequence's predicted experts -> the cache_slots most-voted experts, in load order."""
+    a = np.ascontiguousarray(lists, dtype=np.int32)
+    assert a.ndim == 2
+    out = np.empty(max(cache_slots, 1), dtype=np.int32)
+    n = _L().moe_oracle_pool_prefetch(_p(a), a.shape[0], a.shape[1], n_experts, cache_slots, _p(out))
+    if n < 0:
+        raise ValueError("expert index out of range")
+    return out[:n].copy()
 
 
 def threads() -> int:

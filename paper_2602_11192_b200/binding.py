@@ -25,6 +25,7 @@ EXPORTED_SYMBOLS = [
     "melinoe_moe_last_call_used_gemm", "melinoe_moe_set_policy", "melinoe_moe_cache_counts", "melinoe_moe_expert_bytes_q4",
     "melinoe_moe_pack_expert_q4", "melinoe_moe_register_host_experts_q4", "melinoe_trace_miss_proxies", "melinoe_launch_count",
     "melinoe_last_cuda_error", "melinoe_strerror", "melinoe_moe_ffn_launch_times_ms", "melinoe_debug_fail_host_copy",
+    "melinoe_moe_preload_pooled",
 ]
 
 STATUS_NAMES = {0: "OK", 1: "INVALID", 2: "STATE", 3: "CUDA", 4: "NOMEM", 5: "TIMEOUT", 6: "UNSUPPORTED"}
@@ -89,6 +90,7 @@ def lib():
     L.melinoe_moe_set_policy.argtypes = [vp, i32, C.c_float]
     L.melinoe_moe_cache_counts.argtypes = [vp, vp]
     L.melinoe_moe_preload.argtypes = [vp, vp, i32]
+    L.melinoe_moe_preload_pooled.argtypes = [vp, vp, i32, i32]
     L.melinoe_moe_last_routing.argtypes = [vp, vp, vp]
     L.melinoe_moe_last_logits.argtypes = [vp, vp]
     L.melinoe_moe_last_requests.argtypes = [vp, vp, C.POINTER(i32)]
@@ -261,6 +263,14 @@ class MoELayer:
         import numpy as np
         ids = np.ascontiguousarray(expert_ids, dtype=np.int32)
         self._ck(lib().melinoe_moe_preload(self._h, ids.ctypes.data, ids.size), "melinoe_moe_preload")
+
+    def preload_pooled(self, lists) -> None:
+        """lists [n_seq][per_seq]: every sequence's own predicted set; the most-voted experts are preloaded."""
+        import numpy as np
+        a = np.ascontiguousarray(lists, dtype=np.int32)
+        assert a.ndim == 2
+        self._ck(lib().melinoe_moe_preload_pooled(self._h, a.ctypes.data, a.shape[0], a.shape[1]),
+                 "melinoe_moe_preload_pooled")
 
     # -- inspection (blocking)
     def last_routing(self, n_tokens: int):

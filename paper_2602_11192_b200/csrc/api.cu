@@ -177,6 +177,11 @@ struct melinoe_moe {
 
     // page-locked host memory: the miss queue the planning kernel writes
     HostPlan *hplan = nullptr;
+    // preload: the fetch list (device, and page-locked host copy), its event on the copy stream
+    PreloadList *pre_dev = nullptr, *pre_host = nullptr;
+    cudaEvent_t ev_preload = nullptr;
+    bool preload_pending = false;       // the next forward call has to wait for ev_preload
+    uint32_t preload_seq = 0;
 
     cudaStream_t copy_stream = nullptr;
     cudaEvent_t ev_last = nullptr;      // end of the most recent call on the caller's stream
@@ -532,6 +537,11 @@ int melinoe_moe_create(int d, int F, int E, int k, int C, melinoe_moe_t **out)
     CR(cudaMemcpy(h->cache, &c0, sizeof c0, cudaMemcpyHostToDevice));
     CR(cudaHostAlloc(&h->hplan, sizeof(HostPlan), cudaHostAllocMapped | cudaHostAllocPortable));
     std::memset(h->hplan, 0, sizeof(HostPlan));
+    CR(cudaMalloc(&h->pre_dev, sizeof(PreloadList)));
+    CR(cudaMemset(h->pre_dev, 0, sizeof(PreloadList)));
+    CR(cudaHostAlloc(&h->pre_host, sizeof(PreloadList), cudaHostAllocMapped | cudaHostAllocPortable));
+    std::memset(h->pre_host, 0, sizeof(PreloadList));
+    CR(cudaEventCreateWithFlags(&h->ev_preload, cudaEventDisableTiming));
     CR(cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking));
     CR(cudaEventCreateWithFlags(&h->ev_last, cudaEventDisableTiming));
     CR(cudaEventCreateWithFlags(&h->ev_plan, cudaEventDisableTiming));
@@ -585,6 +595,11 @@ int melinoe_moe_destroy(melinoe_moe_t *h)
     cudaFree(h->stage_stats);
     if (h->hplan)
         cudaFreeHost(h->hplan);
+    cudaFree(h->pre_dev);
+    if (h->pre_host)
+        cudaFreeHost(h->pre_host);
+    if (h->ev_preload)
+        cudaEventDestroy(h->ev_preload);
     if (h->copy_stream)
         cudaStreamDestroy(h->copy_stream);
     if (h->ev_last)
@@ -806,6 +821,11 @@ int forward_on(melinoe_moe *h, const Scratch &sc, void *cuda_stream, const void 
                melinoe_moe_stats *stats_dev)
 {
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    if (h->preload_pending) {
+        // a preload is queued on the copy stream: this call's kernels come after it
+        CU_TRY(cudaStreamWaitEvent(s, h->ev_preload, 0));
+        h->preload_pending = false;
+    }
     const uint32_t gmax = (uint32_t)gmax_for(h, T);
     h->call_seq += 1;
     h->last_T = T;
@@ -1262,62 +1282,111 @@ int melinoe_moe_preload(melinoe_moe_t *h, const int32_t *ids, int n)
 {
     if (!h || n < 0 || (n > 0 && !ids) || n > h->C)
         return MELINOE_ERR_INVALID;
+    for (int i = 0; i < n; ++i)
+        if (ids[i] < 0 || ids[i] >= h->E)
+            return MELINOE_ERR_INVALID;
     if (!h->host_experts[0])
         return MELINOE_ERR_STATE;
-    int rc = wait_idle(h);
-    if (rc != MELINOE_OK)
-        return rc;
-    DevCache c;
-    CU_TRY(cudaMemcpy(&c, h->cache, sizeof c, cudaMemcpyDeviceToHost));
-    for (int i = 0; i < n; ++i) {
-        const int e = ids[i];
-        if (e < 0 || e >= h->E)
-            return MELINOE_ERR_INVALID;
-        c.call_no += 1;
-        const uint64_t st = ++c.counter;
-        if (h->policy == MELINOE_POLICY_COUNT)
-            c.count[e] += 1.0f;
-        if (c.slot_of_expert[e] >= 0) {
-            c.stamp[c.slot_of_expert[e]] = st;
-            c.tot_hits += 1;
-            continue;
-        }
-        int victim = -1;
-        for (int s = 0; s < h->C && victim < 0; ++s)
-            if (c.expert_of_slot[s] < 0)
-                victim = s;
-        if (victim < 0) {
-            for (int s = 0; s < h->C; ++s) {
-                if (victim < 0) {
-                    victim = s;
-                } else if (h->policy == MELINOE_POLICY_COUNT) {
-                    const float cs = c.count[c.expert_of_slot[s]], cv = c.count[c.expert_of_slot[victim]];
-                    if (cs < cv || (cs == cv && c.stamp[s] < c.stamp[victim]))
-                        victim = s;
-                } else if (c.stamp[s] < c.stamp[victim]) {
-                    victim = s;
-                }
+    if (h->sticky.load() != MELINOE_OK)
+        return h->sticky.load();
+    if (n == 0)
+        return MELINOE_OK;
+    // behind everything already queued on the handle (whose kernels may still read the slots)
+    if (h->has_last)
+        CU_TRY(cudaStreamWaitEvent(h->copy_stream, h->ev_last, 0));
+    PreloadParams pp;
+    pp.cache = h->cache;
+    pp.list = h->pre_dev;
+    pp.host_list = nullptr;
+    for (int i = 0; i < kMaxExperts; ++i)
+        pp.ids[i] = i < n ? ids[i] : -1;
+    pp.n = n;
+    pp.C = h->C;
+    pp.policy = h->policy;
+    pp.seq = ++h->preload_seq;
+    if (h->pull_ok) {
+        // the cache requests and the copies both run on the device: nothing to wait for here
+        CU_TRY(launch_preload_plan(h->copy_stream, pp));
+        FetchParams fp;
+        fp.list = h->pre_dev;
+        fp.host_blobs = h->host_dev;
+        fp.slots = h->slots;
+        fp.slot_stride = h->slot_stride;
+        fp.rows = h->F;
+        fp.row_bytes = 6 * h->d;
+        fp.rows_per_piece = 49152 / fp.row_bytes > 0 ? 49152 / fp.row_bytes : 1;
+        fp.piece_bytes = fp.rows_per_piece * fp.row_bytes;
+        fp.err = h->err_word;
+        CU_TRY(launch_fetch_experts(h->copy_stream, h->n_sms, fp));
+        CU_TRY(cudaEventRecord(h->ev_preload, h->copy_stream));
+    } else {
+        // the host issues the copies: it has to see the list the planning kernel wrote
+        void *hl = nullptr;
+        CU_TRY(cudaHostGetDevicePointer(&hl, h->pre_host, 0));
+        pp.host_list = static_cast<PreloadList *>(hl);
+        CU_TRY(launch_preload_plan(h->copy_stream, pp));
+        CU_TRY(cudaStreamSynchronize(h->copy_stream));
+        const volatile PreloadList &vl = *h->pre_host;
+        if (vl.seq != pp.seq || vl.n < 0 || vl.n > n)
+            return MELINOE_ERR_STATE;
+        const int nf = vl.n;
+        for (int i = 0; i < nf; ++i) {
+            const int e = vl.expert[i], slot = vl.slot[i];
+            if (e < 0 || e >= h->E || slot < 0 || slot >= h->C)
+                return MELINOE_ERR_STATE;
+            if (h->store_q4) {
+                const unsigned b = h->q4_turn++ & 1u;
+                char *stage = h->q4_stage + (size_t)b * h->q4_bytes;
+                if (h->q4_used[b])
+                    CU_TRY(cudaStreamWaitEvent(h->copy_stream, h->ev_q4_expanded[b], 0));
+                CU_TRY(cudaMemcpyAsync(stage, h->host_experts[e], h->q4_bytes, cudaMemcpyHostToDevice, h->copy_stream));
+                CU_TRY(cudaEventRecord(h->ev_q4_copied[b], h->copy_stream));
+                CU_TRY(cudaStreamWaitEvent(h->dq_stream, h->ev_q4_copied[b], 0));
+                CU_TRY(launch_dequant_q4(h->dq_stream, stage, h->slots + (size_t)slot * h->slot_stride, h->d, h->F, h->n_sms));
+                CU_TRY(cudaEventRecord(h->ev_q4_expanded[b], h->dq_stream));
+                h->q4_used[b] = true;
+            } else {
+                CU_TRY(cudaMemcpyAsync(h->slots + (size_t)slot * h->slot_stride, h->host_experts[e], h->expert_bytes,
+                                       cudaMemcpyHostToDevice, h->copy_stream));
             }
-            c.slot_of_expert[c.expert_of_slot[victim]] = -1;
-            c.tot_evictions += 1;
         }
         if (h->store_q4) {
-            // the handle is idle (wait_idle above): stage, expand, wait
-            CU_TRY(cudaMemcpy(h->q4_stage, h->host_experts[e], h->q4_bytes, cudaMemcpyHostToDevice));
-            CU_TRY(launch_dequant_q4(h->dq_stream, h->q4_stage, h->slots + (size_t)victim * h->slot_stride, h->d, h->F,
-                                     h->n_sms));
-            CU_TRY(cudaStreamSynchronize(h->dq_stream));
-        } else {
-            CU_TRY(cudaMemcpy(h->slots + (size_t)victim * h->slot_stride, h->host_experts[e], h->expert_bytes,
-                              cudaMemcpyHostToDevice));
+            // the event has to cover the copy stream (planning kernel) and the expansion stream
+            CU_TRY(cudaEventRecord(h->ev_arrive, h->dq_stream));
+            CU_TRY(cudaStreamWaitEvent(h->copy_stream, h->ev_arrive, 0));
         }
-        c.expert_of_slot[victim] = e;
-        c.slot_of_expert[e] = victim;
-        c.stamp[victim] = st;
-        c.tot_misses += 1;
+        CU_TRY(cudaEventRecord(h->ev_preload, h->copy_stream));
     }
-    CU_TRY(cudaMemcpy(h->cache, &c, sizeof c, cudaMemcpyHostToDevice));
+    h->preload_pending = true;
     return MELINOE_OK;
+}
+
+int melinoe_moe_preload_pooled(melinoe_moe_t *h, const int32_t *lists_host, int n_seq, int per_seq)
+{
+    if (!h || !lists_host || n_seq <= 0 || per_seq <= 0)
+        return MELINOE_ERR_INVALID;
+    // votes: in how many sequences' lists an expert appears (once per list)
+    int votes[kMaxExperts] = {0};
+    for (int q = 0; q < n_seq; ++q) {
+        bool seen[kMaxExperts] = {false};
+        for (int j = 0; j < per_seq; ++j) {
+            const int e = lists_host[(size_t)q * per_seq + j];
+            if (e < 0 || e >= h->E)
+                return MELINOE_ERR_INVALID;
+            if (!seen[e]) {
+                seen[e] = true;
+                votes[e] += 1;
+            }
+        }
+    }
+    // the cache_slots experts with the most votes, the lower id first among equals, loaded in that order
+    int32_t chosen[kMaxExperts];
+    int n = 0;
+    for (int v = n_seq; v >= 1 && n < h->C; --v)
+        for (int e = 0; e < h->E && n < h->C; ++e)
+            if (votes[e] == v)
+                chosen[n++] = e;
+    return melinoe_moe_preload(h, chosen, n);
 }
 
 int melinoe_moe_last_routing(melinoe_moe_t *h, int32_t *idx_host, float *gate_host)

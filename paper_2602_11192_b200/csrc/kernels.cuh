@@ -114,6 +114,27 @@ cudaError_t launch_ffn_gemm(cudaStream_t stream, int phase, int n_sms, const Gem
 cudaError_t launch_combine_rows(cudaStream_t stream, const DevPlan *plan, const float *gate, const int32_t *inv_pos,
                                 const float *zs, uint16_t *out, int T, int d, int k, int n_shared, int n_sms);
 
+// ---- preload (Eq. 5): cache requests of a list of experts, and the copy of the missing ones into their slots
+struct PreloadParams {
+    DevCache *cache;
+    PreloadList *list;               // device
+    PreloadList *host_list;          // page-locked host memory as the device sees it, or null
+    int32_t ids[kMaxExperts];
+    int n, C, policy;
+    uint32_t seq;
+};
+struct FetchParams {
+    const PreloadList *list;
+    const char *const *host_blobs;   // device array: the host store as the device sees it
+    char *slots;
+    size_t slot_stride;
+    int rows, row_bytes;             // rows of one expert blob (d_ff) and their size
+    int rows_per_piece, piece_bytes; // rows copied at a time (at most 48 KB)
+    int *err;
+};
+cudaError_t launch_preload_plan(cudaStream_t stream, const PreloadParams &p);
+cudaError_t launch_fetch_experts(cudaStream_t stream, int n_sms, const FetchParams &p);
+
 // ---- cache-miss proxies of a recorded routing trace (Section 3.1, Definition C.1)
 cudaError_t launch_miss_proxies(cudaStream_t stream, const int32_t *idx, int n_layers, int T, int K, int E,
                                 const melinoe_proxy_config *cfgs, int n_cfg, double *soft_mean, long long *hard_total);

@@ -93,6 +93,15 @@ struct __align__(16) HostPlan {
     HostMiss miss[kMaxExperts];
 };
 
+// What a preload has to fetch, written by its planning kernel: device copy for the fetch kernel,
+// and a copy in page-locked host memory (seq written last) where the host issues the copies.
+struct PreloadList {
+    int32_t n;
+    uint32_t seq;
+    int32_t expert[kMaxExperts];
+    int32_t slot[kMaxExperts];
+};
+
 // Device side: publish the miss queue of call `seq` (one 16-byte store per record).
 __device__ inline void store16_host(void *dst, const void *rec)
 {

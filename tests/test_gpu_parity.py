@@ -256,11 +256,37 @@ def test_preload_fills_the_cache_before_the_first_token():
     P = _pair(d, F, E, k, C, seed=15)
     x = gen.hidden_states(15, 0, "decode", 0, 1, d)
     idx, _, _ = oracle.route(x, P.w_r, k)
-    P.gpu.layer.preload(np.array(sorted(idx[0].tolist()), np.int32))
-    res = P.gpu.forward_np(x)
-    assert res["stats"]["misses"] == 0 and res["stats"]["hits"] == k
+    P.preload(sorted(idx[0].tolist()))
+    _, o = P.step(x)
+    assert o["stats"]["misses"] == 0 and o["stats"]["hits"] == k
     eos, tot = P.gpu.layer.cache_state()
     assert tot["misses"] == k and set(eos[:k].tolist()) == set(idx[0].tolist())
+    P.close()
+
+
+@pytest.mark.parametrize("policy", ["lru", "count"])
+def test_preload_is_queued_and_matches_the_oracle(policy):
+    """Preloads in the middle of a stream of calls (on a warm cache: ids that are resident, ids that
+    evict, a full list of cache_slots ids), queued without any host synchronisation between them and
+    the calls around them; slot table, totals, counts and the following calls' traces and outputs
+    agree with the oracle; then the pooled variant for a batch."""
+    d, F, E, k, C = 512, 64, 12, 2, 5
+    P = _pair(d, F, E, k, C, seed=17)
+    if policy == "count":
+        P.set_policy("count", 0.9)
+    step = 0
+    for ids in ([3, 7], [7, 1, 9, 3, 0], [11], [2, 2, 5]):
+        P.preload(ids)
+        for _ in range(2):
+            P.step(gen.hidden_states(17, 0, "decode", step, 3, d))
+            step += 1
+    lists = np.array([[4, 6, 8], [6, 8, 10], [8, 1, 4], [0, 8, 6]], np.int32)
+    want = oracle.pool_prefetch(lists, E, C)
+    assert want.tolist() == [8, 6, 4, 0, 1]
+    P.gpu.layer.preload_pooled(lists)
+    P.cache.preload(want)
+    P.step(gen.hidden_states(17, 0, "decode", step, 4, d))
+    eos, _ = P.gpu.layer.cache_state()
     P.close()
 
 

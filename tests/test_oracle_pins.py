@@ -569,3 +569,23 @@ def test_missing_expert_is_reported():
     x = gen.hidden_states(25, 0, "decode", 0, 1, d)
     with pytest.raises(ValueError):
         oracle.ffn_combine(x, np.array([[1]], np.int32), np.ones((1, 1)), [ex[0], None], F)
+
+
+def test_pooled_prefetch_set_hand_worked_and_against_a_sort():
+    """Pooled prefetch of a batch: the hand-worked sets, then random batches against a plain sort of
+    (-votes, id) computed with collections.Counter; every chosen expert is named by some sequence."""
+    import collections
+    import json
+    g = json.load(open(os.path.join(GOLD, "pooled_prefetch.json")))
+    for c in g["cases"]:
+        got = oracle.pool_prefetch(np.array(c["lists"], np.int32), g["n_experts"], c["cache_slots"])
+        assert got.tolist() == c["expect"]
+    rs = np.random.default_rng(5)
+    for _ in range(50):
+        E, n_seq, m, C = int(rs.integers(4, 40)), int(rs.integers(1, 9)), int(rs.integers(1, 9)), int(rs.integers(1, 12))
+        lists = rs.integers(0, E, size=(n_seq, m)).astype(np.int32)
+        votes = collections.Counter(e for row in lists for e in set(row.tolist()))
+        want = [e for e, _ in sorted(votes.items(), key=lambda kv: (-kv[1], kv[0]))][:C]
+        assert oracle.pool_prefetch(lists, E, C).tolist() == want
+    with pytest.raises(ValueError):
+        oracle.pool_prefetch(np.array([[0, 11]], np.int32), 10, 4)
