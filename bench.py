@@ -219,12 +219,15 @@ class Runner:
         ms = e0.elapsed_time(e1)
         launches = M.melinoe_launch_count() - n0
         per_launch = None
+        self.copy_ms = self.copy_bytes = 0.0
         if with_kernel_timing:
             per_launch = []                                   # [layer] -> times of its K calls' launches
             for ls in st.layers:
                 per_launch.append(ls.layer.ffn_launch_times_ms())
                 ls.layer.ffn_time_ms()
-                ls.layer.transfer_time_ms()
+                cm, cb = ls.layer.transfer_time_ms()          # host-issued transfers only (copy-stream events)
+                self.copy_ms += cm
+                self.copy_bytes += cb
                 ls.layer.enable_timing(False)
         stats = stats_arrays(self.stats_dev[W:W + K])
         if int(stats["status"].max()) != 0:
@@ -285,10 +288,19 @@ def ffn_launch_analysis(cfg, stats, per_launch, hbm_peak, link_peak):
     miss_n = 0
     all_bytes = all_ms = 0.0
     K, L = stats["misses"].shape
+    if any(len(per_launch[l]) != K for l in range(L)):
+        # not one launch per call (calls whose transfers the host issues, one launch per compute group): no
+        # per-call attribution, only the sum over all launches
+        ms = float(sum(float(t.sum()) for t in per_launch))
+        n = int(sum(len(t) for t in per_launch))
+        by = float((stats["n_distinct"].astype(np.int64) + cfg.n_shared).sum()) * B_e
+        g = by / (ms * 1e-3) / 1e9
+        return {"resident": None, "fetching": None,
+                "all": {"launches": n, "avg_launch_us": 1e3 * ms / max(n, 1), "gbs": g, "frac_of_hbm": g / hbm_peak,
+                        "note": "one launch per compute group (the host issues this shape's transfers): experts streamed "
+                                "from their slots x bytes per expert / summed launch times"}}
     for l in range(L):
         t = per_launch[l]
-        if len(t) != K:
-            return None                     # not one launch per call (host-issued transfers): no per-call attribution
         for i in range(K):
             experts = int(stats["n_distinct"][i, l]) + cfg.n_shared
             m = int(stats["misses"][i, l])
@@ -336,6 +348,45 @@ def host_link_gbs(torch):
     return best
 
 
+def preload_record(torch, R, cfg, alpha, C, L, n_steps):
+    """First n_steps decode tokens from an empty cache (no prompt), plain and after melinoe_moe_preload of
+    each layer's C most preferred experts of the sequence (Eq. 5 with the bias standing in for the predictor)."""
+    st = R.stack
+    out = {}
+    for mode in ("cold", "preloaded"):
+        st.reset()
+        st.set_phase("decode")
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        if mode == "preloaded":
+            for l, ls in enumerate(st.layers):
+                pref = np.argsort(-st.bias[l].max(axis=0), kind="stable")[:C].astype(np.int32)
+                ls.layer.preload(pref)
+        t1 = time.perf_counter()
+        torch.cuda.synchronize()
+        t2 = time.perf_counter()
+        R.stats_dev.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for s in range(n_steps):
+            st.forward_all(R.dec_dev[s], R.out_dev, R.stats_dev[s])
+        e1.record()
+        torch.cuda.synchronize()
+        sa = stats_arrays(R.stats_dev[:n_steps])
+        out[mode] = {"decode_ms": e0.elapsed_time(e1), "misses": int(sa["misses"].sum()),
+                     "misses_per_layer_per_token": float(sa["misses"].sum()) / (n_steps * L * cfg.batch)}
+        if mode == "preloaded":
+            out[mode]["preload_queue_ms"] = (t1 - t0) * 1e3
+            out[mode]["preload_ms"] = (t2 - t0) * 1e3
+            out[mode]["preloaded_bytes"] = int(L * C * cfg.expert_bytes)
+    out["tokens"] = n_steps
+    out["saved_ms"] = out["cold"]["decode_ms"] - out["preloaded"]["decode_ms"]
+    out["note"] = ("%d decode tokens from an empty cache; preload = every layer's %d most preferred experts of the sequence's "
+                   "router bias, queued with melinoe_moe_preload (returns at once: preload_queue_ms is the host time of the "
+                   "%d calls, preload_ms the time until the copies have landed)" % (n_steps, C, L))
+    return out
+
+
 def shape_record(torch, M, gen, name, n_layers, K, W, hbm_peak, link_peak, peaks):
     """Decode throughput, FFN roofline and (where the prompt runs the grouped GEMM) the prefill GEMM's
     rate of one of the other workload shapes, at its full width with a reduced number of layers."""
@@ -354,6 +405,10 @@ def shape_record(torch, M, gen, name, n_layers, K, W, hbm_peak, link_peak, peaks
     rec.update(hit_summary(cfg, st, K, n_layers))
     _, _, st2, per_launch = R.timed_device(alpha, with_kernel_timing=True)
     rec["ffn"] = ffn_launch_analysis(cfg, st2, per_launch, hbm_peak, link_peak)
+    if R.copy_ms > 0:
+        g = R.copy_bytes / (R.copy_ms * 1e-3) / 1e9
+        rec["host_issued_transfers"] = {"gbs": g, "frac_of_link": g / link_peak, "bytes": R.copy_bytes,
+                                        "note": "cudaMemcpyAsync waves on the copy stream, events around each wave"}
     # the prompt again with events around the grouped GEMM launches of every compute group
     if cfg.prefill_tokens and cfg.d_ff % 128 == 0 and cfg.batch * cfg.prefill_tokens > 8:
         R.prepare(alpha, timing_prefill=True)
@@ -376,6 +431,13 @@ def shape_record(torch, M, gen, name, n_layers, K, W, hbm_peak, link_peak, peaks
                                "note": "flops = 6 d_model d_ff per (token, expert) pair; time = CUDA events around the two "
                                        "GEMM launches of every compute group, transfers excluded"}
     R.close()
+    # the same shape with every expert resident: the decode kernel in its HBM-bound regime
+    Ra = Runner(torch, M, gen, cfg, alpha, cfg.n_experts, n_layers, K, W)
+    Ra.timed_device(alpha)                                           # warm: the first pass fetches what the prompt did not
+    _, _, st3, pl3 = Ra.timed_device(alpha, with_kernel_timing=True)
+    a3 = ffn_launch_analysis(cfg, st3, pl3, hbm_peak, link_peak)
+    rec["ffn_all_resident"] = a3["resident"] if a3 else None
+    Ra.close()
     return rec
 
 
@@ -489,6 +551,10 @@ def run_ours(args):
             ms_p, _, st_p, _ = R.timed_device(alpha0)
             extra[name] = dict(value=cfg.batch * K / (ms_p * 1e-3), **hit_summary(cfg, st_p, K, L))
         R.stack.set_policy("lru")
+        # cold start with and without a preload of every layer's Top-C of the sequence's router bias (the
+        # stand-in for the paper's activation predictor): misses and time of the first decode tokens
+        phase("cold start with and without preload")
+        extra["preload"] = preload_record(torch, R, cfg, alpha0, C, L, min(64, W + K))
         R.close()
         # 4-bit host store (the paper keeps its experts in 4-bit form): a miss moves 3.76 times fewer bytes
         if cfg.d_ff % 64 == 0:

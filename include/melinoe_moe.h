@@ -68,6 +68,26 @@ typedef struct melinoe_moe_request {
 } melinoe_moe_request;
 
 /*
+ * Request trace (optional, melinoe_moe_set_trace): one record per forward call, written on the device
+ * in stream order by the call's routing / planning kernels, so that routing and cache decisions can
+ * be recorded without synchronising after every call.  A record is melinoe_moe_trace_record_bytes()
+ * long and holds, in this order:
+ *     melinoe_moe_trace_header
+ *     melinoe_moe_request  req[n_experts]         the first n_requests are the call's cache requests in order
+ *     int32_t              idx[max_tokens][top_k] routing indices of the call's first max_tokens tokens
+ *     float                gate[max_tokens][top_k] their gates
+ * (the whole rounded up to 16 bytes).
+ */
+typedef struct melinoe_moe_trace_header {
+    uint64_t call_no;     /* as in melinoe_moe_stats                                        */
+    int32_t n_tokens;     /* T of the call (indices beyond max_tokens are not recorded)     */
+    int32_t n_requests;   /* distinct routed experts of the call                            */
+    int32_t hits, misses;
+    int32_t status;       /* melinoe_status of the device-side part of the call             */
+    int32_t reserved;
+} melinoe_moe_trace_header;
+
+/*
  * Create one layer.  Shapes follow Eq. 1-3: router W_r [n_experts][d_model]; each expert has
  * W_g, W_u [d_ff][d_model] and W_d [d_model][d_ff].  Allocates, on the current device,
  * cache_slots expert slots of melinoe_moe_expert_bytes() each plus small tables, and creates
@@ -365,16 +385,44 @@ int melinoe_moe_ffn_launch_times_ms(melinoe_moe_t *h, float *ms_out, int capacit
 int melinoe_moe_transfer_time_ms(melinoe_moe_t *h, double *ms_out, uint64_t *bytes_out);
 
 /*
+ * Request trace of the handle's forward calls.  trace_buf: device memory (or page-locked host memory
+ * the device can address), 16-byte aligned, borrowed; bytes: its size; max_tokens: tokens per call
+ * whose routing is recorded.  The buffer is used as a ring of bytes / melinoe_moe_trace_record_bytes()
+ * records: the n-th call after this call (n = 1, 2, ...) writes record (n - 1) mod capacity.  The
+ * records of calls that have finished on the device are valid (synchronise the stream, or an event
+ * behind the calls, before reading).  NULL switches the trace off.  melinoe_moe_trace_count returns
+ * the number of calls recorded since the trace was set.  INVALID if the buffer holds no record.
+ * A recorded routing trace (the idx arrays of consecutive calls) is what melinoe_trace_miss_proxies
+ * evaluates.
+ */
+size_t melinoe_moe_trace_record_bytes(melinoe_moe_t *h, int max_tokens);
+int melinoe_moe_set_trace(melinoe_moe_t *h, void *trace_buf, size_t bytes, int max_tokens);
+int64_t melinoe_moe_trace_count(melinoe_moe_t *h);
+
+/*
+ * Per-layer cache sizes under one budget (the paper names per-layer cache budgets as future work in
+ * its limitations; Section 3.1 / Definition C.1 give the miss counts this works on).  Pure host code.
+ * hard_host [n_layers][n_sizes] int64: transfers of layer l with first_size + j slots (what
+ * melinoe_trace_miss_proxies returns as hard totals for consecutive cache sizes).  Every layer starts
+ * at first_size slots; the rest of budget (total slots over all layers) is handed out one slot at a
+ * time to the layer whose next slot saves the most transfers, the lower layer first among equals,
+ * until the budget is spent or no layer can grow.  slots_out [n_layers] receives the sizes.
+ * INVALID if the budget does not cover first_size slots per layer.
+ */
+int melinoe_allocate_slots(const int64_t *hard_host, int n_layers, int n_sizes, int first_size, int64_t budget,
+                           int32_t *slots_out);
+
+/*
  * Kernel timeline for profiling (no counterpart in the paper).  trace_dev: device memory of at
- * least 8 * 8 bytes per SM of the device (melinoe_moe_trace_ctas() * 64 bytes), 8-byte aligned,
+ * least 8 * 8 bytes per SM of the device (melinoe_moe_timeline_ctas() * 64 bytes), 8-byte aligned,
  * borrowed; NULL switches tracing off.  Every launch of the decode FFN kernel then overwrites, per
  * CTA, eight 64-bit nanosecond stamps of the device's global timer: 0 entry, 1 set-up done (plan
- * read, rows dealt out), 2 first tile of weights landed, 3 last tile computed, 4 arrived at the grid
- * barrier, 5 barrier passed, 6 output written, 7 exit.  Stamps of steps a CTA skipped keep their old
- * value.
+ * read, rows dealt out), 2 first tile of weights landed, 3 last tile computed, 4 partial output added
+ * and counted out, 5 (last CTA only) sums complete, 6 (last CTA only) output written, 7 exit.  Stamps of
+ * steps a CTA skipped keep their old value.
  */
-int melinoe_moe_set_trace(melinoe_moe_t *h, void *trace_dev, size_t bytes);
-int melinoe_moe_trace_ctas(melinoe_moe_t *h);
+int melinoe_moe_set_timeline(melinoe_moe_t *h, void *trace_dev, size_t bytes);
+int melinoe_moe_timeline_ctas(melinoe_moe_t *h);
 
 /* 1 if the most recent forward call of the handle ran its expert FFN as the tensor-core grouped
  * GEMM (calls of more than 8 tokens on shapes with d_model % 256 == 0 and d_ff % 128 == 0), 0 if it

@@ -20,7 +20,8 @@ EXPORTED_SYMBOLS = [
     "melinoe_moe_set_router_bias", "melinoe_moe_reserve", "melinoe_moe_forward", "melinoe_moe_forward_host",
     "melinoe_moe_reset_cache", "melinoe_moe_preload", "melinoe_moe_last_routing", "melinoe_moe_last_logits",
     "melinoe_moe_last_requests", "melinoe_moe_last_gather", "melinoe_moe_cache_state",
-    "melinoe_moe_enable_timing", "melinoe_moe_ffn_time_ms", "melinoe_moe_set_trace", "melinoe_moe_trace_ctas",
+    "melinoe_moe_enable_timing", "melinoe_moe_ffn_time_ms", "melinoe_moe_set_trace", "melinoe_moe_trace_count",
+    "melinoe_moe_trace_record_bytes", "melinoe_moe_set_timeline", "melinoe_moe_timeline_ctas", "melinoe_allocate_slots",
     "melinoe_moe_transfer_time_ms", "melinoe_moe_forward_static", "melinoe_moe_static_scratch_bytes",
     "melinoe_moe_last_call_used_gemm", "melinoe_moe_set_policy", "melinoe_moe_cache_counts", "melinoe_moe_expert_bytes_q4",
     "melinoe_moe_pack_expert_q4", "melinoe_moe_register_host_experts_q4", "melinoe_trace_miss_proxies", "melinoe_launch_count",
@@ -101,8 +102,14 @@ def lib():
     L.melinoe_moe_transfer_time_ms.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_uint64)]
     L.melinoe_moe_ffn_launch_times_ms.argtypes = [vp, vp, i32, C.POINTER(i32)]
     L.melinoe_debug_fail_host_copy.argtypes = [i32]
-    L.melinoe_moe_set_trace.argtypes = [vp, vp, sz]
-    L.melinoe_moe_trace_ctas.argtypes = [vp]
+    L.melinoe_moe_set_trace.argtypes = [vp, vp, sz, i32]
+    L.melinoe_moe_trace_count.argtypes = [vp]
+    L.melinoe_moe_trace_count.restype = C.c_int64
+    L.melinoe_moe_trace_record_bytes.argtypes = [vp, i32]
+    L.melinoe_moe_trace_record_bytes.restype = sz
+    L.melinoe_moe_set_timeline.argtypes = [vp, vp, sz]
+    L.melinoe_moe_timeline_ctas.argtypes = [vp]
+    L.melinoe_allocate_slots.argtypes = [vp, i32, i32, i32, C.c_int64, vp]
     L.melinoe_launch_count.restype = C.c_int64
     L.melinoe_last_cuda_error.restype = i32
     L.melinoe_strerror.argtypes = [i32]
@@ -330,12 +337,23 @@ class MoELayer:
         self._ck(lib().melinoe_moe_transfer_time_ms(self._h, C.byref(ms), C.byref(nb)), "melinoe_moe_transfer_time_ms")
         return ms.value, nb.value
 
-    def set_trace(self, trace_dev, n_bytes: int) -> None:
-        self._keep["trace"] = trace_dev
-        self._ck(lib().melinoe_moe_set_trace(self._h, _ptr(trace_dev), n_bytes), "melinoe_moe_set_trace")
+    def set_timeline(self, trace_dev, n_bytes: int) -> None:
+        self._keep["timeline"] = trace_dev
+        self._ck(lib().melinoe_moe_set_timeline(self._h, _ptr(trace_dev), n_bytes), "melinoe_moe_set_timeline")
 
-    def trace_ctas(self) -> int:
-        return int(lib().melinoe_moe_trace_ctas(self._h))
+    def timeline_ctas(self) -> int:
+        return int(lib().melinoe_moe_timeline_ctas(self._h))
+
+    def trace_record_bytes(self, max_tokens: int) -> int:
+        return int(lib().melinoe_moe_trace_record_bytes(self._h, max_tokens))
+
+    def set_trace(self, trace_buf, n_bytes: int, max_tokens: int) -> None:
+        """Request trace: one record per forward call into trace_buf (a ring of records), in stream order."""
+        self._keep["trace"] = trace_buf
+        self._ck(lib().melinoe_moe_set_trace(self._h, _ptr(trace_buf), n_bytes, max_tokens), "melinoe_moe_set_trace")
+
+    def trace_count(self) -> int:
+        return int(lib().melinoe_moe_trace_count(self._h))
 
     def ffn_time_ms(self):
         ms = C.c_double(0.0)

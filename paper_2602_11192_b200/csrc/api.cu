@@ -149,7 +149,11 @@ struct melinoe_moe {
     int cap_shared = -1;
     float *zbuf = nullptr;                 // grouped-GEMM path: expert outputs [sorted rows][d] fp32
     unsigned *sync = nullptr;              // counter of the decode kernel's rare "who is last" step (zero between launches)
-    unsigned long long *trace = nullptr;   // borrowed; see melinoe_moe_set_trace
+    unsigned long long *trace = nullptr;   // borrowed; see melinoe_moe_set_timeline
+    char *req_trace = nullptr;             // borrowed; see melinoe_moe_set_trace
+    size_t req_trace_cap = 0;              // records it holds
+    int req_trace_tokens = 0;
+    long long req_trace_count = 0;
     uint16_t *stage_in = nullptr, *stage_out = nullptr;
     // grouped-GEMM path (calls of more than 8 tokens): gathered activations, h, tensor maps
     bool gemm_ok = false, last_used_gemm = false;
@@ -854,6 +858,14 @@ int forward_on(melinoe_moe *h, const Scratch &sc, void *cuda_stream, const void 
     pp.gamma = h->gamma;
     pp.stats = stats_dev;
     pp.expert_bytes = h->store_q4 ? h->q4_bytes : h->expert_bytes;   // bytes one miss moves over the host link
+    pp.gate = sc.gate;
+    pp.trace_rec = nullptr;
+    pp.trace_max_tokens = h->req_trace_tokens;
+    if (h->req_trace) {
+        const TraceLayout tl = trace_layout(h->E, h->k, h->req_trace_tokens);
+        pp.trace_rec = h->req_trace + (size_t)(h->req_trace_count % (long long)h->req_trace_cap) * tl.bytes;
+        h->req_trace_count += 1;
+    }
     const bool small = route_plan_small_supported(T, h->k, h->d);
     if (small) {
         CU_TRY(launch_route_plan_small(s, static_cast<const uint16_t *>(hidden_dev), h->w_router, h->bias, h->token_seq,
@@ -1500,7 +1512,7 @@ int melinoe_moe_transfer_time_ms(melinoe_moe_t *h, double *ms_out, uint64_t *byt
     return MELINOE_OK;
 }
 
-int melinoe_moe_set_trace(melinoe_moe_t *h, void *trace_dev, size_t bytes)
+int melinoe_moe_set_timeline(melinoe_moe_t *h, void *trace_dev, size_t bytes)
 {
     if (!h)
         return MELINOE_ERR_INVALID;
@@ -1514,7 +1526,73 @@ int melinoe_moe_set_trace(melinoe_moe_t *h, void *trace_dev, size_t bytes)
     return MELINOE_OK;
 }
 
-int melinoe_moe_trace_ctas(melinoe_moe_t *h) { return h ? h->cfg.grid : 0; }
+int melinoe_moe_timeline_ctas(melinoe_moe_t *h) { return h ? h->cfg.grid : 0; }
+
+size_t melinoe_moe_trace_record_bytes(melinoe_moe_t *h, int max_tokens)
+{
+    if (!h || max_tokens <= 0)
+        return 0;
+    return trace_layout(h->E, h->k, max_tokens).bytes;
+}
+
+int melinoe_moe_set_trace(melinoe_moe_t *h, void *trace_buf, size_t bytes, int max_tokens)
+{
+    if (!h)
+        return MELINOE_ERR_INVALID;
+    if (!trace_buf) {
+        h->req_trace = nullptr;
+        h->req_trace_cap = 0;
+        return MELINOE_OK;
+    }
+    if (max_tokens <= 0 || !aligned16(trace_buf))
+        return MELINOE_ERR_INVALID;
+    const size_t rb = trace_layout(h->E, h->k, max_tokens).bytes;
+    if (bytes < rb)
+        return MELINOE_ERR_INVALID;
+    // the device must be able to write it: device memory, or page-locked host memory it can address
+    cudaPointerAttributes a;
+    if (cudaPointerGetAttributes(&a, trace_buf) != cudaSuccess || (a.type != cudaMemoryTypeDevice && a.type != cudaMemoryTypeHost) ||
+        !a.devicePointer) {
+        (void)cudaGetLastError();
+        return MELINOE_ERR_INVALID;
+    }
+    h->req_trace = static_cast<char *>(a.devicePointer);
+    h->req_trace_cap = bytes / rb;
+    h->req_trace_tokens = max_tokens;
+    h->req_trace_count = 0;
+    return MELINOE_OK;
+}
+
+int64_t melinoe_moe_trace_count(melinoe_moe_t *h) { return h ? (int64_t)h->req_trace_count : 0; }
+
+int melinoe_allocate_slots(const int64_t *hard, int n_layers, int n_sizes, int first_size, int64_t budget, int32_t *slots_out)
+{
+    if (!hard || !slots_out || n_layers <= 0 || n_sizes <= 0 || first_size <= 0)
+        return MELINOE_ERR_INVALID;
+    long long left = (long long)budget - (long long)n_layers * first_size;
+    if (left < 0)
+        return MELINOE_ERR_INVALID;
+    std::vector<int> at((size_t)n_layers, 0);
+    while (left > 0) {
+        int best = -1;
+        long long gain = -1;
+        for (int l = 0; l < n_layers; ++l)
+            if (at[l] + 1 < n_sizes) {
+                const long long g = (long long)(hard[(size_t)l * n_sizes + at[l]] - hard[(size_t)l * n_sizes + at[l] + 1]);
+                if (g > gain) {
+                    best = l;
+                    gain = g;
+                }
+            }
+        if (best < 0)
+            break;
+        at[best] += 1;
+        left -= 1;
+    }
+    for (int l = 0; l < n_layers; ++l)
+        slots_out[l] = first_size + at[l];
+    return MELINOE_OK;
+}
 
 int melinoe_moe_last_call_used_gemm(melinoe_moe_t *h) { return h && h->last_used_gemm ? 1 : 0; }
 

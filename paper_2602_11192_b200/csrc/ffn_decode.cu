@@ -704,13 +704,11 @@ cudaError_t ffn_decode_geometry(const DecLaunchCfg &cfg, int d, int F, int token
     geo->row_bytes = 6 * d;
     geo->x_pitch = 2 * d + 16;
     geo->tokens = tokens;
-    // staged hidden rows + the warps' partial tiles; the largest tile (8, 4, 2 or 1 rows) of which two
+    // staged hidden rows + the warps' partial tiles; the largest tile (at most 8 rows) of which two
     // stages fit beside them
     const size_t fixed = (size_t)tokens * geo->x_pitch + (size_t)NW * kBufPitch * sizeof(float);
     int tr = 8;
-    if (const char *ev = std::getenv("MELINOE_DEC_TR"))
-        tr = atoi(ev);
-    for (;; tr /= 2) {
+    for (;; --tr) {
         if (cfg.max_smem >= fixed + (size_t)2 * tr * geo->row_bytes)
             break;
         if (tr == 1)

@@ -37,7 +37,24 @@ struct PlanParams {
     float gamma;              // decay of the count policy
     melinoe_moe_stats *stats; // may be null
     size_t expert_bytes;
+    // request trace (melinoe_moe_set_trace): this call's record, or null; see trace_layout()
+    char *trace_rec;
+    int trace_max_tokens;
+    const float *gate;        // [T][k], for the trace record of calls planned by the general kernel
 };
+// Layout of one request-trace record for a layer of n_experts experts and top_k, max_tokens tokens.
+struct TraceLayout {
+    size_t req_off, idx_off, gate_off, bytes;
+};
+__host__ __device__ inline TraceLayout trace_layout(int n_experts, int top_k, int max_tokens)
+{
+    TraceLayout t;
+    t.req_off = sizeof(melinoe_moe_trace_header);
+    t.idx_off = t.req_off + (size_t)n_experts * sizeof(melinoe_moe_request);
+    t.gate_off = t.idx_off + (size_t)max_tokens * top_k * sizeof(int32_t);
+    t.bytes = (t.gate_off + (size_t)max_tokens * top_k * sizeof(float) + 15) / 16 * 16;
+    return t;
+}
 cudaError_t launch_plan(cudaStream_t stream, const PlanParams &p);
 
 // ---- router and planning in one kernel (one thread-block cluster), for calls of at most 8 tokens
@@ -76,7 +93,7 @@ struct DecLaunchCfg {
 // Shape of the shared-memory ring for one launch.
 struct DecGeometry {
     int n_warps;                     // consumer warps: 8 (d <= 2048) or 16
-    int tile_rows;                   // f rows per tile / ring stage: 8, 4, 2 or 1
+    int tile_rows;                   // f rows per tile / ring stage: at most 8
     int n_stages;
     int row_bytes;                   // bytes of one f row of the blob (its W_g, W_u and W_d^T rows)
     int stage_bytes;

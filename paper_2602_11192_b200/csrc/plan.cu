@@ -409,6 +409,29 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p)
         }
         publish_miss_queue(p.hplan, s_miss, n_miss, s_misc[4], s_misc[6], p.call_seq);
     }
+    // the call's request-trace record, if one is being kept
+    if (p.trace_rec) {
+        const TraceLayout tl = trace_layout(E, p.k, p.trace_max_tokens);
+        melinoe_moe_request *rq = reinterpret_cast<melinoe_moe_request *>(p.trace_rec + tl.req_off);
+        for (int i = tid; i < s_misc[0]; i += kPlanThreads)
+            rq[i] = melinoe_moe_request{s_req[i].expert, s_req[i].slot, s_req[i].hit, s_req[i].evicted};
+        const int nt = p.T < p.trace_max_tokens ? p.T : p.trace_max_tokens;
+        for (int i = tid; i < nt * p.k; i += kPlanThreads) {
+            reinterpret_cast<int32_t *>(p.trace_rec + tl.idx_off)[i] = p.idx[i];
+            reinterpret_cast<float *>(p.trace_rec + tl.gate_off)[i] = p.gate ? p.gate[i] : 0.0f;
+        }
+        if (tid == 0) {
+            melinoe_moe_trace_header th;
+            th.call_no = s_cache.call_no;
+            th.n_tokens = p.T;
+            th.n_requests = s_misc[0];
+            th.hits = s_misc[1];
+            th.misses = s_misc[2];
+            th.status = s_misc[6];
+            th.reserved = 0;
+            *reinterpret_cast<melinoe_moe_trace_header *>(p.trace_rec) = th;
+        }
+    }
     // the plan is complete: announce it (see DevPlan::ready_seq)
     __threadfence();
     __syncthreads();

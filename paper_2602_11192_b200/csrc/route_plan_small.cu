@@ -65,10 +65,13 @@ __device__ __forceinline__ uint64_t ballot64(bool lo, bool hi)
 __device__ __forceinline__ int rank_below(uint64_t mask, int bit) { return __popcll(mask & ((1ull << bit) - 1ull)); }
 
 // The cache half of a request record (the gather warp writes tok_off / n_tok, the other two words).
-__device__ __forceinline__ void write_req(ReqRec *r, int expert, int slot, int hit, int evicted, int at, int group)
+__device__ __forceinline__ void write_req(ReqRec *r, int expert, int slot, int hit, int evicted, int at, int group,
+                                          char *trace_req = nullptr)
 {
     *reinterpret_cast<int4 *>(&r->expert) = make_int4(expert, slot, hit, evicted);
     *reinterpret_cast<int2 *>(&r->vr_start) = make_int2(at, group);
+    if (trace_req)      // the same four words into the call's request-trace record
+        *reinterpret_cast<int4 *>(trace_req) = make_int4(expert, slot, hit, evicted);
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -282,6 +285,11 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
             if (lane < k) {
                 idx_out[(size_t)t * k + lane] = s_idx[t * k + lane];
                 gate_out[(size_t)t * k + lane] = ev / sum;
+                if (p.trace_rec && t < p.trace_max_tokens) {
+                    const TraceLayout tl = trace_layout(E, k, p.trace_max_tokens);
+                    reinterpret_cast<int32_t *>(p.trace_rec + tl.idx_off)[t * k + lane] = s_idx[t * k + lane];
+                    reinterpret_cast<float *>(p.trace_rec + tl.gate_off)[t * k + lane] = ev / sum;
+                }
             }
         }
         // these warps' results are written before the planning warp announces the plan
@@ -378,6 +386,7 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
     }
 
     // ---- the cache requests (warp 0)
+    char *tr_req = p.trace_rec ? p.trace_rec + trace_layout(E, k, p.trace_max_tokens).req_off : nullptr;
     const bool req0 = (need >> e0) & 1ull, req1 = (need >> e1) & 1ull;
     // compute groups: closed form under LRU; under the count policy known only after the misses
     // have been walked, one wave per miss at most
@@ -412,7 +421,7 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
             const unsigned long long st = counter + (unsigned long long)r + 1ull;
             s_key[soe] = (1ull << 63) | st;
             cache->stamp[soe] = st;
-            write_req(&plan->req[r], e, soe, 1, -1, r, 0);
+            write_req(&plan->req[r], e, soe, 1, -1, r, 0, tr_req ? tr_req + 16 * r : nullptr);
             s_grp_of[e] = 0;
             plan->dreq[r] = DecReq{p.slots + (size_t)soe * p.slot_stride, nullptr, e, 0, 0, 0};
         }
@@ -503,7 +512,7 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
                 s_live_occ[slot] = e;
                 s_live_stamp[slot] = st;
                 s_grp_of[e] = cur_group;
-                write_req(&plan->req[n_hits + i], e, slot, 0, ev, vr_at, cur_group);
+                write_req(&plan->req[n_hits + i], e, slot, 0, ev, vr_at, cur_group, tr_req ? tr_req + 16 * (n_hits + i) : nullptr);
                 s_miss_expert[i] = e;
                 s_miss_slot[i] = slot;
                 s_miss_group[i] = cur_group;
@@ -538,7 +547,7 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
                 dep = 0;
             ev_flag[h] = ev >= 0;
             const int vr_at = n_hits + p.n_shared + i;
-            write_req(&plan->req[n_hits + i], e, slot, 0, ev, vr_at, group);
+            write_req(&plan->req[n_hits + i], e, slot, 0, ev, vr_at, group, tr_req ? tr_req + 16 * (n_hits + i) : nullptr);
             // cache update: the last miss that lands in a slot keeps it
             const bool stays = i + C >= n_miss;
             {
@@ -618,6 +627,17 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
         }
         const HostPlanHeader hdr{n_miss, n_groups, status, p.call_seq};
         store16_host(&p.hplan->hdr, &hdr);
+        if (p.trace_rec) {
+            melinoe_moe_trace_header th;
+            th.call_no = call_no;
+            th.n_tokens = T;
+            th.n_requests = n_req;
+            th.hits = n_hits;
+            th.misses = n_miss;
+            th.status = status;
+            th.reserved = 0;
+            *reinterpret_cast<melinoe_moe_trace_header *>(p.trace_rec) = th;
+        }
     }
 }
 

@@ -110,6 +110,60 @@ def test_deepseek_shape_with_shared_experts(alpha):
     _run_stack("deepseek", 4, alpha, 12, decode_steps=32, sample_layers=(3,), y_tokens=8)
 
 
+def test_per_layer_budget_end_to_end_makes_fewer_transfers():
+    """Per-layer cache budgets from a recorded trace, end to end on the OLMoE shape: four layers whose
+    routing runs from concentrated to near-uniform decode 96 tokens with 16 slots each while their request
+    traces are recorded on the device (no synchronisation per call); the routing traces go through the
+    miss-proxy evaluator (Definition C.1's hard cache) for every cache size, the library splits the same
+    total of 64 slots over the layers, and a second stack with those sizes decodes the same tokens.  Both
+    runs' request records equal the oracle's, and the budgeted stack makes fewer transfers."""
+    import torch
+    from paper_2602_11192_b200.budget import allocate_slots, miss_curves, read_trace
+    from paper_2602_11192_b200.workload import Stack
+    cfg = gen.config_by_name("olmoe")
+    L, steps, E, k = 4, 96, cfg.n_experts, cfg.top_k
+    alphas = (0.05, 0.3, 3.0, 30.0)
+
+    def run(slots):
+        st = Stack(cfg, 1.0, slots, n_layers=L)
+        st.bias = [np.stack([gen.router_bias(cfg.seed, l, 0, alphas[l], E)]) for l in range(L)]
+        st.set_phase("decode")
+        bufs = []
+        for ls in st.layers:
+            rb = ls.layer.trace_record_bytes(1)
+            b = torch.zeros(steps * rb, dtype=torch.uint8, device="cuda")
+            ls.layer.set_trace(b, b.numel(), 1)
+            bufs.append(b)
+        out = torch.empty((L, 1, cfg.d_model), dtype=torch.int16, device="cuda")
+        xs = [st.hidden_bits("decode", s) for s in range(steps)]
+        xd = [torch.from_numpy(x.view(np.int16)).cuda() for x in xs]
+        for s in range(steps):
+            st.forward_all(xd[s], out, None)
+        torch.cuda.synchronize()
+        recs = [read_trace(b.cpu().numpy(), steps, E, k, 1) for b in bufs]
+        # against the oracle, request by request
+        Cs = [slots] * L if np.isscalar(slots) else list(slots)
+        for l in range(L):
+            cache = oracle.ExpertCache(Cs[l], E)
+            for s in range(steps):
+                idx, _, _ = oracle.route(xs[s][l], st.w_r[l], k, st.bias[l], np.zeros(1, np.int32))
+                assert np.array_equal(recs[l][s]["idx"], idx)
+                assert np.array_equal(recs[l][s]["req"], cache.call(idx)), (l, s)
+        trace = np.stack([np.stack([r["idx"][0] for r in recs[l]]) for l in range(L)])[:, :, None, :].reshape(L, steps, k)
+        misses = [sum(r["misses"] for r in recs[l]) for l in range(L)]
+        st.close()
+        return trace, misses
+
+    trace, uniform = run(16)
+    sizes = list(range(k, 41))
+    _, hard = miss_curves(trace, E, 0.5, sizes)
+    slots = allocate_slots(hard, sizes, 16 * L)
+    assert sum(slots) == 16 * L and min(slots) >= k
+    assert len(set(slots)) > 1                      # layers with different routing get different sizes
+    _, budgeted = run(slots)
+    assert sum(budgeted) < sum(uniform), (slots, budgeted, uniform)
+
+
 def test_repeated_runs_with_heavy_miss_traffic_are_bit_identical():
     """Two cold-start runs of the same OLMoE-shaped steps (near-uniform routing: several transfers
     per layer and token, miss waves, slot reuse inside a call) give the same output bits and the

@@ -221,6 +221,51 @@ def test_a_failed_host_copy_leaves_the_handle_usable():
     P.close()
 
 
+def test_request_trace_records_calls_without_synchronising():
+    """The request trace: 24 calls (decode-sized ones through the fused planner, two larger ones through the
+    general planner) are queued back to back with no synchronisation in between; afterwards the ring holds
+    the last 16 calls' records, each equal to what the oracle says of that call: routing indices, gates,
+    request records in order, hit and miss counts."""
+    import torch
+    from paper_2602_11192_b200.budget import read_trace
+    from paper_2602_11192_b200.runner import current_stream_ptr, to_dev_bf16
+    d, F, E, k, C = 512, 64, 12, 2, 4
+    P = _pair(d, F, E, k, C, seed=87)
+    L = P.gpu.layer
+    max_tok, cap = 8, 16
+    rb = L.trace_record_bytes(max_tok)
+    assert rb == (32 + 16 * E + 8 * max_tok * k + 15) // 16 * 16
+    buf = torch.zeros(cap * rb, dtype=torch.uint8, device="cuda")
+    L.set_trace(buf, buf.numel(), max_tok)
+    Ts = [1, 3, 8, 1, 20, 2, 1, 5] * 3
+    xs = [gen.hidden_states(87, 0, "decode", i, T, d) for i, T in enumerate(Ts)]
+    outs = [torch.empty((T, d), dtype=torch.int16, device="cuda") for T in Ts]
+    xd = [to_dev_bf16(x) for x in xs]
+    s = current_stream_ptr()
+    for x, o, T in zip(xd, outs, Ts):
+        L.forward(s, x, T, o)                       # nothing waits here
+    torch.cuda.synchronize()
+    assert L.trace_count() == len(Ts)
+    recs = read_trace(buf.cpu().numpy(), cap, E, k, max_tok)
+    want = []
+    for x in xs:
+        idx, gate, _ = oracle.route(x, P.w_r, k)
+        want.append((idx, gate, P.cache.call(idx)))
+    for n in range(len(Ts) - cap, len(Ts)):
+        r = recs[n % cap]
+        idx, gate, req = want[n]
+        nt = min(Ts[n], max_tok)
+        assert r["call_no"] == n + 1 and r["n_tokens"] == Ts[n] and r["status"] == 0
+        assert np.array_equal(r["idx"], idx[:nt]) and np.allclose(r["gate"], gate[:nt], rtol=1e-5, atol=1e-7)
+        assert np.array_equal(r["req"], req)
+        assert r["hits"] == int(req[:, 2].sum()) and r["misses"] == len(req) - int(req[:, 2].sum())
+    L.set_trace(None, 0, 0)
+    L.forward(s, xd[0], Ts[0], outs[0])
+    torch.cuda.synchronize()
+    assert L.trace_count() == len(Ts)               # switched off: nothing more is recorded
+    P.close()
+
+
 def test_forward_host_matches_forward_and_is_deterministic():
     import torch
     from paper_2602_11192_b200.runner import current_stream_ptr

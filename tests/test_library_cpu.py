@@ -82,16 +82,16 @@ def test_pack_expert_q4_matches_the_oracle_bit_for_bit(m):
         m.melinoe_moe_pack_expert_q4(256, 40, w[0].ctypes.data, w[1].ctypes.data, w[2].ctypes.data, blob.ctypes.data)
 
 
-def test_budget_allocation_spends_slots_where_they_save_transfers():
-    """Host logic of the per-layer budget: greedy on the marginal transfers saved."""
-    import importlib.util
-    spec = importlib.util.spec_from_file_location("budget_src", os.path.join(ROOT, "paper_2602_11192_b200", "budget.py"))
-    src = open(spec.origin).read()
-    ns = {}
-    # the allocator itself needs neither the library nor a device: run it from its source
-    start = src.index("def allocate_slots")
-    exec("import numpy as np\nfrom typing import List, Sequence\n" + src[start:], ns)
-    alloc = ns["allocate_slots"]
+def test_budget_allocation_spends_slots_where_they_save_transfers(m):
+    """Host logic of the per-layer budget (melinoe_allocate_slots): greedy on the marginal transfers saved.
+    Pure host code: needs the library, no device."""
+    def alloc(hard, sizes, budget):
+        hard = np.ascontiguousarray(hard, dtype=np.int64)
+        out = np.zeros(hard.shape[0], np.int32)
+        rc = m.lib().melinoe_allocate_slots(hard.ctypes.data, hard.shape[0], hard.shape[1], sizes[0], budget, out.ctypes.data)
+        if rc:
+            raise ValueError("status %d" % rc)
+        return out.tolist()
     sizes = [2, 3, 4, 5, 6]
     hard = np.array([[100, 60, 50, 49, 49],      # layer 0: the third slot is worth 40, then little
                      [100, 95, 90, 85, 80],      # layer 1: every slot is worth 5
