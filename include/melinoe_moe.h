@@ -122,15 +122,20 @@ int melinoe_moe_pack_expert(int d_model, int d_ff, const void *w_gate_host, cons
                             const void *w_down_host, void *blob_out_host);
 
 /*
- * 4-bit host store (Section 3.2 keeps the expert weights in 4-bit form; the calibrated HQQ format
+ * 4-bit expert format (Section 3.2 keeps the expert weights in 4-bit form; the calibrated HQQ format
  * of the paper is a third-party method, what is implemented is plain symmetric group
- * quantisation).  A matrix row is cut into groups of 64 consecutive elements; a group's scale is
+ * quantisation).  Every vector of d_model weights that belongs to one hidden unit f -- W_g[f],
+ * W_u[f] and column f of W_d -- is cut into groups of 64 consecutive elements; a group's scale is
  * bf16(max|w| / 7); code = clamp(rint(w / scale), -8, 7) + 8, ties to even; the weight the layer
  * computes with is bf16(scale * (code - 8)).  Blob of one expert, `melinoe_moe_expert_bytes_q4`
- * long (about 1.59 bytes per three weights, 3.76 times smaller than the bf16 blob): for W_g, W_u,
- * W_d in this order the codes [rows][cols / 2] (even column in the low nibble) then the scales
- * [rows][cols / 64] bf16.  Needs d_ff % 64 == 0 (else the size is 0 and packing returns
- * MELINOE_ERR_UNSUPPORTED).  Pure host code.
+ * long (3.76 times smaller than the bf16 blob): for every hidden unit f a unit of
+ * ceil16(3 * d_model / 2 + 3 * (d_model / 64) * 2) bytes holding
+ *     codes W_g[f] | codes W_u[f] | codes W_d[:, f]    d_model / 2 bytes each, even element in the low nibble
+ *     scales W_g[f] | scales W_u[f] | scales W_d[:, f]  d_model / 64 bf16 each
+ * then zero padding to a multiple of 16 bytes (none when d_model % 512 == 0).  Within each code
+ * vector, the 16-byte pieces of every group of eight sit at position (piece xor (f mod 8)).  As in
+ * the bf16 blob, everything f contributes is one contiguous byte range.  Needs d_model % 256 == 0 and
+ * d_ff % 8 == 0 (else the size is 0 and packing returns MELINOE_ERR_UNSUPPORTED).  Pure host code.
  */
 size_t melinoe_moe_expert_bytes_q4(int d_model, int d_ff);
 int melinoe_moe_pack_expert_q4(int d_model, int d_ff, const void *w_gate_host, const void *w_up_host,

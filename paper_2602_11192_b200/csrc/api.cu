@@ -404,12 +404,15 @@ int melinoe_moe_pack_expert(int d, int F, const void *wg_, const void *wu_, cons
     return MELINOE_OK;
 }
 
+// Bytes of one hidden unit's part of a 4-bit blob: three rows of d codes (d / 2 bytes each), three rows of
+// d / 64 bf16 scales, rounded up to 16 bytes (bulk copies move multiples of 16 bytes).
+static size_t q4_unit_bytes(int d) { return ((size_t)3 * (d / 2) + (size_t)3 * (d / 64) * 2 + 15) / 16 * 16; }
+
 size_t melinoe_moe_expert_bytes_q4(int d_model, int d_ff)
 {
-    if (d_model <= 0 || d_ff <= 0 || d_model % 64 != 0 || d_ff % 64 != 0)
+    if (d_model <= 0 || d_ff <= 0 || d_model % 256 != 0 || d_ff % kUnitRows != 0)
         return 0;
-    const size_t n = (size_t)d_model * (size_t)d_ff;
-    return 3 * (n / 2 + n / 32);
+    return (size_t)d_ff * q4_unit_bytes(d_model);
 }
 
 namespace {
@@ -430,30 +433,28 @@ uint16_t host_f32_to_bf16(float f)
     return (uint16_t)(u >> 16);
 }
 
-// One matrix [rows][cols] into its section: codes [rows][cols / 2], then scales [rows][cols / 64].
-void pack_q4_matrix(const uint16_t *w, size_t rows, size_t cols, unsigned char *section)
+// One vector of d values (read at stride `stride`) into d / 2 code bytes and d / 64 scales: groups of 64
+// consecutive values, scale = bf16(max|w| / 7), code = clamp(rint(w / scale), -8, 7) + 8, ties to even.  The
+// 16-byte pieces of the codes (32 codes each) go to position (piece xor x) within every group of 8 pieces.
+void pack_q4_vector(const uint16_t *w, size_t stride, int d, int x, unsigned char *codes, uint16_t *scales)
 {
-    unsigned char *codes = section;
-    uint16_t *scales = reinterpret_cast<uint16_t *>(section + rows * cols / 2);
-    for (size_t r = 0; r < rows; ++r) {
-        for (size_t g = 0; g < cols / 64; ++g) {
-            const uint16_t *src = w + r * cols + g * 64;
-            float amax = 0.0f;
-            for (int j = 0; j < 64; ++j)
-                amax = std::fmax(amax, std::fabs(host_bf16_to_f32(src[j])));
-            const uint16_t sb = host_f32_to_bf16(amax / 7.0f);
-            const float sc = host_bf16_to_f32(sb);
-            scales[r * (cols / 64) + g] = sb;
-            unsigned char *dst = codes + (r * cols + g * 64) / 2;
-            for (int j = 0; j < 64; j += 2) {
-                int q[2] = {0, 0};
-                for (int h2 = 0; h2 < 2; ++h2)
-                    if (sc > 0.0f) {
-                        const float t = std::nearbyint(host_bf16_to_f32(src[j + h2]) / sc);   // ties to even
-                        q[h2] = (int)std::fmin(7.0f, std::fmax(-8.0f, t));
-                    }
-                dst[j / 2] = (unsigned char)((q[0] + 8) | ((q[1] + 8) << 4));
-            }
+    for (int g = 0; g < d / 64; ++g) {
+        float amax = 0.0f;
+        for (int j = 0; j < 64; ++j)
+            amax = std::fmax(amax, std::fabs(host_bf16_to_f32(w[(size_t)(g * 64 + j) * stride])));
+        const uint16_t sb = host_f32_to_bf16(amax / 7.0f);
+        const float sc = host_bf16_to_f32(sb);
+        scales[g] = sb;
+        for (int j = 0; j < 64; j += 2) {
+            int q[2] = {0, 0};
+            for (int h2 = 0; h2 < 2; ++h2)
+                if (sc > 0.0f) {
+                    const float t = std::nearbyint(host_bf16_to_f32(w[(size_t)(g * 64 + j + h2) * stride]) / sc);   // ties to even
+                    q[h2] = (int)std::fmin(7.0f, std::fmax(-8.0f, t));
+                }
+            const int byte = (g * 64 + j) / 2, piece = byte / 16;
+            const int ppiece = (piece & ~7) | ((piece ^ x) & 7);
+            codes[ppiece * 16 + byte % 16] = (unsigned char)((q[0] + 8) | ((q[1] + 8) << 4));
         }
     }
 }
@@ -466,11 +467,18 @@ int melinoe_moe_pack_expert_q4(int d, int F, const void *wg_, const void *wu_, c
         return MELINOE_ERR_INVALID;
     if (melinoe_moe_expert_bytes_q4(d, F) == 0)
         return MELINOE_ERR_UNSUPPORTED;
-    const size_t n = (size_t)d * F, sec = n / 2 + n / 32;
+    const uint16_t *wg = static_cast<const uint16_t *>(wg_), *wu = static_cast<const uint16_t *>(wu_);
+    const uint16_t *wd = static_cast<const uint16_t *>(wd_);
     unsigned char *blob = static_cast<unsigned char *>(blob_);
-    pack_q4_matrix(static_cast<const uint16_t *>(wg_), (size_t)F, (size_t)d, blob);
-    pack_q4_matrix(static_cast<const uint16_t *>(wu_), (size_t)F, (size_t)d, blob + sec);
-    pack_q4_matrix(static_cast<const uint16_t *>(wd_), (size_t)d, (size_t)F, blob + 2 * sec);
+    const size_t ub = q4_unit_bytes(d);
+    for (int f = 0; f < F; ++f) {
+        unsigned char *u = blob + (size_t)f * ub;
+        std::memset(u, 0, ub);
+        uint16_t *sc = reinterpret_cast<uint16_t *>(u + 3 * (size_t)(d / 2));
+        pack_q4_vector(wg + (size_t)f * d, 1, d, f & 7, u, sc);
+        pack_q4_vector(wu + (size_t)f * d, 1, d, f & 7, u + d / 2, sc + d / 64);
+        pack_q4_vector(wd + f, (size_t)F, d, f & 7, u + 2 * (size_t)(d / 2), sc + 2 * (d / 64));    // column f of W_d
+    }
     return MELINOE_OK;
 }
 

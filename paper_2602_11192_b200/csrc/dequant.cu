@@ -1,12 +1,11 @@
 // Expansion of a 4-bit group-quantised expert into the bf16 blob layout the FFN kernels read.
 //
-// Host store layout of one 4-bit expert (Section 3.2 keeps the experts in 4-bit form; what is
-// stored here is plain symmetric group quantisation): for each of W_g [F][d], W_u [F][d],
-// W_d [d][F], in this order, the codes [rows][cols / 2] (one byte = two columns, the even column
-// in the low nibble) followed by the scales [rows][cols / 64] (bf16).  The weight that the layer
-// computes with is bf16( scale * (code - 8) ): the product is exact in fp32 and is rounded to
-// nearest even.  The output is the bf16 blob of melinoe_moe_pack_expert: per hidden unit f the rows
-// W_g[f] | W_u[f] | W_d[:, f], the 16-byte pieces of every 128-byte group at (piece xor (f mod 8)).
+// Both blobs are organised per hidden unit f (see melinoe_moe_pack_expert / _pack_expert_q4): the
+// 4-bit unit holds the codes of W_g[f], W_u[f], W_d[:, f] (d / 2 bytes each, the even element in the
+// low nibble, the 16-byte pieces of every 128-byte group at (piece xor (f mod 8))), then their
+// scales (d / 64 bf16 each).  The weight that the layer computes with is bf16(scale * (code - 8)):
+// the product is exact in fp32 and is rounded to nearest even.  The bf16 unit holds the three
+// vectors of d bf16 values with the same kind of permutation on its own 16-byte pieces.
 #include "kernels.cuh"
 
 namespace melinoe {
@@ -20,63 +19,37 @@ __device__ __forceinline__ uint32_t bf16_rne_bits(float v)
     return u >> 16;
 }
 
-// A block expands tiles of 64 x 64 weights.  W_g / W_u: 64 rows f x 64 columns, written straight
-// through; W_d: 64 rows c x 64 columns f, transposed through shared memory so that the 64 values
-// c of one f leave as one 128-byte row piece.
-__global__ void __launch_bounds__(256) dequant_q4_kernel(const unsigned char *__restrict__ q, uint16_t *__restrict__ out, int d, int F)
+// One thread expands one 16-byte piece of codes (32 weights) into four 16-byte pieces of bf16.
+__global__ void __launch_bounds__(256) dequant_q4_kernel(const unsigned char *__restrict__ q, uint16_t *__restrict__ out, int d, int F,
+                                                         int unit_bytes)
 {
-    __shared__ uint16_t s_t[64][66];
-    const size_t n = (size_t)d * F;
-    const size_t sec = n / 2 + n / 32;                 // one matrix's section of the 4-bit blob
-    const int tiles_gu = (F / 64) * (d / 64), tiles_d = (d / 64) * (F / 64);
-    const int total = 2 * tiles_gu + tiles_d;
-    const int tid = threadIdx.x;
-    const int r = tid >> 2, part = tid & 3;            // source row of the tile, 16 of its 64 columns
-    for (int t = blockIdx.x; t < total; t += gridDim.x) {
-        const int m = t < tiles_gu ? 0 : (t < 2 * tiles_gu ? 1 : 2);
-        const int tt = t - m * tiles_gu;
-        const int cols = m < 2 ? d : F;
-        const int tr = tt / (cols / 64), tc = tt % (cols / 64);      // tile of source rows, of source columns
-        const unsigned char *codes = q + m * sec;
-        const uint16_t *scales = reinterpret_cast<const uint16_t *>(q + m * sec + n / 2);
-        const size_t row = (size_t)tr * 64 + r;
-        const float sc = __uint_as_float((uint32_t)scales[row * (cols / 64) + tc] << 16);
-        const uint2 c8 = *reinterpret_cast<const uint2 *>(codes + (row * cols + (size_t)tc * 64 + part * 16) / 2);
-        uint32_t o[8];
+    const int pieces = d / 32;                        // code pieces of one vector
+    const size_t total = (size_t)F * 3 * pieces;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const int f = (int)(i / (3 * pieces)), rest = (int)(i % (3 * pieces));
+        const int m = rest / pieces, piece = rest % pieces;            // vector (g, u, d) and logical code piece
+        const unsigned char *unit = q + (size_t)f * unit_bytes;
+        const int x = f & 7;
+        const int ppiece = (piece & ~7) | ((piece ^ x) & 7);
+        const uint4 c = *reinterpret_cast<const uint4 *>(unit + (size_t)m * (d / 2) + (size_t)ppiece * 16);
+        const uint16_t *scales = reinterpret_cast<const uint16_t *>(unit + 3 * (size_t)(d / 2)) + m * (d / 64);
+        const float sc = __uint_as_float((uint32_t)scales[piece / 2] << 16);
+        const uint32_t words[4] = {c.x, c.y, c.z, c.w};
+        uint16_t *row = out + ((size_t)f * 3 + m) * d;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const uint32_t word = i < 4 ? c8.x : c8.y;
-            const uint32_t byte = (word >> (8 * (i & 3))) & 0xffu;
-            const float lo = __fmul_rn(sc, (float)((int)(byte & 15u) - 8));
-            const float hi = __fmul_rn(sc, (float)((int)(byte >> 4) - 8));
-            o[i] = bf16_rne_bits(lo) | (bf16_rne_bits(hi) << 16);
-        }
-        if (m < 2) {
-            // row f = row, columns tc * 64 + part * 16 ..: two 16-byte pieces of the 128-byte group tc
-            const int f = (int)row;
-            uint16_t *dst = out + ((size_t)f * 3 + m) * d + (size_t)tc * 64;
-            const int p0 = (part * 2) ^ (f & 7), p1 = (part * 2 + 1) ^ (f & 7);
-            *reinterpret_cast<uint4 *>(dst + p0 * 8) = make_uint4(o[0], o[1], o[2], o[3]);
-            *reinterpret_cast<uint4 *>(dst + p1 * 8) = make_uint4(o[4], o[5], o[6], o[7]);
-        } else {
-            // source row c = row, source columns f = tc * 64 + part * 16 ..: transpose
-            __syncthreads();
+        for (int w = 0; w < 4; ++w) {
+            uint32_t o[4];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                s_t[part * 16 + 2 * i][r] = (uint16_t)(o[i] & 0xffffu);
-                s_t[part * 16 + 2 * i + 1][r] = (uint16_t)(o[i] >> 16);
+            for (int b = 0; b < 4; ++b) {
+                const uint32_t byte = (words[w] >> (8 * b)) & 0xffu;
+                const float lo = __fmul_rn(sc, (float)((int)(byte & 15u) - 8));
+                const float hi = __fmul_rn(sc, (float)((int)(byte >> 4) - 8));
+                o[b] = bf16_rne_bits(lo) | (bf16_rne_bits(hi) << 16);
             }
-            __syncthreads();
-            // thread: f = tc * 64 + r, 16 of the 64 values c = tr * 64 + part * 16 ..
-            const int f = tc * 64 + r;
-            uint32_t w[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i)
-                w[i] = (uint32_t)s_t[r][part * 16 + 2 * i] | ((uint32_t)s_t[r][part * 16 + 2 * i + 1] << 16);
-            uint16_t *dst = out + ((size_t)f * 3 + 2) * d + (size_t)tr * 64;
-            const int p0 = (part * 2) ^ (f & 7), p1 = (part * 2 + 1) ^ (f & 7);
-            *reinterpret_cast<uint4 *>(dst + p0 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
-            *reinterpret_cast<uint4 *>(dst + p1 * 8) = make_uint4(w[4], w[5], w[6], w[7]);
+            // these 8 weights are elements piece * 32 + w * 8 .. of the vector: bf16 piece 4 * piece + w
+            const int bp = 4 * piece + w;
+            const int pbp = (bp & ~7) | ((bp ^ x) & 7);
+            *reinterpret_cast<uint4 *>(row + (size_t)pbp * 8) = make_uint4(o[0], o[1], o[2], o[3]);
         }
     }
 }
@@ -103,7 +76,9 @@ cudaError_t launch_stage_in(cudaStream_t stream, const void *src_mapped, void *d
 
 cudaError_t launch_dequant_q4(cudaStream_t stream, const void *q4_blob, void *slot, int d, int F, int n_sms)
 {
-    dequant_q4_kernel<<<n_sms * 8, 256, 0, stream>>>(static_cast<const unsigned char *>(q4_blob), static_cast<uint16_t *>(slot), d, F);
+    const int unit_bytes = (3 * (d / 2) + 3 * (d / 64) * 2 + 15) / 16 * 16;
+    dequant_q4_kernel<<<n_sms * 8, 256, 0, stream>>>(static_cast<const unsigned char *>(q4_blob), static_cast<uint16_t *>(slot), d, F,
+                                                      unit_bytes);
     count_launch();
     return cudaGetLastError();
 }

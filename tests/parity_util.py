@@ -27,6 +27,14 @@ def make_weights(seed, layer, E, d, F, n_shared=0):
     return [gen.expert_weights(seed, layer, e, d, F) for e in range(E + n_shared)]
 
 
+def _q4_roundtrip(w):
+    """The weights a 4-bit store defines: W_g and W_u quantised along their rows, W_d along its columns
+    (the quantisation groups follow the d_model axis in all three)."""
+    wg, wu, wd = w
+    q = lambda m: oracle.dequantize_q4(*oracle.quantize_q4(np.ascontiguousarray(m)))
+    return q(wg), q(wu), np.ascontiguousarray(q(wd.T).T)
+
+
 def rel_err_per_token(y_gpu_bits: np.ndarray, y_ref: np.ndarray) -> np.ndarray:
     yg = gen.bf16_bits_to_f32(y_gpu_bits).astype(np.float64)
     num = np.linalg.norm(yg - y_ref, axis=1)
@@ -58,7 +66,7 @@ class Pair:
             # format defines as the layer's weights (its own quantise + dequantise)
             assert n_shared == 0
             self.gpu.set_experts_q4(self.weights)
-            self.weights = [tuple(oracle.dequantize_q4(*oracle.quantize_q4(m)) for m in w) for w in self.weights]
+            self.weights = [_q4_roundtrip(w) for w in self.weights]
             self.bytes_per_miss = melinoe_moe_expert_bytes_q4(d, F)
         else:
             self.gpu.set_experts(self.weights[:E], self.weights[E:])

@@ -59,27 +59,38 @@ def test_pack_expert_layout(m):
 
 
 def test_pack_expert_q4_matches_the_oracle_bit_for_bit(m):
-    """The library's host-side quantiser against the oracle's (independent code, same definition)."""
+    """The library's host-side quantiser against the oracle's (independent code, same definition).  The
+    blob is per hidden unit f: codes of W_g[f], W_u[f], W_d[:, f] (the quantisation groups of W_d run down
+    its columns), then the three scale vectors; 16-byte code pieces at (piece xor (f mod 8)) within every
+    eight."""
     import oracle
-    d, F = 256, 128
-    rs = np.random.default_rng(3)
-    w = [gen.f32_to_bf16_bits(rs.normal(0.0, 0.02, shp).astype(np.float32)) for shp in ((F, d), (F, d), (d, F))]
-    w[0][0, :64] = 0                                            # an all-zero group
-    w[1][1, :8] = gen.f32_to_bf16_bits(np.array([0.875, -0.875, 0.0625, 0.1875, -0.0625, -0.1875, 0.125, 0.0], np.float32))
-    w[1][1, 8:64] = 0                                           # ties exactly between two codes
-    qb = m.melinoe_moe_expert_bytes_q4(d, F)
-    assert qb == 3 * (d * F // 2 + d * F // 32)
-    assert m.melinoe_moe_expert_bytes_q4(256, 40) == 0
-    blob = np.full(qb, 0xAB, np.uint8)
-    m.melinoe_moe_pack_expert_q4(d, F, w[0].ctypes.data, w[1].ctypes.data, w[2].ctypes.data, blob.ctypes.data)
-    sec = d * F // 2 + d * F // 32
-    for i, mat in enumerate(w):
-        codes, scales = oracle.quantize_q4(mat)
-        part = blob[i * sec:(i + 1) * sec]
-        assert np.array_equal(part[:d * F // 2], codes.reshape(-1))
-        assert np.array_equal(part[d * F // 2:].view(np.uint16), scales.reshape(-1))
+    for d, F in ((256, 24), (512, 64)):
+        rs = np.random.default_rng(3)
+        w = [gen.f32_to_bf16_bits(rs.normal(0.0, 0.02, shp).astype(np.float32)) for shp in ((F, d), (F, d), (d, F))]
+        w[0][0, :64] = 0                                            # an all-zero group
+        w[1][1, :8] = gen.f32_to_bf16_bits(np.array([0.875, -0.875, 0.0625, 0.1875, -0.0625, -0.1875, 0.125, 0.0], np.float32))
+        w[1][1, 8:64] = 0                                           # ties exactly between two codes
+        unit = (3 * (d // 2) + 3 * (d // 64) * 2 + 15) // 16 * 16
+        qb = m.melinoe_moe_expert_bytes_q4(d, F)
+        assert qb == F * unit
+        blob = np.full(qb, 0xAB, np.uint8)
+        m.melinoe_moe_pack_expert_q4(d, F, w[0].ctypes.data, w[1].ctypes.data, w[2].ctypes.data, blob.ctypes.data)
+        units = blob.reshape(F, unit)
+        want = [oracle.quantize_q4(w[0]), oracle.quantize_q4(w[1]), oracle.quantize_q4(np.ascontiguousarray(w[2].T))]
+        for f in range(F):
+            for i, (codes, scales) in enumerate(want):
+                stored = units[f, i * (d // 2):(i + 1) * (d // 2)].reshape(-1, 16)
+                plain = np.empty_like(stored)
+                for piece in range(stored.shape[0]):
+                    plain[piece] = stored[(piece & ~7) | ((piece ^ f) & 7)]
+                assert np.array_equal(plain.reshape(-1), codes[f]), (d, f, i)
+                sc = units[f, 3 * (d // 2) + i * (d // 32):3 * (d // 2) + (i + 1) * (d // 32)].view(np.uint16)
+                assert np.array_equal(sc, scales[f]), (d, f, i)
+            assert not units[f, 3 * (d // 2) + 3 * (d // 32):].any()      # padding is zeroed
+    assert m.melinoe_moe_expert_bytes_q4(256, 40) == 40 * 416 and m.melinoe_moe_expert_bytes_q4(256, 36) == 0
+    assert m.melinoe_moe_expert_bytes_q4(320, 64) == 0
     with pytest.raises(m.MelinoeError):
-        m.melinoe_moe_pack_expert_q4(256, 40, w[0].ctypes.data, w[1].ctypes.data, w[2].ctypes.data, blob.ctypes.data)
+        m.melinoe_moe_pack_expert_q4(256, 36, w[0].ctypes.data, w[1].ctypes.data, w[2].ctypes.data, blob.ctypes.data)
 
 
 def test_budget_allocation_spends_slots_where_they_save_transfers(m):
