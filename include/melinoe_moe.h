@@ -98,6 +98,19 @@ typedef struct melinoe_moe_trace_header {
 int melinoe_moe_create(int d_model, int d_ff, int n_experts, int top_k, int cache_slots,
                        melinoe_moe_t **out);
 
+/*
+ * Same layer with 4-bit cache slots (Section 3.2 and Appendix D.5: 4-bit experts let the same memory hold
+ * about 3.76 times as many of them): a slot is melinoe_moe_expert_bytes_q4() long, the store is registered
+ * with melinoe_moe_register_host_experts_q4 and a miss is a plain copy of the 4-bit blob; the compute
+ * kernel expands the codes in registers on their way into the tensor-core fragments, so HBM and the
+ * host link only ever carry 4-bit data.  The layer computes with exactly the weights the format defines
+ * (see melinoe_moe_pack_expert_q4).  Shared experts, if any, are registered as 4-bit blobs too.  Calls of
+ * every size run the decode kernel, 8 tokens per launch (there is no 4-bit grouped GEMM).  Needs
+ * d_model % 512 == 0 on top of the limits above.
+ */
+int melinoe_moe_create_q4(int d_model, int d_ff, int n_experts, int top_k, int cache_slots,
+                          melinoe_moe_t **out);
+
 /* Waits for the handle's outstanding transfers and device work, then frees everything the
  * library allocated.  Caller memory (router, experts, bias) is untouched. */
 int melinoe_moe_destroy(melinoe_moe_t *h);
@@ -159,10 +172,12 @@ int melinoe_moe_set_router(melinoe_moe_t *h, const void *w_router_dev);
  * cudaMemcpyAsync issued by the host.
  */
 int melinoe_moe_register_host_experts(melinoe_moe_t *h, const void *const *expert_host_ptrs,
-                                      size_t bytes_per_expert);
+                                      size_t bytes_per_expert);   /* UNSUPPORTED on a handle with 4-bit slots */
 
 /*
- * Same registration for a store of 4-bit blobs (melinoe_moe_pack_expert_q4): a miss then moves the
+ * Same registration for a store of 4-bit blobs (melinoe_moe_pack_expert_q4).  On a handle with 4-bit slots
+ * (melinoe_moe_create_q4) this is the one way to register the store, and everything said above holds.
+ * On a handle with bf16 slots a miss then moves the
  * 4-bit blob over the host link (3.76 times fewer bytes, which is what a miss costs, Eq. 4) and a
  * kernel expands it into the bf16 slot behind the copy, so the cache slots and the compute kernels
  * are the same as with a bf16 store and the layer computes with exactly the weights the format
@@ -174,8 +189,8 @@ int melinoe_moe_register_host_experts(melinoe_moe_t *h, const void *const *exper
 int melinoe_moe_register_host_experts_q4(melinoe_moe_t *h, const void *const *expert_host_ptrs,
                                          size_t bytes_per_expert);
 
-/* Always-resident shared experts (not in the paper; DeepSeekMoE-style stacks): packed blobs
- * in DEVICE memory, applied to every token with gate 1, never cached, never counted in
+/* Always-resident shared experts (not in the paper; DeepSeekMoE-style stacks): blobs packed in
+ * the format of the handle's slots, in DEVICE memory, applied to every token with gate 1, never cached, never counted in
  * hits or misses.  n_shared <= 8.  Borrowed. */
 int melinoe_moe_register_shared_experts(melinoe_moe_t *h, int n_shared,
                                         const void *const *expert_dev_ptrs);

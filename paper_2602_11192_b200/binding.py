@@ -15,7 +15,7 @@ __all__ = [
 HERE = os.path.dirname(os.path.abspath(__file__))
 
 EXPORTED_SYMBOLS = [
-    "melinoe_moe_create", "melinoe_moe_destroy", "melinoe_moe_expert_bytes", "melinoe_moe_pack_expert",
+    "melinoe_moe_create", "melinoe_moe_create_q4", "melinoe_moe_destroy", "melinoe_moe_expert_bytes", "melinoe_moe_pack_expert",
     "melinoe_moe_set_router", "melinoe_moe_register_host_experts", "melinoe_moe_register_shared_experts",
     "melinoe_moe_set_router_bias", "melinoe_moe_reserve", "melinoe_moe_forward", "melinoe_moe_forward_host",
     "melinoe_moe_reset_cache", "melinoe_moe_preload", "melinoe_moe_last_routing", "melinoe_moe_last_logits",
@@ -68,6 +68,7 @@ def lib():
     L = C.CDLL(path)
     vp, i32, sz = C.c_void_p, C.c_int, C.c_size_t
     L.melinoe_moe_create.argtypes = [i32, i32, i32, i32, i32, C.POINTER(vp)]
+    L.melinoe_moe_create_q4.argtypes = [i32, i32, i32, i32, i32, C.POINTER(vp)]
     L.melinoe_moe_destroy.argtypes = [vp]
     L.melinoe_moe_expert_bytes.argtypes = [i32, i32]
     L.melinoe_moe_expert_bytes.restype = sz
@@ -181,15 +182,18 @@ def _ptr(t) -> Optional[int]:
 class MoELayer:
     """One handle (= one MoE layer).  Methods mirror the C entry points one to one."""
 
-    def __init__(self, d_model: int, d_ff: int, n_experts: int, top_k: int, cache_slots: int):
+    def __init__(self, d_model: int, d_ff: int, n_experts: int, top_k: int, cache_slots: int, slots: str = "bf16"):
         self.d_model, self.d_ff, self.n_experts, self.top_k, self.cache_slots = (
             int(d_model), int(d_ff), int(n_experts), int(top_k), int(cache_slots))
         self._h = C.c_void_p()
         self._keep = {}
-        rc = lib().melinoe_moe_create(d_model, d_ff, n_experts, top_k, cache_slots, C.byref(self._h))
+        assert slots in ("bf16", "q4")
+        self.slots = slots
+        create = lib().melinoe_moe_create if slots == "bf16" else lib().melinoe_moe_create_q4
+        rc = create(d_model, d_ff, n_experts, top_k, cache_slots, C.byref(self._h))
         if rc:
             self._h = C.c_void_p()
-            raise MelinoeError(rc, "melinoe_moe_create")
+            raise MelinoeError(rc, "melinoe_moe_create" if slots == "bf16" else "melinoe_moe_create_q4")
 
     # -- lifetime
     def destroy(self) -> None:

@@ -131,6 +131,7 @@ struct Scratch {
 struct melinoe_moe {
     int d = 0, F = 0, E = 0, k = 0, C = 0, device = 0, n_sms = 0;
     size_t expert_bytes = 0, slot_stride = 0;
+    int fmt = 0;                           // what the slots hold: 0 = bf16 blobs, 1 = 4-bit blobs
     DecLaunchCfg cfg{};
 
     // device memory owned by the handle
@@ -482,14 +483,20 @@ int melinoe_moe_pack_expert_q4(int d, int F, const void *wg_, const void *wu_, c
     return MELINOE_OK;
 }
 
-int melinoe_moe_create(int d, int F, int E, int k, int C, melinoe_moe_t **out)
+static int create_layer(int d, int F, int E, int k, int C, int fmt, melinoe_moe_t **out);
+
+int melinoe_moe_create(int d, int F, int E, int k, int C, melinoe_moe_t **out) { return create_layer(d, F, E, k, C, 0, out); }
+
+int melinoe_moe_create_q4(int d, int F, int E, int k, int C, melinoe_moe_t **out) { return create_layer(d, F, E, k, C, 1, out); }
+
+static int create_layer(int d, int F, int E, int k, int C, int fmt, melinoe_moe_t **out)
 {
     if (!out)
         return MELINOE_ERR_INVALID;
     *out = nullptr;
     if (d <= 0 || F <= 0 || E <= 0 || k <= 0 || C <= 0 || k > E || C < k || C > E)
         return MELINOE_ERR_INVALID;
-    if (!ffn_decode_supported(d, F) || E > kMaxExperts || k > 32)
+    if (!(fmt == 0 ? ffn_decode_supported(d, F) : ffn_decode_supported_q4(d, F)) || E > kMaxExperts || k > 32)
         return MELINOE_ERR_UNSUPPORTED;
     {
         int dev = 0;
@@ -507,7 +514,8 @@ int melinoe_moe_create(int d, int F, int E, int k, int C, melinoe_moe_t **out)
     h->E = E;
     h->k = k;
     h->C = C;
-    h->expert_bytes = melinoe_moe_expert_bytes(d, F);
+    h->fmt = fmt;
+    h->expert_bytes = fmt == 0 ? melinoe_moe_expert_bytes(d, F) : melinoe_moe_expert_bytes_q4(d, F);
     h->slot_stride = (h->expert_bytes + 1023) / 1024 * 1024;
     h->host_experts.assign(E, nullptr);
     int rc = MELINOE_OK;
@@ -565,7 +573,7 @@ int melinoe_moe_create(int d, int F, int E, int k, int C, melinoe_moe_t **out)
     // grouped GEMM for calls of many tokens: the slots are contiguous, so one tensor map per view
     // (W_g rows, W_u rows, W_d^T rows) covers every slot
     std::memset(h->maps_host, 0, sizeof(h->maps_host));
-    if (ffn_gemm_supported(d, F) && h->slot_stride == h->expert_bytes && ffn_gemm_configure() == cudaSuccess) {
+    if (fmt == 0 && ffn_gemm_supported(d, F) && h->slot_stride == h->expert_bytes && ffn_gemm_configure() == cudaSuccess) {
         CR(cudaMalloc(&h->maps_dev, sizeof(h->maps_host)));
         if (encode_weight_maps(&h->maps_host[kMapSlotsG], h->slots, d, (uint64_t)C * F)) {
             CR(cudaMemcpy(h->maps_dev, h->maps_host, sizeof(h->maps_host), cudaMemcpyHostToDevice));
@@ -652,9 +660,22 @@ int melinoe_moe_set_router(melinoe_moe_t *h, const void *w_router_dev)
     return MELINOE_OK;
 }
 
+static int register_store(melinoe_moe *h, const void *const *ptrs, size_t bytes_per_expert);
+
 int melinoe_moe_register_host_experts(melinoe_moe_t *h, const void *const *ptrs, size_t bytes_per_expert)
 {
-    if (!h || !ptrs || bytes_per_expert != h->expert_bytes)
+    if (!h || !ptrs)
+        return MELINOE_ERR_INVALID;
+    if (h->fmt != 0)
+        return MELINOE_ERR_UNSUPPORTED;   // 4-bit slots are filled from a 4-bit store
+    return register_store(h, ptrs, bytes_per_expert);
+}
+
+// The store holds blobs of the slots' own format: a miss is a plain copy, by the device where it can
+// address the store.
+static int register_store(melinoe_moe *h, const void *const *ptrs, size_t bytes_per_expert)
+{
+    if (bytes_per_expert != h->expert_bytes)
         return MELINOE_ERR_INVALID;
     for (int e = 0; e < h->E; ++e) {
         if (!ptrs[e] || !aligned16(ptrs[e]))
@@ -699,6 +720,8 @@ int melinoe_moe_register_host_experts_q4(melinoe_moe_t *h, const void *const *pt
         return MELINOE_ERR_UNSUPPORTED;
     if (bytes_per_expert != qb)
         return MELINOE_ERR_INVALID;
+    if (h->fmt == 1)
+        return register_store(h, ptrs, bytes_per_expert);
     for (int e = 0; e < h->E; ++e) {
         cudaPointerAttributes a;
         if (!ptrs[e] || !aligned16(ptrs[e]) || cudaPointerGetAttributes(&a, ptrs[e]) != cudaSuccess ||
@@ -798,7 +821,7 @@ int launch_decode(melinoe_moe *h, cudaStream_t s, const Scratch &sc, const void 
 {
     const int tokens = T - chunk * kTokPerVr < kTokPerVr ? T - chunk * kTokPerVr : kTokPerVr;
     DecGeometry geo;
-    if (ffn_decode_geometry(h->cfg, h->d, h->F, tokens, 0, &geo) != cudaSuccess)
+    if (ffn_decode_geometry(h->cfg, h->d, h->F, tokens, h->fmt, &geo) != cudaSuccess)
         return MELINOE_ERR_UNSUPPORTED;
     DecParams dp;
     dp.plan = h->plan;
@@ -823,7 +846,7 @@ int launch_decode(melinoe_moe *h, cudaStream_t s, const Scratch &sc, const void 
     dp.n_chunks = (T + kTokPerVr - 1) / kTokPerVr;
     dp.write_back = 1;
     dp.wait_prior = first_of_call ? 0 : 1;
-    dp.fmt = 0;
+    dp.fmt = h->fmt;
     CU_TRY(launch_ffn_decode(s, h->cfg, geo, dp));
     return MELINOE_OK;
 }
@@ -1333,7 +1356,7 @@ int melinoe_moe_preload(melinoe_moe_t *h, const int32_t *ids, int n)
         fp.slots = h->slots;
         fp.slot_stride = h->slot_stride;
         fp.rows = h->F;
-        fp.row_bytes = 6 * h->d;
+        fp.row_bytes = (int)(h->expert_bytes / (size_t)h->F);     // one hidden unit of the slots' format
         fp.rows_per_piece = 49152 / fp.row_bytes > 0 ? 49152 / fp.row_bytes : 1;
         fp.piece_bytes = fp.rows_per_piece * fp.row_bytes;
         fp.err = h->err_word;

@@ -141,6 +141,33 @@ __device__ __forceinline__ uint32_t lds32(uint32_t addr)
     return v;
 }
 
+__device__ __forceinline__ uint4 lds128(uint32_t addr)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds16(uint32_t addr)
+{
+    uint16_t v;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(addr));
+    return v;
+}
+
+// Eight 4-bit codes (one 32-bit word: element j in nibble j) into bf16 weights, as four registers
+// P[j] = (element j, element j + 4).  A nibble n placed in the mantissa of 0x4300 is the bf16 number
+// 128 + n; minus 136 is the integer n - 8, exactly; times the group's scale, rounded once to nearest
+// even, is the weight the format defines.  ss = the scale in both halves.
+__device__ __forceinline__ void dequant8(uint32_t w, uint32_t ss, uint32_t (&P)[4])
+{
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        uint32_t t = ((w >> (4 * j)) & 0x000f000fu) | 0x43004300u;
+        asm("sub.rn.bf16x2 %0, %0, %1;" : "+r"(t) : "r"(0x43084308u));
+        asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(P[j]) : "r"(t), "r"(ss));
+    }
+}
+
 __device__ __forceinline__ uint32_t bf16_rne(float v)
 {
     uint32_t u = __float_as_uint(v);
@@ -174,8 +201,212 @@ constexpr int NW = 16;                           // consumer warps
 constexpr int kThreads = (NW + 1) * 32;          // + the producer warp
 constexpr int kBufPitch = 130;                   // floats between the warps' partial tiles (keeps the column sums conflict-free)
 
-// MT_: k-steps of the gate/up phase and m-tiles of the down phase per warp (d / 256), 0 = taken from d at run time.
+// ---------------------------------------------------------------------------------------------------
+// The consumer warps' work on 4-bit blobs.  One hidden unit f is a unit of geo.row_bytes bytes: the
+// codes of W_g[f], W_u[f], W_d[:, f] (d / 2 bytes each) and their scales (one bf16 per 64 elements).
+// A 32-bit word of codes is eight consecutive elements and expands into four registers that pair
+// element j with element j + 4 (dequant8).  A tensor-core operand register holds two neighbours
+// along the contraction, and a sum does not care in which order its terms are met, so:
+//   gate/up   the contraction runs over the columns: a thread takes one word of its W_g row and one of
+//             its W_u row (columns c .. c + 7) and feeds two products, the k-slots being columns
+//             (c, c + 4, c + 1, c + 5) and (c + 2, c + 6, c + 3, c + 7); the hidden state was staged
+//             in the same pairing, so one 16-byte load is the matching token operand of both.  The
+//             warps split the columns in steps of 32.
+//   down      the contraction runs over f, and the two halves of a register are two COLUMNS of one f.
+//             They are made two k-slots of that f, and the token operand carries h[f][t] in the first
+//             of them for the output columns n = 0..3 (tokens 0..3) and in the second for n = 4..7
+//             (again tokens 0..3): the product's left half is column j of every row of output, its right
+//             half column j + 4.  One product so covers 8 hidden units x 32 output columns x 4 tokens;
+//             tokens 4..7 take a second product.  The warps split the columns in steps of 32.
+constexpr int kMaxWs = 8;                        // 32-column steps per warp (d / 512)
+
 template <int MT_>
+__device__ __forceinline__ void consume_q4(const DecParams &p, const DecGeometry &geo, const SReq *s_req, const float *s_gate,
+                                           float *s_sums, float *buf, uint32_t ring_s, uint32_t xs_s, uint32_t full0,
+                                           uint32_t empty0, volatile int *abort_flag, long long q_lo, long long q_hi,
+                                           unsigned long long *trace)
+{
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, tig = lane & 3;
+    const int d = p.d, F = p.F;
+    const int TR = geo.tile_rows, S = geo.n_stages, RB = geo.row_bytes, STAGE = geo.stage_bytes, XP = geo.x_pitch, Tc = geo.tokens;
+    const int WS = MT_ > 0 ? MT_ / 2 : d / (32 * NW);
+    float acc[kMaxWs][2][4];
+#pragma unroll
+    for (int i = 0; i < kMaxWs; ++i)
+#pragma unroll
+        for (int j = 0; j < 2; ++j)
+            acc[i][j][0] = acc[i][j][1] = acc[i][j][2] = acc[i][j][3] = 0.f;
+    const bool has_tok = g < Tc, two = Tc > 4;
+    const uint32_t xrow = xs_s + g * XP + (warp * WS * 32 + tig * 8) * 2;
+    const uint32_t sc_off = 3 * (uint32_t)(d / 2), sc_len = (uint32_t)(d / 32);     // scales: offset in the unit, bytes per vector
+    const int t0 = g & 3, sh = g < 4 ? 0 : 16;
+    uint32_t n = 0;
+    long long q = q_lo;
+    int a = (int)(q / F), f0 = (int)(q % F);
+    bool first = true;
+    while (q < q_hi) {
+        const int m = (int)min((long long)min(TR, F - f0), q_hi - q);
+        const uint32_t st = n % (uint32_t)S;
+        const uint32_t stage = ring_s + st * STAGE;
+        mbar_wait(full0 + 8 * st, (n / S) & 1u, abort_flag);
+        if (trace && first && tid == 0)
+            trace[2] = globaltimer_ns();
+        first = false;
+        const SReq rq = s_req[a];
+        const bool store_tile = rq.wb != nullptr && tid == 0;
+        if (store_tile)
+            bulk_s2g(rq.wb + (size_t)f0 * RB, stage, (uint32_t)m * RB);
+        // ---- gate/up.  Rows the tile does not have read row 0; their results are dropped below.
+        float cg[4][4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            cg[i][0] = cg[i][1] = cg[i][2] = cg[i][3] = 0.f;
+        {
+            const int rr = g < m ? g : 0;
+            const uint32_t fx = (uint32_t)((f0 + rr) & 7);
+            const uint32_t row = stage + rr * RB;
+            uint32_t sg = 0, su = 0;
+#pragma unroll
+            for (int i = 0; i < kMaxWs; ++i) {
+                if (i < WS) {
+                    const uint32_t ws = (uint32_t)(warp * WS + i);                  // 32-column step = 16-byte piece of codes
+                    const uint32_t pp = (ws & ~7u) | ((ws ^ fx) & 7u);
+                    const uint32_t wg = lds32(row + pp * 16 + tig * 4);
+                    const uint32_t wu = lds32(row + (uint32_t)(d / 2) + pp * 16 + tig * 4);
+                    if ((i & 1) == 0 || WS == 1) {
+                        sg = lds16(row + sc_off + (ws >> 1) * 2) * 0x10001u;
+                        su = lds16(row + sc_off + sc_len + (ws >> 1) * 2) * 0x10001u;
+                    }
+                    uint4 xb = make_uint4(0u, 0u, 0u, 0u);
+                    if (has_tok)
+                        xb = lds128(xrow + i * 64);
+                    uint32_t Pg[4], Pu[4];
+                    dequant8(wg, sg, Pg);
+                    dequant8(wu, su, Pu);
+                    mma_16816(cg[(2 * i) & 3], Pg[0], Pu[0], Pg[1], Pu[1], xb.x, xb.y);
+                    mma_16816(cg[(2 * i + 1) & 3], Pg[2], Pu[2], Pg[3], Pu[3], xb.z, xb.w);
+                }
+            }
+        }
+        // ---- the warps' partial tiles meet (as in the bf16 path)
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            buf[warp * kBufPitch + i * 32 + lane] = (cg[0][i] + cg[1][i]) + (cg[2][i] + cg[3][i]);
+        asm volatile("bar.sync 1, %0;" ::"n"(NW * 32) : "memory");
+        {
+            const int e = warp * 8 + (lane & 7), pg = lane >> 3;
+            float v = buf[(pg * 4) * kBufPitch + e];
+            v += buf[(pg * 4 + 1) * kBufPitch + e];
+            v += buf[(pg * 4 + 2) * kBufPitch + e];
+            v += buf[(pg * 4 + 3) * kBufPitch + e];
+            v += __shfl_xor_sync(0xffffffffu, v, 8);
+            v += __shfl_xor_sync(0xffffffffu, v, 16);
+            if (lane < 8)
+                s_sums[e] = v;
+        }
+        asm volatile("bar.sync 1, %0;" ::"n"(NW * 32) : "memory");
+        // g_f[t] and u_f[t] of the tile sit at (t & 1) * 32 + 4 f + (t >> 1) and 64 further on (the
+        // accumulator layout of the product).  This thread needs h of f = tig, tig + 4 for token g mod 4
+        // (and that token + 4).
+        auto hval = [&](int f, int t) -> uint32_t {
+            const int o = (t & 1) * 32 + f * 4 + (t >> 1);
+            const float vg = s_sums[o], vu = s_sums[64 + o];
+            const float gt = s_gate[rq.gate_row * kTokPerVr + t];
+            const float h = __fdividef(vg, 1.0f + __expf(-vg)) * vu * gt;
+            return (f >= m || gt == 0.0f) ? 0u : bf16_rne(h);
+        };
+        const uint32_t b0 = hval(tig, t0) << sh, b1 = hval(tig + 4, t0) << sh;
+        uint32_t b0h = 0u, b1h = 0u;
+        if (two) {
+            b0h = hval(tig, t0 + 4) << sh;
+            b1h = hval(tig + 4, t0 + 4) << sh;
+        }
+        // ---- down
+        {
+            const int ra = tig < m ? tig : 0, rb = tig + 4 < m ? tig + 4 : 0;
+            const uint32_t fa = (uint32_t)((f0 + ra) & 7), fb = (uint32_t)((f0 + rb) & 7);
+            const uint32_t rowa = stage + ra * RB, rowb = stage + rb * RB;
+            const int hf = warp & 1;
+#pragma unroll
+            for (int b = 0; b < kMaxWs / 2; ++b) {
+                if (2 * b < WS) {
+                    const uint32_t block = (uint32_t)(warp * WS + 2 * b) >> 1;          // 64 output columns = one scale group
+                    const uint32_t piece = block * 2 + (uint32_t)(g >> 2);
+                    const uint32_t wa = lds32(rowa + (uint32_t)d + ((piece & ~7u) | ((piece ^ fa) & 7u)) * 16 + (g & 3) * 4);
+                    const uint32_t wb = lds32(rowb + (uint32_t)d + ((piece & ~7u) | ((piece ^ fb) & 7u)) * 16 + (g & 3) * 4);
+                    const uint32_t sa = lds16(rowa + sc_off + 2 * sc_len + block * 2) * 0x10001u;
+                    const uint32_t sb = lds16(rowb + sc_off + 2 * sc_len + block * 2) * 0x10001u;
+                    uint32_t Pa[4], Pb[4];
+                    dequant8(wa, sa, Pa);
+                    dequant8(wb, sb, Pb);
+                    if (WS == 1) {
+                        // two warps share the block: this one owns its columns j = 2 hf, 2 hf + 1 (and + 4)
+                        const uint32_t a0 = hf ? Pa[2] : Pa[0], a1 = hf ? Pa[3] : Pa[1], a2 = hf ? Pb[2] : Pb[0], a3 = hf ? Pb[3] : Pb[1];
+                        mma_16816(acc[0][0], a0, a1, a2, a3, b0, b1);
+                        if (two)
+                            mma_16816(acc[0][1], a0, a1, a2, a3, b0h, b1h);
+                    } else {
+                        mma_16816(acc[2 * b][0], Pa[0], Pa[1], Pb[0], Pb[1], b0, b1);
+                        mma_16816(acc[2 * b + 1][0], Pa[2], Pa[3], Pb[2], Pb[3], b0, b1);
+                        if (two) {
+                            mma_16816(acc[2 * b][1], Pa[0], Pa[1], Pb[0], Pb[1], b0h, b1h);
+                            mma_16816(acc[2 * b + 1][1], Pa[2], Pa[3], Pb[2], Pb[3], b0h, b1h);
+                        }
+                    }
+                }
+            }
+        }
+        if (store_tile)
+            bulk_wait_read();         // the slot store has read the stage
+        __syncwarp();
+        if (lane == 0)
+            mbar_arrive(empty0 + 8 * st);
+        ++n;
+        q += m;
+        f0 += m;
+        if (f0 == F) {
+            f0 = 0;
+            ++a;
+        }
+    }
+    if (trace && tid == 0)
+        trace[3] = globaltimer_ns();
+    // ---- this CTA's partial output into the call's accumulator (64-bit fixed point, as in the bf16 path).
+    // Accumulator i of the warp is the 32-column step hb = warp * WS + i: block hb / 2, and within the
+    // block's 64 columns, column 8 g + 2 (hb mod 2) + {0, 1} for the product's rows g, g + 8, plus 4
+    // for the product's right half (tig >= 2); its columns there are tokens 2 (tig mod 2), + 1.
+    {
+        unsigned long long *yacc = reinterpret_cast<unsigned long long *>(p.yacc);
+        auto add = [&](int t, int c, float v) {
+            if (t < Tc) {
+                const long long fx = __float2ll_rn(v * 1099511627776.0f);
+                atomicAdd(yacc + (size_t)t * d + c, (unsigned long long)fx);
+            }
+        };
+#pragma unroll
+        for (int i = 0; i < kMaxWs; ++i) {
+            if (i < WS) {
+                const int hb = warp * WS + i;
+                const int c = (hb >> 1) * 64 + 8 * g + 2 * (hb & 1) + 4 * (tig >> 1);
+                const int t = 2 * (tig & 1);
+#pragma unroll
+                for (int tg = 0; tg < 2; ++tg) {
+                    if (tg == 0 || two) {
+                        add(t + 4 * tg, c, acc[i][tg][0]);
+                        add(t + 4 * tg + 1, c, acc[i][tg][1]);
+                        add(t + 4 * tg, c + 1, acc[i][tg][2]);
+                        add(t + 4 * tg + 1, c + 1, acc[i][tg][3]);
+                    }
+                }
+            }
+        }
+    }
+}
+
+// MT_: k-steps of the gate/up phase and m-tiles of the down phase per warp (d / 256), 0 = taken from d at run time.
+// FMT: 0 = bf16 expert blobs, 1 = 4-bit blobs (melinoe_moe_pack_expert_q4), expanded in registers on
+// the way into the tensor-core fragments.
+template <int MT_, int FMT>
 __global__ void __launch_bounds__(kThreads, 1) ffn_decode_kernel(DecParams p, DecGeometry geo)
 {
     extern __shared__ __align__(128) unsigned char smem[];
@@ -278,7 +509,10 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_decode_kernel(DecParams p, De
         const int per_row = d / 8;                  // 16-byte pieces of a hidden row
         for (int i = tid; i < Tc * per_row; i += kThreads) {
             const int t = i / per_row, c = i % per_row;
-            const uint4 v = *reinterpret_cast<const uint4 *>(p.x + (size_t)(tok0 + t) * d + c * 8);
+            uint4 v = *reinterpret_cast<const uint4 *>(p.x + (size_t)(tok0 + t) * d + c * 8);
+            if (FMT == 1)       // elements (0,4) (1,5) (2,6) (3,7): the pairing of the expanded weight registers
+                v = make_uint4(__byte_perm(v.x, v.z, 0x5410), __byte_perm(v.x, v.z, 0x7632), __byte_perm(v.y, v.w, 0x5410),
+                               __byte_perm(v.y, v.w, 0x7632));
             *reinterpret_cast<uint4 *>(xs + (size_t)t * XP + c * 16) = v;
         }
     }
@@ -417,6 +651,9 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_decode_kernel(DecParams p, De
     } else {
         // =================================================================== consumers
         const int g = lane >> 2, tig = lane & 3;
+        if constexpr (FMT == 1) {
+            consume_q4<MT_>(p, geo, s_req, &s_gate[0][0], s_sums, buf, ring_s, xs_s, full0, empty0, abort_flag, q_lo, q_hi, trace);
+        } else {
         float acc[kMaxMt][4];
 #pragma unroll
         for (int i = 0; i < kMaxMt; ++i)
@@ -588,6 +825,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_decode_kernel(DecParams p, De
                 }
             }
         }
+        }
         if (tid == 0)
             bulk_wait_all();              // the slot stores of this thread have completed
     }
@@ -670,12 +908,15 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_decode_kernel(DecParams p, De
 }  // namespace
 
 bool ffn_decode_supported(int d, int F) { return d % 256 == 0 && d >= 256 && d <= 4096 && F % kUnitRows == 0; }
+// 4-bit slots: the warps split the columns in steps of 32 (one 16-byte piece of codes), 16 warps.
+bool ffn_decode_supported_q4(int d, int F) { return ffn_decode_supported(d, F) && d % 512 == 0; }
 
 cudaError_t ffn_decode_configure(int n_sms, size_t max_smem, DecLaunchCfg *cfg)
 {
     size_t stat = 0;
-    const void *fns[3] = {reinterpret_cast<const void *>(ffn_decode_kernel<0>), reinterpret_cast<const void *>(ffn_decode_kernel<8>),
-                          reinterpret_cast<const void *>(ffn_decode_kernel<16>)};
+    const void *fns[6] = {reinterpret_cast<const void *>(ffn_decode_kernel<0, 0>), reinterpret_cast<const void *>(ffn_decode_kernel<8, 0>),
+                          reinterpret_cast<const void *>(ffn_decode_kernel<16, 0>), reinterpret_cast<const void *>(ffn_decode_kernel<0, 1>),
+                          reinterpret_cast<const void *>(ffn_decode_kernel<8, 1>), reinterpret_cast<const void *>(ffn_decode_kernel<16, 1>)};
     for (const void *fn : fns) {
         cudaFuncAttributes fa;
         const cudaError_t e = cudaFuncGetAttributes(&fa, fn);
@@ -698,11 +939,13 @@ cudaError_t ffn_decode_configure(int n_sms, size_t max_smem, DecLaunchCfg *cfg)
 
 cudaError_t ffn_decode_geometry(const DecLaunchCfg &cfg, int d, int F, int tokens, int fmt, DecGeometry *geo)
 {
-    if (!ffn_decode_supported(d, F) || tokens < 1 || tokens > kTokPerVr || fmt != 0)
+    if (!(fmt == 0 ? ffn_decode_supported(d, F) : fmt == 1 && ffn_decode_supported_q4(d, F)) || tokens < 1 || tokens > kTokPerVr)
         return cudaErrorInvalidValue;
     geo->n_warps = NW;
-    geo->row_bytes = 6 * d;
-    geo->x_pitch = 2 * d + 16;
+    // bytes of one hidden unit; pitch of the staged hidden rows (the pad keeps the fragment loads of neighbouring
+    // tokens in different banks: 4-byte loads in the bf16 path, 16-byte loads in the 4-bit path)
+    geo->row_bytes = fmt == 0 ? 6 * d : (3 * (d / 2) + 3 * (d / 64) * 2 + 15) / 16 * 16;
+    geo->x_pitch = fmt == 0 ? 2 * d + 16 : 2 * d + 64;
     geo->tokens = tokens;
     // staged hidden rows + the warps' partial tiles; the largest tile (at most 8 rows) of which two
     // stages fit beside them
@@ -752,9 +995,15 @@ cudaError_t launch_ffn_decode(cudaStream_t stream, const DecLaunchCfg &cfg, cons
     lc.attrs = attr;
     lc.numAttrs = na;
     const int mt = p.d / (16 * NW);
-    const cudaError_t e = mt == 8    ? cudaLaunchKernelEx(&lc, ffn_decode_kernel<8>, p, geo)
-                          : mt == 16 ? cudaLaunchKernelEx(&lc, ffn_decode_kernel<16>, p, geo)
-                                     : cudaLaunchKernelEx(&lc, ffn_decode_kernel<0>, p, geo);
+    cudaError_t e;
+    if (p.fmt == 0)
+        e = mt == 8    ? cudaLaunchKernelEx(&lc, ffn_decode_kernel<8, 0>, p, geo)
+            : mt == 16 ? cudaLaunchKernelEx(&lc, ffn_decode_kernel<16, 0>, p, geo)
+                       : cudaLaunchKernelEx(&lc, ffn_decode_kernel<0, 0>, p, geo);
+    else
+        e = mt == 8    ? cudaLaunchKernelEx(&lc, ffn_decode_kernel<8, 1>, p, geo)
+            : mt == 16 ? cudaLaunchKernelEx(&lc, ffn_decode_kernel<16, 1>, p, geo)
+                       : cudaLaunchKernelEx(&lc, ffn_decode_kernel<0, 1>, p, geo);
     count_launch();
     return e;
 }

@@ -103,6 +103,7 @@ struct DecGeometry {
 };
 cudaError_t ffn_decode_configure(int n_sms, size_t max_smem, DecLaunchCfg *cfg);
 bool ffn_decode_supported(int d, int F);
+bool ffn_decode_supported_q4(int d, int F);
 cudaError_t ffn_decode_geometry(const DecLaunchCfg &cfg, int d, int F, int tokens, int fmt, DecGeometry *geo);
 cudaError_t launch_ffn_decode(cudaStream_t stream, const DecLaunchCfg &cfg, const DecGeometry &geo,
                               const DecParams &p);

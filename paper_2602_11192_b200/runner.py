@@ -29,12 +29,19 @@ def to_dev_bf16(bits: np.ndarray) -> torch.Tensor:
 class LayerSetup:
     """One layer: pinned host store of packed experts, device router, the library handle."""
 
-    def __init__(self, d_model: int, d_ff: int, n_experts: int, top_k: int, cache_slots: int, n_shared: int = 0):
+    def __init__(self, d_model: int, d_ff: int, n_experts: int, top_k: int, cache_slots: int, n_shared: int = 0,
+                 slots: str = "bf16"):
+        """slots = "q4": the cache slots (and therefore the store and the shared experts) hold 4-bit blobs."""
         self.d, self.F, self.E, self.k, self.C, self.n_shared = d_model, d_ff, n_experts, top_k, cache_slots, n_shared
-        self.expert_bytes = B.melinoe_moe_expert_bytes(d_model, d_ff)
-        self.store = torch.empty((n_experts, self.expert_bytes), dtype=torch.uint8, pin_memory=True)
+        self.slots = slots
+        if slots == "q4":
+            self.expert_bytes = B.melinoe_moe_expert_bytes_q4(d_model, d_ff)
+            self.store = None
+        else:
+            self.expert_bytes = B.melinoe_moe_expert_bytes(d_model, d_ff)
+            self.store = torch.empty((n_experts, self.expert_bytes), dtype=torch.uint8, pin_memory=True)
         self.shared_store: Optional[torch.Tensor] = None
-        self.layer = B.MoELayer(d_model, d_ff, n_experts, top_k, cache_slots)
+        self.layer = B.MoELayer(d_model, d_ff, n_experts, top_k, cache_slots, slots=slots)
         self.router_dev: Optional[torch.Tensor] = None
         self.bias_dev = None
         self.seq_dev = None
@@ -70,9 +77,20 @@ class LayerSetup:
             self.layer.register_shared_experts([sb + s * self.expert_bytes for s in range(self.n_shared)],
                                                keep=self.shared_store)
 
-    def set_experts_q4(self, experts: Sequence[Tuple]) -> None:
+    def set_experts_q4(self, experts: Sequence[Tuple], shared: Sequence[Tuple] = ()) -> None:
         """experts[e] = (W_g, W_u, W_d) numpy uint16 (bf16 bits): quantised into a 4-bit pinned store."""
         assert len(experts) == self.E
+        if self.n_shared and self.slots == "q4":
+            assert len(shared) == self.n_shared
+            tmp = torch.empty((self.n_shared, self.expert_bytes), dtype=torch.uint8)
+            for s_, w in enumerate(shared):
+                a = [np.ascontiguousarray(m) for m in w]
+                B.melinoe_moe_pack_expert_q4(self.d, self.F, a[0].ctypes.data, a[1].ctypes.data, a[2].ctypes.data,
+                                             tmp.data_ptr() + s_ * self.expert_bytes)
+            self.shared_store = tmp.cuda()
+            sb = self.shared_store.data_ptr()
+            self.layer.register_shared_experts([sb + s_ * self.expert_bytes for s_ in range(self.n_shared)],
+                                               keep=self.shared_store)
         qb = B.melinoe_moe_expert_bytes_q4(self.d, self.F)
         assert qb > 0, "the 4-bit store needs d_ff % 64 == 0"
         self.store_q4 = torch.empty((self.E, qb), dtype=torch.uint8, pin_memory=True)
@@ -113,9 +131,9 @@ class LayerSetup:
         """Shared experts of the layer: wg/wu [n_shared][F][d], wd [n_shared][d][F] bf16 CPU tensors."""
         assert wg.shape[0] == self.n_shared
         tmp = torch.empty((self.n_shared, self.expert_bytes), dtype=torch.uint8)
+        pack = B.melinoe_moe_pack_expert_q4 if self.slots == "q4" else B.melinoe_moe_pack_expert
         for s in range(self.n_shared):
-            B.melinoe_moe_pack_expert(self.d, self.F, wg[s].data_ptr(), wu[s].data_ptr(), wd[s].data_ptr(),
-                                      tmp.data_ptr() + s * self.expert_bytes)
+            pack(self.d, self.F, wg[s].data_ptr(), wu[s].data_ptr(), wd[s].data_ptr(), tmp.data_ptr() + s * self.expert_bytes)
         self.shared_store = tmp.cuda()
         sb = self.shared_store.data_ptr()
         self.layer.register_shared_experts([sb + s * self.expert_bytes for s in range(self.n_shared)],

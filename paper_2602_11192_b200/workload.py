@@ -44,9 +44,11 @@ class Stack:
         self.bias: List[np.ndarray] = []
         t0 = time.time()
         for l in range(self.L):
-            ls = LayerSetup(cfg.d_model, cfg.d_ff, cfg.n_experts, cfg.top_k, self.C[l], cfg.n_shared)
+            # store: "bf16"; "q4" = 4-bit host store expanded into bf16 slots; "q4slots" = 4-bit store and 4-bit slots
+            ls = LayerSetup(cfg.d_model, cfg.d_ff, cfg.n_experts, cfg.top_k, self.C[l], cfg.n_shared,
+                            slots="q4" if store == "q4slots" else "bf16")
             wg, wu, wd = gen.fill_expert_store_fast(cfg.seed, l, cfg.n_experts + cfg.n_shared, cfg.d_model, cfg.d_ff)
-            if store == "q4":
+            if store in ("q4", "q4slots"):
                 ls.set_experts_stacked_q4(wg[:cfg.n_experts], wu[:cfg.n_experts], wd[:cfg.n_experts])
             else:
                 ls.set_experts_stacked(wg[:cfg.n_experts], wu[:cfg.n_experts], wd[:cfg.n_experts])

@@ -59,13 +59,13 @@ class Pair:
         self.d, self.F, self.E, self.k, self.C, self.n_shared = d, F, E, k, C, n_shared
         self.weights = make_weights(seed, layer, E, d, F, n_shared)
         self.w_r = gen.router_weights(seed, layer, E, d)
-        self.gpu = LayerSetup(d, F, E, k, C, n_shared)
+        self.gpu = LayerSetup(d, F, E, k, C, n_shared, slots="q4" if store == "q4slots" else "bf16")
         self.bytes_per_miss = 3 * d * F * 2
-        if store == "q4":
+        if store in ("q4", "q4slots"):
             # the library quantises the original weights; the oracle computes with what the 4-bit
             # format defines as the layer's weights (its own quantise + dequantise)
-            assert n_shared == 0
-            self.gpu.set_experts_q4(self.weights)
+            assert n_shared == 0 or store == "q4slots"
+            self.gpu.set_experts_q4(self.weights[:E], self.weights[E:])
             self.weights = [_q4_roundtrip(w) for w in self.weights]
             self.bytes_per_miss = melinoe_moe_expert_bytes_q4(d, F)
         else:

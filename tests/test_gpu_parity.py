@@ -414,6 +414,38 @@ def test_q4_host_store_matches_the_oracle_and_a_bf16_store_of_the_same_weights()
     P.close()
 
 
+@pytest.mark.parametrize("d,F,E,k,C,n_shared", [(512, 128, 12, 2, 4, 0), (1024, 72, 16, 4, 8, 1), (2048, 64, 16, 8, 8, 0),
+                                                (4096, 40, 8, 2, 4, 0)])
+def test_q4_slots_match_the_oracle(d, F, E, k, C, n_shared):
+    """4-bit cache slots: host link and HBM carry 4-bit blobs only, the FFN kernel expands the codes in
+    registers.  Routing, cache trace and statistics bit for bit, activations element-wise, against the
+    oracle on the weights the format defines; calls of 1..8 tokens (fetched by the kernel itself), of
+    more tokens than slots allow (copies issued by the host) and of several launches; both entry points."""
+    P = _pair(d, F, E, k, C, seed=61, n_shared=n_shared, store="q4slots")
+    from paper_2602_11192_b200 import melinoe_moe_expert_bytes_q4
+    assert P.bytes_per_miss == melinoe_moe_expert_bytes_q4(d, F) and P.gpu.layer.slots == "q4"
+    n_miss = 0
+    for step, T in enumerate((1, 1, 2, 8, 5, 1, 19, 3, 1, 4)):
+        x = gen.hidden_states(61, 0, "decode", step, T, d)
+        entry = "static" if T <= 8 and T * k <= 64 and step % 2 == 1 else "forward"
+        res, out = P.step(x, entry=entry)
+        n_miss += out["stats"]["misses"]
+        assert not P.gpu.layer.last_call_used_gemm()
+    assert n_miss > 6
+    P.set_policy("count", 0.9)
+    P.reset()
+    P.preload(list(range(min(C, 3))))
+    for step in range(6):
+        P.step(gen.hidden_states(61, 0, "decode", 50 + step, 1 + step % 3, d))
+    # a bf16 store cannot be registered on this handle, nor 4-bit slots made for a width the kernel does not split
+    with pytest.raises(Exception):
+        P.gpu.layer.register_host_experts([0] * E, 3 * d * F * 2)
+    P.close()
+    from paper_2602_11192_b200 import MoELayer
+    with pytest.raises(Exception):
+        MoELayer(768, 64, 8, 2, 4, slots="q4")
+
+
 def test_parity_without_programmatic_launch():
     """The decode kernels are launched with programmatic stream serialisation by default; the
     same parity must hold with the attribute switched off (the switch is read once per process,
