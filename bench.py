@@ -276,12 +276,12 @@ def hit_summary(cfg, stats, K, L):
             "h2d_expert_bytes_per_step": m * cfg.expert_bytes / K}
 
 
-def ffn_launch_analysis(cfg, stats, per_launch, hbm_peak, link_peak):
+def ffn_launch_analysis(cfg, stats, per_launch, hbm_peak, link_peak, expert_bytes=None):
     """Per-launch CUDA-event times of the decode FFN kernel against what each launch moved.
     One launch per call here (the kernel fetches missed experts itself), so launch i of layer l is call i.
     Launches whose experts were all resident are bound by HBM: bytes = experts x bytes per expert.  Launches
     that fetched experts are bound by the host link for those: bytes over the link / launch time."""
-    B_e = cfg.expert_bytes
+    B_e = cfg.expert_bytes if expert_bytes is None else expert_bytes
     res_bytes = res_ms = 0.0
     res_n = 0
     miss_bytes = miss_ms = 0.0
@@ -572,6 +572,32 @@ def run_ours(args):
             extra["store=q4,policy=lfu"] = dict(value=cfg.batch * K / (ms_q * 1e-3), **hit_summary(cfg, st_q, K, L))
             extra["store=q4,policy=lfu"]["h2d_expert_bytes_per_step"] = float(st_q["misses"].sum()) * qb / K
             Rq.close()
+        # 4-bit cache slots (Appendix D.5, Table 12: at equal memory 4-bit experts let about 3.76 times as many stay
+        # resident): the same number of slots, then the number of 4-bit slots that fit the bf16 slots' memory
+        if cfg.d_model % 512 == 0:
+            qb = M.melinoe_moe_expert_bytes_q4(cfg.d_model, cfg.d_ff)
+            C_eq = int(min(cfg.n_experts, C * cfg.expert_bytes // qb))
+            for name, Cq in (("slots=q4,same_count", C), ("slots=q4,equal_memory", C_eq)):
+                phase("4-bit slots: %d per layer" % Cq)
+                Rs = Runner(torch, M, gen, cfg, alpha0, Cq, L, K, W, store="q4slots")
+                vals = []
+                for _ in range(REPEATS):
+                    ms_s, _, st_s, _ = Rs.timed_device(alpha0)
+                    vals.append(cfg.batch * K / (ms_s * 1e-3))
+                _, _, st_s2, pl_s = Rs.timed_device(alpha0, with_kernel_timing=True)
+                ana_s = ffn_launch_analysis(cfg, st_s2, pl_s, hbm_peak, link_peak, expert_bytes=qb)
+                med, best = med_best(vals)
+                rec = {"value": med, "best": best, "cache_slots": Cq, "slot_bytes": qb, "slot_memory_bytes_per_layer": Cq * qb,
+                       "bf16_slot_memory_bytes_per_layer": C * cfg.expert_bytes, **hit_summary(cfg, st_s, K, L)}
+                if ana_s and ana_s["resident"]:
+                    r_ = ana_s["resident"]
+                    rec["ffn_resident"] = {"launches": r_["launches"], "avg_launch_us": r_["avg_launch_us"], "gbs_4bit": r_["gbs"],
+                                           "frac_of_hbm": r_["frac_of_hbm"],
+                                           "bf16_equivalent_gbs": r_["gbs"] * cfg.expert_bytes / qb}
+                if ana_s and ana_s["fetching"]:
+                    rec["ffn_fetching"] = ana_s["fetching"]
+                extra[name] = rec
+                Rs.close()
         # everything resident (cache = all experts, warm): the hit path alone
         phase("all experts resident")
         Rf = Runner(torch, M, gen, cfg, alpha0, cfg.n_experts, L, K, W)

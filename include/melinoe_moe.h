@@ -106,7 +106,7 @@ int melinoe_moe_create(int d_model, int d_ff, int n_experts, int top_k, int cach
  * host link only ever carry 4-bit data.  The layer computes with exactly the weights the format defines
  * (see melinoe_moe_pack_expert_q4).  Shared experts, if any, are registered as 4-bit blobs too.  Calls of
  * every size run the decode kernel, 8 tokens per launch (there is no 4-bit grouped GEMM).  Needs
- * d_model % 512 == 0 on top of the limits above.
+ * d_model = 512, 1024, 2048 or 4096 on top of the limits above.
  */
 int melinoe_moe_create_q4(int d_model, int d_ff, int n_experts, int top_k, int cache_slots,
                           melinoe_moe_t **out);
@@ -146,7 +146,9 @@ int melinoe_moe_pack_expert(int d_model, int d_ff, const void *w_gate_host, cons
  *     codes W_g[f] | codes W_u[f] | codes W_d[:, f]    d_model / 2 bytes each, even element in the low nibble
  *     scales W_g[f] | scales W_u[f] | scales W_d[:, f]  d_model / 64 bf16 each
  * then zero padding to a multiple of 16 bytes (none when d_model % 512 == 0).  Within each code
- * vector, the 16-byte pieces of every group of eight sit at position (piece xor (f mod 8)).  As in
+ * vector, the 16-byte pieces of every group of eight sit at position (piece xor (f mod 8)); in the
+ * codes of W_d[:, f], position p of a group of 64 holds element 8 (p mod 8) + p / 8 of that group (the
+ * order in which the compute kernel's output fragments own the columns).  As in
  * the bf16 blob, everything f contributes is one contiguous byte range.  Needs d_model % 256 == 0 and
  * d_ff % 8 == 0 (else the size is 0 and packing returns MELINOE_ERR_UNSUPPORTED).  Pure host code.
  */

@@ -437,7 +437,8 @@ uint16_t host_f32_to_bf16(float f)
 // One vector of d values (read at stride `stride`) into d / 2 code bytes and d / 64 scales: groups of 64
 // consecutive values, scale = bf16(max|w| / 7), code = clamp(rint(w / scale), -8, 7) + 8, ties to even.  The
 // 16-byte pieces of the codes (32 codes each) go to position (piece xor x) within every group of 8 pieces.
-void pack_q4_vector(const uint16_t *w, size_t stride, int d, int x, unsigned char *codes, uint16_t *scales)
+// interleave: element i of a group sits at code position 8 * (i mod 8) + i / 8 of the group instead of i.
+void pack_q4_vector(const uint16_t *w, size_t stride, int d, int x, bool interleave, unsigned char *codes, uint16_t *scales)
 {
     for (int g = 0; g < d / 64; ++g) {
         float amax = 0.0f;
@@ -446,11 +447,12 @@ void pack_q4_vector(const uint16_t *w, size_t stride, int d, int x, unsigned cha
         const uint16_t sb = host_f32_to_bf16(amax / 7.0f);
         const float sc = host_bf16_to_f32(sb);
         scales[g] = sb;
-        for (int j = 0; j < 64; j += 2) {
+        for (int j = 0; j < 64; j += 2) {       // code positions j, j + 1 of the group share a byte
             int q[2] = {0, 0};
             for (int h2 = 0; h2 < 2; ++h2)
                 if (sc > 0.0f) {
-                    const float t = std::nearbyint(host_bf16_to_f32(w[(size_t)(g * 64 + j + h2) * stride]) / sc);   // ties to even
+                    const int pos = j + h2, i = interleave ? 8 * (pos % 8) + pos / 8 : pos;     // the element at this position
+                    const float t = std::nearbyint(host_bf16_to_f32(w[(size_t)(g * 64 + i) * stride]) / sc);   // ties to even
                     q[h2] = (int)std::fmin(7.0f, std::fmax(-8.0f, t));
                 }
             const int byte = (g * 64 + j) / 2, piece = byte / 16;
@@ -476,9 +478,9 @@ int melinoe_moe_pack_expert_q4(int d, int F, const void *wg_, const void *wu_, c
         unsigned char *u = blob + (size_t)f * ub;
         std::memset(u, 0, ub);
         uint16_t *sc = reinterpret_cast<uint16_t *>(u + 3 * (size_t)(d / 2));
-        pack_q4_vector(wg + (size_t)f * d, 1, d, f & 7, u, sc);
-        pack_q4_vector(wu + (size_t)f * d, 1, d, f & 7, u + d / 2, sc + d / 64);
-        pack_q4_vector(wd + f, (size_t)F, d, f & 7, u + 2 * (size_t)(d / 2), sc + 2 * (d / 64));    // column f of W_d
+        pack_q4_vector(wg + (size_t)f * d, 1, d, f & 7, false, u, sc);
+        pack_q4_vector(wu + (size_t)f * d, 1, d, f & 7, false, u + d / 2, sc + d / 64);
+        pack_q4_vector(wd + f, (size_t)F, d, f & 7, true, u + 2 * (size_t)(d / 2), sc + 2 * (d / 64));    // column f of W_d
     }
     return MELINOE_OK;
 }

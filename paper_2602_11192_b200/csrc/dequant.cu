@@ -2,7 +2,8 @@
 //
 // Both blobs are organised per hidden unit f (see melinoe_moe_pack_expert / _pack_expert_q4): the
 // 4-bit unit holds the codes of W_g[f], W_u[f], W_d[:, f] (d / 2 bytes each, the even element in the
-// low nibble, the 16-byte pieces of every 128-byte group at (piece xor (f mod 8))), then their
+// low nibble, the 16-byte pieces of every 128-byte group at (piece xor (f mod 8)); in W_d[:, f] the
+// code at position p of a group of 64 is element 8 (p mod 8) + p / 8 of the group), then their
 // scales (d / 64 bf16 each).  The weight that the layer computes with is bf16(scale * (code - 8)):
 // the product is exact in fp32 and is rounded to nearest even.  The bf16 unit holds the three
 // vectors of d bf16 values with the same kind of permutation on its own 16-byte pieces.
@@ -46,10 +47,22 @@ __global__ void __launch_bounds__(256) dequant_q4_kernel(const unsigned char *__
                 const float hi = __fmul_rn(sc, (float)((int)(byte >> 4) - 8));
                 o[b] = bf16_rne_bits(lo) | (bf16_rne_bits(hi) << 16);
             }
-            // these 8 weights are elements piece * 32 + w * 8 .. of the vector: bf16 piece 4 * piece + w
-            const int bp = 4 * piece + w;
-            const int pbp = (bp & ~7) | ((bp ^ x) & 7);
-            *reinterpret_cast<uint4 *>(row + (size_t)pbp * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+            if (m < 2) {
+                // these 8 weights are elements piece * 32 + w * 8 .. of the vector: bf16 piece 4 * piece + w
+                const int bp = 4 * piece + w;
+                const int pbp = (bp & ~7) | ((bp ^ x) & 7);
+                *reinterpret_cast<uint4 *>(row + (size_t)pbp * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+            } else {
+                // W_d[:, f]: code position pos of a group of 64 holds element 8 * (pos mod 8) + pos / 8; these are
+                // positions (piece mod 2) * 32 + w * 8 + j, j = 0 .. 7, that is element 8 j + (piece mod 2) * 4 + w
+                const int grp = piece / 2, e0 = (piece & 1) * 4 + w;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const int el = grp * 64 + 8 * j + e0;
+                    const int bp = el / 8, pbp = (bp & ~7) | ((bp ^ x) & 7);
+                    row[(size_t)pbp * 8 + el % 8] = (uint16_t)(j & 1 ? o[j / 2] >> 16 : o[j / 2] & 0xffffu);
+                }
+            }
         }
     }
 }

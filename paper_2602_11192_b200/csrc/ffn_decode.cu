@@ -186,6 +186,12 @@ __device__ __forceinline__ void bulk_s2g(void *dst, uint32_t src, uint32_t bytes
     asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes) : "memory");
     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
+// Add without a return value, on the global address space (a generic atomicAdd compiles to the
+// returning form on the generic space).
+__device__ __forceinline__ void red_add_u64(unsigned long long *addr, unsigned long long v)
+{
+    asm volatile("red.global.add.u64 [%0], %1;" ::"l"(__cvta_generic_to_global(addr)), "l"(v) : "memory");
+}
 __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
@@ -217,14 +223,24 @@ constexpr int kBufPitch = 130;                   // floats between the warps' pa
 //             of them for the output columns n = 0..3 (tokens 0..3) and in the second for n = 4..7
 //             (again tokens 0..3): the product's left half is column j of every row of output, its right
 //             half column j + 4.  One product so covers 8 hidden units x 32 output columns x 4 tokens;
-//             tokens 4..7 take a second product.  The warps split the columns in steps of 32.
+//             tokens 4..7 take a second product.  The warps split the columns in steps of 32.  (The codes
+//             of W_d[:, f] are stored interleaved within every 64, nibble j of word g being column
+//             g + 8 j, so that the lanes of one product row own neighbouring output columns.)
 constexpr int kMaxWs = 8;                        // 32-column steps per warp (d / 512)
+
+// One tile as the loop sees it.
+struct Q4Tile {
+    uint32_t stage, st;   // shared-memory address of its ring stage, index of the stage
+    int m, f0;            // rows, first hidden unit
+    int gate_row;
+    bool stored;          // this thread issued the tile's store into the cache slot
+};
 
 template <int MT_>
 __device__ __forceinline__ void consume_q4(const DecParams &p, const DecGeometry &geo, const SReq *s_req, const float *s_gate,
                                            float *s_sums, float *buf, uint32_t ring_s, uint32_t xs_s, uint32_t full0,
-                                           uint32_t empty0, volatile int *abort_flag, long long q_lo, long long q_hi,
-                                           unsigned long long *trace)
+                                           uint32_t empty0, uint32_t bar_a, uint32_t bar_b, volatile int *abort_flag,
+                                           long long q_lo, long long q_hi, unsigned long long *trace)
 {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, tig = lane & 3;
     const int d = p.d, F = p.F;
@@ -240,162 +256,224 @@ __device__ __forceinline__ void consume_q4(const DecParams &p, const DecGeometry
     const uint32_t xrow = xs_s + g * XP + (warp * WS * 32 + tig * 8) * 2;
     const uint32_t sc_off = 3 * (uint32_t)(d / 2), sc_len = (uint32_t)(d / 32);     // scales: offset in the unit, bytes per vector
     const int t0 = g & 3, sh = g < 4 ? 0 : 16;
-    uint32_t n = 0;
-    long long q = q_lo;
-    int a = (int)(q / F), f0 = (int)(q % F);
+
+    // ---- the tiles of this CTA in order; taking one waits until it has landed and starts its copy into the slot
+    int left = (int)(q_hi - q_lo);                  // rows still to take
+    int a = (int)(q_lo / F), f0 = (int)(q_lo % F);
+    uint32_t st = 0, ph = 0;                        // ring stage of the next tile and the parity of its barrier phase
     bool first = true;
-    while (q < q_hi) {
-        const int m = (int)min((long long)min(TR, F - f0), q_hi - q);
-        const uint32_t st = n % (uint32_t)S;
-        const uint32_t stage = ring_s + st * STAGE;
-        mbar_wait(full0 + 8 * st, (n / S) & 1u, abort_flag);
+    auto take = [&](Q4Tile &t) -> bool {
+        if (left <= 0)
+            return false;
+        t.m = min(min(TR, F - f0), left);
+        t.f0 = f0;
+        t.st = st;
+        t.stage = ring_s + st * STAGE;
+        mbar_wait(full0 + 8 * st, ph, abort_flag);
         if (trace && first && tid == 0)
             trace[2] = globaltimer_ns();
         first = false;
         const SReq rq = s_req[a];
-        const bool store_tile = rq.wb != nullptr && tid == 0;
-        if (store_tile)
-            bulk_s2g(rq.wb + (size_t)f0 * RB, stage, (uint32_t)m * RB);
-        // ---- gate/up.  Rows the tile does not have read row 0; their results are dropped below.
-        float cg[4][4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-            cg[i][0] = cg[i][1] = cg[i][2] = cg[i][3] = 0.f;
-        {
-            const int rr = g < m ? g : 0;
-            const uint32_t fx = (uint32_t)((f0 + rr) & 7);
-            const uint32_t row = stage + rr * RB;
-            uint32_t sg = 0, su = 0;
-#pragma unroll
-            for (int i = 0; i < kMaxWs; ++i) {
-                if (i < WS) {
-                    const uint32_t ws = (uint32_t)(warp * WS + i);                  // 32-column step = 16-byte piece of codes
-                    const uint32_t pp = (ws & ~7u) | ((ws ^ fx) & 7u);
-                    const uint32_t wg = lds32(row + pp * 16 + tig * 4);
-                    const uint32_t wu = lds32(row + (uint32_t)(d / 2) + pp * 16 + tig * 4);
-                    if ((i & 1) == 0 || WS == 1) {
-                        sg = lds16(row + sc_off + (ws >> 1) * 2) * 0x10001u;
-                        su = lds16(row + sc_off + sc_len + (ws >> 1) * 2) * 0x10001u;
-                    }
-                    uint4 xb = make_uint4(0u, 0u, 0u, 0u);
-                    if (has_tok)
-                        xb = lds128(xrow + i * 64);
-                    uint32_t Pg[4], Pu[4];
-                    dequant8(wg, sg, Pg);
-                    dequant8(wu, su, Pu);
-                    mma_16816(cg[(2 * i) & 3], Pg[0], Pu[0], Pg[1], Pu[1], xb.x, xb.y);
-                    mma_16816(cg[(2 * i + 1) & 3], Pg[2], Pu[2], Pg[3], Pu[3], xb.z, xb.w);
-                }
-            }
+        t.gate_row = rq.gate_row;
+        t.stored = rq.wb != nullptr && tid == 0;
+        if (t.stored)
+            bulk_s2g(rq.wb + (size_t)f0 * RB, t.stage, (uint32_t)t.m * RB);
+        if (++st == (uint32_t)S) {
+            st = 0;
+            ph ^= 1u;
         }
-        // ---- the warps' partial tiles meet (as in the bf16 path)
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-            buf[warp * kBufPitch + i * 32 + lane] = (cg[0][i] + cg[1][i]) + (cg[2][i] + cg[3][i]);
-        asm volatile("bar.sync 1, %0;" ::"n"(NW * 32) : "memory");
-        {
-            const int e = warp * 8 + (lane & 7), pg = lane >> 3;
-            float v = buf[(pg * 4) * kBufPitch + e];
-            v += buf[(pg * 4 + 1) * kBufPitch + e];
-            v += buf[(pg * 4 + 2) * kBufPitch + e];
-            v += buf[(pg * 4 + 3) * kBufPitch + e];
-            v += __shfl_xor_sync(0xffffffffu, v, 8);
-            v += __shfl_xor_sync(0xffffffffu, v, 16);
-            if (lane < 8)
-                s_sums[e] = v;
-        }
-        asm volatile("bar.sync 1, %0;" ::"n"(NW * 32) : "memory");
-        // g_f[t] and u_f[t] of the tile sit at (t & 1) * 32 + 4 f + (t >> 1) and 64 further on (the
-        // accumulator layout of the product).  This thread needs h of f = tig, tig + 4 for token g mod 4
-        // (and that token + 4).
-        auto hval = [&](int f, int t) -> uint32_t {
-            const int o = (t & 1) * 32 + f * 4 + (t >> 1);
-            const float vg = s_sums[o], vu = s_sums[64 + o];
-            const float gt = s_gate[rq.gate_row * kTokPerVr + t];
-            const float h = __fdividef(vg, 1.0f + __expf(-vg)) * vu * gt;
-            return (f >= m || gt == 0.0f) ? 0u : bf16_rne(h);
-        };
-        const uint32_t b0 = hval(tig, t0) << sh, b1 = hval(tig + 4, t0) << sh;
-        uint32_t b0h = 0u, b1h = 0u;
-        if (two) {
-            b0h = hval(tig, t0 + 4) << sh;
-            b1h = hval(tig + 4, t0 + 4) << sh;
-        }
-        // ---- down
-        {
-            const int ra = tig < m ? tig : 0, rb = tig + 4 < m ? tig + 4 : 0;
-            const uint32_t fa = (uint32_t)((f0 + ra) & 7), fb = (uint32_t)((f0 + rb) & 7);
-            const uint32_t rowa = stage + ra * RB, rowb = stage + rb * RB;
-            const int hf = warp & 1;
-#pragma unroll
-            for (int b = 0; b < kMaxWs / 2; ++b) {
-                if (2 * b < WS) {
-                    const uint32_t block = (uint32_t)(warp * WS + 2 * b) >> 1;          // 64 output columns = one scale group
-                    const uint32_t piece = block * 2 + (uint32_t)(g >> 2);
-                    const uint32_t wa = lds32(rowa + (uint32_t)d + ((piece & ~7u) | ((piece ^ fa) & 7u)) * 16 + (g & 3) * 4);
-                    const uint32_t wb = lds32(rowb + (uint32_t)d + ((piece & ~7u) | ((piece ^ fb) & 7u)) * 16 + (g & 3) * 4);
-                    const uint32_t sa = lds16(rowa + sc_off + 2 * sc_len + block * 2) * 0x10001u;
-                    const uint32_t sb = lds16(rowb + sc_off + 2 * sc_len + block * 2) * 0x10001u;
-                    uint32_t Pa[4], Pb[4];
-                    dequant8(wa, sa, Pa);
-                    dequant8(wb, sb, Pb);
-                    if (WS == 1) {
-                        // two warps share the block: this one owns its columns j = 2 hf, 2 hf + 1 (and + 4)
-                        const uint32_t a0 = hf ? Pa[2] : Pa[0], a1 = hf ? Pa[3] : Pa[1], a2 = hf ? Pb[2] : Pb[0], a3 = hf ? Pb[3] : Pb[1];
-                        mma_16816(acc[0][0], a0, a1, a2, a3, b0, b1);
-                        if (two)
-                            mma_16816(acc[0][1], a0, a1, a2, a3, b0h, b1h);
-                    } else {
-                        mma_16816(acc[2 * b][0], Pa[0], Pa[1], Pb[0], Pb[1], b0, b1);
-                        mma_16816(acc[2 * b + 1][0], Pa[2], Pa[3], Pb[2], Pb[3], b0, b1);
-                        if (two) {
-                            mma_16816(acc[2 * b][1], Pa[0], Pa[1], Pb[0], Pb[1], b0h, b1h);
-                            mma_16816(acc[2 * b + 1][1], Pa[2], Pa[3], Pb[2], Pb[3], b0h, b1h);
-                        }
-                    }
-                }
-            }
-        }
-        if (store_tile)
-            bulk_wait_read();         // the slot store has read the stage
-        __syncwarp();
-        if (lane == 0)
-            mbar_arrive(empty0 + 8 * st);
-        ++n;
-        q += m;
-        f0 += m;
+        left -= t.m;
+        f0 += t.m;
         if (f0 == F) {
             f0 = 0;
             ++a;
         }
+        return true;
+    };
+    // ---- gate/up of one tile: this warp's columns, into registers.  Rows the tile does not have read row 0;
+    // their results are dropped when h is formed.
+    auto gate_up = [&](const Q4Tile &t, float (&cg)[4][4]) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            cg[i][0] = cg[i][1] = cg[i][2] = cg[i][3] = 0.f;
+        const int rr = g < t.m ? g : 0;
+        const uint32_t fx16 = (uint32_t)((t.f0 + rr) & 7) << 4;
+        const uint32_t row = t.stage + rr * RB;
+        // piece ws of the codes sits at ((ws & ~7) | ((ws ^ f) & 7)) * 16: the warp's first step, then xor per step
+        const uint32_t ws0 = (uint32_t)(warp * WS);
+        const uint32_t cbase = row + (ws0 & ~7u) * 16 + tig * 4, sbase = row + sc_off + (ws0 >> 1) * 2;
+        uint32_t sg = 0, su = 0;
+#pragma unroll
+        for (int i = 0; i < kMaxWs; ++i) {
+            if (i < WS) {
+                const uint32_t wsl = (ws0 & 7u) + (uint32_t)i;
+                const uint32_t off = ((wsl << 4) ^ fx16) & 0x70u, hi = (wsl >> 3) * 128u;
+                const uint32_t wg = lds32(cbase + hi + off);
+                const uint32_t wu = lds32(cbase + hi + off + (uint32_t)(d / 2));
+                if ((i & 1) == 0 || WS == 1) {
+                    sg = lds16(sbase + (i >> 1) * 2) * 0x10001u;
+                    su = lds16(sbase + (i >> 1) * 2 + sc_len) * 0x10001u;
+                }
+                uint4 xb = make_uint4(0u, 0u, 0u, 0u);
+                if (has_tok)
+                    xb = lds128(xrow + i * 64);
+                uint32_t Pg[4], Pu[4];
+                dequant8(wg, sg, Pg);
+                dequant8(wu, su, Pu);
+                mma_16816(cg[(2 * i) & 3], Pg[0], Pu[0], Pg[1], Pu[1], xb.x, xb.y);
+                mma_16816(cg[(2 * i + 1) & 3], Pg[2], Pu[2], Pg[3], Pu[3], xb.z, xb.w);
+            }
+        }
+    };
+    // The warps' partial tiles meet in shared memory: every warp stores its 128 partial values, warp w sums
+    // 8 of the 128 over all warps (four lanes per value, each adding four warps' parts in warp order, then a
+    // fixed tree), and every warp reads the complete tile.  Two sets of buffers and two counting barriers
+    // (all warps have stored / all sums are there) let a warp do other work between arriving at a barrier
+    // and needing what it guards: the loop below is arranged so that it always has some.
+    auto store_partials = [&](const float (&cg)[4][4], uint32_t sel) {
+        float *b = buf + sel * (NW * kBufPitch) + warp * kBufPitch;
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            b[i * 32 + lane] = (cg[0][i] + cg[1][i]) + (cg[2][i] + cg[3][i]);
+        __syncwarp();
+        if (lane == 0)
+            mbar_arrive(bar_a);
+    };
+    auto column_sums = [&](uint32_t sel) {
+        const float *b = buf + sel * (NW * kBufPitch);
+        const int e = warp * 8 + (lane & 7), pg = lane >> 3;
+        float v = b[(pg * 4) * kBufPitch + e];
+        v += b[(pg * 4 + 1) * kBufPitch + e];
+        v += b[(pg * 4 + 2) * kBufPitch + e];
+        v += b[(pg * 4 + 3) * kBufPitch + e];
+        v += __shfl_xor_sync(0xffffffffu, v, 8);
+        v += __shfl_xor_sync(0xffffffffu, v, 16);
+        if (lane < 8)
+            s_sums[sel * 128 + e] = v;
+        __syncwarp();
+        if (lane == 0)
+            mbar_arrive(bar_b);
+    };
+    // ---- h of the tile from the complete sums, then the down product
+    auto down = [&](const Q4Tile &t, uint32_t sel) {
+        // g_f[t] and u_f[t] of the tile sit at (t & 1) * 32 + 4 f + (t >> 1) and 64 further on (the
+        // accumulator layout of the product).  This thread needs h of f = tig, tig + 4 for token g mod 4
+        // (and that token + 4).
+        const float *sums = s_sums + sel * 128;
+        // (h rounded to bf16 once, to nearest even; it goes to the register half of this thread's output column)
+        auto hval = [&](int f, int tk) -> uint32_t {
+            const int o = (tk & 1) * 32 + f * 4 + (tk >> 1);
+            const float vg = sums[o], vu = sums[64 + o];
+            const float gt = s_gate[t.gate_row * kTokPerVr + tk];
+            float h = __fdividef(vg, 1.0f + __expf(-vg)) * vu * gt;
+            if (f >= t.m || gt == 0.0f)
+                h = 0.f;
+            uint32_t r;
+            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(sh ? h : 0.f), "f"(sh ? 0.f : h));
+            return r;
+        };
+        const uint32_t b0 = hval(tig, t0), b1 = hval(tig + 4, t0);
+        uint32_t b0h = 0u, b1h = 0u;
+        if (two) {
+            b0h = hval(tig, t0 + 4);
+            b1h = hval(tig + 4, t0 + 4);
+        }
+        const int ra = tig < t.m ? tig : 0, rb = tig + 4 < t.m ? tig + 4 : 0;
+        const uint32_t fa16 = (uint32_t)((t.f0 + ra) & 7) << 4, fb16 = (uint32_t)((t.f0 + rb) & 7) << 4;
+        const uint32_t rowa = t.stage + ra * RB, rowb = t.stage + rb * RB;
+        const int hf = warp & 1;
+        // block = 64 output columns = one scale group = two 16-byte pieces of codes; this thread's word is in piece
+        // 2 block + g / 4
+        const uint32_t blk0 = (uint32_t)(warp * WS) >> 1, pc0 = blk0 * 2 + (uint32_t)(g >> 2);
+        const uint32_t cofs = (uint32_t)d + (pc0 & ~7u) * 16 + (g & 3) * 4, sofs = sc_off + 2 * sc_len + blk0 * 2;
+#pragma unroll
+        for (int b = 0; b < kMaxWs / 2; ++b) {
+            if (2 * b < WS) {
+                // (pc0 + 2 b) & 7 = (pc0 & 7) + 2 b for b < 4: pc0 & 7 is 0, 1 (four blocks), 0..5 (two), 0..7 (one or half)
+                const uint32_t pin = ((pc0 & 7u) + 2u * (uint32_t)b) << 4;
+                const uint32_t hi = (pin >> 7) * 128u;
+                const uint32_t wa = lds32(rowa + cofs + hi + ((pin ^ fa16) & 0x70u));
+                const uint32_t wb = lds32(rowb + cofs + hi + ((pin ^ fb16) & 0x70u));
+                const uint32_t sa = lds16(rowa + sofs + b * 2) * 0x10001u;
+                const uint32_t sb = lds16(rowb + sofs + b * 2) * 0x10001u;
+                uint32_t Pa[4], Pb[4];
+                dequant8(wa, sa, Pa);
+                dequant8(wb, sb, Pb);
+                if (WS == 1) {
+                    // two warps share the block: this one owns the product rows made of nibbles 2 hf, 2 hf + 1 (and + 4)
+                    const uint32_t a0 = hf ? Pa[2] : Pa[0], a1 = hf ? Pa[3] : Pa[1], a2 = hf ? Pb[2] : Pb[0], a3 = hf ? Pb[3] : Pb[1];
+                    mma_16816(acc[0][0], a0, a1, a2, a3, b0, b1);
+                    if (two)
+                        mma_16816(acc[0][1], a0, a1, a2, a3, b0h, b1h);
+                } else {
+                    mma_16816(acc[2 * b][0], Pa[0], Pa[1], Pb[0], Pb[1], b0, b1);
+                    mma_16816(acc[2 * b + 1][0], Pa[2], Pa[3], Pb[2], Pb[3], b0, b1);
+                    if (two) {
+                        mma_16816(acc[2 * b][1], Pa[0], Pa[1], Pb[0], Pb[1], b0h, b1h);
+                        mma_16816(acc[2 * b + 1][1], Pa[2], Pa[3], Pb[2], Pb[3], b0h, b1h);
+                    }
+                }
+            }
+        }
+        if (t.stored)
+            bulk_wait_read();         // the slot store has read the stage
+        __syncwarp();
+        if (lane == 0)
+            mbar_arrive(empty0 + 8 * t.st);
+    };
+
+    // ---- the loop, one tile ahead: while the partial sums of tile i travel through shared memory, the warp
+    // computes the gate/up products of tile i + 1, and it forms the down product of tile i after it has handed
+    // on the partial sums of tile i + 1.
+    Q4Tile cur, nxt;
+    float cg[4][4];
+    bool has_cur = take(cur);
+    if (has_cur) {
+        gate_up(cur, cg);
+        store_partials(cg, 0u);
+    }
+    for (uint32_t i = 0; has_cur; ++i) {
+        const bool has_nxt = take(nxt);
+        if (has_nxt)
+            gate_up(nxt, cg);
+        mbar_wait(bar_a, i & 1u, abort_flag);             // every warp's partial sums of tile i are stored
+        column_sums(i & 1u);
+        if (has_nxt)
+            store_partials(cg, (i + 1) & 1u);
+        mbar_wait(bar_b, i & 1u, abort_flag);             // the complete sums of tile i are there
+        down(cur, i & 1u);
+        cur = nxt;
+        has_cur = has_nxt;
     }
     if (trace && tid == 0)
         trace[3] = globaltimer_ns();
     // ---- this CTA's partial output into the call's accumulator (64-bit fixed point, as in the bf16 path).
     // Accumulator i of the warp is the 32-column step hb = warp * WS + i: block hb / 2, and within the
-    // block's 64 columns, column 8 g + 2 (hb mod 2) + {0, 1} for the product's rows g, g + 8, plus 4
-    // for the product's right half (tig >= 2); its columns there are tokens 2 (tig mod 2), + 1.
+    // block's 64 columns (whose codes are stored interleaved: nibble j of word g is column g + 8 j),
+    // column g + 16 (hb mod 2) + {0, 8} for the product's rows g, g + 8, plus 32 for the product's right
+    // half (tig >= 2); its columns there are tokens 2 (tig mod 2), + 1.  Eight lanes of an add are
+    // eight neighbouring columns.
     {
         unsigned long long *yacc = reinterpret_cast<unsigned long long *>(p.yacc);
         auto add = [&](int t, int c, float v) {
             if (t < Tc) {
                 const long long fx = __float2ll_rn(v * 1099511627776.0f);
-                atomicAdd(yacc + (size_t)t * d + c, (unsigned long long)fx);
+                red_add_u64(yacc + (size_t)t * d + c, (unsigned long long)fx);
             }
         };
 #pragma unroll
         for (int i = 0; i < kMaxWs; ++i) {
             if (i < WS) {
                 const int hb = warp * WS + i;
-                const int c = (hb >> 1) * 64 + 8 * g + 2 * (hb & 1) + 4 * (tig >> 1);
+                const int c = (hb >> 1) * 64 + g + 16 * (hb & 1) + 32 * (tig >> 1);
                 const int t = 2 * (tig & 1);
 #pragma unroll
                 for (int tg = 0; tg < 2; ++tg) {
                     if (tg == 0 || two) {
                         add(t + 4 * tg, c, acc[i][tg][0]);
                         add(t + 4 * tg + 1, c, acc[i][tg][1]);
-                        add(t + 4 * tg, c + 1, acc[i][tg][2]);
-                        add(t + 4 * tg + 1, c + 1, acc[i][tg][3]);
+                        add(t + 4 * tg, c + 8, acc[i][tg][2]);
+                        add(t + 4 * tg + 1, c + 8, acc[i][tg][3]);
                     }
                 }
             }
@@ -419,8 +497,8 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_decode_kernel(DecParams p, De
     __shared__ int32_t s_of_expert[kMaxReq];        // request of an expert id (routed 0..E-1, shared E..), -1 = none
     __shared__ int32_t s_idx[kTokPerVr * 32];
     __shared__ float s_gw[kTokPerVr * 32];
-    __shared__ float s_sums[128];
-    __shared__ __align__(8) uint64_t s_bars[2 * kMaxStages + 1];
+    __shared__ float s_sums[256];
+    __shared__ __align__(8) uint64_t s_bars[2 * kMaxStages + 3];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int d = p.d, F = p.F;
@@ -449,6 +527,8 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_decode_kernel(DecParams p, De
             mbar_init(empty0 + 8 * i, NW);
         }
         mbar_init(hzbar, 1);
+        mbar_init(hzbar + 8, NW);
+        mbar_init(hzbar + 16, NW);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     for (int i = tid; i < kMaxReq; i += kThreads) {
@@ -652,7 +732,8 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_decode_kernel(DecParams p, De
         // =================================================================== consumers
         const int g = lane >> 2, tig = lane & 3;
         if constexpr (FMT == 1) {
-            consume_q4<MT_>(p, geo, s_req, &s_gate[0][0], s_sums, buf, ring_s, xs_s, full0, empty0, abort_flag, q_lo, q_hi, trace);
+            consume_q4<MT_>(p, geo, s_req, &s_gate[0][0], s_sums, buf, ring_s, xs_s, full0, empty0, hzbar + 8, hzbar + 16, abort_flag,
+                            q_lo, q_hi, trace);
         } else {
         float acc[kMaxMt][4];
 #pragma unroll
@@ -808,7 +889,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_decode_kernel(DecParams p, De
             unsigned long long *yacc = reinterpret_cast<unsigned long long *>(p.yacc);
             auto add = [&](int t, int c, float v) {
                 const long long fx = __float2ll_rn(v * 1099511627776.0f);    // exact scaling, then to the nearest 2^-40
-                atomicAdd(yacc + (size_t)t * d + c, (unsigned long long)fx);
+                red_add_u64(yacc + (size_t)t * d + c, (unsigned long long)fx);
             };
 #pragma unroll
             for (int mi = 0; mi < kMaxMt; ++mi) {
@@ -908,8 +989,12 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_decode_kernel(DecParams p, De
 }  // namespace
 
 bool ffn_decode_supported(int d, int F) { return d % 256 == 0 && d >= 256 && d <= 4096 && F % kUnitRows == 0; }
-// 4-bit slots: the warps split the columns in steps of 32 (one 16-byte piece of codes), 16 warps.
-bool ffn_decode_supported_q4(int d, int F) { return ffn_decode_supported(d, F) && d % 512 == 0; }
+// 4-bit slots: the warps split the columns in steps of 32 (one 16-byte piece of codes), 16 warps; a warp's
+// steps are 1, 2, 4 or 8 (whole scale groups, or half of one shared by two warps).
+bool ffn_decode_supported_q4(int d, int F)
+{
+    return ffn_decode_supported(d, F) && (d == 512 || d == 1024 || d == 2048 || d == 4096);
+}
 
 cudaError_t ffn_decode_configure(int n_sms, size_t max_smem, DecLaunchCfg *cfg)
 {
@@ -949,7 +1034,7 @@ cudaError_t ffn_decode_geometry(const DecLaunchCfg &cfg, int d, int F, int token
     geo->tokens = tokens;
     // staged hidden rows + the warps' partial tiles; the largest tile (at most 8 rows) of which two
     // stages fit beside them
-    const size_t fixed = (size_t)tokens * geo->x_pitch + (size_t)NW * kBufPitch * sizeof(float);
+    const size_t fixed = (size_t)tokens * geo->x_pitch + (size_t)(fmt == 0 ? 1 : 2) * NW * kBufPitch * sizeof(float);
     int tr = 8;
     for (;; --tr) {
         if (cfg.max_smem >= fixed + (size_t)2 * tr * geo->row_bytes)

@@ -443,7 +443,7 @@ def test_q4_slots_match_the_oracle(d, F, E, k, C, n_shared):
     P.close()
     from paper_2602_11192_b200 import MoELayer
     with pytest.raises(Exception):
-        MoELayer(768, 64, 8, 2, 4, slots="q4")
+        MoELayer(1536, 64, 8, 2, 4, slots="q4")
 
 
 def test_parity_without_programmatic_launch():

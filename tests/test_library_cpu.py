@@ -62,7 +62,7 @@ def test_pack_expert_q4_matches_the_oracle_bit_for_bit(m):
     """The library's host-side quantiser against the oracle's (independent code, same definition).  The
     blob is per hidden unit f: codes of W_g[f], W_u[f], W_d[:, f] (the quantisation groups of W_d run down
     its columns), then the three scale vectors; 16-byte code pieces at (piece xor (f mod 8)) within every
-    eight."""
+    eight; the codes of W_d[:, f] are interleaved within every group of 64 (position p = element 8 (p mod 8) + p // 8)."""
     import oracle
     for d, F in ((256, 24), (512, 64)):
         rs = np.random.default_rng(3)
@@ -83,7 +83,13 @@ def test_pack_expert_q4_matches_the_oracle_bit_for_bit(m):
                 plain = np.empty_like(stored)
                 for piece in range(stored.shape[0]):
                     plain[piece] = stored[(piece & ~7) | ((piece ^ f) & 7)]
-                assert np.array_equal(plain.reshape(-1), codes[f]), (d, f, i)
+                got = plain.reshape(-1)
+                if i == 2:
+                    # W_d[:, f]: within a group of 64, code position p holds element 8 (p mod 8) + p // 8
+                    nib = np.stack([got & 15, got >> 4], axis=1).reshape(-1, 8, 8)       # group, element mod 8, element // 8
+                    nib = nib.transpose(0, 2, 1).reshape(-1, 2)
+                    got = (nib[:, 0] | (nib[:, 1] << 4)).astype(np.uint8)
+                assert np.array_equal(got, codes[f]), (d, f, i)
                 sc = units[f, 3 * (d // 2) + i * (d // 32):3 * (d // 2) + (i + 1) * (d // 32)].view(np.uint16)
                 assert np.array_equal(sc, scales[f]), (d, f, i)
             assert not units[f, 3 * (d // 2) + 3 * (d // 32):].any()      # padding is zeroed
