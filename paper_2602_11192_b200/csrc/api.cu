@@ -966,8 +966,12 @@ int forward_on(melinoe_moe *h, const Scratch &sc, void *cuda_stream, const void 
         }
         if (use_gemm) {
             gp.group = g;
-            CU_TRY(launch_ffn_gemm(s, 1, h->n_sms, gp));
-            CU_TRY(launch_ffn_gemm(s, 2, h->n_sms, gp));
+            // CTA pairs share one weight tile over two m-tiles: worth it where an expert has several m-tiles
+            // (on average at least two here); MELINOE_MOE_GEMM_SINGLE in the environment keeps the single-CTA form
+            static const bool single_only = std::getenv("MELINOE_MOE_GEMM_SINGLE") != nullptr;
+            const bool pairs = !single_only && (long long)T * h->k >= 256ll * h->E;
+            CU_TRY(launch_ffn_gemm(s, 1, h->n_sms, pairs, gp));
+            CU_TRY(launch_ffn_gemm(s, 2, h->n_sms, pairs, gp));
         } else {
             for (int c = 0; c < n_chunks; ++c) {
                 int rc = launch_decode(h, s, sc, hidden_dev, out_dev, T, g, c, g == 0 && c == 0);

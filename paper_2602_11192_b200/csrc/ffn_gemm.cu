@@ -31,6 +31,17 @@
 // Ragged M: an m-tile may run past its expert's last row; those rows are computed on whatever
 // the next rows hold (or zeros past the end of the buffer) and never stored.
 //
+// CTA pairs (template parameter CG = 2, used where the experts have enough tokens): two CTAs of a
+// cluster on neighbouring SMs take two adjacent m-tiles of the same expert and n-tile and run them
+// as ONE tensor-core operation of M = 256 (tcgen05.mma.cta_group::2, issued by the even CTA).  Each
+// CTA stages its own 128 activation rows but only HALF of the weight tile (128 of its 256 columns);
+// the tensor cores of both SMs read both halves.  Per CTA and k-block that is 32 KB instead of 48 KB
+// through shared memory for the same arithmetic, which is what limits the single-CTA form, and the
+// ring holds 6 stages instead of 4.  Both CTAs' loads complete on the even CTA's barrier; its MMA
+// thread frees a stage, and hands over an accumulator, in both CTAs at once (commit with cluster
+// multicast); the odd CTA's epilogue warps report to the even CTA's barrier.  Each CTA drains its own
+// accumulator rows.
+//
 // Every wait is bounded; on a timeout the CTA raises its abort flag, every role leaves its
 // loops, tensor memory is freed and the error word tells the host.
 #include <cuda.h>
@@ -44,8 +55,10 @@ namespace {
 constexpr int kGemmThreads = 192;          // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
 constexpr int kBM = 128, kBK = 64;         // tile rows (tokens), K elements per stage (128 bytes)
 constexpr int kBN = 256;                   // accumulator columns: 128 g + 128 u, or 256 outputs
-constexpr int kStages = 4;
-constexpr int kABytes = kBM * kBK * 2, kBBytes = kBN * kBK * 2, kStageBytes = kABytes + kBBytes;
+constexpr int kABytes = kBM * kBK * 2, kBBytes = kBN * kBK * 2;
+// ring stages and bytes of a stage for the single-CTA form (CG = 1) and the CTA-pair form (CG = 2)
+__host__ __device__ constexpr int gemm_stages(int cg) { return cg == 2 ? 6 : 4; }
+__host__ __device__ constexpr int gemm_stage_bytes(int cg) { return kABytes + kBBytes / cg; }
 constexpr long long kGemmWaitCycles = 4000000000ll;
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -105,6 +118,32 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
         : "memory");
 }
 
+// The same from a CTA of a pair: the completion may be counted on the peer CTA's barrier (bar is an
+// address in the cluster's shared window).
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+// Address of this CTA's shared-memory location `addr` in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t cluster_addr(uint32_t addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 // Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes, groups
 // of 8 rows 1024 bytes apart.
 __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr)
@@ -154,6 +193,24 @@ __device__ __forceinline__ void umma_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
+// The pair forms: one operation over both CTAs' tensor cores; the commit arrives on the barrier at this
+// offset in both CTAs of the pair.
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                               uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"((uint16_t)3)
+                 : "memory");
+}
 
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
 {
@@ -184,14 +241,16 @@ struct GemmItem {
 };
 
 // PHASE 1: h = SiLU(Xs W_g^T) * (Xs W_u^T) -> hs (bf16).  PHASE 2: z = hs W_d^T -> zs (fp32).
-template <int PHASE>
+template <int PHASE, int CG>
 __global__ void __launch_bounds__(kGemmThreads, 1) ffn_gemm_kernel(GemmParams p)
 {
+    constexpr int kStages = gemm_stages(CG), kStageBytes = gemm_stage_bytes(CG);
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     __shared__ uint64_t s_bars[2 * kStages + 4];
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
-    __shared__ int s_req[kMaxReq], s_tile0[kMaxReq + 1], s_nreq;
+    __shared__ int s_tile0[kMaxReq + 1], s_nreq;
+    __shared__ int4 s_rec[kMaxReq];                          // tok_off, n_tok, slot, expert of the launch's requests
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const DevPlan *plan = p.plan;
@@ -203,8 +262,14 @@ __global__ void __launch_bounds__(kGemmThreads, 1) ffn_gemm_kernel(GemmParams p)
     const uint32_t full0 = smem_u32(s_bars), empty0 = full0 + 8 * kStages;
     const uint32_t tfull0 = empty0 + 8 * kStages, tempty0 = tfull0 + 16;
     volatile int *abort_flag = &s_abort;
+    // rank within the CTA pair; the even CTA issues the MMAs, owns the "stage full" barriers and counts
+    // the drained accumulators of both
+    uint32_t rank = 0;
+    if (CG == 2)
+        asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
+    const int n_units = (int)gridDim.x / CG, unit = (int)blockIdx.x / CG;    // CTAs, or CTA pairs, that share out the items
 
-    // ---- the launch's requests and their m-tiles
+    // ---- the launch's requests and their m-tiles (CG = 2: pairs of m-tiles)
     const int K = PHASE == 1 ? p.d : p.F;                 // reduction length
     const int n_tiles_n = PHASE == 1 ? p.F / 128 : p.d / kBN;
     if (tid == 0) {
@@ -214,9 +279,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) ffn_gemm_kernel(GemmParams p)
         for (int r = 0; r < n_req_total; ++r) {
             const ReqRec rec = plan->req[r];
             if (rec.group == p.group && rec.n_tok > 0) {
-                s_req[n] = r;
+                s_rec[n] = make_int4(rec.tok_off, rec.n_tok, rec.slot, rec.expert);
                 s_tile0[n] = tiles;
-                tiles += (rec.n_tok + kBM - 1) / kBM * n_tiles_n;
+                tiles += (rec.n_tok + CG * kBM - 1) / (CG * kBM) * n_tiles_n;
                 ++n;
             }
         }
@@ -228,8 +293,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) ffn_gemm_kernel(GemmParams p)
         }
         mbar_init(tfull0, 1);
         mbar_init(tfull0 + 8, 1);
-        mbar_init(tempty0, 4);
-        mbar_init(tempty0 + 8, 4);
+        mbar_init(tempty0, 4 * CG);
+        mbar_init(tempty0 + 8, 4 * CG);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -238,10 +303,20 @@ __global__ void __launch_bounds__(kGemmThreads, 1) ffn_gemm_kernel(GemmParams p)
     if (total_items == 0)
         return;
 
+    // (the barriers of both CTAs exist before either signals the other's)
+    if (CG == 2)
+        cluster_sync_all();
     if (warp == 2) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)),
-                     "r"(512));
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
+        if (CG == 1) {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)),
+                         "r"(512));
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
+        } else {
+            // the same warp of both CTAs, the same destination: one allocation over the pair
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)),
+                         "r"(512));
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;");
+        }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -254,15 +329,15 @@ __global__ void __launch_bounds__(kGemmThreads, 1) ffn_gemm_kernel(GemmParams p)
         int q = 0;
         while (q + 1 < n_reqs && s_tile0[q + 1] <= w)
             ++q;
-        const ReqRec rec = plan->req[s_req[q]];
+        const int4 rec = s_rec[q];                                  // tok_off, n_tok, slot, expert
         const int local = w - s_tile0[q];
-        const int mtiles = (rec.n_tok + kBM - 1) / kBM;
+        const int mtiles = (rec.y + CG * kBM - 1) / (CG * kBM);
         const int nt = local / mtiles, mt = local % mtiles;
         GemmItem it;
-        it.row0 = rec.tok_off + mt * kBM;
-        it.row_end = rec.tok_off + rec.n_tok;
-        it.shared = rec.slot >= 0 ? -1 : rec.expert - p.E;
-        it.b_row = (rec.slot >= 0 ? rec.slot : 0) * p.F;          // shared experts have maps of their own
+        it.row0 = rec.x + (mt * CG + (int)rank) * kBM;              // this CTA's 128 rows of the item
+        it.row_end = rec.x + rec.y;
+        it.shared = rec.z >= 0 ? -1 : rec.w - p.E;
+        it.b_row = (rec.z >= 0 ? rec.z : 0) * p.F;                  // shared experts have maps of their own
         it.n0 = PHASE == 1 ? nt * 128 : nt * kBN;
         return it;
     };
@@ -273,7 +348,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) ffn_gemm_kernel(GemmParams p)
         if (lane == 0) {
             const CUtensorMap *map_a = p.maps + (PHASE == 1 ? kMapXs : kMapHs);
             uint32_t n = 0;
-            for (int w = blockIdx.x; w < total_items && !*abort_flag; w += gridDim.x) {
+            for (int w = unit; w < total_items && !*abort_flag; w += n_units) {
                 const GemmItem it = item_of(w);
                 // W_g rows, W_u rows, W_d^T rows of the slots, or of the shared expert
                 const CUtensorMap *map_w = it.shared < 0 ? p.maps + kMapSlotsG : p.maps + kMapShared0 + 3 * it.shared;
@@ -281,28 +356,50 @@ __global__ void __launch_bounds__(kGemmThreads, 1) ffn_gemm_kernel(GemmParams p)
                     const uint32_t s = n % kStages;
                     if (n >= (uint32_t)kStages && !mbar_wait(empty0 + 8 * s, ((n / kStages) - 1u) & 1u, abort_flag))
                         break;
-                    const uint32_t bar = full0 + 8 * s;
                     const uint32_t a_dst = ring_s + s * kStageBytes, b_dst = a_dst + kABytes;
-                    mbar_expect(bar, kStageBytes);
-                    tma_load_2d(a_dst, map_a, kb * kBK, it.row0, bar);
-                    if (PHASE == 1) {
-                        tma_load_2d(b_dst, map_w, kb * kBK, it.b_row + it.n0, bar);                   // 128 rows of W_g
-                        tma_load_2d(b_dst + kBBytes / 2, map_w + 1, kb * kBK, it.b_row + it.n0, bar); // 128 rows of W_u
-                    } else {
-                        // 64 rows f of W_d^T, four boxes of 64 output columns
+                    if (CG == 1) {
+                        const uint32_t bar = full0 + 8 * s;
+                        mbar_expect(bar, kStageBytes);
+                        tma_load_2d(a_dst, map_a, kb * kBK, it.row0, bar);
+                        if (PHASE == 1) {
+                            tma_load_2d(b_dst, map_w, kb * kBK, it.b_row + it.n0, bar);                   // 128 rows of W_g
+                            tma_load_2d(b_dst + kBBytes / 2, map_w + 1, kb * kBK, it.b_row + it.n0, bar); // 128 rows of W_u
+                        } else {
+                            // 64 rows f of W_d^T, four boxes of 64 output columns
 #pragma unroll
-                        for (int i = 0; i < kBN / 64; ++i)
-                            tma_load_2d(b_dst + i * 8192, map_w + 2, it.n0 + 64 * i, it.b_row + kb * kBK, bar);
+                            for (int i = 0; i < kBN / 64; ++i)
+                                tma_load_2d(b_dst + i * 8192, map_w + 2, it.n0 + 64 * i, it.b_row + kb * kBK, bar);
+                        }
+                    } else {
+                        // the bytes of both CTAs are expected, once, on the even CTA's barrier
+                        const uint32_t bar = cluster_addr(full0 + 8 * s, 0);
+                        if (rank == 0)
+                            mbar_expect(full0 + 8 * s, 2 * kStageBytes);
+                        tma_load_2d_pair(a_dst, map_a, kb * kBK, it.row0, bar);
+                        if (PHASE == 1) {
+                            // columns 0..127 of the accumulator (g) come from the even CTA's half, 128..255 (u) from the odd one's
+                            tma_load_2d_pair(b_dst, map_w + rank, kb * kBK, it.b_row + it.n0, bar);
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 2; ++i)
+                                tma_load_2d_pair(b_dst + i * 8192, map_w + 2, it.n0 + 64 * (2 * (int)rank + i), it.b_row + kb * kBK, bar);
+                        }
                     }
                 }
             }
+            if (CG == 2) {
+                // The MMA thread's commits arrive on this CTA's barriers from outside: wait for the last
+                // ones so that none is still under way when the CTA ends.
+                for (uint32_t j = n > (uint32_t)kStages ? n - kStages : 0; j < n && !*abort_flag; ++j)
+                    mbar_wait(empty0 + 8 * (j % kStages), (j / kStages) & 1u, abort_flag);
+            }
         }
     } else if (warp == 1) {
-        // ============================================================ MMA issuer
-        if (lane == 0) {
-            const uint32_t idesc = instr_desc_bf16(kBM, kBN, PHASE == 2);
+        // ============================================================ MMA issuer (of a pair: the even CTA's)
+        if (lane == 0 && rank == 0) {
+            const uint32_t idesc = instr_desc_bf16(CG * kBM, kBN, PHASE == 2);
             uint32_t n = 0, item = 0;
-            for (int w = blockIdx.x; w < total_items && !*abort_flag; w += gridDim.x, ++item) {
+            for (int w = unit; w < total_items && !*abort_flag; w += n_units, ++item) {
                 const uint32_t acc = item & 1u;
                 if (item >= 2 && !mbar_wait(tempty0 + 8 * acc, ((item >> 1) - 1u) & 1u, abort_flag))
                     break;
@@ -323,20 +420,32 @@ __global__ void __launch_bounds__(kGemmThreads, 1) ffn_gemm_kernel(GemmParams p)
                     // in an N-major box (128 units)
                     constexpr int kBStep = PHASE == 1 ? 2 : 128;
 #pragma unroll
-                    for (int ks = 0; ks < kBK / 16; ++ks)
-                        umma_bf16(d_tmem, a_desc + 2 * ks, b_desc + kBStep * ks, idesc, (kb | ks) != 0);
-                    umma_commit(empty0 + 8 * s);             // the stage is free once these MMAs have read it
+                    for (int ks = 0; ks < kBK / 16; ++ks) {
+                        if (CG == 1)
+                            umma_bf16(d_tmem, a_desc + 2 * ks, b_desc + kBStep * ks, idesc, (kb | ks) != 0);
+                        else
+                            umma_bf16_pair(d_tmem, a_desc + 2 * ks, b_desc + kBStep * ks, idesc, (kb | ks) != 0);
+                    }
+                    // the stage is free once these MMAs have read it
+                    if (CG == 1)
+                        umma_commit(empty0 + 8 * s);
+                    else
+                        umma_commit_pair(empty0 + 8 * s);
                 }
                 if (!ok)
                     break;
-                umma_commit(tfull0 + 8 * acc);               // the accumulator is complete
+                // the accumulator is complete
+                if (CG == 1)
+                    umma_commit(tfull0 + 8 * acc);
+                else
+                    umma_commit_pair(tfull0 + 8 * acc);
             }
         }
     } else {
         // ============================================================ epilogue (warps 2..5)
         const int quarter = warp & 3;                        // the 32 accumulator rows this warp may read
         uint32_t item = 0;
-        for (int w = blockIdx.x; w < total_items && !*abort_flag; w += gridDim.x, ++item) {
+        for (int w = unit; w < total_items && !*abort_flag; w += n_units, ++item) {
             const GemmItem it = item_of(w);
             const uint32_t acc = item & 1u;
             if (!mbar_wait(tfull0 + 8 * acc, (item >> 1) & 1u, abort_flag))
@@ -384,8 +493,12 @@ __global__ void __launch_bounds__(kGemmThreads, 1) ffn_gemm_kernel(GemmParams p)
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
-            if (lane == 0)
-                mbar_arrive(tempty0 + 8 * acc);
+            if (lane == 0) {
+                if (CG == 1 || rank == 0)
+                    mbar_arrive(tempty0 + 8 * acc);
+                else
+                    mbar_arrive_cluster(cluster_addr(tempty0 + 8 * acc, 0));
+            }
         }
     }
 
@@ -393,8 +506,15 @@ __global__ void __launch_bounds__(kGemmThreads, 1) ffn_gemm_kernel(GemmParams p)
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    if (warp == 2)
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512));
+    // (a pair: neither CTA goes while the other may still signal it or read its shared memory)
+    if (CG == 2)
+        cluster_sync_all();
+    if (warp == 2) {
+        if (CG == 1)
+            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512));
+        else
+            asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512));
+    }
     if (*abort_flag && tid == 0)
         atomicExch(p.err, MELINOE_ERR_TIMEOUT);
 }
@@ -448,7 +568,7 @@ __global__ void __launch_bounds__(256) combine_rows_kernel(const DevPlan *plan, 
     }
 }
 
-constexpr size_t kGemmSmem = (size_t)kStages * kStageBytes + 1024;
+constexpr size_t gemm_smem(int cg) { return (size_t)gemm_stages(cg) * gemm_stage_bytes(cg) + 1024; }
 
 }  // namespace
 
@@ -456,10 +576,14 @@ bool ffn_gemm_supported(int d, int F) { return d % kBN == 0 && F % 128 == 0 && d
 
 cudaError_t ffn_gemm_configure()
 {
-    cudaError_t e = cudaFuncSetAttribute(ffn_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmem);
-    if (e != cudaSuccess)
-        return e;
-    return cudaFuncSetAttribute(ffn_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmem);
+    cudaError_t e = cudaFuncSetAttribute(ffn_gemm_kernel<1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem(1));
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(ffn_gemm_kernel<2, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem(1));
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(ffn_gemm_kernel<1, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem(2));
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(ffn_gemm_kernel<2, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem(2));
+    return e;
 }
 
 cudaError_t launch_gather_rows(cudaStream_t stream, const DevPlan *plan, const uint16_t *x, const int32_t *tok_of_sorted,
@@ -471,14 +595,32 @@ cudaError_t launch_gather_rows(cudaStream_t stream, const DevPlan *plan, const u
     return cudaGetLastError();
 }
 
-cudaError_t launch_ffn_gemm(cudaStream_t stream, int phase, int n_sms, const GemmParams &p)
+cudaError_t launch_ffn_gemm(cudaStream_t stream, int phase, int n_sms, bool pairs, const GemmParams &p)
 {
-    if (phase == 1)
-        ffn_gemm_kernel<1><<<n_sms, kGemmThreads, kGemmSmem, stream>>>(p);
-    else
-        ffn_gemm_kernel<2><<<n_sms, kGemmThreads, kGemmSmem, stream>>>(p);
+    if (!pairs) {
+        if (phase == 1)
+            ffn_gemm_kernel<1, 1><<<n_sms, kGemmThreads, gemm_smem(1), stream>>>(p);
+        else
+            ffn_gemm_kernel<2, 1><<<n_sms, kGemmThreads, gemm_smem(1), stream>>>(p);
+        count_launch();
+        return cudaGetLastError();
+    }
+    // clusters of two CTAs on neighbouring SMs
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3(n_sms / 2 * 2);
+    lc.blockDim = dim3(kGemmThreads);
+    lc.dynamicSmemBytes = gemm_smem(2);
+    lc.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    const cudaError_t e = phase == 1 ? cudaLaunchKernelEx(&lc, ffn_gemm_kernel<1, 2>, p) : cudaLaunchKernelEx(&lc, ffn_gemm_kernel<2, 2>, p);
     count_launch();
-    return cudaGetLastError();
+    return e;
 }
 
 cudaError_t launch_combine_rows(cudaStream_t stream, const DevPlan *plan, const float *gate, const int32_t *inv_pos,

@@ -128,7 +128,7 @@ bool ffn_gemm_supported(int d, int F);
 cudaError_t ffn_gemm_configure();
 cudaError_t launch_gather_rows(cudaStream_t stream, const DevPlan *plan, const uint16_t *x, const int32_t *tok_of_sorted,
                                uint16_t *xs, int d, int n_sorted, int n_sms);
-cudaError_t launch_ffn_gemm(cudaStream_t stream, int phase, int n_sms, const GemmParams &p);
+cudaError_t launch_ffn_gemm(cudaStream_t stream, int phase, int n_sms, bool pairs, const GemmParams &p);
 cudaError_t launch_combine_rows(cudaStream_t stream, const DevPlan *plan, const float *gate, const int32_t *inv_pos,
                                 const float *zs, uint16_t *out, int T, int d, int k, int n_shared, int n_sms);
 

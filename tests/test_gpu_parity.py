@@ -142,6 +142,7 @@ def test_prefill_then_decode_with_waves():
     (1024, 384, 6, 2, 3, 2, (257, 20)),          # shared experts, ragged last m-tile
     (512, 256, 4, 2, 4, 0, (600, 385, 40)),      # many tokens per expert, ragged
     (1024, 384, 4, 2, 2, 1, (700,)),             # many tokens per expert with a shared expert and miss waves
+    (256, 256, 2, 2, 2, 0, (1100, 520)),         # every token to both experts: nine m-tiles (CTA pairs, the last one half empty)
 ])
 def test_prefill_grouped_gemm(d, F, E, k, C, n_shared, Ts):
     """Calls of more than 8 tokens run the tensor-core grouped GEMM (d_ff a multiple of 128)."""
