@@ -27,9 +27,10 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the decode FFN kernel divided by the launch's
-# algorithmic bytes (8 experts x 12.58 MB), from an ncu capture of a two-layer case of this workload; traffic
-# grows in proportion to the experts streamed.  None until the counters have been taken for the current kernel.
-DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE = None
+# algorithmic bytes (8 experts x 12.58 MB), from an ncu capture of a two-layer case of this workload (100.75 MB
+# read + 3.5 MB written against 100.66 MB); traffic grows in proportion to the experts streamed.  To be set to
+# None when the kernel changes, until the counters have been taken again.
+DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.036
 
 METRIC = "decode tokens/s (OLMoE-shaped, cache-limited)"
 UNIT = "tokens/s"
@@ -56,6 +57,13 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--alpha", type=float, default=None, help="headline router-bias concentration (default: the workload's first)")
     ap.add_argument("--layers", type=int, default=None, help="use fewer layers (debugging only; marks the line)")
+    ap.add_argument("--store", default="bf16", choices=["bf16", "q4", "q4slots"],
+                    help="expert format of the headline run (profiling aid; anything but bf16 marks the line): "
+                         "q4 = 4-bit host store expanded into bf16 slots, q4slots = 4-bit store and 4-bit slots")
+    ap.add_argument("--slots", type=int, default=None, help="cache slots per layer of the headline run (marks the line)")
+    ap.add_argument("--shape", default=None, choices=["mixtral", "phi35", "deepseek"],
+                    help="profiling aid: run only that workload shape's record (decode, FFN analysis, prefill GEMM) on "
+                         "--layers layers (default 1), print it and exit; not a benchmark line")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extra", action="store_true", help="skip the other alphas and the resident-cache run")
     return ap.parse_args()
@@ -463,12 +471,12 @@ def run_ours(args):
     import paper_2602_11192_b200 as M
 
     cfg = gen.config_by_name(WORKLOAD)
-    C = cfg.cache_slots[0]
+    C = cfg.cache_slots[0] if args.slots is None else args.slots
     alpha0 = cfg.alphas[0] if args.alpha is None else args.alpha
     L = cfg.n_layers if args.layers is None else args.layers
     K, W = args.steps, args.warmup
     d = cfg.d_model
-    B_e = cfg.expert_bytes
+    B_e = cfg.expert_bytes if args.store != "q4slots" else M.melinoe_moe_expert_bytes_q4(cfg.d_model, cfg.d_ff)
     peaks = {}
     try:
         peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
@@ -476,9 +484,13 @@ def run_ours(args):
         pass
     hbm_peak = float(peaks.get("hbm_gbs", 6650.0))
     peak_src = "measured" if "hbm_gbs" in peaks else "fallback"
+    if args.shape is not None:
+        rec = shape_record(torch, M, gen, args.shape, args.layers or 1, min(K, 64), W, hbm_peak, host_link_gbs(torch), peaks)
+        print(json.dumps({"shape_only": args.shape, "record": rec}), flush=True)
+        return
 
     phase("building the stack: %d layers x %d experts x %.1f MB in pinned host memory" % (L, cfg.n_experts, B_e / 1e6))
-    R = Runner(torch, M, gen, cfg, alpha0, C, L, K, W, dist=dist)
+    R = Runner(torch, M, gen, cfg, alpha0, C, L, K, W, store=args.store, dist=dist)
 
     gpu_index = local
     vis = os.environ.get("CUDA_VISIBLE_DEVICES")
@@ -517,7 +529,7 @@ def run_ours(args):
     phase("same region with per-launch events around the FFN kernel")
     link_peak = host_link_gbs(torch)
     _, _, st2, per_launch = R.timed_device(alpha0, with_kernel_timing=True)
-    ana = ffn_launch_analysis(cfg, st2, per_launch, hbm_peak, link_peak)
+    ana = ffn_launch_analysis(cfg, st2, per_launch, hbm_peak, link_peak, expert_bytes=B_e)
     res = ana["resident"] if ana and ana["resident"] else {"gbs": 0.0, "launches": 0, "avg_launch_us": None, "bytes_per_launch": 0.0}
     roofline = {"bound": "hbm", "kernel": "ffn_decode_kernel", "achieved": res["gbs"], "peak": hbm_peak, "unit": "GB/s",
                 "frac": res["gbs"] / hbm_peak, "peak_source": peak_src,
@@ -639,6 +651,10 @@ def run_ours(args):
         }
         if args.layers is not None:
             line["config"]["reduced_layers"] = True
+        if args.store != "bf16":
+            line["config"]["store"] = args.store
+        if args.slots is not None:
+            line["config"]["slots_override"] = args.slots
         print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
