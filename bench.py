@@ -601,6 +601,7 @@ def run_ours(args):
                 med, best = med_best(vals)
                 rec = {"value": med, "best": best, "cache_slots": Cq, "slot_bytes": qb, "slot_memory_bytes_per_layer": Cq * qb,
                        "bf16_slot_memory_bytes_per_layer": C * cfg.expert_bytes, **hit_summary(cfg, st_s, K, L)}
+                rec["h2d_expert_bytes_per_step"] = float(st_s["misses"].sum()) * qb / K
                 if ana_s and ana_s["resident"]:
                     r_ = ana_s["resident"]
                     rec["ffn_resident"] = {"launches": r_["launches"], "avg_launch_us": r_["avg_launch_us"], "gbs_4bit": r_["gbs"],
