@@ -327,9 +327,10 @@ __device__ __forceinline__ void consume_q4(const DecParams &p, const DecGeometry
     };
     // The warps' partial tiles meet in shared memory: every warp stores its 128 partial values, warp w sums
     // 8 of the 128 over all warps (four lanes per value, each adding four warps' parts in warp order, then a
-    // fixed tree), and every warp reads the complete tile.  Two sets of buffers and two counting barriers
-    // (all warps have stored / all sums are there) let a warp do other work between arriving at a barrier
-    // and needing what it guards: the loop below is arranged so that it always has some.
+    // fixed tree), and every warp reads the complete tile.  Two counting barriers order this (all warps
+    // have stored / all sums are there); the buffers alternate from tile to tile.  (Running the loop one tile
+    // ahead, so that a warp has other work between arriving at a barrier and needing what it guards, was
+    // measured and made no difference: this path is bound by instruction issue, not by waiting.)
     auto store_partials = [&](const float (&cg)[4][4], uint32_t sel) {
         float *b = buf + sel * (NW * kBufPitch) + warp * kBufPitch;
 #pragma unroll
@@ -422,28 +423,15 @@ __device__ __forceinline__ void consume_q4(const DecParams &p, const DecGeometry
             mbar_arrive(empty0 + 8 * t.st);
     };
 
-    // ---- the loop, one tile ahead: while the partial sums of tile i travel through shared memory, the warp
-    // computes the gate/up products of tile i + 1, and it forms the down product of tile i after it has handed
-    // on the partial sums of tile i + 1.
-    Q4Tile cur, nxt;
+    Q4Tile cur;
     float cg[4][4];
-    bool has_cur = take(cur);
-    if (has_cur) {
+    for (uint32_t i = 0; take(cur); ++i) {
         gate_up(cur, cg);
-        store_partials(cg, 0u);
-    }
-    for (uint32_t i = 0; has_cur; ++i) {
-        const bool has_nxt = take(nxt);
-        if (has_nxt)
-            gate_up(nxt, cg);
-        mbar_wait(bar_a, i & 1u, abort_flag);             // every warp's partial sums of tile i are stored
+        store_partials(cg, i & 1u);
+        mbar_wait(bar_a, i & 1u, abort_flag);             // every warp's partial sums of the tile are stored
         column_sums(i & 1u);
-        if (has_nxt)
-            store_partials(cg, (i + 1) & 1u);
-        mbar_wait(bar_b, i & 1u, abort_flag);             // the complete sums of tile i are there
+        mbar_wait(bar_b, i & 1u, abort_flag);             // the complete sums of the tile are there
         down(cur, i & 1u);
-        cur = nxt;
-        has_cur = has_nxt;
     }
     if (trace && tid == 0)
         trace[3] = globaltimer_ns();
