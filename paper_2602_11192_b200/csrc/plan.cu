@@ -172,11 +172,11 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p)
                 s_miss_expert[rank_below(miss_mask, e)] = e;
         }
         __syncwarp();
-        // V: rank of each slot among the keys (keys are distinct)
+        // V: rank of each slot among the keys (keys are distinct); only misses under LRU take victims from it
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             const int sl = lane + 32 * h;
-            if (sl < C) {
+            if (sl < C && n_miss > 0 && p.policy != MELINOE_POLICY_COUNT) {
                 const uint64_t mine = s_key[sl];
                 int r = 0;
 #pragma unroll 8

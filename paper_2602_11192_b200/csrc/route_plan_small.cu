@@ -429,11 +429,11 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
             s_miss_expert[rank_below(miss_mask, e)] = e;
     }
     __syncwarp();
-    // V: rank of each slot among the keys (keys are distinct)
+    // V: rank of each slot among the keys (keys are distinct); only misses take victims
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
         const int s = lane + 32 * h;
-        if (s < C) {
+        if (s < C && n_miss > 0 && !by_count) {
             const unsigned long long mine = s_key[s];
             int r = 0;
 #pragma unroll 8
@@ -599,12 +599,11 @@ route_plan_small_kernel(const uint16_t *__restrict__ x, const uint16_t *__restri
     }
     // The plan is complete: announce it.  The decode FFN kernel behind this one in the stream may
     // already be running (programmatic launch) and waits for this word, not for this grid to drain.
-    // (The barrier orders the other warps' and lanes' writes before lane 0's release.)
+    // (The barrier orders the other warps' and lanes' writes before lane 0's release, which is cumulative:
+    // whoever acquires the word sees them all.)
     asm volatile("bar.sync 2, %0;" ::"n"(kThreads) : "memory");
-    if (lane == 0) {
-        __threadfence();
+    if (lane == 0)
         asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(&plan->ready_seq), "r"(p.call_seq) : "memory");
-    }
     // What may live in host memory goes out last, so that no fence above has to wait for the host link:
     // the statistics, and the miss queue for calls whose transfers the host issues.
     for (int i = lane; i < n_miss; i += 32)
