@@ -239,8 +239,7 @@ struct Q4Tile {
 template <int MT_>
 __device__ __forceinline__ void consume_q4(const DecParams &p, const DecGeometry &geo, const SReq *s_req, const float *s_gate,
                                            float *s_sums, float *buf, uint32_t ring_s, uint32_t xs_s, uint32_t full0,
-                                           uint32_t empty0, uint32_t bar_a, uint32_t bar_b, volatile int *abort_flag,
-                                           long long q_lo, long long q_hi, unsigned long long *trace)
+                                           uint32_t empty0, volatile int *abort_flag, long long q_lo, long long q_hi, unsigned long long *trace)
 {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, tig = lane & 3;
     const int d = p.d, F = p.F;
@@ -327,18 +326,16 @@ __device__ __forceinline__ void consume_q4(const DecParams &p, const DecGeometry
     };
     // The warps' partial tiles meet in shared memory: every warp stores its 128 partial values, warp w sums
     // 8 of the 128 over all warps (four lanes per value, each adding four warps' parts in warp order, then a
-    // fixed tree), and every warp reads the complete tile.  Two counting barriers order this (all warps
-    // have stored / all sums are there); the buffers alternate from tile to tile.  (Running the loop one tile
-    // ahead, so that a warp has other work between arriving at a barrier and needing what it guards, was
-    // measured and made no difference: this path is bound by instruction issue, not by waiting.)
+    // fixed tree), and every warp reads the complete tile.  Two block-wide named barriers order this; the
+    // buffers alternate from tile to tile.  (Measured and dropped: counting mbarriers in their place, with
+    // the loop running one tile ahead so that a warp has other work between arriving and waiting -- the
+    // hardware barrier is the cheaper way for 16 warps to meet; and h formed once per tile by the summing
+    // warps instead of by every warp for itself -- it lengthens the path between the two barriers.)
     auto store_partials = [&](const float (&cg)[4][4], uint32_t sel) {
         float *b = buf + sel * (NW * kBufPitch) + warp * kBufPitch;
 #pragma unroll
         for (int i = 0; i < 4; ++i)
             b[i * 32 + lane] = (cg[0][i] + cg[1][i]) + (cg[2][i] + cg[3][i]);
-        __syncwarp();
-        if (lane == 0)
-            mbar_arrive(bar_a);
     };
     auto column_sums = [&](uint32_t sel) {
         const float *b = buf + sel * (NW * kBufPitch);
@@ -351,9 +348,6 @@ __device__ __forceinline__ void consume_q4(const DecParams &p, const DecGeometry
         v += __shfl_xor_sync(0xffffffffu, v, 16);
         if (lane < 8)
             s_sums[sel * 128 + e] = v;
-        __syncwarp();
-        if (lane == 0)
-            mbar_arrive(bar_b);
     };
     // ---- h of the tile from the complete sums, then the down product
     auto down = [&](const Q4Tile &t, uint32_t sel) {
@@ -428,9 +422,9 @@ __device__ __forceinline__ void consume_q4(const DecParams &p, const DecGeometry
     for (uint32_t i = 0; take(cur); ++i) {
         gate_up(cur, cg);
         store_partials(cg, i & 1u);
-        mbar_wait(bar_a, i & 1u, abort_flag);             // every warp's partial sums of the tile are stored
+        asm volatile("bar.sync 1, %0;" ::"n"(NW * 32) : "memory");      // every warp's partial sums of the tile are stored
         column_sums(i & 1u);
-        mbar_wait(bar_b, i & 1u, abort_flag);             // the complete sums of the tile are there
+        asm volatile("bar.sync 1, %0;" ::"n"(NW * 32) : "memory");      // the complete sums of the tile are there
         down(cur, i & 1u);
     }
     if (trace && tid == 0)
@@ -486,7 +480,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_decode_kernel(DecParams p, De
     __shared__ int32_t s_idx[kTokPerVr * 32];
     __shared__ float s_gw[kTokPerVr * 32];
     __shared__ float s_sums[256];
-    __shared__ __align__(8) uint64_t s_bars[2 * kMaxStages + 3];
+    __shared__ __align__(8) uint64_t s_bars[2 * kMaxStages + 1];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int d = p.d, F = p.F;
@@ -515,8 +509,6 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_decode_kernel(DecParams p, De
             mbar_init(empty0 + 8 * i, NW);
         }
         mbar_init(hzbar, 1);
-        mbar_init(hzbar + 8, NW);
-        mbar_init(hzbar + 16, NW);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     for (int i = tid; i < kMaxReq; i += kThreads) {
@@ -720,8 +712,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_decode_kernel(DecParams p, De
         // =================================================================== consumers
         const int g = lane >> 2, tig = lane & 3;
         if constexpr (FMT == 1) {
-            consume_q4<MT_>(p, geo, s_req, &s_gate[0][0], s_sums, buf, ring_s, xs_s, full0, empty0, hzbar + 8, hzbar + 16, abort_flag,
-                            q_lo, q_hi, trace);
+            consume_q4<MT_>(p, geo, s_req, &s_gate[0][0], s_sums, buf, ring_s, xs_s, full0, empty0, abort_flag, q_lo, q_hi, trace);
         } else {
         float acc[kMaxMt][4];
 #pragma unroll
