@@ -395,13 +395,14 @@ def preload_record(torch, R, cfg, alpha, C, L, n_steps):
     return out
 
 
-def shape_record(torch, M, gen, name, n_layers, K, W, hbm_peak, link_peak, peaks):
+def shape_record(torch, M, gen, name, n_layers, K, W, hbm_peak, link_peak, peaks, store="bf16"):
     """Decode throughput, FFN roofline and (where the prompt runs the grouped GEMM) the prefill GEMM's
     rate of one of the other workload shapes, at its full width with a reduced number of layers."""
     cfg = gen.config_by_name(name)
     C, alpha = cfg.cache_slots[0], cfg.alphas[0]
-    R = Runner(torch, M, gen, cfg, alpha, C, n_layers, K, W)
-    rec = {"workload": "%s-shaped: d_model=%d, d_ff=%d, %d experts (+%d shared), top-%d, cache %d/layer, batch %d, "
+    eb = M.melinoe_moe_expert_bytes_q4(cfg.d_model, cfg.d_ff) if store == "q4slots" else cfg.expert_bytes
+    R = Runner(torch, M, gen, cfg, alpha, C, n_layers, K, W, store=store)
+    rec = {"store": store, "slot_bytes": eb, "workload": "%s-shaped: d_model=%d, d_ff=%d, %d experts (+%d shared), top-%d, cache %d/layer, batch %d, "
                        "%d-token prompts, alpha=%g" % (name, cfg.d_model, cfg.d_ff, cfg.n_experts, cfg.n_shared, cfg.top_k, C,
                                                        cfg.batch, cfg.prefill_tokens, alpha),
            "layers": n_layers, "reduced_layers": n_layers != cfg.n_layers, "decode_steps": K}
@@ -412,13 +413,13 @@ def shape_record(torch, M, gen, name, n_layers, K, W, hbm_peak, link_peak, peaks
     rec["tokens_per_s_median"], rec["tokens_per_s_best"] = med_best(vals)
     rec.update(hit_summary(cfg, st, K, n_layers))
     _, _, st2, per_launch = R.timed_device(alpha, with_kernel_timing=True)
-    rec["ffn"] = ffn_launch_analysis(cfg, st2, per_launch, hbm_peak, link_peak)
+    rec["ffn"] = ffn_launch_analysis(cfg, st2, per_launch, hbm_peak, link_peak, expert_bytes=eb)
     if R.copy_ms > 0:
         g = R.copy_bytes / (R.copy_ms * 1e-3) / 1e9
         rec["host_issued_transfers"] = {"gbs": g, "frac_of_link": g / link_peak, "bytes": R.copy_bytes,
                                         "note": "cudaMemcpyAsync waves on the copy stream, events around each wave"}
     # the prompt again with events around the grouped GEMM launches of every compute group
-    if cfg.prefill_tokens and cfg.d_ff % 128 == 0 and cfg.batch * cfg.prefill_tokens > 8:
+    if cfg.prefill_tokens and cfg.d_ff % 128 == 0 and cfg.batch * cfg.prefill_tokens > 8 and store != "q4slots":
         R.prepare(alpha, timing_prefill=True)
         ms_sum, n = 0.0, 0
         for ls in R.stack.layers:
@@ -440,10 +441,10 @@ def shape_record(torch, M, gen, name, n_layers, K, W, hbm_peak, link_peak, peaks
                                        "GEMM launches of every compute group, transfers excluded"}
     R.close()
     # the same shape with every expert resident: the decode kernel in its HBM-bound regime
-    Ra = Runner(torch, M, gen, cfg, alpha, cfg.n_experts, n_layers, K, W)
+    Ra = Runner(torch, M, gen, cfg, alpha, cfg.n_experts, n_layers, K, W, store=store)
     Ra.timed_device(alpha)                                           # warm: the first pass fetches what the prompt did not
     _, _, st3, pl3 = Ra.timed_device(alpha, with_kernel_timing=True)
-    a3 = ffn_launch_analysis(cfg, st3, pl3, hbm_peak, link_peak)
+    a3 = ffn_launch_analysis(cfg, st3, pl3, hbm_peak, link_peak, expert_bytes=eb)
     rec["ffn_all_resident"] = a3["resident"] if a3 else None
     Ra.close()
     return rec
@@ -485,7 +486,8 @@ def run_ours(args):
     hbm_peak = float(peaks.get("hbm_gbs", 6650.0))
     peak_src = "measured" if "hbm_gbs" in peaks else "fallback"
     if args.shape is not None:
-        rec = shape_record(torch, M, gen, args.shape, args.layers or 1, min(K, 64), W, hbm_peak, host_link_gbs(torch), peaks)
+        rec = shape_record(torch, M, gen, args.shape, args.layers or 1, min(K, 64), W, hbm_peak, host_link_gbs(torch), peaks,
+                           store=args.store)
         print(json.dumps({"shape_only": args.shape, "record": rec}), flush=True)
         return
 
