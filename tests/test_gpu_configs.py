@@ -14,24 +14,27 @@ import pytest
 
 import gen
 import oracle
-from parity_util import elementwise_excess
+from parity_util import _q4_roundtrip, elementwise_excess
 
 pytestmark = pytest.mark.gpu
 
 REL_TOL = 2e-2          # the specified bound at full size
 
 
-def _run_stack(name, n_layers, alpha, C, decode_steps, sample_layers, prefill=True, y_tokens=8):
+def _run_stack(name, n_layers, alpha, C, decode_steps, sample_layers, prefill=True, y_tokens=8, store="bf16"):
     import torch
     from paper_2602_11192_b200.workload import Stack, bits_of, stats_rows
     cfg = gen.config_by_name(name)
-    st = Stack(cfg, alpha, C, n_layers=n_layers)
+    st = Stack(cfg, alpha, C, n_layers=n_layers, store=store)
     L, B, k, E, d = st.L, cfg.batch, cfg.top_k, cfg.n_experts, cfg.d_model
     caches = [oracle.ExpertCache(C, E) for _ in range(L)]
     weights = {}
     for l in sample_layers:
         wg, wu, wd = st.layer_weights(l)
-        weights[l] = ([(bits_of(wg[e]), bits_of(wu[e]), bits_of(wd[e])) for e in range(E + cfg.n_shared)], (wg, wu, wd))
+        ws = [(bits_of(wg[e]), bits_of(wu[e]), bits_of(wd[e])) for e in range(E + cfg.n_shared)]
+        if store == "q4slots":
+            ws = [_q4_roundtrip(w) for w in ws]        # the weights the 4-bit format defines
+        weights[l] = (ws, (wg, wu, wd))
 
     def check(phase, step, T, seq):
         x = st.hidden_bits(phase, step)                                  # [L][T][d]
@@ -55,7 +58,7 @@ def _run_stack(name, n_layers, alpha, C, decode_steps, sample_layers, prefill=Tr
             hits = int(req_o[:, 2].sum())
             assert sr["status"][l] == 0 and sr["n_distinct"][l] == len(req_o)
             assert sr["hits"][l] == hits and sr["misses"][l] == len(req_o) - hits
-            assert layer.last_call_used_gemm() == (T > 8 and cfg.d_ff % 128 == 0)
+            assert layer.last_call_used_gemm() == (T > 8 and cfg.d_ff % 128 == 0 and store == "bf16")
             if l in weights:
                 toks = sorted(set(np.linspace(0, T - 1, min(T, y_tokens)).astype(int).tolist()))
                 y = oracle.ffn_combine(x[l], idx_o, gate_o, weights[l][0], cfg.d_ff, cfg.n_shared, toks)
@@ -108,6 +111,18 @@ def test_deepseek_shape_with_shared_experts(alpha):
     """configs[4]: d 2048, d_ff 1408, 64 routed + 2 shared experts, top-6, 12 slots, 4 sequences:
     8192-token prefill, then 32 decode steps of 4 tokens; 4 of the 28 layers."""
     _run_stack("deepseek", 4, alpha, 12, decode_steps=32, sample_layers=(3,), y_tokens=8)
+
+
+@pytest.mark.parametrize("name,n_layers,alpha,C,steps,prefill", [
+    ("olmoe", 4, 0.1, 16, 32, True),          # d 2048; the 128-token prompt runs as 16 launches of 8 tokens
+    ("mixtral", 2, 0.2, 4, 16, False),        # d 4096, one token
+    ("phi35", 2, 0.3, 6, 16, False),          # d 4096, eight tokens (both token groups of the down product)
+    ("deepseek", 2, 0.1, 12, 16, False),      # shared experts (4-bit as well), four tokens
+])
+def test_four_bit_slots_at_full_width(name, n_layers, alpha, C, steps, prefill):
+    """The workload shapes with 4-bit cache slots (codes expanded inside the FFN kernel): routing, traces and
+    statistics bit for bit, activations element-wise against the oracle on the weights the format defines."""
+    _run_stack(name, n_layers, alpha, C, decode_steps=steps, sample_layers=(n_layers - 1,), prefill=prefill, store="q4slots")
 
 
 def test_per_layer_budget_end_to_end_makes_fewer_transfers():
