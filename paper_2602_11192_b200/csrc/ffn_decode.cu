@@ -17,7 +17,7 @@
 //     of shared-memory banks (the xor), so the tensor-core fragment loads (ldmatrix) are free of
 //     bank conflicts although the rows sit at a pitch that is a multiple of 128 bytes.
 //
-// One CTA per SM: NW consumer warps (8 for d <= 2048, else 16) and one producer warp.
+// One CTA per SM: 16 consumer warps and one producer warp.
 //   producer  one thread; per tile (up to 8 rows f of one expert) one cp.async.bulk into a ring
 //             stage, completion on the stage's mbarrier.  A missed expert's rows come straight from
 //             the page-locked host store (the device reads host memory over the link).
@@ -40,11 +40,12 @@
 //             itself out on the handle's counter and exits; the CTA that finds all the others gone
 //             converts the sums to bf16, writes the output and clears accumulator and counter.  No CTA
 //             ever waits for another.
+//   4-bit     the same structure on 4-bit blobs (melinoe_moe_pack_expert_q4): the codes are expanded in
+//   blobs     registers on their way into the tensor-core fragments, see consume_q4 below.
 //
 // Every wait is bounded: when an mbarrier or the wait for the plan does not complete in time the warp
 // raises the CTA's abort flag, later waits fall through, copies in flight are given a bounded time
 // to land, the kernel ends normally and the error word tells the host.
-#include <cstdlib>
 
 #include "kernels.cuh"
 
@@ -200,7 +201,7 @@ struct SReq {
     const char *src;      // where its rows are streamed from: the slot, a shared expert's blob, or the host store
     char *wb;             // null, or the slot the fetched rows are also stored into
     int32_t gate_row;     // its row of the gate table (= its index among the launch's requests)
-    int32_t deferred;     // the slot is written only after the grid barrier (it is still being computed with)
+    int32_t deferred;     // the slot is written by the last CTA once every CTA is done (it is still being computed with)
 };
 
 constexpr int NW = 16;                           // consumer warps
@@ -1035,22 +1036,15 @@ cudaError_t ffn_decode_geometry(const DecLaunchCfg &cfg, int d, int F, int token
 cudaError_t launch_ffn_decode(cudaStream_t stream, const DecLaunchCfg &cfg, const DecGeometry &geo, const DecParams &p)
 {
     // Programmatic stream serialisation: the CTAs may be scheduled, and set up their barriers, while the
-    // kernel ahead in the stream is still draining; the kernel waits for it before it reads the plan.
-    // All CTAs are resident at once (one per SM, the grid is the SM count), which the grid barrier at
-    // the end relies on; MELINOE_MOE_COOP in the environment asks the driver to guarantee it.
-    static const bool coop = std::getenv("MELINOE_MOE_COOP") != nullptr;
+    // kernel ahead in the stream is still running; the kernel waits for the plan word before it reads
+    // anything that kernel writes.  No CTA waits for another, so nothing depends on co-residency.
     cudaLaunchConfig_t lc = {};
     lc.gridDim = dim3(cfg.grid);
     lc.blockDim = dim3(kThreads);
     lc.dynamicSmemBytes = geo.smem_bytes;
     lc.stream = stream;
-    cudaLaunchAttribute attr[2];
+    cudaLaunchAttribute attr[1];
     int na = 0;
-    if (coop) {
-        attr[na].id = cudaLaunchAttributeCooperative;
-        attr[na].val.cooperative = 1;
-        ++na;
-    }
     if (cfg.pdl) {
         attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[na].val.programmaticStreamSerializationAllowed = 1;
