@@ -15,10 +15,14 @@
  *    be ordered with respect to each other on the device (same stream, or caller-made
  *    dependencies): a call's cache decisions depend on the previous call's.
  *  - melinoe_moe_forward is asynchronous with respect to the host: for calls of at most 8 tokens
- *    on a bf16 host store it queues two kernels and returns (the missed experts are fetched by the
+ *    (and no more token-expert pairs than cache slots) it queues two kernels and returns (the missed experts are fetched by the
  *    compute kernel itself); otherwise it returns once the call's cache decisions are known to
  *    the host and all of its transfers and kernels are queued.  It never waits for transfers or
  *    compute.
+ *  - Environment switches, read once per process (for measurements and tests; none changes results):
+ *    MELINOE_MOE_NO_PDL          launch the decode kernels without programmatic stream serialisation;
+ *    MELINOE_MOE_HOST_COPIES     every expert transfer is a cudaMemcpyAsync issued by the host;
+ *    MELINOE_MOE_GEMM_SINGLE     the prefill GEMM never pairs CTAs (tcgen05 cta_group::1 only).
  */
 #ifndef MELINOE_MOE_H_
 #define MELINOE_MOE_H_

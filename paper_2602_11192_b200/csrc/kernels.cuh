@@ -92,8 +92,8 @@ struct DecLaunchCfg {
 };
 // Shape of the shared-memory ring for one launch.
 struct DecGeometry {
-    int n_warps;                     // consumer warps: 8 (d <= 2048) or 16
-    int tile_rows;                   // f rows per tile / ring stage: at most 8
+    int n_warps;                     // consumer warps (16)
+    int tile_rows;                   // f rows per tile = ring stage: at most 8
     int n_stages;
     int row_bytes;                   // bytes of one f row of the blob (its W_g, W_u and W_d^T rows)
     int stage_bytes;
