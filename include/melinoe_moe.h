@@ -15,8 +15,8 @@
  *    be ordered with respect to each other on the device (same stream, or caller-made
  *    dependencies): a call's cache decisions depend on the previous call's.
  *  - melinoe_moe_forward is asynchronous with respect to the host: for calls of at most 8 tokens
- *    (and no more token-expert pairs than cache slots) it queues two kernels and returns (the missed experts are fetched by the
- *    compute kernel itself); otherwise it returns once the call's cache decisions are known to
+ *    (and no more token-expert pairs than cache slots) it queues two kernels and returns (the
+ *    missed experts are fetched by the compute kernel itself); otherwise it returns once the call's cache decisions are known to
  *    the host and all of its transfers and kernels are queued.  It never waits for transfers or
  *    compute.
  *  - Environment switches, read once per process (for measurements and tests; none changes results):
