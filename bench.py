@@ -538,6 +538,7 @@ def run_ours(args):
                 "traffic": (DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE * res["bytes_per_launch"]) if DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE else None,
                 "launches": res["launches"], "avg_launch_us": res["avg_launch_us"], "bytes_per_launch": res["bytes_per_launch"],
                 "all_launches": ana["all"] if ana else None,
+                "target_frac": 0.70, "target_met": bool(res["gbs"] / hbm_peak >= 0.70),
                 "note": "launches whose experts were all resident (HBM-bound): bytes = experts streamed x bytes per expert, "
                         "time = CUDA events around each launch; the launches that also fetched experts over the host link "
                         "are in miss_path, all launches together in all_launches"}
