@@ -169,6 +169,28 @@ __device__ __forceinline__ void dequant8(uint32_t w, uint32_t ss, uint32_t (&P)[
     }
 }
 
+// Tensor memory as a per-thread operand store: 32 consecutive 32-bit columns of the thread's own lane.
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+          "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]),
+          "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]),
+          "r"(r[30]), "r"(r[31])
+        : "memory");
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_ld4(uint32_t taddr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3)
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
 __device__ __forceinline__ uint32_t bf16_rne(float v)
 {
     uint32_t u = __float_as_uint(v);
@@ -467,9 +489,14 @@ __device__ __forceinline__ void consume_q4(const DecParams &p, const DecGeometry
 // MT_: k-steps of the gate/up phase and m-tiles of the down phase per warp (d / 256), 0 = taken from d at run time.
 // FMT: 0 = bf16 expert blobs, 1 = 4-bit blobs (melinoe_moe_pack_expert_q4), expanded in registers on
 // the way into the tensor-core fragments.
-template <int MT_, int FMT>
+// XT: 1 = the hidden states' tensor-core operand fragments are kept in tensor memory instead of shared
+// memory (bf16 blobs, d_model 4096 and more than 4 tokens: 64 KB of shared memory go to the ring instead,
+// which doubles the height of the tiles that fit).
+template <int MT_, int FMT, int XT = 0>
 __global__ void __launch_bounds__(kThreads, 1) ffn_decode_kernel(DecParams p, DecGeometry geo)
 {
+    static_assert(XT == 0 || (FMT == 0 && MT_ == 16), "tensor-memory operands: bf16 blobs, d_model 4096");
+    __shared__ uint32_t s_tmem;
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ int s_abort, s_nact, s_last;
     __shared__ int s_hdr[4];                        // status, n_groups, first request, one past the last
@@ -497,7 +524,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_decode_kernel(DecParams p, De
     // ring | staged hidden rows | the warps' partial gate/up tiles
     unsigned char *ring = smem;
     unsigned char *xs = smem + (size_t)S * STAGE;
-    float *buf = reinterpret_cast<float *>(xs + (size_t)Tc * XP);                   // [NW][kBufPitch]
+    float *buf = reinterpret_cast<float *>(xs + (XT ? 0 : (size_t)Tc * XP));        // [NW][kBufPitch]
     const uint32_t ring_s = smem_u32(ring), xs_s = smem_u32(xs);
     const uint32_t full0 = smem_u32(s_bars), empty0 = full0 + 8 * kMaxStages, hzbar = empty0 + 8 * kMaxStages;
     volatile int *abort_flag = &s_abort;
@@ -566,7 +593,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_decode_kernel(DecParams p, De
         s_idx[i] = p.idx[(size_t)tok0 * p.k + i];
         s_gw[i] = p.gate[(size_t)tok0 * p.k + i];
     }
-    {
+    if (XT == 0) {
         const int per_row = d / 8;                  // 16-byte pieces of a hidden row
         for (int i = tid; i < Tc * per_row; i += kThreads) {
             const int t = i / per_row, c = i % per_row;
@@ -593,6 +620,14 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_decode_kernel(DecParams p, De
                 *p.sync = 0u;
         }
         return;
+    }
+    if (XT) {
+        // 128 columns of tensor memory: 16 warps x 32 columns of operand fragments (see below)
+        if (warp == 0) {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)), "r"(128));
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     }
     // gate of every (request, token): the token's gate for that expert if the router chose it
     for (int i = tid; i < nrq * kTokPerVr; i += kThreads) {
@@ -721,6 +756,22 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_decode_kernel(DecParams p, De
             acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f;
         const bool has_tok = g < Tc;
         const uint32_t xrow = xs_s + g * XP + tig * 4 + warp * MT * 32;     // this warp's columns of token g
+        // XT: the token operand of this thread's 16 gate/up steps (two registers each) never changes, so it is
+        // written once into the thread's own lane of tensor memory (warp w may use lanes 32 (w mod 4) ..,
+        // the four warps of a lane quarter take 32 columns each) and fetched from there step by step.
+        uint32_t xt = 0;
+        if constexpr (XT == 1) {
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            xt = s_tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(warp >> 2) * 32;
+            uint32_t r[32];
+            const uint16_t *xr = p.x + (size_t)(tok0 + (has_tok ? g : 0)) * d + warp * 256 + 2 * tig;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                r[2 * i] = has_tok ? __ldcg(reinterpret_cast<const uint32_t *>(xr + i * 16)) : 0u;
+                r[2 * i + 1] = has_tok ? __ldcg(reinterpret_cast<const uint32_t *>(xr + i * 16 + 8)) : 0u;
+            }
+            tmem_st32(xt, r);
+        }
         // ldmatrix lane roles.  gate/up: matrices (W_g rows, k low), (W_u rows, k low), (W_g rows, k high),
         // (W_u rows, k high); down: four consecutive 8-column pieces of the W_d^T rows
         const int r8 = lane & 7, sel_gu = (lane >> 3) & 1, kh = lane >> 4, mat = lane >> 3;
@@ -765,8 +816,15 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_decode_kernel(DecParams p, De
                         for (int j = 0; j < GG; ++j) {
                             const int i = i0 + j < MT ? i0 + j : i0;     // beyond the warp's last step: a valid address, product unused
                             ldmatrix_x4(arow + (((ch0 + 2 * i) ^ swz) << 4), af[j][0], af[j][1], af[j][2], af[j][3]);
-                            bf[j][0] = has_tok ? lds32(xrow + i * 32) : 0u;
-                            bf[j][1] = has_tok ? lds32(xrow + i * 32 + 16) : 0u;
+                            if constexpr (XT == 0) {
+                                bf[j][0] = has_tok ? lds32(xrow + i * 32) : 0u;
+                                bf[j][1] = has_tok ? lds32(xrow + i * 32 + 16) : 0u;
+                            }
+                        }
+                        if constexpr (XT == 1) {
+                            static_assert(XT == 0 || GG == 2, "two steps per group");
+                            tmem_ld4(xt + 2 * i0, bf[0][0], bf[0][1], bf[GG - 1][0], bf[GG - 1][1]);
+                            tmem_wait_ld();
                         }
 #pragma unroll
                         for (int j = 0; j < GG; ++j)
@@ -892,7 +950,14 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_decode_kernel(DecParams p, De
     }
 
     // ---- the CTA that finishes last turns the sums into the output; all others are done
+    if (XT)
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
+    if (XT) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (warp == 0)
+            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(s_tmem), "r"(128));
+    }
     if (tid == 0) {
         __threadfence();
         const unsigned ticket = atomicAdd(p.sync, 1u);
@@ -979,7 +1044,8 @@ bool ffn_decode_supported_q4(int d, int F)
 cudaError_t ffn_decode_configure(int n_sms, size_t max_smem, DecLaunchCfg *cfg)
 {
     size_t stat = 0;
-    const void *fns[6] = {reinterpret_cast<const void *>(ffn_decode_kernel<0, 0>), reinterpret_cast<const void *>(ffn_decode_kernel<8, 0>),
+    const void *fns[7] = {reinterpret_cast<const void *>(ffn_decode_kernel<16, 0, 1>),
+                          reinterpret_cast<const void *>(ffn_decode_kernel<0, 0>), reinterpret_cast<const void *>(ffn_decode_kernel<8, 0>),
                           reinterpret_cast<const void *>(ffn_decode_kernel<16, 0>), reinterpret_cast<const void *>(ffn_decode_kernel<0, 1>),
                           reinterpret_cast<const void *>(ffn_decode_kernel<8, 1>), reinterpret_cast<const void *>(ffn_decode_kernel<16, 1>)};
     for (const void *fn : fns) {
@@ -1012,9 +1078,13 @@ cudaError_t ffn_decode_geometry(const DecLaunchCfg &cfg, int d, int F, int token
     geo->row_bytes = fmt == 0 ? 6 * d : (3 * (d / 2) + 3 * (d / 64) * 2 + 15) / 16 * 16;
     geo->x_pitch = fmt == 0 ? 2 * d + 16 : 2 * d + 64;
     geo->tokens = tokens;
+    // Wide models with many tokens: the hidden states would take a third of the shared memory and leave
+    // room for tiles of two rows only, at which the per-tile work of the warps, not HBM, sets the pace.
+    // Their operand fragments go to tensor memory instead.
+    geo->x_tmem = fmt == 0 && d == 4096 && tokens > 4 ? 1 : 0;
     // staged hidden rows + the warps' partial tiles; the largest tile (at most 8 rows) of which two
     // stages fit beside them
-    const size_t fixed = (size_t)tokens * geo->x_pitch + (size_t)(fmt == 0 ? 1 : 2) * NW * kBufPitch * sizeof(float);
+    const size_t fixed = (geo->x_tmem ? 0 : (size_t)tokens * geo->x_pitch) + (size_t)(fmt == 0 ? 1 : 2) * NW * kBufPitch * sizeof(float);
     int tr = 8;
     for (;; --tr) {
         if (cfg.max_smem >= fixed + (size_t)2 * tr * geo->row_bytes)
@@ -1056,7 +1126,8 @@ cudaError_t launch_ffn_decode(cudaStream_t stream, const DecLaunchCfg &cfg, cons
     cudaError_t e;
     if (p.fmt == 0)
         e = mt == 8    ? cudaLaunchKernelEx(&lc, ffn_decode_kernel<8, 0>, p, geo)
-            : mt == 16 ? cudaLaunchKernelEx(&lc, ffn_decode_kernel<16, 0>, p, geo)
+            : mt == 16 ? (geo.x_tmem ? cudaLaunchKernelEx(&lc, ffn_decode_kernel<16, 0, 1>, p, geo)
+                                     : cudaLaunchKernelEx(&lc, ffn_decode_kernel<16, 0>, p, geo))
                        : cudaLaunchKernelEx(&lc, ffn_decode_kernel<0, 0>, p, geo);
     else
         e = mt == 8    ? cudaLaunchKernelEx(&lc, ffn_decode_kernel<8, 1>, p, geo)

@@ -99,6 +99,7 @@ struct DecGeometry {
     int stage_bytes;
     int x_pitch;                     // bytes between token rows of the staged hidden states
     int tokens;                      // tokens of the launch (1..8)
+    int x_tmem;                      // 1: the hidden states' operand fragments live in tensor memory, not in shared memory
     size_t smem_bytes;
 };
 cudaError_t ffn_decode_configure(int n_sms, size_t max_smem, DecLaunchCfg *cfg);

@@ -56,6 +56,28 @@ def test_shapes_and_token_counts(d, F, E, k, C):
     P.close()
 
 
+def test_wide_model_with_many_tokens_keeps_its_token_operands_in_tensor_memory():
+    """d_model 4096 with 5 to 8 tokens per call: the decode kernel writes the hidden states' tensor-core
+    operands into tensor memory once and reads them from there (the shared memory goes to taller weight
+    tiles).  Calls whose missed experts the kernel fetches itself (token-expert pairs <= slots), with a
+    shared expert, between calls of fewer tokens that take the shared-memory form; then the same bits
+    again from a warm cache (the sum over the SMs is exact, so residency must not change the output)."""
+    d, F, E, k, C = 4096, 48, 20, 2, 16
+    P = _pair(d, F, E, k, C, seed=77, n_shared=1)
+    P.set_bias(_bias(9, E, 0.5, 4), None)
+    outs = {}
+    for rnd in range(2):
+        for step, T in enumerate((8, 5, 2, 7, 6, 1, 8)):
+            P.set_bias(P.bias, (np.arange(T) % 4).astype(np.int32))
+            res, o = P.step(gen.hidden_states(77, 0, "decode", step, T, d))
+            if rnd == 0:
+                outs[step] = res["out_bits"].copy()
+            else:
+                assert np.array_equal(outs[step], res["out_bits"]), "output bits depend on the cache state"
+    assert not P.gpu.layer.last_call_used_gemm()
+    P.close()
+
+
 def test_largest_supported_sizes_and_empty_call():
     """d_model, n_experts and top_k at their limits; T * k = 64 is the largest call the fused
     decode planner takes, T = 3 already goes through the general kernels; T = 0 is a no-op."""
