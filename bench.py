@@ -64,6 +64,10 @@ def parse_args():
     ap.add_argument("--shape", default=None, choices=["mixtral", "phi35", "deepseek"],
                     help="profiling aid: run only that workload shape's record (decode, FFN analysis, prefill GEMM) on "
                          "--layers layers (default 1), print it and exit; not a benchmark line")
+    ap.add_argument("--timeline", action="store_true",
+                    help="profiling aid: per-CTA time stamps of the decode FFN kernel (melinoe_moe_set_timeline) on a "
+                         "--layers (default 2) layer stack with --slots slots (default: every expert resident), "
+                         "printed as medians and maxima over the CTAs; not a benchmark line")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extra", action="store_true", help="skip the other alphas and the resident-cache run")
     return ap.parse_args()
@@ -450,6 +454,41 @@ def shape_record(torch, M, gen, name, n_layers, K, W, hbm_peak, link_peak, peaks
     return rec
 
 
+def timeline_record(torch, gen, cfg, alpha, C, n_layers, store, steps=24, warm=8):
+    """Where a decode launch spends its time: the kernel stamps %globaltimer per CTA at entry, set-up done (plan
+    seen), first tile landed, last tile done, partial sums added, (last CTA only: counter passed, output written),
+    exit.  Stamps of the stack's last layer, microseconds after its first CTA entered, median and maximum over
+    the CTAs, one row per decode step."""
+    from paper_2602_11192_b200.workload import Stack
+    st = Stack(cfg, alpha, C, n_layers=n_layers, store=store)
+    lay = st.layers[-1].layer
+    n_cta = lay.timeline_ctas()
+    tr = torch.zeros((n_cta, 8), dtype=torch.int64, device="cuda")
+    out = torch.empty((n_layers, cfg.batch, cfg.d_model), dtype=torch.int16, device="cuda")
+    stats = torch.zeros((n_layers, 12), dtype=torch.int32, device="cuda")
+    xs = [torch.from_numpy(st.hidden_bits("decode", s).view(np.int16)).cuda() for s in range(steps)]
+    for s in range(warm):
+        st.forward_all(xs[s], out, stats)
+    torch.cuda.synchronize()
+    lay.set_timeline(tr, n_cta * 64)
+    rows = []
+    for s in range(warm, steps):
+        st.forward_all(xs[s], out, stats)
+        torch.cuda.synchronize()
+        t = tr.cpu().numpy().astype(np.int64)
+        rel = (t - t[:, 0].min()) / 1e3
+        live = [0, 1, 2, 3, 4, 7]                    # stamps every CTA writes
+        rows.append({"misses": int(stats.cpu()[-1, 4]),
+                     "median_us": [round(float(np.median(rel[:, i])), 2) for i in live],
+                     "max_us": [round(float(rel[:, i].max()), 2) for i in range(8)]})
+    st.close()
+    return {"timeline": "decode FFN kernel, last of %d layers, %d slots, store %s" % (n_layers, C, store),
+            "stamps_median": ["entry", "set-up done", "first tile landed", "last tile done", "partial sums added", "exit"],
+            "stamps_max": ["entry", "set-up done", "first tile landed", "last tile done", "partial sums added",
+                           "last CTA: counter passed", "last CTA: output written", "exit"],
+            "steps": rows}
+
+
 def run_ours(args):
     import torch
     import gen
@@ -485,6 +524,10 @@ def run_ours(args):
         pass
     hbm_peak = float(peaks.get("hbm_gbs", 6650.0))
     peak_src = "measured" if "hbm_gbs" in peaks else "fallback"
+    if args.timeline:
+        print(json.dumps(timeline_record(torch, gen, cfg, alpha0, cfg.n_experts if args.slots is None else args.slots,
+                                         args.layers or 2, args.store)), flush=True)
+        return
     if args.shape is not None:
         rec = shape_record(torch, M, gen, args.shape, args.layers or 1, min(K, 64), W, hbm_peak, host_link_gbs(torch), peaks,
                            store=args.store)
