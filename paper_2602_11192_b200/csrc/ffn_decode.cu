@@ -982,17 +982,33 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_decode_kernel(DecParams p, De
         const bool acc_in = p.group > 0, acc_out = p.group >= 0 && p.group < n_groups - 1;
         long long *yacc = p.yacc;
         const int N = Tc * d;
-        for (int e = tid; e < N; e += kThreads) {
-            const long long fx = __ldcg(yacc + e);
-            yacc[e] = 0;                                     // the accumulator is left clean for the next launch
-            float v = __ll2float_rn(fx) * (1.0f / 1099511627776.0f);     // one rounding, then an exact scaling
-            const size_t o = (size_t)tok0 * d + e;           // element e of the launch's [tokens][d] block
-            if (acc_in)
-                v += __ldcg(p.ybuf + o);
-            if (acc_out)
-                p.ybuf[o] = v;
-            else
-                p.out[o] = (uint16_t)bf16_rne(v);
+        // four elements per thread at a time, all their loads before any store: this CTA is the whole
+        // grid's critical path, and a load behind a store that may alias it would wait for it
+        constexpr int kBatch = 4;
+        for (int e0 = tid; e0 < N; e0 += kBatch * kThreads) {
+            long long fx[kBatch];
+            float carry[kBatch];
+#pragma unroll
+            for (int j = 0; j < kBatch; ++j) {
+                const int e = e0 + j * kThreads;
+                fx[j] = e < N ? __ldcg(yacc + e) : 0ll;
+                carry[j] = (acc_in && e < N) ? __ldcg(p.ybuf + (size_t)tok0 * d + e) : 0.0f;
+            }
+#pragma unroll
+            for (int j = 0; j < kBatch; ++j) {
+                const int e = e0 + j * kThreads;
+                if (e < N) {
+                    yacc[e] = 0;                                 // the accumulator is left clean for the next launch
+                    float v = __ll2float_rn(fx[j]) * (1.0f / 1099511627776.0f);     // one rounding, then an exact scaling
+                    const size_t o = (size_t)tok0 * d + e;       // element e of the launch's [tokens][d] block
+                    if (acc_in)
+                        v += carry[j];
+                    if (acc_out)
+                        p.ybuf[o] = v;
+                    else
+                        p.out[o] = (uint16_t)bf16_rne(v);
+                }
+            }
         }
     }
     if (trace && tid == 0)
