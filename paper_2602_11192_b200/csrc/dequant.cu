@@ -71,9 +71,14 @@ __global__ void __launch_bounds__(256) dequant_q4_kernel(const unsigned char *__
 
 // Copy of a few KB from device-mapped page-locked host memory into device memory by the SMs
 // themselves: for decode-sized inputs this takes the stream less time than a copy-engine operation.
+// Launched with programmatic stream serialisation: it is scheduled while the kernel ahead in the stream
+// drains and lets the router behind it be scheduled at once; it touches memory only after the kernel ahead
+// has finished (dst may still be read by it, and src may be what it wrote: a caller may chain layers
+// through host buffers on one stream).
 __global__ void __launch_bounds__(256) stage_in_kernel(const uint4 *__restrict__ src, uint4 *__restrict__ dst, int n16)
 {
-    asm volatile("griddepcontrol.wait;" ::: "memory");      // dst may still be read by the kernel ahead in the stream
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += gridDim.x * blockDim.x)
         dst[i] = src[i];
 }
@@ -82,9 +87,18 @@ cudaError_t launch_stage_in(cudaStream_t stream, const void *src_mapped, void *d
 {
     const int n16 = (int)(bytes / 16);
     const int blocks = (n16 + 255) / 256 < 32 ? (n16 + 255) / 256 : 32;
-    stage_in_kernel<<<blocks, 256, 0, stream>>>(static_cast<const uint4 *>(src_mapped), static_cast<uint4 *>(dst), n16);
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3(blocks);
+    lc.blockDim = dim3(256);
+    lc.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = pdl_enabled() ? 1 : 0;
+    const cudaError_t e = cudaLaunchKernelEx(&lc, stage_in_kernel, static_cast<const uint4 *>(src_mapped), static_cast<uint4 *>(dst), n16);
     count_launch();
-    return cudaGetLastError();
+    return e;
 }
 
 cudaError_t launch_dequant_q4(cudaStream_t stream, const void *q4_blob, void *slot, int d, int F, int n_sms)
