@@ -491,6 +491,37 @@ def test_parity_without_programmatic_launch():
     assert r.returncode == 0 and "child ok" in r.stdout, r.stdout[-2000:] + r.stderr[-2000:]
 
 
+def _child(code_body, env_extra):
+    import os
+    import subprocess
+    import sys
+    here = os.path.dirname(os.path.abspath(__file__))
+    code = ("import sys; sys.path.insert(0, %r); sys.path.insert(0, %r)\n"
+            "import numpy as np, gen\nfrom parity_util import Pair\n" % (os.path.dirname(here), here)) + code_body + "print('child ok')\n"
+    r = subprocess.run([sys.executable, "-c", code], env=dict(os.environ, **env_extra), capture_output=True, text=True,
+                       timeout=600)
+    assert r.returncode == 0 and "child ok" in r.stdout, r.stdout[-2000:] + r.stderr[-2000:]
+
+
+def test_parity_with_every_transfer_issued_by_the_host():
+    """MELINOE_MOE_HOST_COPIES: decode calls, too, wait for their plan on the host and fetch with
+    cudaMemcpyAsync (the switch is read once per process, hence the child process)."""
+    _child("P = Pair(512, 64, 16, 2, 4, seed=62)\n"
+           "for step, T in enumerate((1, 2, 1, 8, 2, 1, 12, 1)):\n"
+           "    P.step(gen.hidden_states(62, 0, 'decode', step, T, 512))\n"
+           "P.close()\n", {"MELINOE_MOE_HOST_COPIES": "1"})
+
+
+def test_parity_of_the_single_cta_gemm_on_a_call_of_many_tokens():
+    """MELINOE_MOE_GEMM_SINGLE: a call that would pair CTAs (300 tokens per expert) through the
+    cta_group::1 form of the grouped GEMM."""
+    _child("P = Pair(512, 256, 4, 2, 4, seed=63)\n"
+           "x = gen.hidden_states(63, 0, 'prefill', 0, 600, 512)\n"
+           "P.step(x, tokens=sorted(set([0, 1, 598, 599] + list(range(0, 600, 7)))))\n"
+           "assert P.gpu.layer.last_call_used_gemm()\n"
+           "P.close()\n", {"MELINOE_MOE_GEMM_SINGLE": "1"})
+
+
 def test_trace_miss_proxies_match_the_oracle():
     """Soft (Section 3.1) and hard (Definition C.1) miss proxies of recorded traces, every cache size
     at once: hard misses exact, soft proxy to fp64 rounding; then a budget split over the layers."""
